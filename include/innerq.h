@@ -1,0 +1,159 @@
+/*
+ * innerq.h - C ABI of libinnerq: decode-step attention over a KV cache quantised
+ * group-wise along the inner dimension of each vector-matrix product (InnerQ),
+ * for NVIDIA B200 (sm_100a).
+ *
+ * Conventions (all entry points)
+ *   - Every tensor pointer is a DEVICE pointer unless the parameter is documented as
+ *     host memory.  Tensors are contiguous, row-major, fp16 (IEEE binary16) unless
+ *     stated otherwise.  The caller owns every device byte: the library never calls
+ *     cudaMalloc/cudaFree and never synchronises the device; it enqueues work on the
+ *     caller's stream (`cuda_stream` is a cudaStream_t passed as void*) and returns.
+ *   - Every call returns an int status: INNERQ_OK (0) or a negative INNERQ_ERR_* code.
+ *     Arguments are validated on the host before anything is launched; a failed call
+ *     leaves the cache unchanged.  Nothing aborts, throws or traps.
+ *   - The token count N of a cache lives in the host handle; which tokens are in the
+ *     fp16 windows and which are quantised is a function of N alone.
+ *   - (batch b, KV head h) is called a "unit" u = b * n_kv_heads + h.  Query head j
+ *     reads KV head j / (n_q_heads / n_kv_heads).
+ *   - Supported shapes: head_dim == 128; group in {32, 64, 128}; bits in {2, 3, 4};
+ *     n_q_heads a multiple of n_kv_heads.
+ */
+#ifndef INNERQ_H_
+#define INNERQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  INNERQ_OK = 0,
+  INNERQ_ERR_INVALID_ARG = -1,      /* null pointer, negative size, inconsistent config          */
+  INNERQ_ERR_UNSUPPORTED = -2,      /* bits / group / head_dim combination not implemented       */
+  INNERQ_ERR_CAPACITY = -3,         /* token count would exceed max_tokens                        */
+  INNERQ_ERR_BUFFER_TOO_SMALL = -4, /* caller's cache or workspace buffer smaller than required   */
+  INNERQ_ERR_CUDA = -5              /* a CUDA runtime call or launch failed                       */
+};
+
+enum { INNERQ_MODE_SYM = 0, INNERQ_MODE_ASYM = 1, INNERQ_MODE_HYBRID = 2 };
+enum { INNERQ_SYM_FULLRANGE = 0, INNERQ_SYM_PAPER_LITERAL = 1 };
+enum { INNERQ_GROUPING_INNER = 0, INNERQ_GROUPING_OUTER = 1, INNERQ_GROUPING_FP16 = 2 };
+
+/* Hyper-parameters of a cache (Section "Quantization Scheme": b-bit group-wise quantisation with
+ * group size G; Section "High-precision Window": w_sink, w_recent). */
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim;
+  int32_t max_tokens;   /* capacity: N never exceeds this                                        */
+  int32_t group;        /* G                                                                     */
+  int32_t k_bits, v_bits;
+  int32_t k_mode, v_mode;   /* INNERQ_MODE_*; per-group choice when HYBRID (Section "Hybrid Quantization") */
+  int32_t sym_variant;  /* INNERQ_SYM_*: FULLRANGE  S = max|G|/(2^(b-1)-1), codes in [-(2^(b-1)-1), 2^(b-1)-1];
+                           PAPER_LITERAL  S = max|G|/(2^b-1) as printed, codes clipped to [-2^(b-1), 2^(b-1)-1] */
+  int32_t w_sink, w_recent;
+  int32_t grouping;     /* INNER: K grouped along head_dim inside a token, V along tokens inside a channel
+                           (Section "InnerQ"); OUTER: the reverse, asymmetric, no key normalisation (the
+                           outer-grouped method the paper compares against); FP16: unquantised cache     */
+  int32_t k_normalize;  /* 1: per-channel key normalisation (Section "Per-channel Normalization of K")  */
+  float sm_scale;       /* softmax scale; 0 selects 1/sqrt(head_dim)                                     */
+} innerq_config_t;
+
+typedef struct innerq_cache innerq_cache_t;   /* opaque host handle: layout, views, host copy of N */
+
+/* Canonical (unpacked) view of a cache, for inspection, tests and checkpoints.  All pointers are
+ * DEVICE buffers provided by the caller, or NULL to skip that array.  Shapes use the capacity
+ * cap = max_tokens; tokens are oldest first; only the first n_* entries are written.
+ *   k_code, v_code    uint8  [units][cap][head_dim]     unsigned codes (offset-binary for symmetric groups)
+ *   k_scale, k_zero   uint16 [units][cap][head_dim/G]   (INNER)  or [units][cap/G + 1][head_dim] (OUTER)
+ *   v_scale, v_zero   uint16 [units][cap/G + 1][head_dim] (INNER) or [units][cap][head_dim/G]    (OUTER)
+ *                     fp16 bit patterns; bit 15 of a scale is the hybrid mask M; zero is 0 when M = 0
+ *   norm              float  [units][head_dim]
+ *   k_sink, v_sink    fp16   [units][w_sink][head_dim]
+ *   k_recent,v_recent fp16   [units][w_recent + G][head_dim]
+ * The counts are filled in by innerq_cache_export (host fields). */
+typedef struct {
+  uint8_t *k_code, *v_code;
+  uint16_t *k_scale, *k_zero, *v_scale, *v_zero;
+  float *norm;
+  uint16_t *k_sink, *v_sink, *k_recent, *v_recent;
+  int32_t n_tokens, n_sink, n_qk, n_qv, n_k_recent, n_v_recent;
+} innerq_export_t;
+
+/* Size query.  Writes the number of device bytes the caller must provide for the packed cache
+ * (codes, fp16 scale/zero pairs with the mask in the scale's sign bit, fp16 window ring buffers,
+ * key norms) and for the scratch workspace (split partials of the decode kernel, reduction
+ * scratch of the prefill).  Host pointers.  Errors: INVALID_ARG, UNSUPPORTED. */
+int innerq_cache_bytes(const innerq_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Size of the packed, per-token payload only: bytes of codes + scales + zero-points that one
+ * quantised token of one unit occupies for K (`k_bytes`) and V (`v_bytes`), as double so that the
+ * per-group metadata of V is amortised over its G tokens.  Used to check the effective bit-widths
+ * of Table "bits".  Host pointers. */
+int innerq_token_payload_bytes(const innerq_config_t* cfg, double* k_bytes, double* v_bytes);
+
+/* Create a handle over caller-provided device buffers (256-byte aligned, sizes from
+ * innerq_cache_bytes).  The cache starts empty (N = 0, norm = 1).  The buffers must stay valid
+ * until innerq_cache_destroy.  `*out` receives the handle.  Enqueues a clear of the buffers on
+ * `cuda_stream`.  Errors: INVALID_ARG, UNSUPPORTED, BUFFER_TOO_SMALL, CUDA. */
+int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cache_bytes,
+                        void* dev_workspace, size_t workspace_bytes, void* cuda_stream,
+                        innerq_cache_t** out);
+
+/* Frees the host handle only. */
+int innerq_cache_destroy(innerq_cache_t* cache);
+
+/* Number of tokens currently cached (host value), or a negative error code. */
+int innerq_cache_n_tokens(const innerq_cache_t* cache);
+
+/* Prefill quantisation (Section "High-precision Window", window-split equation; Section
+ * "Per-channel Normalization of K").  Resets the cache to exactly n_tokens tokens taken from
+ * k, v: fp16 [batch][n_kv_heads][n_tokens][head_dim].  Computes norm[c] = sqrt(max_t |K[t,c]|)
+ * per unit over all n_tokens (when k_normalize), keeps the first w_sink and the last w_recent
+ * tokens in fp16, and quantises the middle: per group statistics, symmetric / asymmetric
+ * candidates, the hybrid choice, bit-packing.  Tokens grouped G at a time (V under INNER) that do
+ * not fill a group stay fp16 in front of the recent window.  0 <= n_tokens <= max_tokens.
+ * Errors: INVALID_ARG, CAPACITY, CUDA. */
+int innerq_quantize_prefill(innerq_cache_t* cache, const void* k, const void* v, int32_t n_tokens,
+                            void* cuda_stream);
+
+/* Append the decode step's own token (Section "High-precision Window", last paragraph; Section
+ * "Latency": one key token is quantised every step, G value tokens every G steps; the reverse
+ * under OUTER).  k_new, v_new: fp16 [batch][n_kv_heads][head_dim].  The token enters the sink
+ * window while it is not full, else the recent window; tokens leaving the recent window are
+ * normalised with the norm fixed at prefill (keys) and quantised into the packed cache.
+ * Errors: INVALID_ARG, CAPACITY, CUDA. */
+int innerq_append_token(innerq_cache_t* cache, const void* k_new, const void* v_new, void* cuda_stream);
+
+/* Decode attention (attention equations S = QK^T, P = softmax(S / sqrt(d_h)), O = PV with
+ * N_Q = 1, over K = [K_sink; dequant(K^); K_recent] and the same for V; hybrid dequantisation
+ * S*K^ + M*Z; Section "InnerQ").  q: fp16 [batch][n_q_heads][head_dim]; out: fp16, same shape,
+ * fully overwritten.  Attends over all N cached tokens (append the step's token first); N >= 1.
+ * Scores of quantised key rows use q' = q * norm; dequantisation happens in registers, scale and
+ * zero-point are applied once per group.  Uses the workspace; two decodes on the same cache must
+ * not overlap.  Errors: INVALID_ARG (N == 0 included), CUDA. */
+int innerq_decode_attention(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
+
+/* Unpack the cache into canonical arrays (see innerq_export_t).  `ex` is a host struct holding
+ * device pointers; counts are written to it before the call returns, array contents when the
+ * stream reaches the enqueued kernels.  Errors: INVALID_ARG, CUDA. */
+int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_stream);
+
+/* Tuning knobs for experiments; both default to 0 = automatic.
+ *   n_splits : number of token ranges each unit is split into by the decode kernel.
+ *   variant  : 0 automatic, 1 plain SIMT kernel, 2 warp-MMA kernel (where supported).
+ * Errors: INVALID_ARG. */
+int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
+
+/* Number of kernels the last call of each kind launched (for launch accounting):
+ * which = 0 prefill, 1 append, 2 decode.  Returns the count or a negative error code. */
+int innerq_last_launch_count(const innerq_cache_t* cache, int32_t which);
+
+/* Static string for a status code; never NULL. */
+const char* innerq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INNERQ_H_ */

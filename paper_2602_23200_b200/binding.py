@@ -1,0 +1,244 @@
+"""ctypes binding over libinnerq.so: argument marshalling only.
+
+Function names mirror the C ABI (include/innerq.h).  PyTorch is used for device memory and
+streams; every step of the path runs in the library's CUDA kernels.  There is no CPU fallback:
+if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libinnerq.so")
+
+MODE_SYM, MODE_ASYM, MODE_HYBRID = 0, 1, 2
+SYM_FULLRANGE, SYM_PAPER_LITERAL = 0, 1
+GROUPING_INNER, GROUPING_OUTER, GROUPING_FP16 = 0, 1, 2
+
+EXPORTED_SYMBOLS = (
+    "innerq_cache_bytes", "innerq_token_payload_bytes", "innerq_cache_create", "innerq_cache_destroy",
+    "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
+    "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_status_string",
+)
+
+
+class InnerQError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+class innerq_config_t(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "batch", "n_q_heads", "n_kv_heads", "head_dim", "max_tokens", "group", "k_bits", "v_bits",
+        "k_mode", "v_mode", "sym_variant", "w_sink", "w_recent", "grouping", "k_normalize")] + [("sm_scale", C.c_float)]
+
+
+class innerq_export_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "k_code", "v_code", "k_scale", "k_zero", "v_scale", "v_zero", "norm",
+        "k_sink", "v_sink", "k_recent", "v_recent")] + [(n, C.c_int32) for n in (
+        "n_tokens", "n_sink", "n_qk", "n_qv", "n_k_recent", "n_v_recent")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libinnerq.so (built in-tree by paper_2602_23200_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_23200_b200.build` "
+                           "(there is no fallback path)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    cfgp = C.POINTER(innerq_config_t)
+    L.innerq_cache_bytes.argtypes = [cfgp, C.POINTER(sz), C.POINTER(sz)]
+    L.innerq_token_payload_bytes.argtypes = [cfgp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.innerq_cache_create.argtypes = [cfgp, vp, sz, vp, sz, vp, C.POINTER(vp)]
+    L.innerq_cache_destroy.argtypes = [vp]
+    L.innerq_cache_n_tokens.argtypes = [vp]
+    L.innerq_quantize_prefill.argtypes = [vp, vp, vp, i32, vp]
+    L.innerq_append_token.argtypes = [vp, vp, vp, vp]
+    L.innerq_decode_attention.argtypes = [vp, vp, vp, vp]
+    L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
+    L.innerq_set_decode_options.argtypes = [vp, i32, i32]
+    L.innerq_last_launch_count.argtypes = [vp, i32]
+    L.innerq_status_string.argtypes = [C.c_int]
+    L.innerq_status_string.restype = C.c_char_p
+    for name in EXPORTED_SYMBOLS:
+        if name != "innerq_status_string":
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().innerq_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> int:
+    if status < 0:
+        raise InnerQError(status, what)
+    return status
+
+
+def make_config(w=None, **kw) -> innerq_config_t:
+    """Build an innerq_config_t from a workload-like object (attribute names of synth.Workload) and/or keywords."""
+    vals = dict(batch=1, n_q_heads=1, n_kv_heads=1, head_dim=128, max_tokens=0, group=32, k_bits=2, v_bits=2,
+                k_mode=MODE_HYBRID, v_mode=MODE_HYBRID, sym_variant=0, w_sink=4, w_recent=128,
+                grouping=GROUPING_INNER, k_normalize=1, sm_scale=0.0)
+    if w is not None:
+        for k in vals:
+            if hasattr(w, k):
+                vals[k] = getattr(w, k)
+        if not kw.get("max_tokens") and hasattr(w, "n_tokens"):
+            vals["max_tokens"] = w.n_tokens
+    vals.update(kw)
+    cfg = innerq_config_t()
+    for k, v in vals.items():
+        setattr(cfg, k, v)
+    return cfg
+
+
+def innerq_cache_bytes(cfg: innerq_config_t):
+    cb, wb = C.c_size_t(), C.c_size_t()
+    _check(lib().innerq_cache_bytes(C.byref(cfg), C.byref(cb), C.byref(wb)), "innerq_cache_bytes")
+    return cb.value, wb.value
+
+
+def innerq_token_payload_bytes(cfg: innerq_config_t):
+    kb, vb = C.c_double(), C.c_double()
+    _check(lib().innerq_token_payload_bytes(C.byref(cfg), C.byref(kb), C.byref(vb)), "innerq_token_payload_bytes")
+    return kb.value, vb.value
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _dev_ptr(t, name: str, shape) -> int:
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float16 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA fp16 tensor")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+    return t.data_ptr()
+
+
+class InnerQCache:
+    """A packed KV cache living in caller-side torch device buffers, driven through the C ABI."""
+
+    def __init__(self, cfg: innerq_config_t, device="cuda:0", stream=None):
+        import torch
+        self.cfg = cfg
+        self.device = torch.device(device)
+        cb, wb = innerq_cache_bytes(cfg)
+        self.cache_bytes, self.workspace_bytes = cb, wb
+        with torch.cuda.device(self.device):
+            self._cache_buf = torch.empty(cb, dtype=torch.uint8, device=self.device)
+            self._ws_buf = torch.empty(wb, dtype=torch.uint8, device=self.device)
+            h = C.c_void_p()
+            _check(lib().innerq_cache_create(C.byref(cfg), self._cache_buf.data_ptr(), cb, self._ws_buf.data_ptr(), wb,
+                                             _stream_ptr(stream), C.byref(h)), "innerq_cache_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().innerq_cache_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    @property
+    def n_tokens(self) -> int:
+        return _check(lib().innerq_cache_n_tokens(self._h), "innerq_cache_n_tokens")
+
+    @property
+    def units(self) -> int:
+        return self.cfg.batch * self.cfg.n_kv_heads
+
+    def innerq_quantize_prefill(self, k, v, stream=None):
+        c = self.cfg
+        n = int(k.shape[2]) if k.dim() == 4 else -1
+        shape = (c.batch, c.n_kv_heads, n, c.head_dim)
+        kp, vp = (_dev_ptr(k, "k", shape), _dev_ptr(v, "v", shape)) if n > 0 else (k.data_ptr(), v.data_ptr())
+        _check(lib().innerq_quantize_prefill(self._h, kp, vp, n, _stream_ptr(stream)), "innerq_quantize_prefill")
+
+    def innerq_append_token(self, k_new, v_new, stream=None):
+        c = self.cfg
+        shape = (c.batch, c.n_kv_heads, c.head_dim)
+        _check(lib().innerq_append_token(self._h, _dev_ptr(k_new, "k_new", shape), _dev_ptr(v_new, "v_new", shape),
+                                         _stream_ptr(stream)), "innerq_append_token")
+
+    def innerq_decode_attention(self, q, out=None, stream=None):
+        import torch
+        c = self.cfg
+        shape = (c.batch, c.n_q_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float16, device=self.device)
+        _check(lib().innerq_decode_attention(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
+                                             _stream_ptr(stream)), "innerq_decode_attention")
+        return out
+
+    def innerq_set_decode_options(self, n_splits: int = 0, variant: int = 0):
+        _check(lib().innerq_set_decode_options(self._h, n_splits, variant), "innerq_set_decode_options")
+
+    def innerq_last_launch_count(self, which: int) -> int:
+        return _check(lib().innerq_last_launch_count(self._h, which), "innerq_last_launch_count")
+
+    def innerq_cache_export(self, stream=None, codes: bool = True) -> dict:
+        """Canonical (unpacked) cache contents as numpy arrays trimmed to the live counts."""
+        import torch
+        c = self.cfg
+        U, D, G, cap = self.units, c.head_dim, c.group, c.max_tokens
+        fp16 = c.grouping == GROUPING_FP16
+        inner = c.grouping == GROUPING_INNER
+        dev = self.device
+
+        def buf(shape, dtype):
+            return torch.zeros(shape, dtype=dtype, device=dev)
+
+        row_meta, blk_meta = (U, cap, D // G), (U, cap // G + 1, D)
+        t = {}
+        if not fp16:
+            if codes:
+                t["k_code"], t["v_code"] = buf((U, cap, D), torch.uint8), buf((U, cap, D), torch.uint8)
+            km, vm = (row_meta, blk_meta) if inner else (blk_meta, row_meta)
+            t["k_scale"], t["k_zero"] = buf(km, torch.int16), buf(km, torch.int16)
+            t["v_scale"], t["v_zero"] = buf(vm, torch.int16), buf(vm, torch.int16)
+            t["k_recent"] = buf((U, c.w_recent + G, D), torch.float16)
+            t["v_recent"] = buf((U, c.w_recent + G, D), torch.float16)
+        t["norm"] = buf((U, D), torch.float32)
+        sink_cap = cap if fp16 else c.w_sink
+        t["k_sink"], t["v_sink"] = buf((U, max(sink_cap, 1), D), torch.float16), buf((U, max(sink_cap, 1), D), torch.float16)
+        ex = innerq_export_t()
+        for name, ten in t.items():
+            setattr(ex, name, ten.data_ptr())
+        _check(lib().innerq_cache_export(self._h, C.byref(ex), _stream_ptr(stream)), "innerq_cache_export")
+        torch.cuda.synchronize(dev)
+        out = {k: getattr(ex, k) for k in ("n_tokens", "n_sink", "n_qk", "n_qv", "n_k_recent", "n_v_recent")}
+        host = {k: v.cpu().numpy() for k, v in t.items()}
+        out["norm"] = host["norm"]
+        out["k_sink"], out["v_sink"] = host["k_sink"][:, :out["n_sink"]], host["v_sink"][:, :out["n_sink"]]
+        if fp16:
+            return out
+        out["k_recent"] = host["k_recent"][:, :out["n_k_recent"]]
+        out["v_recent"] = host["v_recent"][:, :out["n_v_recent"]]
+        nk_meta = out["n_qk"] if inner else out["n_qk"] // G
+        nv_meta = out["n_qv"] // G if inner else out["n_qv"]
+        if codes:
+            out["k_code"], out["v_code"] = host["k_code"][:, :out["n_qk"]], host["v_code"][:, :out["n_qv"]]
+        out["k_scale"] = host["k_scale"].view(np.uint16)[:, :nk_meta]
+        out["k_zero"] = host["k_zero"].view(np.uint16)[:, :nk_meta]
+        out["v_scale"] = host["v_scale"].view(np.uint16)[:, :nv_meta]
+        out["v_zero"] = host["v_zero"].view(np.uint16)[:, :nv_meta]
+        return out

@@ -1,0 +1,263 @@
+// C ABI of libinnerq (see include/innerq.h): argument validation, layout computation, host-side
+// token bookkeeping, kernel dispatch.  No device allocation, no synchronisation.
+#include <cstring>
+#include <new>
+
+#include "../../include/innerq.h"
+#include "innerq_kernels.h"
+
+using namespace iq;
+
+struct innerq_cache {
+  innerq_config_t cfg;
+  Layout L;
+  unsigned char* cache;
+  unsigned char* ws;
+  int N;
+  int opt_splits, opt_variant;
+  int launches[3];
+};
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool valid_bits(int b) { return b == 2 || b == 3 || b == 4; }
+bool valid_mode(int m) { return m >= 0 && m <= 2; }
+
+int check_config(const innerq_config_t* c) {
+  if (!c) return INNERQ_ERR_INVALID_ARG;
+  if (c->batch <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->max_tokens <= 0 || c->w_sink < 0 ||
+      c->w_recent < 0 || c->n_q_heads % c->n_kv_heads != 0 || !(c->sm_scale >= 0.f))
+    return INNERQ_ERR_INVALID_ARG;
+  if (c->grouping < 0 || c->grouping > 2 || c->sym_variant < 0 || c->sym_variant > 1) return INNERQ_ERR_INVALID_ARG;
+  if (c->head_dim != kD) return INNERQ_ERR_UNSUPPORTED;
+  if (c->grouping != INNERQ_GROUPING_FP16) {
+    if (!valid_mode(c->k_mode) || !valid_mode(c->v_mode)) return INNERQ_ERR_INVALID_ARG;
+    if (!valid_bits(c->k_bits) || !valid_bits(c->v_bits)) return INNERQ_ERR_UNSUPPORTED;
+    if (c->group != 32 && c->group != 64 && c->group != 128) return INNERQ_ERR_UNSUPPORTED;
+    if (c->grouping == INNERQ_GROUPING_OUTER && c->k_normalize) return INNERQ_ERR_INVALID_ARG;
+  }
+  if ((long long)c->batch * c->n_kv_heads > 65535) return INNERQ_ERR_UNSUPPORTED;
+  return INNERQ_OK;
+}
+
+void place_store(Store& S, int kind, int bits, int mode, const innerq_config_t& c, int U, size_t& off) {
+  std::memset(&S, 0, sizeof(S));
+  S.kind = kind;
+  S.bits = bits;
+  S.mode = mode;
+  if (kind == kNone) {
+    S.sink_stride = (size_t)c.max_tokens * kD * 2;
+    S.sink_off = off;
+    off = align_up(off + S.sink_stride * U, 256);
+    return;
+  }
+  const int G = c.group;
+  int mid = c.max_tokens - c.w_sink - c.w_recent;
+  if (mid < 1) mid = 1;
+  S.cap_q = (int)align_up((size_t)mid, kTile);
+  S.ring_cap = kind == kRow ? c.w_recent + 1 : c.w_recent + G;
+  S.n_groups = kind == kRow ? kD / G : kD;
+  S.meta_bytes = mode == INNERQ_MODE_SYM ? 2 : 4;
+  S.sink_stride = (size_t)c.w_sink * kD * 2;
+  S.ring_stride = (size_t)S.ring_cap * kD * 2;
+  if (kind == kRow) {
+    S.code_stride = (size_t)S.cap_q * row_bytes(bits);
+    S.meta_stride = (size_t)S.cap_q * S.n_groups * S.meta_bytes;
+  } else {
+    S.code_stride = (size_t)(S.cap_q / kChunk) * chunk_bytes(bits);
+    S.meta_stride = (size_t)(S.cap_q / G) * kD * S.meta_bytes;
+  }
+  S.sink_off = off; off = align_up(off + S.sink_stride * U, 256);
+  S.ring_off = off; off = align_up(off + S.ring_stride * U, 256);
+  S.code_off = off; off = align_up(off + S.code_stride * U, 256);
+  S.meta_off = off; off = align_up(off + S.meta_stride * U, 256);
+}
+
+void make_layout(const innerq_config_t& c, Layout& L) {
+  std::memset(&L, 0, sizeof(L));
+  L.B = c.batch; L.Hq = c.n_q_heads; L.Hkv = c.n_kv_heads;
+  L.U = c.batch * c.n_kv_heads;
+  L.r = c.n_q_heads / c.n_kv_heads;
+  L.G = c.grouping == INNERQ_GROUPING_FP16 ? 32 : c.group;
+  L.w_sink = c.w_sink; L.w_recent = c.w_recent;
+  L.sym_variant = c.sym_variant; L.grouping = c.grouping;
+  L.k_normalize = (c.grouping == INNERQ_GROUPING_INNER && c.k_normalize) ? 1 : 0;
+  L.max_tokens = c.max_tokens;
+  L.sm_scale = c.sm_scale > 0.f ? c.sm_scale : 0.08838834764831845f;   // 1/sqrt(128)
+  int ms = (4 * 148 + L.U - 1) / L.U;
+  L.max_splits = ms < 1 ? 1 : (ms > 64 ? 64 : ms);
+  size_t off = 0;
+  L.norm_off = off; off = align_up(off + (size_t)L.U * kD * 4, 256);
+  if (c.grouping == INNERQ_GROUPING_FP16) {
+    place_store(L.k, kNone, 16, 0, c, L.U, off);
+    place_store(L.v, kNone, 16, 0, c, L.U, off);
+  } else if (c.grouping == INNERQ_GROUPING_INNER) {
+    place_store(L.k, kRow, c.k_bits, c.k_mode, c, L.U, off);
+    place_store(L.v, kBlock, c.v_bits, c.v_mode, c, L.U, off);
+  } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
+    place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);
+    place_store(L.v, kRow, c.v_bits, INNERQ_MODE_ASYM, c, L.U, off);
+  }
+  L.cache_bytes = off;
+  size_t w = 0;
+  L.ws_partial_off = w; w = align_up(w + (size_t)L.B * L.Hq * L.max_splits * kPartialStride * 4, 256);
+  L.ws_absmax_off = w; w = align_up(w + (size_t)L.U * kD * 4, 256);
+  L.ws_ticket_off = w; w = align_up(w + (size_t)L.U * 4, 256);
+  L.workspace_bytes = w;
+}
+
+}  // namespace
+
+extern "C" {
+
+int innerq_cache_bytes(const innerq_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes) {
+  int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  if (!cache_bytes || !workspace_bytes) return INNERQ_ERR_INVALID_ARG;
+  Layout L;
+  make_layout(*cfg, L);
+  *cache_bytes = L.cache_bytes;
+  *workspace_bytes = L.workspace_bytes;
+  return INNERQ_OK;
+}
+
+int innerq_token_payload_bytes(const innerq_config_t* cfg, double* k_bytes, double* v_bytes) {
+  int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  if (!k_bytes || !v_bytes) return INNERQ_ERR_INVALID_ARG;
+  Layout L;
+  make_layout(*cfg, L);
+  const Store* S[2] = {&L.k, &L.v};
+  double out[2];
+  for (int i = 0; i < 2; ++i) {
+    if (S[i]->kind == kNone) out[i] = kD * 2.0;
+    else if (S[i]->kind == kRow) out[i] = row_bytes(S[i]->bits) + (double)S[i]->n_groups * S[i]->meta_bytes;
+    else out[i] = chunk_bytes(S[i]->bits) / (double)kChunk + (double)kD * S[i]->meta_bytes / L.G;
+  }
+  *k_bytes = out[0];
+  *v_bytes = out[1];
+  return INNERQ_OK;
+}
+
+int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cache_bytes, void* dev_workspace,
+                        size_t workspace_bytes, void* cuda_stream, innerq_cache_t** out) {
+  int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  if (!dev_cache || !dev_workspace || !out) return INNERQ_ERR_INVALID_ARG;
+  if (((uintptr_t)dev_cache & 255u) || ((uintptr_t)dev_workspace & 255u)) return INNERQ_ERR_INVALID_ARG;
+  innerq_cache* c = new (std::nothrow) innerq_cache();
+  if (!c) return INNERQ_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  make_layout(*cfg, c->L);
+  if (cache_bytes < c->L.cache_bytes || workspace_bytes < c->L.workspace_bytes) {
+    delete c;
+    return INNERQ_ERR_BUFFER_TOO_SMALL;
+  }
+  c->cache = static_cast<unsigned char*>(dev_cache);
+  c->ws = static_cast<unsigned char*>(dev_workspace);
+  c->N = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(c->cache, 0, c->L.cache_bytes, s) != cudaSuccess ||
+      cudaMemsetAsync(c->ws, 0, c->L.workspace_bytes, s) != cudaSuccess) {
+    delete c;
+    return INNERQ_ERR_CUDA;
+  }
+  // norm = 1 until a prefill computes it
+  if (launch_prefill(c->L, c->cache, c->ws, nullptr, nullptr, 0, s) < 0) {
+    delete c;
+    return INNERQ_ERR_CUDA;
+  }
+  *out = c;
+  return INNERQ_OK;
+}
+
+int innerq_cache_destroy(innerq_cache_t* cache) {
+  if (!cache) return INNERQ_ERR_INVALID_ARG;
+  delete cache;
+  return INNERQ_OK;
+}
+
+int innerq_cache_n_tokens(const innerq_cache_t* cache) { return cache ? cache->N : INNERQ_ERR_INVALID_ARG; }
+
+int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int32_t n_tokens, void* cuda_stream) {
+  if (!c || n_tokens < 0 || (n_tokens > 0 && (!k || !v))) return INNERQ_ERR_INVALID_ARG;
+  if (n_tokens > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  int n = launch_prefill(c->L, c->cache, c->ws, static_cast<const __half*>(k), static_cast<const __half*>(v), n_tokens,
+                         static_cast<cudaStream_t>(cuda_stream));
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->N = n_tokens;
+  c->launches[0] = n;
+  return INNERQ_OK;
+}
+
+int innerq_append_token(innerq_cache_t* c, const void* k_new, const void* v_new, void* cuda_stream) {
+  if (!c || !k_new || !v_new) return INNERQ_ERR_INVALID_ARG;
+  if (c->N + 1 > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  int n = launch_append(c->L, c->cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new), c->N + 1,
+                        static_cast<cudaStream_t>(cuda_stream));
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->N += 1;
+  c->launches[1] = n;
+  return INNERQ_OK;
+}
+
+int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* cuda_stream) {
+  if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int n = -2;
+  if (c->opt_variant != 1 && decode_mma_supported(c->L))
+    n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                          c->opt_splits, s);
+  if (n == -2) {
+    if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
+    n = launch_decode_simt(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                           c->opt_splits, s);
+  }
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->launches[2] = n;
+  return INNERQ_OK;
+}
+
+int innerq_cache_export(innerq_cache_t* c, innerq_export_t* ex, void* cuda_stream) {
+  if (!c || !ex) return INNERQ_ERR_INVALID_ARG;
+  const Counts cn = counts_for(c->L, c->N);
+  const bool fp16 = c->L.k.kind == kNone;
+  ex->n_tokens = cn.N;
+  ex->n_sink = fp16 ? cn.N : cn.n_sink;
+  ex->n_qk = cn.n_qk;
+  ex->n_qv = cn.n_qv;
+  ex->n_k_recent = fp16 ? 0 : cn.n_k_recent;
+  ex->n_v_recent = fp16 ? 0 : cn.n_v_recent;
+  ExportPtrs p{ex->k_code, ex->v_code, ex->k_scale, ex->k_zero, ex->v_scale, ex->v_zero,
+               ex->norm,   ex->k_sink, ex->v_sink,  ex->k_recent, ex->v_recent};
+  if (launch_export(c->L, c->cache, c->N, p, static_cast<cudaStream_t>(cuda_stream)) < 0) return INNERQ_ERR_CUDA;
+  return INNERQ_OK;
+}
+
+int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t variant) {
+  if (!c || n_splits < 0 || variant < 0 || variant > 2) return INNERQ_ERR_INVALID_ARG;
+  c->opt_splits = n_splits;
+  c->opt_variant = variant;
+  return INNERQ_OK;
+}
+
+int innerq_last_launch_count(const innerq_cache_t* c, int32_t which) {
+  if (!c || which < 0 || which > 2) return INNERQ_ERR_INVALID_ARG;
+  return c->launches[which];
+}
+
+const char* innerq_status_string(int status) {
+  switch (status) {
+    case INNERQ_OK: return "ok";
+    case INNERQ_ERR_INVALID_ARG: return "invalid argument";
+    case INNERQ_ERR_UNSUPPORTED: return "unsupported configuration";
+    case INNERQ_ERR_CAPACITY: return "token capacity exceeded";
+    case INNERQ_ERR_BUFFER_TOO_SMALL: return "caller buffer too small";
+    case INNERQ_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

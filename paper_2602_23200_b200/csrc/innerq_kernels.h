@@ -1,0 +1,33 @@
+// Host-callable launchers of the library's kernels (internal interface between the .cu files).
+// Each returns the number of kernels it launched, or -1 on a CUDA error.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "innerq_layout.h"
+
+namespace iq {
+
+struct ExportPtrs {
+  uint8_t *k_code, *v_code;
+  uint16_t *k_scale, *k_zero, *v_scale, *v_zero;
+  float* norm;
+  uint16_t *k_sink, *v_sink, *k_recent, *v_recent;
+};
+
+int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, const __half* K, const __half* V, int N,
+                   cudaStream_t st);
+int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
+                  cudaStream_t st);
+int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st);
+
+// Generic SIMT decode (any store kinds, bits, group sizes): split kernel + merge kernel.
+int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
+                       __half* out, int n_splits, cudaStream_t st);
+
+// Warp-MMA decode for the INNER layout.  Returns -2 if the configuration is not supported.
+int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
+                      __half* out, int n_splits, cudaStream_t st);
+bool decode_mma_supported(const Layout& L);
+
+}  // namespace iq

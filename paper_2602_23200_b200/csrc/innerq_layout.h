@@ -1,0 +1,141 @@
+// Packed cache layout in HBM (head_dim = 128).  Shared by the quantise, append, decode and
+// export kernels of this library.
+//
+// A quantised tensor lives in one of two stores:
+//
+//   ROW store   (per-token groups along channels; InnerQ keys).  One row of 16*b bytes per
+//               token, rows contiguous, so one evicted token is one contiguous write and a
+//               tile of tokens is one contiguous range.  Metadata: one 32-bit word per
+//               (token, group) = fp16 scale (mask M in the sign bit) | fp16 zero-point << 16;
+//               in symmetric mode only the 16-bit scale is stored.
+//   BLOCK store (per-channel groups along tokens; InnerQ values).  Chunks of 32 tokens x 128
+//               channels, 512*b bytes each, chunks contiguous.  Metadata: one word per
+//               (group of G tokens, channel), reused by the G tokens of the group.
+//
+// Inside a row / chunk the codes are permuted so that a 32-lane warp reads its tensor-core
+// operand fragments with 64/128-bit loads and extracts them with one LOP3 per pair:
+// lane L = 4*gid + tid4 owns the fragment entries that mma.m16n8k16 assigns to it, and a
+// 32-bit word holds pairs (low half, high half) at equal field positions, so that
+// `word & (mask << pos)` is a half2 of two codes scaled by 2^pos (as fp16 subnormals).
+//
+// b = 3 is stored as a 2-bit plane followed by a 1-bit plane (code = lo + 4*hi).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+#ifdef __CUDACC__
+#define IQ_HD __host__ __device__ __forceinline__
+#else
+#define IQ_HD inline
+#endif
+
+namespace iq {
+
+constexpr int kD = 128;           // head_dim
+constexpr int kChunk = 32;        // tokens per BLOCK-store chunk
+constexpr int kTile = 128;        // capacity granularity in tokens
+
+enum StoreKind : int { kRow = 0, kBlock = 1, kNone = 2 };
+
+struct Store {
+  int kind;            // StoreKind
+  int bits, mode;
+  int ring_cap;        // slots of the recent ring: w_recent + 1 (ROW) or w_recent + G (BLOCK)
+  int cap_q;           // capacity in quantised tokens (multiple of kTile)
+  int n_groups;        // metadata entries per row (ROW: D/G) or per group (BLOCK: D)
+  int meta_bytes;      // 4: fp16 scale | fp16 zero << 16;  2: fp16 scale only (symmetric mode stores no zero-points)
+  size_t sink_off, ring_off, code_off, meta_off;              // byte offsets of unit 0
+  size_t sink_stride, ring_stride, code_stride, meta_stride;  // bytes per unit
+};
+
+struct Layout {
+  int B, Hq, Hkv, U, r;
+  int G, w_sink, w_recent, sym_variant, grouping, k_normalize;
+  int max_tokens, max_splits;
+  float sm_scale;
+  size_t norm_off;     // float [U][D]
+  size_t cache_bytes;
+  // workspace
+  size_t ws_partial_off;   // float [B*Hq][max_splits][kPartialStride]
+  size_t ws_absmax_off;    // uint32 [U][D]
+  size_t ws_ticket_off;    // uint32 [U]
+  size_t workspace_bytes;
+  Store k, v;
+};
+
+constexpr int kPartialStride = kD + 4;   // acc[D], m, l, pad, pad
+
+// Token bookkeeping: a function of N alone.
+struct Counts {
+  int N, n_sink, n_qk, n_qv, n_k_recent, n_v_recent;
+};
+
+IQ_HD int n_quantised(int kind, int N, int w_sink, int w_recent, int G) {
+  int mid = N - w_sink - w_recent;
+  if (kind == kNone || mid <= 0) return 0;
+  return kind == kRow ? mid : (mid / G) * G;
+}
+
+IQ_HD Counts counts_for(const Layout& L, int N) {
+  Counts c;
+  c.N = N;
+  c.n_sink = N < L.w_sink ? N : L.w_sink;
+  c.n_qk = n_quantised(L.k.kind, N, L.w_sink, L.w_recent, L.G);
+  c.n_qv = n_quantised(L.v.kind, N, L.w_sink, L.w_recent, L.G);
+  c.n_k_recent = N - c.n_sink - c.n_qk;
+  c.n_v_recent = N - c.n_sink - c.n_qv;
+  return c;
+}
+
+// ---------------------------------------------------------------- code positions
+// ROW store: bit position of channel c inside a row of 16*b bytes.
+//   k-step s = c / 16 (16 channels feed one mma k-step), col = c % 16,
+//   tid4 = (col % 8) / 2 owns the column pair, hf = col % 2 selects the half-word,
+//   odd = col / 8 selects the second pair of the k-step.
+struct BitPos { int word; int bit; };      // 32-bit word index inside the row/chunk, bit inside the word
+
+IQ_HD BitPos row_pos_plane(int c, int plane_bits) {
+  int s = c >> 4, col = c & 15;
+  int j = (col & 7) >> 1, hf = col & 1, odd = col >> 3;
+  BitPos p;
+  if (plane_bits == 2) {         // lane chunk = 2 words; word serves 4 k-steps, 2 fields each
+    p.word = 2 * j + (s >> 2);
+    p.bit = 16 * hf + 2 * (2 * (s & 3) + odd);
+  } else if (plane_bits == 4) {  // lane chunk = 4 words; word serves 2 k-steps
+    p.word = 4 * j + (s >> 1);
+    p.bit = 16 * hf + 4 * (2 * (s & 1) + odd);
+  } else {                       // 1-bit plane: lane chunk = 1 word; 8 k-steps x 2 fields
+    p.word = j;
+    p.bit = 16 * hf + (2 * s + odd);
+  }
+  return p;
+}
+
+// BLOCK store: position of (token tau in 0..31, channel c) inside a chunk.
+//   PV mma: row = channel, k = token.  m = c / 16 is the m-tile, gid = c % 8, rh = (c / 8) % 2 the
+//   upper row half; ks = tau / 16 the k-step, kh = (tau / 8) % 2, tid4 = (tau % 8) / 2, tp = tau % 2.
+IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
+  int ks = tau >> 4, kh = (tau >> 3) & 1, j = (tau & 7) >> 1, tp = tau & 1;
+  int m = c >> 4, gid = c & 7, rh = (c >> 3) & 1;
+  int lane = 4 * gid + j;
+  BitPos p;
+  if (plane_bits == 2) {         // 8 words per lane: word = m; fields (rh, ks, kh)
+    p.word = (m >> 2) * 128 + lane * 4 + (m & 3);
+    p.bit = 16 * tp + 2 * (4 * rh + 2 * ks + kh);
+  } else if (plane_bits == 4) {  // 16 words per lane: word = (ks, m); fields (rh, kh)
+    p.word = ks * 256 + (m >> 2) * 128 + lane * 4 + (m & 3);
+    p.bit = 16 * tp + 4 * (2 * rh + kh);
+  } else {                       // 1-bit plane, 4 words per lane: word = m / 2; fields (m % 2, rh, ks, kh)
+    p.word = lane * 4 + (m >> 1);
+    p.bit = 16 * tp + (((m & 1) * 2 + rh) * 4 + 2 * ks + kh);
+  }
+  return p;
+}
+
+IQ_HD int row_bytes(int bits) { return 16 * bits; }
+IQ_HD int chunk_bytes(int bits) { return 512 * bits; }
+// word offset of the 1-bit plane of a 3-bit row / chunk
+IQ_HD int row_hi_plane_word() { return 8; }
+IQ_HD int chunk_hi_plane_word() { return 256; }
+
+}  // namespace iq

@@ -1,0 +1,376 @@
+// Quantise-side kernels: per-channel key norm, group quantisation into the ROW / BLOCK stores
+// (prefill and quantise-on-evict share the same device routines), window copies, canonical export.
+#include "innerq_device.cuh"
+#include "innerq_kernels.h"
+
+namespace iq {
+
+// ------------------------------------------------------------------ key norm
+// absmax[u][c] = max_t |K[u][t][c]| as fp32 bit patterns (non-negative floats order like uints).
+__global__ void __launch_bounds__(256) k_absmax_kernel(const __half* __restrict__ K, int N, int rows_per_block,
+                                                       uint32_t* __restrict__ absmax) {
+  const int u = blockIdx.y;
+  const int t0 = blockIdx.x * rows_per_block;
+  const int t1 = min(N, t0 + rows_per_block);
+  const int cg = threadIdx.x & 15;      // 8 channels each
+  const int rg = threadIdx.x >> 4;      // 16 rows in flight
+  const uint4* base = reinterpret_cast<const uint4*>(K + (size_t)u * N * kD);
+  __half2 m[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) m[i] = __float2half2_rn(0.f);
+  for (int t = t0 + rg; t < t1; t += 16) {
+    uint4 v = __ldg(base + (size_t)t * 16 + cg);
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m[i] = __hmax2(m[i], __habs2(h[i]));
+  }
+  __shared__ float red[16][kD];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    red[rg][cg * 8 + 2 * i] = __low2float(m[i]);
+    red[rg][cg * 8 + 2 * i + 1] = __high2float(m[i]);
+  }
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    float v = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v = fmaxf(v, red[i][threadIdx.x]);
+    atomicMax(absmax + (size_t)u * kD + threadIdx.x, __float_as_uint(v));
+  }
+}
+
+// norm = sqrt(absmax), 0 -> 1  (Section "Per-channel Normalization of K")
+__global__ void finalize_norm_kernel(const uint32_t* __restrict__ absmax, float* __restrict__ norm, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    float n_ = __fsqrt_rn(__uint_as_float(absmax[i]));
+    norm[i] = n_ == 0.f ? 1.0f : n_;
+  }
+}
+
+__global__ void fill_float_kernel(float* p, float v, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+
+// ------------------------------------------------------------------ ROW store quantiser
+// One warp quantises one token: lane l holds channels 4l..4l+3; a group of G channels is G/4
+// adjacent lanes.  `stage` is this warp's zero-initialised packed row in shared memory.
+__device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src, const float* __restrict__ norm,
+                                                  const Layout& L, const Store& S, uint32_t* stage,
+                                                  uint32_t* __restrict__ dst_row, void* __restrict__ dst_meta, size_t meta_idx) {
+  const int lane = threadIdx.x & 31;
+  const int gl = L.G >> 2;   // lanes per group
+  float x[4];
+  {
+    uint2 raw = *reinterpret_cast<const uint2*>(src + 4 * lane);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+    float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
+    x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+  }
+  if (norm) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) x[i] = __fmul_rn(x[i], __fdiv_rn(1.0f, norm[4 * lane + i]));
+  }
+  float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+  float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+  float am = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+  for (int o = gl >> 1; o > 0; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+  }
+  GroupParams p = group_params(mn, mx, am, S.bits, L.sym_variant);
+  float ua[4], qs[4], ea = 0.f, es = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    ua[i] = asym_code(p, x[i]);
+    qs[i] = sym_code(p, x[i]);
+    ea += asym_err(p, x[i], ua[i]);
+    es += sym_err(p, x[i], qs[i]);
+  }
+  for (int o = gl >> 1; o > 0; o >>= 1) {
+    ea += __shfl_xor_sync(0xffffffffu, ea, o);
+    es += __shfl_xor_sync(0xffffffffu, es, o);
+  }
+  const bool asym = choose_asym(S.mode, ea, es);
+  const int words = row_bytes(S.bits) / 4;
+  if (lane < words) stage[lane] = 0u;
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
+    row_put(stage, 4 * lane + i, S.bits, code);
+  }
+  __syncwarp();
+  if (lane < words) dst_row[lane] = stage[lane];
+  if ((lane % gl) == 0) store_meta(dst_meta, meta_idx + lane / gl, S.meta_bytes, group_meta(p, asym));
+  __syncwarp();
+}
+
+// Prefill: rows [0, n_q) of every unit; token of row i is w_sink + i.
+__global__ void __launch_bounds__(128) quantize_rows_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
+                                                            int n_q, unsigned char* __restrict__ cache,
+                                                            bool use_norm) {
+  __shared__ uint32_t stage[4][16];
+  const int u = blockIdx.y, warp = threadIdx.x >> 5;
+  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
+  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
+  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  const int rw = row_bytes(S.bits) / 4;
+  for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4) {
+    const __half* src = X + ((size_t)u * N + L.w_sink + i) * kD;
+    quantize_row_warp(src, norm, L, S, stage[warp], codes + (size_t)i * rw, meta, (size_t)i * S.n_groups);
+  }
+}
+
+// ------------------------------------------------------------------ BLOCK store quantiser
+// A 128-thread CTA quantises one group of G tokens x 128 channels; thread c owns channel c.
+// tile: fp16 [G][D] staging; words: packed chunks of the group (zeroed here).
+__device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* __restrict__ norm, const Layout& L,
+                                   const Store& S, __half* tile, uint32_t* words, uint32_t* __restrict__ dst_chunks,
+                                   void* __restrict__ dst_meta, size_t meta_idx) {
+  const int G = L.G, c = threadIdx.x;
+  const int cw = chunk_bytes(S.bits) / 4;
+  const int n_words = (G / kChunk) * cw;
+  for (int i = threadIdx.x; i < G * 16; i += 128) {        // 16 x 16-byte pieces per token row
+    int t = i >> 4, piece = i & 15;
+    reinterpret_cast<uint4*>(tile)[i] = *reinterpret_cast<const uint4*>(src.row(t_first + t) + piece * 8);
+  }
+  for (int i = threadIdx.x; i < n_words; i += 128) words[i] = 0u;
+  __syncthreads();
+  const float inv = norm ? __fdiv_rn(1.0f, norm[c]) : 1.0f;
+  float mn = INFINITY, mx = -INFINITY, am = 0.f;
+  for (int t = 0; t < G; ++t) {
+    float x = __half2float(tile[t * kD + c]);
+    if (norm) x = __fmul_rn(x, inv);
+    mn = fminf(mn, x); mx = fmaxf(mx, x); am = fmaxf(am, fabsf(x));
+  }
+  GroupParams p = group_params(mn, mx, am, S.bits, L.sym_variant);
+  float ea = 0.f, es = 0.f;
+  if (S.mode == 2) {
+    for (int t = 0; t < G; ++t) {
+      float x = __half2float(tile[t * kD + c]);
+      if (norm) x = __fmul_rn(x, inv);
+      ea += asym_err(p, x, asym_code(p, x));
+      es += sym_err(p, x, sym_code(p, x));
+    }
+  }
+  const bool asym = choose_asym(S.mode, ea, es);
+  for (int t = 0; t < G; ++t) {
+    float x = __half2float(tile[t * kD + c]);
+    if (norm) x = __fmul_rn(x, inv);
+    uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
+    chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
+  }
+  store_meta(dst_meta, meta_idx + c, S.meta_bytes, group_meta(p, asym));
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_words; i += 128) dst_chunks[i] = words[i];
+  __syncthreads();
+}
+
+// Prefill: groups [0, n_q / G) of every unit; group j covers tokens w_sink + jG .. + G - 1.
+__global__ void __launch_bounds__(128) quantize_blocks_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
+                                                              int n_q, unsigned char* __restrict__ cache,
+                                                              bool use_norm) {
+  __shared__ __align__(16) __half tile[128 * kD];
+  __shared__ uint32_t words[4 * 512];
+  const int u = blockIdx.y;
+  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
+  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
+  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  const int cw = chunk_bytes(S.bits) / 4, cpg = L.G / kChunk;
+  TokSrc src{X + (size_t)u * N * kD, 0, 0};
+  for (int j = blockIdx.x; j < n_q / L.G; j += gridDim.x)
+    quantize_block_cta(src, L.w_sink + j * L.G, norm, L, S, tile, words, codes + (size_t)j * cpg * cw,
+                       meta, (size_t)j * kD);
+}
+
+// ------------------------------------------------------------------ window copies (prefill)
+// Copies tokens [t0, t1) of the input into the sink (t < w_sink) or the recent ring.
+__global__ void copy_window_kernel(Layout L, Store S, const __half* __restrict__ X, int N, int t0, int t1,
+                                   unsigned char* __restrict__ cache) {
+  const int u = blockIdx.y;
+  const int n = (t1 - t0) * 16;
+  __half* sink = reinterpret_cast<__half*>(cache + S.sink_off + (size_t)u * S.sink_stride);
+  __half* ring = reinterpret_cast<__half*>(cache + S.ring_off + (size_t)u * S.ring_stride);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    int t = t0 + (i >> 4), piece = i & 15;
+    uint4 v = *reinterpret_cast<const uint4*>(X + ((size_t)u * N + t) * kD + piece * 8);
+    __half* dst = t < L.w_sink ? sink + (size_t)t * kD : ring + (size_t)((t - L.w_sink) % S.ring_cap) * kD;
+    *reinterpret_cast<uint4*>(dst + piece * 8) = v;
+  }
+}
+
+// ------------------------------------------------------------------ append (quantise-on-evict)
+// One CTA per unit.  N is the token count after this append.  Writes the new token into the sink
+// or ring; then, if the store's recent window overflows, quantises the oldest token (ROW) or the
+// oldest G tokens (BLOCK) out of the ring.  Which of these happens is a function of N alone.
+__device__ void append_store(const Layout& L, const Store& S, const __half* __restrict__ x_new, int N, int u,
+                             unsigned char* __restrict__ cache, bool use_norm, __half* tile, uint32_t* words) {
+  if (S.kind == kNone) {       // unquantised cache: everything lives in the "sink" array
+    __half* sink = reinterpret_cast<__half*>(cache + S.sink_off + (size_t)u * S.sink_stride);
+    sink[(size_t)(N - 1) * kD + threadIdx.x] = x_new[threadIdx.x];
+    return;
+  }
+  const int t_new = N - 1;
+  __half* sink = reinterpret_cast<__half*>(cache + S.sink_off + (size_t)u * S.sink_stride);
+  __half* ring = reinterpret_cast<__half*>(cache + S.ring_off + (size_t)u * S.ring_stride);
+  if (t_new < L.w_sink) {
+    sink[(size_t)t_new * kD + threadIdx.x] = x_new[threadIdx.x];
+    return;
+  }
+  ring[(size_t)((t_new - L.w_sink) % S.ring_cap) * kD + threadIdx.x] = x_new[threadIdx.x];
+  const int nq_before = n_quantised(S.kind, N - 1, L.w_sink, L.w_recent, L.G);
+  const int nq_after = n_quantised(S.kind, N, L.w_sink, L.w_recent, L.G);
+  if (nq_after == nq_before) return;
+  __syncthreads();      // the ring row written above may be among the evicted tokens
+  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
+  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
+  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  TokSrc src{ring, S.ring_cap, L.w_sink};
+  if (S.kind == kRow) {
+    if (threadIdx.x < 32)
+      quantize_row_warp(src.row(L.w_sink + nq_before), norm, L, S, words, codes + (size_t)nq_before * (row_bytes(S.bits) / 4),
+                        meta, (size_t)nq_before * S.n_groups);
+  } else {
+    const int j = nq_before / L.G;
+    quantize_block_cta(src, L.w_sink + nq_before, norm, L, S, tile, words,
+                       codes + (size_t)j * (L.G / kChunk) * (chunk_bytes(S.bits) / 4), meta, (size_t)j * kD);
+  }
+}
+
+__global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
+                                                     const __half* __restrict__ v_new, int N,
+                                                     unsigned char* __restrict__ cache) {
+  __shared__ __align__(16) __half tile[128 * kD];
+  __shared__ uint32_t words[4 * 512];
+  const int u = blockIdx.x;
+  append_store(L, L.k, k_new + (size_t)u * kD, N, u, cache, L.k_normalize != 0, tile, words);
+  __syncthreads();
+  append_store(L, L.v, v_new + (size_t)u * kD, N, u, cache, false, tile, words);
+}
+
+// ------------------------------------------------------------------ canonical export
+__global__ void export_store_kernel(Layout L, Store S, const unsigned char* __restrict__ cache, int n_q, int n_sink,
+                                    int n_recent, uint8_t* __restrict__ code, uint16_t* __restrict__ scale,
+                                    uint16_t* __restrict__ zero, uint16_t* __restrict__ sink_out,
+                                    uint16_t* __restrict__ recent_out) {
+  const int u = blockIdx.y;
+  const int cap = L.max_tokens;
+  const uint32_t* codes = reinterpret_cast<const uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
+  const void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  const int stride = gridDim.x * blockDim.x, tid0 = blockIdx.x * blockDim.x + threadIdx.x;
+  if (code && S.kind != kNone) {
+    for (int i = tid0; i < n_q * kD; i += stride) {
+      int t = i / kD, c = i % kD;
+      uint32_t v = S.kind == kRow
+                       ? row_code(codes + (size_t)t * (row_bytes(S.bits) / 4), c, S.bits)
+                       : chunk_code(codes + (size_t)(t / kChunk) * (chunk_bytes(S.bits) / 4), t % kChunk, c, S.bits);
+      code[((size_t)u * cap + t) * kD + c] = (uint8_t)v;
+    }
+  }
+  if (S.kind != kNone) {
+    const int n_meta_rows = S.kind == kRow ? n_q : n_q / L.G;
+    const int rows_cap = S.kind == kRow ? cap : cap / L.G + 1;
+    for (int i = tid0; i < n_meta_rows * S.n_groups; i += stride) {
+      uint32_t m = load_meta(meta, i, S.meta_bytes);
+      size_t o = (size_t)u * rows_cap * S.n_groups + i;
+      if (scale) scale[o] = (uint16_t)(m & 0xFFFFu);
+      if (zero) zero[o] = (uint16_t)(m >> 16);
+    }
+  }
+  const uint16_t* sink = reinterpret_cast<const uint16_t*>(cache + S.sink_off + (size_t)u * S.sink_stride);
+  const uint16_t* ring = reinterpret_cast<const uint16_t*>(cache + S.ring_off + (size_t)u * S.ring_stride);
+  const int sink_cap = S.kind == kNone ? L.max_tokens : L.w_sink;
+  if (sink_out)
+    for (int i = tid0; i < n_sink * kD; i += stride) sink_out[(size_t)u * sink_cap * kD + i] = sink[i];
+  if (recent_out && S.kind != kNone) {
+    const int t_first = n_sink + n_q;   // absolute token of the oldest recent entry
+    for (int i = tid0; i < n_recent * kD; i += stride) {
+      int t = t_first + i / kD, c = i % kD;
+      recent_out[(size_t)u * (L.w_recent + L.G) * kD + i] = ring[(size_t)((t - L.w_sink) % S.ring_cap) * kD + c];
+    }
+  }
+}
+
+// ------------------------------------------------------------------ host launchers
+static inline int grid_for(int n, int per_block, int cap) {
+  int g = (n + per_block - 1) / per_block;
+  return g < 1 ? 1 : (g > cap ? cap : g);
+}
+
+int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, const __half* K, const __half* V, int N,
+                   cudaStream_t st) {
+  int launches = 0;
+  const Counts cn = counts_for(L, N);
+  float* norm = reinterpret_cast<float*>(cache + L.norm_off);
+  const bool use_norm = L.k_normalize != 0 && L.k.kind != kNone;
+  if (use_norm && N > 0) {
+    uint32_t* absmax = reinterpret_cast<uint32_t*>(ws + L.ws_absmax_off);
+    if (cudaMemsetAsync(absmax, 0, (size_t)L.U * kD * 4, st) != cudaSuccess) return -1;
+    const int rows_per_block = 512;
+    dim3 g((N + rows_per_block - 1) / rows_per_block, L.U);
+    k_absmax_kernel<<<g, 256, 0, st>>>(K, N, rows_per_block, absmax);
+    finalize_norm_kernel<<<(L.U * kD + 255) / 256, 256, 0, st>>>(absmax, norm, L.U * kD);
+    launches += 2;
+  } else {
+    fill_float_kernel<<<(L.U * kD + 255) / 256, 256, 0, st>>>(norm, 1.0f, L.U * kD);
+    launches += 1;
+  }
+  const Store* stores[2] = {&L.k, &L.v};
+  const __half* srcs[2] = {K, V};
+  const int nq[2] = {cn.n_qk, cn.n_qv};
+  for (int i = 0; i < 2; ++i) {
+    const Store& S = *stores[i];
+    if (N == 0) break;
+    if (S.kind == kNone) {      // unquantised: the whole input goes to the "sink" array
+      Layout Lf = L;
+      Lf.w_sink = L.max_tokens;
+      copy_window_kernel<<<dim3(grid_for(N * 16, 256, 1024), L.U), 256, 0, st>>>(Lf, S, srcs[i], N, 0, N, cache);
+      launches += 1;
+      continue;
+    }
+    const bool nrm = use_norm && i == 0;
+    if (nq[i] > 0) {
+      if (S.kind == kRow)
+        quantize_rows_kernel<<<dim3(grid_for(nq[i], 4 * 8, 4096), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i], cache, nrm);
+      else
+        quantize_blocks_kernel<<<dim3(grid_for(nq[i] / L.G, 1, 8192), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i], cache,
+                                                                                       nrm);
+      launches += 1;
+    }
+    // fp16 windows: sink, then everything after the quantised middle
+    if (cn.n_sink > 0) {
+      copy_window_kernel<<<dim3(1, L.U), 256, 0, st>>>(L, S, srcs[i], N, 0, cn.n_sink, cache);
+      launches += 1;
+    }
+    const int t_rec = cn.n_sink + nq[i];
+    if (N > t_rec) {
+      copy_window_kernel<<<dim3(grid_for((N - t_rec) * 16, 256, 64), L.U), 256, 0, st>>>(L, S, srcs[i], N, t_rec, N, cache);
+      launches += 1;
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
+                  cudaStream_t st) {
+  append_kernel<<<L.U, 128, 0, st>>>(L, k_new, v_new, N_after, cache);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st) {
+  const Counts cn = counts_for(L, N);
+  const bool fp16 = L.k.kind == kNone;
+  export_store_kernel<<<dim3(64, L.U), 256, 0, st>>>(L, L.k, cache, cn.n_qk, fp16 ? N : cn.n_sink, cn.n_k_recent, e.k_code,
+                                                    e.k_scale, e.k_zero, e.k_sink, e.k_recent);
+  export_store_kernel<<<dim3(64, L.U), 256, 0, st>>>(L, L.v, cache, cn.n_qv, fp16 ? N : cn.n_sink, cn.n_v_recent, e.v_code,
+                                                    e.v_scale, e.v_zero, e.v_sink, e.v_recent);
+  if (e.norm)
+    if (cudaMemcpyAsync(e.norm, cache + L.norm_off, (size_t)L.U * kD * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return -1;
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+}  // namespace iq

@@ -1,0 +1,75 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates arguments, and its packed layout has the paper's effective bit-widths."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2602_23200_b200 import binding as B
+from paper_2602_23200_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "innerq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(innerq_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 10
+    assert sorted(B.EXPORTED_SYMBOLS) == names
+    lib = C.CDLL(B.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_status_strings():
+    for code in range(-5, 1):
+        assert B.status_string(code) not in ("", "unknown status")
+    assert B.status_string(-99) == "unknown status"
+
+
+def test_config_validation_without_gpu():
+    ok = B.make_config(synth.config1())
+    cb, wb = B.innerq_cache_bytes(ok)
+    assert cb > 0 and wb > 0 and cb % 256 == 0
+    for field, bad, status in [("head_dim", 64, -2), ("group", 48, -2), ("k_bits", 5, -2), ("batch", 0, -1),
+                               ("n_q_heads", 3, -1), ("max_tokens", 0, -1), ("k_mode", 7, -1), ("grouping", 3, -1)]:
+        cfg = B.make_config(synth.config1().with_(n_q_heads=2, n_kv_heads=2), **{field: bad})
+        with pytest.raises(B.InnerQError) as ei:
+            B.innerq_cache_bytes(cfg)
+        assert ei.value.status == status, field
+    with pytest.raises(B.InnerQError):      # the outer-grouped method has no key normalisation
+        B.innerq_cache_bytes(B.make_config(synth.config1(), grouping=B.GROUPING_OUTER, k_normalize=1))
+
+
+def test_packed_payload_matches_table_bits():
+    # Table "bits" (G = 32, head dim 128): effective bits per cached number = payload bytes * 8 / 128.
+    rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table_bits.txt"))
+            if l.strip() and not l.startswith("#")]
+    for name, kb, kz, vb, vz, eff in rows:
+        if name == "KIVI":
+            cfg = B.make_config(synth.config1(), k_bits=int(kb), v_bits=int(vb), grouping=B.GROUPING_OUTER,
+                                k_normalize=0, k_mode=B.MODE_ASYM, v_mode=B.MODE_ASYM)
+        else:
+            cfg = B.make_config(synth.config1(), k_bits=int(kb), v_bits=int(vb),
+                                k_mode=B.MODE_HYBRID if int(kz) else B.MODE_SYM,
+                                v_mode=B.MODE_HYBRID if int(vz) else B.MODE_SYM)
+        k_bytes, v_bytes = B.innerq_token_payload_bytes(cfg)
+        assert (k_bytes + v_bytes) * 8 / (2 * 128) == pytest.approx(float(eff)), name
+
+
+def test_cache_size_tracks_payload():
+    # the buffer the caller must provide is the payload plus windows, norms and alignment: within 2 %
+    # for a long context
+    w = synth.config4()
+    cfg = B.make_config(w)
+    cb, _ = B.innerq_cache_bytes(cfg)
+    k_bytes, v_bytes = B.innerq_token_payload_bytes(cfg)
+    payload = w.n_units * w.n_tokens * (k_bytes + v_bytes)
+    assert payload <= cb <= 1.02 * payload
+    assert cb < 0.16 * (2 * w.n_units * w.n_tokens * 128 * 2)      # 2.25 bits vs 16 bits per number

@@ -1,0 +1,185 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+
+from oracle import innerq_oracle as O
+from paper_2602_23200_b200 import synth
+from tests import _parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def gpu_cache(w, max_tokens=None, **opts):
+    from paper_2602_23200_b200 import binding as B
+    cfg = B.make_config(w, max_tokens=max_tokens or w.n_tokens + 300)
+    return B.InnerQCache(cfg)
+
+
+def dev(x):
+    torch = _torch()
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def run_prefill_both(w, max_tokens=None):
+    K, V = synth.kv_all(w)
+    oc = O.from_workload(w, max_tokens=max_tokens or w.n_tokens + 300)
+    oc.prefill(K, V)
+    gc = gpu_cache(w, max_tokens)
+    gc.innerq_quantize_prefill(dev(K), dev(V))
+    return oc, gc, K, V
+
+
+def check_decode(w, oc, gc, step=0, variants=(0,), splits=(0,)):
+    q = synth.query(w, step)
+    ref = oc.decode(q)
+    worst = 0.0
+    for variant in variants:
+        for s in splits:
+            gc.innerq_set_decode_options(s, variant)
+            out = gc.innerq_decode_attention(dev(q)).cpu().numpy()
+            worst = max(worst, P.assert_outputs_close(out, ref, f"{w.name} variant={variant} splits={s}"))
+    gc.innerq_set_decode_options(0, 0)
+    return worst
+
+
+CASES = [
+    # bits, G, mode, sym_variant, N
+    (2, 32, O.HYBRID, 0, 333),
+    (2, 32, O.HYBRID, 1, 333),
+    (2, 64, O.ASYM, 0, 420),
+    (2, 128, O.HYBRID, 0, 700),
+    (3, 32, O.HYBRID, 0, 333),
+    (3, 64, O.SYM, 0, 300),
+    (4, 64, O.HYBRID, 0, 420),
+    (4, 32, O.SYM, 1, 333),
+    (4, 128, O.ASYM, 0, 541),
+]
+
+
+@pytest.mark.parametrize("bits,G,mode,variant,N", CASES)
+def test_prefill_and_decode_inner(bits, G, mode, variant, N):
+    w = synth.tiny(n_tokens=N, group=G, k_bits=bits, v_bits=bits, k_mode=mode, v_mode=mode, sym_variant=variant)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, mode == O.HYBRID, mode == O.HYBRID)
+    check_decode(w, oc, gc, variants=(0, 1), splits=(0, 1, 3, 7))
+
+
+@pytest.mark.parametrize("bits,G,N", [(2, 32, 333), (3, 64, 420), (4, 128, 541)])
+def test_prefill_and_decode_outer(bits, G, N):
+    w = synth.tiny(n_tokens=N, group=G, k_bits=bits, v_bits=bits, grouping=O.OUTER, k_normalize=0,
+                   k_mode=O.ASYM, v_mode=O.ASYM)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.OUTER, G, False, False)
+    check_decode(w, oc, gc, splits=(0, 2))
+
+
+def test_fp16_cache_decode():
+    w = synth.tiny(n_tokens=500, grouping=O.FP16, k_normalize=0)
+    oc, gc, K, V = run_prefill_both(w)
+    e = gc.innerq_cache_export()
+    assert e["n_tokens"] == 500 and np.array_equal(e["k_sink"].reshape(K.shape), K)
+    check_decode(w, oc, gc, splits=(0, 1, 5))
+    for step in range(3):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+    check_decode(w, oc, gc, step=1)
+
+
+def test_mixed_bits_and_modes():
+    w = synth.tiny(n_tokens=400, group=32, k_bits=3, v_bits=2, k_mode=O.SYM, v_mode=O.HYBRID)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, 32, False, True)
+    check_decode(w, oc, gc, variants=(0, 1))
+
+
+@pytest.mark.parametrize("N", [1, 3, 4, 5, 19, 20, 21, 52, 53])
+def test_short_contexts_and_window_edges(N):
+    # N <= w_sink, N <= w_sink + w_recent (nothing quantised), first quantised key token, first value group
+    w = synth.tiny(n_tokens=N)
+    oc, gc, K, V = run_prefill_both(w)
+    e, eo = gc.innerq_cache_export(), oc.export()
+    P.assert_export_equal(e, eo, O.INNER, w.group)
+    check_decode(w, oc, gc, variants=(0, 1))
+    if N <= w.w_sink + w.w_recent:
+        # every token is in a window: the result is plain attention on the fp16 inputs
+        q = synth.query(w)
+        out = gc.innerq_decode_attention(dev(q)).cpu().numpy()
+        for b in range(w.batch):
+            for j in range(w.n_q_heads):
+                h = j // w.q_per_kv
+                ref = O.dense_attention(q[b, j], K[b, h], V[b, h])
+                P.assert_outputs_close(out[b, j][None], ref[None], "all-window")
+
+
+def test_empty_prefill_then_appends_through_every_phase():
+    # start from an empty cache; append through sink fill, recent fill, first key eviction, value evictions
+    w = synth.tiny(n_tokens=0, w_sink=4, w_recent=16, group=32)
+    oc = O.from_workload(w, max_tokens=200)
+    gc = gpu_cache(w, max_tokens=200)
+    torch = _torch()
+    gc.innerq_quantize_prefill(torch.empty((w.batch, w.n_kv_heads, 0, 128), dtype=torch.float16, device="cuda"),
+                               torch.empty((w.batch, w.n_kv_heads, 0, 128), dtype=torch.float16, device="cuda"))
+    for step in range(120):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        if step in (0, 3, 4, 19, 20, 21, 51, 52, 83, 84, 119):
+            P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
+            check_decode(w, oc, gc, step=step, variants=(0, 1))
+
+
+@pytest.mark.parametrize("grouping", [O.INNER, O.OUTER])
+def test_prefill_then_appends_matches_oracle(grouping):
+    w = synth.tiny(n_tokens=150, grouping=grouping, k_normalize=int(grouping == O.INNER), append_scale=0.5,
+                   k_mode=O.HYBRID if grouping == O.INNER else O.ASYM,
+                   v_mode=O.HYBRID if grouping == O.INNER else O.ASYM)
+    oc, gc, _, _ = run_prefill_both(w)
+    for step in range(100):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        if step % 33 == 32:
+            check_decode(w, oc, gc, step=step)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), grouping, w.group,
+                          grouping == O.INNER, grouping == O.INNER)
+    check_decode(w, oc, gc, step=1000, variants=(0, 1) if grouping == O.INNER else (0,))
+
+
+def test_capacity_and_argument_errors():
+    from paper_2602_23200_b200 import binding as B
+    torch = _torch()
+    w = synth.tiny(n_tokens=40)
+    gc = gpu_cache(w, max_tokens=41)
+    K, V = synth.kv_all(w)
+    gc.innerq_quantize_prefill(dev(K), dev(V))
+    k1, v1 = synth.new_token(w, 0)
+    gc.innerq_append_token(dev(k1), dev(v1))
+    with pytest.raises(B.InnerQError) as ei:
+        gc.innerq_append_token(dev(k1), dev(v1))
+    assert ei.value.status == -3 and gc.n_tokens == 41
+    K2, V2 = synth.kv_all(w.with_(n_tokens=42))
+    with pytest.raises(B.InnerQError) as ei:
+        gc.innerq_quantize_prefill(dev(K2), dev(V2))
+    assert ei.value.status == -3 and gc.n_tokens == 41
+    empty = gpu_cache(w, max_tokens=41)
+    q = dev(synth.query(w))
+    with pytest.raises(B.InnerQError) as ei:
+        empty.innerq_decode_attention(q)
+    assert ei.value.status == -1
+    # the context is still healthy
+    out = gc.innerq_decode_attention(q)
+    assert torch.isfinite(out.float()).all()
+
+
+def test_config1_full_parity():
+    w = synth.config1()
+    oc, gc, _, _ = run_prefill_both(w)
+    flips = P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
+    worst = check_decode(w, oc, gc, variants=(0, 1), splits=(0, 1, 4, 13))
+    print(f"config1: contested flips {flips}, worst err/tol {worst:.3f}")
