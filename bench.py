@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the InnerQ decode path on B200.
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: innerq_append_token
+(one new fp16 token per KV head, quantise-on-evict) followed by innerq_decode_attention over the
+whole packed cache.  The default workload is the 7B-class MHA configuration (32 heads, head_dim
+128, batch 1, 32768 tokens of context, 2-bit, group 32, sink 4, recent 128).
+
+The packed cache of that workload (about 100 MB) would fit in the 126 MB L2, so the bench rotates
+over several independent cache instances (same contents, different memory; total several times
+the L2 size) and step i uses instance i mod R: every decode streams its cache from HBM.
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead (host cores).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2602_23200_b200 import synth  # noqa: E402
+
+D = 128
+
+
+def workload_by_name(name: str):
+    if name == "c1":
+        return synth.config1()
+    if name == "c2":
+        return synth.config2()
+    if name == "c3_4bit":
+        return synth.config3(4)
+    if name == "c3_2bit":
+        return synth.config3(2)
+    if name == "c4":
+        return synth.config4()
+    raise SystemExit(f"unknown workload {name}")
+
+
+def payload_bytes(w):
+    """(bytes per quantised K token, bytes per quantised V token) of one unit, dense zero-points."""
+    def row(bits, mode):
+        return 16 * bits + (D // w.group) * (2 if mode == synth.SYM else 4)
+
+    def blk(bits, mode):
+        return 16 * bits + D * (2 if mode == synth.SYM else 4) / w.group
+    if w.grouping == synth.FP16:
+        return 2 * D, 2 * D
+    if w.grouping == synth.INNER:
+        return row(w.k_bits, w.k_mode), blk(w.v_bits, w.v_mode)
+    return blk(w.k_bits, synth.ASYM), row(w.v_bits, synth.ASYM)
+
+
+def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
+    """Bytes one decode call must move: packed codes, scale/zero pairs, fp16 windows, q, out, norm.
+
+    Returns (dense, minimal): `dense` counts the zero-point of every group (they are stored dense);
+    `minimal` leaves out the zero-points of symmetric groups, which the result does not depend on."""
+    U = w.n_units
+    ws, wr, G = w.w_sink, w.w_recent, w.group
+    if w.grouping == synth.FP16:
+        b = U * N * 2 * D * 2 + 2 * w.batch * w.n_q_heads * D * 2
+        return b, b
+    mid = max(0, N - ws - wr)
+    row_q, blk_q = mid, (mid // G) * G
+    n_qk, n_qv = (row_q, blk_q) if w.grouping == synth.INNER else (blk_q, row_q)
+    kb, vb = payload_bytes(w)
+    n_sink = min(N, ws)
+    per_unit = n_qk * kb + n_qv * vb + (N - n_qk) * 2 * D + (N - n_qv) * 2 * D
+    extra = 2 * w.batch * w.n_q_heads * D * 2 + (U * D * 4 if w.k_normalize else 0)
+    dense = U * per_unit + extra
+    k_groups = n_qk * (D // G) if w.grouping == synth.INNER else (n_qk // G) * D
+    v_groups = (n_qv // G) * D if w.grouping == synth.INNER else n_qv * (D // G)
+    k_has_z = (w.k_mode != synth.SYM) or w.grouping == synth.OUTER
+    v_has_z = (w.v_mode != synth.SYM) or w.grouping == synth.OUTER
+    minimal = dense - U * 2 * (k_groups * sym_frac_k * k_has_z + v_groups * sym_frac_v * v_has_z)
+    del n_sink
+    return float(dense), float(minimal)
+
+
+class ClockSampler(threading.Thread):
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self._stop_evt = index, [], threading.Event()
+
+    def run(self):
+        while not self._stop_evt.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                if len(f) >= 6:
+                    self.samples.append(f)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.05)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=6)
+        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+def measured_peak_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def stored_traffic(workload: str):
+    """DRAM bytes per decode launch from the committed ncu summary, if any."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "decode_traffic.json")) as f:
+            return json.load(f).get(workload)
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------------------------- oracle legs
+def oracle_steps(w, n_steps, units=None):
+    """Times the CPU oracle on `n_steps` steps (append + decode).  Returns (seconds per step, bytes per step, cores)."""
+    from oracle import innerq_oracle as O
+    sub = w if units is None else w.with_(batch=1, n_q_heads=units * w.q_per_kv, n_kv_heads=units)
+    K, V = synth.kv_all(sub)
+    oc = O.from_workload(sub, max_tokens=sub.n_tokens + n_steps + 8)
+    oc.prefill(K, V)
+    del K, V
+    times, nbytes = [], []
+    for step in range(n_steps):
+        k1, v1 = synth.new_token(sub, step)
+        q = synth.query(sub, step)
+        t0 = time.perf_counter()
+        oc.append(k1, v1)
+        oc.decode(q)
+        times.append(time.perf_counter() - t0)
+        nbytes.append(decode_algorithmic_bytes(sub, oc.N)[0])
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    return float(np.mean(times)), float(np.mean(nbytes)), cores
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    units = min(w.n_units, 4)
+    for _ in range(args.warmup and 1):
+        pass
+    t, b, cores = oracle_steps(w, max(1, min(args.steps, 8)), units=units)
+    gbs = b / t / 1e9
+    line = {"impl": "reference", "metric": "decode_step_algorithmic_hbm_gbs", "value": gbs, "unit": "GB/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+            "us_per_step": t * 1e6 * (w.n_units / units), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w, args),
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{units} of {w.n_units} KV heads, {max(1, min(args.steps, 8))} steps of append+decode"},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_dict(w, args):
+    return {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+            "head_dim": w.head_dim, "context": w.n_tokens, "k_bits": w.k_bits, "v_bits": w.v_bits, "group": w.group,
+            "w_sink": w.w_sink, "w_recent": w.w_recent, "grouping": ["inner", "outer", "fp16"][w.grouping],
+            "step": "innerq_append_token + innerq_decode_attention",
+            "l2": f"rotating {args.instances} cache instances (> L2) so every decode streams from HBM"}
+
+
+# ------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_23200_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    R, Kst, W = args.instances, args.steps, max(args.warmup, 3)
+    total_steps = W + Kst
+    e2e_steps = max(4, min(Kst, 32))
+    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps) // R + 8)
+    Kh, Vh = synth.kv_all(w)
+    Kd, Vd = torch.from_numpy(Kh).cuda(), torch.from_numpy(Vh).cuda()
+    caches = []
+    for _ in range(R):
+        c = B.InnerQCache(cfg)
+        c.innerq_quantize_prefill(Kd, Vd)
+        if args.splits or args.variant:
+            c.innerq_set_decode_options(args.splits, args.variant)
+        caches.append(c)
+    # fraction of symmetric groups (their zero-points are not needed by the result)
+    ex = caches[0].innerq_cache_export(codes=False)
+    sym_k = float(1.0 - ((ex["k_scale"] & 0x8000) != 0).mean()) if "k_scale" in ex and ex["k_scale"].size else 0.0
+    sym_v = float(1.0 - ((ex["v_scale"] & 0x8000) != 0).mean()) if "v_scale" in ex and ex["v_scale"].size else 0.0
+    del Kd, Vd, Kh, Vh, ex
+    torch.cuda.empty_cache()
+
+    n_in = total_steps + e2e_steps
+    toks = [synth.new_token(w, s) for s in range(n_in)]
+    qs = [synth.query(w, s) for s in range(n_in)]
+    k_new = torch.from_numpy(np.stack([t[0] for t in toks])).cuda()
+    v_new = torch.from_numpy(np.stack([t[1] for t in toks])).cuda()
+    q_all = torch.from_numpy(np.stack(qs)).cuda()
+    out = torch.empty_like(q_all[0])
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        c = caches[i % R]
+        c.innerq_append_token(k_new[i], v_new[i])
+        c.innerq_decode_attention(q_all[i], out)
+        return c
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(W):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.15)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dec_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Kst)]
+    launches = 0
+    bytes_dense = bytes_min = 0.0
+    barrier()
+    ev0.record(stream)
+    for j in range(Kst):
+        i = W + j
+        c = caches[i % R]
+        c.innerq_append_token(k_new[i], v_new[i])
+        dec_ev[j][0].record(stream)
+        c.innerq_decode_attention(q_all[i], out)
+        dec_ev[j][1].record(stream)
+        launches += c.innerq_last_launch_count(1) + c.innerq_last_launch_count(2)
+        bd, bm = decode_algorithmic_bytes(w, c.n_tokens, sym_k, sym_v)
+        bytes_dense += bd
+        bytes_min += bm
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    dec_ms = [a.elapsed_time(b) for a, b in dec_ev]
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / Kst
+    value_gbs = world * (bytes_min / Kst) / (ms_step * 1e-3) / 1e9
+
+    # end to end: host buffers in, host buffer out, copies inside the timed region
+    kh = torch.from_numpy(np.stack([t[0] for t in toks])).pin_memory()
+    vh = torch.from_numpy(np.stack([t[1] for t in toks])).pin_memory()
+    qh = torch.from_numpy(np.stack(qs)).pin_memory()
+    oh = torch.empty_like(qh[0]).pin_memory()
+    kd, vd, qd = torch.empty_like(k_new[0]), torch.empty_like(v_new[0]), torch.empty_like(q_all[0])
+
+    def e2e_step(i):
+        c = caches[i % R]
+        kd.copy_(kh[i], non_blocking=True)
+        vd.copy_(vh[i], non_blocking=True)
+        qd.copy_(qh[i], non_blocking=True)
+        c.innerq_append_token(kd, vd)
+        c.innerq_decode_attention(qd, out)
+        oh.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+        return c
+
+    base = total_steps
+    e2e_step(base)
+    barrier()
+    t0 = time.perf_counter()
+    e2e_bytes = 0.0
+    for j in range(1, e2e_steps):
+        c = e2e_step(base + j)
+        e2e_bytes += decode_algorithmic_bytes(w, c.n_tokens, sym_k, sym_v)[1]
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / (e2e_steps - 1)
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_gbs = world * (e2e_bytes / (e2e_steps - 1)) / e2e_s / 1e9
+    h2d = (kh[0].numel() + vh[0].numel() + qh[0].numel()) * 2
+    d2h = oh.numel() * 2
+
+    if rank == 0:
+        peak, which = measured_peak_gbs()
+        dec_us = float(np.mean(dec_ms)) * 1e3
+        achieved = (bytes_min / Kst) / (dec_us * 1e-6) / 1e9
+        line = {
+            "metric": "decode_step_algorithmic_hbm_gbs", "value": value_gbs, "unit": "GB/s", "n_gpus": world,
+            "steps": Kst, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
+            "us_per_decode": dec_us, "us_per_decode_median": float(np.median(dec_ms)) * 1e3,
+            "us_per_decode_min": float(np.min(dec_ms)) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config_dict(w, args),
+            "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
+                                 "sym_group_fraction": {"k": sym_k, "v": sym_v}},
+            "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": which, "traffic": stored_traffic(w.name),
+                         "kernel": "innerq_decode_attention (split + merge)"},
+            "e2e": {"value": e2e_gbs, "unit": "GB/s", "us_per_step": e2e_s * 1e6, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches, "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            units = min(w.n_units, 4)
+            t, b, cores = oracle_steps(w, 3, units=units)
+            line["cpu_baseline"] = {"value": b / t / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                    "us_per_step_full_workload": t * 1e6 * (w.n_units / units),
+                                    "sample": f"{units} of {w.n_units} KV heads, 3 steps of append+decode"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--instances", type=int, default=4, help="cache instances rotated to defeat L2 residency")
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = workload_by_name(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
