@@ -146,6 +146,13 @@ int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_s
  * Errors: INVALID_ARG. */
 int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
 
+/* The decode kernel waits for its asynchronous copies with a bounded number of polls; if a wait ever
+ * runs out it records that in a device-side error word, contributes nothing for the affected token
+ * range and returns normally.  This call copies the word to the host and SYNCHRONISES `cuda_stream`
+ * (the only entry point that does).  Returns 0 (no error), 1 (a wait ran out since the cache was
+ * created) or a negative error code. */
+int innerq_read_device_error(innerq_cache_t* cache, void* cuda_stream);
+
 /* Number of kernels the last call of each kind launched (for launch accounting):
  * which = 0 prefill, 1 append, 2 decode.  Returns the count or a negative error code. */
 int innerq_last_launch_count(const innerq_cache_t* cache, int32_t which);

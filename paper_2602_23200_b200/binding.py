@@ -22,7 +22,8 @@ GROUPING_INNER, GROUPING_OUTER, GROUPING_FP16 = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "innerq_cache_bytes", "innerq_token_payload_bytes", "innerq_cache_create", "innerq_cache_destroy",
     "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
-    "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_status_string",
+    "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
+    "innerq_status_string",
 )
 
 
@@ -70,6 +71,7 @@ def lib() -> C.CDLL:
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
+    L.innerq_read_device_error.argtypes = [vp, vp]
     L.innerq_status_string.argtypes = [C.c_int]
     L.innerq_status_string.restype = C.c_char_p
     for name in EXPORTED_SYMBOLS:
@@ -191,6 +193,9 @@ class InnerQCache:
 
     def innerq_set_decode_options(self, n_splits: int = 0, variant: int = 0):
         _check(lib().innerq_set_decode_options(self._h, n_splits, variant), "innerq_set_decode_options")
+
+    def innerq_read_device_error(self, stream=None) -> int:
+        return _check(lib().innerq_read_device_error(self._h, _stream_ptr(stream)), "innerq_read_device_error")
 
     def innerq_last_launch_count(self, which: int) -> int:
         return _check(lib().innerq_last_launch_count(self._h, which), "innerq_last_launch_count")

@@ -86,8 +86,10 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   L.k_normalize = (c.grouping == INNERQ_GROUPING_INNER && c.k_normalize) ? 1 : 0;
   L.max_tokens = c.max_tokens;
   L.sm_scale = c.sm_scale > 0.f ? c.sm_scale : 0.08838834764831845f;   // 1/sqrt(128)
+  // partial slots per query head: token-range splits plus one per 32 tokens of the fp16 tail
   int ms = (4 * 148 + L.U - 1) / L.U;
-  L.max_splits = ms < 1 ? 1 : (ms > 64 ? 64 : ms);
+  ms = ms < 1 ? 1 : (ms > 64 ? 64 : ms);
+  L.max_splits = ms + (c.w_sink + c.w_recent + L.G + 31) / 32 + 1;
   size_t off = 0;
   L.norm_off = off; off = align_up(off + (size_t)L.U * kD * 4, 256);
   if (c.grouping == INNERQ_GROUPING_FP16) {
@@ -104,7 +106,7 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   size_t w = 0;
   L.ws_partial_off = w; w = align_up(w + (size_t)L.B * L.Hq * L.max_splits * kPartialStride * 4, 256);
   L.ws_absmax_off = w; w = align_up(w + (size_t)L.U * kD * 4, 256);
-  L.ws_ticket_off = w; w = align_up(w + (size_t)L.U * 4, 256);
+  L.ws_ticket_off = w; w = align_up(w + (size_t)(L.U + 8) * 4, 256);   // tickets [U], then the device error word
   L.workspace_bytes = w;
 }
 
@@ -241,6 +243,16 @@ int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t varia
   c->opt_splits = n_splits;
   c->opt_variant = variant;
   return INNERQ_OK;
+}
+
+int innerq_read_device_error(innerq_cache_t* c, void* cuda_stream) {
+  if (!c) return INNERQ_ERR_INVALID_ARG;
+  unsigned int flag = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&flag, c->ws + c->L.ws_ticket_off + (size_t)c->L.U * 4, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return INNERQ_ERR_CUDA;
+  return (int)flag;
 }
 
 int innerq_last_launch_count(const innerq_cache_t* c, int32_t which) {

@@ -1,11 +1,681 @@
-// Warp-MMA decode kernel for the INNER layout (placeholder until the kernel lands).
+// Fused decode attention over the packed InnerQ cache (INNER layout), one launch:
+//   q.K^T on packed key rows  ->  online softmax  ->  p.V on packed value chunks, split over token
+//   ranges, fp16 windows and the K/V skew zone in a tail CTA, cross-CTA merge by the last CTA to finish.
+//
+// Work decomposition.  A CTA owns one (batch, KV head) unit and a range of value groups; each of its
+// 8 warps owns a contiguous sub-range and streams it chunk by chunk (32 tokens) through a private ring
+// of shared-memory stages filled by 1-D bulk async copies (cp.async.bulk + mbarrier): packed key rows,
+// key scale/zero words, the packed value chunk and, at the end of each value group, its scale/zero
+// words.  The warp never synchronises with other warps until the final merge.
+//
+// Arithmetic.  Codes are never dequantised element by element.  Inner-dimension grouping lets scale and
+// zero-point leave the inner sum (Section "InnerQ": one scale per group, reused):
+//     q'.x^_t = sum_g ( S_tg * sum_{c in g} q'_c u_tc  +  z_tg * sum_{c in g} q'_c )
+//     sum_t p_t v^_tc = sum_j ( S_jc * sum_{t in j} p_t u_tc  +  z_jc * sum_{t in j} p_t )
+// The raw-code sums run on the tensor pipe (mma.sync m16n8k16, fp32 accumulate) so that the ALU pipe only
+// unpacks: `word & (field << pos)` is already an fp16 pair (two codes as subnormals scaled by 2^pos,
+// the scale folded into the other operand).  The other operand (q' or p) is split into fp16 hi + lo
+// columns, so the products carry fp32-level accuracy; up to 4 query heads of the KV head share one pass
+// over the codes (the 8 mma columns are 4 heads x {hi, lo}).  Scale and zero-point are then applied once
+// per (token, group) for keys and once per (group, channel) for values, in fp32.
 #include "innerq_device.cuh"
 #include "innerq_kernels.h"
 
 namespace iq {
-bool decode_mma_supported(const Layout&) { return false; }
-int launch_decode_mma(const Layout&, const unsigned char*, unsigned char*, int, const __half*, __half*, int,
-                      cudaStream_t) {
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kHeads = 4;              // query heads per pass (hi/lo columns: 8 mma columns)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait: gives up after kWaitLimit polls and reports it (the caller records an error and
+// skips the data instead of spinning forever).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+// fp16 hi / lo split of x, packed (hi in the low half-word, lo in the high half-word)
+__device__ __forceinline__ uint32_t split_hi_lo(float x) {
+  const __half hi = __float2half_rn(x);
+  const __half lo = __float2half_rn(x - __half2float(hi));
+  return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+}
+__device__ __forceinline__ float pow2i(int e) { return __int_as_float((e + 127) << 23); }   // 2^e, -126 <= e <= 127
+
+// Per bit-width constants of the packed formats (see innerq_layout.h).
+template <int BITS> struct Fmt;
+template <> struct Fmt<2> {
+  static constexpr uint32_t kField = 0x00030003u;
+  static constexpr int kKstepsPerWindow = 2;   // an 8-bit window of each half-word feeds 2 key k-steps
+  static constexpr int kRowWordsPerLane = 2;
+  static constexpr int kChunkWordsPerLane = 8;
+};
+template <> struct Fmt<4> {
+  static constexpr uint32_t kField = 0x000F000Fu;
+  static constexpr int kKstepsPerWindow = 1;
+  static constexpr int kRowWordsPerLane = 4;
+  static constexpr int kChunkWordsPerLane = 16;
+};
+
+template <int BITS, int G> struct StageLayout {
+  static constexpr int kNG = kD / G;
+  static constexpr int kKCodes = kChunk * 16 * BITS;
+  static constexpr int kKMeta = kChunk * kNG * 4;
+  static constexpr int kVCodes = 512 * BITS;
+  static constexpr int kVMeta = kD * 4;
+  static constexpr int kOffKMeta = kKCodes;
+  static constexpr int kOffVCodes = kOffKMeta + kKMeta;
+  static constexpr int kOffVMeta = kOffVCodes + kVCodes;
+  static constexpr int kBytes = kOffVMeta + kVMeta;
+  static constexpr int kStages = BITS == 2 ? 4 : 2;
+  static constexpr int kWarpBytes = kBytes * kStages;
+  static constexpr int kCtaBytes = kWarpBytes * kWarps + 1024;   // + barriers and small tables
+};
+
+struct DecodeArgs {
+  const unsigned char* cache;
+  unsigned char* ws;
+  const __half* q;
+  __half* out;
+  int n_splits;          // fast-path CTAs per unit (blockIdx.y < n_splits); blockIdx.y >= n_splits are tail CTAs
+  int n_tail_tiles;      // tail CTAs per unit, 32 list entries each
+  int groups_per_split;
+  int head0;             // first query head (within the KV head's r) handled by this launch
+};
+
+// ---- tail: fp16 windows, and key rows whose values are still fp16 (plain SIMT, small) ---------------
+// Token list of the tail: [0, n_sink) and [n_sink + n_qv, N).  One tail CTA handles one tile of 32 list
+// entries: it stages the tile's key rows (fp16 window rows, or dequantised skew-zone rows) and value rows
+// in shared memory with independent 128-bit loads, then scores, soft-maxes and accumulates from there.
+struct TailSmem {
+  float q_raw[kHeads][kD], q_nrm[kHeads][kD];
+  float k[32][kD + 4];
+  __half v[32][kD];
+  float sc[32][kHeads];
+  float m[kHeads], l[kHeads];
+  float acc2[kHeads][kD];
+  int quant[32];
+};
+
+__device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a, int u, int nh, int tile, TailSmem& S,
+                         float (&acc)[kHeads], float (&m_out)[kHeads], float (&l_out)[kHeads]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const Store& Ks = L.k;
+  const Store& Vs = L.v;
+  const __half* k_sink = reinterpret_cast<const __half*>(a.cache + Ks.sink_off + (size_t)u * Ks.sink_stride);
+  const __half* k_ring = reinterpret_cast<const __half*>(a.cache + Ks.ring_off + (size_t)u * Ks.ring_stride);
+  const __half* v_sink = reinterpret_cast<const __half*>(a.cache + Vs.sink_off + (size_t)u * Vs.sink_stride);
+  const __half* v_ring = reinterpret_cast<const __half*>(a.cache + Vs.ring_off + (size_t)u * Vs.ring_stride);
+  const uint32_t* k_codes = reinterpret_cast<const uint32_t*>(a.cache + Ks.code_off + (size_t)u * Ks.code_stride);
+  const void* k_meta = a.cache + Ks.meta_off + (size_t)u * Ks.meta_stride;
+  const int n_tail = cn.n_sink + (cn.N - cn.n_sink - cn.n_qv);
+  const int i0 = tile * 32;
+  // ---- stage the tile: 32 rows x 16 pieces of 8 channels
+#pragma unroll
+  for (int rep = 0; rep < 2; ++rep) {
+    const int idx = tid + rep * kThreads;
+    const int tt = idx >> 4, piece = idx & 15;
+    const int i = i0 + tt;
+    uint4 vraw = make_uint4(0u, 0u, 0u, 0u);
+    float kx[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    int quant = 0;
+    if (i < n_tail) {
+      const int t = i < cn.n_sink ? i : cn.n_qv + i;
+      const int iq = t - cn.n_sink;   // index among the packed key rows, if < n_qk
+      const __half* vrow = t < cn.n_sink ? v_sink + (size_t)t * kD : v_ring + (size_t)((t - L.w_sink) % Vs.ring_cap) * kD;
+      vraw = *reinterpret_cast<const uint4*>(vrow + piece * 8);
+      if (t < cn.n_sink || iq >= cn.n_qk) {
+        const __half* row = t < cn.n_sink ? k_sink + (size_t)t * kD : k_ring + (size_t)((t - L.w_sink) % Ks.ring_cap) * kD;
+        const uint4 raw = *reinterpret_cast<const uint4*>(row + piece * 8);
+        const __half2* hh = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 x = __half22float2(hh[e]);
+          kx[2 * e] = x.x; kx[2 * e + 1] = x.y;
+        }
+      } else {
+        quant = 1;
+        float s_, z_;
+        decode_meta(load_meta(k_meta, (size_t)iq * Ks.n_groups + (piece * 8) / L.G, Ks.meta_bytes), Ks.bits, s_, z_);
+        const uint32_t* row = k_codes + (size_t)iq * (row_bytes(Ks.bits) / 4);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) kx[e] = fmaf(s_, (float)row_code(row, piece * 8 + e, Ks.bits), z_);
+      }
+    }
+    *reinterpret_cast<uint4*>(&S.v[tt][piece * 8]) = vraw;
+    *reinterpret_cast<float4*>(&S.k[tt][piece * 8]) = make_float4(kx[0], kx[1], kx[2], kx[3]);
+    *reinterpret_cast<float4*>(&S.k[tt][piece * 8 + 4]) = make_float4(kx[4], kx[5], kx[6], kx[7]);
+    if (piece == 0) S.quant[tt] = quant;
+  }
+  __syncthreads();
+  // ---- scores: warp w takes rows w, w + 8, w + 16, w + 24; lane takes channels 4*lane .. +3
+#pragma unroll
+  for (int rr = 0; rr < 4; ++rr) {
+    const int tt = warp + rr * kWarps;
+    const float4 kx = *reinterpret_cast<const float4*>(&S.k[tt][4 * lane]);
+    const bool quant = S.quant[tt] != 0;
+#pragma unroll
+    for (int h = 0; h < kHeads; ++h) {
+      const float4 qv = *reinterpret_cast<const float4*>(quant ? &S.q_nrm[h][4 * lane] : &S.q_raw[h][4 * lane]);
+      float v = fmaf(kx.x, qv.x, fmaf(kx.y, qv.y, fmaf(kx.z, qv.z, kx.w * qv.w)));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) S.sc[tt][h] = (i0 + tt) < n_tail ? v : -INFINITY;
+    }
+  }
+  __syncthreads();
+  if (warp < kHeads) {
+    const int h = warp;
+    const float sv = S.sc[lane][h];
+    float mt = sv;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, o));
+    const float p = exp2f(sv - mt);
+    float ps = p;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    S.sc[lane][h] = p;
+    if (lane == 0) { S.m[h] = mt; S.l[h] = ps; }
+  }
+  __syncthreads();
+  // ---- values: thread owns channel c_own and every second row
+  const int c_own = tid & (kD - 1), half_id = tid >> 7;
+#pragma unroll
+  for (int h = 0; h < kHeads; ++h) acc[h] = 0.f;
+#pragma unroll
+  for (int r2 = 0; r2 < 16; ++r2) {
+    const int tt = 2 * r2 + half_id;
+    const float vx = __half2float(S.v[tt][c_own]);
+    const float4 p4 = *reinterpret_cast<const float4*>(&S.sc[tt][0]);
+    acc[0] = fmaf(p4.x, vx, acc[0]); acc[1] = fmaf(p4.y, vx, acc[1]);
+    acc[2] = fmaf(p4.z, vx, acc[2]); acc[3] = fmaf(p4.w, vx, acc[3]);
+  }
+  if (half_id == 1) {
+#pragma unroll
+    for (int h = 0; h < kHeads; ++h) S.acc2[h][c_own] = acc[h];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int h = 0; h < kHeads; ++h) {
+    if (half_id == 0) acc[h] += S.acc2[h][c_own];
+    m_out[h] = S.m[h];
+    l_out[h] = S.l[h];
+  }
+  (void)nh;
+}
+
+// ---- the kernel -------------------------------------------------------------------------------------
+template <int BITS, int G>
+__global__ void __launch_bounds__(kThreads, BITS == 2 ? 2 : 2)
+decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
+  using F = Fmt<BITS>;
+  using SL = StageLayout<BITS, G>;
+  constexpr int NG = SL::kNG;                   // key groups per token
+  constexpr int KS_PER_G = G / 16;              // key k-steps per group
+  constexpr int CH_PER_G = G / kChunk;          // chunks per value group
+  constexpr int NST = SL::kStages;
+  constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
+  constexpr int RWL = F::kRowWordsPerLane;
+  constexpr int KPW = F::kKstepsPerWindow;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, j = lane & 3;
+  const int u = blockIdx.x, split = blockIdx.y;
+  const int b = u / L.Hkv, hkv = u % L.Hkv;
+  const int nh = min(kHeads, L.r - a.head0);
+  const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
+  const int n_parts = a.n_splits + a.n_tail_tiles;
+
+  // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
+  // Tables are staged in the ring memory of warp 0..: they are consumed into registers and the CTA
+  // synchronises before the first bulk copy is issued.
+  float* q_nrm_s = reinterpret_cast<float*>(smem);                 // [4][128]
+  float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
+  float* qg_s = q_raw_s + kHeads * kD;                             // [4][NG]
+  int* qe_s = reinterpret_cast<int*>(qg_s + kHeads * 4);           // [4] exponent of max|q''|
+  const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
+  for (int i = tid; i < kHeads * kD; i += kThreads) {
+    const int h = i >> 7, c = i & (kD - 1);
+    float v = 0.f;
+    if (h < nh) v = __half2float(a.q[(size_t)(head_base + h) * kD + c]) * (L.sm_scale * kLog2e);
+    q_raw_s[i] = v;
+    q_nrm_s[i] = L.k_normalize ? v * norm[c] : v;
+  }
+  __syncthreads();
+  if (tid < kHeads * NG) {
+    const int h = tid / NG, g = tid % NG;
+    float sum = 0.f;
+    for (int c = 0; c < G; ++c) sum += q_nrm_s[h * kD + g * G + c];
+    qg_s[h * 4 + g] = sum;
+  }
+  if (tid < kHeads) {
+    float am = 0.f;
+    for (int c = 0; c < kD; ++c) am = fmaxf(am, fabsf(q_nrm_s[tid * kD + c]));
+    int e = 0;
+    if (am > 0.f && am < INFINITY) frexpf(am, &e);
+    qe_s[tid] = e;     // am < 2^e
+  }
+  __syncthreads();
+
+  if (split >= a.n_splits) {
+    // ======================= tail CTA ==============================================================
+    TailSmem& TS = *reinterpret_cast<TailSmem*>(smem + 8192);
+    for (int i = tid; i < kHeads * kD; i += kThreads) {
+      TS.q_raw[i >> 7][i & (kD - 1)] = q_raw_s[i];
+      TS.q_nrm[i >> 7][i & (kD - 1)] = q_nrm_s[i];
+    }
+    __syncthreads();
+    float acc[kHeads], m_t[kHeads], l_t[kHeads];
+    tail_cta(L, cn, a, u, nh, split - a.n_splits, TS, acc, m_t, l_t);
+    float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
+    if (tid < kD) {
+      for (int h = 0; h < nh; ++h) {
+        float* P = partials + ((size_t)(head_base + h) * L.max_splits + split) * kPartialStride;
+        P[tid] = acc[h];
+        if (tid == 0) { P[kD] = m_t[h]; P[kD + 1] = l_t[h]; }
+      }
+    }
+  } else {
+    // ======================= fast path: packed keys and values ===================================
+    // this warp's range of value groups -> chunks
+    const int n_groups_total = cn.n_qv / G;
+    const int g_lo = min(n_groups_total, split * a.groups_per_split);
+    const int g_hi = min(n_groups_total, g_lo + a.groups_per_split);
+    const int n_g = g_hi - g_lo;
+    const int wg_lo = g_lo + (int)(((long long)n_g * warp) / kWarps);
+    const int wg_hi = g_lo + (int)(((long long)n_g * (warp + 1)) / kWarps);
+    const int c_lo = wg_lo * CH_PER_G, n_chunks = (wg_hi - wg_lo) * CH_PER_G;
+
+    // per-thread constants: B fragments of q'' (hi/lo split, pre-scaled), group sums, exponents
+    const int my_head = gid >> 1, my_part = gid & 1;   // as a B-fragment owner: column gid = (head, hi|lo)
+    const int e_b = qe_s[my_head];
+    const float bscale = pow2i(14 - e_b);              // |q''| * bscale < 2^14
+    uint32_t Bq[8][2];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int kk = (s % (2 * KPW)) % KPW;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const int pos = 2 * kk + rr;
+        const float sc = bscale * pow2i(-BITS * pos);
+        const int c0 = 16 * s + 2 * j + 8 * rr;
+        const uint32_t v0 = split_hi_lo(q_nrm_s[my_head * kD + c0] * sc);
+        const uint32_t v1 = split_hi_lo(q_nrm_s[my_head * kD + c0 + 1] * sc);
+        Bq[s][rr] = my_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
+      }
+    }
+    // as a C-fragment owner: columns 2j, 2j+1 = head j (hi, lo)
+    const float kfac = pow2i(24 - (14 - qe_s[j]));     // undoes the 2^-24 of the subnormal codes and bscale
+    const float inv_kfac = pow2i(-(24 - (14 - qe_s[j])));
+    float Qg[NG];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
+    __syncthreads();   // tables consumed: ring memory may now be overwritten by bulk copies
+
+    unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kWarpBytes * kWarps) + warp * NST;
+    const unsigned char* gk_codes = a.cache + L.k.code_off + (size_t)u * L.k.code_stride;
+    const unsigned char* gk_meta = a.cache + L.k.meta_off + (size_t)u * L.k.meta_stride;
+    const unsigned char* gv_codes = a.cache + L.v.code_off + (size_t)u * L.v.code_stride;
+    const unsigned char* gv_meta = a.cache + L.v.meta_off + (size_t)u * L.v.meta_stride;
+
+    auto issue = [&](int st, int ci) {   // one lane: arm the barrier, start the copies of chunk ci into stage st
+      const uint32_t bar = smem_u32(&bars[st]);
+      const uint32_t dst = smem_u32(ring + (size_t)st * SL::kBytes);
+      const bool with_vmeta = (ci % CH_PER_G) == CH_PER_G - 1;
+      mbar_expect_tx(bar, SL::kKCodes + SL::kKMeta + SL::kVCodes + (with_vmeta ? SL::kVMeta : 0));
+      bulk_g2s(dst, gk_codes + (size_t)ci * SL::kKCodes, SL::kKCodes, bar);
+      bulk_g2s(dst + SL::kOffKMeta, gk_meta + (size_t)ci * SL::kKMeta, SL::kKMeta, bar);
+      bulk_g2s(dst + SL::kOffVCodes, gv_codes + (size_t)ci * SL::kVCodes, SL::kVCodes, bar);
+      if (with_vmeta) bulk_g2s(dst + SL::kOffVMeta, gv_meta + (size_t)(ci / CH_PER_G) * SL::kVMeta, SL::kVMeta, bar);
+    };
+    if (lane == 0) {
+#pragma unroll
+      for (int s = 0; s < NST; ++s) mbar_init(smem_u32(&bars[s]), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+#pragma unroll
+      for (int s = 0; s < NST; ++s)
+        if (s < n_chunks) issue(s, c_lo + s);
+    }
+    __syncwarp();
+
+    float m_run = -INFINITY, l_part = 0.f, psum = 0.f;
+    float out_acc[8][2];
+    float accg[8][4];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      out_acc[m][0] = out_acc[m][1] = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
+    }
+    bool failed = false;
+
+    for (int it = 0; it < n_chunks; ++it) {
+      const int st = it % NST;
+      const uint32_t parity = (uint32_t)(it / NST) & 1u;
+      if (!mbar_wait(smem_u32(&bars[st]), parity)) { failed = true; break; }
+      const unsigned char* sp = ring + (size_t)st * SL::kBytes;
+      const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp);
+      const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::kOffKMeta);
+      const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::kOffVCodes);
+      const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::kOffVMeta);
+
+      // ---------------- scores of 32 tokens: two m-tiles of 16 -------------------------------------
+      float sc[2][2];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const int rA = 16 * mt + gid, rB = rA + 8;
+        uint32_t wa[RWL], wb[RWL];
+        if constexpr (RWL == 2) {
+          const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
+          const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
+          wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
+        } else {
+          const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
+          const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
+          wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
+          wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
+        }
+        uint32_t ma[NG], mb[NG];
+        if constexpr (NG == 4) {
+          const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
+          const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
+          ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
+          mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
+        } else if constexpr (NG == 2) {
+          const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
+          const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
+          ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
+        } else {
+          ma[0] = km[rA]; mb[0] = km[rB];
+        }
+        float sA = 0.f, sB = 0.f;
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          float c4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int ks = 0; ks < KS_PER_G; ++ks) {
+            const int s = g * KS_PER_G + ks;
+            const int wi = s / (2 * KPW), sw = s % (2 * KPW);
+            const int window = sw / KPW, kk = sw % KPW;
+            const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
+            const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
+            const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
+            mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[s][0], Bq[s][1]);
+          }
+          float s_, z_;
+          decode_meta(ma[g], BITS, s_, z_);
+          sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
+          decode_meta(mb[g], BITS, s_, z_);
+          sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
+        }
+        sc[mt][0] = sA * kfac;
+        sc[mt][1] = sB * kfac;
+      }
+
+      // ---------------- online softmax (head j, log2 domain) ---------------------------------------
+      float cmax = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
+      const float m_new = fmaxf(m_run, cmax);
+      if (__any_sync(0xffffffffu, m_new > m_run)) {
+        const float alpha = exp2f(m_run - m_new);     // 0 on the first chunk (m_run = -inf)
+        l_part *= alpha;
+        psum *= alpha;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
+        }
+      }
+      m_run = m_new;
+      uint32_t Bp[2][2];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float p = exp2f(sc[mt][h] - m_new);
+          l_part += p;
+          psum += p;
+          const int pos = BITS == 2 ? 2 * mt + h : h;
+          Bp[mt][h] = movmatrix_trans(split_hi_lo(p * pow2i(10 - BITS * pos)));
+        }
+      }
+
+      // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
+      if constexpr (BITS == 2) {
+        const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
+        const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
+        const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks) {
+            const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
+            mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
+            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int mm = 0; mm < 4; ++mm) {
+              const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
+              const uint32_t m0 = F::kField, m1 = F::kField << 4;
+              mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+            }
+          }
+        }
+      }
+
+      // ---------------- end of a value group: apply scale / zero-point once per channel -----------
+      if ((it % CH_PER_G) == CH_PER_G - 1) {
+        float pg = psum;
+        pg += __shfl_xor_sync(0xffffffffu, pg, 4);
+        pg += __shfl_xor_sync(0xffffffffu, pg, 8);
+        pg += __shfl_xor_sync(0xffffffffu, pg, 16);
+        pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
+        const uint4* vm4 = reinterpret_cast<const uint4*>(vm + gid * 16);
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const uint4 mw = vm4[q4];
+          const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
+            float s_, z_;
+            decode_meta(mws[e], BITS, s_, z_);
+            out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
+            accg[m][2 * rh] = 0.f;
+            accg[m][2 * rh + 1] = 0.f;
+          }
+        }
+        psum = 0.f;
+      }
+
+      __syncwarp();
+      if (lane == 0 && it + NST < n_chunks) issue(st, c_lo + it + NST);
+    }
+
+    if (failed) {
+      // a copy never arrived: flag it for the host and contribute nothing
+      if (lane == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);
+      m_run = -INFINITY;
+      l_part = 0.f;
+    }
+
+    // ---------------- warp result -> shared memory -> CTA partial ---------------------------------
+    l_part += __shfl_xor_sync(0xffffffffu, l_part, 4);
+    l_part += __shfl_xor_sync(0xffffffffu, l_part, 8);
+    l_part += __shfl_xor_sync(0xffffffffu, l_part, 16);
+    __syncthreads();                                   // every warp is done with its ring
+    float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
+    {
+      float* mine = wres + ((size_t)warp * kHeads + j) * (kD + 2);
+#pragma unroll
+      for (int m = 0; m < 8; ++m) {
+        mine[16 * m + gid] = n_chunks > 0 ? out_acc[m][0] * 0x1p14f : 0.f;
+        mine[16 * m + 8 + gid] = n_chunks > 0 ? out_acc[m][1] * 0x1p14f : 0.f;
+      }
+      if (gid == 0) {
+        mine[kD] = n_chunks > 0 ? m_run : -INFINITY;
+        mine[kD + 1] = n_chunks > 0 ? l_part : 0.f;
+      }
+    }
+    __syncthreads();
+    float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
+    for (int i = tid; i < nh * kD; i += kThreads) {
+      const int h = i >> 7, c = i & (kD - 1);
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wres[((size_t)w * kHeads + h) * (kD + 2) + kD]);
+      float num = 0.f, den = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const float* r_ = wres + ((size_t)w * kHeads + h) * (kD + 2);
+        const float wgt = r_[kD] == -INFINITY ? 0.f : exp2f(r_[kD] - M);
+        num = fmaf(r_[c], wgt, num);
+        den = fmaf(r_[kD + 1], wgt, den);
+      }
+      float* P = partials + ((size_t)(head_base + h) * L.max_splits + split) * kPartialStride;
+      P[c] = num;
+      if (c == 0) { P[kD] = M; P[kD + 1] = den; }
+    }
+  }
+
+  // ---------------- cross-CTA merge: the last CTA of the unit to arrive combines all parts -----------
+  __shared__ unsigned int s_ticket;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+  __syncthreads();
+  if (s_ticket != (unsigned int)(n_parts - 1)) return;
+  __threadfence();
+  const float* partials = reinterpret_cast<const float*>(a.ws + L.ws_partial_off);
+  for (int i = tid; i < nh * kD; i += kThreads) {
+    const int h = i >> 7, c = i & (kD - 1);
+    const float* P = partials + (size_t)(head_base + h) * L.max_splits * kPartialStride;
+    float M = -INFINITY;
+    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, __ldcg(P + s * kPartialStride + kD));
+    float num = 0.f, den = 0.f;
+    for (int s = 0; s < n_parts; ++s) {
+      const float ms = __ldcg(P + s * kPartialStride + kD);
+      if (ms == -INFINITY) continue;
+      const float wgt = exp2f(ms - M);
+      num = fmaf(__ldcg(P + s * kPartialStride + c), wgt, num);
+      den = fmaf(__ldcg(P + s * kPartialStride + kD + 1), wgt, den);
+    }
+    a.out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
+  }
+  if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
+}
+
+template <int BITS, int G>
+int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, dim3 grid, cudaStream_t st) {
+  using SL = StageLayout<BITS, G>;
+  constexpr int kSmem = SL::kCtaBytes > 8192 + (int)sizeof(TailSmem) ? SL::kCtaBytes : 8192 + (int)sizeof(TailSmem);
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+      return -1;
+    configured = true;
+  }
+  int launches = 0;
+  for (int h0 = 0; h0 < L.r; h0 += kHeads) {
+    a.head0 = h0;
+    decode_mma_kernel<BITS, G><<<grid, kThreads, kSmem, st>>>(L, cn, a);
+    ++launches;
+  }
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+}  // namespace
+
+bool decode_mma_supported(const Layout& L) {
+  return L.grouping == 0 && L.k.kind == kRow && L.v.kind == kBlock && L.k.bits == L.v.bits &&
+         (L.k.bits == 2 || L.k.bits == 4) && L.k.meta_bytes == 4 && L.v.meta_bytes == 4;
+}
+
+int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
+                      __half* out, int n_splits, cudaStream_t st) {
+  if (!decode_mma_supported(L)) return -2;
+  const Counts cn = counts_for(L, N);
+  const int n_groups = cn.n_qv / L.G;
+  if (n_splits <= 0) {
+    n_splits = (2 * 148 + L.U - 1) / L.U - 1;   // about two resident CTAs per SM; the (short) tail CTAs launch last
+    if (n_splits < 1) n_splits = 1;
+  }
+  const int by_work = (n_groups + kWarps - 1) / kWarps;      // at least one group per warp
+  if (n_splits > by_work) n_splits = by_work;
+  { const int room = L.max_splits - (cn.N - cn.n_qv + 31) / 32; if (n_splits > room) n_splits = room; }
+  if (n_groups == 0) n_splits = 0;
+  DecodeArgs a;
+  a.cache = cache; a.ws = ws; a.q = q; a.out = out;
+  a.n_splits = n_splits;
+  a.groups_per_split = n_splits ? (n_groups + n_splits - 1) / n_splits : 0;
+  a.head0 = 0;
+  a.n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
+  if (n_splits + a.n_tail_tiles > L.max_splits) return -2;
+  dim3 grid(L.U, n_splits + a.n_tail_tiles);
+  const int bits = L.k.bits;
+  if (bits == 2 && L.G == 32) return launch_one<2, 32>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 64) return launch_one<2, 64>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 128) return launch_one<2, 128>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 32) return launch_one<4, 32>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 64) return launch_one<4, 64>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 128) return launch_one<4, 128>(L, cn, a, grid, st);
   return -2;
 }
+
 }  // namespace iq

@@ -46,7 +46,7 @@ __device__ __forceinline__ float element(const TensorView& v, int G, int t, int 
     decode_meta(load_meta(v.meta, (size_t)i * v.n_groups + c / G, v.meta_bytes), v.bits, s, z);
     code = row_code(v.codes + (size_t)i * (row_bytes(v.bits) / 4), c, v.bits);
   } else {
-    decode_meta(load_meta(v.meta, (size_t)(i / G) * kD + c, v.meta_bytes), v.bits, s, z);
+    decode_meta(load_meta(v.meta, (size_t)(i / G) * kD + block_meta_index(c), v.meta_bytes), v.bits, s, z);
     code = chunk_code(v.codes + (size_t)(i / kChunk) * (chunk_bytes(v.bits) / 4), i % kChunk, c, v.bits);
   }
   return fmaf(s, (float)code, z);

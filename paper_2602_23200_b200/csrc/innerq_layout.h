@@ -132,6 +132,11 @@ IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
   return p;
 }
 
+// BLOCK store metadata: the 128 per-channel entries of a group are ordered so that the 16 channels a
+// lane owns in the PV fragments (channel = 16*m + 8*rh + gid) are contiguous: 4 x 128-bit loads.
+IQ_HD int block_meta_index(int c) { return (c & 7) * 16 + (c >> 3); }
+IQ_HD int block_meta_channel(int pos) { return (pos & 15) * 8 + (pos >> 4); }
+
 IQ_HD int row_bytes(int bits) { return 16 * bits; }
 IQ_HD int chunk_bytes(int bits) { return 512 * bits; }
 // word offset of the 1-bit plane of a 3-bit row / chunk

@@ -163,7 +163,7 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
     chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
   }
-  store_meta(dst_meta, meta_idx + c, S.meta_bytes, group_meta(p, asym));
+  store_meta(dst_meta, meta_idx + block_meta_index(c), S.meta_bytes, group_meta(p, asym));
   __syncthreads();
   for (int i = threadIdx.x; i < n_words; i += 128) dst_chunks[i] = words[i];
   __syncthreads();
@@ -275,7 +275,8 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
     const int rows_cap = S.kind == kRow ? cap : cap / L.G + 1;
     for (int i = tid0; i < n_meta_rows * S.n_groups; i += stride) {
       uint32_t m = load_meta(meta, i, S.meta_bytes);
-      size_t o = (size_t)u * rows_cap * S.n_groups + i;
+      const int ic = S.kind == kRow ? i : (i / kD) * kD + block_meta_channel(i % kD);   // canonical position
+      size_t o = (size_t)u * rows_cap * S.n_groups + ic;
       if (scale) scale[o] = (uint16_t)(m & 0xFFFFu);
       if (zero) zero[o] = (uint16_t)(m >> 16);
     }

@@ -44,6 +44,7 @@ def check_decode(w, oc, gc, step=0, variants=(0,), splits=(0,)):
             out = gc.innerq_decode_attention(dev(q)).cpu().numpy()
             worst = max(worst, P.assert_outputs_close(out, ref, f"{w.name} variant={variant} splits={s}"))
     gc.innerq_set_decode_options(0, 0)
+    assert gc.innerq_read_device_error() == 0      # no bounded wait inside a kernel ever ran out
     return worst
 
 
