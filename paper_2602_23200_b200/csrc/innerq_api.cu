@@ -62,17 +62,33 @@ void place_store(Store& S, int kind, int bits, int mode, const innerq_config_t& 
   S.meta_bytes = mode == INNERQ_MODE_SYM ? 2 : 4;
   S.sink_stride = (size_t)c.w_sink * kD * 2;
   S.ring_stride = (size_t)S.ring_cap * kD * 2;
-  if (kind == kRow) {
-    S.code_stride = (size_t)S.cap_q * row_bytes(bits);
-    S.meta_stride = (size_t)S.cap_q * S.n_groups * S.meta_bytes;
-  } else {
-    S.code_stride = (size_t)(S.cap_q / kChunk) * chunk_bytes(bits);
-    S.meta_stride = (size_t)(S.cap_q / G) * kD * S.meta_bytes;
-  }
   S.sink_off = off; off = align_up(off + S.sink_stride * U, 256);
   S.ring_off = off; off = align_up(off + S.ring_stride * U, 256);
-  S.code_off = off; off = align_up(off + S.code_stride * U, 256);
-  S.meta_off = off; off = align_up(off + S.meta_stride * U, 256);
+}
+
+// Geometry of the shared record area of a ROW store and a BLOCK store (see struct Store).
+void place_records(Store& row, Store& blk, int G, int U, size_t& off) {
+  const int row_codes = kChunk * row_bytes(row.bits);
+  const int row_meta = kChunk * row.n_groups * row.meta_bytes;
+  const int blk_codes = chunk_bytes(blk.bits);
+  const int blk_meta = kD * blk.meta_bytes;
+  const int chunk_stride = row_codes + row_meta + blk_codes;
+  const int cpg = G / kChunk;
+  const int group_stride = cpg * chunk_stride + blk_meta;
+  const size_t unit = align_up((size_t)(row.cap_q / G) * group_stride, 256);
+  Store* both[2] = {&row, &blk};
+  for (Store* S : both) {
+    S->rec_off = off;
+    S->rec_unit_stride = unit;
+    S->group_stride = group_stride;
+    S->chunk_stride = chunk_stride;
+    S->chunks_per_group = cpg;
+  }
+  row.code_in_rec = 0;
+  row.meta_in_rec = row_codes;
+  blk.code_in_rec = row_codes + row_meta;
+  blk.meta_in_rec = cpg * chunk_stride;
+  off = align_up(off + unit * U, 256);
 }
 
 void make_layout(const innerq_config_t& c, Layout& L) {
@@ -98,9 +114,11 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   } else if (c.grouping == INNERQ_GROUPING_INNER) {
     place_store(L.k, kRow, c.k_bits, c.k_mode, c, L.U, off);
     place_store(L.v, kBlock, c.v_bits, c.v_mode, c, L.U, off);
+    place_records(L.k, L.v, L.G, L.U, off);
   } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
     place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);
     place_store(L.v, kRow, c.v_bits, INNERQ_MODE_ASYM, c, L.U, off);
+    place_records(L.v, L.k, L.G, L.U, off);
   }
   L.cache_bytes = off;
   size_t w = 0;

@@ -148,8 +148,7 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a,
   const __half* k_ring = reinterpret_cast<const __half*>(a.cache + Ks.ring_off + (size_t)u * Ks.ring_stride);
   const __half* v_sink = reinterpret_cast<const __half*>(a.cache + Vs.sink_off + (size_t)u * Vs.sink_stride);
   const __half* v_ring = reinterpret_cast<const __half*>(a.cache + Vs.ring_off + (size_t)u * Vs.ring_stride);
-  const uint32_t* k_codes = reinterpret_cast<const uint32_t*>(a.cache + Ks.code_off + (size_t)u * Ks.code_stride);
-  const void* k_meta = a.cache + Ks.meta_off + (size_t)u * Ks.meta_stride;
+  const unsigned char* k_rec = a.cache + Ks.rec_off + (size_t)u * Ks.rec_unit_stride;
   const int n_tail = cn.n_sink + (cn.N - cn.n_sink - cn.n_qv);
   const int i0 = tile * 32;
   // ---- stage the tile: 32 rows x 16 pieces of 8 channels
@@ -178,8 +177,8 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a,
       } else {
         quant = 1;
         float s_, z_;
-        decode_meta(load_meta(k_meta, (size_t)iq * Ks.n_groups + (piece * 8) / L.G, Ks.meta_bytes), Ks.bits, s_, z_);
-        const uint32_t* row = k_codes + (size_t)iq * (row_bytes(Ks.bits) / 4);
+        decode_meta(load_meta(k_rec + row_meta_off(Ks, iq), (piece * 8) / L.G, Ks.meta_bytes), Ks.bits, s_, z_);
+        const uint32_t* row = reinterpret_cast<const uint32_t*>(k_rec + row_code_off(Ks, iq));
 #pragma unroll
         for (int e = 0; e < 8; ++e) kx[e] = fmaf(s_, (float)row_code(row, piece * 8 + e, Ks.bits), z_);
       }
@@ -357,20 +356,18 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 
     unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kWarpBytes * kWarps) + warp * NST;
-    const unsigned char* gk_codes = a.cache + L.k.code_off + (size_t)u * L.k.code_stride;
-    const unsigned char* gk_meta = a.cache + L.k.meta_off + (size_t)u * L.k.meta_stride;
-    const unsigned char* gv_codes = a.cache + L.v.code_off + (size_t)u * L.v.code_stride;
-    const unsigned char* gv_meta = a.cache + L.v.meta_off + (size_t)u * L.v.meta_stride;
+    const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
 
     auto issue = [&](int st, int ci) {   // one lane: arm the barrier, start the copies of chunk ci into stage st
       const uint32_t bar = smem_u32(&bars[st]);
       const uint32_t dst = smem_u32(ring + (size_t)st * SL::kBytes);
+      // a chunk record is contiguous; the value group's scale/zero words sit right behind its last chunk
       const bool with_vmeta = (ci % CH_PER_G) == CH_PER_G - 1;
-      mbar_expect_tx(bar, SL::kKCodes + SL::kKMeta + SL::kVCodes + (with_vmeta ? SL::kVMeta : 0));
-      bulk_g2s(dst, gk_codes + (size_t)ci * SL::kKCodes, SL::kKCodes, bar);
-      bulk_g2s(dst + SL::kOffKMeta, gk_meta + (size_t)ci * SL::kKMeta, SL::kKMeta, bar);
-      bulk_g2s(dst + SL::kOffVCodes, gv_codes + (size_t)ci * SL::kVCodes, SL::kVCodes, bar);
-      if (with_vmeta) bulk_g2s(dst + SL::kOffVMeta, gv_meta + (size_t)(ci / CH_PER_G) * SL::kVMeta, SL::kVMeta, bar);
+      const uint32_t bytes = SL::kOffVMeta + (with_vmeta ? SL::kVMeta : 0);
+      const unsigned char* src = g_rec + (size_t)(ci / CH_PER_G) * (CH_PER_G * SL::kOffVMeta + SL::kVMeta) +
+                                 (size_t)(ci % CH_PER_G) * SL::kOffVMeta;
+      mbar_expect_tx(bar, bytes);
+      bulk_g2s(dst, src, bytes, bar);
     };
     if (lane == 0) {
 #pragma unroll

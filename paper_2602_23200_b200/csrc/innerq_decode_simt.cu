@@ -13,8 +13,8 @@ constexpr int kSimtTile = 32;
 struct TensorView {              // one unit's view of a store
   const __half* sink;
   const __half* ring;
-  const uint32_t* codes;
-  const void* meta;
+  const unsigned char* rec;
+  Store S;
   int kind, bits, ring_cap, n_groups, meta_bytes;
   int n_sink, n_q, w_sink;
 };
@@ -24,8 +24,8 @@ __device__ __forceinline__ TensorView make_view(const Layout& L, const Store& S,
   TensorView v;
   v.sink = reinterpret_cast<const __half*>(cache + S.sink_off + (size_t)u * S.sink_stride);
   v.ring = reinterpret_cast<const __half*>(cache + S.ring_off + (size_t)u * S.ring_stride);
-  v.codes = reinterpret_cast<const uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
-  v.meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  v.rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  v.S = S;
   v.meta_bytes = S.meta_bytes;
   v.kind = S.kind; v.bits = S.bits; v.ring_cap = S.ring_cap; v.n_groups = S.n_groups;
   v.n_sink = n_sink; v.n_q = n_q; v.w_sink = L.w_sink;
@@ -43,11 +43,11 @@ __device__ __forceinline__ float element(const TensorView& v, int G, int t, int 
   float s, z;
   uint32_t code;
   if (v.kind == kRow) {
-    decode_meta(load_meta(v.meta, (size_t)i * v.n_groups + c / G, v.meta_bytes), v.bits, s, z);
-    code = row_code(v.codes + (size_t)i * (row_bytes(v.bits) / 4), c, v.bits);
+    decode_meta(load_meta(v.rec + row_meta_off(v.S, i), c / G, v.meta_bytes), v.bits, s, z);
+    code = row_code(reinterpret_cast<const uint32_t*>(v.rec + row_code_off(v.S, i)), c, v.bits);
   } else {
-    decode_meta(load_meta(v.meta, (size_t)(i / G) * kD + block_meta_index(c), v.meta_bytes), v.bits, s, z);
-    code = chunk_code(v.codes + (size_t)(i / kChunk) * (chunk_bytes(v.bits) / 4), i % kChunk, c, v.bits);
+    decode_meta(load_meta(v.rec + block_meta_off(v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
+    code = chunk_code(reinterpret_cast<const uint32_t*>(v.rec + block_code_off(v.S, i / kChunk)), i % kChunk, c, v.bits);
   }
   return fmaf(s, (float)code, z);
 }

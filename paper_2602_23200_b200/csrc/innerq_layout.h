@@ -4,13 +4,15 @@
 // A quantised tensor lives in one of two stores:
 //
 //   ROW store   (per-token groups along channels; InnerQ keys).  One row of 16*b bytes per
-//               token, rows contiguous, so one evicted token is one contiguous write and a
-//               tile of tokens is one contiguous range.  Metadata: one 32-bit word per
-//               (token, group) = fp16 scale (mask M in the sign bit) | fp16 zero-point << 16;
-//               in symmetric mode only the 16-bit scale is stored.
+//               token, so one evicted token is one contiguous write.  Metadata: one 32-bit
+//               word per (token, group) = fp16 scale (mask M in the sign bit) | fp16
+//               zero-point << 16; in symmetric mode only the 16-bit scale is stored.
 //   BLOCK store (per-channel groups along tokens; InnerQ values).  Chunks of 32 tokens x 128
-//               channels, 512*b bytes each, chunks contiguous.  Metadata: one word per
-//               (group of G tokens, channel), reused by the G tokens of the group.
+//               channels, 512*b bytes each.  Metadata: one word per (group of G tokens,
+//               channel), reused by the G tokens of the group.
+//
+// Both stores of a cache are interleaved in "chunk records" of 32 tokens (see struct Store), so
+// that everything a decode step needs for 32 tokens is one contiguous, 16-byte aligned range.
 //
 // Inside a row / chunk the codes are permuted so that a 32-lane warp reads its tensor-core
 // operand fragments with 64/128-bit loads and extracts them with one LOP3 per pair:
@@ -44,9 +46,35 @@ struct Store {
   int cap_q;           // capacity in quantised tokens (multiple of kTile)
   int n_groups;        // metadata entries per row (ROW: D/G) or per group (BLOCK: D)
   int meta_bytes;      // 4: fp16 scale | fp16 zero << 16;  2: fp16 scale only (symmetric mode stores no zero-points)
-  size_t sink_off, ring_off, code_off, meta_off;              // byte offsets of unit 0
-  size_t sink_stride, ring_stride, code_stride, meta_stride;  // bytes per unit
+  size_t sink_off, ring_off;          // byte offsets of unit 0's fp16 windows
+  size_t sink_stride, ring_stride;    // bytes per unit
+  // Packed records.  The ROW store and the BLOCK store of a cache share one record area per unit:
+  // for every group of G tokens, G/32 chunk records followed by the BLOCK store's metadata of the group;
+  // a chunk record holds, for 32 consecutive tokens, the ROW store's packed rows, the ROW store's
+  // metadata rows and the BLOCK store's packed chunk.  A decoding warp fetches a chunk record (plus the
+  // group metadata behind the last chunk of a group) with ONE contiguous bulk copy.
+  size_t rec_off, rec_unit_stride;    // byte offset of unit 0's record area, bytes per unit
+  int group_stride, chunk_stride;     // bytes per group record / per chunk record
+  int chunks_per_group;               // G / 32
+  int code_in_rec;                    // offset of this store's codes inside a chunk record
+  int meta_in_rec;                    // ROW: offset of its metadata rows inside a chunk record;
+                                      // BLOCK: offset of the group's metadata inside a group record
 };
+
+// Byte offset (from the unit's record area) of chunk record ci.
+IQ_HD size_t chunk_rec_off(const Store& S, int ci) {
+  return (size_t)(ci / S.chunks_per_group) * S.group_stride + (size_t)(ci % S.chunks_per_group) * S.chunk_stride;
+}
+// ROW store: packed row of quantised token i, and index base of its metadata entries.
+IQ_HD size_t row_code_off(const Store& S, int i) {
+  return chunk_rec_off(S, i / kChunk) + S.code_in_rec + (size_t)(i % kChunk) * (16 * S.bits);
+}
+IQ_HD size_t row_meta_off(const Store& S, int i) {
+  return chunk_rec_off(S, i / kChunk) + S.meta_in_rec + (size_t)(i % kChunk) * S.n_groups * S.meta_bytes;
+}
+// BLOCK store: packed chunk ci, metadata of group j.
+IQ_HD size_t block_code_off(const Store& S, int ci) { return chunk_rec_off(S, ci) + S.code_in_rec; }
+IQ_HD size_t block_meta_off(const Store& S, int j) { return (size_t)j * S.group_stride + S.meta_in_rec; }
 
 struct Layout {
   int B, Hq, Hkv, U, r;

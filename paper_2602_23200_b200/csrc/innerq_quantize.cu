@@ -115,12 +115,11 @@ __global__ void __launch_bounds__(128) quantize_rows_kernel(Layout L, Store S, c
   __shared__ uint32_t stage[4][16];
   const int u = blockIdx.y, warp = threadIdx.x >> 5;
   const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
-  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
-  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
-  const int rw = row_bytes(S.bits) / 4;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4) {
     const __half* src = X + ((size_t)u * N + L.w_sink + i) * kD;
-    quantize_row_warp(src, norm, L, S, stage[warp], codes + (size_t)i * rw, meta, (size_t)i * S.n_groups);
+    quantize_row_warp(src, norm, L, S, stage[warp], reinterpret_cast<uint32_t*>(rec + row_code_off(S, i)),
+                      rec + row_meta_off(S, i), 0);
   }
 }
 
@@ -128,8 +127,7 @@ __global__ void __launch_bounds__(128) quantize_rows_kernel(Layout L, Store S, c
 // A 128-thread CTA quantises one group of G tokens x 128 channels; thread c owns channel c.
 // tile: fp16 [G][D] staging; words: packed chunks of the group (zeroed here).
 __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* __restrict__ norm, const Layout& L,
-                                   const Store& S, __half* tile, uint32_t* words, uint32_t* __restrict__ dst_chunks,
-                                   void* __restrict__ dst_meta, size_t meta_idx) {
+                                   const Store& S, __half* tile, uint32_t* words, unsigned char* __restrict__ rec, int group_j) {
   const int G = L.G, c = threadIdx.x;
   const int cw = chunk_bytes(S.bits) / 4;
   const int n_words = (G / kChunk) * cw;
@@ -163,9 +161,12 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
     chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
   }
-  store_meta(dst_meta, meta_idx + block_meta_index(c), S.meta_bytes, group_meta(p, asym));
+  store_meta(rec + block_meta_off(S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
   __syncthreads();
-  for (int i = threadIdx.x; i < n_words; i += 128) dst_chunks[i] = words[i];
+  for (int i = threadIdx.x; i < n_words; i += 128) {
+    const int ch = i / cw;
+    reinterpret_cast<uint32_t*>(rec + block_code_off(S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
+  }
   __syncthreads();
 }
 
@@ -177,13 +178,10 @@ __global__ void __launch_bounds__(128) quantize_blocks_kernel(Layout L, Store S,
   __shared__ uint32_t words[4 * 512];
   const int u = blockIdx.y;
   const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
-  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
-  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
-  const int cw = chunk_bytes(S.bits) / 4, cpg = L.G / kChunk;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   TokSrc src{X + (size_t)u * N * kD, 0, 0};
   for (int j = blockIdx.x; j < n_q / L.G; j += gridDim.x)
-    quantize_block_cta(src, L.w_sink + j * L.G, norm, L, S, tile, words, codes + (size_t)j * cpg * cw,
-                       meta, (size_t)j * kD);
+    quantize_block_cta(src, L.w_sink + j * L.G, norm, L, S, tile, words, rec, j);
 }
 
 // ------------------------------------------------------------------ window copies (prefill)
@@ -226,17 +224,14 @@ __device__ void append_store(const Layout& L, const Store& S, const __half* __re
   if (nq_after == nq_before) return;
   __syncthreads();      // the ring row written above may be among the evicted tokens
   const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
-  uint32_t* codes = reinterpret_cast<uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
-  void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   TokSrc src{ring, S.ring_cap, L.w_sink};
   if (S.kind == kRow) {
     if (threadIdx.x < 32)
-      quantize_row_warp(src.row(L.w_sink + nq_before), norm, L, S, words, codes + (size_t)nq_before * (row_bytes(S.bits) / 4),
-                        meta, (size_t)nq_before * S.n_groups);
+      quantize_row_warp(src.row(L.w_sink + nq_before), norm, L, S, words,
+                        reinterpret_cast<uint32_t*>(rec + row_code_off(S, nq_before)), rec + row_meta_off(S, nq_before), 0);
   } else {
-    const int j = nq_before / L.G;
-    quantize_block_cta(src, L.w_sink + nq_before, norm, L, S, tile, words,
-                       codes + (size_t)j * (L.G / kChunk) * (chunk_bytes(S.bits) / 4), meta, (size_t)j * kD);
+    quantize_block_cta(src, L.w_sink + nq_before, norm, L, S, tile, words, rec, nq_before / L.G);
   }
 }
 
@@ -258,15 +253,15 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
                                     uint16_t* __restrict__ recent_out) {
   const int u = blockIdx.y;
   const int cap = L.max_tokens;
-  const uint32_t* codes = reinterpret_cast<const uint32_t*>(cache + S.code_off + (size_t)u * S.code_stride);
-  const void* meta = cache + S.meta_off + (size_t)u * S.meta_stride;
+  const unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   const int stride = gridDim.x * blockDim.x, tid0 = blockIdx.x * blockDim.x + threadIdx.x;
   if (code && S.kind != kNone) {
     for (int i = tid0; i < n_q * kD; i += stride) {
       int t = i / kD, c = i % kD;
       uint32_t v = S.kind == kRow
-                       ? row_code(codes + (size_t)t * (row_bytes(S.bits) / 4), c, S.bits)
-                       : chunk_code(codes + (size_t)(t / kChunk) * (chunk_bytes(S.bits) / 4), t % kChunk, c, S.bits);
+                       ? row_code(reinterpret_cast<const uint32_t*>(rec + row_code_off(S, t)), c, S.bits)
+                       : chunk_code(reinterpret_cast<const uint32_t*>(rec + block_code_off(S, t / kChunk)), t % kChunk, c,
+                                    S.bits);
       code[((size_t)u * cap + t) * kD + c] = (uint8_t)v;
     }
   }
@@ -274,8 +269,10 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
     const int n_meta_rows = S.kind == kRow ? n_q : n_q / L.G;
     const int rows_cap = S.kind == kRow ? cap : cap / L.G + 1;
     for (int i = tid0; i < n_meta_rows * S.n_groups; i += stride) {
-      uint32_t m = load_meta(meta, i, S.meta_bytes);
-      const int ic = S.kind == kRow ? i : (i / kD) * kD + block_meta_channel(i % kD);   // canonical position
+      const int mr = i / S.n_groups, me = i % S.n_groups;
+      uint32_t m = S.kind == kRow ? load_meta(rec + row_meta_off(S, mr), me, S.meta_bytes)
+                                  : load_meta(rec + block_meta_off(S, mr), me, S.meta_bytes);
+      const int ic = S.kind == kRow ? i : mr * kD + block_meta_channel(me);   // canonical position
       size_t o = (size_t)u * rows_cap * S.n_groups + ic;
       if (scale) scale[o] = (uint16_t)(m & 0xFFFFu);
       if (zero) zero[o] = (uint16_t)(m >> 16);
