@@ -70,6 +70,27 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// same with a zero accumulator input (lets the assembler use the zero register instead of clearing four)
+__device__ __forceinline__ void mma16816_z(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                           uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Decoder parameters from a metadata word (fp16 scale with the mask in its sign bit | fp16 zero << 16):
+// s = |scale|, z = Z if the mask is set (scale <= -0), else -s * 2^(b-1) (Z is stored as 0 then).
+__device__ __forceinline__ void decode_fast(uint32_t meta, float neg_half, float& s, float& z) {
+  const __half2 h = *reinterpret_cast<const __half2*>(&meta);
+  const float sg = __low2float(h), Z = __high2float(h);
+  s = fabsf(sg);
+  z = fmaf(neg_half, fmaxf(sg, 0.f), Z);
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -111,7 +132,10 @@ template <int BITS, int G> struct StageLayout {
   static constexpr int kBytes = kOffVMeta + kVMeta;
   static constexpr int kStages = BITS == 2 ? 4 : 2;
   static constexpr int kWarpBytes = kBytes * kStages;
-  static constexpr int kCtaBytes = kWarpBytes * kWarps + 1024;   // + barriers and small tables
+  static constexpr int kSideBytes = 4 * kVMeta;                  // per warp: value metadata of the last 4 groups
+  static constexpr int kOffSide = kWarpBytes * kWarps;
+  static constexpr int kOffBars = kOffSide + kSideBytes * kWarps;
+  static constexpr int kCtaBytes = kOffBars + 256;
 };
 
 struct DecodeArgs {
@@ -246,8 +270,14 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a,
 }
 
 // ---- the kernel -------------------------------------------------------------------------------------
-template <int BITS, int G>
-__global__ void __launch_bounds__(kThreads, BITS == 2 ? 2 : 2)
+// SPLIT (one query head per KV head, G = 32): the 8 mma columns are not 4 heads x {hi, lo} but
+// 4 groups x {hi, lo}: for keys, column pair g holds q'' restricted to channel group g, so one accumulator
+// chain over all 8 k-steps yields the four per-group code sums at once and lane j of each quad applies the
+// scale / zero-point of group j only (then the quad adds up); for values, column pair w holds p
+// restricted to the w-th value group of a window of four, and lane j applies group j's metadata once per
+// window.  This removes the 4x redundancy a quad otherwise has in decoding per-group metadata.
+template <int BITS, int G, bool SPLIT>
+__global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   using F = Fmt<BITS>;
   using SL = StageLayout<BITS, G>;
@@ -258,22 +288,25 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
   constexpr int RWL = F::kRowWordsPerLane;
   constexpr int KPW = F::kKstepsPerWindow;
+  constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
+  static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
+  static_assert((NST & (NST - 1)) == 0, "stage count must be a power of two");
 
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, j = lane & 3;
   const int u = blockIdx.x, split = blockIdx.y;
   const int b = u / L.Hkv, hkv = u % L.Hkv;
-  const int nh = min(kHeads, L.r - a.head0);
+  const int nh = min(SPLIT ? 1 : kHeads, L.r - a.head0);
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
   const int n_parts = a.n_splits + a.n_tail_tiles;
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
-  // Tables are staged in the ring memory of warp 0..: they are consumed into registers and the CTA
+  // Tables are staged in the ring memory of warp 0: they are consumed into registers and the CTA
   // synchronises before the first bulk copy is issued.
   float* q_nrm_s = reinterpret_cast<float*>(smem);                 // [4][128]
   float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
-  float* qg_s = q_raw_s + kHeads * kD;                             // [4][NG]
+  float* qg_s = q_raw_s + kHeads * kD;                             // [4][4]
   int* qe_s = reinterpret_cast<int*>(qg_s + kHeads * 4);           // [4] exponent of max|q''|
   const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
   for (int i = tid; i < kHeads * kD; i += kThreads) {
@@ -328,10 +361,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     const int wg_hi = g_lo + (int)(((long long)n_g * (warp + 1)) / kWarps);
     const int c_lo = wg_lo * CH_PER_G, n_chunks = (wg_hi - wg_lo) * CH_PER_G;
 
-    // per-thread constants: B fragments of q'' (hi/lo split, pre-scaled), group sums, exponents
-    const int my_head = gid >> 1, my_part = gid & 1;   // as a B-fragment owner: column gid = (head, hi|lo)
-    const int e_b = qe_s[my_head];
-    const float bscale = pow2i(14 - e_b);              // |q''| * bscale < 2^14
+    // ---- per-thread constants.  As owner of B-fragment column gid: (head, hi|lo) or, in SPLIT, (group, hi|lo).
+    const int col_head = SPLIT ? 0 : (gid >> 1), col_group = gid >> 1, col_part = gid & 1;
+    const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
     uint32_t Bq[8][2];
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
@@ -339,39 +371,51 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
       for (int rr = 0; rr < 2; ++rr) {
         const int pos = 2 * kk + rr;
-        const float sc = bscale * pow2i(-BITS * pos);
+        const float scl = bscale * pow2i(-BITS * pos);
         const int c0 = 16 * s + 2 * j + 8 * rr;
-        const uint32_t v0 = split_hi_lo(q_nrm_s[my_head * kD + c0] * sc);
-        const uint32_t v1 = split_hi_lo(q_nrm_s[my_head * kD + c0 + 1] * sc);
-        Bq[s][rr] = my_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
+        const uint32_t v0 = split_hi_lo(q_nrm_s[col_head * kD + c0] * scl);
+        const uint32_t v1 = split_hi_lo(q_nrm_s[col_head * kD + c0 + 1] * scl);
+        uint32_t v = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
+        if (SPLIT && (s / KS_PER_G) != col_group) v = 0u;
+        Bq[s][rr] = v;
       }
     }
-    // as a C-fragment owner: columns 2j, 2j+1 = head j (hi, lo)
-    const float kfac = pow2i(24 - (14 - qe_s[j]));     // undoes the 2^-24 of the subnormal codes and bscale
-    const float inv_kfac = pow2i(-(24 - (14 - qe_s[j])));
-    float Qg[NG];
+    // ---- as owner of C-fragment columns 2j, 2j+1: head j, or in SPLIT (head 0, key group j)
+    const int my_head = SPLIT ? 0 : j;
+    const int e_c = qe_s[my_head];
+    const float kfac = pow2i(24 - (14 - e_c));       // undoes the 2^-24 of the subnormal codes and bscale
+    const float inv_kfac = pow2i(-(24 - (14 - e_c)));
+    float Qg[SPLIT ? 1 : NG];
+    if constexpr (SPLIT) {
+      Qg[0] = qg_s[j] * inv_kfac;                     // NG == 4: every lane of the quad owns one group
+    } else {
 #pragma unroll
-    for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
+      for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
+    }
+    const float neg_half = -(float)(1 << (BITS - 1));
     __syncthreads();   // tables consumed: ring memory may now be overwritten by bulk copies
 
     unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kWarpBytes * kWarps) + warp * NST;
+    uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
     const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
+    const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
 
-    auto issue = [&](int st, int ci) {   // one lane: arm the barrier, start the copies of chunk ci into stage st
-      const uint32_t bar = smem_u32(&bars[st]);
-      const uint32_t dst = smem_u32(ring + (size_t)st * SL::kBytes);
+    auto issue = [&](int st, int ci) {   // one lane: arm the barrier, start the copy of chunk ci into stage st
       // a chunk record is contiguous; the value group's scale/zero words sit right behind its last chunk
       const bool with_vmeta = (ci % CH_PER_G) == CH_PER_G - 1;
       const uint32_t bytes = SL::kOffVMeta + (with_vmeta ? SL::kVMeta : 0);
       const unsigned char* src = g_rec + (size_t)(ci / CH_PER_G) * (CH_PER_G * SL::kOffVMeta + SL::kVMeta) +
                                  (size_t)(ci % CH_PER_G) * SL::kOffVMeta;
-      mbar_expect_tx(bar, bytes);
-      bulk_g2s(dst, src, bytes, bar);
+      mbar_expect_tx(bars_u32 + 8 * st, bytes);
+      bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
     };
+    if constexpr (SPLIT) {
+      for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
+    }
     if (lane == 0) {
 #pragma unroll
-      for (int s = 0; s < NST; ++s) mbar_init(smem_u32(&bars[s]), 1);
+      for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 #pragma unroll
@@ -391,158 +435,207 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
     bool failed = false;
 
+    // The loop body is deliberately not unrolled over chunks: it is a few hundred instructions and two
+    // CTAs of eight warps each walk it at different phases, so it has to stay resident in the
+    // instruction cache.
+#pragma unroll 1
     for (int it = 0; it < n_chunks; ++it) {
-      const int st = it % NST;
-      const uint32_t parity = (uint32_t)(it / NST) & 1u;
-      if (!mbar_wait(smem_u32(&bars[st]), parity)) { failed = true; break; }
-      const unsigned char* sp = ring + (size_t)st * SL::kBytes;
-      const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp);
-      const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::kOffKMeta);
-      const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::kOffVCodes);
-      const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::kOffVMeta);
-
-      // ---------------- scores of 32 tokens: two m-tiles of 16 -------------------------------------
-      float sc[2][2];
+      {
+        {
+          const int st = it & (NST - 1);
+          const int s = SPLIT ? (it & (WIN - 1)) : (it % CH_PER_G);      // slot in the window / chunk in the group
+          const uint32_t parity = (uint32_t)(it / NST) & 1u;
+          if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
+          const unsigned char* sp = ring + st * SL::kBytes;
+          const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp);
+          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::kOffKMeta);
+          const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::kOffVCodes);
+          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::kOffVMeta);
+          const bool group_start = s == 0;                  // value accumulators start from zero
+          const bool group_end = SPLIT ? (s == WIN - 1 || it == n_chunks - 1) : (s == CH_PER_G - 1);
+          constexpr bool kFreshEveryChunk = !SPLIT && CH_PER_G == 1;      // then the first value mma takes a zero C
+          if (!kFreshEveryChunk && group_start) {
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const int rA = 16 * mt + gid, rB = rA + 8;
-        uint32_t wa[RWL], wb[RWL];
-        if constexpr (RWL == 2) {
-          const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
-          const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
-          wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
-        } else {
-          const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
-          const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
-          wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
-          wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
-        }
-        uint32_t ma[NG], mb[NG];
-        if constexpr (NG == 4) {
-          const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
-          const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
-          ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
-          mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
-        } else if constexpr (NG == 2) {
-          const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
-          const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
-          ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
-        } else {
-          ma[0] = km[rA]; mb[0] = km[rB];
-        }
-        float sA = 0.f, sB = 0.f;
+            for (int m = 0; m < 8; ++m)
 #pragma unroll
-        for (int g = 0; g < NG; ++g) {
-          float c4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-          for (int ks = 0; ks < KS_PER_G; ++ks) {
-            const int s = g * KS_PER_G + ks;
-            const int wi = s / (2 * KPW), sw = s % (2 * KPW);
-            const int window = sw / KPW, kk = sw % KPW;
-            const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
-            const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
-            const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
-            mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[s][0], Bq[s][1]);
+              for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
           }
-          float s_, z_;
-          decode_meta(ma[g], BITS, s_, z_);
-          sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
-          decode_meta(mb[g], BITS, s_, z_);
-          sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
-        }
-        sc[mt][0] = sA * kfac;
-        sc[mt][1] = sB * kfac;
-      }
 
-      // ---------------- online softmax (head j, log2 domain) ---------------------------------------
-      float cmax = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
-      const float m_new = fmaxf(m_run, cmax);
-      if (__any_sync(0xffffffffu, m_new > m_run)) {
-        const float alpha = exp2f(m_run - m_new);     // 0 on the first chunk (m_run = -inf)
-        l_part *= alpha;
-        psum *= alpha;
+          // ---------------- raw scores of 32 tokens: two m-tiles of 16 ------------------------------
+          float sc[2][2];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
+          for (int mt = 0; mt < 2; ++mt) {
+            const int rA = 16 * mt + gid, rB = rA + 8;
+            uint32_t wa[RWL], wb[RWL];
+            if constexpr (RWL == 2) {
+              const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
+              const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
+              wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
+            } else {
+              const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
+              const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
+              wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
+              wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
+            }
+            auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
+              const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
+              const int window = sw / KPW, kk = sw % KPW;
+              const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
+              const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
+              const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
+              if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+              else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+            };
+            float sA, sB;
+            if constexpr (SPLIT) {
+              float c4[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
-        }
-      }
-      m_run = m_new;
-      uint32_t Bp[2][2];
+              for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
+              float s_, z_;
+              decode_fast(km[rA * NG + j], neg_half, s_, z_);
+              sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
+              decode_fast(km[rB * NG + j], neg_half, s_, z_);
+              sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
+              sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+              sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+              sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+              sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+            } else {
+              uint32_t ma[NG], mb[NG];
+              if constexpr (NG == 4) {
+                const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
+                const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
+                ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
+                mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
+              } else if constexpr (NG == 2) {
+                const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
+                const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
+                ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
+              } else {
+                ma[0] = km[rA]; mb[0] = km[rB];
+              }
+              sA = 0.f; sB = 0.f;
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
+              for (int g = 0; g < NG; ++g) {
+                float c4[4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float p = exp2f(sc[mt][h] - m_new);
-          l_part += p;
-          psum += p;
-          const int pos = BITS == 2 ? 2 * mt + h : h;
-          Bp[mt][h] = movmatrix_trans(split_hi_lo(p * pow2i(10 - BITS * pos)));
-        }
-      }
-
-      // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
-      if constexpr (BITS == 2) {
-        const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
-        const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
-        const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
-#pragma unroll
-          for (int ks = 0; ks < 2; ++ks) {
-            const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
-            mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
+                float s_, z_;
+                decode_fast(ma[g], neg_half, s_, z_);
+                sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
+                decode_fast(mb[g], neg_half, s_, z_);
+                sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
+              }
+            }
+            sc[mt][0] = sA;
+            sc[mt][1] = sB;
           }
-        }
-      } else {
+
+          // ---------------- online softmax (log2 domain; raw scores still carry 1/kfac) -------------
+          float cmax = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
+          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
+          const float m_new = fmaxf(m_run, cmax * kfac);
+          if (__any_sync(0xffffffffu, m_new > m_run)) {
+            const float alpha = ex2_approx(m_run - m_new);     // 0 on the first chunk (m_run = -inf)
+            l_part *= alpha;
+            psum *= alpha;
 #pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
+            for (int m = 0; m < 8; ++m) {
+              out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
+              if (!kFreshEveryChunk) {
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
-            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int mm = 0; mm < 4; ++mm) {
-              const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
-              const uint32_t m0 = F::kField, m1 = F::kField << 4;
-              mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
+              }
             }
           }
-        }
-      }
-
-      // ---------------- end of a value group: apply scale / zero-point once per channel -----------
-      if ((it % CH_PER_G) == CH_PER_G - 1) {
-        float pg = psum;
-        pg += __shfl_xor_sync(0xffffffffu, pg, 4);
-        pg += __shfl_xor_sync(0xffffffffu, pg, 8);
-        pg += __shfl_xor_sync(0xffffffffu, pg, 16);
-        pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
-        const uint4* vm4 = reinterpret_cast<const uint4*>(vm + gid * 16);
+          m_run = m_new;
+          uint32_t Bp[2][2];
+          float psum_c = 0.f;
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const uint4 mw = vm4[q4];
-          const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+          for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
-            float s_, z_;
-            decode_meta(mws[e], BITS, s_, z_);
-            out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
-            accg[m][2 * rh] = 0.f;
-            accg[m][2 * rh + 1] = 0.f;
+            for (int h = 0; h < 2; ++h) {
+              const float p = ex2_approx(fmaf(sc[mt][h], kfac, -m_new));
+              psum_c += p;
+              const int pos = BITS == 2 ? 2 * mt + h : h;
+              uint32_t pk = split_hi_lo(p * pow2i(10 - BITS * pos));
+              if (SPLIT && j != s) pk = 0u;                     // column pair of this chunk's window slot only
+              Bp[mt][h] = movmatrix_trans(pk);
+            }
           }
-        }
-        psum = 0.f;
-      }
+          l_part += psum_c;
+          if constexpr (SPLIT) psum += (j == s) ? psum_c : 0.f;
+          else psum += psum_c;
 
-      __syncwarp();
-      if (lane == 0 && it + NST < n_chunks) issue(st, c_lo + it + NST);
+          // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ----------------
+          if constexpr (BITS == 2) {
+            const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
+            const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
+            const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+              const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
+#pragma unroll
+              for (int ks = 0; ks < 2; ++ks) {
+                const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
+                if (kFreshEveryChunk && ks == 0) mma16816_z(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
+                const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int mm = 0; mm < 4; ++mm) {
+                  const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
+                  const uint32_t m0 = F::kField, m1 = F::kField << 4;
+                  if (kFreshEveryChunk && ks == 0)
+                    mma16816_z(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                  else
+                    mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                }
+              }
+            }
+          }
+
+          // ---------------- end of a value group: apply scale / zero-point once per channel ---------
+          if constexpr (SPLIT) {
+            // keep this group's metadata for the end of the window (the stage will be refilled)
+            *reinterpret_cast<uint4*>(side + s * kD + lane * 4) = *reinterpret_cast<const uint4*>(vm + lane * 4);
+          }
+          if (group_end) {
+            if constexpr (SPLIT) __syncwarp();
+            float pg = psum;
+            pg += __shfl_xor_sync(0xffffffffu, pg, 4);
+            pg += __shfl_xor_sync(0xffffffffu, pg, 8);
+            pg += __shfl_xor_sync(0xffffffffu, pg, 16);
+            pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
+            const uint4* vm4 = reinterpret_cast<const uint4*>((SPLIT ? side + j * kD : vm) + gid * 16);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const uint4 mw = vm4[q4];
+              const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
+                float s_, z_;
+                decode_fast(mws[e], neg_half, s_, z_);
+                out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
+              }
+            }
+            psum = 0.f;
+          }
+
+          __syncwarp();
+          if (lane == 0 && it + NST < n_chunks) issue(st, c_lo + it + NST);
+        }
+      }
     }
 
     if (failed) {
@@ -556,10 +649,23 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     l_part += __shfl_xor_sync(0xffffffffu, l_part, 4);
     l_part += __shfl_xor_sync(0xffffffffu, l_part, 8);
     l_part += __shfl_xor_sync(0xffffffffu, l_part, 16);
+    if constexpr (SPLIT) {
+      // the four lanes of a quad hold the contributions of different window slots: add them up
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+          float v = out_acc[m][rh];
+          v += __shfl_xor_sync(0xffffffffu, v, 1);
+          v += __shfl_xor_sync(0xffffffffu, v, 2);
+          out_acc[m][rh] = v;
+        }
+    }
     __syncthreads();                                   // every warp is done with its ring
     float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
-    {
-      float* mine = wres + ((size_t)warp * kHeads + j) * (kD + 2);
+    const bool writer = SPLIT ? (j == 0) : true;
+    if (writer) {
+      float* mine = wres + ((size_t)warp * kHeads + (SPLIT ? 0 : j)) * (kD + 2);
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
         mine[16 * m + gid] = n_chunks > 0 ? out_acc[m][0] * 0x1p14f : 0.f;
@@ -618,20 +724,22 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
 }
 
-template <int BITS, int G>
+template <int BITS, int G, bool SPLIT>
 int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, dim3 grid, cudaStream_t st) {
   using SL = StageLayout<BITS, G>;
   constexpr int kSmem = SL::kCtaBytes > 8192 + (int)sizeof(TailSmem) ? SL::kCtaBytes : 8192 + (int)sizeof(TailSmem);
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
+        cudaSuccess)
       return -1;
     configured = true;
   }
   int launches = 0;
-  for (int h0 = 0; h0 < L.r; h0 += kHeads) {
+  const int step = SPLIT ? 1 : kHeads;
+  for (int h0 = 0; h0 < L.r; h0 += step) {
     a.head0 = h0;
-    decode_mma_kernel<BITS, G><<<grid, kThreads, kSmem, st>>>(L, cn, a);
+    decode_mma_kernel<BITS, G, SPLIT><<<grid, kThreads, kSmem, st>>>(L, cn, a);
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -649,29 +757,32 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   if (!decode_mma_supported(L)) return -2;
   const Counts cn = counts_for(L, N);
   const int n_groups = cn.n_qv / L.G;
+  const int n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
   if (n_splits <= 0) {
     n_splits = (2 * 148 + L.U - 1) / L.U - 1;   // about two resident CTAs per SM; the (short) tail CTAs launch last
     if (n_splits < 1) n_splits = 1;
   }
   const int by_work = (n_groups + kWarps - 1) / kWarps;      // at least one group per warp
   if (n_splits > by_work) n_splits = by_work;
-  { const int room = L.max_splits - (cn.N - cn.n_qv + 31) / 32; if (n_splits > room) n_splits = room; }
+  if (n_splits > L.max_splits - n_tail_tiles) n_splits = L.max_splits - n_tail_tiles;
   if (n_groups == 0) n_splits = 0;
+  if (n_splits < 0 || n_splits + n_tail_tiles > L.max_splits) return -2;
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
+  a.n_tail_tiles = n_tail_tiles;
   a.groups_per_split = n_splits ? (n_groups + n_splits - 1) / n_splits : 0;
   a.head0 = 0;
-  a.n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
-  if (n_splits + a.n_tail_tiles > L.max_splits) return -2;
-  dim3 grid(L.U, n_splits + a.n_tail_tiles);
+  dim3 grid(L.U, n_splits + n_tail_tiles);
   const int bits = L.k.bits;
-  if (bits == 2 && L.G == 32) return launch_one<2, 32>(L, cn, a, grid, st);
-  if (bits == 2 && L.G == 64) return launch_one<2, 64>(L, cn, a, grid, st);
-  if (bits == 2 && L.G == 128) return launch_one<2, 128>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 32) return launch_one<4, 32>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 64) return launch_one<4, 64>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 128) return launch_one<4, 128>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 32 && L.r == 1) return launch_one<2, 32, true>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 32 && L.r == 1) return launch_one<4, 32, true>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 32) return launch_one<2, 32, false>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 64) return launch_one<2, 64, false>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 128) return launch_one<2, 128, false>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 32) return launch_one<4, 32, false>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 64) return launch_one<4, 64, false>(L, cn, a, grid, st);
+  if (bits == 4 && L.G == 128) return launch_one<4, 128, false>(L, cn, a, grid, st);
   return -2;
 }
 
