@@ -135,6 +135,25 @@ int innerq_append_token(innerq_cache_t* cache, const void* k_new, const void* v_
  * not overlap.  Errors: INVALID_ARG (N == 0 included), CUDA. */
 int innerq_decode_attention(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
 
+/* Same computation and arguments as innerq_decode_attention, for callers that cannot give the decode
+ * step any scratch memory of their own.  (The paper has no counterpart; this is an integration aid.)
+ * Typical cases: the workspace passed to innerq_cache_create was only lent for the prefill and has gone
+ * back to a pool; or the decode runs in a part of a program (a serving loop with a frozen memory plan,
+ * a plug-in without access to the host's allocator) where device memory cannot be allocated, so no
+ * workspace can be produced on demand.  Here the kernel's scratch (per-split partial results, merge
+ * tickets, error word) lives in a 4 MiB array that is part of the library image on every GPU that loads
+ * the library, until the process exits.  The call allocates nothing and frees nothing.
+ *   - Limit: the configuration's workspace size (innerq_cache_bytes) must not exceed 4 MiB; otherwise
+ *     the call returns INNERQ_ERR_BUFFER_TOO_SMALL and launches nothing.
+ *   - The first call on each device looks up the array's device address (one runtime query, made with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All caches and all calls on a device share the one array, which keeps the contents of the previous
+ *     call; the parts that must start at zero are cleared on `cuda_stream` before the launch.  Two such
+ *     calls must not overlap on the GPU (different streams without ordering): they would race on the array.
+ *   - The caller's workspace is not touched, so innerq_read_device_error does not see this call.
+ * Errors: INVALID_ARG (N == 0 included), BUFFER_TOO_SMALL, UNSUPPORTED, CUDA. */
+int innerq_decode_attention_static(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
+
 /* Unpack the cache into canonical arrays (see innerq_export_t).  `ex` is a host struct holding
  * device pointers; counts are written to it before the call returns, array contents when the
  * stream reaches the enqueued kernels.  Errors: INVALID_ARG, CUDA. */

@@ -22,6 +22,7 @@ GROUPING_INNER, GROUPING_OUTER, GROUPING_FP16 = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "innerq_cache_bytes", "innerq_token_payload_bytes", "innerq_cache_create", "innerq_cache_destroy",
     "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
+    "innerq_decode_attention_static",
     "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
@@ -68,6 +69,7 @@ def lib() -> C.CDLL:
     L.innerq_quantize_prefill.argtypes = [vp, vp, vp, i32, vp]
     L.innerq_append_token.argtypes = [vp, vp, vp, vp]
     L.innerq_decode_attention.argtypes = [vp, vp, vp, vp]
+    L.innerq_decode_attention_static.argtypes = [vp, vp, vp, vp]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
@@ -189,6 +191,19 @@ class InnerQCache:
             out = torch.empty(shape, dtype=torch.float16, device=self.device)
         _check(lib().innerq_decode_attention(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
                                              _stream_ptr(stream)), "innerq_decode_attention")
+        return out
+
+    def innerq_decode_attention_static(self, q, out=None, stream=None):
+        """Decode on the library's built-in scratch array: for callers that cannot supply device scratch
+        themselves.  Allocates nothing inside the library (the `out` tensor, if not passed, is still a
+        normal torch allocation made here in the binding)."""
+        import torch
+        c = self.cfg
+        shape = (c.batch, c.n_q_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float16, device=self.device)
+        _check(lib().innerq_decode_attention_static(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
+                                                    _stream_ptr(stream)), "innerq_decode_attention_static")
         return out
 
     def innerq_set_decode_options(self, n_splits: int = 0, variant: int = 0):

@@ -1,6 +1,7 @@
 // C ABI of libinnerq (see include/innerq.h): argument validation, layout computation, host-side
 // token bookkeeping, kernel dispatch.  No device allocation, no synchronisation.
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/innerq.h"
@@ -233,6 +234,57 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   if (n == -2) {
     if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
     n = launch_decode_simt(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                           c->opt_splits, s);
+  }
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->launches[2] = n;
+  return INNERQ_OK;
+}
+
+// ---- decode on library-owned scratch ---------------------------------------------------------------
+// The split partials, merge tickets and error word of the decode kernel normally live in the workspace
+// the caller handed to innerq_cache_create.  This variant keeps them in a fixed array inside the library
+// image instead, so it needs no device memory from the caller beyond inputs and outputs.
+constexpr size_t kStaticScratchBytes = 4u << 20;     // 4 MiB per GPU that loads the library, held until exit
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can use:
+// the device address has to be looked up, once per device, while that device is current.
+int static_scratch_for_current_device(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INNERQ_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return INNERQ_ERR_CUDA;
+    g_scratch_ptr[dev] = p;
+  }
+  *out = static_cast<unsigned char*>(g_scratch_ptr[dev]);
+  return INNERQ_OK;
+}
+}  // namespace
+
+int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, void* cuda_stream) {
+  if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
+  if (c->L.workspace_bytes > kStaticScratchBytes) return INNERQ_ERR_BUFFER_TOO_SMALL;
+  unsigned char* scratch = nullptr;
+  int st = static_scratch_for_current_device(&scratch);
+  if (st != INNERQ_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps whatever the previous call (of any cache) left: tickets and the error word must start at zero
+  if (cudaMemsetAsync(scratch + c->L.ws_ticket_off, 0, (size_t)(c->L.U + 8) * 4, s) != cudaSuccess) return INNERQ_ERR_CUDA;
+  int n = -2;
+  if (c->opt_variant != 1 && decode_mma_supported(c->L))
+    n = launch_decode_mma(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                          c->opt_splits, s);
+  if (n == -2) {
+    if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
+    n = launch_decode_simt(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
   }
   if (n < 0) return INNERQ_ERR_CUDA;
