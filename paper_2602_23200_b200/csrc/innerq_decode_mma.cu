@@ -120,21 +120,30 @@ template <> struct Fmt<4> {
   static constexpr int kChunkWordsPerLane = 16;
 };
 
-template <int BITS, int G> struct StageLayout {
+// Shared-memory stage = the byte range of CPI consecutive chunk records as it lies in HBM (value metadata
+// follows the last chunk of each value group), fetched with one bulk copy.
+template <int BITS, int G, int CPI> struct StageLayout {
   static constexpr int kNG = kD / G;
+  static constexpr int kCH = G / kChunk;                          // chunks per value group
   static constexpr int kKCodes = kChunk * 16 * BITS;
   static constexpr int kKMeta = kChunk * kNG * 4;
   static constexpr int kVCodes = 512 * BITS;
   static constexpr int kVMeta = kD * 4;
   static constexpr int kOffKMeta = kKCodes;
   static constexpr int kOffVCodes = kOffKMeta + kKMeta;
-  static constexpr int kOffVMeta = kOffVCodes + kVCodes;
-  static constexpr int kBytes = kOffVMeta + kVMeta;
-  static constexpr int kStages = BITS == 2 ? 4 : 2;
+  static constexpr int kRec = kOffVCodes + kVCodes;               // bytes of one chunk record
+  static constexpr int kGroupRec = kCH * kRec + kVMeta;           // bytes of one group record
+  // offset of chunk cc of an iteration inside the stage (iterations start on a group boundary or, when a
+  // group spans several iterations, inside one group)
+  __host__ __device__ static constexpr int off(int cc) { return cc * kRec + (cc / kCH) * kVMeta; }
+  static constexpr int kBytes = CPI * kRec + (CPI / kCH > 0 ? CPI / kCH : 1) * kVMeta;
+  static constexpr int kStages = (BITS == 2 ? 4 : 2) / CPI > 1 ? (BITS == 2 ? 4 : 2) / CPI : 2;
   static constexpr int kWarpBytes = kBytes * kStages;
-  static constexpr int kSideBytes = 4 * kVMeta;                  // per warp: value metadata of the last 4 groups
+  static constexpr int kSideBytes = 4 * kVMeta;                   // per warp: value metadata of the last 4 groups
+  static constexpr int kTableBytes = 5120;                        // q tables of the prologue
   static constexpr int kOffSide = kWarpBytes * kWarps;
-  static constexpr int kOffBars = kOffSide + kSideBytes * kWarps;
+  static constexpr int kSideArea = kSideBytes * kWarps > kTableBytes ? kSideBytes * kWarps : kTableBytes;
+  static constexpr int kOffBars = kOffSide + kSideArea;
   static constexpr int kCtaBytes = kOffBars + 256;
 };
 
@@ -145,7 +154,7 @@ struct DecodeArgs {
   __half* out;
   int n_splits;          // fast-path CTAs per unit (blockIdx.y < n_splits); blockIdx.y >= n_splits are tail CTAs
   int n_tail_tiles;      // tail CTAs per unit, 32 list entries each
-  int groups_per_split;
+  int units_per_split;   // range units (max(value group, iteration) of chunks) per fast-path CTA
   int head0;             // first query head (within the KV head's r) handled by this launch
 };
 
@@ -270,27 +279,31 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a,
 }
 
 // ---- the kernel -------------------------------------------------------------------------------------
+// CPI = chunks (of 32 tokens) a warp processes per loop iteration: one barrier wait, one soft-max update and
+// one refill per iteration, and CPI*2 independent key accumulator chains in flight.
 // SPLIT (one query head per KV head, G = 32): the 8 mma columns are not 4 heads x {hi, lo} but
 // 4 groups x {hi, lo}: for keys, column pair g holds q'' restricted to channel group g, so one accumulator
 // chain over all 8 k-steps yields the four per-group code sums at once and lane j of each quad applies the
 // scale / zero-point of group j only (then the quad adds up); for values, column pair w holds p
 // restricted to the w-th value group of a window of four, and lane j applies group j's metadata once per
 // window.  This removes the 4x redundancy a quad otherwise has in decoding per-group metadata.
-template <int BITS, int G, bool SPLIT>
+template <int BITS, int G, bool SPLIT, int CPI>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   using F = Fmt<BITS>;
-  using SL = StageLayout<BITS, G>;
+  using SL = StageLayout<BITS, G, CPI>;
   constexpr int NG = SL::kNG;                   // key groups per token
   constexpr int KS_PER_G = G / 16;              // key k-steps per group
-  constexpr int CH_PER_G = G / kChunk;          // chunks per value group
+  constexpr int CH = SL::kCH;                   // chunks per value group
   constexpr int NST = SL::kStages;
   constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
   constexpr int RWL = F::kRowWordsPerLane;
   constexpr int KPW = F::kKstepsPerWindow;
+  constexpr int RU = CH > CPI ? CH : CPI;       // chunks per range unit (whole groups and whole iterations)
   constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
   static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
   static_assert((NST & (NST - 1)) == 0, "stage count must be a power of two");
+  static_assert(CPI == 1 || CPI == 2, "one or two chunks per iteration");
 
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -300,11 +313,46 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int nh = min(SPLIT ? 1 : kHeads, L.r - a.head0);
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
   const int n_parts = a.n_splits + a.n_tail_tiles;
+  const bool fast = split < a.n_splits;
+
+  // ---------------- this warp's token range; start its first copies before anything else -------------
+  const int n_chunks_total = cn.n_qv / kChunk;
+  const int n_units_total = (n_chunks_total + RU - 1) / RU;
+  const int u_lo = min(n_units_total, split * a.units_per_split);
+  const int u_hi = min(n_units_total, u_lo + a.units_per_split);
+  const int n_u = fast ? u_hi - u_lo : 0;
+  const int wu_lo = u_lo + (int)(((long long)n_u * warp) / kWarps);
+  const int wu_hi = u_lo + (int)(((long long)n_u * (warp + 1)) / kWarps);
+  const int c_lo = wu_lo * RU;                                  // first chunk
+  const int n_iters = (wu_hi - wu_lo) * (RU / CPI);
+
+  unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
+  uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
+  const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
+  const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
+
+  auto issue = [&](int st, int it) {   // one lane: arm the barrier, start the copy of iteration `it` into stage st
+    const int ci = c_lo + it * CPI;
+    const unsigned char* src = g_rec + (size_t)(ci / CH) * SL::kGroupRec + (size_t)(ci % CH) * SL::kRec;
+    // the value group's scale/zero words sit right behind its last chunk
+    const int n_meta = CPI >= CH ? CPI / CH : (((ci + CPI) % CH) == 0 ? 1 : 0);
+    const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
+    mbar_expect_tx(bars_u32 + 8 * st, bytes);
+    bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
+  };
+  if (fast && lane == 0) {
+#pragma unroll
+    for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+#pragma unroll
+    for (int s = 0; s < NST; ++s)
+      if (s < n_iters) issue(s, s);
+  }
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
-  // Tables are staged in the ring memory of warp 0: they are consumed into registers and the CTA
-  // synchronises before the first bulk copy is issued.
-  float* q_nrm_s = reinterpret_cast<float*>(smem);                 // [4][128]
+  float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
   float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
   float* qg_s = q_raw_s + kHeads * kD;                             // [4][4]
   int* qe_s = reinterpret_cast<int*>(qg_s + kHeads * 4);           // [4] exponent of max|q''|
@@ -317,24 +365,33 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     q_nrm_s[i] = L.k_normalize ? v * norm[c] : v;
   }
   __syncthreads();
-  if (tid < kHeads * NG) {
-    const int h = tid / NG, g = tid % NG;
-    float sum = 0.f;
-    for (int c = 0; c < G; ++c) sum += q_nrm_s[h * kD + g * G + c];
-    qg_s[h * 4 + g] = sum;
-  }
-  if (tid < kHeads) {
-    float am = 0.f;
-    for (int c = 0; c < kD; ++c) am = fmaxf(am, fabsf(q_nrm_s[tid * kD + c]));
-    int e = 0;
-    if (am > 0.f && am < INFINITY) frexpf(am, &e);
-    qe_s[tid] = e;     // am < 2^e
+  if (warp < kHeads) {      // warp h: group sums and max |q''| of head h
+    float v[4], am = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { v[e] = q_nrm_s[warp * kD + e * 32 + lane]; am = fmaxf(am, fabsf(v[e])); }
+    // channel c = e * 32 + lane belongs to group c / G
+    float gs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) gs[(e * 32) / G] += v[e];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+#pragma unroll
+      for (int g = 0; g < 4; ++g) gs[g] += __shfl_xor_sync(0xffffffffu, gs[g], o);
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) qg_s[warp * 4 + g] = gs[g];
+      int e = 0;
+      if (am > 0.f && am < INFINITY) frexpf(am, &e);
+      qe_s[warp] = e;     // am < 2^e
+    }
   }
   __syncthreads();
 
-  if (split >= a.n_splits) {
+  if (!fast) {
     // ======================= tail CTA ==============================================================
-    TailSmem& TS = *reinterpret_cast<TailSmem*>(smem + 8192);
+    TailSmem& TS = *reinterpret_cast<TailSmem*>(smem);
     for (int i = tid; i < kHeads * kD; i += kThreads) {
       TS.q_raw[i >> 7][i & (kD - 1)] = q_raw_s[i];
       TS.q_nrm[i >> 7][i & (kD - 1)] = q_nrm_s[i];
@@ -352,15 +409,6 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
   } else {
     // ======================= fast path: packed keys and values ===================================
-    // this warp's range of value groups -> chunks
-    const int n_groups_total = cn.n_qv / G;
-    const int g_lo = min(n_groups_total, split * a.groups_per_split);
-    const int g_hi = min(n_groups_total, g_lo + a.groups_per_split);
-    const int n_g = g_hi - g_lo;
-    const int wg_lo = g_lo + (int)(((long long)n_g * warp) / kWarps);
-    const int wg_hi = g_lo + (int)(((long long)n_g * (warp + 1)) / kWarps);
-    const int c_lo = wg_lo * CH_PER_G, n_chunks = (wg_hi - wg_lo) * CH_PER_G;
-
     // ---- per-thread constants.  As owner of B-fragment column gid: (head, hi|lo) or, in SPLIT, (group, hi|lo).
     const int col_head = SPLIT ? 0 : (gid >> 1), col_group = gid >> 1, col_part = gid & 1;
     const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
@@ -393,36 +441,11 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
     }
     const float neg_half = -(float)(1 << (BITS - 1));
-    __syncthreads();   // tables consumed: ring memory may now be overwritten by bulk copies
-
-    unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
-    uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
-    const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
-    const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
-
-    auto issue = [&](int st, int ci) {   // one lane: arm the barrier, start the copy of chunk ci into stage st
-      // a chunk record is contiguous; the value group's scale/zero words sit right behind its last chunk
-      const bool with_vmeta = (ci % CH_PER_G) == CH_PER_G - 1;
-      const uint32_t bytes = SL::kOffVMeta + (with_vmeta ? SL::kVMeta : 0);
-      const unsigned char* src = g_rec + (size_t)(ci / CH_PER_G) * (CH_PER_G * SL::kOffVMeta + SL::kVMeta) +
-                                 (size_t)(ci % CH_PER_G) * SL::kOffVMeta;
-      mbar_expect_tx(bars_u32 + 8 * st, bytes);
-      bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
-    };
+    __syncthreads();   // tables consumed: the side area may now be used
     if constexpr (SPLIT) {
       for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
+      __syncwarp();
     }
-    if (lane == 0) {
-#pragma unroll
-      for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-#pragma unroll
-      for (int s = 0; s < NST; ++s)
-        if (s < n_chunks) issue(s, c_lo + s);
-    }
-    __syncwarp();
 
     float m_run = -INFINITY, l_part = 0.f, psum = 0.f;
     float out_acc[8][2];
@@ -435,207 +458,218 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
     bool failed = false;
 
-    // The loop body is deliberately not unrolled over chunks: it is a few hundred instructions and two
-    // CTAs of eight warps each walk it at different phases, so it has to stay resident in the
-    // instruction cache.
+    // The loop body is deliberately not unrolled over iterations: two CTAs of eight warps walk it at
+    // different phases, so it has to stay resident in the instruction cache.
 #pragma unroll 1
-    for (int it = 0; it < n_chunks; ++it) {
-      {
-        {
-          const int st = it & (NST - 1);
-          const int s = SPLIT ? (it & (WIN - 1)) : (it % CH_PER_G);      // slot in the window / chunk in the group
-          const uint32_t parity = (uint32_t)(it / NST) & 1u;
-          if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
-          const unsigned char* sp = ring + st * SL::kBytes;
-          const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp);
-          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::kOffKMeta);
-          const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::kOffVCodes);
-          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::kOffVMeta);
-          const bool group_start = s == 0;                  // value accumulators start from zero
-          const bool group_end = SPLIT ? (s == WIN - 1 || it == n_chunks - 1) : (s == CH_PER_G - 1);
-          constexpr bool kFreshEveryChunk = !SPLIT && CH_PER_G == 1;      // then the first value mma takes a zero C
-          if (!kFreshEveryChunk && group_start) {
-#pragma unroll
-            for (int m = 0; m < 8; ++m)
-#pragma unroll
-              for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
-          }
+    for (int it = 0; it < n_iters; ++it) {
+      const int st = it & (NST - 1);
+      const uint32_t parity = (uint32_t)(it / NST) & 1u;
+      if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
+      const unsigned char* sp = ring + st * SL::kBytes;
+      const int ci0 = c_lo + it * CPI;                           // first chunk of this iteration (unit-relative)
+      const bool last_valid = CPI == 1 || (ci0 + 1 < n_chunks_total);   // odd chunk count: the last half is empty
 
-          // ---------------- raw scores of 32 tokens: two m-tiles of 16 ------------------------------
-          float sc[2][2];
+      // ---------------- raw scores: CPI * 2 m-tiles of 16 tokens -------------------------------------
+      float sc[CPI][2][2];
 #pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            const int rA = 16 * mt + gid, rB = rA + 8;
-            uint32_t wa[RWL], wb[RWL];
-            if constexpr (RWL == 2) {
-              const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
-              const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
-              wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
+      for (int cc = 0; cc < CPI; ++cc) {
+        const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc));
+        const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const int rA = 16 * mt + gid, rB = rA + 8;
+          uint32_t wa[RWL], wb[RWL];
+          if constexpr (RWL == 2) {
+            const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
+            const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
+            wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
+          } else {
+            const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
+            const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
+            wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
+            wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
+          }
+          auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
+            const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
+            const int window = sw / KPW, kk = sw % KPW;
+            const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
+            const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
+            const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
+            if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+            else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+          };
+          float sA, sB;
+          if constexpr (SPLIT) {
+            float c4[4];
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
+            float s_, z_;
+            decode_fast(km[rA * NG + j], neg_half, s_, z_);
+            sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
+            decode_fast(km[rB * NG + j], neg_half, s_, z_);
+            sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
+            sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+            sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+            sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+            sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+          } else {
+            uint32_t ma[NG], mb[NG];
+            if constexpr (NG == 4) {
+              const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
+              const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
+              ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
+              mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
+            } else if constexpr (NG == 2) {
+              const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
+              const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
+              ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
             } else {
-              const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
-              const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
-              wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
-              wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
+              ma[0] = km[rA]; mb[0] = km[rB];
             }
-            auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
-              const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
-              const int window = sw / KPW, kk = sw % KPW;
-              const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
-              const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
-              const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
-              if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-              else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-            };
-            float sA, sB;
-            if constexpr (SPLIT) {
+            sA = 0.f; sB = 0.f;
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
               float c4[4];
 #pragma unroll
-              for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
+              for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
               float s_, z_;
-              decode_fast(km[rA * NG + j], neg_half, s_, z_);
-              sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
-              decode_fast(km[rB * NG + j], neg_half, s_, z_);
-              sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
-              sA += __shfl_xor_sync(0xffffffffu, sA, 1);
-              sB += __shfl_xor_sync(0xffffffffu, sB, 1);
-              sA += __shfl_xor_sync(0xffffffffu, sA, 2);
-              sB += __shfl_xor_sync(0xffffffffu, sB, 2);
-            } else {
-              uint32_t ma[NG], mb[NG];
-              if constexpr (NG == 4) {
-                const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
-                const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
-                ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
-                mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
-              } else if constexpr (NG == 2) {
-                const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
-                const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
-                ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
-              } else {
-                ma[0] = km[rA]; mb[0] = km[rB];
-              }
-              sA = 0.f; sB = 0.f;
-#pragma unroll
-              for (int g = 0; g < NG; ++g) {
-                float c4[4];
-#pragma unroll
-                for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
-                float s_, z_;
-                decode_fast(ma[g], neg_half, s_, z_);
-                sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
-                decode_fast(mb[g], neg_half, s_, z_);
-                sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
-              }
-            }
-            sc[mt][0] = sA;
-            sc[mt][1] = sB;
-          }
-
-          // ---------------- online softmax (log2 domain; raw scores still carry 1/kfac) -------------
-          float cmax = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
-          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
-          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-          cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
-          const float m_new = fmaxf(m_run, cmax * kfac);
-          if (__any_sync(0xffffffffu, m_new > m_run)) {
-            const float alpha = ex2_approx(m_run - m_new);     // 0 on the first chunk (m_run = -inf)
-            l_part *= alpha;
-            psum *= alpha;
-#pragma unroll
-            for (int m = 0; m < 8; ++m) {
-              out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
-              if (!kFreshEveryChunk) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
-              }
+              decode_fast(ma[g], neg_half, s_, z_);
+              sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
+              decode_fast(mb[g], neg_half, s_, z_);
+              sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
             }
           }
-          m_run = m_new;
-          uint32_t Bp[2][2];
-          float psum_c = 0.f;
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const float p = ex2_approx(fmaf(sc[mt][h], kfac, -m_new));
-              psum_c += p;
-              const int pos = BITS == 2 ? 2 * mt + h : h;
-              uint32_t pk = split_hi_lo(p * pow2i(10 - BITS * pos));
-              if (SPLIT && j != s) pk = 0u;                     // column pair of this chunk's window slot only
-              Bp[mt][h] = movmatrix_trans(pk);
-            }
-          }
-          l_part += psum_c;
-          if constexpr (SPLIT) psum += (j == s) ? psum_c : 0.f;
-          else psum += psum_c;
-
-          // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ----------------
-          if constexpr (BITS == 2) {
-            const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
-            const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
-            const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-            for (int m = 0; m < 8; ++m) {
-              const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
-#pragma unroll
-              for (int ks = 0; ks < 2; ++ks) {
-                const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
-                if (kFreshEveryChunk && ks == 0) mma16816_z(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-                else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-              }
-            }
-          } else {
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
-#pragma unroll
-              for (int hh = 0; hh < 2; ++hh) {
-                const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
-                const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int mm = 0; mm < 4; ++mm) {
-                  const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
-                  const uint32_t m0 = F::kField, m1 = F::kField << 4;
-                  if (kFreshEveryChunk && ks == 0)
-                    mma16816_z(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-                  else
-                    mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-                }
-              }
-            }
-          }
-
-          // ---------------- end of a value group: apply scale / zero-point once per channel ---------
-          if constexpr (SPLIT) {
-            // keep this group's metadata for the end of the window (the stage will be refilled)
-            *reinterpret_cast<uint4*>(side + s * kD + lane * 4) = *reinterpret_cast<const uint4*>(vm + lane * 4);
-          }
-          if (group_end) {
-            if constexpr (SPLIT) __syncwarp();
-            float pg = psum;
-            pg += __shfl_xor_sync(0xffffffffu, pg, 4);
-            pg += __shfl_xor_sync(0xffffffffu, pg, 8);
-            pg += __shfl_xor_sync(0xffffffffu, pg, 16);
-            pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
-            const uint4* vm4 = reinterpret_cast<const uint4*>((SPLIT ? side + j * kD : vm) + gid * 16);
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              const uint4 mw = vm4[q4];
-              const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
-                float s_, z_;
-                decode_fast(mws[e], neg_half, s_, z_);
-                out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
-              }
-            }
-            psum = 0.f;
-          }
-
-          __syncwarp();
-          if (lane == 0 && it + NST < n_chunks) issue(st, c_lo + it + NST);
+          const bool valid = cc == 0 || last_valid;
+          sc[cc][mt][0] = valid ? sA : -INFINITY;
+          sc[cc][mt][1] = valid ? sB : -INFINITY;
         }
       }
+
+      // ---------------- online softmax (log2 domain; raw scores still carry 1/kfac) -------------------
+      float cmax = -INFINITY;
+#pragma unroll
+      for (int cc = 0; cc < CPI; ++cc)
+        cmax = fmaxf(cmax, fmaxf(fmaxf(sc[cc][0][0], sc[cc][0][1]), fmaxf(sc[cc][1][0], sc[cc][1][1])));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
+      const float m_new = fmaxf(m_run, cmax * kfac);
+      if (__any_sync(0xffffffffu, m_new > m_run)) {
+        const float alpha = ex2_approx(m_run - m_new);     // 0 on the first iteration (m_run = -inf)
+        l_part *= alpha;
+        psum *= alpha;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
+        }
+      }
+      m_run = m_new;
+
+#pragma unroll
+      for (int cc = 0; cc < CPI; ++cc) {
+        const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffVCodes);
+        const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
+        const int ci = ci0 + cc;
+        // slot: position of this chunk's value group in the SPLIT window / position of the chunk in its group
+        const int slot = SPLIT ? (ci - c_lo) & (WIN - 1) : ci % CH;
+        const bool group_start = slot == 0;
+        const bool group_end = SPLIT ? (slot == WIN - 1 || (it == n_iters - 1 && (cc == CPI - 1 || !last_valid)))
+                                     : (slot == CH - 1);
+        constexpr bool kFreshEveryChunk = !SPLIT && CH == 1;   // then the first value mma takes a zero C
+        if (!kFreshEveryChunk && group_start) {
+#pragma unroll
+          for (int m = 0; m < 8; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
+        }
+        uint32_t Bp[2][2];
+        float psum_c = 0.f;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const float p = ex2_approx(fmaf(sc[cc][mt][h], kfac, -m_new));
+            psum_c += p;
+            const int pos = BITS == 2 ? 2 * mt + h : h;
+            uint32_t pk = split_hi_lo(p * pow2i(10 - BITS * pos));
+            if (SPLIT && j != slot) pk = 0u;                 // column pair of this chunk's window slot only
+            Bp[mt][h] = movmatrix_trans(pk);
+          }
+        }
+        l_part += psum_c;
+        if constexpr (SPLIT) psum += (j == slot) ? psum_c : 0.f;
+        else psum += psum_c;
+
+        // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
+        if constexpr (BITS == 2) {
+          const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
+          const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
+          const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+          for (int m = 0; m < 8; ++m) {
+            const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+              const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
+              if (kFreshEveryChunk && ks == 0) mma16816_z(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+              else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
+              const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int mm = 0; mm < 4; ++mm) {
+                const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
+                const uint32_t m0 = F::kField, m1 = F::kField << 4;
+                if (kFreshEveryChunk && ks == 0)
+                  mma16816_z(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                else
+                  mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+              }
+            }
+          }
+        }
+
+        // ---------------- end of a value group: apply scale / zero-point once per channel -----------
+        const bool chunk_valid = cc == 0 || last_valid;
+        if constexpr (SPLIT) {
+          // keep this group's metadata for the end of the window (the stage will be refilled)
+          if (chunk_valid)
+            *reinterpret_cast<uint4*>(side + slot * kD + lane * 4) = *reinterpret_cast<const uint4*>(vm + lane * 4);
+        }
+        if (group_end && chunk_valid) {
+          if constexpr (SPLIT) __syncwarp();
+          float pg = psum;
+          pg += __shfl_xor_sync(0xffffffffu, pg, 4);
+          pg += __shfl_xor_sync(0xffffffffu, pg, 8);
+          pg += __shfl_xor_sync(0xffffffffu, pg, 16);
+          pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
+          const uint4* vm4 = reinterpret_cast<const uint4*>((SPLIT ? side + j * kD : vm) + gid * 16);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 mw = vm4[q4];
+            const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
+              float s_, z_;
+              decode_fast(mws[e], neg_half, s_, z_);
+              out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
+            }
+          }
+          psum = 0.f;
+        }
+      }
+
+      __syncwarp();
+      if (lane == 0 && it + NST < n_iters) issue(st, it + NST);
     }
 
     if (failed) {
@@ -664,16 +698,17 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     __syncthreads();                                   // every warp is done with its ring
     float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
     const bool writer = SPLIT ? (j == 0) : true;
+    const bool any = n_iters > 0;
     if (writer) {
       float* mine = wres + ((size_t)warp * kHeads + (SPLIT ? 0 : j)) * (kD + 2);
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
-        mine[16 * m + gid] = n_chunks > 0 ? out_acc[m][0] * 0x1p14f : 0.f;
-        mine[16 * m + 8 + gid] = n_chunks > 0 ? out_acc[m][1] * 0x1p14f : 0.f;
+        mine[16 * m + gid] = any ? out_acc[m][0] * 0x1p14f : 0.f;
+        mine[16 * m + 8 + gid] = any ? out_acc[m][1] * 0x1p14f : 0.f;
       }
       if (gid == 0) {
-        mine[kD] = n_chunks > 0 ? m_run : -INFINITY;
-        mine[kD + 1] = n_chunks > 0 ? l_part : 0.f;
+        mine[kD] = any ? m_run : -INFINITY;
+        mine[kD + 1] = any ? l_part : 0.f;
       }
     }
     __syncthreads();
@@ -724,25 +759,44 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
 }
 
-template <int BITS, int G, bool SPLIT>
-int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, dim3 grid, cudaStream_t st) {
-  using SL = StageLayout<BITS, G>;
-  constexpr int kSmem = SL::kCtaBytes > 8192 + (int)sizeof(TailSmem) ? SL::kCtaBytes : 8192 + (int)sizeof(TailSmem);
+int g_chunks_per_iter = 0;    // tuning knob: 0 automatic, else 1 or 2 chunks of 32 tokens per loop iteration
+
+template <int BITS, int G, bool SPLIT, int CPI>
+int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
+  using SL = StageLayout<BITS, G, CPI>;
+  constexpr int kSmem = SL::kCtaBytes > (int)sizeof(TailSmem) ? SL::kCtaBytes : (int)sizeof(TailSmem);
+  constexpr int RU = SL::kCH > CPI ? SL::kCH : CPI;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G, SPLIT, CPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSmem) != cudaSuccess)
       return -1;
     configured = true;
   }
+  const int n_chunks = cn.n_qv / kChunk;
+  const int n_units = (n_chunks + RU - 1) / RU;
+  const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
+  if (n_splits > by_work) n_splits = by_work;
+  if (n_units == 0) n_splits = 0;
+  a.n_splits = n_splits;
+  a.units_per_split = n_splits ? (n_units + n_splits - 1) / n_splits : 0;
+  dim3 grid(L.U, n_splits + a.n_tail_tiles);
   int launches = 0;
   const int step = SPLIT ? 1 : kHeads;
   for (int h0 = 0; h0 < L.r; h0 += step) {
     a.head0 = h0;
-    decode_mma_kernel<BITS, G, SPLIT><<<grid, kThreads, kSmem, st>>>(L, cn, a);
+    decode_mma_kernel<BITS, G, SPLIT, CPI><<<grid, kThreads, kSmem, st>>>(L, cn, a);
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+template <int BITS, int G, bool SPLIT>
+int launch_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, cudaStream_t st) {
+  // two chunks per iteration need twice the stage bytes: with 4-bit codes that would cost the second resident CTA
+  const int cpi = g_chunks_per_iter ? g_chunks_per_iter : (BITS == 2 ? 2 : 1);
+  if (cpi == 1) return launch_one<BITS, G, SPLIT, 1>(L, cn, a, n_splits, st);
+  return launch_one<BITS, G, SPLIT, 2>(L, cn, a, n_splits, st);
 }
 
 }  // namespace
@@ -752,37 +806,34 @@ bool decode_mma_supported(const Layout& L) {
          (L.k.bits == 2 || L.k.bits == 4) && L.k.meta_bytes == 4 && L.v.meta_bytes == 4;
 }
 
+void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
+
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                       __half* out, int n_splits, cudaStream_t st) {
   if (!decode_mma_supported(L)) return -2;
   const Counts cn = counts_for(L, N);
-  const int n_groups = cn.n_qv / L.G;
   const int n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
   if (n_splits <= 0) {
     n_splits = (2 * 148 + L.U - 1) / L.U - 1;   // about two resident CTAs per SM; the (short) tail CTAs launch last
     if (n_splits < 1) n_splits = 1;
   }
-  const int by_work = (n_groups + kWarps - 1) / kWarps;      // at least one group per warp
-  if (n_splits > by_work) n_splits = by_work;
   if (n_splits > L.max_splits - n_tail_tiles) n_splits = L.max_splits - n_tail_tiles;
-  if (n_groups == 0) n_splits = 0;
-  if (n_splits < 0 || n_splits + n_tail_tiles > L.max_splits) return -2;
+  if (n_splits < 0) return -2;
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
   a.n_tail_tiles = n_tail_tiles;
-  a.groups_per_split = n_splits ? (n_groups + n_splits - 1) / n_splits : 0;
+  a.units_per_split = 0;
   a.head0 = 0;
-  dim3 grid(L.U, n_splits + n_tail_tiles);
   const int bits = L.k.bits;
-  if (bits == 2 && L.G == 32 && L.r == 1) return launch_one<2, 32, true>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 32 && L.r == 1) return launch_one<4, 32, true>(L, cn, a, grid, st);
-  if (bits == 2 && L.G == 32) return launch_one<2, 32, false>(L, cn, a, grid, st);
-  if (bits == 2 && L.G == 64) return launch_one<2, 64, false>(L, cn, a, grid, st);
-  if (bits == 2 && L.G == 128) return launch_one<2, 128, false>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 32) return launch_one<4, 32, false>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 64) return launch_one<4, 64, false>(L, cn, a, grid, st);
-  if (bits == 4 && L.G == 128) return launch_one<4, 128, false>(L, cn, a, grid, st);
+  if (bits == 2 && L.G == 32 && L.r == 1) return launch_cpi<2, 32, true>(L, cn, a, n_splits, st);
+  if (bits == 4 && L.G == 32 && L.r == 1) return launch_cpi<4, 32, true>(L, cn, a, n_splits, st);
+  if (bits == 2 && L.G == 32) return launch_cpi<2, 32, false>(L, cn, a, n_splits, st);
+  if (bits == 2 && L.G == 64) return launch_cpi<2, 64, false>(L, cn, a, n_splits, st);
+  if (bits == 2 && L.G == 128) return launch_cpi<2, 128, false>(L, cn, a, n_splits, st);
+  if (bits == 4 && L.G == 32) return launch_cpi<4, 32, false>(L, cn, a, n_splits, st);
+  if (bits == 4 && L.G == 64) return launch_cpi<4, 64, false>(L, cn, a, n_splits, st);
+  if (bits == 4 && L.G == 128) return launch_cpi<4, 128, false>(L, cn, a, n_splits, st);
   return -2;
 }
 

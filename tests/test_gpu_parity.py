@@ -67,7 +67,8 @@ def test_prefill_and_decode_inner(bits, G, mode, variant, N):
     w = synth.tiny(n_tokens=N, group=G, k_bits=bits, v_bits=bits, k_mode=mode, v_mode=mode, sym_variant=variant)
     oc, gc, _, _ = run_prefill_both(w)
     P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, mode == O.HYBRID, mode == O.HYBRID)
-    check_decode(w, oc, gc, variants=(0, 1), splits=(0, 1, 3, 7))
+    fast = (3, 4) if bits in (2, 4) and mode != O.SYM else ()
+    check_decode(w, oc, gc, variants=(0, 1) + fast, splits=(0, 1, 3, 7))
 
 
 @pytest.mark.parametrize("bits,G,N", [(2, 32, 333), (3, 64, 420), (4, 128, 541)])
@@ -182,5 +183,5 @@ def test_config1_full_parity():
     w = synth.config1()
     oc, gc, _, _ = run_prefill_both(w)
     flips = P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
-    worst = check_decode(w, oc, gc, variants=(0, 1), splits=(0, 1, 4, 13))
+    worst = check_decode(w, oc, gc, variants=(0, 1, 3, 4), splits=(0, 1, 4, 13))
     print(f"config1: contested flips {flips}, worst err/tol {worst:.3f}")
