@@ -156,11 +156,15 @@ class InnerQCache:
         self._h = h
 
     def close(self):
-        if getattr(self, "_h", None):
-            lib().innerq_cache_destroy(self._h)
-            self._h = None
+        h, self._h = getattr(self, "_h", None), None
+        if h and _lib is not None:
+            _lib.innerq_cache_destroy(h)
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:       # interpreter shutdown: globals may already be gone
+            pass
 
     @property
     def n_tokens(self) -> int:

@@ -152,8 +152,8 @@ struct DecodeArgs {
   unsigned char* ws;
   const __half* q;
   __half* out;
-  int n_splits;          // fast-path CTAs per unit (blockIdx.y < n_splits); blockIdx.y >= n_splits are tail CTAs
-  int n_tail_tiles;      // tail CTAs per unit, 32 list entries each
+  int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
+  int n_tail_tiles;      // tiles of 32 entries of the fp16 tail; CTA y handles tiles y, y + gridDim.y, ...
   int units_per_split;   // range units (max(value group, iteration) of chunks) per fast-path CTA
   int head0;             // first query head (within the KV head's r) handled by this launch
 };
@@ -314,6 +314,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
   const int n_parts = a.n_splits + a.n_tail_tiles;
   const bool fast = split < a.n_splits;
+  const bool has_tail = split < a.n_tail_tiles;      // this CTA also handles tail tiles (done first)
 
   // ---------------- this warp's token range; start its first copies before anything else -------------
   const int n_chunks_total = cn.n_qv / kChunk;
@@ -341,15 +342,18 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
     bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
   };
-  if (fast && lane == 0) {
+  auto start_copies = [&]() {
+    if (fast && lane == 0) {
 #pragma unroll
-    for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 #pragma unroll
-    for (int s = 0; s < NST; ++s)
-      if (s < n_iters) issue(s, s);
-  }
+      for (int s = 0; s < NST; ++s)
+        if (s < n_iters) issue(s, s);
+    }
+  };
+  if (!has_tail) start_copies();     // otherwise the ring memory first serves the tail tiles
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
   float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
@@ -389,25 +393,30 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   }
   __syncthreads();
 
-  if (!fast) {
-    // ======================= tail CTA ==============================================================
+  if (has_tail) {
+    // ======================= tail tiles (fp16 windows, skew zone) ==================================
     TailSmem& TS = *reinterpret_cast<TailSmem*>(smem);
     for (int i = tid; i < kHeads * kD; i += kThreads) {
       TS.q_raw[i >> 7][i & (kD - 1)] = q_raw_s[i];
       TS.q_nrm[i >> 7][i & (kD - 1)] = q_nrm_s[i];
     }
     __syncthreads();
-    float acc[kHeads], m_t[kHeads], l_t[kHeads];
-    tail_cta(L, cn, a, u, nh, split - a.n_splits, TS, acc, m_t, l_t);
     float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
-    if (tid < kD) {
-      for (int h = 0; h < nh; ++h) {
-        float* P = partials + ((size_t)(head_base + h) * L.max_splits + split) * kPartialStride;
-        P[tid] = acc[h];
-        if (tid == 0) { P[kD] = m_t[h]; P[kD + 1] = l_t[h]; }
+    for (int tile = split; tile < a.n_tail_tiles; tile += gridDim.y) {
+      float acc[kHeads], m_t[kHeads], l_t[kHeads];
+      tail_cta(L, cn, a, u, nh, tile, TS, acc, m_t, l_t);
+      if (tid < kD) {
+        for (int h = 0; h < nh; ++h) {
+          float* P = partials + ((size_t)(head_base + h) * L.max_splits + a.n_splits + tile) * kPartialStride;
+          P[tid] = acc[h];
+          if (tid == 0) { P[kD] = m_t[h]; P[kD + 1] = l_t[h]; }
+        }
       }
+      __syncthreads();
     }
-  } else {
+    start_copies();
+  }
+  if (fast) {
     // ======================= fast path: packed keys and values ===================================
     // ---- per-thread constants.  As owner of B-fragment column gid: (head, hi|lo) or, in SPLIT, (group, hi|lo).
     const int col_head = SPLIT ? 0 : (gid >> 1), col_group = gid >> 1, col_part = gid & 1;
@@ -738,21 +747,42 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   __syncthreads();
   if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
   __syncthreads();
-  if (s_ticket != (unsigned int)(n_parts - 1)) return;
+  if (s_ticket != gridDim.y - 1) return;
   __threadfence();
   const float* partials = reinterpret_cast<const float*>(a.ws + L.ws_partial_off);
+  float* mw = reinterpret_cast<float*>(smem);          // [head][part]: max, then weight
+  float* lw = mw + kHeads * 128;                        // [head][part]: l
+  for (int i = tid; i < nh * n_parts; i += kThreads) {
+    const int h = i / n_parts, s = i % n_parts;
+    const float* P = partials + ((size_t)(head_base + h) * L.max_splits + s) * kPartialStride;
+    mw[h * 128 + s] = __ldcg(P + kD);
+    lw[h * 128 + s] = __ldcg(P + kD + 1);
+  }
+  __syncthreads();
   for (int i = tid; i < nh * kD; i += kThreads) {
     const int h = i >> 7, c = i & (kD - 1);
-    const float* P = partials + (size_t)(head_base + h) * L.max_splits * kPartialStride;
+    const float* P = partials + (size_t)(head_base + h) * L.max_splits * kPartialStride + c;
     float M = -INFINITY;
-    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, __ldcg(P + s * kPartialStride + kD));
+    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, mw[h * 128 + s]);
     float num = 0.f, den = 0.f;
-    for (int s = 0; s < n_parts; ++s) {
-      const float ms = __ldcg(P + s * kPartialStride + kD);
-      if (ms == -INFINITY) continue;
-      const float wgt = exp2f(ms - M);
-      num = fmaf(__ldcg(P + s * kPartialStride + c), wgt, num);
-      den = fmaf(__ldcg(P + s * kPartialStride + kD + 1), wgt, den);
+    int s = 0;
+    for (; s + 4 <= n_parts; s += 4) {                  // four independent loads in flight
+      float v[4], wgt[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] = __ldcg(P + (size_t)(s + e) * kPartialStride);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float ms = mw[h * 128 + s + e];
+        wgt[e] = ms == -INFINITY ? 0.f : exp2f(ms - M);
+        num = fmaf(v[e], wgt[e], num);
+        den = fmaf(lw[h * 128 + s + e], wgt[e], den);
+      }
+    }
+    for (; s < n_parts; ++s) {
+      const float ms = mw[h * 128 + s];
+      const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
+      num = fmaf(__ldcg(P + (size_t)s * kPartialStride), wgt, num);
+      den = fmaf(lw[h * 128 + s], wgt, den);
     }
     a.out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
   }
@@ -780,7 +810,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   if (n_units == 0) n_splits = 0;
   a.n_splits = n_splits;
   a.units_per_split = n_splits ? (n_units + n_splits - 1) / n_splits : 0;
-  dim3 grid(L.U, n_splits + a.n_tail_tiles);
+  dim3 grid(L.U, n_splits > 0 ? n_splits : a.n_tail_tiles);
   int launches = 0;
   const int step = SPLIT ? 1 : kHeads;
   for (int h0 = 0; h0 < L.r; h0 += step) {
@@ -814,11 +844,11 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   const Counts cn = counts_for(L, N);
   const int n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
   if (n_splits <= 0) {
-    n_splits = (2 * 148 + L.U - 1) / L.U - 1;   // about two resident CTAs per SM; the (short) tail CTAs launch last
+    n_splits = (2 * 148) / L.U;                  // two resident CTAs per SM, one wave
     if (n_splits < 1) n_splits = 1;
   }
   if (n_splits > L.max_splits - n_tail_tiles) n_splits = L.max_splits - n_tail_tiles;
-  if (n_splits < 0) return -2;
+  if (n_splits < 0 || n_splits + n_tail_tiles > 128) return -2;
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
