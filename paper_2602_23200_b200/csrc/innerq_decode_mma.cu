@@ -140,7 +140,7 @@ template <int BITS, int G, int CPI> struct StageLayout {
   static constexpr int kStages = (BITS == 2 ? 4 : 2) / CPI > 1 ? (BITS == 2 ? 4 : 2) / CPI : 2;
   static constexpr int kWarpBytes = kBytes * kStages;
   static constexpr int kSideBytes = 4 * kVMeta;                   // per warp: value metadata of the last 4 groups
-  static constexpr int kTableBytes = 5120;                        // q tables of the prologue
+  static constexpr int kTableBytes = 6400;                        // q tables and B fragments of the prologue
   static constexpr int kOffSide = kWarpBytes * kWarps;
   static constexpr int kSideArea = kSideBytes * kWarps > kTableBytes ? kSideBytes * kWarps : kTableBytes;
   static constexpr int kOffBars = kOffSide + kSideArea;
@@ -153,130 +153,15 @@ struct DecodeArgs {
   const __half* q;
   __half* out;
   int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
-  int n_tail_tiles;      // tiles of 32 entries of the fp16 tail; CTA y handles tiles y, y + gridDim.y, ...
-  int units_per_split;   // range units (max(value group, iteration) of chunks) per fast-path CTA
+  int n_tail_tiles;      // mini-tiles of 8 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
+                         // tile x belongs to CTA x % gridDim.y, warp (x / gridDim.y) % 8
+  int n_skew_tiles;      // of those, tiles whose keys are packed rows (values still fp16)
+  int tiles_q0, tiles_rem;   // n_tail_tiles / gridDim.y and n_tail_tiles % gridDim.y
+  int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
+  int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
+  int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
   int head0;             // first query head (within the KV head's r) handled by this launch
 };
-
-// ---- tail: fp16 windows, and key rows whose values are still fp16 (plain SIMT, small) ---------------
-// Token list of the tail: [0, n_sink) and [n_sink + n_qv, N).  One tail CTA handles one tile of 32 list
-// entries: it stages the tile's key rows (fp16 window rows, or dequantised skew-zone rows) and value rows
-// in shared memory with independent 128-bit loads, then scores, soft-maxes and accumulates from there.
-struct TailSmem {
-  float q_raw[kHeads][kD], q_nrm[kHeads][kD];
-  float k[32][kD + 4];
-  __half v[32][kD];
-  float sc[32][kHeads];
-  float m[kHeads], l[kHeads];
-  float acc2[kHeads][kD];
-  int quant[32];
-};
-
-__device__ void tail_cta(const Layout& L, const Counts& cn, const DecodeArgs& a, int u, int nh, int tile, TailSmem& S,
-                         float (&acc)[kHeads], float (&m_out)[kHeads], float (&l_out)[kHeads]) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const Store& Ks = L.k;
-  const Store& Vs = L.v;
-  const __half* k_sink = reinterpret_cast<const __half*>(a.cache + Ks.sink_off + (size_t)u * Ks.sink_stride);
-  const __half* k_ring = reinterpret_cast<const __half*>(a.cache + Ks.ring_off + (size_t)u * Ks.ring_stride);
-  const __half* v_sink = reinterpret_cast<const __half*>(a.cache + Vs.sink_off + (size_t)u * Vs.sink_stride);
-  const __half* v_ring = reinterpret_cast<const __half*>(a.cache + Vs.ring_off + (size_t)u * Vs.ring_stride);
-  const unsigned char* k_rec = a.cache + Ks.rec_off + (size_t)u * Ks.rec_unit_stride;
-  const int n_tail = cn.n_sink + (cn.N - cn.n_sink - cn.n_qv);
-  const int i0 = tile * 32;
-  // ---- stage the tile: 32 rows x 16 pieces of 8 channels
-#pragma unroll
-  for (int rep = 0; rep < 2; ++rep) {
-    const int idx = tid + rep * kThreads;
-    const int tt = idx >> 4, piece = idx & 15;
-    const int i = i0 + tt;
-    uint4 vraw = make_uint4(0u, 0u, 0u, 0u);
-    float kx[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    int quant = 0;
-    if (i < n_tail) {
-      const int t = i < cn.n_sink ? i : cn.n_qv + i;
-      const int iq = t - cn.n_sink;   // index among the packed key rows, if < n_qk
-      const __half* vrow = t < cn.n_sink ? v_sink + (size_t)t * kD : v_ring + (size_t)((t - L.w_sink) % Vs.ring_cap) * kD;
-      vraw = *reinterpret_cast<const uint4*>(vrow + piece * 8);
-      if (t < cn.n_sink || iq >= cn.n_qk) {
-        const __half* row = t < cn.n_sink ? k_sink + (size_t)t * kD : k_ring + (size_t)((t - L.w_sink) % Ks.ring_cap) * kD;
-        const uint4 raw = *reinterpret_cast<const uint4*>(row + piece * 8);
-        const __half2* hh = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 x = __half22float2(hh[e]);
-          kx[2 * e] = x.x; kx[2 * e + 1] = x.y;
-        }
-      } else {
-        quant = 1;
-        float s_, z_;
-        decode_meta(load_meta(k_rec + row_meta_off(Ks, iq), (piece * 8) / L.G, Ks.meta_bytes), Ks.bits, s_, z_);
-        const uint32_t* row = reinterpret_cast<const uint32_t*>(k_rec + row_code_off(Ks, iq));
-#pragma unroll
-        for (int e = 0; e < 8; ++e) kx[e] = fmaf(s_, (float)row_code(row, piece * 8 + e, Ks.bits), z_);
-      }
-    }
-    *reinterpret_cast<uint4*>(&S.v[tt][piece * 8]) = vraw;
-    *reinterpret_cast<float4*>(&S.k[tt][piece * 8]) = make_float4(kx[0], kx[1], kx[2], kx[3]);
-    *reinterpret_cast<float4*>(&S.k[tt][piece * 8 + 4]) = make_float4(kx[4], kx[5], kx[6], kx[7]);
-    if (piece == 0) S.quant[tt] = quant;
-  }
-  __syncthreads();
-  // ---- scores: warp w takes rows w, w + 8, w + 16, w + 24; lane takes channels 4*lane .. +3
-#pragma unroll
-  for (int rr = 0; rr < 4; ++rr) {
-    const int tt = warp + rr * kWarps;
-    const float4 kx = *reinterpret_cast<const float4*>(&S.k[tt][4 * lane]);
-    const bool quant = S.quant[tt] != 0;
-#pragma unroll
-    for (int h = 0; h < kHeads; ++h) {
-      const float4 qv = *reinterpret_cast<const float4*>(quant ? &S.q_nrm[h][4 * lane] : &S.q_raw[h][4 * lane]);
-      float v = fmaf(kx.x, qv.x, fmaf(kx.y, qv.y, fmaf(kx.z, qv.z, kx.w * qv.w)));
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) S.sc[tt][h] = (i0 + tt) < n_tail ? v : -INFINITY;
-    }
-  }
-  __syncthreads();
-  if (warp < kHeads) {
-    const int h = warp;
-    const float sv = S.sc[lane][h];
-    float mt = sv;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, o));
-    const float p = exp2f(sv - mt);
-    float ps = p;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
-    S.sc[lane][h] = p;
-    if (lane == 0) { S.m[h] = mt; S.l[h] = ps; }
-  }
-  __syncthreads();
-  // ---- values: thread owns channel c_own and every second row
-  const int c_own = tid & (kD - 1), half_id = tid >> 7;
-#pragma unroll
-  for (int h = 0; h < kHeads; ++h) acc[h] = 0.f;
-#pragma unroll
-  for (int r2 = 0; r2 < 16; ++r2) {
-    const int tt = 2 * r2 + half_id;
-    const float vx = __half2float(S.v[tt][c_own]);
-    const float4 p4 = *reinterpret_cast<const float4*>(&S.sc[tt][0]);
-    acc[0] = fmaf(p4.x, vx, acc[0]); acc[1] = fmaf(p4.y, vx, acc[1]);
-    acc[2] = fmaf(p4.z, vx, acc[2]); acc[3] = fmaf(p4.w, vx, acc[3]);
-  }
-  if (half_id == 1) {
-#pragma unroll
-    for (int h = 0; h < kHeads; ++h) S.acc2[h][c_own] = acc[h];
-  }
-  __syncthreads();
-#pragma unroll
-  for (int h = 0; h < kHeads; ++h) {
-    if (half_id == 0) acc[h] += S.acc2[h][c_own];
-    m_out[h] = S.m[h];
-    l_out[h] = S.l[h];
-  }
-  (void)nh;
-}
 
 // ---- the kernel -------------------------------------------------------------------------------------
 // CPI = chunks (of 32 tokens) a warp processes per loop iteration: one barrier wait, one soft-max update and
@@ -312,18 +197,33 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int b = u / L.Hkv, hkv = u % L.Hkv;
   const int nh = min(SPLIT ? 1 : kHeads, L.r - a.head0);
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
-  const int n_parts = a.n_splits + a.n_tail_tiles;
+  const int n_parts = gridDim.y;
   const bool fast = split < a.n_splits;
-  const bool has_tail = split < a.n_tail_tiles;      // this CTA also handles tail tiles (done first)
+  constexpr int kTailBytes = 2048 + SL::kOffVCodes;                 // 8 fp16 value rows + a chunk's packed key part
+  constexpr int TS = SL::kBytes >= kTailBytes ? 1 : 2;               // ring stages lent to a tail tile
+  static_assert(TS * SL::kBytes >= kTailBytes && 2048 + 2048 <= TS * SL::kBytes && NST >= TS, "tail tile must fit");
 
-  // ---------------- this warp's token range; start its first copies before anything else -------------
+  // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
+  // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
+  // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
+  const int Gy = gridDim.y, cst = a.tail_cost_units;
   const int n_chunks_total = cn.n_qv / kChunk;
   const int n_units_total = (n_chunks_total + RU - 1) / RU;
-  const int u_lo = min(n_units_total, split * a.units_per_split);
-  const int u_hi = min(n_units_total, u_lo + a.units_per_split);
+  const int q_cta = a.tiles_q0 + (split < a.tiles_rem ? 1 : 0);                 // tail tiles of this CTA
+  const int tiles_before = split * a.tiles_q0 + min(split, a.tiles_rem);         // ... of the CTAs before it
+  auto tiles_of_warp = [&](int q, int w) { return (q >> 3) + (w < (q & 7) ? 1 : 0); };
+  const int u_lo = max(0, min(n_units_total, split * a.units_per_split - cst * tiles_before));
+  const int u_hi = split == a.n_splits - 1
+                       ? n_units_total
+                       : max(u_lo, min(n_units_total, (split + 1) * a.units_per_split - cst * (tiles_before + q_cta)));
   const int n_u = fast ? u_hi - u_lo : 0;
-  const int wu_lo = u_lo + (int)(((long long)n_u * warp) / kWarps);
-  const int wu_hi = u_lo + (int)(((long long)n_u * (warp + 1)) / kWarps);
+  const int n_virtual = n_u + cst * q_cta;
+  const int tw_before = warp * (q_cta >> 3) + min(warp, q_cta & 7);
+  const int tw = tiles_of_warp(q_cta, warp);                        // tail tiles of this warp
+  const int wu_lo = u_lo + max(0, min(n_u, ((n_virtual * warp) >> 3) - cst * tw_before));
+  const int wu_hi = warp == kWarps - 1
+                        ? u_lo + n_u
+                        : max(wu_lo, u_lo + max(0, min(n_u, ((n_virtual * (warp + 1)) >> 3) - cst * (tw_before + tw))));
   const int c_lo = wu_lo * RU;                                  // first chunk
   const int n_iters = (wu_hi - wu_lo) * (RU / CPI);
 
@@ -332,6 +232,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
   const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
+  unsigned char* tail_buf = ring + (NST - TS) * SL::kBytes;      // [8 value rows][key rows | packed key part]
 
   auto issue = [&](int st, int it) {   // one lane: arm the barrier, start the copy of iteration `it` into stage st
     const int ci = c_lo + it * CPI;
@@ -342,18 +243,70 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
     bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
   };
-  auto start_copies = [&]() {
-    if (fast && lane == 0) {
-#pragma unroll
-      for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-#pragma unroll
-      for (int s = 0; s < NST; ++s)
-        if (s < n_iters) issue(s, s);
+  // Tail tile x: up to 8 tokens.  Skew tiles (x < n_skew_tiles): keys are packed rows n_qv + 8x .. of one
+  // chunk record, values fp16 ring rows.  Other tiles: entries of the list [sink tokens, recent key tokens].
+  const int n_skew = cn.n_qk - cn.n_qv, n_list = cn.n_sink + cn.n_k_recent;
+  auto tail_tile = [&](int k, bool& skew, int& e0, int& cnt) {
+    const int x = split + Gy * (warp + kWarps * k);
+    skew = x < a.n_skew_tiles;
+    e0 = 8 * (skew ? x : x - a.n_skew_tiles);
+    cnt = min(8, (skew ? n_skew : n_list) - e0);
+  };
+  // Rows of consecutive entries are contiguous in memory except where a ring wraps or the list passes from the
+  // sink to the ring: copy maximal runs (typically one 2 KB copy for the values, one for the keys).
+  auto issue_tail = [&](int k) {       // one lane: copy the rows of this warp's k-th tail tile into tail_buf
+    bool skew; int e0, cnt;
+    tail_tile(k, skew, e0, cnt);
+    const uint32_t bar = bars_u32 + 8 * (NST - 1), dst = smem_u32(tail_buf);
+    mbar_expect_tx(bar, (uint32_t)cnt * 256u + (skew ? (uint32_t)SL::kOffVCodes : (uint32_t)cnt * 256u));
+    const unsigned char* v_sink = a.cache + L.v.sink_off + (size_t)u * L.v.sink_stride;
+    const unsigned char* v_ring = a.cache + L.v.ring_off + (size_t)u * L.v.ring_stride;
+    const unsigned char* k_sink = a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride;
+    const unsigned char* k_ring = a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride;
+    // row address of list entry e: sink rows, else ring slot = (first slot + offset) wrapped once
+    auto v_row = [&](int e) -> const unsigned char* {
+      if (!skew && e < cn.n_sink) return v_sink + (size_t)e * 256;
+      int slot = a.v_ring_pos0 + (skew ? e : n_skew + (e - cn.n_sink));
+      if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
+      return v_ring + (size_t)slot * 256;
+    };
+    auto k_row = [&](int e) -> const unsigned char* {
+      if (e < cn.n_sink) return k_sink + (size_t)e * 256;
+      int slot = a.k_ring_pos0 + (e - cn.n_sink);
+      if (slot >= L.k.ring_cap) slot -= L.k.ring_cap;
+      return k_ring + (size_t)slot * 256;
+    };
+    for (int i = 0; i < cnt;) {
+      const unsigned char* src = v_row(e0 + i);
+      int run = 1;
+      while (i + run < cnt && v_row(e0 + i + run) == src + run * 256) ++run;
+      bulk_g2s(dst + i * 256, src, run * 256, bar);
+      i += run;
+    }
+    if (skew) {
+      const int ci = (cn.n_qv + e0) / kChunk;
+      bulk_g2s(dst + 2048, g_rec + (size_t)(ci / CH) * SL::kGroupRec + (size_t)(ci % CH) * SL::kRec, SL::kOffVCodes, bar);
+    } else {
+      for (int i = 0; i < cnt;) {
+        const unsigned char* src = k_row(e0 + i);
+        int run = 1;
+        while (i + run < cnt && k_row(e0 + i + run) == src + run * 256) ++run;
+        bulk_g2s(dst + 2048 + i * 256, src, run * 256, bar);
+        i += run;
+      }
     }
   };
-  if (!has_tail) start_copies();     // otherwise the ring memory first serves the tail tiles
+  const int early_stages = tw > 0 ? NST - TS : NST;              // stages free for packed chunks right away
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (tw > 0) issue_tail(0);
+#pragma unroll
+    for (int s = 0; s < NST; ++s)
+      if (s < early_stages && s < n_iters) issue(s, s);
+  }
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
   float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
@@ -393,37 +346,16 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   }
   __syncthreads();
 
-  if (has_tail) {
-    // ======================= tail tiles (fp16 windows, skew zone) ==================================
-    TailSmem& TS = *reinterpret_cast<TailSmem*>(smem);
-    for (int i = tid; i < kHeads * kD; i += kThreads) {
-      TS.q_raw[i >> 7][i & (kD - 1)] = q_raw_s[i];
-      TS.q_nrm[i >> 7][i & (kD - 1)] = q_nrm_s[i];
-    }
-    __syncthreads();
-    float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
-    for (int tile = split; tile < a.n_tail_tiles; tile += gridDim.y) {
-      float acc[kHeads], m_t[kHeads], l_t[kHeads];
-      tail_cta(L, cn, a, u, nh, tile, TS, acc, m_t, l_t);
-      if (tid < kD) {
-        for (int h = 0; h < nh; ++h) {
-          float* P = partials + ((size_t)(head_base + h) * L.max_splits + a.n_splits + tile) * kPartialStride;
-          P[tid] = acc[h];
-          if (tid == 0) { P[kD] = m_t[h]; P[kD + 1] = l_t[h]; }
-        }
-      }
-      __syncthreads();
-    }
-    start_copies();
-  }
-  if (fast) {
+  {
     // ======================= fast path: packed keys and values ===================================
     // ---- per-thread constants.  As owner of B-fragment column gid: (head, hi|lo) or, in SPLIT, (group, hi|lo).
     const int col_head = SPLIT ? 0 : (gid >> 1), col_group = gid >> 1, col_part = gid & 1;
-    const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
-    uint32_t Bq[8][2];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
+    // The fragment values depend on (lane, k-step, register) only, not on the warp: warp w computes the
+    // k-step-w entries for every lane once, all warps then read their 16 registers from shared memory.
+    uint32_t* bq_s = reinterpret_cast<uint32_t*>(qe_s + 16);      // [8 k-steps][2][32 lanes]
+    {
+      const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
+      const int s = warp;
       const int kk = (s % (2 * KPW)) % KPW;
 #pragma unroll
       for (int rr = 0; rr < 2; ++rr) {
@@ -434,8 +366,15 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         const uint32_t v1 = split_hi_lo(q_nrm_s[col_head * kD + c0 + 1] * scl);
         uint32_t v = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
         if (SPLIT && (s / KS_PER_G) != col_group) v = 0u;
-        Bq[s][rr] = v;
+        bq_s[(s * 2 + rr) * 32 + lane] = v;
       }
+    }
+    __syncthreads();
+    uint32_t Bq[8][2];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      Bq[s][0] = bq_s[(s * 2) * 32 + lane];
+      Bq[s][1] = bq_s[(s * 2 + 1) * 32 + lane];
     }
     // ---- as owner of C-fragment columns 2j, 2j+1: head j, or in SPLIT (head 0, key group j)
     const int my_head = SPLIT ? 0 : j;
@@ -450,8 +389,13 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
     }
     const float neg_half = -(float)(1 << (BITS - 1));
-    __syncthreads();   // tables consumed: the side area may now be used
+    // SPLIT reuses the table area for its side ring, so it takes what the tail tiles need of q into
+    // registers (one head: 4 channels per lane) and releases the tables now, while all warps are in step.
+    float4 qraw4 = make_float4(0.f, 0.f, 0.f, 0.f), qnrm4 = qraw4;
     if constexpr (SPLIT) {
+      qraw4 = *reinterpret_cast<const float4*>(q_raw_s + 4 * lane);
+      qnrm4 = *reinterpret_cast<const float4*>(q_nrm_s + 4 * lane);
+      __syncthreads();
       for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
       __syncwarp();
     }
@@ -467,12 +411,82 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
     bool failed = false;
 
+    // ---------------- tail tiles of this warp: fp16 windows and the K/V skew zone, plain SIMT ---------
+    // (8 tokens at a time, straight into the warp's running soft-max state; no CTA-wide synchronisation)
+    for (int k = 0; k < tw && !failed; ++k) {
+      bool skew; int e0, cnt;
+      tail_tile(k, skew, e0, cnt);
+      if (!mbar_wait(bars_u32 + 8 * (NST - 1), (uint32_t)k & 1u)) { failed = true; break; }
+      const __half* vbuf = reinterpret_cast<const __half*>(tail_buf);
+      const unsigned char* kbuf = tail_buf + 2048;
+      constexpr int NHT = SPLIT ? 1 : kHeads;
+      float s_mine[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        float kx[4];
+        if (!skew) {
+          const uint2 raw = *reinterpret_cast<const uint2*>(kbuf + t * 256 + lane * 8);
+          const __half2* hh = reinterpret_cast<const __half2*>(&raw);
+          const float2 x0 = __half22float2(hh[0]), x1 = __half22float2(hh[1]);
+          kx[0] = x0.x; kx[1] = x0.y; kx[2] = x1.x; kx[3] = x1.y;
+        } else {
+          const int rc = (cn.n_qv + e0 + t) % kChunk;            // row inside the chunk record
+          const uint32_t* row = reinterpret_cast<const uint32_t*>(kbuf + rc * (16 * BITS));
+          float s_, z_;
+          decode_fast(reinterpret_cast<const uint32_t*>(kbuf + SL::kOffKMeta)[rc * NG + (4 * lane) / G], neg_half, s_, z_);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) kx[e] = fmaf(s_, (float)row_code(row, 4 * lane + e, BITS), z_);
+        }
+        float mine = 0.f;
+#pragma unroll
+        for (int h = 0; h < NHT; ++h) {
+          const float4 qv = SPLIT ? (skew ? qnrm4 : qraw4)
+                                  : *reinterpret_cast<const float4*>((skew ? q_nrm_s : q_raw_s) + h * kD + 4 * lane);
+          float d = fmaf(kx[0], qv.x, fmaf(kx[1], qv.y, fmaf(kx[2], qv.z, kx[3] * qv.w)));
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+          if (h == my_head) mine = d;
+        }
+        s_mine[t] = t < cnt ? mine : -INFINITY;
+      }
+      float cmax = s_mine[0];
+#pragma unroll
+      for (int t = 1; t < 8; ++t) cmax = fmaxf(cmax, s_mine[t]);
+      const float m_new = fmaxf(m_run, cmax);
+      const float alpha = ex2_approx(m_run - m_new);            // 0 while m_run = -inf
+      m_run = m_new;
+      l_part *= alpha;
+#pragma unroll
+      for (int m = 0; m < 8; ++m) { out_acc[m][0] *= alpha; out_acc[m][1] *= alpha; }
+      // out_acc is kept in units of 2^-14 (see the packed path); in SPLIT only lane 0 of a quad contributes
+      const float unit = (SPLIT && j != 0) ? 0.f : 0x1p-14f;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const float p = ex2_approx(s_mine[t] - m_new);          // 0 for the padding tokens
+        if (t == gid) l_part += p;                              // every token counted once per head
+        if (t < cnt) {
+          const float pu = p * unit;
+#pragma unroll
+          for (int m = 0; m < 8; ++m) {
+            out_acc[m][0] = fmaf(pu, __half2float(vbuf[t * kD + 16 * m + gid]), out_acc[m][0]);
+            out_acc[m][1] = fmaf(pu, __half2float(vbuf[t * kD + 16 * m + 8 + gid]), out_acc[m][1]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0 && k + 1 < tw) issue_tail(k + 1);
+    }
+    if (tw > 0 && lane == 0) {     // the lent stages go back to the packed stream
+#pragma unroll
+      for (int s = 0; s < NST; ++s)
+        if (s >= early_stages && s < n_iters) issue(s, s);
+    }
     // The loop body is deliberately not unrolled over iterations: two CTAs of eight warps walk it at
     // different phases, so it has to stay resident in the instruction cache.
 #pragma unroll 1
     for (int it = 0; it < n_iters; ++it) {
       const int st = it & (NST - 1);
-      const uint32_t parity = (uint32_t)(it / NST) & 1u;
+      const uint32_t parity = ((uint32_t)(it / NST) + (st == NST - 1 ? (uint32_t)tw : 0u)) & 1u;   // tail tiles used phases of the last barrier
       if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
       const unsigned char* sp = ring + st * SL::kBytes;
       const int ci0 = c_lo + it * CPI;                           // first chunk of this iteration (unit-relative)
@@ -707,7 +721,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     __syncthreads();                                   // every warp is done with its ring
     float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
     const bool writer = SPLIT ? (j == 0) : true;
-    const bool any = n_iters > 0;
+    const bool any = n_iters > 0 || tw > 0;
     if (writer) {
       float* mine = wres + ((size_t)warp * kHeads + (SPLIT ? 0 : j)) * (kD + 2);
 #pragma unroll
@@ -765,24 +779,19 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     float M = -INFINITY;
     for (int s = 0; s < n_parts; ++s) M = fmaxf(M, mw[h * 128 + s]);
     float num = 0.f, den = 0.f;
-    int s = 0;
-    for (; s + 4 <= n_parts; s += 4) {                  // four independent loads in flight
-      float v[4], wgt[4];
+    for (int s0 = 0; s0 < n_parts; s0 += 16) {          // sixteen independent loads in flight
+      float v[16];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) v[e] = __ldcg(P + (size_t)(s + e) * kPartialStride);
+      for (int e = 0; e < 16; ++e) v[e] = s0 + e < n_parts ? __ldcg(P + (size_t)(s0 + e) * kPartialStride) : 0.f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float ms = mw[h * 128 + s + e];
-        wgt[e] = ms == -INFINITY ? 0.f : exp2f(ms - M);
-        num = fmaf(v[e], wgt[e], num);
-        den = fmaf(lw[h * 128 + s + e], wgt[e], den);
+      for (int e = 0; e < 16; ++e) {
+        if (s0 + e < n_parts) {
+          const float ms = mw[h * 128 + s0 + e];
+          const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
+          num = fmaf(v[e], wgt, num);
+          den = fmaf(lw[h * 128 + s0 + e], wgt, den);
+        }
       }
-    }
-    for (; s < n_parts; ++s) {
-      const float ms = mw[h * 128 + s];
-      const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
-      num = fmaf(__ldcg(P + (size_t)s * kPartialStride), wgt, num);
-      den = fmaf(lw[h * 128 + s], wgt, den);
     }
     a.out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
   }
@@ -794,7 +803,7 @@ int g_chunks_per_iter = 0;    // tuning knob: 0 automatic, else 1 or 2 chunks of
 template <int BITS, int G, bool SPLIT, int CPI>
 int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
   using SL = StageLayout<BITS, G, CPI>;
-  constexpr int kSmem = SL::kCtaBytes > (int)sizeof(TailSmem) ? SL::kCtaBytes : (int)sizeof(TailSmem);
+  constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH > CPI ? SL::kCH : CPI;
   static bool configured = false;
   if (!configured) {
@@ -808,9 +817,19 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
   if (n_splits > by_work) n_splits = by_work;
   if (n_units == 0) n_splits = 0;
+  // without packed chunks the CTAs only share the tail tiles (eight per CTA)
+  int grid_y = n_splits > 0 ? n_splits : (a.n_tail_tiles + kWarps - 1) / kWarps;
+  if (grid_y < 1) grid_y = 1;
+  if (grid_y > L.max_splits) grid_y = L.max_splits;
   a.n_splits = n_splits;
-  a.units_per_split = n_splits ? (n_units + n_splits - 1) / n_splits : 0;
-  dim3 grid(L.U, n_splits > 0 ? n_splits : a.n_tail_tiles);
+  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about one loop iteration
+  {
+    const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
+    a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
+  }
+  a.tiles_q0 = a.n_tail_tiles / grid_y;
+  a.tiles_rem = a.n_tail_tiles % grid_y;
+  dim3 grid(L.U, grid_y);
   int launches = 0;
   const int step = SPLIT ? 1 : kHeads;
   for (int h0 = 0; h0 < L.r; h0 += step) {
@@ -842,18 +861,22 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
                       __half* out, int n_splits, cudaStream_t st) {
   if (!decode_mma_supported(L)) return -2;
   const Counts cn = counts_for(L, N);
-  const int n_tail_tiles = (cn.N - cn.n_qv + 31) / 32;
   if (n_splits <= 0) {
     n_splits = (2 * 148) / L.U;                  // two resident CTAs per SM, one wave
     if (n_splits < 1) n_splits = 1;
   }
-  if (n_splits > L.max_splits - n_tail_tiles) n_splits = L.max_splits - n_tail_tiles;
-  if (n_splits < 0 || n_splits + n_tail_tiles > 128) return -2;
+  if (n_splits > L.max_splits) n_splits = L.max_splits;
+  if (n_splits > 128) n_splits = 128;            // slots of the merge tables in shared memory
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
-  a.n_tail_tiles = n_tail_tiles;
+  a.n_skew_tiles = (cn.n_qk - cn.n_qv + 7) / 8;
+  a.n_tail_tiles = a.n_skew_tiles + (cn.n_sink + cn.n_k_recent + 7) / 8;
   a.units_per_split = 0;
+  a.tail_cost_units = 0;
+  a.tiles_q0 = a.tiles_rem = 0;
+  a.k_ring_pos0 = L.k.ring_cap ? cn.n_qk % L.k.ring_cap : 0;
+  a.v_ring_pos0 = L.v.ring_cap ? cn.n_qv % L.v.ring_cap : 0;
   a.head0 = 0;
   const int bits = L.k.bits;
   if (bits == 2 && L.G == 32 && L.r == 1) return launch_cpi<2, 32, true>(L, cn, a, n_splits, st);
