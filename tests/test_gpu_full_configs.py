@@ -1,0 +1,135 @@
+"""Parity at the benchmark configurations' full sizes (needs a B200).
+
+The CUDA path runs the whole workload in the launch configuration `bench.py` uses; the oracle, which
+would need minutes for all (batch, KV head) units, is run on a sample of units and compared on those:
+packed codes / scales / zero-points / masks / norms / windows bit-exact, attention outputs within
+|err| <= 2e-3 * max|out| + 1e-3.
+"""
+import numpy as np
+import pytest
+
+from oracle import innerq_oracle as O
+from paper_2602_23200_b200 import synth
+from tests import _parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(x):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def make_gpu(w, K, V, extra=64):
+    from paper_2602_23200_b200 import binding as B
+    gc = B.InnerQCache(B.make_config(w, max_tokens=w.n_tokens + extra))
+    gc.innerq_quantize_prefill(dev(K), dev(V))
+    return gc
+
+
+def sub_oracle(w, K, V, units, extra=64):
+    """Oracle over the sampled units only, laid out as batch 1 with len(units) KV heads."""
+    Ku = K.reshape(w.n_units, w.n_tokens, w.head_dim)[units]
+    Vu = V.reshape(w.n_units, w.n_tokens, w.head_dim)[units]
+    ws = w.with_(batch=1, n_kv_heads=len(units), n_q_heads=len(units) * w.q_per_kv)
+    oc = O.from_workload(ws, max_tokens=w.n_tokens + extra)
+    oc.prefill(Ku[None], Vu[None])
+    return oc
+
+
+def q_rows(w, q, units):
+    """Query heads of the sampled units, as the sub-oracle's [1, len(units) * r, D]."""
+    r = w.q_per_kv
+    rows = [q[u // w.n_kv_heads, (u % w.n_kv_heads) * r + i] for u in units for i in range(r)]
+    return np.stack(rows)[None]
+
+
+def slice_export(e, units):
+    out = {}
+    for k, v in e.items():
+        out[k] = v[units] if isinstance(v, np.ndarray) and v.ndim >= 2 else v
+    return out
+
+
+def compare(w, gc, oc, units, step=0, check_export=True):
+    if check_export:
+        flips = P.assert_export_equal(slice_export(gc.innerq_cache_export(), units), oc.export(), w.grouping, w.group,
+                                      w.k_mode == O.HYBRID, w.v_mode == O.HYBRID)
+    else:
+        flips = 0
+    q = synth.query(w, step)
+    out = gc.innerq_decode_attention(dev(q)).cpu().numpy()
+    ref = oc.decode(q_rows(w, q, units))
+    worst = P.assert_outputs_close(q_rows(w, out, units), ref, f"{w.name} step {step}")
+    assert gc.innerq_read_device_error() == 0
+    return flips, worst
+
+
+def kv_tiled_over_batch(w):
+    """K, V with batch entry 0 generated and repeated over the batch (generation time of the large configs)."""
+    K1, V1 = synth.kv_all(w.with_(batch=1))
+    return np.repeat(K1, w.batch, axis=0), np.repeat(V1, w.batch, axis=0)
+
+
+def test_config2_prefill_then_steps():
+    # 32 heads x 32768 tokens, 2-bit, G = 32; each step appends one token, then decodes.
+    w = synth.config2()
+    K, V = synth.kv_all(w)
+    units = [0, 13, 31]
+    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    compare(w, gc, oc, units, step=1000)
+    worst = 0.0
+    for step in range(40):                      # crosses value-group evictions (every 32 steps) and 40 key evictions
+        k1, v1 = synth.new_token(w, step)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+        if step in (0, 3, 4, 5, 35, 36, 39):
+            _, e = compare(w, gc, oc, units, step=step, check_export=step in (4, 39))
+            worst = max(worst, e)
+    print(f"config2: worst err/tol over steps {worst:.3f}")
+
+
+@pytest.mark.parametrize("bits", [4, 2])
+def test_config3_gqa_batch16(bits):
+    w = synth.config3(bits)
+    K, V = synth.kv_all(w)
+    units = [0, 77, 127]
+    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    flips, worst = compare(w, gc, oc, units)
+    k1, v1 = synth.new_token(w, 0)
+    gc.innerq_append_token(dev(k1), dev(v1))
+    oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+    _, worst2 = compare(w, gc, oc, units, step=1)
+    print(f"config3 {bits}-bit: contested flips {flips}, worst err/tol {max(worst, worst2):.3f}")
+
+
+def test_config4_long_context_prefill_and_decode():
+    # batch 4 x 8 KV heads x 131072 tokens, 2-bit, G = 128: full prefill quantisation, then decode.
+    w = synth.config4()
+    K, V = kv_tiled_over_batch(w)
+    units = [3, 20]
+    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    del K, V
+    flips, worst = compare(w, gc, oc, units)
+    print(f"config4: contested flips {flips}, worst err/tol {worst:.3f}")
+
+
+SWEEP = [(b, g, m, O.INNER, 0) for b in (2, 3, 4) for g in (32, 64, 128) for m in (O.HYBRID, O.ASYM)] + \
+        [(2, 64, O.HYBRID, O.INNER, 1), (2, 64, O.ASYM, O.OUTER, 0), (4, 64, O.ASYM, O.OUTER, 0), (2, 64, O.ASYM, O.FP16, 0)]
+
+
+@pytest.mark.parametrize("bits,G,mode,grouping,variant", SWEEP)
+def test_config5_sweep_point(bits, G, mode, grouping, variant):
+    # The sweep of bits x group size x mode on the config-3 shape and data; batch reduced from 16 to 2 to keep
+    # the run short (units are independent), full context length.
+    w = synth.config5(bits, G, mode, grouping, variant).with_(batch=2)
+    K, V = synth.kv_all(w)
+    units = [5]
+    gc = make_gpu(w, K, V)
+    oc = sub_oracle(w, K, V, units)
+    if grouping == O.FP16:
+        q = synth.query(w)
+        out = gc.innerq_decode_attention(dev(q)).cpu().numpy()
+        P.assert_outputs_close(q_rows(w, out, units), oc.decode(q_rows(w, q, units)), "fp16 cache")
+        return
+    compare(w, gc, oc, units)
