@@ -89,35 +89,47 @@ def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
 
 
 class ClockSampler(threading.Thread):
-    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and clock-event (throttle) reasons through NVML while the timed region runs.
 
-    def __init__(self, index: int):
+    Read-only queries; nothing about the GPU is changed."""
+    REASONS = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40, "sw_power_cap": 0x4}
+
+    def __init__(self, index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
-        self.index, self.samples, self._stop_evt = index, [], threading.Event()
+        self.index, self.period = index, period_s
+        self.sm, self.mask, self.sm_max = [], 0, None
+        self._stop_evt = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
 
     def run(self):
+        if self._h is None:
+            return
+        nv = self._nv
         while not self._stop_evt.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                f = [x.strip() for x in out.strip().split(",")]
-                if len(f) >= 6:
-                    self.samples.append(f)
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
             except Exception:
-                pass
-            self._stop_evt.wait(0.05)
+                try:
+                    self.mask |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                except Exception:
+                    pass
+            self._stop_evt.wait(self.period)
 
     def stop(self):
         self._stop_evt.set()
-        self.join(timeout=6)
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.samples)}
+        self.join(timeout=2)
+        reasons = [n for n, bit in self.REASONS.items() if self.mask & bit]
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.sm_max,
+                "reasons": reasons, "samples": len(self.sm)}
 
 
 def measured_peak_gbs():
@@ -189,6 +201,22 @@ def config_dict(w, args):
             "w_sink": w.w_sink, "w_recent": w.w_recent, "grouping": ["inner", "outer", "fp16"][w.grouping],
             "step": "innerq_append_token + innerq_decode_attention",
             "l2": f"rotating {args.instances} cache instances (> L2) so every decode streams from HBM"}
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    """Maximum of a per-rank time over all ranks (each rank times its own replica on the device)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_step_per_rank: float, seconds_per_step: float, world: int) -> float:
+    """Weak scaling: every rank runs its own batch of sequences; no data-path collective exists on this path."""
+    return world * bytes_per_step_per_rank / seconds_per_step / 1e9
 
 
 # ------------------------------------------------------------------------------------- CUDA arm
@@ -279,12 +307,9 @@ def run_ours(args, w):
     assert all(caches[r].n_tokens == n_now[r] for r in range(R))
     ms_total = ev0.elapsed_time(ev1)
     dec_ms = [a.elapsed_time(b) for a, b in dec_ev]
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, "cuda")
     ms_step = ms_total / Kst
-    value_gbs = world * (bytes_min / Kst) / (ms_step * 1e-3) / 1e9
+    value_gbs = whole_job_gbs(bytes_min / Kst, ms_step * 1e-3, world)
 
     # end to end: host buffers in, host buffer out, copies inside the timed region
     kh = torch.from_numpy(np.stack([t[0] for t in toks])).pin_memory()
@@ -314,11 +339,8 @@ def run_ours(args, w):
         e2e_bytes += decode_algorithmic_bytes(w, c.n_tokens, sym_k, sym_v)[1]
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / (e2e_steps - 1)
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_gbs = world * (e2e_bytes / (e2e_steps - 1)) / e2e_s / 1e9
+    e2e_s = max_over_ranks(e2e_s, "cuda")
+    e2e_gbs = whole_job_gbs(e2e_bytes / (e2e_steps - 1), e2e_s, world)
     # decode kernel alone, launches back to back (no host work between them), same rotation over instances
     b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     nb = max(16, min(Kst, 64))
@@ -367,7 +389,7 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
