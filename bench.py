@@ -34,6 +34,15 @@ D = 128
 
 
 def workload_by_name(name: str):
+    """c1 .. c4 (c3_4bit / c3_2bit); a suffix "+fp16" or "+outer" selects the comparison cache of the same shape."""
+    if "+" in name:
+        base, variant = name.split("+", 1)
+        w = workload_by_name(base)
+        if variant == "fp16":
+            return w.with_(name=w.name + "+fp16", grouping=synth.FP16, k_normalize=0)
+        if variant == "outer":
+            return w.with_(name=w.name + "+outer", grouping=synth.OUTER, k_normalize=0, k_mode=synth.ASYM, v_mode=synth.ASYM)
+        raise SystemExit(f"unknown variant {variant}")
     if name == "c1":
         return synth.config1()
     if name == "c2":

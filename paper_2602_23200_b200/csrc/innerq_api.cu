@@ -228,7 +228,10 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int n = -2;
-  if (c->opt_variant != 1 && decode_mma_supported(c->L))
+  if (c->opt_variant != 1 && c->L.k.kind == kNone)
+    n = launch_decode_fp16(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                           c->opt_splits, s);
+  else if (c->opt_variant != 1 && decode_mma_supported(c->L))
     n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                           c->opt_splits, s);
   if (n == -2) {
@@ -279,7 +282,10 @@ int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, 
   // the array keeps whatever the previous call (of any cache) left: tickets and the error word must start at zero
   if (cudaMemsetAsync(scratch + c->L.ws_ticket_off, 0, (size_t)(c->L.U + 8) * 4, s) != cudaSuccess) return INNERQ_ERR_CUDA;
   int n = -2;
-  if (c->opt_variant != 1 && decode_mma_supported(c->L))
+  if (c->opt_variant != 1 && c->L.k.kind == kNone)
+    n = launch_decode_fp16(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                           c->opt_splits, s);
+  else if (c->opt_variant != 1 && decode_mma_supported(c->L))
     n = launch_decode_mma(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                           c->opt_splits, s);
   if (n == -2) {

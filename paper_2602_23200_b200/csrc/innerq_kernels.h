@@ -29,6 +29,10 @@ int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned cha
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                       __half* out, int n_splits, cudaStream_t st);
 bool decode_mma_supported(const Layout& L);
+
+// Warp-MMA decode over an unquantised fp16 cache (grouping = FP16).  Returns -2 for other layouts.
+int launch_decode_fp16(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
+                       __half* out, int n_splits, cudaStream_t st);
 void decode_mma_set_chunks_per_iter(int n);   // tuning: 32-token chunks per loop iteration (1 or 2)
 
 }  // namespace iq
