@@ -65,7 +65,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -73,7 +73,7 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
 // same with a zero accumulator input (lets the assembler use the zero register instead of clearing four)
 __device__ __forceinline__ void mma16816_z(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                            uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
       : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
@@ -93,7 +93,7 @@ __device__ __forceinline__ void decode_fast(uint32_t meta, float neg_half, float
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
   return d;
 }
 
@@ -184,7 +184,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
   constexpr int RWL = F::kRowWordsPerLane;
   constexpr int KPW = F::kKstepsPerWindow;
-  constexpr int RU = CH > CPI ? CH : CPI;       // chunks per range unit (whole groups and whole iterations)
+  constexpr int RU = CH;                        // chunks per range unit: one value group
   constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
   static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
   static_assert((NST & (NST - 1)) == 0, "stage count must be a power of two");
@@ -199,6 +199,18 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
   const int n_parts = gridDim.y;
   const bool fast = split < a.n_splits;
+  // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
+  // hundred KB of queued chunk data per SM they would take microseconds to arrive.
+  float q_early[2], n_early[2];
+  {
+    const float* norm_g = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
+      q_early[e] = h < nh ? __half2float(a.q[(size_t)(head_base + h) * kD + c]) : 0.f;
+      n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
+    }
+  }
   constexpr int kTailBytes = 2048 + SL::kOffVCodes;                 // 8 fp16 value rows + a chunk's packed key part
   constexpr int TS = SL::kBytes >= kTailBytes ? 1 : 2;               // ring stages lent to a tail tile
   static_assert(TS * SL::kBytes >= kTailBytes && 2048 + 2048 <= TS * SL::kBytes && NST >= TS, "tail tile must fit");
@@ -225,7 +237,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
                         ? u_lo + n_u
                         : max(wu_lo, u_lo + max(0, min(n_u, ((n_virtual * (warp + 1)) >> 3) - cst * (tw_before + tw))));
   const int c_lo = wu_lo * RU;                                  // first chunk
-  const int n_iters = (wu_hi - wu_lo) * (RU / CPI);
+  const int n_chunks_w = (wu_hi - wu_lo) * RU;                  // chunks of this warp (may be odd when CPI = 2)
+  const int n_iters = (n_chunks_w + CPI - 1) / CPI;
 
   unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
   uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
@@ -313,13 +326,12 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
   float* qg_s = q_raw_s + kHeads * kD;                             // [4][4]
   int* qe_s = reinterpret_cast<int*>(qg_s + kHeads * 4);           // [4] exponent of max|q''|
-  const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-  for (int i = tid; i < kHeads * kD; i += kThreads) {
-    const int h = i >> 7, c = i & (kD - 1);
-    float v = 0.f;
-    if (h < nh) v = __half2float(a.q[(size_t)(head_base + h) * kD + c]) * (L.sm_scale * kLog2e);
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int i = tid + e * kThreads;
+    const float v = q_early[e] * (L.sm_scale * kLog2e);
     q_raw_s[i] = v;
-    q_nrm_s[i] = L.k_normalize ? v * norm[c] : v;
+    q_nrm_s[i] = v * n_early[e];
   }
   __syncthreads();
   if (warp < kHeads) {      // warp h: group sums and max |q''| of head h
@@ -490,12 +502,16 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
       const unsigned char* sp = ring + st * SL::kBytes;
       const int ci0 = c_lo + it * CPI;                           // first chunk of this iteration (unit-relative)
-      const bool last_valid = CPI == 1 || (ci0 + 1 < n_chunks_total);   // odd chunk count: the last half is empty
+      const bool last_valid = CPI == 1 || (it * CPI + 1 < n_chunks_w);   // odd chunk count: the last half is empty
 
       // ---------------- raw scores: CPI * 2 m-tiles of 16 tokens -------------------------------------
       float sc[CPI][2][2];
 #pragma unroll
       for (int cc = 0; cc < CPI; ++cc) {
+        if (cc > 0 && !last_valid) {      // nothing there: this warp's range ends in the middle of the iteration
+          sc[cc][0][0] = sc[cc][0][1] = sc[cc][1][0] = sc[cc][1][1] = -INFINITY;
+          continue;
+        }
         const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc));
         const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
@@ -592,6 +608,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 
 #pragma unroll
       for (int cc = 0; cc < CPI; ++cc) {
+        if (cc > 0 && !last_valid) continue;
         const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffVCodes);
         const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
         const int ci = ci0 + cc;
@@ -804,7 +821,7 @@ template <int BITS, int G, bool SPLIT, int CPI>
 int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
   using SL = StageLayout<BITS, G, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
-  constexpr int RU = SL::kCH > CPI ? SL::kCH : CPI;
+  constexpr int RU = SL::kCH;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G, SPLIT, CPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -822,7 +839,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   if (grid_y < 1) grid_y = 1;
   if (grid_y > L.max_splits) grid_y = L.max_splits;
   a.n_splits = n_splits;
-  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about one loop iteration
+  a.tail_cost_units = n_splits ? (3 / RU > 1 ? 3 / RU : 1) : 0;     // a tail tile costs a warp about three chunks' time
   {
     const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
     a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
