@@ -140,7 +140,7 @@ template <int BITS, int G, int CPI> struct StageLayout {
   static constexpr int kStages = (BITS == 2 ? 4 : 2) / CPI > 1 ? (BITS == 2 ? 4 : 2) / CPI : 2;
   static constexpr int kWarpBytes = kBytes * kStages;
   static constexpr int kSideBytes = 4 * kVMeta;                   // per warp: value metadata of the last 4 groups
-  static constexpr int kTableBytes = 6400;                        // q tables and B fragments of the prologue
+  static constexpr int kTableBytes = 8448;                        // q tables and B fragments of the prologue
   static constexpr int kOffSide = kWarpBytes * kWarps;
   static constexpr int kSideArea = kSideBytes * kWarps > kTableBytes ? kSideBytes * kWarps : kTableBytes;
   static constexpr int kOffBars = kOffSide + kSideArea;
@@ -153,7 +153,7 @@ struct DecodeArgs {
   const __half* q;
   __half* out;
   int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
-  int n_tail_tiles;      // mini-tiles of 8 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
+  int n_tail_tiles;      // tiles of 16 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
                          // tile x belongs to CTA x % gridDim.y, warp (x / gridDim.y) % 8
   int n_skew_tiles;      // of those, tiles whose keys are packed rows (values still fp16)
   int tiles_q0, tiles_rem;   // n_tail_tiles / gridDim.y and n_tail_tiles % gridDim.y
@@ -211,10 +211,6 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
     }
   }
-  constexpr int kTailBytes = 2048 + SL::kOffVCodes;                 // 8 fp16 value rows + a chunk's packed key part
-  constexpr int TS = SL::kBytes >= kTailBytes ? 1 : 2;               // ring stages lent to a tail tile
-  static_assert(TS * SL::kBytes >= kTailBytes && 2048 + 2048 <= TS * SL::kBytes && NST >= TS, "tail tile must fit");
-
   // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
   // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
   // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
@@ -245,7 +241,6 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
   const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
-  unsigned char* tail_buf = ring + (NST - TS) * SL::kBytes;      // [8 value rows][key rows | packed key part]
 
   auto issue = [&](int st, int it) {   // one lane: arm the barrier, start the copy of iteration `it` into stage st
     const int ci = c_lo + it * CPI;
@@ -256,69 +251,41 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
     bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
   };
-  // Tail tile x: up to 8 tokens.  Skew tiles (x < n_skew_tiles): keys are packed rows n_qv + 8x .. of one
-  // chunk record, values fp16 ring rows.  Other tiles: entries of the list [sink tokens, recent key tokens].
+  // Tail tile x: up to 16 tokens outside the range where both K and V are packed.  Skew tiles
+  // (x < n_skew_tiles): keys are packed rows n_qv + 16x .. of one chunk record, values fp16 ring rows.
+  // Other tiles: entries of the list [sink tokens, recent key tokens], keys and values fp16.
   const int n_skew = cn.n_qk - cn.n_qv, n_list = cn.n_sink + cn.n_k_recent;
   auto tail_tile = [&](int k, bool& skew, int& e0, int& cnt) {
     const int x = split + Gy * (warp + kWarps * k);
     skew = x < a.n_skew_tiles;
-    e0 = 8 * (skew ? x : x - a.n_skew_tiles);
-    cnt = min(8, (skew ? n_skew : n_list) - e0);
+    e0 = 16 * (skew ? x : x - a.n_skew_tiles);
+    cnt = min(16, (skew ? n_skew : n_list) - e0);
   };
-  // Rows of consecutive entries are contiguous in memory except where a ring wraps or the list passes from the
-  // sink to the ring: copy maximal runs (typically one 2 KB copy for the values, one for the keys).
-  auto issue_tail = [&](int k) {       // one lane: copy the rows of this warp's k-th tail tile into tail_buf
-    bool skew; int e0, cnt;
-    tail_tile(k, skew, e0, cnt);
-    const uint32_t bar = bars_u32 + 8 * (NST - 1), dst = smem_u32(tail_buf);
-    mbar_expect_tx(bar, (uint32_t)cnt * 256u + (skew ? (uint32_t)SL::kOffVCodes : (uint32_t)cnt * 256u));
-    const unsigned char* v_sink = a.cache + L.v.sink_off + (size_t)u * L.v.sink_stride;
-    const unsigned char* v_ring = a.cache + L.v.ring_off + (size_t)u * L.v.ring_stride;
-    const unsigned char* k_sink = a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride;
-    const unsigned char* k_ring = a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride;
-    // row address of list entry e: sink rows, else ring slot = (first slot + offset) wrapped once
-    auto v_row = [&](int e) -> const unsigned char* {
-      if (!skew && e < cn.n_sink) return v_sink + (size_t)e * 256;
-      int slot = a.v_ring_pos0 + (skew ? e : n_skew + (e - cn.n_sink));
-      if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
-      return v_ring + (size_t)slot * 256;
-    };
-    auto k_row = [&](int e) -> const unsigned char* {
-      if (e < cn.n_sink) return k_sink + (size_t)e * 256;
-      int slot = a.k_ring_pos0 + (e - cn.n_sink);
-      if (slot >= L.k.ring_cap) slot -= L.k.ring_cap;
-      return k_ring + (size_t)slot * 256;
-    };
-    for (int i = 0; i < cnt;) {
-      const unsigned char* src = v_row(e0 + i);
-      int run = 1;
-      while (i + run < cnt && v_row(e0 + i + run) == src + run * 256) ++run;
-      bulk_g2s(dst + i * 256, src, run * 256, bar);
-      i += run;
-    }
-    if (skew) {
-      const int ci = (cn.n_qv + e0) / kChunk;
-      bulk_g2s(dst + 2048, g_rec + (size_t)(ci / CH) * SL::kGroupRec + (size_t)(ci % CH) * SL::kRec, SL::kOffVCodes, bar);
-    } else {
-      for (int i = 0; i < cnt;) {
-        const unsigned char* src = k_row(e0 + i);
-        int run = 1;
-        while (i + run < cnt && k_row(e0 + i + run) == src + run * 256) ++run;
-        bulk_g2s(dst + 2048 + i * 256, src, run * 256, bar);
-        i += run;
-      }
-    }
+  // fp16 row of list entry e: sink rows, else ring slot = (first slot + offset), wrapped once
+  const uint4* v_sink4 = reinterpret_cast<const uint4*>(a.cache + L.v.sink_off + (size_t)u * L.v.sink_stride);
+  const uint4* v_ring4 = reinterpret_cast<const uint4*>(a.cache + L.v.ring_off + (size_t)u * L.v.ring_stride);
+  const uint4* k_sink4 = reinterpret_cast<const uint4*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
+  const uint4* k_ring4 = reinterpret_cast<const uint4*>(a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride);
+  auto v_row = [&](bool skew, int e) -> const uint4* {
+    if (!skew && e < cn.n_sink) return v_sink4 + (size_t)e * 16;
+    int slot = a.v_ring_pos0 + (skew ? e : n_skew + (e - cn.n_sink));
+    if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
+    return v_ring4 + (size_t)slot * 16;
   };
-  const int early_stages = tw > 0 ? NST - TS : NST;              // stages free for packed chunks right away
+  auto k_row = [&](int e) -> const uint4* {
+    if (e < cn.n_sink) return k_sink4 + (size_t)e * 16;
+    int slot = a.k_ring_pos0 + (e - cn.n_sink);
+    if (slot >= L.k.ring_cap) slot -= L.k.ring_cap;
+    return k_ring4 + (size_t)slot * 16;
+  };
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (tw > 0) issue_tail(0);
 #pragma unroll
     for (int s = 0; s < NST; ++s)
-      if (s < early_stages && s < n_iters) issue(s, s);
+      if (s < n_iters) issue(s, s);
   }
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
@@ -335,9 +302,13 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   }
   __syncthreads();
   if (warp < kHeads) {      // warp h: group sums and max |q''| of head h
-    float v[4], am = 0.f;
+    float v[4], am = 0.f, amr = 0.f;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { v[e] = q_nrm_s[warp * kD + e * 32 + lane]; am = fmaxf(am, fabsf(v[e])); }
+    for (int e = 0; e < 4; ++e) {
+      v[e] = q_nrm_s[warp * kD + e * 32 + lane];
+      am = fmaxf(am, fabsf(v[e]));
+      amr = fmaxf(amr, fabsf(q_raw_s[warp * kD + e * 32 + lane]));
+    }
     // channel c = e * 32 + lane belongs to group c / G
     float gs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -345,6 +316,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+      amr = fmaxf(amr, __shfl_xor_sync(0xffffffffu, amr, o));
 #pragma unroll
       for (int g = 0; g < 4; ++g) gs[g] += __shfl_xor_sync(0xffffffffu, gs[g], o);
     }
@@ -354,6 +326,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       int e = 0;
       if (am > 0.f && am < INFINITY) frexpf(am, &e);
       qe_s[warp] = e;     // am < 2^e
+      int er = 0;
+      if (amr > 0.f && amr < INFINITY) frexpf(amr, &er);
+      qe_s[4 + warp] = er;
     }
   }
   __syncthreads();
@@ -365,6 +340,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     // The fragment values depend on (lane, k-step, register) only, not on the warp: warp w computes the
     // k-step-w entries for every lane once, all warps then read their 16 registers from shared memory.
     uint32_t* bq_s = reinterpret_cast<uint32_t*>(qe_s + 16);      // [8 k-steps][2][32 lanes]
+    uint32_t* bqr_s = bq_s + 512;                                  // same for raw q against fp16 key rows
     {
       const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
       const int s = warp;
@@ -379,6 +355,16 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         uint32_t v = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
         if (SPLIT && (s / KS_PER_G) != col_group) v = 0u;
         bq_s[(s * 2 + rr) * 32 + lane] = v;
+      }
+      // raw q'' for fp16 key rows: k rows follow the 16-byte-piece order of a row load (piece tid4 + 4*i holds
+      // the column pairs of k-steps 2i and 2i+1); one head per column pair also in SPLIT (pair 0 only)
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const int c0 = 8 * (j + 4 * (s >> 1)) + 4 * (s & 1) + 2 * rr;
+        const int h = gid >> 1;
+        const float bs = pow2i(14 - qe_s[4 + h]);
+        const uint32_t v0 = split_hi_lo(q_raw_s[h * kD + c0] * bs), v1 = split_hi_lo(q_raw_s[h * kD + c0 + 1] * bs);
+        bqr_s[(s * 2 + rr) * 32 + lane] = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
       }
     }
     __syncthreads();
@@ -401,12 +387,85 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
     }
     const float neg_half = -(float)(1 << (BITS - 1));
-    // SPLIT reuses the table area for its side ring, so it takes what the tail tiles need of q into
-    // registers (one head: 4 channels per lane) and releases the tables now, while all warps are in step.
-    float4 qraw4 = make_float4(0.f, 0.f, 0.f, 0.f), qnrm4 = qraw4;
+    // Raw scores (still carrying 1/kfac) of the 16 packed key rows r0 .. r0+15 of a chunk: this lane's rows are
+    // r0 + gid and r0 + gid + 8.  kc / km: packed rows and metadata rows of the chunk (shared or global memory).
+    auto k_mtile = [&](const uint32_t* kc, const uint32_t* km, int r0, float& sA_out, float& sB_out) {
+      const int rA = r0 + gid, rB = rA + 8;
+      uint32_t wa[RWL], wb[RWL];
+      if constexpr (RWL == 2) {
+        const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
+        const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
+        wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
+      } else {
+        const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
+        const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
+        wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
+        wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
+      }
+      auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
+        const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
+        const int window = sw / KPW, kk = sw % KPW;
+        const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
+        const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
+        const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
+        if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+        else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
+      };
+      float sA, sB;
+      if constexpr (SPLIT) {
+        float c4[4];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
+        float s_, z_;
+        decode_fast(km[rA * NG + j], neg_half, s_, z_);
+        sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
+        decode_fast(km[rB * NG + j], neg_half, s_, z_);
+        sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
+        sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+        sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+        sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+        sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+      } else {
+        uint32_t ma[NG], mb[NG];
+        if constexpr (NG == 4) {
+          const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
+          const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
+          ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
+          mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
+        } else if constexpr (NG == 2) {
+          const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
+          const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
+          ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
+        } else {
+          ma[0] = km[rA]; mb[0] = km[rB];
+        }
+        sA = 0.f; sB = 0.f;
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          float c4[4];
+#pragma unroll
+          for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
+          float s_, z_;
+          decode_fast(ma[g], neg_half, s_, z_);
+          sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
+          decode_fast(mb[g], neg_half, s_, z_);
+          sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
+        }
+      }
+      sA_out = sA;
+      sB_out = sB;
+    };
+
+    // Fragments of raw q'' for the fp16 key rows of this warp's tail tiles (registers only while those run).
+    // SPLIT reuses the table area for its side ring, so the tables are released now, while all warps are in step.
+    uint32_t Bqr[8][2];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      Bqr[s][0] = tw > 0 ? bqr_s[(s * 2) * 32 + lane] : 0u;
+      Bqr[s][1] = tw > 0 ? bqr_s[(s * 2 + 1) * 32 + lane] : 0u;
+    }
+    const float kfac_raw = pow2i(-(14 - qe_s[4 + my_head]));       // fp16 key rows: accumulator * kfac_raw
     if constexpr (SPLIT) {
-      qraw4 = *reinterpret_cast<const float4*>(q_raw_s + 4 * lane);
-      qnrm4 = *reinterpret_cast<const float4*>(q_nrm_s + 4 * lane);
       __syncthreads();
       for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
       __syncwarp();
@@ -423,82 +482,89 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
     bool failed = false;
 
-    // ---------------- tail tiles of this warp: fp16 windows and the K/V skew zone, plain SIMT ---------
-    // (8 tokens at a time, straight into the warp's running soft-max state; no CTA-wide synchronisation)
-    for (int k = 0; k < tw && !failed; ++k) {
+    // ---------------- tail tiles of this warp: fp16 windows and the K/V skew zone -------------------
+    // 16 tokens at a time, operands straight from global memory (coalesced 128-bit loads), into the warp's
+    // running soft-max state.  Keys: fp16 rows against raw q'' (pieces tid4 + 4i of rows gid, gid + 8), or the
+    // packed rows of the skew zone through the same path as the main loop.  Values: fp16 rows, pieces gid and
+    // gid + 8 of token rows 2*tid4, 2*tid4 + 1 (+8), byte-permuted into (channel; token pair) fragments.
+    for (int k = 0; k < tw; ++k) {
       bool skew; int e0, cnt;
       tail_tile(k, skew, e0, cnt);
-      if (!mbar_wait(bars_u32 + 8 * (NST - 1), (uint32_t)k & 1u)) { failed = true; break; }
-      const __half* vbuf = reinterpret_cast<const __half*>(tail_buf);
-      const unsigned char* kbuf = tail_buf + 2048;
-      constexpr int NHT = SPLIT ? 1 : kHeads;
-      float s_mine[8];
+      float sA, sB;                                            // true log2-domain scores of entries e0+gid, e0+gid+8
+      if (skew) {
+        const int iq = cn.n_qv + e0;                           // first packed key row of the tile (16-aligned)
+        const unsigned char* rec = g_rec + (size_t)((iq / kChunk) / CH) * SL::kGroupRec +
+                                   (size_t)((iq / kChunk) % CH) * SL::kRec;
+        k_mtile(reinterpret_cast<const uint32_t*>(rec), reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta),
+                iq % kChunk, sA, sB);
+        sA *= kfac;
+        sB *= kfac;
+      } else {
+        const uint4* ra = k_row(e0 + min(gid, cnt - 1));
+        const uint4* rb = k_row(e0 + min(gid + 8, cnt - 1));
+        uint4 ka[4], kb[4];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        float kx[4];
-        if (!skew) {
-          const uint2 raw = *reinterpret_cast<const uint2*>(kbuf + t * 256 + lane * 8);
-          const __half2* hh = reinterpret_cast<const __half2*>(&raw);
-          const float2 x0 = __half22float2(hh[0]), x1 = __half22float2(hh[1]);
-          kx[0] = x0.x; kx[1] = x0.y; kx[2] = x1.x; kx[3] = x1.y;
-        } else {
-          const int rc = (cn.n_qv + e0 + t) % kChunk;            // row inside the chunk record
-          const uint32_t* row = reinterpret_cast<const uint32_t*>(kbuf + rc * (16 * BITS));
-          float s_, z_;
-          decode_fast(reinterpret_cast<const uint32_t*>(kbuf + SL::kOffKMeta)[rc * NG + (4 * lane) / G], neg_half, s_, z_);
+        for (int i = 0; i < 4; ++i) { ka[i] = __ldg(ra + j + 4 * i); kb[i] = __ldg(rb + j + 4 * i); }
+        float c4[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) kx[e] = fmaf(s_, (float)row_code(row, 4 * lane + e, BITS), z_);
+        for (int i = 0; i < 4; ++i) {
+          if (i == 0) mma16816_z(c4, ka[i].x, kb[i].x, ka[i].y, kb[i].y, Bqr[0][0], Bqr[0][1]);
+          else mma16816(c4, ka[i].x, kb[i].x, ka[i].y, kb[i].y, Bqr[2 * i][0], Bqr[2 * i][1]);
+          mma16816(c4, ka[i].z, kb[i].z, ka[i].w, kb[i].w, Bqr[2 * i + 1][0], Bqr[2 * i + 1][1]);
         }
-        float mine = 0.f;
-#pragma unroll
-        for (int h = 0; h < NHT; ++h) {
-          const float4 qv = SPLIT ? (skew ? qnrm4 : qraw4)
-                                  : *reinterpret_cast<const float4*>((skew ? q_nrm_s : q_raw_s) + h * kD + 4 * lane);
-          float d = fmaf(kx[0], qv.x, fmaf(kx[1], qv.y, fmaf(kx[2], qv.z, kx[3] * qv.w)));
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-          if (h == my_head) mine = d;
+        sA = (c4[0] + c4[1]) * kfac_raw;
+        sB = (c4[2] + c4[3]) * kfac_raw;
+        if constexpr (SPLIT) {       // only column pair 0 carries the head: hand its sums to the whole quad
+          sA = __shfl_sync(0xffffffffu, sA, lane & ~3);
+          sB = __shfl_sync(0xffffffffu, sB, lane & ~3);
         }
-        s_mine[t] = t < cnt ? mine : -INFINITY;
       }
-      float cmax = s_mine[0];
-#pragma unroll
-      for (int t = 1; t < 8; ++t) cmax = fmaxf(cmax, s_mine[t]);
+      if (gid >= cnt) sA = -INFINITY;
+      if (gid + 8 >= cnt) sB = -INFINITY;
+      float cmax = fmaxf(sA, sB);
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
       const float m_new = fmaxf(m_run, cmax);
       const float alpha = ex2_approx(m_run - m_new);            // 0 while m_run = -inf
       m_run = m_new;
       l_part *= alpha;
 #pragma unroll
       for (int m = 0; m < 8; ++m) { out_acc[m][0] *= alpha; out_acc[m][1] *= alpha; }
-      // out_acc is kept in units of 2^-14 (see the packed path); in SPLIT only lane 0 of a quad contributes
-      const float unit = (SPLIT && j != 0) ? 0.f : 0x1p-14f;
+      const float pA = ex2_approx(sA - m_new), pB = ex2_approx(sB - m_new);
+      l_part += pA + pB;
+      uint32_t pkA = split_hi_lo(pA * 1024.f), pkB = split_hi_lo(pB * 1024.f);
+      if (SPLIT && j != 0) { pkA = 0u; pkB = 0u; }              // SPLIT: lane 0 of each quad takes the tail's sums
+      const uint32_t b0 = movmatrix_trans(pkA), b1 = movmatrix_trans(pkB);
+      const uint4* vr[4] = {v_row(skew, e0 + min(2 * j, cnt - 1)), v_row(skew, e0 + min(2 * j + 1, cnt - 1)),
+                            v_row(skew, e0 + min(2 * j + 8, cnt - 1)), v_row(skew, e0 + min(2 * j + 9, cnt - 1))};
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        const float p = ex2_approx(s_mine[t] - m_new);          // 0 for the padding tokens
-        if (t == gid) l_part += p;                              // every token counted once per head
-        if (t < cnt) {
-          const float pu = p * unit;
+      for (int hh = 0; hh < 2; ++hh) {
+        uint4 v4[4];
 #pragma unroll
-          for (int m = 0; m < 8; ++m) {
-            out_acc[m][0] = fmaf(pu, __half2float(vbuf[t * kD + 16 * m + gid]), out_acc[m][0]);
-            out_acc[m][1] = fmaf(pu, __half2float(vbuf[t * kD + 16 * m + 8 + gid]), out_acc[m][1]);
-          }
+        for (int r = 0; r < 4; ++r) v4[r] = __ldg(vr[r] + gid + 8 * hh);
+        const uint32_t* T0 = reinterpret_cast<const uint32_t*>(&v4[0]);
+        const uint32_t* T1 = reinterpret_cast<const uint32_t*>(&v4[1]);
+        const uint32_t* T8 = reinterpret_cast<const uint32_t*>(&v4[2]);
+        const uint32_t* T9 = reinterpret_cast<const uint32_t*>(&v4[3]);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {                        // m-tile 4*hh + kk: channels 64*hh + 8*gid + 2*kk (+1)
+          float c4[4];
+          mma16816_z(c4, __byte_perm(T0[kk], T1[kk], 0x5410), __byte_perm(T0[kk], T1[kk], 0x7632),
+                     __byte_perm(T8[kk], T9[kk], 0x5410), __byte_perm(T8[kk], T9[kk], 0x7632), b0, b1);
+          // out_acc is kept in units of 2^-14; these sums carry p * 2^10
+          out_acc[4 * hh + kk][0] = fmaf(c4[0] + c4[1], 0x1p-24f, out_acc[4 * hh + kk][0]);
+          out_acc[4 * hh + kk][1] = fmaf(c4[2] + c4[3], 0x1p-24f, out_acc[4 * hh + kk][1]);
         }
       }
-      __syncwarp();
-      if (lane == 0 && k + 1 < tw) issue_tail(k + 1);
     }
-    if (tw > 0 && lane == 0) {     // the lent stages go back to the packed stream
-#pragma unroll
-      for (int s = 0; s < NST; ++s)
-        if (s >= early_stages && s < n_iters) issue(s, s);
-    }
+
     // The loop body is deliberately not unrolled over iterations: two CTAs of eight warps walk it at
     // different phases, so it has to stay resident in the instruction cache.
 #pragma unroll 1
     for (int it = 0; it < n_iters; ++it) {
       const int st = it & (NST - 1);
-      const uint32_t parity = ((uint32_t)(it / NST) + (st == NST - 1 ? (uint32_t)tw : 0u)) & 1u;   // tail tiles used phases of the last barrier
+      const uint32_t parity = (uint32_t)(it / NST) & 1u;
       if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
       const unsigned char* sp = ring + st * SL::kBytes;
       const int ci0 = c_lo + it * CPI;                           // first chunk of this iteration (unit-relative)
@@ -516,68 +582,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
-          const int rA = 16 * mt + gid, rB = rA + 8;
-          uint32_t wa[RWL], wb[RWL];
-          if constexpr (RWL == 2) {
-            const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
-            const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
-            wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
-          } else {
-            const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
-            const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
-            wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
-            wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
-          }
-          auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
-            const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
-            const int window = sw / KPW, kk = sw % KPW;
-            const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
-            const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
-            const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
-            if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-            else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-          };
           float sA, sB;
-          if constexpr (SPLIT) {
-            float c4[4];
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
-            float s_, z_;
-            decode_fast(km[rA * NG + j], neg_half, s_, z_);
-            sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
-            decode_fast(km[rB * NG + j], neg_half, s_, z_);
-            sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
-            sA += __shfl_xor_sync(0xffffffffu, sA, 1);
-            sB += __shfl_xor_sync(0xffffffffu, sB, 1);
-            sA += __shfl_xor_sync(0xffffffffu, sA, 2);
-            sB += __shfl_xor_sync(0xffffffffu, sB, 2);
-          } else {
-            uint32_t ma[NG], mb[NG];
-            if constexpr (NG == 4) {
-              const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
-              const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
-              ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
-              mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
-            } else if constexpr (NG == 2) {
-              const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
-              const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
-              ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
-            } else {
-              ma[0] = km[rA]; mb[0] = km[rB];
-            }
-            sA = 0.f; sB = 0.f;
-#pragma unroll
-            for (int g = 0; g < NG; ++g) {
-              float c4[4];
-#pragma unroll
-              for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
-              float s_, z_;
-              decode_fast(ma[g], neg_half, s_, z_);
-              sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
-              decode_fast(mb[g], neg_half, s_, z_);
-              sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
-            }
-          }
+          k_mtile(kc, km, 16 * mt, sA, sB);
           const bool valid = cc == 0 || last_valid;
           sc[cc][mt][0] = valid ? sA : -INFINITY;
           sc[cc][mt][1] = valid ? sB : -INFINITY;
@@ -743,8 +749,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       float* mine = wres + ((size_t)warp * kHeads + (SPLIT ? 0 : j)) * (kD + 2);
 #pragma unroll
       for (int m = 0; m < 8; ++m) {
-        mine[16 * m + gid] = any ? out_acc[m][0] * 0x1p14f : 0.f;
-        mine[16 * m + 8 + gid] = any ? out_acc[m][1] * 0x1p14f : 0.f;
+        mine[block_row_channel(m, 0, gid)] = any ? out_acc[m][0] * 0x1p14f : 0.f;
+        mine[block_row_channel(m, 1, gid)] = any ? out_acc[m][1] * 0x1p14f : 0.f;
       }
       if (gid == 0) {
         mine[kD] = any ? m_run : -INFINITY;
@@ -839,7 +845,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   if (grid_y < 1) grid_y = 1;
   if (grid_y > L.max_splits) grid_y = L.max_splits;
   a.n_splits = n_splits;
-  a.tail_cost_units = n_splits ? (3 / RU > 1 ? 3 / RU : 1) : 0;     // a tail tile costs a warp about three chunks' time
+  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about as much as one value group's chunks
   {
     const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
     a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
@@ -887,8 +893,8 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
-  a.n_skew_tiles = (cn.n_qk - cn.n_qv + 7) / 8;
-  a.n_tail_tiles = a.n_skew_tiles + (cn.n_sink + cn.n_k_recent + 7) / 8;
+  a.n_skew_tiles = (cn.n_qk - cn.n_qv + 15) / 16;
+  a.n_tail_tiles = a.n_skew_tiles + (cn.n_sink + cn.n_k_recent + 15) / 16;
   a.units_per_split = 0;
   a.tail_cost_units = 0;
   a.tiles_q0 = a.tiles_rem = 0;

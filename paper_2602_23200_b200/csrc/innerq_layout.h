@@ -140,11 +140,14 @@ IQ_HD BitPos row_pos_plane(int c, int plane_bits) {
 }
 
 // BLOCK store: position of (token tau in 0..31, channel c) inside a chunk.
-//   PV mma: row = channel, k = token.  m = c / 16 is the m-tile, gid = c % 8, rh = (c / 8) % 2 the
-//   upper row half; ks = tau / 16 the k-step, kh = (tau / 8) % 2, tid4 = (tau % 8) / 2, tp = tau % 2.
+//   PV mma: row = channel, k = token.  ks = tau / 16 is the k-step, kh = (tau / 8) % 2, tid4 = (tau % 8) / 2,
+//   tp = tau % 2.  Channels are dealt to fragment rows so that the 16 channels a lane owns are two
+//   contiguous runs of 8 (c = 64*h + 8*gid + 2*k + rh): the same ownership an unquantised fp16 value row
+//   gives when a lane loads its 16-byte pieces gid and gid + 8, so fp16 window tokens and packed tokens
+//   accumulate into the same registers.  m-tile m = 4*h + k, rh = upper row half.
 IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
   int ks = tau >> 4, kh = (tau >> 3) & 1, j = (tau & 7) >> 1, tp = tau & 1;
-  int m = c >> 4, gid = c & 7, rh = (c >> 3) & 1;
+  int m = 4 * (c >> 6) + ((c >> 1) & 3), gid = (c >> 3) & 7, rh = c & 1;
   int lane = 4 * gid + j;
   BitPos p;
   if (plane_bits == 2) {         // 8 words per lane: word = m; fields (rh, ks, kh)
@@ -161,9 +164,11 @@ IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
 }
 
 // BLOCK store metadata: the 128 per-channel entries of a group are ordered so that the 16 channels a
-// lane owns in the PV fragments (channel = 16*m + 8*rh + gid) are contiguous: 4 x 128-bit loads.
-IQ_HD int block_meta_index(int c) { return (c & 7) * 16 + (c >> 3); }
-IQ_HD int block_meta_channel(int pos) { return (pos & 15) * 8 + (pos >> 4); }
+// lane owns in the PV fragments are contiguous (entry 2*m + rh of lane gid): 4 x 128-bit loads.
+IQ_HD int block_meta_index(int c) { return ((c >> 3) & 7) * 16 + (c >> 6) * 8 + (c & 7); }
+IQ_HD int block_meta_channel(int pos) { return ((pos >> 3) & 1) * 64 + (pos >> 4) * 8 + (pos & 7); }
+// channel of fragment row (m-tile m, row half rh) of lane group gid
+IQ_HD int block_row_channel(int m, int rh, int gid) { return 64 * (m >> 2) + 8 * gid + 2 * (m & 3) + rh; }
 
 IQ_HD int row_bytes(int bits) { return 16 * bits; }
 IQ_HD int chunk_bytes(int bits) { return 512 * bits; }
