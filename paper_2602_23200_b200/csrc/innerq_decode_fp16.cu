@@ -223,9 +223,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fp16_kernel(const Layout L
   }
 
   // ---- cross-CTA merge by the last CTA of the unit to arrive
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's fence below
+  if (tid == 0) {
+    __threadfence();               // cumulative: publishes the whole CTA's partial before the ticket is taken
+    s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+  }
   __syncthreads();
   if (s_ticket != gridDim.y - 1) return;
   __threadfence();

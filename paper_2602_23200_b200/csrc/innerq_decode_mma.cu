@@ -780,9 +780,11 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 
   // ---------------- cross-CTA merge: the last CTA of the unit to arrive combines all parts -----------
   __shared__ unsigned int s_ticket;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's fence below
+  if (tid == 0) {
+    __threadfence();               // cumulative: publishes the whole CTA's partial before the ticket is taken
+    s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+  }
   __syncthreads();
   if (s_ticket != gridDim.y - 1) return;
   __threadfence();
