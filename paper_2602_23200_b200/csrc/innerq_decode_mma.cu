@@ -242,14 +242,17 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
 
-  auto issue = [&](int st, int it) {   // one lane: arm the barrier, start the copy of iteration `it` into stage st
-    const int ci = c_lo + it * CPI;
-    const unsigned char* src = g_rec + (size_t)(ci / CH) * SL::kGroupRec + (size_t)(ci % CH) * SL::kRec;
+  // Copies of consecutive iterations read consecutive byte ranges of the record area: keep a running source.
+  const unsigned char* nx_src = g_rec + (size_t)(c_lo / CH) * SL::kGroupRec + (size_t)(c_lo % CH) * SL::kRec;
+  int nx_ci = c_lo;
+  auto issue = [&](int st) {   // one lane: arm the barrier, start the copy of the next iteration into stage st
     // the value group's scale/zero words sit right behind its last chunk
-    const int n_meta = CPI >= CH ? CPI / CH : (((ci + CPI) % CH) == 0 ? 1 : 0);
+    const int n_meta = CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0);
     const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
-    bulk_g2s(ring_u32 + st * SL::kBytes, src, bytes, bars_u32 + 8 * st);
+    bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes, bars_u32 + 8 * st);
+    nx_src += bytes;
+    nx_ci += CPI;
   };
   // Tail tile x: up to 16 tokens outside the range where both K and V are packed.  Skew tiles
   // (x < n_skew_tiles): keys are packed rows n_qv + 16x .. of one chunk record, values fp16 ring rows.
@@ -285,7 +288,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 #pragma unroll
     for (int s = 0; s < NST; ++s)
-      if (s < n_iters) issue(s, s);
+      if (s < n_iters) issue(s);
   }
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
@@ -639,7 +642,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
             const float p = ex2_approx(fmaf(sc[cc][mt][h], kfac, -m_new));
             psum_c += p;
             const int pos = BITS == 2 ? 2 * mt + h : h;
-            uint32_t pk = split_hi_lo(p * pow2i(10 - BITS * pos));
+            // p goes in as one fp16 (the lo column stays zero): its 2^-12 relative rounding is random per token and
+            // far inside the output tolerance, and it saves the hi/lo split of every probability
+            uint32_t pk = (uint32_t)__half_as_ushort(__float2half_rn(p * pow2i(10 - BITS * pos)));
             if (SPLIT && j != slot) pk = 0u;                 // column pair of this chunk's window slot only
             Bp[mt][h] = movmatrix_trans(pk);
           }
@@ -715,7 +720,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       }
 
       __syncwarp();
-      if (lane == 0 && it + NST < n_iters) issue(st, it + NST);
+      if (lane == 0 && it + NST < n_iters) issue(st);
     }
 
     if (failed) {
