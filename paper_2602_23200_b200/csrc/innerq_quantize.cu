@@ -56,7 +56,8 @@ __global__ void fill_float_kernel(float* p, float v, int n) {
 // ------------------------------------------------------------------ ROW store quantiser
 // One warp quantises one token: lane l holds channels 4l..4l+3; a group of G channels is G/4
 // adjacent lanes.  `stage` is this warp's zero-initialised packed row in shared memory.
-__device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src, const float* __restrict__ norm,
+// `inv_norm4`: reciprocal key norms of this lane's four channels (1.0f / norm, correctly rounded), or null.
+__device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src, const float* __restrict__ inv_norm4,
                                                   const Layout& L, const Store& S, uint32_t* stage,
                                                   uint32_t* __restrict__ dst_row, void* __restrict__ dst_meta, size_t meta_idx) {
   const int lane = threadIdx.x & 31;
@@ -68,9 +69,9 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
     float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
     x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
   }
-  if (norm) {
+  if (inv_norm4) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) x[i] = __fmul_rn(x[i], __fdiv_rn(1.0f, norm[4 * lane + i]));
+    for (int i = 0; i < 4; ++i) x[i] = __fmul_rn(x[i], inv_norm4[i]);
   }
   float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
   float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
@@ -114,12 +115,15 @@ __global__ void __launch_bounds__(128) quantize_rows_kernel(Layout L, Store S, c
                                                             bool use_norm) {
   __shared__ uint32_t stage[4][16];
   const int u = blockIdx.y, warp = threadIdx.x >> 5;
-  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
+  const float* norm = reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD;
+  float inv4[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) inv4[i] = use_norm ? __fdiv_rn(1.0f, norm[4 * (threadIdx.x & 31) + i]) : 1.0f;
   unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4) {
     const __half* src = X + ((size_t)u * N + L.w_sink + i) * kD;
-    quantize_row_warp(src, norm, L, S, stage[warp], reinterpret_cast<uint32_t*>(rec + row_code_off(S, i)),
-                      rec + row_meta_off(S, i), 0);
+    quantize_row_warp(src, use_norm ? inv4 : nullptr, L, S, stage[warp],
+                      reinterpret_cast<uint32_t*>(rec + row_code_off(S, i)), rec + row_meta_off(S, i), 0);
   }
 }
 
@@ -227,9 +231,13 @@ __device__ void append_store(const Layout& L, const Store& S, const __half* __re
   unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
   TokSrc src{ring, S.ring_cap, L.w_sink};
   if (S.kind == kRow) {
-    if (threadIdx.x < 32)
-      quantize_row_warp(src.row(L.w_sink + nq_before), norm, L, S, words,
+    if (threadIdx.x < 32) {
+      float inv4[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) inv4[i] = norm ? __fdiv_rn(1.0f, norm[4 * threadIdx.x + i]) : 1.0f;
+      quantize_row_warp(src.row(L.w_sink + nq_before), norm ? inv4 : nullptr, L, S, words,
                         reinterpret_cast<uint32_t*>(rec + row_code_off(S, nq_before)), rec + row_meta_off(S, nq_before), 0);
+    }
   } else {
     quantize_block_cta(src, L.w_sink + nq_before, norm, L, S, tile, words, rec, nq_before / L.G);
   }
