@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libinnerq.so")
-SOURCES = ["innerq_api.cu", "innerq_quantize.cu", "innerq_decode_simt.cu", "innerq_decode_mma.cu", "innerq_decode_fp16.cu"]
+# every .cu of csrc/: the C ABI, the quantise kernels, the decode kernels (the fused kernel one file per packed format)
+SOURCES = sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 NVCC_FLAGS = [*ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 

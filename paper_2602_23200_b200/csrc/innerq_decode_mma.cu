@@ -1,895 +1,44 @@
-// Fused decode attention over the packed InnerQ cache (INNER layout), one launch:
-//   q.K^T on packed key rows  ->  online softmax  ->  p.V on packed value chunks, split over token
-//   ranges, fp16 windows and the K/V skew zone in a tail CTA, cross-CTA merge by the last CTA to finish.
-//
-// Work decomposition.  A CTA owns one (batch, KV head) unit and a range of value groups; each of its
-// 8 warps owns a contiguous sub-range and streams it chunk by chunk (32 tokens) through a private ring
-// of shared-memory stages filled by 1-D bulk async copies (cp.async.bulk + mbarrier): packed key rows,
-// key scale/zero words, the packed value chunk and, at the end of each value group, its scale/zero
-// words.  The warp never synchronises with other warps until the final merge.
-//
-// Arithmetic.  Codes are never dequantised element by element.  Inner-dimension grouping lets scale and
-// zero-point leave the inner sum (Section "InnerQ": one scale per group, reused):
-//     q'.x^_t = sum_g ( S_tg * sum_{c in g} q'_c u_tc  +  z_tg * sum_{c in g} q'_c )
-//     sum_t p_t v^_tc = sum_j ( S_jc * sum_{t in j} p_t u_tc  +  z_jc * sum_{t in j} p_t )
-// The raw-code sums run on the tensor pipe (mma.sync m16n8k16, fp32 accumulate) so that the ALU pipe only
-// unpacks: `word & (field << pos)` is already an fp16 pair (two codes as subnormals scaled by 2^pos,
-// the scale folded into the other operand).  The other operand (q' or p) is split into fp16 hi + lo
-// columns, so the products carry fp32-level accuracy; up to 4 query heads of the KV head share one pass
-// over the codes (the 8 mma columns are 4 heads x {hi, lo}).  Scale and zero-point are then applied once
-// per (token, group) for keys and once per (group, channel) for values, in fp32.
-#include "innerq_device.cuh"
+// Host side of the fused decode kernel over the packed InnerQ cache: picks the kernel family of the cache's
+// packed format and fills the launch parameters.  The kernels are in innerq_decode_mma.cuh and are compiled
+// one translation unit per format (innerq_decode_mma_k*v*_m*.cu).
+#include "innerq_decode_mma.h"
 #include "innerq_kernels.h"
 
 namespace iq {
 
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kHeads = 4;              // query heads per pass (hi/lo columns: 8 mma columns)
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr uint32_t kWaitLimit = 1u << 22;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-// Bounded wait: gives up after kWaitLimit polls and reports it (the caller records an error and
-// skips the data instead of spinning forever).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// same with a zero accumulator input (lets the assembler use the zero register instead of clearing four)
-__device__ __forceinline__ void mma16816_z(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                           uint32_t b1) {
-  asm(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// Decoder parameters from a metadata word (fp16 scale with the mask in its sign bit | fp16 zero << 16):
-// s = |scale|, z = Z if the mask is set (scale <= -0), else -s * 2^(b-1) (Z is stored as 0 then).
-__device__ __forceinline__ void decode_fast(uint32_t meta, float neg_half, float& s, float& z) {
-  const __half2 h = *reinterpret_cast<const __half2*>(&meta);
-  const float sg = __low2float(h), Z = __high2float(h);
-  s = fabsf(sg);
-  z = fmaf(neg_half, fmaxf(sg, 0.f), Z);
-}
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
-  uint32_t d;
-  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-  return d;
-}
-
-// fp16 hi / lo split of x, packed (hi in the low half-word, lo in the high half-word)
-__device__ __forceinline__ uint32_t split_hi_lo(float x) {
-  const __half hi = __float2half_rn(x);
-  const __half lo = __float2half_rn(x - __half2float(hi));
-  return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
-}
-__device__ __forceinline__ float pow2i(int e) { return __int_as_float((e + 127) << 23); }   // 2^e, -126 <= e <= 127
-
-// Per bit-width constants of the packed formats (see innerq_layout.h).
-template <int BITS> struct Fmt;
-template <> struct Fmt<2> {
-  static constexpr uint32_t kField = 0x00030003u;
-  static constexpr int kKstepsPerWindow = 2;   // an 8-bit window of each half-word feeds 2 key k-steps
-  static constexpr int kRowWordsPerLane = 2;
-  static constexpr int kChunkWordsPerLane = 8;
-};
-template <> struct Fmt<4> {
-  static constexpr uint32_t kField = 0x000F000Fu;
-  static constexpr int kKstepsPerWindow = 1;
-  static constexpr int kRowWordsPerLane = 4;
-  static constexpr int kChunkWordsPerLane = 16;
-};
-
-// Shared-memory stage = the byte range of CPI consecutive chunk records as it lies in HBM (value metadata
-// follows the last chunk of each value group), fetched with one bulk copy.
-template <int BITS, int G, int CPI> struct StageLayout {
-  static constexpr int kNG = kD / G;
-  static constexpr int kCH = G / kChunk;                          // chunks per value group
-  static constexpr int kKCodes = kChunk * 16 * BITS;
-  static constexpr int kKMeta = kChunk * kNG * 4;
-  static constexpr int kVCodes = 512 * BITS;
-  static constexpr int kVMeta = kD * 4;
-  static constexpr int kOffKMeta = kKCodes;
-  static constexpr int kOffVCodes = kOffKMeta + kKMeta;
-  static constexpr int kRec = kOffVCodes + kVCodes;               // bytes of one chunk record
-  static constexpr int kGroupRec = kCH * kRec + kVMeta;           // bytes of one group record
-  // offset of chunk cc of an iteration inside the stage (iterations start on a group boundary or, when a
-  // group spans several iterations, inside one group)
-  __host__ __device__ static constexpr int off(int cc) { return cc * kRec + (cc / kCH) * kVMeta; }
-  static constexpr int kBytes = CPI * kRec + (CPI / kCH > 0 ? CPI / kCH : 1) * kVMeta;
-  static constexpr int kStages = (BITS == 2 ? 4 : 2) / CPI > 1 ? (BITS == 2 ? 4 : 2) / CPI : 2;
-  static constexpr int kWarpBytes = kBytes * kStages;
-  static constexpr int kSideBytes = 4 * kVMeta;                   // per warp: value metadata of the last 4 groups
-  static constexpr int kTableBytes = 8448;                        // q tables and B fragments of the prologue
-  static constexpr int kOffSide = kWarpBytes * kWarps;
-  static constexpr int kSideArea = kSideBytes * kWarps > kTableBytes ? kSideBytes * kWarps : kTableBytes;
-  static constexpr int kOffBars = kOffSide + kSideArea;
-  static constexpr int kCtaBytes = kOffBars + 256;
-};
-
-struct DecodeArgs {
-  const unsigned char* cache;
-  unsigned char* ws;
-  const __half* q;
-  __half* out;
-  int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
-  int n_tail_tiles;      // tiles of 16 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
-                         // tile x belongs to CTA x % gridDim.y, warp (x / gridDim.y) % 8
-  int n_skew_tiles;      // of those, tiles whose keys are packed rows (values still fp16)
-  int tiles_q0, tiles_rem;   // n_tail_tiles / gridDim.y and n_tail_tiles % gridDim.y
-  int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
-  int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
-  int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
-  int head0;             // first query head (within the KV head's r) handled by this launch
-};
-
-// ---- the kernel -------------------------------------------------------------------------------------
-// CPI = chunks (of 32 tokens) a warp processes per loop iteration: one barrier wait, one soft-max update and
-// one refill per iteration, and CPI*2 independent key accumulator chains in flight.
-// SPLIT (one query head per KV head, G = 32): the 8 mma columns are not 4 heads x {hi, lo} but
-// 4 groups x {hi, lo}: for keys, column pair g holds q'' restricted to channel group g, so one accumulator
-// chain over all 8 k-steps yields the four per-group code sums at once and lane j of each quad applies the
-// scale / zero-point of group j only (then the quad adds up); for values, column pair w holds p
-// restricted to the w-th value group of a window of four, and lane j applies group j's metadata once per
-// window.  This removes the 4x redundancy a quad otherwise has in decoding per-group metadata.
-template <int BITS, int G, bool SPLIT, int CPI>
-__global__ void __launch_bounds__(kThreads, 2)
-decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  using F = Fmt<BITS>;
-  using SL = StageLayout<BITS, G, CPI>;
-  constexpr int NG = SL::kNG;                   // key groups per token
-  constexpr int KS_PER_G = G / 16;              // key k-steps per group
-  constexpr int CH = SL::kCH;                   // chunks per value group
-  constexpr int NST = SL::kStages;
-  constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
-  constexpr int RWL = F::kRowWordsPerLane;
-  constexpr int KPW = F::kKstepsPerWindow;
-  constexpr int RU = CH;                        // chunks per range unit: one value group
-  constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
-  static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
-  static_assert((NST & (NST - 1)) == 0, "stage count must be a power of two");
-  static_assert(CPI == 1 || CPI == 2, "one or two chunks per iteration");
-
-  extern __shared__ __align__(128) unsigned char smem[];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gid = lane >> 2, j = lane & 3;
-  const int u = blockIdx.x, split = blockIdx.y;
-  const int b = u / L.Hkv, hkv = u % L.Hkv;
-  const int nh = min(SPLIT ? 1 : kHeads, L.r - a.head0);
-  const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
-  const int n_parts = gridDim.y;
-  const bool fast = split < a.n_splits;
-  // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
-  // hundred KB of queued chunk data per SM they would take microseconds to arrive.
-  float q_early[2], n_early[2];
-  {
-    const float* norm_g = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
-      q_early[e] = h < nh ? __half2float(a.q[(size_t)(head_base + h) * kD + c]) : 0.f;
-      n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
-    }
-  }
-  // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
-  // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
-  // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
-  const int Gy = gridDim.y, cst = a.tail_cost_units;
-  const int n_chunks_total = cn.n_qv / kChunk;
-  const int n_units_total = (n_chunks_total + RU - 1) / RU;
-  const int q_cta = a.tiles_q0 + (split < a.tiles_rem ? 1 : 0);                 // tail tiles of this CTA
-  const int tiles_before = split * a.tiles_q0 + min(split, a.tiles_rem);         // ... of the CTAs before it
-  auto tiles_of_warp = [&](int q, int w) { return (q >> 3) + (w < (q & 7) ? 1 : 0); };
-  const int u_lo = max(0, min(n_units_total, split * a.units_per_split - cst * tiles_before));
-  const int u_hi = split == a.n_splits - 1
-                       ? n_units_total
-                       : max(u_lo, min(n_units_total, (split + 1) * a.units_per_split - cst * (tiles_before + q_cta)));
-  const int n_u = fast ? u_hi - u_lo : 0;
-  const int n_virtual = n_u + cst * q_cta;
-  const int tw_before = warp * (q_cta >> 3) + min(warp, q_cta & 7);
-  const int tw = tiles_of_warp(q_cta, warp);                        // tail tiles of this warp
-  const int wu_lo = u_lo + max(0, min(n_u, ((n_virtual * warp) >> 3) - cst * tw_before));
-  const int wu_hi = warp == kWarps - 1
-                        ? u_lo + n_u
-                        : max(wu_lo, u_lo + max(0, min(n_u, ((n_virtual * (warp + 1)) >> 3) - cst * (tw_before + tw))));
-  const int c_lo = wu_lo * RU;                                  // first chunk
-  const int n_chunks_w = (wu_hi - wu_lo) * RU;                  // chunks of this warp (may be odd when CPI = 2)
-  const int n_iters = (n_chunks_w + CPI - 1) / CPI;
-
-  unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
-  uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
-  const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
-  const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
-
-  // Copies of consecutive iterations read consecutive byte ranges of the record area: keep a running source.
-  const unsigned char* nx_src = g_rec + (size_t)(c_lo / CH) * SL::kGroupRec + (size_t)(c_lo % CH) * SL::kRec;
-  int nx_ci = c_lo;
-  auto issue = [&](int st) {   // one lane: arm the barrier, start the copy of the next iteration into stage st
-    // the value group's scale/zero words sit right behind its last chunk
-    const int n_meta = CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0);
-    const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
-    mbar_expect_tx(bars_u32 + 8 * st, bytes);
-    bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes, bars_u32 + 8 * st);
-    nx_src += bytes;
-    nx_ci += CPI;
-  };
-  // Tail tile x: up to 16 tokens outside the range where both K and V are packed.  Skew tiles
-  // (x < n_skew_tiles): keys are packed rows n_qv + 16x .. of one chunk record, values fp16 ring rows.
-  // Other tiles: entries of the list [sink tokens, recent key tokens], keys and values fp16.
-  const int n_skew = cn.n_qk - cn.n_qv, n_list = cn.n_sink + cn.n_k_recent;
-  auto tail_tile = [&](int k, bool& skew, int& e0, int& cnt) {
-    const int x = split + Gy * (warp + kWarps * k);
-    skew = x < a.n_skew_tiles;
-    e0 = 16 * (skew ? x : x - a.n_skew_tiles);
-    cnt = min(16, (skew ? n_skew : n_list) - e0);
-  };
-  // fp16 row of list entry e: sink rows, else ring slot = (first slot + offset), wrapped once
-  const uint4* v_sink4 = reinterpret_cast<const uint4*>(a.cache + L.v.sink_off + (size_t)u * L.v.sink_stride);
-  const uint4* v_ring4 = reinterpret_cast<const uint4*>(a.cache + L.v.ring_off + (size_t)u * L.v.ring_stride);
-  const uint4* k_sink4 = reinterpret_cast<const uint4*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
-  const uint4* k_ring4 = reinterpret_cast<const uint4*>(a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride);
-  auto v_row = [&](bool skew, int e) -> const uint4* {
-    if (!skew && e < cn.n_sink) return v_sink4 + (size_t)e * 16;
-    int slot = a.v_ring_pos0 + (skew ? e : n_skew + (e - cn.n_sink));
-    if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
-    return v_ring4 + (size_t)slot * 16;
-  };
-  auto k_row = [&](int e) -> const uint4* {
-    if (e < cn.n_sink) return k_sink4 + (size_t)e * 16;
-    int slot = a.k_ring_pos0 + (e - cn.n_sink);
-    if (slot >= L.k.ring_cap) slot -= L.k.ring_cap;
-    return k_ring4 + (size_t)slot * 16;
-  };
-  if (lane == 0) {
-#pragma unroll
-    for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-#pragma unroll
-    for (int s = 0; s < NST; ++s)
-      if (s < n_iters) issue(s);
-  }
-
-  // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
-  float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
-  float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
-  float* qg_s = q_raw_s + kHeads * kD;                             // [4][4]
-  int* qe_s = reinterpret_cast<int*>(qg_s + kHeads * 4);           // [4] exponent of max|q''|
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const int i = tid + e * kThreads;
-    const float v = q_early[e] * (L.sm_scale * kLog2e);
-    q_raw_s[i] = v;
-    q_nrm_s[i] = v * n_early[e];
-  }
-  __syncthreads();
-  if (warp < kHeads) {      // warp h: group sums and max |q''| of head h
-    float v[4], am = 0.f, amr = 0.f;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      v[e] = q_nrm_s[warp * kD + e * 32 + lane];
-      am = fmaxf(am, fabsf(v[e]));
-      amr = fmaxf(amr, fabsf(q_raw_s[warp * kD + e * 32 + lane]));
-    }
-    // channel c = e * 32 + lane belongs to group c / G
-    float gs[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) gs[(e * 32) / G] += v[e];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
-      amr = fmaxf(amr, __shfl_xor_sync(0xffffffffu, amr, o));
-#pragma unroll
-      for (int g = 0; g < 4; ++g) gs[g] += __shfl_xor_sync(0xffffffffu, gs[g], o);
-    }
-    if (lane == 0) {
-#pragma unroll
-      for (int g = 0; g < 4; ++g) qg_s[warp * 4 + g] = gs[g];
-      int e = 0;
-      if (am > 0.f && am < INFINITY) frexpf(am, &e);
-      qe_s[warp] = e;     // am < 2^e
-      int er = 0;
-      if (amr > 0.f && amr < INFINITY) frexpf(amr, &er);
-      qe_s[4 + warp] = er;
-    }
-  }
-  __syncthreads();
-
-  {
-    // ======================= fast path: packed keys and values ===================================
-    // ---- per-thread constants.  As owner of B-fragment column gid: (head, hi|lo) or, in SPLIT, (group, hi|lo).
-    const int col_head = SPLIT ? 0 : (gid >> 1), col_group = gid >> 1, col_part = gid & 1;
-    // The fragment values depend on (lane, k-step, register) only, not on the warp: warp w computes the
-    // k-step-w entries for every lane once, all warps then read their 16 registers from shared memory.
-    uint32_t* bq_s = reinterpret_cast<uint32_t*>(qe_s + 16);      // [8 k-steps][2][32 lanes]
-    uint32_t* bqr_s = bq_s + 512;                                  // same for raw q against fp16 key rows
-    {
-      const float bscale = pow2i(14 - qe_s[col_head]);   // |q''| * bscale < 2^14
-      const int s = warp;
-      const int kk = (s % (2 * KPW)) % KPW;
-#pragma unroll
-      for (int rr = 0; rr < 2; ++rr) {
-        const int pos = 2 * kk + rr;
-        const float scl = bscale * pow2i(-BITS * pos);
-        const int c0 = 16 * s + 2 * j + 8 * rr;
-        const uint32_t v0 = split_hi_lo(q_nrm_s[col_head * kD + c0] * scl);
-        const uint32_t v1 = split_hi_lo(q_nrm_s[col_head * kD + c0 + 1] * scl);
-        uint32_t v = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
-        if (SPLIT && (s / KS_PER_G) != col_group) v = 0u;
-        bq_s[(s * 2 + rr) * 32 + lane] = v;
-      }
-      // raw q'' for fp16 key rows: k rows follow the 16-byte-piece order of a row load (piece tid4 + 4*i holds
-      // the column pairs of k-steps 2i and 2i+1); one head per column pair also in SPLIT (pair 0 only)
-#pragma unroll
-      for (int rr = 0; rr < 2; ++rr) {
-        const int c0 = 8 * (j + 4 * (s >> 1)) + 4 * (s & 1) + 2 * rr;
-        const int h = gid >> 1;
-        const float bs = pow2i(14 - qe_s[4 + h]);
-        const uint32_t v0 = split_hi_lo(q_raw_s[h * kD + c0] * bs), v1 = split_hi_lo(q_raw_s[h * kD + c0 + 1] * bs);
-        bqr_s[(s * 2 + rr) * 32 + lane] = col_part ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
-      }
-    }
-    __syncthreads();
-    uint32_t Bq[8][2];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      Bq[s][0] = bq_s[(s * 2) * 32 + lane];
-      Bq[s][1] = bq_s[(s * 2 + 1) * 32 + lane];
-    }
-    // ---- as owner of C-fragment columns 2j, 2j+1: head j, or in SPLIT (head 0, key group j)
-    const int my_head = SPLIT ? 0 : j;
-    const int e_c = qe_s[my_head];
-    const float kfac = pow2i(24 - (14 - e_c));       // undoes the 2^-24 of the subnormal codes and bscale
-    const float inv_kfac = pow2i(-(24 - (14 - e_c)));
-    float Qg[SPLIT ? 1 : NG];
-    if constexpr (SPLIT) {
-      Qg[0] = qg_s[j] * inv_kfac;                     // NG == 4: every lane of the quad owns one group
-    } else {
-#pragma unroll
-      for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g] * inv_kfac;
-    }
-    const float neg_half = -(float)(1 << (BITS - 1));
-    // Raw scores (still carrying 1/kfac) of the 16 packed key rows r0 .. r0+15 of a chunk: this lane's rows are
-    // r0 + gid and r0 + gid + 8.  kc / km: packed rows and metadata rows of the chunk (shared or global memory).
-    auto k_mtile = [&](const uint32_t* kc, const uint32_t* km, int r0, float& sA_out, float& sB_out) {
-      const int rA = r0 + gid, rB = rA + 8;
-      uint32_t wa[RWL], wb[RWL];
-      if constexpr (RWL == 2) {
-        const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + j * RWL);
-        const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + j * RWL);
-        wa[0] = xa.x; wa[1] = xa.y; wb[0] = xb.x; wb[1] = xb.y;
-      } else {
-        const uint4 xa = *reinterpret_cast<const uint4*>(kc + rA * RW + j * RWL);
-        const uint4 xb = *reinterpret_cast<const uint4*>(kc + rB * RW + j * RWL);
-        wa[0] = xa.x; wa[1] = xa.y; wa[2] = xa.z; wa[3] = xa.w;
-        wb[0] = xb.x; wb[1] = xb.y; wb[2] = xb.z; wb[3] = xb.w;
-      }
-      auto kstep = [&](float (&c4)[4], int ks, bool zero_c) {
-        const int wi = ks / (2 * KPW), sw = ks % (2 * KPW);
-        const int window = sw / KPW, kk = sw % KPW;
-        const uint32_t xa = window ? (wa[wi] >> 8) : wa[wi];
-        const uint32_t xb = window ? (wb[wi] >> 8) : wb[wi];
-        const uint32_t m0 = F::kField << (BITS * (2 * kk)), m1 = F::kField << (BITS * (2 * kk + 1));
-        if (zero_c) mma16816_z(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-        else mma16816(c4, xa & m0, xb & m0, xa & m1, xb & m1, Bq[ks][0], Bq[ks][1]);
-      };
-      float sA, sB;
-      if constexpr (SPLIT) {
-        float c4[4];
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
-        float s_, z_;
-        decode_fast(km[rA * NG + j], neg_half, s_, z_);
-        sA = fmaf(s_, c4[0] + c4[1], z_ * Qg[0]);
-        decode_fast(km[rB * NG + j], neg_half, s_, z_);
-        sB = fmaf(s_, c4[2] + c4[3], z_ * Qg[0]);
-        sA += __shfl_xor_sync(0xffffffffu, sA, 1);
-        sB += __shfl_xor_sync(0xffffffffu, sB, 1);
-        sA += __shfl_xor_sync(0xffffffffu, sA, 2);
-        sB += __shfl_xor_sync(0xffffffffu, sB, 2);
-      } else {
-        uint32_t ma[NG], mb[NG];
-        if constexpr (NG == 4) {
-          const uint4 xa = *reinterpret_cast<const uint4*>(km + rA * NG);
-          const uint4 xb = *reinterpret_cast<const uint4*>(km + rB * NG);
-          ma[0] = xa.x; ma[1] = xa.y; ma[2] = xa.z; ma[3] = xa.w;
-          mb[0] = xb.x; mb[1] = xb.y; mb[2] = xb.z; mb[3] = xb.w;
-        } else if constexpr (NG == 2) {
-          const uint2 xa = *reinterpret_cast<const uint2*>(km + rA * NG);
-          const uint2 xb = *reinterpret_cast<const uint2*>(km + rB * NG);
-          ma[0] = xa.x; ma[1] = xa.y; mb[0] = xb.x; mb[1] = xb.y;
-        } else {
-          ma[0] = km[rA]; mb[0] = km[rB];
-        }
-        sA = 0.f; sB = 0.f;
-#pragma unroll
-        for (int g = 0; g < NG; ++g) {
-          float c4[4];
-#pragma unroll
-          for (int ks = 0; ks < KS_PER_G; ++ks) kstep(c4, g * KS_PER_G + ks, ks == 0);
-          float s_, z_;
-          decode_fast(ma[g], neg_half, s_, z_);
-          sA = fmaf(s_, c4[0] + c4[1], fmaf(z_, Qg[g], sA));
-          decode_fast(mb[g], neg_half, s_, z_);
-          sB = fmaf(s_, c4[2] + c4[3], fmaf(z_, Qg[g], sB));
-        }
-      }
-      sA_out = sA;
-      sB_out = sB;
-    };
-
-    // Fragments of raw q'' for the fp16 key rows of this warp's tail tiles (registers only while those run).
-    // SPLIT reuses the table area for its side ring, so the tables are released now, while all warps are in step.
-    uint32_t Bqr[8][2];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      Bqr[s][0] = tw > 0 ? bqr_s[(s * 2) * 32 + lane] : 0u;
-      Bqr[s][1] = tw > 0 ? bqr_s[(s * 2 + 1) * 32 + lane] : 0u;
-    }
-    const float kfac_raw = pow2i(-(14 - qe_s[4 + my_head]));       // fp16 key rows: accumulator * kfac_raw
-    if constexpr (SPLIT) {
-      __syncthreads();
-      for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
-      __syncwarp();
-    }
-
-    float m_run = -INFINITY, l_part = 0.f, psum = 0.f;
-    float out_acc[8][2];
-    float accg[8][4];
-#pragma unroll
-    for (int m = 0; m < 8; ++m) {
-      out_acc[m][0] = out_acc[m][1] = 0.f;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
-    }
-    bool failed = false;
-
-    // ---------------- tail tiles of this warp: fp16 windows and the K/V skew zone -------------------
-    // 16 tokens at a time, operands straight from global memory (coalesced 128-bit loads), into the warp's
-    // running soft-max state.  Keys: fp16 rows against raw q'' (pieces tid4 + 4i of rows gid, gid + 8), or the
-    // packed rows of the skew zone through the same path as the main loop.  Values: fp16 rows, pieces gid and
-    // gid + 8 of token rows 2*tid4, 2*tid4 + 1 (+8), byte-permuted into (channel; token pair) fragments.
-    for (int k = 0; k < tw; ++k) {
-      bool skew; int e0, cnt;
-      tail_tile(k, skew, e0, cnt);
-      float sA, sB;                                            // true log2-domain scores of entries e0+gid, e0+gid+8
-      if (skew) {
-        const int iq = cn.n_qv + e0;                           // first packed key row of the tile (16-aligned)
-        const unsigned char* rec = g_rec + (size_t)((iq / kChunk) / CH) * SL::kGroupRec +
-                                   (size_t)((iq / kChunk) % CH) * SL::kRec;
-        k_mtile(reinterpret_cast<const uint32_t*>(rec), reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta),
-                iq % kChunk, sA, sB);
-        sA *= kfac;
-        sB *= kfac;
-      } else {
-        const uint4* ra = k_row(e0 + min(gid, cnt - 1));
-        const uint4* rb = k_row(e0 + min(gid + 8, cnt - 1));
-        uint4 ka[4], kb[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { ka[i] = __ldg(ra + j + 4 * i); kb[i] = __ldg(rb + j + 4 * i); }
-        float c4[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          if (i == 0) mma16816_z(c4, ka[i].x, kb[i].x, ka[i].y, kb[i].y, Bqr[0][0], Bqr[0][1]);
-          else mma16816(c4, ka[i].x, kb[i].x, ka[i].y, kb[i].y, Bqr[2 * i][0], Bqr[2 * i][1]);
-          mma16816(c4, ka[i].z, kb[i].z, ka[i].w, kb[i].w, Bqr[2 * i + 1][0], Bqr[2 * i + 1][1]);
-        }
-        sA = (c4[0] + c4[1]) * kfac_raw;
-        sB = (c4[2] + c4[3]) * kfac_raw;
-        if constexpr (SPLIT) {       // only column pair 0 carries the head: hand its sums to the whole quad
-          sA = __shfl_sync(0xffffffffu, sA, lane & ~3);
-          sB = __shfl_sync(0xffffffffu, sB, lane & ~3);
-        }
-      }
-      if (gid >= cnt) sA = -INFINITY;
-      if (gid + 8 >= cnt) sB = -INFINITY;
-      float cmax = fmaxf(sA, sB);
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
-      const float m_new = fmaxf(m_run, cmax);
-      const float alpha = ex2_approx(m_run - m_new);            // 0 while m_run = -inf
-      m_run = m_new;
-      l_part *= alpha;
-#pragma unroll
-      for (int m = 0; m < 8; ++m) { out_acc[m][0] *= alpha; out_acc[m][1] *= alpha; }
-      const float pA = ex2_approx(sA - m_new), pB = ex2_approx(sB - m_new);
-      l_part += pA + pB;
-      uint32_t pkA = split_hi_lo(pA * 1024.f), pkB = split_hi_lo(pB * 1024.f);
-      if (SPLIT && j != 0) { pkA = 0u; pkB = 0u; }              // SPLIT: lane 0 of each quad takes the tail's sums
-      const uint32_t b0 = movmatrix_trans(pkA), b1 = movmatrix_trans(pkB);
-      const uint4* vr[4] = {v_row(skew, e0 + min(2 * j, cnt - 1)), v_row(skew, e0 + min(2 * j + 1, cnt - 1)),
-                            v_row(skew, e0 + min(2 * j + 8, cnt - 1)), v_row(skew, e0 + min(2 * j + 9, cnt - 1))};
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint4 v4[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) v4[r] = __ldg(vr[r] + gid + 8 * hh);
-        const uint32_t* T0 = reinterpret_cast<const uint32_t*>(&v4[0]);
-        const uint32_t* T1 = reinterpret_cast<const uint32_t*>(&v4[1]);
-        const uint32_t* T8 = reinterpret_cast<const uint32_t*>(&v4[2]);
-        const uint32_t* T9 = reinterpret_cast<const uint32_t*>(&v4[3]);
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {                        // m-tile 4*hh + kk: channels 64*hh + 8*gid + 2*kk (+1)
-          float c4[4];
-          mma16816_z(c4, __byte_perm(T0[kk], T1[kk], 0x5410), __byte_perm(T0[kk], T1[kk], 0x7632),
-                     __byte_perm(T8[kk], T9[kk], 0x5410), __byte_perm(T8[kk], T9[kk], 0x7632), b0, b1);
-          // out_acc is kept in units of 2^-14; these sums carry p * 2^10
-          out_acc[4 * hh + kk][0] = fmaf(c4[0] + c4[1], 0x1p-24f, out_acc[4 * hh + kk][0]);
-          out_acc[4 * hh + kk][1] = fmaf(c4[2] + c4[3], 0x1p-24f, out_acc[4 * hh + kk][1]);
-        }
-      }
-    }
-
-    // The loop body is deliberately not unrolled over iterations: two CTAs of eight warps walk it at
-    // different phases, so it has to stay resident in the instruction cache.
-#pragma unroll 1
-    for (int it = 0; it < n_iters; ++it) {
-      const int st = it & (NST - 1);
-      const uint32_t parity = (uint32_t)(it / NST) & 1u;
-      if (!mbar_wait(bars_u32 + 8 * st, parity)) { failed = true; break; }
-      const unsigned char* sp = ring + st * SL::kBytes;
-      const int ci0 = c_lo + it * CPI;                           // first chunk of this iteration (unit-relative)
-      const bool last_valid = CPI == 1 || (it * CPI + 1 < n_chunks_w);   // odd chunk count: the last half is empty
-
-      // ---------------- raw scores: CPI * 2 m-tiles of 16 tokens -------------------------------------
-      float sc[CPI][2][2];
-#pragma unroll
-      for (int cc = 0; cc < CPI; ++cc) {
-        if (cc > 0 && !last_valid) {      // nothing there: this warp's range ends in the middle of the iteration
-          sc[cc][0][0] = sc[cc][0][1] = sc[cc][1][0] = sc[cc][1][1] = -INFINITY;
-          continue;
-        }
-        const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc));
-        const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          float sA, sB;
-          k_mtile(kc, km, 16 * mt, sA, sB);
-          const bool valid = cc == 0 || last_valid;
-          sc[cc][mt][0] = valid ? sA : -INFINITY;
-          sc[cc][mt][1] = valid ? sB : -INFINITY;
-        }
-      }
-
-      // ---------------- online softmax (log2 domain; raw scores still carry 1/kfac) -------------------
-      float cmax = -INFINITY;
-#pragma unroll
-      for (int cc = 0; cc < CPI; ++cc)
-        cmax = fmaxf(cmax, fmaxf(fmaxf(sc[cc][0][0], sc[cc][0][1]), fmaxf(sc[cc][1][0], sc[cc][1][1])));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
-      const float m_new = fmaxf(m_run, cmax * kfac);
-      if (__any_sync(0xffffffffu, m_new > m_run)) {
-        const float alpha = ex2_approx(m_run - m_new);     // 0 on the first iteration (m_run = -inf)
-        l_part *= alpha;
-        psum *= alpha;
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
-        }
-      }
-      m_run = m_new;
-
-#pragma unroll
-      for (int cc = 0; cc < CPI; ++cc) {
-        if (cc > 0 && !last_valid) continue;
-        const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffVCodes);
-        const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
-        const int ci = ci0 + cc;
-        // slot: position of this chunk's value group in the SPLIT window / position of the chunk in its group
-        const int slot = SPLIT ? (ci - c_lo) & (WIN - 1) : ci % CH;
-        const bool group_start = slot == 0;
-        const bool group_end = SPLIT ? (slot == WIN - 1 || (it == n_iters - 1 && (cc == CPI - 1 || !last_valid)))
-                                     : (slot == CH - 1);
-        constexpr bool kFreshEveryChunk = !SPLIT && CH == 1;   // then the first value mma takes a zero C
-        if (!kFreshEveryChunk && group_start) {
-#pragma unroll
-          for (int m = 0; m < 8; ++m)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
-        }
-        uint32_t Bp[2][2];
-        float psum_c = 0.f;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const float p = ex2_approx(fmaf(sc[cc][mt][h], kfac, -m_new));
-            psum_c += p;
-            const int pos = BITS == 2 ? 2 * mt + h : h;
-            // p goes in as one fp16 (the lo column stays zero): its 2^-12 relative rounding is random per token and
-            // far inside the output tolerance, and it saves the hi/lo split of every probability
-            uint32_t pk = (uint32_t)__half_as_ushort(__float2half_rn(p * pow2i(10 - BITS * pos)));
-            if (SPLIT && j != slot) pk = 0u;                 // column pair of this chunk's window slot only
-            Bp[mt][h] = movmatrix_trans(pk);
-          }
-        }
-        l_part += psum_c;
-        if constexpr (SPLIT) psum += (j == slot) ? psum_c : 0.f;
-        else psum += psum_c;
-
-        // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
-        if constexpr (BITS == 2) {
-          const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
-          const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
-          const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-          for (int m = 0; m < 8; ++m) {
-            const uint32_t w0 = vw[m], w1 = vw[m] >> 8;
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
-              const uint32_t m0 = F::kField << (2 * (2 * ks)), m1 = F::kField << (2 * (2 * ks + 1));
-              if (kFreshEveryChunk && ks == 0) mma16816_z(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-              else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-            }
-          }
-        } else {
-#pragma unroll
-          for (int ks = 0; ks < 2; ++ks) {
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-              const uint4 v = *reinterpret_cast<const uint4*>(vc + ks * 256 + hh * 128 + lane * 4);
-              const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-              for (int mm = 0; mm < 4; ++mm) {
-                const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
-                const uint32_t m0 = F::kField, m1 = F::kField << 4;
-                if (kFreshEveryChunk && ks == 0)
-                  mma16816_z(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-                else
-                  mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-              }
-            }
-          }
-        }
-
-        // ---------------- end of a value group: apply scale / zero-point once per channel -----------
-        const bool chunk_valid = cc == 0 || last_valid;
-        if constexpr (SPLIT) {
-          // keep this group's metadata for the end of the window (the stage will be refilled)
-          if (chunk_valid)
-            *reinterpret_cast<uint4*>(side + slot * kD + lane * 4) = *reinterpret_cast<const uint4*>(vm + lane * 4);
-        }
-        if (group_end && chunk_valid) {
-          if constexpr (SPLIT) __syncwarp();
-          float pg = psum;
-          pg += __shfl_xor_sync(0xffffffffu, pg, 4);
-          pg += __shfl_xor_sync(0xffffffffu, pg, 8);
-          pg += __shfl_xor_sync(0xffffffffu, pg, 16);
-          pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
-          const uint4* vm4 = reinterpret_cast<const uint4*>((SPLIT ? side + j * kD : vm) + gid * 16);
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const uint4 mw = vm4[q4];
-            const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // channel 16 m + 8 rh + gid
-              float s_, z_;
-              decode_fast(mws[e], neg_half, s_, z_);
-              out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
-            }
-          }
-          psum = 0.f;
-        }
-      }
-
-      __syncwarp();
-      if (lane == 0 && it + NST < n_iters) issue(st);
-    }
-
-    if (failed) {
-      // a copy never arrived: flag it for the host and contribute nothing
-      if (lane == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);
-      m_run = -INFINITY;
-      l_part = 0.f;
-    }
-
-    // ---------------- warp result -> shared memory -> CTA partial ---------------------------------
-    l_part += __shfl_xor_sync(0xffffffffu, l_part, 4);
-    l_part += __shfl_xor_sync(0xffffffffu, l_part, 8);
-    l_part += __shfl_xor_sync(0xffffffffu, l_part, 16);
-    if constexpr (SPLIT) {
-      // the four lanes of a quad hold the contributions of different window slots: add them up
-#pragma unroll
-      for (int m = 0; m < 8; ++m)
-#pragma unroll
-        for (int rh = 0; rh < 2; ++rh) {
-          float v = out_acc[m][rh];
-          v += __shfl_xor_sync(0xffffffffu, v, 1);
-          v += __shfl_xor_sync(0xffffffffu, v, 2);
-          out_acc[m][rh] = v;
-        }
-    }
-    __syncthreads();                                   // every warp is done with its ring
-    float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
-    const bool writer = SPLIT ? (j == 0) : true;
-    const bool any = n_iters > 0 || tw > 0;
-    if (writer) {
-      float* mine = wres + ((size_t)warp * kHeads + (SPLIT ? 0 : j)) * (kD + 2);
-#pragma unroll
-      for (int m = 0; m < 8; ++m) {
-        mine[block_row_channel(m, 0, gid)] = any ? out_acc[m][0] * 0x1p14f : 0.f;
-        mine[block_row_channel(m, 1, gid)] = any ? out_acc[m][1] * 0x1p14f : 0.f;
-      }
-      if (gid == 0) {
-        mine[kD] = any ? m_run : -INFINITY;
-        mine[kD + 1] = any ? l_part : 0.f;
-      }
-    }
-    __syncthreads();
-    float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
-    for (int i = tid; i < nh * kD; i += kThreads) {
-      const int h = i >> 7, c = i & (kD - 1);
-      float M = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wres[((size_t)w * kHeads + h) * (kD + 2) + kD]);
-      float num = 0.f, den = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const float* r_ = wres + ((size_t)w * kHeads + h) * (kD + 2);
-        const float wgt = r_[kD] == -INFINITY ? 0.f : exp2f(r_[kD] - M);
-        num = fmaf(r_[c], wgt, num);
-        den = fmaf(r_[kD + 1], wgt, den);
-      }
-      float* P = partials + ((size_t)(head_base + h) * L.max_splits + split) * kPartialStride;
-      P[c] = num;
-      if (c == 0) { P[kD] = M; P[kD + 1] = den; }
-    }
-  }
-
-  // ---------------- cross-CTA merge: the last CTA of the unit to arrive combines all parts -----------
-  __shared__ unsigned int s_ticket;
-  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's fence below
-  if (tid == 0) {
-    __threadfence();               // cumulative: publishes the whole CTA's partial before the ticket is taken
-    s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
-  }
-  __syncthreads();
-  if (s_ticket != gridDim.y - 1) return;
-  __threadfence();
-  const float* partials = reinterpret_cast<const float*>(a.ws + L.ws_partial_off);
-  float* mw = reinterpret_cast<float*>(smem);          // [head][part]: max, then weight
-  float* lw = mw + kHeads * 128;                        // [head][part]: l
-  for (int i = tid; i < nh * n_parts; i += kThreads) {
-    const int h = i / n_parts, s = i % n_parts;
-    const float* P = partials + ((size_t)(head_base + h) * L.max_splits + s) * kPartialStride;
-    mw[h * 128 + s] = __ldcg(P + kD);
-    lw[h * 128 + s] = __ldcg(P + kD + 1);
-  }
-  __syncthreads();
-  for (int i = tid; i < nh * kD; i += kThreads) {
-    const int h = i >> 7, c = i & (kD - 1);
-    const float* P = partials + (size_t)(head_base + h) * L.max_splits * kPartialStride + c;
-    float M = -INFINITY;
-    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, mw[h * 128 + s]);
-    float num = 0.f, den = 0.f;
-    for (int s0 = 0; s0 < n_parts; s0 += 16) {          // sixteen independent loads in flight
-      float v[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) v[e] = s0 + e < n_parts ? __ldcg(P + (size_t)(s0 + e) * kPartialStride) : 0.f;
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        if (s0 + e < n_parts) {
-          const float ms = mw[h * 128 + s0 + e];
-          const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
-          num = fmaf(v[e], wgt, num);
-          den = fmaf(lw[h * 128 + s0 + e], wgt, den);
-        }
-      }
-    }
-    a.out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
-  }
-  if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
-}
-
 int g_chunks_per_iter = 0;    // tuning knob: 0 automatic, else 1 or 2 chunks of 32 tokens per loop iteration
 
-template <int BITS, int G, bool SPLIT, int CPI>
-int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
-  using SL = StageLayout<BITS, G, CPI>;
-  constexpr int kSmem = SL::kCtaBytes;
-  constexpr int RU = SL::kCH;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_kernel<BITS, G, SPLIT, CPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSmem) != cudaSuccess)
-      return -1;
-    configured = true;
-  }
-  const int n_chunks = cn.n_qv / kChunk;
-  const int n_units = (n_chunks + RU - 1) / RU;
-  const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
-  if (n_splits > by_work) n_splits = by_work;
-  if (n_units == 0) n_splits = 0;
-  // without packed chunks the CTAs only share the tail tiles (eight per CTA)
-  int grid_y = n_splits > 0 ? n_splits : (a.n_tail_tiles + kWarps - 1) / kWarps;
-  if (grid_y < 1) grid_y = 1;
-  if (grid_y > L.max_splits) grid_y = L.max_splits;
-  a.n_splits = n_splits;
-  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about as much as one value group's chunks
-  {
-    const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
-    a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
-  }
-  a.tiles_q0 = a.n_tail_tiles / grid_y;
-  a.tiles_rem = a.n_tail_tiles % grid_y;
-  dim3 grid(L.U, grid_y);
-  int launches = 0;
-  const int step = SPLIT ? 1 : kHeads;
-  for (int h0 = 0; h0 < L.r; h0 += step) {
-    a.head0 = h0;
-    decode_mma_kernel<BITS, G, SPLIT, CPI><<<grid, kThreads, kSmem, st>>>(L, cn, a);
-    ++launches;
-  }
-  return cudaGetLastError() == cudaSuccess ? launches : -1;
-}
+using FormatLauncher = int (*)(const Layout&, const Counts&, const DecodeArgs&, int, int, cudaStream_t);
 
-template <int BITS, int G, bool SPLIT>
-int launch_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, cudaStream_t st) {
-  // two chunks per iteration need twice the stage bytes: with 4-bit codes that would cost the second resident CTA
-  const int cpi = g_chunks_per_iter ? g_chunks_per_iter : (BITS == 2 ? 2 : 1);
-  if (cpi == 1) return launch_one<BITS, G, SPLIT, 1>(L, cn, a, n_splits, st);
-  return launch_one<BITS, G, SPLIT, 2>(L, cn, a, n_splits, st);
+// The formats with kernels: equal key and value bit widths with full or symmetric-only metadata, and the mixed
+// 3-bit-key / 2-bit-value combinations with symmetric keys.
+FormatLauncher format_launcher(const Layout& L) {
+  if (L.grouping != 0 || L.k.kind != kRow || L.v.kind != kBlock) return nullptr;
+  if (L.G != 32 && L.G != 64 && L.G != 128) return nullptr;
+  const int kb = L.k.bits, vb = L.v.bits, km = L.k.meta_bytes, vm = L.v.meta_bytes;
+  if (kb == 2 && vb == 2 && km == 4 && vm == 4) return &launch_decode_mma_k2v2_m44;
+  if (kb == 4 && vb == 4 && km == 4 && vm == 4) return &launch_decode_mma_k4v4_m44;
+  if (kb == 3 && vb == 3 && km == 4 && vm == 4) return &launch_decode_mma_k3v3_m44;
+  if (kb == 2 && vb == 2 && km == 2 && vm == 2) return &launch_decode_mma_k2v2_m22;
+  if (kb == 3 && vb == 3 && km == 2 && vm == 2) return &launch_decode_mma_k3v3_m22;
+  if (kb == 4 && vb == 4 && km == 2 && vm == 2) return &launch_decode_mma_k4v4_m22;
+  if (kb == 3 && vb == 2 && km == 2 && vm == 2) return &launch_decode_mma_k3v2_m22;
+  if (kb == 3 && vb == 2 && km == 2 && vm == 4) return &launch_decode_mma_k3v2_m24;
+  return nullptr;
 }
 
 }  // namespace
 
-bool decode_mma_supported(const Layout& L) {
-  return L.grouping == 0 && L.k.kind == kRow && L.v.kind == kBlock && L.k.bits == L.v.bits &&
-         (L.k.bits == 2 || L.k.bits == 4) && L.k.meta_bytes == 4 && L.v.meta_bytes == 4;
-}
+bool decode_mma_supported(const Layout& L) { return format_launcher(L) != nullptr; }
 
 void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
 
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                       __half* out, int n_splits, cudaStream_t st) {
-  if (!decode_mma_supported(L)) return -2;
+  const FormatLauncher launch = format_launcher(L);
+  if (!launch) return -2;
   const Counts cn = counts_for(L, N);
   if (n_splits <= 0) {
     n_splits = (2 * 148) / L.U;                  // two resident CTAs per SM, one wave
@@ -908,16 +57,7 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.k_ring_pos0 = L.k.ring_cap ? cn.n_qk % L.k.ring_cap : 0;
   a.v_ring_pos0 = L.v.ring_cap ? cn.n_qv % L.v.ring_cap : 0;
   a.head0 = 0;
-  const int bits = L.k.bits;
-  if (bits == 2 && L.G == 32 && L.r == 1) return launch_cpi<2, 32, true>(L, cn, a, n_splits, st);
-  if (bits == 4 && L.G == 32 && L.r == 1) return launch_cpi<4, 32, true>(L, cn, a, n_splits, st);
-  if (bits == 2 && L.G == 32) return launch_cpi<2, 32, false>(L, cn, a, n_splits, st);
-  if (bits == 2 && L.G == 64) return launch_cpi<2, 64, false>(L, cn, a, n_splits, st);
-  if (bits == 2 && L.G == 128) return launch_cpi<2, 128, false>(L, cn, a, n_splits, st);
-  if (bits == 4 && L.G == 32) return launch_cpi<4, 32, false>(L, cn, a, n_splits, st);
-  if (bits == 4 && L.G == 64) return launch_cpi<4, 64, false>(L, cn, a, n_splits, st);
-  if (bits == 4 && L.G == 128) return launch_cpi<4, 128, false>(L, cn, a, n_splits, st);
-  return -2;
+  return launch(L, cn, a, n_splits, g_chunks_per_iter, st);
 }
 
 }  // namespace iq

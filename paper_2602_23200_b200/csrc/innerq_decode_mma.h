@@ -1,0 +1,39 @@
+// Interface between the host side of the fused decode kernel (innerq_decode_mma.cu) and the translation
+// units that compile its kernels, one per packed format (innerq_decode_mma_k*v*_m*.cu).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "innerq_layout.h"
+
+namespace iq {
+
+// Launch parameters shared by every format's kernels (filled by launch_decode_mma).
+struct DecodeArgs {
+  const unsigned char* cache;
+  unsigned char* ws;
+  const __half* q;
+  __half* out;
+  int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
+  int n_tail_tiles;      // tiles of 16 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
+                         // tile x belongs to CTA x % gridDim.y, warp (x / gridDim.y) % 8
+  int n_skew_tiles;      // of those, tiles whose keys are packed rows (values still fp16)
+  int tiles_q0, tiles_rem;   // n_tail_tiles / gridDim.y and n_tail_tiles % gridDim.y
+  int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
+  int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
+  int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
+  int head0;             // first query head (within the KV head's r) handled by this launch
+};
+
+// Launchers by format: k<key bits>v<value bits>_m<bytes per key metadata entry><bytes per value metadata entry>.
+// cpi: chunks of 32 tokens per loop iteration (0 = automatic).  Return the number of launches, or < 0.
+int launch_decode_mma_k2v2_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k4v4_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k3v3_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k2v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k3v3_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k4v4_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k3v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_k3v2_m24(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+
+}  // namespace iq

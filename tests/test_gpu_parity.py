@@ -67,8 +67,7 @@ def test_prefill_and_decode_inner(bits, G, mode, variant, N):
     w = synth.tiny(n_tokens=N, group=G, k_bits=bits, v_bits=bits, k_mode=mode, v_mode=mode, sym_variant=variant)
     oc, gc, _, _ = run_prefill_both(w)
     P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, mode == O.HYBRID, mode == O.HYBRID)
-    fast = (3, 4) if bits in (2, 4) and mode != O.SYM else ()
-    check_decode(w, oc, gc, variants=(0, 1) + fast, splits=(0, 1, 3, 7))
+    check_decode(w, oc, gc, variants=(0, 1, 3, 4), splits=(0, 1, 3, 7))
 
 
 @pytest.mark.parametrize("bits,G,N", [(2, 32, 333), (3, 64, 420), (4, 128, 541)])
@@ -97,7 +96,37 @@ def test_mixed_bits_and_modes():
     w = synth.tiny(n_tokens=400, group=32, k_bits=3, v_bits=2, k_mode=O.SYM, v_mode=O.HYBRID)
     oc, gc, _, _ = run_prefill_both(w)
     P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, 32, False, True)
-    check_decode(w, oc, gc, variants=(0, 1))
+    check_decode(w, oc, gc, variants=(0, 1, 3))
+
+
+# key bits, value bits, key mode, value mode, G, query heads per KV head, N: the packed formats the fused kernel
+# is built for beyond equal-width hybrid ones (3-bit planes, symmetric-only 2-byte metadata, 3-bit keys with
+# 2-bit values), with one query head per KV head (group-per-column kernel), several, and two passes of four
+FORMATS = [
+    (3, 3, O.HYBRID, O.HYBRID, 32, 1, 700),
+    (3, 3, O.SYM, O.SYM, 32, 1, 700),
+    (3, 2, O.SYM, O.SYM, 32, 1, 600),
+    (3, 2, O.SYM, O.HYBRID, 32, 1, 1500),
+    (3, 2, O.SYM, O.HYBRID, 64, 4, 600),
+    (3, 2, O.SYM, O.SYM, 128, 2, 900),
+    (2, 2, O.SYM, O.SYM, 128, 2, 900),
+    (4, 4, O.SYM, O.SYM, 32, 1, 500),
+    (3, 3, O.ASYM, O.ASYM, 128, 8, 900),
+    (3, 3, O.SYM, O.SYM, 64, 8, 555),
+]
+
+
+@pytest.mark.parametrize("kb,vb,km,vm,G,r,N", FORMATS)
+def test_fused_kernel_formats(kb, vb, km, vm, G, r, N):
+    w = synth.tiny(n_tokens=N, group=G, k_bits=kb, v_bits=vb, k_mode=km, v_mode=vm, n_q_heads=2 * r)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, km == O.HYBRID, vm == O.HYBRID)
+    check_decode(w, oc, gc, variants=(3, 1), splits=(0, 2, 5))       # 3: the fused kernel or an error, 1: generic kernel
+    for step in range(G + 3):                                          # across a value-group eviction
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+    check_decode(w, oc, gc, step=7, variants=(3,), splits=(0, 3))
 
 
 @pytest.mark.parametrize("N", [1, 3, 4, 5, 19, 20, 21, 52, 53])
