@@ -17,6 +17,10 @@ struct ExportPtrs {
 
 int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, const __half* K, const __half* V, int N,
                    cudaStream_t st);
+// Prefill quantiser of one store: rows / groups [0, n_q) of every unit from X ([U][N][128] fp16).
+// inv_norm: reciprocal key norms [U][128], or null.
+int launch_quantize_store_prefill(const Layout& L, const Store& S, const __half* X, int N, int n_q, unsigned char* cache,
+                                  const float* inv_norm, cudaStream_t st);
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
                   cudaStream_t st);
 int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st);

@@ -39,12 +39,15 @@ __global__ void __launch_bounds__(256) k_absmax_kernel(const __half* __restrict_
   }
 }
 
-// norm = sqrt(absmax), 0 -> 1  (Section "Per-channel Normalization of K")
-__global__ void finalize_norm_kernel(const uint32_t* __restrict__ absmax, float* __restrict__ norm, int n) {
+// norm = sqrt(absmax), 0 -> 1  (Section "Per-channel Normalization of K"); the absmax word is replaced by the
+// reciprocal 1 / norm (correctly rounded) that the quantisers multiply keys with
+__global__ void finalize_norm_kernel(uint32_t* __restrict__ absmax, float* __restrict__ norm, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     float n_ = __fsqrt_rn(__uint_as_float(absmax[i]));
-    norm[i] = n_ == 0.f ? 1.0f : n_;
+    n_ = n_ == 0.f ? 1.0f : n_;
+    norm[i] = n_;
+    absmax[i] = __float_as_uint(__fdiv_rn(1.0f, n_));
   }
 }
 
@@ -109,24 +112,6 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
   __syncwarp();
 }
 
-// Prefill: rows [0, n_q) of every unit; token of row i is w_sink + i.
-__global__ void __launch_bounds__(128) quantize_rows_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
-                                                            int n_q, unsigned char* __restrict__ cache,
-                                                            bool use_norm) {
-  __shared__ uint32_t stage[4][16];
-  const int u = blockIdx.y, warp = threadIdx.x >> 5;
-  const float* norm = reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD;
-  float inv4[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) inv4[i] = use_norm ? __fdiv_rn(1.0f, norm[4 * (threadIdx.x & 31) + i]) : 1.0f;
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
-  for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4) {
-    const __half* src = X + ((size_t)u * N + L.w_sink + i) * kD;
-    quantize_row_warp(src, use_norm ? inv4 : nullptr, L, S, stage[warp],
-                      reinterpret_cast<uint32_t*>(rec + row_code_off(S, i)), rec + row_meta_off(S, i), 0);
-  }
-}
-
 // ------------------------------------------------------------------ BLOCK store quantiser
 // A 128-thread CTA quantises one group of G tokens x 128 channels; thread c owns channel c.
 // tile: fp16 [G][D] staging; words: packed chunks of the group (zeroed here).
@@ -172,20 +157,6 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     reinterpret_cast<uint32_t*>(rec + block_code_off(S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
   }
   __syncthreads();
-}
-
-// Prefill: groups [0, n_q / G) of every unit; group j covers tokens w_sink + jG .. + G - 1.
-__global__ void __launch_bounds__(128) quantize_blocks_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
-                                                              int n_q, unsigned char* __restrict__ cache,
-                                                              bool use_norm) {
-  __shared__ __align__(16) __half tile[128 * kD];
-  __shared__ uint32_t words[4 * 512];
-  const int u = blockIdx.y;
-  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
-  TokSrc src{X + (size_t)u * N * kD, 0, 0};
-  for (int j = blockIdx.x; j < n_q / L.G; j += gridDim.x)
-    quantize_block_cta(src, L.w_sink + j * L.G, norm, L, S, tile, words, rec, j);
 }
 
 // ------------------------------------------------------------------ window copies (prefill)
@@ -339,11 +310,8 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
     }
     const bool nrm = use_norm && i == 0;
     if (nq[i] > 0) {
-      if (S.kind == kRow)
-        quantize_rows_kernel<<<dim3(grid_for(nq[i], 4 * 8, 4096), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i], cache, nrm);
-      else
-        quantize_blocks_kernel<<<dim3(grid_for(nq[i] / L.G, 1, 8192), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i], cache,
-                                                                                       nrm);
+      const float* inv_norm = nrm ? reinterpret_cast<const float*>(ws + L.ws_absmax_off) : nullptr;
+      if (launch_quantize_store_prefill(L, S, srcs[i], N, nq[i], cache, inv_norm, st) < 0) return -1;
       launches += 1;
     }
     // fp16 windows: sink, then everything after the quantised middle

@@ -1,0 +1,322 @@
+// Prefill quantisers: the middle tokens of every unit into the ROW store (groups of G channels inside a token,
+// Section "InnerQ" for keys) and the BLOCK store (per-channel groups of G tokens, values).
+//
+// Both are built around one work item: 32 values of one group held in the registers of one thread (a group of
+// 64 or 128 values is 2 or 4 such threads, which exchange their minima / maxima and error sums).  The thread
+// makes the passes the method needs over its registers: min / max, then (hybrid mode only) the L1 errors of both
+// candidates, then the codes of the chosen mode.  All value arithmetic is the same sequence of single, correctly
+// rounded fp32 operations as in group_params / asym_code / sym_code, so stored bits do not depend on the kernel:
+// rounding to an integer is done by adding 1.5 * 2^23 (round-to-nearest-even at unit granularity, identical to
+// rintf for |t| < 2^22; codes are bounded by a few times 2^b), which leaves the code in the low mantissa bits.
+#include "innerq_device.cuh"
+#include "innerq_kernels.h"
+
+namespace iq {
+
+namespace {
+
+constexpr float kMagic = 12582912.0f;       // 1.5 * 2^23
+constexpr int kSeg = 32;                    // values per thread
+
+struct SegCoder {
+  float z_a, inv_a, s_a, lo_a, hi_a;        // asymmetric: clamp bounds in the magic domain
+  float inv_s, s_s, off_s, lo_s, hi_s;      // symmetric (offset-binary): magic + 2^(b-1), bounds
+  __device__ __forceinline__ explicit SegCoder(const GroupParams& p) {
+    z_a = p.z_a; inv_a = p.inv_a; s_a = p.s_a; lo_a = kMagic; hi_a = kMagic + p.L;
+    inv_s = p.inv_s; s_s = p.s_s; off_s = kMagic + p.half; lo_s = off_s + p.q_lo; hi_s = off_s + p.q_hi;
+  }
+  // clamped code plus magic (asymmetric) / plus magic + 2^(b-1) (symmetric): the low mantissa bits are the stored code
+  __device__ __forceinline__ float asym(float x) const {
+    const float t = __fadd_rn(__fmul_rn(__fsub_rn(x, z_a), inv_a), kMagic);
+    return fminf(fmaxf(t, lo_a), hi_a);
+  }
+  __device__ __forceinline__ float sym(float x) const {
+    const float t = __fadd_rn(__fmul_rn(x, inv_s), off_s);
+    return fminf(fmaxf(t, lo_s), hi_s);
+  }
+  // L1 reconstruction errors of one value (used only to pick the mode of a hybrid group)
+  __device__ __forceinline__ float err_asym(float x) const {
+    return fabsf(__fmaf_rn(-s_a, asym(x) - kMagic, __fsub_rn(x, z_a)));
+  }
+  __device__ __forceinline__ float err_sym(float x) const { return fabsf(__fmaf_rn(-s_s, sym(x) - off_s, x)); }
+};
+
+// The coder of the chosen mode as one formula, clamp(((x - z) * inv) + off): symmetric is z = 0 (x - 0 is exact).
+struct ChosenCoder {
+  float z, inv, off, lo, hi;
+  __device__ __forceinline__ ChosenCoder(const SegCoder& c, bool asym)
+      : z(asym ? c.z_a : 0.f), inv(asym ? c.inv_a : c.inv_s), off(asym ? kMagic : c.off_s), lo(asym ? c.lo_a : c.lo_s),
+        hi(asym ? c.hi_a : c.hi_s) {}
+  __device__ __forceinline__ uint32_t code_bits(float x) const {     // the code is in the low mantissa bits
+    const float t = __fadd_rn(__fmul_rn(__fsub_rn(x, z), inv), off);
+    return __float_as_uint(fminf(fmaxf(t, lo), hi));
+  }
+};
+
+// min / max of 32 registers
+__device__ __forceinline__ void seg_minmax(const float (&x)[kSeg], float& mn, float& mx) {
+  mn = x[0]; mx = x[0];
+#pragma unroll
+  for (int e = 1; e < kSeg; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+}
+
+__device__ __forceinline__ void seg_errors(const SegCoder& sc, const float (&x)[kSeg], float& ea, float& es) {
+  float a0 = 0.f, a1 = 0.f, s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int e = 0; e < kSeg; e += 2) {
+    a0 += sc.err_asym(x[e]); a1 += sc.err_asym(x[e + 1]);
+    s0 += sc.err_sym(x[e]);  s1 += sc.err_sym(x[e + 1]);
+  }
+  ea = a0 + a1; es = s0 + s1;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* x) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(h[i]);
+    x[2 * i] = f.x; x[2 * i + 1] = f.y;
+  }
+}
+
+// ------------------------------------------------------------------ ROW store
+// A warp quantises 8 consecutive tokens per iteration: lane = 4 * (token in the batch) + segment, segment =
+// channels 32*seg .. 32*seg+31.  The 8 packed rows and their metadata entries are contiguous in the chunk record.
+// Positions of the segment's codes (see row_pos_plane): element e of segment 0 sits in local word j = tid4(e);
+// for segment seg the word index and the bit offset move by a per-plane amount that depends on seg only.
+template <int BITS, bool NORM>
+__global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
+                                                                    int n_q, unsigned char* __restrict__ cache,
+                                                                    const float* __restrict__ inv_norm) {
+  constexpr int RW = 4 * BITS;                // 32-bit words per packed row
+  constexpr int PB = BITS == 3 ? 2 : BITS;    // bits of the primary plane
+  __shared__ uint32_t stage_all[4][8 * RW];
+  const int u = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int seg = lane & 3, tk = lane >> 2;
+  const int gl = L.G >> 5;                    // lanes per group: 1, 2 or 4
+  uint32_t* stage = stage_all[warp];
+#pragma unroll
+  for (int k = 0; k < RW / 4; ++k) stage[lane + 32 * k] = 0u;
+  float inv[NORM ? kSeg : 1];
+  if constexpr (NORM) {
+    const float4* p = reinterpret_cast<const float4*>(inv_norm + (size_t)u * kD + kSeg * seg);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float4 v = __ldg(p + k);
+      inv[4 * k] = v.x; inv[4 * k + 1] = v.y; inv[4 * k + 2] = v.z; inv[4 * k + 3] = v.w;
+    }
+  }
+  // where this segment's local words go inside the row, and by how much its fields are shifted
+  constexpr int WM = PB == 2 ? 2 : 4;        // row words between consecutive local words
+  const int w_add = PB == 2 ? (seg >> 1) : seg;
+  const int sh_lo = PB == 2 ? 8 * (seg & 1) : 0, sh_hi = 4 * seg;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD + kSeg * seg;
+  const int n_batches = (n_q + 7) >> 3;
+  const int stride = gridDim.x * 4;
+  int bi = blockIdx.x * 4 + warp;
+  uint4 raw[4];
+  if (bi < n_batches) {
+    const uint4* src = reinterpret_cast<const uint4*>(Xu + (size_t)min(bi * 8 + tk, n_q - 1) * kD);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) raw[k] = __ldg(src + k);
+  }
+  for (; bi < n_batches; bi += stride) {
+    const int i0 = bi * 8;
+    float x[kSeg];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) unpack8(raw[k], x + 8 * k);
+    if (bi + stride < n_batches) {            // next batch's rows are requested before this one is worked on
+      const uint4* src = reinterpret_cast<const uint4*>(Xu + (size_t)min((bi + stride) * 8 + tk, n_q - 1) * kD);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) raw[k] = __ldg(src + k);
+    }
+    if constexpr (NORM) {
+#pragma unroll
+      for (int e = 0; e < kSeg; ++e) x[e] = __fmul_rn(x[e], inv[e]);
+    }
+    float mn, mx;
+    seg_minmax(x, mn, mx);
+    for (int o = 1; o < gl; o <<= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
+    const SegCoder sc(p);
+    bool asym = S.mode == 1;
+    if (S.mode == 2) {
+      float ea, es;
+      seg_errors(sc, x, ea, es);
+      for (int o = 1; o < gl; o <<= 1) {
+        ea += __shfl_xor_sync(0xffffffffu, ea, o);
+        es += __shfl_xor_sync(0xffffffffu, es, o);
+      }
+      asym = ea < es;
+    }
+    const ChosenCoder cc(sc, asym);
+    uint32_t lw[4] = {0u, 0u, 0u, 0u}, hw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int e = 0; e < kSeg; ++e) {
+      const uint32_t code = cc.code_bits(x[e]);
+      const BitPos lo = row_pos_plane(e, PB);            // constants: segment 0's positions
+      lw[lo.word / WM] |= (code & ((1u << PB) - 1u)) << lo.bit;
+      if constexpr (BITS == 3) {
+        const BitPos hi = row_pos_plane(e, 1);
+        hw[hi.word] |= ((code >> 2) & 1u) << hi.bit;
+      }
+    }
+    __syncwarp();                                          // the stage is zero and no longer being read
+    uint32_t* row = stage + tk * RW;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      atomicOr(&row[WM * jj + w_add], lw[jj] << sh_lo);
+      if constexpr (BITS == 3) atomicOr(&row[row_hi_plane_word() + jj], hw[jj] << sh_hi);
+    }
+    const int i = i0 + tk;
+    if (i < n_q && (lane & (gl - 1)) == 0)
+      store_meta(rec + row_meta_off(S, i0), (size_t)tk * S.n_groups + (seg >> (gl >> 1)), S.meta_bytes, group_meta(p, asym));
+    __syncwarp();
+    uint32_t* dst = reinterpret_cast<uint32_t*>(rec + row_code_off(S, i0));
+#pragma unroll
+    for (int k = 0; k < RW / 4; ++k) {
+      const int idx = lane + 32 * k;
+      if (i0 + idx / RW < n_q) dst[idx] = stage[idx];
+      stage[idx] = 0u;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ BLOCK store
+// A CTA of 128 * (G / 32) threads quantises one group of G tokens x 128 channels per iteration: thread
+// (channel c, chunk k) owns tokens 32k .. 32k+31 of channel c, read from an fp16 tile in shared memory that
+// the CTA fills with coalesced loads.  Packed chunks are assembled in shared memory and stored coalesced.
+template <int BITS, bool NORM>
+__global__ void __launch_bounds__(512) quantize_blocks_prefill_kernel(Layout L, Store S, const __half* __restrict__ X,
+                                                                      int N, int n_q, unsigned char* __restrict__ cache,
+                                                                      const float* __restrict__ inv_norm) {
+  constexpr int PB = BITS == 3 ? 2 : BITS;
+  constexpr int CW = 128 * BITS;                // words per packed chunk
+  extern __shared__ __align__(16) unsigned char smem_q[];
+  const int G = L.G, CH = G >> 5, nthr = 128 * CH;
+  __half* tile = reinterpret_cast<__half*>(smem_q);                               // [G][128]
+  uint32_t* words = reinterpret_cast<uint32_t*>(smem_q + (size_t)G * kD * 2);     // [CH][CW]
+  float4* red = reinterpret_cast<float4*>(words + CH * CW);                       // [CH][128]: mn, mx, ea, es
+  const int u = blockIdx.y, tid = threadIdx.x, c = tid & 127, k = tid >> 7;
+  const float inv = NORM ? inv_norm[(size_t)u * kD + c] : 1.0f;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD;
+  // positions (see block_pos_plane): fragment coordinates of this channel
+  const int m = 4 * (c >> 6) + ((c >> 1) & 3), gid = (c >> 3) & 7, rh = c & 1;
+  const int base_lo = (m >> 2) * 128 + 16 * gid + (m & 3);                        // + 4 * tid4 (+ 256 * k-step for 4 bits)
+  const int base_hi = chunk_hi_plane_word() + 16 * gid + (m >> 1);
+  const int sh_lo = 8 * rh, sh_hi = 4 * (2 * (m & 1) + rh);
+  for (int i = tid; i < CH * CW; i += nthr) words[i] = 0u;
+  for (int j = blockIdx.x; j < n_q / G; j += gridDim.x) {
+    const uint4* src = reinterpret_cast<const uint4*>(Xu + (size_t)j * G * kD);
+    for (int i = tid; i < G * 16; i += nthr) reinterpret_cast<uint4*>(tile)[i] = __ldg(src + i);
+    __syncthreads();
+    float x[kSeg];
+#pragma unroll
+    for (int t = 0; t < kSeg; ++t) {
+      x[t] = __half2float(tile[(kSeg * k + t) * kD + c]);
+      if constexpr (NORM) x[t] = __fmul_rn(x[t], inv);
+    }
+    float mn, mx;
+    seg_minmax(x, mn, mx);
+    if (CH > 1) {
+      red[k * 128 + c] = make_float4(mn, mx, 0.f, 0.f);
+      __syncthreads();
+      for (int kk = 0; kk < CH; ++kk) {
+        const float4 o = red[kk * 128 + c];
+        mn = fminf(mn, o.x); mx = fmaxf(mx, o.y);
+      }
+    }
+    const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
+    const SegCoder sc(p);
+    bool asym = S.mode == 1;
+    if (S.mode == 2) {
+      float ea, es;
+      seg_errors(sc, x, ea, es);
+      if (CH > 1) {
+        red[k * 128 + c].z = ea;
+        red[k * 128 + c].w = es;
+        __syncthreads();
+        ea = 0.f; es = 0.f;
+        for (int kk = 0; kk < CH; ++kk) {
+          const float4 o = red[kk * 128 + c];
+          ea += o.z; es += o.w;
+        }
+      }
+      asym = ea < es;
+    }
+    uint32_t lw[PB == 4 ? 8 : 4], hw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < (PB == 4 ? 8 : 4); ++i) lw[i] = 0u;
+    const ChosenCoder cc(sc, asym);
+#pragma unroll
+    for (int t = 0; t < kSeg; ++t) {
+      const uint32_t code = cc.code_bits(x[t]);
+      const BitPos lo = block_pos_plane(t, 0, PB);       // constants: channel 0's positions
+      const int li = PB == 4 ? (lo.word >> 8) * 4 + ((lo.word >> 2) & 3) : (lo.word >> 2) & 3;   // (k-step,) tid4
+      lw[li] |= (code & ((1u << PB) - 1u)) << lo.bit;
+      if constexpr (BITS == 3) {
+        const BitPos hi = block_pos_plane(t, 0, 1);
+        hw[(hi.word >> 2) & 3] |= ((code >> 2) & 1u) << hi.bit;
+      }
+    }
+    uint32_t* wk = words + k * CW;
+#pragma unroll
+    for (int i = 0; i < (PB == 4 ? 8 : 4); ++i)
+      atomicOr(&wk[base_lo + 4 * (i & 3) + 256 * (i >> 2)], lw[i] << sh_lo);
+    if constexpr (BITS == 3) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) atomicOr(&wk[base_hi + 4 * i], hw[i] << sh_hi);
+    }
+    if (k == 0) store_meta(rec + block_meta_off(S, j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
+    __syncthreads();
+    for (int i = tid; i < CH * CW; i += nthr) {
+      const int ch = i / CW;
+      reinterpret_cast<uint32_t*>(rec + block_code_off(S, j * CH + ch))[i - ch * CW] = words[i];
+      words[i] = 0u;
+    }
+    __syncthreads();       // tile, words and red are free again
+  }
+}
+
+}  // namespace
+
+static inline int grid_cap(int n, int cap) { return n < 1 ? 1 : (n > cap ? cap : n); }
+
+template <int BITS>
+static int launch_store_bits(const Layout& L, const Store& S, const __half* X, int N, int n_q, unsigned char* cache,
+                             const float* inv_norm, cudaStream_t st) {
+  if (S.kind == kRow) {
+    // a warp takes batches of 8 tokens; several batches per warp amortise its set-up (32 reciprocal norms)
+    const int n_batches = (n_q + 7) / 8;
+    const int per_unit = grid_cap((n_batches + 4 * 8 - 1) / (4 * 8), grid_cap(148 * 16 / L.U, 1 << 16));
+    dim3 grid(per_unit, L.U);
+    if (inv_norm) quantize_rows_prefill_kernel<BITS, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
+    else quantize_rows_prefill_kernel<BITS, false><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
+  } else {
+    const int CH = L.G / kChunk;
+    const int smem = L.G * kD * 2 + CH * 128 * BITS * 4 + CH * 128 * 16;
+    auto kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true> : quantize_blocks_prefill_kernel<BITS, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
+    const int n_groups = n_q / L.G;
+    dim3 grid(grid_cap(n_groups, grid_cap(148 * 8 / L.U, 1 << 16)), L.U);
+    kern<<<grid, 128 * CH, smem, st>>>(L, S, X, N, n_q, cache, inv_norm);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// Quantises rows / groups [0, n_q) of every unit of store S from the prefill input X ([U][N][128] fp16; the token
+// of row i is w_sink + i).  inv_norm: reciprocal key norms [U][128], or null for unnormalised values.
+int launch_quantize_store_prefill(const Layout& L, const Store& S, const __half* X, int N, int n_q, unsigned char* cache,
+                                  const float* inv_norm, cudaStream_t st) {
+  if (S.bits == 2) return launch_store_bits<2>(L, S, X, N, n_q, cache, inv_norm, st);
+  if (S.bits == 3) return launch_store_bits<3>(L, S, X, N, n_q, cache, inv_norm, st);
+  if (S.bits == 4) return launch_store_bits<4>(L, S, X, N, n_q, cache, inv_norm, st);
+  return -1;
+}
+
+}  // namespace iq
