@@ -25,20 +25,28 @@ struct SegCoder {
     z_a = p.z_a; inv_a = p.inv_a; s_a = p.s_a; lo_a = kMagic; hi_a = kMagic + p.L;
     inv_s = p.inv_s; s_s = p.s_s; off_s = kMagic + p.half; lo_s = off_s + p.q_lo; hi_s = off_s + p.q_hi;
   }
-  // clamped code plus magic (asymmetric) / plus magic + 2^(b-1) (symmetric): the low mantissa bits are the stored code
-  __device__ __forceinline__ float asym(float x) const {
+  // code plus magic (asymmetric) / plus magic + 2^(b-1) (symmetric): the low mantissa bits are the stored code.
+  // CLAMP = false leaves out the clamp to the code range, for groups where no_clip() holds.
+  template <bool CLAMP> __device__ __forceinline__ float asym(float x) const {
     const float t = __fadd_rn(__fmul_rn(__fsub_rn(x, z_a), inv_a), kMagic);
-    return fminf(fmaxf(t, lo_a), hi_a);
+    return CLAMP ? fminf(fmaxf(t, lo_a), hi_a) : t;
   }
-  __device__ __forceinline__ float sym(float x) const {
+  template <bool CLAMP> __device__ __forceinline__ float sym(float x) const {
     const float t = __fadd_rn(__fmul_rn(x, inv_s), off_s);
-    return fminf(fmaxf(t, lo_s), hi_s);
+    return CLAMP ? fminf(fmaxf(t, lo_s), hi_s) : t;
+  }
+  // Both coders are non-decreasing in x (each step is a correctly rounded monotone operation and the reciprocal
+  // scales are >= 0), so if the group's minimum and maximum land inside the code range, every value does.
+  __device__ __forceinline__ bool no_clip(float mn, float mx) const {
+    return asym<false>(mn) >= lo_a && asym<false>(mx) <= hi_a && sym<false>(mn) >= lo_s && sym<false>(mx) <= hi_s;
   }
   // L1 reconstruction errors of one value (used only to pick the mode of a hybrid group)
-  __device__ __forceinline__ float err_asym(float x) const {
-    return fabsf(__fmaf_rn(-s_a, asym(x) - kMagic, __fsub_rn(x, z_a)));
+  template <bool CLAMP> __device__ __forceinline__ float err_asym(float x) const {
+    return fabsf(__fmaf_rn(-s_a, asym<CLAMP>(x) - kMagic, __fsub_rn(x, z_a)));
   }
-  __device__ __forceinline__ float err_sym(float x) const { return fabsf(__fmaf_rn(-s_s, sym(x) - off_s, x)); }
+  template <bool CLAMP> __device__ __forceinline__ float err_sym(float x) const {
+    return fabsf(__fmaf_rn(-s_s, sym<CLAMP>(x) - off_s, x));
+  }
 };
 
 // The coder of the chosen mode as one formula, clamp(((x - z) * inv) + off): symmetric is z = 0 (x - 0 is exact).
@@ -47,27 +55,97 @@ struct ChosenCoder {
   __device__ __forceinline__ ChosenCoder(const SegCoder& c, bool asym)
       : z(asym ? c.z_a : 0.f), inv(asym ? c.inv_a : c.inv_s), off(asym ? kMagic : c.off_s), lo(asym ? c.lo_a : c.lo_s),
         hi(asym ? c.hi_a : c.hi_s) {}
-  __device__ __forceinline__ uint32_t code_bits(float x) const {     // the code is in the low mantissa bits
+  // bits of (1.5 * 2^23 + code): 0x4B400000 + code
+  template <bool CLAMP> __device__ __forceinline__ uint32_t code_bits(float x) const {
     const float t = __fadd_rn(__fmul_rn(__fsub_rn(x, z), inv), off);
-    return __float_as_uint(fminf(fmaxf(t, lo), hi));
+    return __float_as_uint(CLAMP ? fminf(fmaxf(t, lo), hi) : t);
   }
 };
 
-// min / max of 32 registers
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float r;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// min / max of 32 registers (three-input min / max: two values per instruction)
 __device__ __forceinline__ void seg_minmax(const float (&x)[kSeg], float& mn, float& mx) {
-  mn = x[0]; mx = x[0];
+  float a = fminf(x[0], x[1]), b = fmaxf(x[0], x[1]);
 #pragma unroll
-  for (int e = 1; e < kSeg; ++e) { mn = fminf(mn, x[e]); mx = fmaxf(mx, x[e]); }
+  for (int e = 2; e < kSeg; e += 2) { a = min3(a, x[e], x[e + 1]); b = max3(b, x[e], x[e + 1]); }
+  mn = a; mx = b;
 }
 
+template <bool CLAMP>
 __device__ __forceinline__ void seg_errors(const SegCoder& sc, const float (&x)[kSeg], float& ea, float& es) {
   float a0 = 0.f, a1 = 0.f, s0 = 0.f, s1 = 0.f;
 #pragma unroll
   for (int e = 0; e < kSeg; e += 2) {
-    a0 += sc.err_asym(x[e]); a1 += sc.err_asym(x[e + 1]);
-    s0 += sc.err_sym(x[e]);  s1 += sc.err_sym(x[e + 1]);
+    a0 += sc.template err_asym<CLAMP>(x[e]); a1 += sc.template err_asym<CLAMP>(x[e + 1]);
+    s0 += sc.template err_sym<CLAMP>(x[e]);  s1 += sc.template err_sym<CLAMP>(x[e + 1]);
   }
   ea = a0 + a1; es = s0 + s1;
+}
+
+constexpr uint32_t kMagicBits = 0x4B400000u;     // bit pattern of kMagic
+
+// Packs the 32 codes of a ROW-store segment into its local words (positions of segment 0, see the kernel).
+// Codes arrive as kMagicBits + code; with 2 or 4 bits the fields are filled by wrap-around adds of the shifted
+// patterns, the shifted kMagicBits being taken off at the end (a compile-time constant per word).
+template <int BITS, bool CLAMP>
+__device__ __forceinline__ void pack_row_segment(const ChosenCoder& cc, const float (&x)[kSeg], uint32_t (&lw)[4],
+                                                 uint32_t (&hw)[4]) {
+  constexpr int PB = BITS == 3 ? 2 : BITS, WM = PB == 2 ? 2 : 4;
+  uint32_t cw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { lw[i] = 0u; hw[i] = 0u; }
+#pragma unroll
+  for (int e = 0; e < kSeg; ++e) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[e]);
+    const BitPos lo = row_pos_plane(e, PB);            // constants: segment 0's positions
+    if constexpr (BITS == 3) {
+      const BitPos hi = row_pos_plane(e, 1);
+      lw[lo.word / WM] |= (code & 3u) << lo.bit;
+      hw[hi.word] |= ((code >> 2) & 1u) << hi.bit;
+    } else {
+      lw[lo.word / WM] += code << lo.bit;
+      cw[lo.word / WM] += kMagicBits << lo.bit;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) lw[i] -= cw[i];
+}
+
+// Same for a BLOCK-store segment (32 tokens of one channel; positions of channel 0).
+template <int BITS, bool CLAMP>
+__device__ __forceinline__ void pack_block_segment(const ChosenCoder& cc, const float (&x)[kSeg],
+                                                   uint32_t (&lw)[BITS == 4 ? 8 : 4], uint32_t (&hw)[4]) {
+  constexpr int PB = BITS == 3 ? 2 : BITS, NW = PB == 4 ? 8 : 4;
+  uint32_t cw[NW];
+#pragma unroll
+  for (int i = 0; i < NW; ++i) { lw[i] = 0u; cw[i] = 0u; }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) hw[i] = 0u;
+#pragma unroll
+  for (int t = 0; t < kSeg; ++t) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[t]);
+    const BitPos lo = block_pos_plane(t, 0, PB);       // constants: channel 0's positions
+    const int li = PB == 4 ? (lo.word >> 8) * 4 + ((lo.word >> 2) & 3) : (lo.word >> 2) & 3;   // (k-step,) tid4
+    if constexpr (BITS == 3) {
+      const BitPos hi = block_pos_plane(t, 0, 1);
+      lw[li] |= (code & 3u) << lo.bit;
+      hw[(hi.word >> 2) & 3] |= ((code >> 2) & 1u) << hi.bit;
+    } else {
+      lw[li] += code << lo.bit;
+      cw[li] += kMagicBits << lo.bit;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < NW; ++i) lw[i] -= cw[i];
 }
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* x) {
@@ -143,10 +221,12 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
     }
     const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
     const SegCoder sc(p);
+    const bool no_clip = sc.no_clip(mn, mx);        // the same for all lanes of a group
     bool asym = S.mode == 1;
     if (S.mode == 2) {
       float ea, es;
-      seg_errors(sc, x, ea, es);
+      if (no_clip) seg_errors<false>(sc, x, ea, es);
+      else seg_errors<true>(sc, x, ea, es);
       for (int o = 1; o < gl; o <<= 1) {
         ea += __shfl_xor_sync(0xffffffffu, ea, o);
         es += __shfl_xor_sync(0xffffffffu, es, o);
@@ -154,17 +234,9 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
       asym = ea < es;
     }
     const ChosenCoder cc(sc, asym);
-    uint32_t lw[4] = {0u, 0u, 0u, 0u}, hw[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int e = 0; e < kSeg; ++e) {
-      const uint32_t code = cc.code_bits(x[e]);
-      const BitPos lo = row_pos_plane(e, PB);            // constants: segment 0's positions
-      lw[lo.word / WM] |= (code & ((1u << PB) - 1u)) << lo.bit;
-      if constexpr (BITS == 3) {
-        const BitPos hi = row_pos_plane(e, 1);
-        hw[hi.word] |= ((code >> 2) & 1u) << hi.bit;
-      }
-    }
+    uint32_t lw[4], hw[4];
+    if (no_clip) pack_row_segment<BITS, false>(cc, x, lw, hw);
+    else pack_row_segment<BITS, true>(cc, x, lw, hw);
     __syncwarp();                                          // the stage is zero and no longer being read
     uint32_t* row = stage + tk * RW;
 #pragma unroll
@@ -233,10 +305,12 @@ __global__ void __launch_bounds__(512) quantize_blocks_prefill_kernel(Layout L, 
     }
     const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
     const SegCoder sc(p);
+    const bool no_clip = sc.no_clip(mn, mx);
     bool asym = S.mode == 1;
     if (S.mode == 2) {
       float ea, es;
-      seg_errors(sc, x, ea, es);
+      if (no_clip) seg_errors<false>(sc, x, ea, es);
+      else seg_errors<true>(sc, x, ea, es);
       if (CH > 1) {
         red[k * 128 + c].z = ea;
         red[k * 128 + c].w = es;
@@ -249,21 +323,10 @@ __global__ void __launch_bounds__(512) quantize_blocks_prefill_kernel(Layout L, 
       }
       asym = ea < es;
     }
-    uint32_t lw[PB == 4 ? 8 : 4], hw[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int i = 0; i < (PB == 4 ? 8 : 4); ++i) lw[i] = 0u;
     const ChosenCoder cc(sc, asym);
-#pragma unroll
-    for (int t = 0; t < kSeg; ++t) {
-      const uint32_t code = cc.code_bits(x[t]);
-      const BitPos lo = block_pos_plane(t, 0, PB);       // constants: channel 0's positions
-      const int li = PB == 4 ? (lo.word >> 8) * 4 + ((lo.word >> 2) & 3) : (lo.word >> 2) & 3;   // (k-step,) tid4
-      lw[li] |= (code & ((1u << PB) - 1u)) << lo.bit;
-      if constexpr (BITS == 3) {
-        const BitPos hi = block_pos_plane(t, 0, 1);
-        hw[(hi.word >> 2) & 3] |= ((code >> 2) & 1u) << hi.bit;
-      }
-    }
+    uint32_t lw[BITS == 4 ? 8 : 4], hw[4];
+    if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
+    else pack_block_segment<BITS, true>(cc, x, lw, hw);
     uint32_t* wk = words + k * CW;
 #pragma unroll
     for (int i = 0; i < (PB == 4 ? 8 : 4); ++i)
