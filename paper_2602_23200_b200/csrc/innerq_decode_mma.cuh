@@ -152,6 +152,68 @@ template <int KB, int VB, int G, int KM, int VM, int CPI> struct StageLayout {
 };
 
 
+// Cross-CTA merge, run by the last CTA of a unit to finish: log-sum-exp combination of the n_parts partial results
+// (rows of kPartialStride floats: acc[128], max, sum) of nh query heads starting at head_base, fp16 result to out.
+// Kept out of line so that its registers do not add to the streaming loop's.
+__device__ __noinline__ void merge_parts(const float* __restrict__ partials, float* wm, __half* __restrict__ out, int nh,
+                                         int n_parts, int head_base, int max_splits) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // Warp w merges parts w, w + 8, ... (four parts per round of loads, lane l the channels 4l .. 4l+3, running
+  // max / rescale as in the streaming loop), then the eight warp results are combined through shared memory.
+  // The loops over heads and rounds stay rolled: this code runs once per unit on a cold instruction cache,
+  // where its size costs more than its latency.
+#pragma unroll 1
+  for (int h = 0; h < nh; ++h) {
+    float M = -INFINITY, den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+    const float* Ph = partials + (size_t)(head_base + h) * max_splits * kPartialStride;
+#pragma unroll 1
+    for (int s0 = warp; s0 < n_parts; s0 += 4 * kWarps) {
+      float4 v[4];
+      float2 ml[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int s = s0 + e * kWarps;
+        const float* P = Ph + (size_t)(s < n_parts ? s : s0) * kPartialStride;
+        v[e] = __ldcg(reinterpret_cast<const float4*>(P) + lane);
+        ml[e] = __ldcg(reinterpret_cast<const float2*>(P + kD));
+        if (s >= n_parts) ml[e] = make_float2(-INFINITY, 0.f);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float m_new = fmaxf(M, ml[e].x);
+        const float a_old = M == -INFINITY ? 0.f : ex2_approx(M - m_new);
+        const float a_new = ml[e].x == -INFINITY ? 0.f : ex2_approx(ml[e].x - m_new);
+        M = m_new;
+        den = fmaf(den, a_old, ml[e].y * a_new);
+        n0 = fmaf(n0, a_old, v[e].x * a_new);
+        n1 = fmaf(n1, a_old, v[e].y * a_new);
+        n2 = fmaf(n2, a_old, v[e].z * a_new);
+        n3 = fmaf(n3, a_old, v[e].w * a_new);
+      }
+    }
+    float* mine = wm + ((size_t)warp * kHeads + h) * (kD + 2);
+    *reinterpret_cast<float2*>(mine + 4 * lane) = make_float2(n0, n1);
+    *reinterpret_cast<float2*>(mine + 4 * lane + 2) = make_float2(n2, n3);
+    if (lane == 0) { mine[kD] = M; mine[kD + 1] = den; }
+  }
+  __syncthreads();
+  for (int i = tid; i < nh * kD; i += kThreads) {
+    const int h = i >> 7, c = i & (kD - 1);
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wm[((size_t)w * kHeads + h) * (kD + 2) + kD]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float* r_ = wm + ((size_t)w * kHeads + h) * (kD + 2);
+      const float wgt = r_[kD] == -INFINITY ? 0.f : ex2_approx(r_[kD] - M);
+      num = fmaf(r_[c], wgt, num);
+      den = fmaf(r_[kD + 1], wgt, den);
+    }
+    out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
+  }
+}
+
 // ---- the kernel -------------------------------------------------------------------------------------
 // CPI = chunks (of 32 tokens) a warp processes per loop iteration: one barrier wait, one soft-max update and
 // one refill per iteration, and CPI*2 independent key accumulator chains in flight.
@@ -836,38 +898,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   __syncthreads();
   if (s_ticket != gridDim.y - 1) return;
   __threadfence();
-  const float* partials = reinterpret_cast<const float*>(a.ws + L.ws_partial_off);
-  float* mw = reinterpret_cast<float*>(smem);          // [head][part]: max, then weight
-  float* lw = mw + kHeads * 128;                        // [head][part]: l
-  for (int i = tid; i < nh * n_parts; i += kThreads) {
-    const int h = i / n_parts, s = i % n_parts;
-    const float* P = partials + ((size_t)(head_base + h) * L.max_splits + s) * kPartialStride;
-    mw[h * 128 + s] = __ldcg(P + kD);
-    lw[h * 128 + s] = __ldcg(P + kD + 1);
-  }
-  __syncthreads();
-  for (int i = tid; i < nh * kD; i += kThreads) {
-    const int h = i >> 7, c = i & (kD - 1);
-    const float* P = partials + (size_t)(head_base + h) * L.max_splits * kPartialStride + c;
-    float M = -INFINITY;
-    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, mw[h * 128 + s]);
-    float num = 0.f, den = 0.f;
-    for (int s0 = 0; s0 < n_parts; s0 += 16) {          // sixteen independent loads in flight
-      float v[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) v[e] = s0 + e < n_parts ? __ldcg(P + (size_t)(s0 + e) * kPartialStride) : 0.f;
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        if (s0 + e < n_parts) {
-          const float ms = mw[h * 128 + s0 + e];
-          const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - M);
-          num = fmaf(v[e], wgt, num);
-          den = fmaf(lw[h * 128 + s0 + e], wgt, den);
-        }
-      }
-    }
-    a.out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
-  }
+  merge_parts(reinterpret_cast<const float*>(a.ws + L.ws_partial_off), reinterpret_cast<float*>(smem), a.out, nh, n_parts,
+              head_base, L.max_splits);
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
 }
 

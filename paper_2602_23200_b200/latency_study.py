@@ -1,0 +1,131 @@
+"""Decode latency over context length for the paper's presets (Section "Latency", Tables of dequantisation
+latencies and the hybrid ablation), on the shape of one decoder layer of an 8B-class GQA model:
+batch 1, 32 query heads, 8 KV heads, head_dim 128, group 32, sink 32, recent 96.
+
+Presets: Base (3-bit symmetric K and V), Hybrid (3-bit symmetric K, 2-bit hybrid V), Small (3-bit symmetric K,
+2-bit symmetric V), the 2-bit and 4-bit hybrid caches of the benchmark configurations, an outer-grouped
+(per-channel K, per-token V) 2-bit cache and the unquantised fp16 cache.  The hybrid mask density cannot be
+forced from outside (it is decided by the data), so the mask rows use the two readings of the symmetric formula
+and the all-asymmetric mode to reach about 0 %, 2 %, 93 % and 100 % flagged groups; the measured fraction is
+printed.  Key side and value side are one fused kernel here and are not timed separately.
+
+    python -m paper_2602_23200_b200.latency_study [--out table.md] [--lengths 512,4096,32768]
+
+Each cell is the time of one innerq_decode_attention call: "cold" with L2 flushed before the call (CUDA events
+around the single launch, median of `--reps`), "warm" as the mean of back-to-back calls on the same cache.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+import sys
+
+import numpy as np
+
+from . import synth
+
+PRESETS = [
+    # name, overrides
+    ("Base K3s/V3s", dict(k_bits=3, v_bits=3, k_mode=synth.SYM, v_mode=synth.SYM)),
+    ("Hybrid K3s/V2h", dict(k_bits=3, v_bits=2, k_mode=synth.SYM, v_mode=synth.HYBRID)),
+    ("Small K3s/V2s", dict(k_bits=3, v_bits=2, k_mode=synth.SYM, v_mode=synth.SYM)),
+    ("2-bit hybrid", dict(k_bits=2, v_bits=2)),
+    ("2-bit hybrid, literal sym", dict(k_bits=2, v_bits=2, sym_variant=1)),
+    ("2-bit all-asym", dict(k_bits=2, v_bits=2, k_mode=synth.ASYM, v_mode=synth.ASYM)),
+    ("2-bit all-sym", dict(k_bits=2, v_bits=2, k_mode=synth.SYM, v_mode=synth.SYM)),
+    ("4-bit hybrid", dict(k_bits=4, v_bits=4)),
+    ("outer-grouped 2-bit", dict(k_bits=2, v_bits=2, grouping=synth.OUTER, k_normalize=0, k_mode=synth.ASYM,
+                                 v_mode=synth.ASYM)),
+    ("fp16", dict(grouping=synth.FP16, k_normalize=0)),
+]
+
+
+def layer_workload(n_tokens: int, **kw) -> synth.Workload:
+    base = synth.Workload("layer8b", 21, batch=1, n_q_heads=32, n_kv_heads=8, n_tokens=n_tokens, group=32,
+                          w_sink=32, w_recent=96, v_dist="student_t4", n_hashed_outliers=3, outlier_lo=10.0,
+                          outlier_hi=30.0)
+    return base.with_(**kw)
+
+
+def time_decode(cache, q, out, flush, reps: int):
+    import torch
+    for _ in range(3):
+        cache.innerq_decode_attention(q, out)
+    torch.cuda.synchronize()
+    cold = []
+    for _ in range(reps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cache.innerq_decode_attention(q, out)
+        e1.record()
+        torch.cuda.synchronize()
+        cold.append(e0.elapsed_time(e1) * 1e3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 4 * reps
+    e0.record()
+    for _ in range(n):
+        cache.innerq_decode_attention(q, out)
+    e1.record()
+    torch.cuda.synchronize()
+    return statistics.median(cold), e0.elapsed_time(e1) * 1e3 / n
+
+
+def asym_fraction(cache, which: str) -> float:
+    e = cache.innerq_cache_export(codes=False)
+    s = e.get(which)
+    if s is None or s.size == 0:
+        return float("nan")
+    return float(((s & 0x8000) != 0).mean())
+
+
+def main(argv=None) -> int:
+    ap = argparse.ArgumentParser(description=__doc__.split("\n\n")[0])
+    ap.add_argument("--lengths", default="512,1024,2048,4096,8192,16384,32768")
+    ap.add_argument("--reps", type=int, default=15)
+    ap.add_argument("--out", default="")
+    args = ap.parse_args(argv)
+    import torch
+    from . import binding as B
+
+    lengths = [int(x) for x in args.lengths.split(",")]
+    n_max = max(lengths)
+    K, V = synth.kv_all(layer_workload(n_max))
+    Kd, Vd = torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than L2
+    rows, records = [], []
+    for name, kw in PRESETS:
+        cells = []
+        frac_v = float("nan")
+        for n in lengths:
+            w = layer_workload(n, **kw)
+            cache = B.InnerQCache(B.make_config(w, max_tokens=n + 64))
+            cache.innerq_quantize_prefill(Kd[:, :, :n].contiguous(), Vd[:, :, :n].contiguous())
+            q = torch.from_numpy(synth.query(w)).cuda()
+            out = torch.empty_like(q)
+            cold, warm = time_decode(cache, q, out, flush, args.reps)
+            if cache.innerq_read_device_error() != 0:
+                raise RuntimeError("a bounded wait inside the decode kernel ran out")
+            if n == n_max and w.grouping == synth.INNER:
+                frac_v = asym_fraction(cache, "v_scale")
+            cells.append((cold, warm))
+            records.append({"preset": name, "n_tokens": n, "cold_us": round(cold, 2), "warm_us": round(warm, 2)})
+            cache.close()
+        rows.append((name, frac_v, cells))
+        print(f"{name:28s} " + " ".join(f"{c:7.1f}/{wm:<7.1f}" for c, wm in cells), flush=True)
+    lines = ["| preset (asym fraction of V groups) | " + " | ".join(str(n) for n in lengths) + " |",
+             "|---|" + "---|" * len(lengths)]
+    for name, fv, cells in rows:
+        tag = name if np.isnan(fv) else f"{name} ({100 * fv:.0f} %)"
+        lines.append(f"| {tag} | " + " | ".join(f"{c:.1f} / {wm:.1f}" for c, wm in cells) + " |")
+    table = "\n".join(lines)
+    print("\nµs per decode call, cold (L2 flushed) / warm (back to back):\n" + table)
+    if args.out:
+        with open(args.out, "w") as f:
+            f.write(table + "\n\n" + "\n".join(json.dumps(r) for r in records) + "\n")
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
