@@ -179,60 +179,71 @@ __global__ void copy_window_kernel(Layout L, Store S, const __half* __restrict__
 // N is the token count after this append.  Which evictions happen is a function of N alone.
 // One CTA of 128 threads per unit.  The per-step work (ring writes, eviction of one ROW-store token) is a chain of
 // dependent memory accesses, so everything whose address is known up front is requested at once: the new key and
-// value rows, the evicted token's row (in the ring since w_recent steps, or the new row itself if w_recent = 0) and
-// the key norms.  Warp 0 quantises the ROW store's evicted token while the others write the rings; the BLOCK
+// value rows, the evicted token's row (in the ring since w_recent steps, or the new row itself if w_recent = 0)
+// and the key norms.  Warp 0 quantises the ROW store's evicted token while the others write the rings; the BLOCK
 // store's eviction (G tokens, every G steps) then runs on the whole CTA.
+
+// ROW store: eviction of its oldest recent token, if this append causes one (warp 0 only).
+__device__ __forceinline__ void append_evict_row(const Layout& L, const Store& R, const __half* __restrict__ x_new, int N,
+                                                 int u, unsigned char* __restrict__ cache, bool use_norm, uint32_t* words) {
+  const int t_new = N - 1;
+  if (R.kind != kRow || t_new < L.w_sink || threadIdx.x >= 32) return;
+  const int nq_before = n_quantised(kRow, N - 1, L.w_sink, L.w_recent, L.G);
+  if (n_quantised(kRow, N, L.w_sink, L.w_recent, L.G) == nq_before) return;
+  const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
+  const float* norm = reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD;
+  float inv4[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) inv4[e] = use_norm ? __fdiv_rn(1.0f, norm[4 * threadIdx.x + e]) : 1.0f;
+  unsigned char* rec = cache + R.rec_off + (size_t)u * R.rec_unit_stride;
+  TokSrc src{ring, R.ring_cap, L.w_sink};
+  // with an empty recent window the evicted token is the new one, which is not in the ring yet
+  const __half* row = L.w_sink + nq_before == t_new ? x_new : src.row(L.w_sink + nq_before);
+  quantize_row_warp(row, use_norm ? inv4 : nullptr, L, R, words, reinterpret_cast<uint32_t*>(rec + row_code_off(R, nq_before)),
+                    rec + row_meta_off(R, nq_before), 0);
+}
+
+// The new token goes to the sink or the ring of the store.
+__device__ __forceinline__ void append_write(const Layout& L, const Store& R, __half x, int N, int u,
+                                             unsigned char* __restrict__ cache) {
+  const int t_new = N - 1;
+  __half* sink = reinterpret_cast<__half*>(cache + R.sink_off + (size_t)u * R.sink_stride);
+  __half* ring = reinterpret_cast<__half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
+  if (R.kind == kNone || t_new < L.w_sink) sink[(size_t)t_new * kD + threadIdx.x] = x;
+  else ring[(size_t)((t_new - L.w_sink) % R.ring_cap) * kD + threadIdx.x] = x;
+}
+
+// BLOCK store: every G steps the oldest G tokens of its ring (the row written by this append may be among them).
+__device__ __forceinline__ void append_evict_block(const Layout& L, const Store& R, int N, int u,
+                                                   unsigned char* __restrict__ cache, bool use_norm, __half* tile,
+                                                   uint32_t* words) {
+  if (R.kind != kBlock || N - 1 < L.w_sink) return;
+  const int nq_before = n_quantised(kBlock, N - 1, L.w_sink, L.w_recent, L.G);
+  if (n_quantised(kBlock, N, L.w_sink, L.w_recent, L.G) == nq_before) return;
+  __syncthreads();
+  const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
+  const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
+  TokSrc src{ring, R.ring_cap, L.w_sink};
+  quantize_block_cta(src, L.w_sink + nq_before, norm, L, R, tile, words, cache + R.rec_off + (size_t)u * R.rec_unit_stride,
+                     nq_before / L.G);
+}
+
 __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
                                                      const __half* __restrict__ v_new, int N,
                                                      unsigned char* __restrict__ cache) {
   __shared__ __align__(16) __half tile[128 * kD];
   __shared__ uint32_t words[4 * 512];
-  const int u = blockIdx.x, tid = threadIdx.x;
-  const Store* S[2] = {&L.k, &L.v};
-  const __half* x_new[2] = {k_new + (size_t)u * kD, v_new + (size_t)u * kD};
-  const __half xv[2] = {x_new[0][tid], x_new[1][tid]};
-  const int t_new = N - 1;
-  // ---- ROW store (at most one of the two): its eviction, by warp 0, from registers filled before any store
-  for (int i = 0; i < 2; ++i) {
-    const Store& R = *S[i];
-    if (R.kind != kRow || t_new < L.w_sink || tid >= 32) continue;
-    const int nq_before = n_quantised(kRow, N - 1, L.w_sink, L.w_recent, L.G);
-    if (n_quantised(kRow, N, L.w_sink, L.w_recent, L.G) == nq_before) continue;
-    const bool use_norm = i == 0 && L.k_normalize != 0;
-    const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
-    const float* norm = reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD;
-    float inv4[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) inv4[e] = use_norm ? __fdiv_rn(1.0f, norm[4 * tid + e]) : 1.0f;
-    unsigned char* rec = cache + R.rec_off + (size_t)u * R.rec_unit_stride;
-    TokSrc src{ring, R.ring_cap, L.w_sink};
-    // with an empty recent window the evicted token is the new one, which is not in the ring yet
-    const __half* row = L.w_sink + nq_before == t_new ? x_new[i] : src.row(L.w_sink + nq_before);
-    quantize_row_warp(row, use_norm ? inv4 : nullptr, L, R, words,
-                      reinterpret_cast<uint32_t*>(rec + row_code_off(R, nq_before)), rec + row_meta_off(R, nq_before), 0);
-  }
-  // ---- the new token goes to the sink or the ring of both stores
-  for (int i = 0; i < 2; ++i) {
-    const Store& R = *S[i];
-    __half* sink = reinterpret_cast<__half*>(cache + R.sink_off + (size_t)u * R.sink_stride);
-    __half* ring = reinterpret_cast<__half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
-    if (R.kind == kNone || t_new < L.w_sink) sink[(size_t)t_new * kD + tid] = xv[i];
-    else ring[(size_t)((t_new - L.w_sink) % R.ring_cap) * kD + tid] = xv[i];
-  }
-  // ---- BLOCK store: every G steps the oldest G tokens of its ring (the row written above may be among them)
-  for (int i = 0; i < 2; ++i) {
-    const Store& R = *S[i];
-    if (R.kind != kBlock || t_new < L.w_sink) continue;
-    const int nq_before = n_quantised(kBlock, N - 1, L.w_sink, L.w_recent, L.G);
-    if (n_quantised(kBlock, N, L.w_sink, L.w_recent, L.G) == nq_before) continue;
-    __syncthreads();
-    const bool use_norm = i == 0 && L.k_normalize != 0;
-    const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
-    const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
-    TokSrc src{ring, R.ring_cap, L.w_sink};
-    quantize_block_cta(src, L.w_sink + nq_before, norm, L, R, tile, words,
-                       cache + R.rec_off + (size_t)u * R.rec_unit_stride, nq_before / L.G);
-  }
+  const int u = blockIdx.x;
+  const __half* xk = k_new + (size_t)u * kD;
+  const __half* xv = v_new + (size_t)u * kD;
+  const __half k_x = xk[threadIdx.x], v_x = xv[threadIdx.x];
+  const bool k_norm = L.k_normalize != 0;
+  append_evict_row(L, L.k, xk, N, u, cache, k_norm, words);
+  append_evict_row(L, L.v, xv, N, u, cache, false, words);
+  append_write(L, L.k, k_x, N, u, cache);
+  append_write(L, L.v, v_x, N, u, cache);
+  append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
+  append_evict_block(L, L.v, N, u, cache, false, tile, words);
 }
 
 // ------------------------------------------------------------------ canonical export
