@@ -135,6 +135,25 @@ int innerq_append_token(innerq_cache_t* cache, const void* k_new, const void* v_
  * not overlap.  Errors: INVALID_ARG (N == 0 included), CUDA. */
 int innerq_decode_attention(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
 
+/* One decode step from HOST buffers (the sequence the paper's Section "Latency" times per generated token:
+ * quantise-on-evict of the step's own token, then attention over the cache): enqueues on `cuda_stream`
+ *   host -> device copies of k_new, v_new ([batch][n_kv_heads][head_dim] fp16) and q ([batch][n_q_heads][head_dim]),
+ *   innerq_append_token, innerq_decode_attention, device -> host copy of out ([batch][n_q_heads][head_dim] fp16).
+ * `dev_staging` is caller-owned device memory of at least innerq_step_staging_bytes(cfg) bytes, 256-byte aligned,
+ * used for the device copies of the four tensors; it must stay untouched until the stream has passed this step.
+ * If all four host buffers are pinned (page-locked and mapped, e.g. cudaHostAlloc / cudaHostRegister), the kernels
+ * read the inputs and write the result in place over the bus and no copy is enqueued; otherwise the tensors are
+ * staged through `dev_staging` with one copy each (pageable memory makes those copies block the caller).
+ * `out_host` holds the result once `cuda_stream` has been synchronised.  The call itself does not synchronise
+ * and allocates nothing.  INVALID_ARG and CAPACITY are detected before anything is enqueued; after a CUDA error
+ * the step may be partly enqueued.
+ * Errors: INVALID_ARG, CAPACITY, UNSUPPORTED, CUDA. */
+int innerq_decode_step_host(innerq_cache_t* cache, const void* k_new_host, const void* v_new_host, const void* q_host,
+                            void* out_host, void* dev_staging, void* cuda_stream);
+
+/* Bytes of device staging innerq_decode_step_host needs for this configuration.  Errors: INVALID_ARG. */
+int innerq_step_staging_bytes(const innerq_config_t* cfg, size_t* bytes);
+
 /* Same computation and arguments as innerq_decode_attention, for callers that cannot give the decode
  * step any scratch memory of their own.  (The paper has no counterpart; this is an integration aid.)
  * Typical cases: the workspace passed to innerq_cache_create was only lent for the prefill and has gone

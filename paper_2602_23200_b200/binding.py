@@ -22,7 +22,7 @@ GROUPING_INNER, GROUPING_OUTER, GROUPING_FP16 = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "innerq_cache_bytes", "innerq_token_payload_bytes", "innerq_cache_create", "innerq_cache_destroy",
     "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
-    "innerq_decode_attention_static",
+    "innerq_decode_attention_static", "innerq_decode_step_host", "innerq_step_staging_bytes",
     "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
     L.innerq_append_token.argtypes = [vp, vp, vp, vp]
     L.innerq_decode_attention.argtypes = [vp, vp, vp, vp]
     L.innerq_decode_attention_static.argtypes = [vp, vp, vp, vp]
+    L.innerq_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.innerq_step_staging_bytes.argtypes = [cfgp, C.POINTER(sz)]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
@@ -209,6 +211,26 @@ class InnerQCache:
         _check(lib().innerq_decode_attention_static(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
                                                     _stream_ptr(stream)), "innerq_decode_attention_static")
         return out
+
+    def innerq_decode_step_host(self, k_new_host, v_new_host, q_host, out_host, stream=None):
+        """One step (append + decode) from pinned host tensors into a pinned host tensor; enqueues only, the
+        caller synchronises the stream before reading `out_host`.  The device staging buffer the C call needs
+        is a torch allocation made here on first use."""
+        import torch
+        c = self.cfg
+        kv_shape, q_shape = (c.batch, c.n_kv_heads, c.head_dim), (c.batch, c.n_q_heads, c.head_dim)
+        for t, name, shape in ((k_new_host, "k_new_host", kv_shape), (v_new_host, "v_new_host", kv_shape),
+                               (q_host, "q_host", q_shape), (out_host, "out_host", q_shape)):
+            if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == torch.float16 and t.is_contiguous()
+                    and tuple(t.shape) == shape):
+                raise TypeError(f"{name} must be a contiguous host fp16 tensor of shape {shape}")
+        if getattr(self, "_staging", None) is None:
+            n = C.c_size_t()
+            _check(lib().innerq_step_staging_bytes(C.byref(c), C.byref(n)), "innerq_step_staging_bytes")
+            self._staging = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+        _check(lib().innerq_decode_step_host(self._h, k_new_host.data_ptr(), v_new_host.data_ptr(), q_host.data_ptr(),
+                                             out_host.data_ptr(), self._staging.data_ptr(), _stream_ptr(stream)),
+               "innerq_decode_step_host")
 
     def innerq_set_decode_options(self, n_splits: int = 0, variant: int = 0):
         _check(lib().innerq_set_decode_options(self._h, n_splits, variant), "innerq_set_decode_options")

@@ -244,6 +244,57 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   return INNERQ_OK;
 }
 
+// ---- one step from host buffers ----------------------------------------------------------------------
+static size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+int innerq_step_staging_bytes(const innerq_config_t* cfg, size_t* bytes) {
+  if (!cfg || !bytes || check_config(cfg) != INNERQ_OK) return INNERQ_ERR_INVALID_ARG;
+  const size_t kv = align256((size_t)cfg->batch * cfg->n_kv_heads * cfg->head_dim * 2);
+  const size_t qo = align256((size_t)cfg->batch * cfg->n_q_heads * cfg->head_dim * 2);
+  *bytes = 2 * kv + 2 * qo;
+  return INNERQ_OK;
+}
+
+int innerq_decode_step_host(innerq_cache_t* c, const void* k_new_host, const void* v_new_host, const void* q_host,
+                            void* out_host, void* dev_staging, void* cuda_stream) {
+  if (!c || !k_new_host || !v_new_host || !q_host || !out_host || !dev_staging) return INNERQ_ERR_INVALID_ARG;
+  if (c->N + 1 > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t kv_bytes = (size_t)c->L.U * kD * 2, q_bytes = (size_t)c->L.B * c->L.Hq * kD * 2;
+  unsigned char* d = static_cast<unsigned char*>(dev_staging);
+  unsigned char* dk = d;
+  unsigned char* dv = dk + align256(kv_bytes);
+  unsigned char* dq = dv + align256(kv_bytes);
+  unsigned char* dout = dq + align256(q_bytes);
+  // Pinned (page-locked, mapped) host buffers are addressable by the GPU: the kernels then read the 10-30 KB of
+  // inputs and write the result in place over the bus, and no copy is enqueued at all.  Anything else is staged.
+  const void* src[3] = {k_new_host, v_new_host, q_host};
+  void* mapped[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool zero_copy = true;
+  for (int i = 0; i < 4 && zero_copy; ++i) {
+    cudaPointerAttributes at;
+    const void* p = i < 3 ? src[i] : out_host;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); zero_copy = false; break; }
+    if (at.type != cudaMemoryTypeHost || at.devicePointer == nullptr) zero_copy = false;
+    else mapped[i] = at.devicePointer;
+  }
+  if (zero_copy) {
+    int st = innerq_append_token(c, mapped[0], mapped[1], cuda_stream);
+    if (st != INNERQ_OK) return st;
+    return innerq_decode_attention(c, mapped[2], mapped[3], cuda_stream);
+  }
+  if (cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return INNERQ_ERR_CUDA;
+  int st = innerq_append_token(c, dk, dv, cuda_stream);
+  if (st != INNERQ_OK) return st;
+  st = innerq_decode_attention(c, dq, dout, cuda_stream);
+  if (st != INNERQ_OK) return st;
+  if (cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return INNERQ_ERR_CUDA;
+  return INNERQ_OK;
+}
+
 // ---- decode on library-owned scratch ---------------------------------------------------------------
 // The split partials, merge tickets and error word of the decode kernel normally live in the workspace
 // the caller handed to innerq_cache_create.  This variant keeps them in a fixed array inside the library

@@ -182,6 +182,30 @@ def test_prefill_then_appends_matches_oracle(grouping):
     check_decode(w, oc, gc, step=1000, variants=(0, 1) if grouping == O.INNER else (0,))
 
 
+def test_step_from_host_buffers_matches_separate_calls_and_oracle():
+    # innerq_decode_step_host = copies in + append + decode + copy out; across a value-group eviction
+    torch = _torch()
+    w = synth.tiny(n_tokens=300, k_bits=3, v_bits=2, k_mode=O.SYM, v_mode=O.HYBRID)
+    oc, gc, K, V = run_prefill_both(w)
+    gc2 = gpu_cache(w)
+    gc2.innerq_quantize_prefill(dev(K), dev(V))
+    out_h = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float16).pin_memory()
+    for step in range(40):
+        k1, v1 = synth.new_token(w, step)
+        q = synth.query(w, step)
+        oc.append(k1, v1)
+        pin = (lambda t: t.pin_memory()) if step % 2 == 0 else (lambda t: t)    # in-place over the bus / staged copies
+        gc.innerq_decode_step_host(pin(torch.from_numpy(k1)), pin(torch.from_numpy(v1)), pin(torch.from_numpy(q)), out_h)
+        torch.cuda.synchronize()
+        gc2.innerq_append_token(dev(k1), dev(v1))
+        ref2 = gc2.innerq_decode_attention(dev(q)).cpu()
+        assert torch.equal(out_h, ref2)                       # same kernels, same inputs: identical bits
+        if step % 13 == 0 or step == 39:
+            P.assert_outputs_close(out_h.numpy(), oc.decode(q), f"host step {step}")
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group, False, True)
+    assert gc.n_tokens == 340
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
