@@ -303,16 +303,24 @@ def run_ours(args, w):
     sampler.start()
     time.sleep(0.15)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    dec_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Kst)]
+    # The decode kernel is bracketed by its own events on every 8th step only: an event between append and decode
+    # keeps the decode from being launched as a programmatic dependent of the append, so the other steps run the
+    # way a serving loop would.  The bracketed decodes are the ones the roofline figure is computed from.
+    ev_every = 8
+    dec_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range((Kst + ev_every - 1) // ev_every)]
     barrier()
     ev0.record(stream)
     for j in range(Kst):
         i = W + j
         c = caches[i % R]
         c.innerq_append_token(k_new[i], v_new[i])
-        dec_ev[j][0].record(stream)
-        c.innerq_decode_attention(q_all[i], out)
-        dec_ev[j][1].record(stream)
+        if j % ev_every == 0:
+            dec_ev[j // ev_every][0].record(stream)
+            c.innerq_decode_attention(q_all[i], out)
+            dec_ev[j // ev_every][1].record(stream)
+        else:
+            c.innerq_decode_attention(q_all[i], out)
     ev1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -374,7 +382,7 @@ def run_ours(args, w):
     if rank == 0:
         peak, which = measured_peak_gbs()
         dec_us = float(np.mean(dec_ms)) * 1e3
-        achieved = (bytes_min / Kst) / (dec_us * 1e-6) / 1e9
+        achieved = (bytes_min / Kst) / (dec_us * 1e-6) / 1e9      # bytes per decode vary by < 0.1 % over the steps
         line = {
             "metric": "decode_step_algorithmic_hbm_gbs", "value": value_gbs, "unit": "GB/s", "n_gpus": world,
             "steps": Kst, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
@@ -388,6 +396,11 @@ def run_ours(args, w):
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
+                         "note": "achieved is from decodes bracketed by their own events (every 8th step), which "
+                                 "cannot overlap their neighbours; back to back the same kernel averages "
+                                 "us_per_decode_back_to_back",
+                         "achieved_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9,
+                         "frac_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9 / peak,
                          "kernel": "innerq_decode_attention (split + merge)"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "us_per_step": e2e_s * 1e6, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},

@@ -81,6 +81,10 @@ __device__ __forceinline__ void mma16816_z(float (&c)[4], uint32_t a0, uint32_t 
       : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
+// Programmatic dependent launch: wait for the kernels this one depends on (no-op without the launch attribute);
+// allow the next kernel in the stream to be launched before this one has finished.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -256,18 +260,6 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
   const int n_parts = gridDim.y;
   const bool fast = split < a.n_splits;
-  // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
-  // hundred KB of queued chunk data per SM they would take microseconds to arrive.
-  float q_early[2], n_early[2];
-  {
-    const float* norm_g = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
-      q_early[e] = h < nh ? __half2float(a.q[(size_t)(head_base + h) * kD + c]) : 0.f;
-      n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
-    }
-  }
   // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
   // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
   // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
@@ -343,6 +335,24 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     for (int s = 0; s < NST; ++s) mbar_init(bars_u32 + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  // Everything above touches no global memory: under a programmatic dependent launch it runs while the kernel
+  // before this one in the stream (the step's append, or the previous decode's merge) is still finishing.
+  // From here on its results are needed.
+  grid_dependency_wait();
+  // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
+  // hundred KB of queued chunk data per SM they would take microseconds to arrive.
+  float q_early[2], n_early[2];
+  {
+    const float* norm_g = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
+      q_early[e] = h < nh ? __half2float(a.q[(size_t)(head_base + h) * kD + c]) : 0.f;
+      n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
+    }
+  }
+  if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < NST; ++s)
       if (s < n_iters) issue(s);
@@ -828,6 +838,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       if (lane == 0 && it + NST < n_iters) issue(st);
     }
 
+    grid_launch_dependents();     // the next kernel in the stream may start its own set-up during this epilogue
     if (failed) {
       // a copy never arrived: flag it for the host and contribute nothing
       if (lane == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);
@@ -937,7 +948,15 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   const int step = SPLIT ? 1 : kHeads;
   for (int h0 = 0; h0 < L.r; h0 += step) {
     a.head0 = h0;
-    decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI><<<grid, kThreads, kSmem, st>>>(L, cn, a);
+    // launched as a programmatic dependent of whatever precedes it in the stream: its set-up overlaps that
+    // kernel's tail, its first global access waits for it (grid_dependency_wait)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, L, cn, a) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -234,6 +234,10 @@ __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __r
   __shared__ __align__(16) __half tile[128 * kD];
   __shared__ uint32_t words[4 * 512];
   const int u = blockIdx.x;
+  // Programmatic dependent launch: the decode that follows may set itself up while this kernel runs (it waits
+  // for this kernel's completion before its first global access); this kernel in turn waits for its predecessor.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const __half* xk = k_new + (size_t)u * kD;
   const __half* xv = v_new + (size_t)u * kD;
   const __half k_x = xk[threadIdx.x], v_x = xv[threadIdx.x];
@@ -351,8 +355,13 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
 
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
                   cudaStream_t st) {
-  append_kernel<<<L.U, 128, 0, st>>>(L, k_new, v_new, N_after, cache);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, append_kernel, L, k_new, v_new, N_after, cache) == cudaSuccess ? 1 : -1;
 }
 
 int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st) {
