@@ -48,6 +48,7 @@ void place_store(Store& S, int kind, int bits, int mode, const innerq_config_t& 
   S.kind = kind;
   S.bits = bits;
   S.mode = mode;
+  S.code_kind = kind;
   if (kind == kNone) {
     S.sink_stride = (size_t)c.max_tokens * kD * 2;
     S.sink_off = off;
@@ -92,6 +93,37 @@ void place_records(Store& row, Store& blk, int G, int U, size_t& off) {
   off = align_up(off + unit * U, 256);
 }
 
+// Outer grouping: keys are grouped per channel along tokens (kBlock metadata) but keep one packed row per token,
+// values are grouped per token along channels (kRow metadata) but keep 32-token chunks.  A chunk record holds the
+// key rows, the values' metadata rows and the value chunk; the keys' per-group metadata comes FIRST in the group
+// record, because scores need it from the group's first token on.
+void place_records_outer(Store& k, Store& v, int G, int U, size_t& off) {
+  k.code_kind = kRow;
+  v.code_kind = kBlock;
+  const int row_codes = kChunk * row_bytes(k.bits);
+  const int row_meta = kChunk * v.n_groups * v.meta_bytes;
+  const int blk_codes = chunk_bytes(v.bits);
+  const int blk_meta = kD * k.meta_bytes;
+  const int chunk_stride = row_codes + row_meta + blk_codes;
+  const int cpg = G / kChunk;
+  const int group_stride = blk_meta + cpg * chunk_stride;
+  const size_t unit = align_up((size_t)(v.cap_q / G) * group_stride, 256);
+  Store* both[2] = {&k, &v};
+  for (Store* S : both) {
+    S->rec_off = off;
+    S->rec_unit_stride = unit;
+    S->group_stride = group_stride;
+    S->chunk_stride = chunk_stride;
+    S->chunks_per_group = cpg;
+    S->chunk0 = blk_meta;
+  }
+  k.code_in_rec = 0;
+  k.meta_in_rec = 0;
+  v.meta_in_rec = row_codes;
+  v.code_in_rec = row_codes + row_meta;
+  off = align_up(off + unit * U, 256);
+}
+
 void make_layout(const innerq_config_t& c, Layout& L) {
   std::memset(&L, 0, sizeof(L));
   L.B = c.batch; L.Hq = c.n_q_heads; L.Hkv = c.n_kv_heads;
@@ -119,7 +151,7 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
     place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);
     place_store(L.v, kRow, c.v_bits, INNERQ_MODE_ASYM, c, L.U, off);
-    place_records(L.v, L.k, L.G, L.U, off);
+    place_records_outer(L.k, L.v, L.G, L.U, off);
   }
   L.cache_bytes = off;
   size_t w = 0;

@@ -42,13 +42,12 @@ __device__ __forceinline__ float element(const TensorView& v, int G, int t, int 
   quant = true;
   float s, z;
   uint32_t code;
-  if (v.kind == kRow) {
-    decode_meta(load_meta(v.rec + row_meta_off(v.S, i), c / G, v.meta_bytes), v.bits, s, z);
+  if (v.kind == kRow) decode_meta(load_meta(v.rec + row_meta_off(v.S, i), c / G, v.meta_bytes), v.bits, s, z);
+  else decode_meta(load_meta(v.rec + block_meta_off(v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
+  if (v.S.code_kind == kRow)
     code = row_code(reinterpret_cast<const uint32_t*>(v.rec + row_code_off(v.S, i)), c, v.bits);
-  } else {
-    decode_meta(load_meta(v.rec + block_meta_off(v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
+  else
     code = chunk_code(reinterpret_cast<const uint32_t*>(v.rec + block_code_off(v.S, i / kChunk)), i % kChunk, c, v.bits);
-  }
   return fmaf(s, (float)code, z);
 }
 

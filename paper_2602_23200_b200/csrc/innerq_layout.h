@@ -40,7 +40,11 @@ constexpr int kTile = 128;        // capacity granularity in tokens
 enum StoreKind : int { kRow = 0, kBlock = 1, kNone = 2 };
 
 struct Store {
-  int kind;            // StoreKind
+  int kind;            // StoreKind: how the tensor is grouped (kRow: groups of G channels inside a token, metadata
+                       // per token; kBlock: per-channel groups of G tokens, metadata per group)
+  int code_kind;       // how its codes are laid out: kRow = one packed row per token (the operand order of q.K^T),
+                       // kBlock = 32-token chunks (the operand order of p.V).  Equal to `kind` under inner grouping;
+                       // under outer grouping keys keep rows and values keep chunks, only the metadata changes sides.
   int bits, mode;
   int ring_cap;        // slots of the recent ring: w_recent + 1 (ROW) or w_recent + G (BLOCK)
   int cap_q;           // capacity in quantised tokens (multiple of kTile)
@@ -56,6 +60,8 @@ struct Store {
   size_t rec_off, rec_unit_stride;    // byte offset of unit 0's record area, bytes per unit
   int group_stride, chunk_stride;     // bytes per group record / per chunk record
   int chunks_per_group;               // G / 32
+  int chunk0;                         // offset of the first chunk record inside a group record (non-zero when the
+                                      // per-group metadata comes first: outer grouping, where keys need it up front)
   int code_in_rec;                    // offset of this store's codes inside a chunk record
   int meta_in_rec;                    // ROW: offset of its metadata rows inside a chunk record;
                                       // BLOCK: offset of the group's metadata inside a group record
@@ -63,16 +69,16 @@ struct Store {
 
 // Byte offset (from the unit's record area) of chunk record ci.
 IQ_HD size_t chunk_rec_off(const Store& S, int ci) {
-  return (size_t)(ci / S.chunks_per_group) * S.group_stride + (size_t)(ci % S.chunks_per_group) * S.chunk_stride;
+  return (size_t)(ci / S.chunks_per_group) * S.group_stride + S.chunk0 + (size_t)(ci % S.chunks_per_group) * S.chunk_stride;
 }
-// ROW store: packed row of quantised token i, and index base of its metadata entries.
+// Row-coded tensor: packed row of quantised token i.  kRow tensor: index base of token i's metadata entries.
 IQ_HD size_t row_code_off(const Store& S, int i) {
   return chunk_rec_off(S, i / kChunk) + S.code_in_rec + (size_t)(i % kChunk) * (16 * S.bits);
 }
 IQ_HD size_t row_meta_off(const Store& S, int i) {
   return chunk_rec_off(S, i / kChunk) + S.meta_in_rec + (size_t)(i % kChunk) * S.n_groups * S.meta_bytes;
 }
-// BLOCK store: packed chunk ci, metadata of group j.
+// Chunk-coded tensor: packed chunk ci.  kBlock tensor: metadata of group j.
 IQ_HD size_t block_code_off(const Store& S, int ci) { return chunk_rec_off(S, ci) + S.code_in_rec; }
 IQ_HD size_t block_meta_off(const Store& S, int j) { return (size_t)j * S.group_stride + S.meta_in_rec; }
 

@@ -57,12 +57,14 @@ __global__ void fill_float_kernel(float* p, float v, int n) {
 }
 
 // ------------------------------------------------------------------ ROW store quantiser
-// One warp quantises one token: lane l holds channels 4l..4l+3; a group of G channels is G/4
-// adjacent lanes.  `stage` is this warp's zero-initialised packed row in shared memory.
+// One warp quantises one token (quantised row i of the unit whose record area is `rec`): lane l holds channels
+// 4l..4l+3; a group of G channels is G/4 adjacent lanes.  `stage` is this warp's packed row in shared memory.
 // `inv_norm4`: reciprocal key norms of this lane's four channels (1.0f / norm, correctly rounded), or null.
+// Codes go to the token's packed row, or (chunk-coded tensor) are OR-ed into the token's 32-token chunk in
+// global memory, whose words other tokens share: that area must be zero before its first token arrives.
 __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src, const float* __restrict__ inv_norm4,
                                                   const Layout& L, const Store& S, uint32_t* stage,
-                                                  uint32_t* __restrict__ dst_row, void* __restrict__ dst_meta, size_t meta_idx) {
+                                                  unsigned char* __restrict__ rec, int i_row) {
   const int lane = threadIdx.x & 31;
   const int gl = L.G >> 2;   // lanes per group
   float x[4];
@@ -98,28 +100,39 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
     es += __shfl_xor_sync(0xffffffffu, es, o);
   }
   const bool asym = choose_asym(S.mode, ea, es);
-  const int words = row_bytes(S.bits) / 4;
-  if (lane < words) stage[lane] = 0u;
-  __syncwarp();
+  if (S.code_kind == kRow) {
+    const int words = row_bytes(S.bits) / 4;
+    uint32_t* dst_row = reinterpret_cast<uint32_t*>(rec + row_code_off(S, i_row));
+    if (lane < words) stage[lane] = 0u;
+    __syncwarp();
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
-    row_put(stage, 4 * lane + i, S.bits, code);
+    for (int i = 0; i < 4; ++i) {
+      uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
+      row_put(stage, 4 * lane + i, S.bits, code);
+    }
+    __syncwarp();
+    if (lane < words) dst_row[lane] = stage[lane];
+  } else {
+    uint32_t* chunk = reinterpret_cast<uint32_t*>(rec + block_code_off(S, i_row / kChunk));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
+      chunk_put(chunk, i_row % kChunk, 4 * lane + i, S.bits, code);
+    }
   }
-  __syncwarp();
-  if (lane < words) dst_row[lane] = stage[lane];
-  if ((lane % gl) == 0) store_meta(dst_meta, meta_idx + lane / gl, S.meta_bytes, group_meta(p, asym));
+  if ((lane % gl) == 0) store_meta(rec + row_meta_off(S, i_row), lane / gl, S.meta_bytes, group_meta(p, asym));
   __syncwarp();
 }
 
 // ------------------------------------------------------------------ BLOCK store quantiser
 // A 128-thread CTA quantises one group of G tokens x 128 channels; thread c owns channel c.
-// tile: fp16 [G][D] staging; words: packed chunks of the group (zeroed here).
+// tile: fp16 [G][D] staging; words: the group's packed chunks, or its packed rows (row-coded tensor), zeroed here.
 __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* __restrict__ norm, const Layout& L,
                                    const Store& S, __half* tile, uint32_t* words, unsigned char* __restrict__ rec, int group_j) {
   const int G = L.G, c = threadIdx.x;
-  const int cw = chunk_bytes(S.bits) / 4;
-  const int n_words = (G / kChunk) * cw;
+  const int cw = chunk_bytes(S.bits) / 4, rw = row_bytes(S.bits) / 4;
+  const bool rows = S.code_kind == kRow;
+  const int n_words = (G / kChunk) * cw;                   // = G * rw
   for (int i = threadIdx.x; i < G * 16; i += 128) {        // 16 x 16-byte pieces per token row
     int t = i >> 4, piece = i & 15;
     reinterpret_cast<uint4*>(tile)[i] = *reinterpret_cast<const uint4*>(src.row(t_first + t) + piece * 8);
@@ -148,15 +161,42 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     float x = __half2float(tile[t * kD + c]);
     if (norm) x = __fmul_rn(x, inv);
     uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
-    chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
+    if (rows) row_put(words + t * rw, c, S.bits, code);
+    else chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
   }
   store_meta(rec + block_meta_off(S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
   __syncthreads();
   for (int i = threadIdx.x; i < n_words; i += 128) {
-    const int ch = i / cw;
-    reinterpret_cast<uint32_t*>(rec + block_code_off(S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
+    if (rows) {
+      const int t = i / rw;
+      reinterpret_cast<uint32_t*>(rec + row_code_off(S, group_j * G + t))[i - t * rw] = words[i];
+    } else {
+      const int ch = i / cw;
+      reinterpret_cast<uint32_t*>(rec + block_code_off(S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
+    }
   }
   __syncthreads();
+}
+
+// Prefill with these generic routines (tensors whose code layout differs from their grouping: the outer-grouped
+// comparison cache).  One warp per token / one CTA per group of G tokens.
+__global__ void __launch_bounds__(128) quantize_rows_generic_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
+                                                                    int n_q, unsigned char* __restrict__ cache) {
+  __shared__ uint32_t stage[4][16];
+  const int u = blockIdx.y, warp = threadIdx.x >> 5;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4)
+    quantize_row_warp(X + ((size_t)u * N + L.w_sink + i) * kD, nullptr, L, S, stage[warp], rec, i);
+}
+__global__ void __launch_bounds__(128) quantize_blocks_generic_kernel(Layout L, Store S, const __half* __restrict__ X,
+                                                                      int N, int n_q, unsigned char* __restrict__ cache) {
+  __shared__ __align__(16) __half tile[128 * kD];
+  __shared__ uint32_t words[4 * 512];
+  const int u = blockIdx.y;
+  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  TokSrc src{X + (size_t)u * N * kD, 0, 0};
+  for (int j = blockIdx.x; j < n_q / L.G; j += gridDim.x)
+    quantize_block_cta(src, L.w_sink + j * L.G, nullptr, L, S, tile, words, rec, j);
 }
 
 // ------------------------------------------------------------------ window copies (prefill)
@@ -199,8 +239,7 @@ __device__ __forceinline__ void append_evict_row(const Layout& L, const Store& R
   TokSrc src{ring, R.ring_cap, L.w_sink};
   // with an empty recent window the evicted token is the new one, which is not in the ring yet
   const __half* row = L.w_sink + nq_before == t_new ? x_new : src.row(L.w_sink + nq_before);
-  quantize_row_warp(row, use_norm ? inv4 : nullptr, L, R, words, reinterpret_cast<uint32_t*>(rec + row_code_off(R, nq_before)),
-                    rec + row_meta_off(R, nq_before), 0);
+  quantize_row_warp(row, use_norm ? inv4 : nullptr, L, R, words, rec, nq_before);
 }
 
 // The new token goes to the sink or the ring of the store.
@@ -262,7 +301,7 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
   if (code && S.kind != kNone) {
     for (int i = tid0; i < n_q * kD; i += stride) {
       int t = i / kD, c = i % kD;
-      uint32_t v = S.kind == kRow
+      uint32_t v = S.code_kind == kRow
                        ? row_code(reinterpret_cast<const uint32_t*>(rec + row_code_off(S, t)), c, S.bits)
                        : chunk_code(reinterpret_cast<const uint32_t*>(rec + block_code_off(S, t / kChunk)), t % kChunk, c,
                                     S.bits);
@@ -320,6 +359,10 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
     fill_float_kernel<<<(L.U * kD + 255) / 256, 256, 0, st>>>(norm, 1.0f, L.U * kD);
     launches += 1;
   }
+  if (L.k.kind != kNone && L.k.code_kind != L.k.kind) {
+    // chunk words of the outer-grouped cache are filled token by token with OR: they start from zero
+    if (cudaMemsetAsync(cache + L.k.rec_off, 0, L.k.rec_unit_stride * L.U, st) != cudaSuccess) return -1;
+  }
   const Store* stores[2] = {&L.k, &L.v};
   const __half* srcs[2] = {K, V};
   const int nq[2] = {cn.n_qk, cn.n_qv};
@@ -334,7 +377,14 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
       continue;
     }
     const bool nrm = use_norm && i == 0;
-    if (nq[i] > 0) {
+    if (nq[i] > 0 && S.code_kind != S.kind) {      // outer-grouped comparison cache: generic routines, no key norm
+      if (S.kind == kRow)
+        quantize_rows_generic_kernel<<<dim3(grid_for(nq[i], 4 * 8, 4096), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i], cache);
+      else
+        quantize_blocks_generic_kernel<<<dim3(grid_for(nq[i] / L.G, 1, 8192), L.U), 128, 0, st>>>(L, S, srcs[i], N, nq[i],
+                                                                                               cache);
+      launches += 1;
+    } else if (nq[i] > 0) {
       const float* inv_norm = nrm ? reinterpret_cast<const float*>(ws + L.ws_absmax_off) : nullptr;
       if (launch_quantize_store_prefill(L, S, srcs[i], N, nq[i], cache, inv_norm, st) < 0) return -1;
       launches += 1;
