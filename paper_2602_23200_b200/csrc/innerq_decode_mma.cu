@@ -15,8 +15,15 @@ using FormatLauncher = int (*)(const Layout&, const Counts&, const DecodeArgs&, 
 // The formats with kernels: equal key and value bit widths with full or symmetric-only metadata, and the mixed
 // 3-bit-key / 2-bit-value combinations with symmetric keys.
 FormatLauncher format_launcher(const Layout& L) {
-  if (L.grouping != 0 || L.k.kind != kRow || L.v.kind != kBlock) return nullptr;
   if (L.G != 32 && L.G != 64 && L.G != 128) return nullptr;
+  if (L.grouping == 1) {      // outer grouping: per-channel key groups on token rows, per-token value groups on chunks
+    if (L.k.kind != kBlock || L.k.code_kind != kRow || L.v.kind != kRow || L.v.code_kind != kBlock) return nullptr;
+    if (L.k.meta_bytes != 4 || L.v.meta_bytes != 4 || L.k.bits != L.v.bits) return nullptr;
+    if (L.k.bits == 2) return &launch_decode_mma_outer_k2v2;
+    if (L.k.bits == 4) return &launch_decode_mma_outer_k4v4;
+    return nullptr;
+  }
+  if (L.grouping != 0 || L.k.kind != kRow || L.v.kind != kBlock) return nullptr;
   const int kb = L.k.bits, vb = L.v.bits, km = L.k.meta_bytes, vm = L.v.meta_bytes;
   if (kb == 2 && vb == 2 && km == 4 && vm == 4) return &launch_decode_mma_k2v2_m44;
   if (kb == 4 && vb == 4 && km == 4 && vm == 4) return &launch_decode_mma_k4v4_m44;
@@ -49,8 +56,10 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   DecodeArgs a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
-  a.n_skew_tiles = (cn.n_qk - cn.n_qv + 15) / 16;
-  a.n_tail_tiles = a.n_skew_tiles + (cn.n_sink + cn.n_k_recent + 15) / 16;
+  // tokens where only one tensor is packed (inner: keys, outer: values), then the tokens that are fp16 in both
+  const bool outer = L.grouping == 1;
+  a.n_skew_tiles = ((outer ? cn.n_qv - cn.n_qk : cn.n_qk - cn.n_qv) + 15) / 16;
+  a.n_tail_tiles = a.n_skew_tiles + (cn.n_sink + (outer ? cn.n_v_recent : cn.n_k_recent) + 15) / 16;
   a.units_per_split = 0;
   a.tail_cost_units = 0;
   a.tiles_q0 = a.tiles_rem = 0;

@@ -229,7 +229,13 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 // scale / zero-point of group j only (then the quad adds up); for values, column pair w holds p
 // restricted to the w-th value group of a window of four, and lane j applies group j's metadata once per
 // window.  This removes the 4x redundancy a quad otherwise has in decoding per-group metadata.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI>
+// OUTER: the outer-grouped comparison cache (keys grouped per channel along tokens, values per token along
+// channels, asymmetric).  Same records, same pipeline, other arithmetic: the scale can no longer leave the inner
+// sum, so it goes INTO the second operand: for keys q'' * S_j (rebuilt for every group of G tokens from the group's
+// metadata, which leads the group record), for values p_t * S_{t,g} (one operand set per channel group the
+// m-tile's rows fall into); zero-points contribute sum_c q''_c Z_jc per group and sum_t p_t Z_{t,g} per channel
+// group.  One chunk per iteration, four heads per pass.
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   constexpr int KP = KB == 3 ? 2 : KB, VP = VB == 3 ? 2 : VB;     // bits of the primary code plane
@@ -248,6 +254,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   // q'' fragments are scaled below 2^QE; the 1-bit plane of 3-bit keys reuses them times up to 2^2 * 2^0
   constexpr int QE = KB == 3 ? 12 : 14;
   static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
+  static_assert(!OUTER || (!SPLIT && CPI == 1 && KM == 4 && VM == 4 && KB != 3 && VB != 3), "OUTER: plain variant only");
+  constexpr int VBASE = 4;                      // OUTER: p * S enters the value MMA scaled by 2^(VBASE - field position)
   static_assert((NST & (NST - 1)) == 0, "stage count must be a power of two");
   static_assert(CPI == 1 || CPI == 2, "one or two chunks per iteration");
 
@@ -264,7 +272,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
   // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
   const int Gy = gridDim.y, cst = a.tail_cost_units;
-  const int n_chunks_total = cn.n_qv / kChunk;
+  const int n_chunks_total = (OUTER ? cn.n_qk : cn.n_qv) / kChunk;   // chunks in which keys AND values are packed
   const int n_units_total = (n_chunks_total + RU - 1) / RU;
   const int q_cta = a.tiles_q0 + (split < a.tiles_rem ? 1 : 0);                 // tail tiles of this CTA
   const int tiles_before = split * a.tiles_q0 + min(split, a.tiles_rem);         // ... of the CTAs before it
@@ -296,7 +304,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   int nx_ci = c_lo;
   auto issue = [&](int st) {   // one lane: arm the barrier, start the copy of the next iteration into stage st
     // the value group's scale/zero words sit right behind its last chunk
-    const int n_meta = CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0);
+    // (OUTER: the key group's words sit in front of its first chunk)
+    const int n_meta = OUTER ? ((nx_ci & (CH - 1)) == 0 ? 1 : 0)
+                             : (CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0));
     const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
     bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes, bars_u32 + 8 * st);
@@ -306,7 +316,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   // Tail tile x: up to 16 tokens outside the range where both K and V are packed.  Skew tiles
   // (x < n_skew_tiles): keys are packed rows n_qv + 16x .. of one chunk record, values fp16 ring rows.
   // Other tiles: entries of the list [sink tokens, recent key tokens], keys and values fp16.
-  const int n_skew = cn.n_qk - cn.n_qv, n_list = cn.n_sink + cn.n_k_recent;
+  // (OUTER: the skew zone has packed values and fp16 keys, and the list ends with the recent VALUE tokens)
+  const int n_skew = OUTER ? cn.n_qv - cn.n_qk : cn.n_qk - cn.n_qv;
+  const int n_list = cn.n_sink + (OUTER ? cn.n_v_recent : cn.n_k_recent);
   auto tail_tile = [&](int k, bool& skew, int& e0, int& cnt) {
     const int x = split + Gy * (warp + kWarps * k);
     skew = x < a.n_skew_tiles;
@@ -318,15 +330,16 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const uint4* v_ring4 = reinterpret_cast<const uint4*>(a.cache + L.v.ring_off + (size_t)u * L.v.ring_stride);
   const uint4* k_sink4 = reinterpret_cast<const uint4*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
   const uint4* k_ring4 = reinterpret_cast<const uint4*>(a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride);
+  // the tensor that is still fp16 in the skew zone (values; OUTER: keys) has the zone's tokens at the head of its ring
   auto v_row = [&](bool skew, int e) -> const uint4* {
     if (!skew && e < cn.n_sink) return v_sink4 + (size_t)e * 16;
-    int slot = a.v_ring_pos0 + (skew ? e : n_skew + (e - cn.n_sink));
+    int slot = a.v_ring_pos0 + (OUTER ? e - cn.n_sink : (skew ? e : n_skew + (e - cn.n_sink)));
     if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
     return v_ring4 + (size_t)slot * 16;
   };
-  auto k_row = [&](int e) -> const uint4* {
-    if (e < cn.n_sink) return k_sink4 + (size_t)e * 16;
-    int slot = a.k_ring_pos0 + (e - cn.n_sink);
+  auto k_row = [&](bool skew, int e) -> const uint4* {
+    if (!skew && e < cn.n_sink) return k_sink4 + (size_t)e * 16;
+    int slot = a.k_ring_pos0 + (OUTER ? (skew ? e : n_skew + (e - cn.n_sink)) : e - cn.n_sink);
     if (slot >= L.k.ring_cap) slot -= L.k.ring_cap;
     return k_ring4 + (size_t)slot * 16;
   };
@@ -503,7 +516,13 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         }
       };
       float sA, sB;
-      if constexpr (SPLIT) {
+      if constexpr (OUTER) {          // the scales are inside Bq: the sums over all 128 channels are the scores
+        float c4[4];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
+        sA = c4[0] + c4[1];
+        sB = c4[2] + c4[3];
+      } else if constexpr (SPLIT) {
         float c4[4];
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) kstep(c4, ks, ks == 0);
@@ -534,6 +553,47 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       sB_out = sB;
     };
 
+    // OUTER: operand fragments and constants of one key group (G tokens) from its 128 metadata words `kmj` (scale |
+    // zero-point << 16, ordered like block_meta_index): Bq <- q'' * S_j, hi / lo split, scaled below 2^QE by the
+    // group's largest scale; kconst <- sum_c q''_c Z_jc of this lane's accumulator head; kfac_cur undoes the scaling.
+    float kconst = 0.f, kfac_cur = 0.f;
+    auto outer_group = [&](const uint32_t* kmj) {
+      auto entry = [&](int ks, int rr) { return ((2 * ks + rr) & 7) * 16 + (ks >> 2) * 8 + 2 * j; };   // channels 16ks+2j+8rr, +1
+      float smax = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          const uint2 w = *reinterpret_cast<const uint2*>(kmj + entry(ks, rr));
+          smax = fmaxf(smax, fmaxf(fabsf(__low2float(*reinterpret_cast<const __half2*>(&w.x))),
+                                   fabsf(__low2float(*reinterpret_cast<const __half2*>(&w.y)))));
+        }
+      smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, 1));
+      smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, 2));
+      const int eS = smax > 0.f ? ((__float_as_int(smax) >> 23) & 0xff) - 126 : 0;     // smax < 2^eS
+      const int bexp = QE - qe_s[4 + (gid >> 1)] - eS;          // qe_s[4 + h]: exponent of max |q''| of head h
+      float zc = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          const uint2 w = *reinterpret_cast<const uint2*>(kmj + entry(ks, rr));
+          const __half2 h0 = *reinterpret_cast<const __half2*>(&w.x), h1 = *reinterpret_cast<const __half2*>(&w.y);
+          const int c0 = 16 * ks + 2 * j + 8 * rr;
+          const float q0 = q_raw_s[(gid >> 1) * kD + c0], q1 = q_raw_s[(gid >> 1) * kD + c0 + 1];
+          const int kk = (ks % (2 * KPW)) % KPW;
+          const float scl = pow2i(bexp - KP * (2 * kk + rr));
+          const uint32_t v0 = split_hi_lo(q0 * fabsf(__low2float(h0)) * scl);
+          const uint32_t v1 = split_hi_lo(q1 * fabsf(__low2float(h1)) * scl);
+          Bq[ks][rr] = (gid & 1) ? ((v0 >> 16) | (v1 & 0xFFFF0000u)) : ((v0 & 0xFFFFu) | (v1 << 16));
+          zc = fmaf(q0, __high2float(h0), fmaf(q1, __high2float(h1), zc));
+        }
+      zc += __shfl_xor_sync(0xffffffffu, zc, 1);
+      zc += __shfl_xor_sync(0xffffffffu, zc, 2);
+      kconst = __shfl_sync(0xffffffffu, zc, 8 * j);          // lanes 8j .. 8j+7 hold head j's sum
+      kfac_cur = pow2i(24 - (QE - qe_s[4 + j] - eS));
+    };
+
     // Fragments of raw q'' for the fp16 key rows of this warp's tail tiles (registers only while those run).
     // SPLIT reuses the table area for its side ring, so the tables are released now, while all warps are in step.
     uint32_t Bqr[8][2];
@@ -559,6 +619,32 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
     }
     bool failed = false;
+    // OUTER: sum_t p_t Z_{t,g} per channel group (this lane's tokens, head tid4), and the value operand of 16 tokens:
+    // p * S_{t,g} as fp16, one set per half of the m-tiles when there is more than one channel group (G = 32: the
+    // two groups an m-tile's rows fall into share a set as its two column variants).
+    constexpr int NSET = OUTER && NG > 1 ? 2 : 1;
+    float zacc[OUTER ? NG : 1];
+#pragma unroll
+    for (int g = 0; g < (OUTER ? NG : 1); ++g) zacc[g] = 0.f;
+    // meta_rows: the chunk's value metadata rows [token][NG]; tok: token inside the chunk; pos: field position
+    auto outer_v_operand = [&](const uint32_t* meta_rows, int tok, float p, int pos, uint32_t (&pk)[NSET]) {
+      float ps[NG];
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        const uint32_t w = meta_rows[tok * NG + g];
+        const __half2 h2 = *reinterpret_cast<const __half2*>(&w);
+        zacc[g] = fmaf(p, __high2float(h2), zacc[g]);
+        ps[g] = p * fabsf(__low2float(h2)) * pow2i(VBASE - VP * pos);
+      }
+#pragma unroll
+      for (int st_ = 0; st_ < NSET; ++st_) {
+        if constexpr (NG == 4)
+          pk[st_] = (uint32_t)__half_as_ushort(__float2half_rn(ps[2 * st_])) |
+                    ((uint32_t)__half_as_ushort(__float2half_rn(ps[2 * st_ + 1])) << 16);
+        else
+          pk[st_] = (uint32_t)__half_as_ushort(__float2half_rn(ps[NG == 2 ? st_ : 0]));
+      }
+    };
 
     // ---------------- tail tiles of this warp: fp16 windows and the K/V skew zone -------------------
     // 16 tokens at a time, operands straight from global memory (coalesced 128-bit loads), into the warp's
@@ -569,7 +655,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       bool skew; int e0, cnt;
       tail_tile(k, skew, e0, cnt);
       float sA, sB;                                            // true log2-domain scores of entries e0+gid, e0+gid+8
-      if (skew) {
+      if (skew && !OUTER) {
         const int iq = cn.n_qv + e0;                           // first packed key row of the tile (16-aligned)
         const unsigned char* rec = g_rec + (size_t)((iq / kChunk) / CH) * SL::kGroupRec +
                                    (size_t)((iq / kChunk) % CH) * SL::kRec;
@@ -578,8 +664,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         sA *= kfac;
         sB *= kfac;
       } else {
-        const uint4* ra = k_row(e0 + min(gid, cnt - 1));
-        const uint4* rb = k_row(e0 + min(gid + 8, cnt - 1));
+        const uint4* ra = k_row(skew, e0 + min(gid, cnt - 1));
+        const uint4* rb = k_row(skew, e0 + min(gid + 8, cnt - 1));
         uint4 ka[4], kb[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) { ka[i] = __ldg(ra + j + 4 * i); kb[i] = __ldg(rb + j + 4 * i); }
@@ -609,8 +695,55 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       l_part *= alpha;
 #pragma unroll
       for (int m = 0; m < 8; ++m) { out_acc[m][0] *= alpha; out_acc[m][1] *= alpha; }
+      if constexpr (OUTER) {
+#pragma unroll
+        for (int g = 0; g < NG; ++g) zacc[g] *= alpha;
+#pragma unroll
+        for (int m = 0; m < 8; ++m)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
+      }
       const float pA = ex2_approx(sA - m_new), pB = ex2_approx(sB - m_new);
       l_part += pA + pB;
+      if (OUTER && skew) {
+        // values of the skew zone are packed (half a chunk: one k-step of 16 tokens), read straight from global memory
+        const int iq = cn.n_qk + e0, ci = iq / kChunk, ks = (iq % kChunk) / 16;
+        const unsigned char* rec = g_rec + (size_t)(ci / CH) * SL::kGroupRec + SL::kVMeta + (size_t)(ci % CH) * SL::kRec;
+        const uint32_t* vmr = reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta);
+        const uint32_t* vcg = reinterpret_cast<const uint32_t*>(rec + SL::kOffVCodes);
+        uint32_t Bt[NSET][2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t pk[NSET];
+          outer_v_operand(vmr, 16 * ks + gid + 8 * h, h ? pB : pA, h, pk);   // fields are shifted down to position h below
+#pragma unroll
+          for (int st_ = 0; st_ < NSET; ++st_) Bt[st_][h] = movmatrix_trans(pk[st_]);
+        }
+        if constexpr (VP == 2) {
+          const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(vcg + lane * 4));
+          const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(vcg + 128 + lane * 4));
+          const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+          for (int m = 0; m < 8; ++m) {
+            const uint32_t w0 = vw[m] >> (4 * ks), w1 = w0 >> 8;          // this k-step's fields at positions 0 and 1
+            const uint32_t m0 = FV::kField, m1 = FV::kField << 2;
+            mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bt[NSET > 1 ? m >> 2 : 0][0], Bt[NSET > 1 ? m >> 2 : 0][1]);
+          }
+        } else {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(vcg + ks * 256 + hh * 128 + lane * 4));
+            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int mm = 0; mm < 4; ++mm) {
+              const uint32_t w0 = vw[mm], w1 = vw[mm] >> 8;
+              const uint32_t m0 = FV::kField, m1 = FV::kField << 4;
+              mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bt[NSET > 1 ? hh : 0][0], Bt[NSET > 1 ? hh : 0][1]);
+            }
+          }
+        }
+        continue;
+      }
       uint32_t pkA = split_hi_lo(pA * 1024.f), pkB = split_hi_lo(pB * 1024.f);
       if (SPLIT && j != 0) { pkA = 0u; pkB = 0u; }              // SPLIT: lane 0 of each quad takes the tail's sums
       const uint32_t b0 = movmatrix_trans(pkA), b1 = movmatrix_trans(pkB);
@@ -656,12 +789,21 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
           sc[cc][0][0] = sc[cc][0][1] = sc[cc][1][0] = sc[cc][1][1] = -INFINITY;
           continue;
         }
-        const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc));
-        const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
+        // OUTER: a group's first chunk is preceded in the stage by the key group's metadata
+        const int lead = OUTER && ((ci0 + cc) & (CH - 1)) == 0 ? SL::kVMeta : 0;
+        if constexpr (OUTER) {
+          if (lead) outer_group(reinterpret_cast<const uint32_t*>(sp));
+        }
+        const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + lead + SL::off(cc));
+        const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + lead + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           float sA, sB;
           k_mtile(kc, km, 16 * mt, sA, sB);
+          if constexpr (OUTER) {       // true log2-domain scores right away (the scaling changes from group to group)
+            sA = fmaf(sA, kfac_cur, kconst);
+            sB = fmaf(sB, kfac_cur, kconst);
+          }
           const bool valid = cc == 0 || last_valid;
           sc[cc][mt][0] = valid ? sA : -INFINITY;
           sc[cc][mt][1] = valid ? sB : -INFINITY;
@@ -676,11 +818,16 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
-      const float m_new = fmaxf(m_run, cmax * kfac);
+      const float kf = OUTER ? 1.0f : kfac;                    // what the raw scores still have to be multiplied by
+      const float m_new = fmaxf(m_run, cmax * kf);
       if (__any_sync(0xffffffffu, m_new > m_run)) {
         const float alpha = ex2_approx(m_run - m_new);     // 0 on the first iteration (m_run = -inf)
         l_part *= alpha;
         psum *= alpha;
+        if constexpr (OUTER) {
+#pragma unroll
+          for (int g = 0; g < NG; ++g) zacc[g] *= alpha;
+        }
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
           out_acc[m][0] *= alpha; out_acc[m][1] *= alpha;
@@ -693,30 +840,40 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
       for (int cc = 0; cc < CPI; ++cc) {
         if (cc > 0 && !last_valid) continue;
-        const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffVCodes);
-        const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
         const int ci = ci0 + cc;
+        const int lead = OUTER && (ci & (CH - 1)) == 0 ? SL::kVMeta : 0;
+        const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + lead + SL::off(cc) + SL::kOffVCodes);
+        const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
         // slot: position of this chunk's value group in the SPLIT window / position of the chunk in its group
         const int slot = SPLIT ? (ci - c_lo) & (WIN - 1) : ci % CH;
         const bool group_start = slot == 0;
         const bool group_end = SPLIT ? (slot == WIN - 1 || (it == n_iters - 1 && (cc == CPI - 1 || !last_valid)))
                                      : (slot == CH - 1);
-        constexpr bool kFreshEveryChunk = !SPLIT && CH == 1;   // then the first value mma takes a zero C
-        if (!kFreshEveryChunk && group_start) {
+        constexpr bool kFreshEveryChunk = !SPLIT && !OUTER && CH == 1;   // then the first value mma takes a zero C
+        if (!OUTER && !kFreshEveryChunk && group_start) {
 #pragma unroll
           for (int m = 0; m < 8; ++m)
 #pragma unroll
             for (int e = 0; e < 4; ++e) accg[m][e] = 0.f;
         }
-        uint32_t Bp[2][2];
+        uint32_t Bps[NSET][2][2];
+        uint32_t (&Bp)[2][2] = Bps[0];
         float psum_c = 0.f;
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            const float p = ex2_approx(fmaf(sc[cc][mt][h], kfac, -m_new));
+            const float p = ex2_approx(fmaf(sc[cc][mt][h], kf, -m_new));
             psum_c += p;
             const int pos = VP == 2 ? 2 * mt + h : h;
+            if constexpr (OUTER) {
+              uint32_t pks[NSET];
+              outer_v_operand(reinterpret_cast<const uint32_t*>(sp + lead + SL::off(cc) + SL::kOffKMeta), 16 * mt + gid + 8 * h, p,
+                              pos, pks);
+#pragma unroll
+              for (int st_ = 0; st_ < NSET; ++st_) Bps[st_][mt][h] = movmatrix_trans(pks[st_]);
+              continue;
+            }
             // p goes in as one fp16 (the lo column stays zero): its 2^-12 relative rounding is random per token and
             // far inside the output tolerance, and it saves the hi/lo split of every probability
             uint32_t pk = (uint32_t)__half_as_ushort(__float2half_rn(p * pow2i(10 - VP * pos)));
@@ -740,7 +897,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
             for (int ks = 0; ks < 2; ++ks) {
               const uint32_t m0 = FV::kField << (2 * (2 * ks)), m1 = FV::kField << (2 * (2 * ks + 1));
               if (kFreshEveryChunk && ks == 0) mma16816_z(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
-              else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+              else mma16816(accg[m], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bps[NSET > 1 ? m >> 2 : 0][ks][0], Bps[NSET > 1 ? m >> 2 : 0][ks][1]);
             }
           }
         } else {
@@ -757,7 +914,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
                 if (kFreshEveryChunk && ks == 0)
                   mma16816_z(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
                 else
-                  mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bp[ks][0], Bp[ks][1]);
+                  mma16816(accg[hh * 4 + mm], w0 & m0, w1 & m0, w0 & m1, w1 & m1, Bps[NSET > 1 ? hh : 0][ks][0], Bps[NSET > 1 ? hh : 0][ks][1]);
               }
             }
           }
@@ -794,7 +951,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
           if (chunk_valid && lane * 16 < SL::kVMeta)
             *reinterpret_cast<uint4*>(side + slot * (SL::kVMeta / 4) + lane * 4) = *reinterpret_cast<const uint4*>(vm + lane * 4);
         }
-        if (group_end && chunk_valid) {
+        if (!OUTER && group_end && chunk_valid) {
           if constexpr (SPLIT) __syncwarp();
           float pg = psum;
           pg += __shfl_xor_sync(0xffffffffu, pg, 4);
@@ -862,6 +1019,30 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
           out_acc[m][rh] = v;
         }
     }
+    if constexpr (OUTER) {
+      // the value accumulators carry sum p S u * 2^(VBASE - 24); zero-points: lanes of the same head add their tokens
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        zacc[g] += __shfl_xor_sync(0xffffffffu, zacc[g], 4);
+        zacc[g] += __shfl_xor_sync(0xffffffffu, zacc[g], 8);
+        zacc[g] += __shfl_xor_sync(0xffffffffu, zacc[g], 16);
+      }
+      const bool up = (gid >> 2) != 0;                 // G = 32: rows of lanes 16..31 belong to the m-tile's second group
+#pragma unroll
+      for (int m = 0; m < 8; ++m)
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+          float sel, zz;
+          if constexpr (NG == 4) {
+            sel = up ? accg[m][2 * rh + 1] : accg[m][2 * rh];
+            zz = up ? zacc[2 * (m >> 2) + 1] : zacc[2 * (m >> 2)];
+          } else {
+            sel = accg[m][2 * rh];
+            zz = zacc[NG == 2 ? (m >> 2) : 0];
+          }
+          out_acc[m][rh] += sel * pow2i(10 - VBASE) + zz * 0x1p-14f;
+        }
+    }
     __syncthreads();                                   // every warp is done with its ring
     float* wres = reinterpret_cast<float*>(smem);      // [warp][head][kD + 2]
     const bool writer = SPLIT ? (j == 0) : true;
@@ -914,19 +1095,19 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
 }
 
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
 int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
   using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kSmem) != cudaSuccess)
       return -1;
     configured = true;
   }
-  const int n_chunks = cn.n_qv / kChunk;
+  const int n_chunks = (OUTER ? cn.n_qk : cn.n_qv) / kChunk;
   const int n_units = (n_chunks + RU - 1) / RU;
   const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
   if (n_splits > by_work) n_splits = by_work;
@@ -956,7 +1137,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, L, cn, a) != cudaSuccess) return -1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, cn, a) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -982,6 +1163,15 @@ int launch_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_
   return -2;
 }
 
+// The outer-grouped comparison cache with KB-bit keys and VB-bit values at every group size.
+template <int KB, int VB>
+int launch_format_outer(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, cudaStream_t st) {
+  if (L.G == 32) return launch_one<KB, VB, 32, 4, 4, false, 1, true>(L, cn, a, n_splits, st);
+  if (L.G == 64) return launch_one<KB, VB, 64, 4, 4, false, 1, true>(L, cn, a, n_splits, st);
+  if (L.G == 128) return launch_one<KB, VB, 128, 4, 4, false, 1, true>(L, cn, a, n_splits, st);
+  return -2;
+}
+
 }  // namespace
 
 // Defines the externally visible launcher of one format in the translation unit that compiles its kernels.
@@ -990,6 +1180,12 @@ int launch_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_
   int IQ_MMA_FORMAT_NAME(KB, VB, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, \
                                          int cpi, cudaStream_t st) {                                            \
     return launch_format<KB, VB, KM, VM>(L, cn, a, n_splits, cpi, st);                                          \
+  }
+
+#define IQ_DEFINE_MMA_OUTER_FORMAT(KB, VB)                                                                          \
+  int launch_decode_mma_outer_k##KB##v##VB(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,    \
+                                           int, cudaStream_t st) {                                                   \
+    return launch_format_outer<KB, VB>(L, cn, a, n_splits, st);                                                      \
   }
 
 }  // namespace iq

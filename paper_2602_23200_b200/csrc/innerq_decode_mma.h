@@ -36,4 +36,8 @@ int launch_decode_mma_k4v4_m22(const Layout& L, const Counts& cn, const DecodeAr
 int launch_decode_mma_k3v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
 int launch_decode_mma_k3v2_m24(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
 
+// Outer-grouped comparison cache (same argument list; cpi is ignored).
+int launch_decode_mma_outer_k2v2(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_outer_k4v4(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+
 }  // namespace iq

@@ -79,6 +79,25 @@ def test_prefill_and_decode_outer(bits, G, N):
     check_decode(w, oc, gc, splits=(0, 2))
 
 
+@pytest.mark.parametrize("bits,G,r,N", [(2, 32, 1, 700), (2, 64, 4, 600), (2, 128, 2, 900), (4, 32, 4, 500),
+                                        (4, 64, 8, 555), (4, 128, 1, 1300)])
+def test_outer_grouped_fused_kernel(bits, G, r, N):
+    # the outer-grouped comparison cache on the fused kernel (variant 3 refuses to fall back), against the generic
+    # kernel (variant 1) and the oracle; then appends through the reversed skew zone (packed values, fp16 keys)
+    w = synth.tiny(n_tokens=N, group=G, k_bits=bits, v_bits=bits, grouping=O.OUTER, k_normalize=0, k_mode=O.ASYM,
+                   v_mode=O.ASYM, n_q_heads=2 * r)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.OUTER, G, False, False)
+    check_decode(w, oc, gc, variants=(3, 1), splits=(0, 2, 5))
+    for step in range(G + 5):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        if step in (0, 1, 15, 16, 17, G - 1, G, G + 4):
+            check_decode(w, oc, gc, step=step, variants=(3,), splits=(0, 3))
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.OUTER, G, False, False)
+
+
 def test_fp16_cache_decode():
     w = synth.tiny(n_tokens=500, grouping=O.FP16, k_normalize=0)
     oc, gc, K, V = run_prefill_both(w)
