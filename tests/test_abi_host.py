@@ -47,6 +47,18 @@ def test_config_validation_without_gpu():
         B.innerq_cache_bytes(B.make_config(synth.config1(), grouping=B.GROUPING_OUTER, k_normalize=1))
 
 
+def test_step_staging_size_without_gpu():
+    # device staging of innerq_decode_step_host: k_new, v_new, q and out, each rounded up to 256 bytes
+    need = C.c_size_t()
+    cfg = B.make_config(batch=3, n_q_heads=8, n_kv_heads=2, max_tokens=64)
+    assert B.lib().innerq_step_staging_bytes(C.byref(cfg), C.byref(need)) == 0
+    kv, q = 3 * 2 * 128 * 2, 3 * 8 * 128 * 2
+    assert need.value == 2 * ((kv + 255) // 256 * 256) + 2 * ((q + 255) // 256 * 256)
+    bad = B.make_config(batch=3, n_q_heads=8, n_kv_heads=3, max_tokens=64)
+    assert B.lib().innerq_step_staging_bytes(C.byref(bad), C.byref(need)) == -1
+    assert B.lib().innerq_step_staging_bytes(C.byref(cfg), None) == -1
+
+
 def test_packed_payload_matches_table_bits():
     # Table "bits" (G = 32, head dim 128): effective bits per cached number = payload bytes * 8 / 128.
     rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table_bits.txt"))
