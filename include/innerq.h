@@ -182,6 +182,7 @@ int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_s
  *   n_splits : number of token ranges each unit is split into by the decode kernel.
  *   variant  : 0 automatic, 1 plain SIMT kernel, 2 warp-MMA kernel (where supported; UNSUPPORTED otherwise),
  *              3 / 4 warp-MMA kernel with one / two 32-token chunks per loop iteration (sets a process-wide knob).
+ *              5 tcgen05 kernel (2-bit keys and values, group 32, one query head per KV head; UNSUPPORTED otherwise).
  * Errors: INVALID_ARG. */
 int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
 

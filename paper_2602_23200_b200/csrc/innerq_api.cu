@@ -260,7 +260,11 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int n = -2;
-  if (c->opt_variant != 1 && c->L.k.kind == kNone)
+  if (c->opt_variant == 5) {          // tcgen05 kernel, where it exists; no fallback
+    n = launch_decode_tc5(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                          c->opt_splits, s);
+    if (n == -2) return INNERQ_ERR_UNSUPPORTED;
+  } else if (c->opt_variant != 1 && c->L.k.kind == kNone)
     n = launch_decode_fp16(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L))
@@ -398,7 +402,7 @@ int innerq_cache_export(innerq_cache_t* c, innerq_export_t* ex, void* cuda_strea
 }
 
 int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t variant) {
-  if (!c || n_splits < 0 || variant < 0 || variant > 4) return INNERQ_ERR_INVALID_ARG;
+  if (!c || n_splits < 0 || variant < 0 || variant > 5) return INNERQ_ERR_INVALID_ARG;
   c->opt_splits = n_splits;
   // variants 3 and 4 force the fast kernel with one / two 32-token chunks per loop iteration (process-wide knob)
   if (variant == 3 || variant == 4) { decode_mma_set_chunks_per_iter(variant - 2); variant = 2; }
