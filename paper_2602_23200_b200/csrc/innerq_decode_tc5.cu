@@ -406,31 +406,27 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
     const int p_off = b_offset(warp, val_k_index(warp, lane));
     const float p_scale = pow2i(10 - 2 * val_field(lane));
 
-    for (int it = 0; it < n_my; ++it) {
-      const int st = it % kStages, ti = t_lo + it;
-      const int nv = min(kChunksPerTile, n_chunks - kChunksPerTile * ti);
-      // (a wait that runs out does not leave the loop: every thread keeps passing the same CTA barriers; later
-      // waits are skipped and the result is discarded)
-      if (!failed && !mbar_wait(bar_full + 8 * st, (uint32_t)(it / kStages) & 1u)) failed = true;
-      const unsigned char* sp = smem + st * kTileBytes;
-      // ---------------- keys: row of token `tid` -> A_k ------------------------------------------------------------
-      {
-        const uint4* row = reinterpret_cast<const uint4*>(sp + warp * kRecBytes + lane * kKRow);
-        const uint4 r0 = row[0], r1 = row[1];
-        const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+    // Software pipeline over the tiles of this CTA.  The two MMAs of a tile run asynchronously; while they do, the
+    // threads expand the next operand:   MMA-K(i) || expand V(i);   MMA-V(i) || expand K(i+1);   MMA-K(i+1) || output(i).
+    // (A wait that runs out does not leave the loop: every thread keeps passing the same CTA barriers; later waits
+    // are skipped and the result is discarded.)
+    auto expand_keys = [&](const unsigned char* sp) {       // packed row of token `tid` -> row `tid` of A_k
+      const uint4* row = reinterpret_cast<const uint4*>(sp + warp * kRecBytes + lane * kKRow);
+      const uint4 r0 = row[0], r1 = row[1];
+      const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          uint32_t regs[16];
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t regs[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int wi = 2 * q4 + (i >> 3), fld = i & 7;
-            const uint32_t x = fld >= 4 ? (w[wi] >> 8) : w[wi];
-            regs[i] = x & (0x00030003u << (2 * (fld & 3)));
-          }
-          tmem_st16(t_lane + kColAk + 16 * q4, regs);
+        for (int i = 0; i < 16; ++i) {
+          const int wi = 2 * q4 + (i >> 3), fld = i & 7;
+          const uint32_t x = fld >= 4 ? (w[wi] >> 8) : w[wi];
+          regs[i] = x & (0x00030003u << (2 * (fld & 3)));
         }
+        tmem_st16(t_lane + kColAk + 16 * q4, regs);
       }
-      // ---------------- values: codes of channel `tid` for the tile's tokens -> A_v --------------------------------
+    };
+    auto expand_values = [&](const unsigned char* sp) {     // codes of channel `tid` for the tile's tokens -> A_v
 #pragma unroll
       for (int ch = 0; ch < kChunksPerTile; ++ch) {
         const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVCodes);
@@ -444,17 +440,28 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
         }
         tmem_st16(t_lane + kColAv + 16 * ch, regs);
       }
+    };
+    auto issue_mma = [&](int col_d, int col_a, int off_b, uint32_t bar) {   // thread 0
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        mma_ts(tbase + col_d, tbase + col_a + 8 * ks, smem_desc(smem_u32(smem + off_b) + 512 * ks, 256, 128), ks > 0);
+      mma_commit(bar);
+    };
+    if (n_my > 0) {
+      if (!mbar_wait(bar_full, 0u)) failed = true;
+      expand_keys(smem);
       tc_wait_st();
       tc_fence_before();
       __syncthreads();
-      if (tid == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_ts(tbase + kColDk, tbase + kColAk + 8 * ks, smem_desc(smem_u32(smem + kOffBq) + 512 * ks, 256, 128), ks > 0);
-        mma_commit(bar_k);
-      }
-      // ---------------- scores of token `tid` -----------------------------------------------------------------------
+      if (tid == 0) issue_mma(kColDk, kColAk, kOffBq, bar_k);
+    }
+    for (int it = 0; it < n_my; ++it) {
+      const int st = it % kStages, ti = t_lo + it;
+      const int nv = min(kChunksPerTile, n_chunks - kChunksPerTile * ti);
+      const unsigned char* sp = smem + st * kTileBytes;
+      expand_values(sp);                                                       // || MMA-K(it)
+      // ---------------- scores of token `tid`; probabilities relative to the chunk's own maximum -------------------
       if (!failed && !mbar_wait(bar_k, (uint32_t)it & 1u)) failed = true;
       tc_fence_after();
       float d[8];
@@ -476,48 +483,60 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
       float wmax = s;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
-      if (lane == 0) redmax[warp] = wmax;
-      __syncthreads();
-      const float m_new = fmaxf(m_run, fmaxf(fmaxf(redmax[0], redmax[1]), fmaxf(redmax[2], redmax[3])));
-      const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
-      const float p = warp < nv ? ex2_approx(s - m_new) : 0.f;
+      const float p = warp < nv ? ex2_approx(s - wmax) : 0.f;                  // chunk = warp = one column of B_p
       float wsum = p;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-      if (lane == 0) redsum[warp] = wsum;
+      if (lane == 0) { redmax[warp] = wmax; redsum[warp] = wsum; }
       *reinterpret_cast<__half*>(smem + kOffBp + p_off) = __float2half_rn(p * p_scale);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_wait_st();                                                            // A_v
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");             // B_p
       tc_fence_before();
       __syncthreads();
-      if (tid == 0) {
-        tc_fence_after();
+      if (tid == 0) issue_mma(kColDv, kColAv, kOffBp, bar_v);
+      // the chunks' maxima and sums, brought to the new running maximum
+      float cm[4], cs[4];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_ts(tbase + kColDv, tbase + kColAv + 8 * ks, smem_desc(smem_u32(smem + kOffBp) + 512 * ks, 256, 128), ks > 0);
-        mma_commit(bar_v);
-      }
-      const float ps4[4] = {redsum[0], redsum[1], redsum[2], redsum[3]};
-      l_run = l_run * alpha + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+      for (int ch = 0; ch < 4; ++ch) { cm[ch] = redmax[ch]; cs[ch] = redsum[ch]; }
+      const float m_new = fmaxf(m_run, fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])));
+      const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
+      float cw[4];
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) cw[ch] = cm[ch] == -INFINITY ? 0.f : ex2_approx(cm[ch] - m_new);
+      l_run = l_run * alpha + ((cs[0] * cw[0] + cs[1] * cw[1]) + (cs[2] * cw[2] + cs[3] * cw[3]));
       m_run = m_new;
-      // ---------------- output channel `tid` ------------------------------------------------------------------------
+      // value metadata of channel `tid` (the stage is handed back before it is used)
+      uint32_t vmeta[4];
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch)
+        vmeta[ch] = *reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVMeta + 4 * v_meta_idx);
+      if (it + 1 < n_my) {                                                     // || MMA-V(it)
+        const int st1 = (it + 1) % kStages;
+        if (!failed && !mbar_wait(bar_full + 8 * st1, (uint32_t)((it + 1) / kStages) & 1u)) failed = true;
+        expand_keys(smem + st1 * kTileBytes);
+        tc_wait_st();
+      }
       if (!failed && !mbar_wait(bar_v, (uint32_t)it & 1u)) failed = true;
       tc_fence_after();
       float dv[4];
       tmem_ld4(t_lane + kColDv, dv);
+      tc_fence_before();
+      __syncthreads();               // A_k(it+1) is complete; D_v, B_p, the reduction words and stage `st` are free
+      if (tid == 0) {
+        if (it + 1 < n_my) issue_mma(kColDk, kColAk, kOffBq, bar_k);
+        if (it + kStages < n_my) issue(it + kStages);
+      }
+      // ---------------- output channel `tid` ------------------------------------------------- || MMA-K(it+1) ------
       out_c *= alpha;
 #pragma unroll
       for (int ch = 0; ch < kChunksPerTile; ++ch) {
         if (ch < nv) {
-          const uint32_t mwv = *reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVMeta + 4 * v_meta_idx);
-          const __half2 h2 = *reinterpret_cast<const __half2*>(&mwv);
+          const __half2 h2 = *reinterpret_cast<const __half2*>(&vmeta[ch]);
           const float sg = __low2float(h2);
           const float z = fmaf(-2.0f, fmaxf(sg, 0.f), __high2float(h2));
-          out_c = fmaf(fabsf(sg), dv[ch] * 0x1p14f, fmaf(z, ps4[ch], out_c));
+          out_c = fmaf(cw[ch], fmaf(fabsf(sg), dv[ch] * 0x1p14f, z * cs[ch]), out_c);
         }
       }
-      tc_fence_before();
-      __syncthreads();               // the stage, the operands in tensor memory and the reduction words are free again
-      if (tid == 0 && it + kStages < n_my) issue(it + kStages);
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     failed = __syncthreads_or(failed ? 1 : 0) != 0;
