@@ -407,10 +407,10 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
       for (int g = 0; g < 4; ++g) qg_s[warp * 4 + g] = gs[g];
       int e = 0;
-      if (am > 0.f && am < INFINITY) frexpf(am, &e);
+      if (am > 0.f && am < INFINITY) e = ((__float_as_int(am) >> 23) & 0xff) - 126;
       qe_s[warp] = e;     // am < 2^e
       int er = 0;
-      if (amr > 0.f && amr < INFINITY) frexpf(amr, &er);
+      if (amr > 0.f && amr < INFINITY) er = ((__float_as_int(amr) >> 23) & 0xff) - 126;
       qe_s[4 + warp] = er;
     }
   }
@@ -1070,7 +1070,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) {
         const float* r_ = wres + ((size_t)w * kHeads + h) * (kD + 2);
-        const float wgt = r_[kD] == -INFINITY ? 0.f : exp2f(r_[kD] - M);
+        const float wgt = r_[kD] == -INFINITY ? 0.f : ex2_approx(r_[kD] - M);
         num = fmaf(r_[c], wgt, num);
         den = fmaf(r_[kD + 1], wgt, den);
       }
