@@ -259,90 +259,104 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
 }
 
 // ------------------------------------------------------------------ BLOCK store
-// A CTA of 128 * (G / 32) threads quantises one group of G tokens x 128 channels per iteration: thread
-// (channel c, chunk k) owns tokens 32k .. 32k+31 of channel c, read from an fp16 tile in shared memory that
-// the CTA fills with coalesced loads.  Packed chunks are assembled in shared memory and stored coalesced.
+// A CTA of 64 * (G / 32) threads quantises one group of G tokens x 128 channels per iteration: thread
+// (channel pair cp, chunk k) owns tokens 32k .. 32k+31 of channels 2cp and 2cp+1, read straight from global memory
+// (one 32-bit load per token: a warp reads 128 contiguous bytes of each token row).  The two channels of a pair
+// are the two row halves of one MMA fragment row pair, so between them they fill whole words of the packed chunk
+// and no staging or atomics are needed (3-bit: the 1-bit plane's words are shared with the neighbouring pair).
 template <int BITS, bool NORM>
-__global__ void __launch_bounds__(512) quantize_blocks_prefill_kernel(Layout L, Store S, const __half* __restrict__ X,
+__global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, Store S, const __half* __restrict__ X,
                                                                       int N, int n_q, unsigned char* __restrict__ cache,
                                                                       const float* __restrict__ inv_norm) {
   constexpr int PB = BITS == 3 ? 2 : BITS;
-  constexpr int CW = 128 * BITS;                // words per packed chunk
+  constexpr int NW = PB == 4 ? 8 : 4;
   extern __shared__ __align__(16) unsigned char smem_q[];
-  const int G = L.G, CH = G >> 5, nthr = 128 * CH;
-  __half* tile = reinterpret_cast<__half*>(smem_q);                               // [G][128]
-  uint32_t* words = reinterpret_cast<uint32_t*>(smem_q + (size_t)G * kD * 2);     // [CH][CW]
-  float4* red = reinterpret_cast<float4*>(words + CH * CW);                       // [CH][128]: mn, mx, ea, es
-  const int u = blockIdx.y, tid = threadIdx.x, c = tid & 127, k = tid >> 7;
-  const float inv = NORM ? inv_norm[(size_t)u * kD + c] : 1.0f;
+  const int G = L.G, CH = G >> 5;
+  float4* red = reinterpret_cast<float4*>(smem_q);                               // [CH][128]: mn, mx, ea, es
+  const int u = blockIdx.y, tid = threadIdx.x, cp = tid & 63, k = tid >> 6, c0 = 2 * cp;
+  float inv[2] = {1.0f, 1.0f};
+  if constexpr (NORM) { inv[0] = inv_norm[(size_t)u * kD + c0]; inv[1] = inv_norm[(size_t)u * kD + c0 + 1]; }
   unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
-  const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD;
-  // positions (see block_pos_plane): fragment coordinates of this channel
-  const int m = 4 * (c >> 6) + ((c >> 1) & 3), gid = (c >> 3) & 7, rh = c & 1;
+  const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD + c0;
+  // positions (see block_pos_plane): fragment coordinates of the pair (row halves rh = 0, 1)
+  const int m = 4 * (c0 >> 6) + ((c0 >> 1) & 3), gid = (c0 >> 3) & 7;
   const int base_lo = (m >> 2) * 128 + 16 * gid + (m & 3);                        // + 4 * tid4 (+ 256 * k-step for 4 bits)
   const int base_hi = chunk_hi_plane_word() + 16 * gid + (m >> 1);
-  const int sh_lo = 8 * rh, sh_hi = 4 * (2 * (m & 1) + rh);
-  for (int i = tid; i < CH * CW; i += nthr) words[i] = 0u;
   for (int j = blockIdx.x; j < n_q / G; j += gridDim.x) {
-    const uint4* src = reinterpret_cast<const uint4*>(Xu + (size_t)j * G * kD);
-    for (int i = tid; i < G * 16; i += nthr) reinterpret_cast<uint4*>(tile)[i] = __ldg(src + i);
-    __syncthreads();
-    float x[kSeg];
+    uint32_t raw[kSeg];
+    const __half* src = Xu + ((size_t)j * G + kSeg * k) * kD;
 #pragma unroll
-    for (int t = 0; t < kSeg; ++t) {
-      x[t] = __half2float(tile[(kSeg * k + t) * kD + c]);
-      if constexpr (NORM) x[t] = __fmul_rn(x[t], inv);
-    }
-    float mn, mx;
-    seg_minmax(x, mn, mx);
-    if (CH > 1) {
-      red[k * 128 + c] = make_float4(mn, mx, 0.f, 0.f);
-      __syncthreads();
-      for (int kk = 0; kk < CH; ++kk) {
-        const float4 o = red[kk * 128 + c];
-        mn = fminf(mn, o.x); mx = fmaxf(mx, o.y);
+    for (int t = 0; t < kSeg; ++t) raw[t] = __ldg(reinterpret_cast<const uint32_t*>(src + (size_t)t * kD));
+    uint32_t wlo[NW], whi[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < NW; ++i) wlo[i] = 0u;
+    uint32_t meta2[2];
+    if (CH > 1) __syncthreads();       // the previous group's reduction words are no longer read
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+      float x[kSeg];
+#pragma unroll
+      for (int t = 0; t < kSeg; ++t) {
+        const __half2 h2 = *reinterpret_cast<const __half2*>(&raw[t]);
+        x[t] = rh ? __high2float(h2) : __low2float(h2);
+        if constexpr (NORM) x[t] = __fmul_rn(x[t], inv[rh]);
       }
-    }
-    const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
-    const SegCoder sc(p);
-    const bool no_clip = sc.no_clip(mn, mx);
-    bool asym = S.mode == 1;
-    if (S.mode == 2) {
-      float ea, es;
-      if (no_clip) seg_errors<false>(sc, x, ea, es);
-      else seg_errors<true>(sc, x, ea, es);
+      float mn, mx;
+      seg_minmax(x, mn, mx);
       if (CH > 1) {
-        red[k * 128 + c].z = ea;
-        red[k * 128 + c].w = es;
+        red[k * 128 + c0 + rh] = make_float4(mn, mx, 0.f, 0.f);
         __syncthreads();
-        ea = 0.f; es = 0.f;
         for (int kk = 0; kk < CH; ++kk) {
-          const float4 o = red[kk * 128 + c];
-          ea += o.z; es += o.w;
+          const float4 o = red[kk * 128 + c0 + rh];
+          mn = fminf(mn, o.x); mx = fmaxf(mx, o.y);
         }
       }
-      asym = ea < es;
-    }
-    const ChosenCoder cc(sc, asym);
-    uint32_t lw[BITS == 4 ? 8 : 4], hw[4];
-    if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
-    else pack_block_segment<BITS, true>(cc, x, lw, hw);
-    uint32_t* wk = words + k * CW;
+      const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), BITS, L.sym_variant);
+      const SegCoder sc(p);
+      const bool no_clip = sc.no_clip(mn, mx);
+      bool asym = S.mode == 1;
+      if (S.mode == 2) {
+        float ea, es;
+        if (no_clip) seg_errors<false>(sc, x, ea, es);
+        else seg_errors<true>(sc, x, ea, es);
+        if (CH > 1) {
+          red[k * 128 + c0 + rh].z = ea;
+          red[k * 128 + c0 + rh].w = es;
+          __syncthreads();
+          ea = 0.f; es = 0.f;
+          for (int kk = 0; kk < CH; ++kk) {
+            const float4 o = red[kk * 128 + c0 + rh];
+            ea += o.z; es += o.w;
+          }
+        }
+        asym = ea < es;
+      }
+      const ChosenCoder cc(sc, asym);
+      uint32_t lw[NW], hw[4];
+      if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
+      else pack_block_segment<BITS, true>(cc, x, lw, hw);
 #pragma unroll
-    for (int i = 0; i < (PB == 4 ? 8 : 4); ++i)
-      atomicOr(&wk[base_lo + 4 * (i & 3) + 256 * (i >> 2)], lw[i] << sh_lo);
+      for (int i = 0; i < NW; ++i) wlo[i] |= lw[i] << (8 * rh);
+      if constexpr (BITS == 3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) whi[i] |= hw[i] << (4 * (2 * (m & 1) + rh));
+      }
+      meta2[rh] = group_meta(p, asym);
+    }
+    uint32_t* chunk = reinterpret_cast<uint32_t*>(rec + block_code_off(S, j * CH + k));
+#pragma unroll
+    for (int i = 0; i < NW; ++i) chunk[base_lo + 4 * (i & 3) + 256 * (i >> 2)] = wlo[i];
     if constexpr (BITS == 3) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) atomicOr(&wk[base_hi + 4 * i], hw[i] << sh_hi);
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t full = whi[i] | __shfl_xor_sync(0xffffffffu, whi[i], 1);   // the pair with the other m & 1
+        if ((cp & 1) == 0) chunk[base_hi + 4 * i] = full;
+      }
     }
-    if (k == 0) store_meta(rec + block_meta_off(S, j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
-    __syncthreads();
-    for (int i = tid; i < CH * CW; i += nthr) {
-      const int ch = i / CW;
-      reinterpret_cast<uint32_t*>(rec + block_code_off(S, j * CH + ch))[i - ch * CW] = words[i];
-      words[i] = 0u;
+    if (k == 0) {
+      store_meta(rec + block_meta_off(S, j), block_meta_index(c0), S.meta_bytes, meta2[0]);
+      store_meta(rec + block_meta_off(S, j), block_meta_index(c0 + 1), S.meta_bytes, meta2[1]);
     }
-    __syncthreads();       // tile, words and red are free again
   }
 }
 
@@ -362,12 +376,11 @@ static int launch_store_bits(const Layout& L, const Store& S, const __half* X, i
     else quantize_rows_prefill_kernel<BITS, false><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
   } else {
     const int CH = L.G / kChunk;
-    const int smem = L.G * kD * 2 + CH * 128 * BITS * 4 + CH * 128 * 16;
+    const int smem = CH * 128 * 16;                   // reduction words of groups spanning several chunks
     auto kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true> : quantize_blocks_prefill_kernel<BITS, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
     const int n_groups = n_q / L.G;
-    dim3 grid(grid_cap(n_groups, grid_cap(148 * 8 / L.U, 1 << 16)), L.U);
-    kern<<<grid, 128 * CH, smem, st>>>(L, S, X, N, n_q, cache, inv_norm);
+    dim3 grid(grid_cap(n_groups, grid_cap(148 * 16 / L.U, 1 << 16)), L.U);
+    kern<<<grid, 64 * CH, smem, st>>>(L, S, X, N, n_q, cache, inv_norm);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
