@@ -1,6 +1,7 @@
 // Fused decode attention over the packed InnerQ cache (INNER layout), one launch:
 //   q.K^T on packed key rows  ->  online softmax  ->  p.V on packed value chunks, split over token
-//   ranges, fp16 windows and the K/V skew zone in a tail CTA, cross-CTA merge by the last CTA to finish.
+//   ranges, fp16 windows and the K/V skew zone as 16-token tiles dealt to the same warps, cross-CTA merge by
+//   the last CTA to finish.
 //
 // Work decomposition.  A CTA owns one (batch, KV head) unit and a range of value groups; each of its
 // 8 warps owns a contiguous sub-range and streams it chunk by chunk (32 tokens) through a private ring

@@ -87,6 +87,11 @@ def test_config2_prefill_then_steps():
             _, e = compare(w, gc, oc, units, step=step, check_export=step in (4, 39))
             worst = max(worst, e)
     print(f"config2: worst err/tol over steps {worst:.3f}")
+    # the tcgen05 kernel on the same cache (full size, its default split), same tolerance
+    gc.innerq_set_decode_options(0, 5)
+    _, e5 = compare(w, gc, oc, units, step=77, check_export=False)
+    gc.innerq_set_decode_options(0, 0)
+    print(f"config2, tcgen05 kernel: err/tol {e5:.3f}")
 
 
 @pytest.mark.parametrize("bits", [4, 2])
