@@ -42,8 +42,10 @@ constexpr int kOffBp = kOffBq + 4096;              // B_p: 16 columns x 128 toke
 constexpr int kOffMisc = kOffBp + 4096;            // barriers, reductions, tensor-memory base address
 constexpr int kT5Smem = kOffMisc + 512;
 
-// tensor memory columns (32-bit each, 128 lanes): A_k 64, A_v 64, D_k 16, D_v 16
-constexpr int kColAk = 0, kColAv = 64, kColDk = 128, kColDv = 144, kTmemCols = 256;
+// tensor memory (32-bit columns, 128 lanes), two allocations so that three CTAs fit into the SM's 512 columns:
+// operands A_k 64 + A_v 64, accumulators D_k 16 + D_v 16
+constexpr int kColAk = 0, kColAv = 64, kTmemColsA = 128;
+constexpr int kColDk = 0, kColDv = 16, kTmemColsD = 32;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -89,6 +91,8 @@ __device__ __forceinline__ uint32_t split_hi_lo(float x) {
 // ---- tensor memory and tcgen05 ---------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {       // one full warp
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_done() {                                  // after the CTA's last allocation
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {        // the same warp
@@ -328,13 +332,13 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const T5Args& a, int
   acc_out = acc; m_out = m_run; l_out = l_run;
 }
 
-__global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout L, const Counts cn, const T5Args a) {
+__global__ void __launch_bounds__(kT5Threads, 3) decode_tc5_kernel(const Layout L, const Counts cn, const T5Args a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x, split = blockIdx.y;
   unsigned char* misc = smem + kOffMisc;
   const uint32_t bar_full = smem_u32(misc), bar_k = bar_full + 8 * kStages, bar_v = bar_k + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48);       // [0] operands, [1] accumulators
   float* redmax = reinterpret_cast<float*>(misc + 64);
   float* redsum = reinterpret_cast<float*>(misc + 80);
   float* qg_s = reinterpret_cast<float*>(misc + 96);
@@ -367,7 +371,11 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    if (warp == 0) {
+      tmem_alloc(smem_u32(tmem_slot), kTmemColsA);
+      tmem_alloc(smem_u32(tmem_slot + 1), kTmemColsD);
+      tmem_alloc_done();
+    }
     for (int i = tid; i < 8192 / 16; i += kT5Threads) reinterpret_cast<uint4*>(smem + kOffBq)[i] = make_uint4(0u, 0u, 0u, 0u);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // ---------------- q'' and the B_q operand ---------------------------------------------------------------------
@@ -394,8 +402,9 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tbase = *tmem_slot;
+    const uint32_t tbase = tmem_slot[0], tbase_d = tmem_slot[1];
     const uint32_t t_lane = tbase + ((uint32_t)(32 * warp) << 16);   // this warp's quarter of the 128 lanes
+    const uint32_t t_lane_d = tbase_d + ((uint32_t)(32 * warp) << 16);
     const float kfac = pow2i(24 - (14 - e_q)), inv_kfac = pow2i(-(24 - (14 - e_q)));
     const float Qg[4] = {qg_s[0] * inv_kfac, qg_s[1] * inv_kfac, qg_s[2] * inv_kfac, qg_s[3] * inv_kfac};
     // this thread as a channel of the value side
@@ -434,7 +443,7 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj) {
           const uint32_t wv = vc[v_word0 + 4 * jj];
-          const uint32_t x = vrh ? (wv >> 8) : wv;
+          const uint32_t x = wv >> (8 * vrh);
 #pragma unroll
           for (int fld = 0; fld < 4; ++fld) regs[4 * jj + fld] = x & (0x00030003u << (2 * fld));
         }
@@ -445,7 +454,7 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
-        mma_ts(tbase + col_d, tbase + col_a + 8 * ks, smem_desc(smem_u32(smem + off_b) + 512 * ks, 256, 128), ks > 0);
+        mma_ts(tbase_d + col_d, tbase + col_a + 8 * ks, smem_desc(smem_u32(smem + off_b) + 512 * ks, 256, 128), ks > 0);
       mma_commit(bar);
     };
     if (n_my > 0) {
@@ -465,7 +474,7 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
       if (!failed && !mbar_wait(bar_k, (uint32_t)it & 1u)) failed = true;
       tc_fence_after();
       float d[8];
-      tmem_ld8(t_lane + kColDk, d);
+      tmem_ld8(t_lane_d + kColDk, d);
       float s;
       {
         const uint4 mw = *reinterpret_cast<const uint4*>(sp + warp * kRecBytes + kOffKMeta + lane * kKMetaRow);
@@ -519,7 +528,7 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
       if (!failed && !mbar_wait(bar_v, (uint32_t)it & 1u)) failed = true;
       tc_fence_after();
       float dv[4];
-      tmem_ld4(t_lane + kColDv, dv);
+      tmem_ld4(t_lane_d + kColDv, dv);
       tc_fence_before();
       __syncthreads();               // A_k(it+1) is complete; D_v, B_p, the reduction words and stage `st` are free
       if (tid == 0) {
@@ -540,7 +549,10 @@ __global__ void __launch_bounds__(kT5Threads, 2) decode_tc5_kernel(const Layout 
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     failed = __syncthreads_or(failed ? 1 : 0) != 0;
-    if (warp == 0) tmem_dealloc(*tmem_slot, kTmemCols);
+    if (warp == 0) {
+      tmem_dealloc(tmem_slot[0], kTmemColsA);
+      tmem_dealloc(tmem_slot[1], kTmemColsD);
+    }
     if (failed) {
       if (tid == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);
       m_run = -INFINITY; l_run = 0.f; out_c = 0.f;
@@ -584,7 +596,7 @@ int launch_decode_tc5(const Layout& L, const unsigned char* cache, unsigned char
     configured = true;
   }
   const int n_tiles = (cn.n_qv / kChunk + kChunksPerTile - 1) / kChunksPerTile;
-  if (n_splits <= 0) n_splits = (2 * 148) / L.U - 1;     // two CTAs per SM, one of a unit's CTAs takes the fp16 tail
+  if (n_splits <= 0) n_splits = (3 * 148) / L.U - 1;     // three CTAs per SM, one of a unit's CTAs takes the fp16 tail
   if (n_splits < 1) n_splits = 1;
   if (n_splits > n_tiles) n_splits = n_tiles;
   if (n_splits > L.max_splits - 1) n_splits = L.max_splits - 1;
