@@ -106,7 +106,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
-        self.sm, self.mask, self.sm_max = [], 0, None
+        self.sm, self.mem, self.mask, self.sm_max = [], [], 0, None
         self._stop_evt = threading.Event()
         self._h = None
         try:
@@ -125,6 +125,7 @@ class ClockSampler(threading.Thread):
         while not self._stop_evt.is_set():
             try:
                 self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.mem.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_MEM)))
                 self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
             except Exception:
                 try:
@@ -138,7 +139,7 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         reasons = [n for n, bit in self.REASONS.items() if self.mask & bit]
         return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.sm_max,
-                "reasons": reasons, "samples": len(self.sm)}
+                "mem_mhz": float(np.median(self.mem)) if self.mem else None, "reasons": reasons, "samples": len(self.sm)}
 
 
 def measured_peak_gbs():
@@ -246,7 +247,8 @@ def run_ours(args, w):
     R, Kst, W = args.instances, args.steps, max(args.warmup, 3)
     total_steps = W + Kst
     e2e_steps = max(4, min(Kst, 32))
-    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps) // R + 8)
+    split_steps = 2 * R * w.group if w.grouping != synth.FP16 else 0     # extra steps timed one by one (below)
+    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps + split_steps) // R + 8)
     Kh, Vh = synth.kv_all(w)
     Kd, Vd = torch.from_numpy(Kh).cuda(), torch.from_numpy(Vh).cuda()
     caches = []
@@ -276,7 +278,7 @@ def run_ours(args, w):
     del Kd, Vd, Kh, Vh, ex
     torch.cuda.empty_cache()
 
-    n_in = total_steps + e2e_steps
+    n_in = total_steps + e2e_steps + split_steps
     toks = [synth.new_token(w, s) for s in range(n_in)]
     qs = [synth.query(w, s) for s in range(n_in)]
     k_new = torch.from_numpy(np.stack([t[0] for t in toks])).cuda()
@@ -376,6 +378,29 @@ def run_ours(args, w):
     b1.record(stream)
     torch.cuda.synchronize()
     b2b_us = b0.elapsed_time(b1) / nb * 1e3
+    # steps timed one by one (events around append + decode): those on which a value group (inner grouping) or a key
+    # group (outer grouping) of G tokens is quantised, against the others
+    step_split = None
+    if split_steps:
+        base2 = total_steps + e2e_steps
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(split_steps)]
+        evict = []
+        for j in range(split_steps):
+            i = base2 + j
+            c = caches[i % R]
+            n_before = c.n_tokens
+            evs[j][0].record(stream)
+            c.innerq_append_token(k_new[i], v_new[i])
+            c.innerq_decode_attention(q_all[i], out)
+            evs[j][1].record(stream)
+            mid0, mid1 = n_before - w.w_sink - w.w_recent, n_before + 1 - w.w_sink - w.w_recent
+            evict.append(mid1 > 0 and mid1 // w.group > max(mid0, 0) // w.group)
+        torch.cuda.synchronize()
+        t_us = np.array([a_.elapsed_time(b_) * 1e3 for a_, b_ in evs])
+        ev_mask = np.array(evict)
+        step_split = {"steps": split_steps, "group_eviction_steps": int(ev_mask.sum()),
+                      "us_median_group_eviction": float(np.median(t_us[ev_mask])) if ev_mask.any() else None,
+                      "us_median_other": float(np.median(t_us[~ev_mask])) if (~ev_mask).any() else None}
     h2d = (kh[0].numel() + vh[0].numel() + qh[0].numel()) * 2
     d2h = oh.numel() * 2
 
@@ -393,6 +418,7 @@ def run_ours(args, w):
             "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
+            "step_us_by_kind": step_split,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
