@@ -248,6 +248,22 @@ def test_step_from_host_buffers_matches_separate_calls_and_oracle():
     assert gc.n_tokens == 340
 
 
+@pytest.mark.parametrize("w_sink,w_recent", [(0, 0), (0, 7), (5, 0)])
+def test_degenerate_windows(w_sink, w_recent):
+    # no sink and / or no recent window: every token (w_recent = 0: even the newest) is quantised
+    w = synth.tiny(n_tokens=230, w_sink=w_sink, w_recent=w_recent)
+    oc, gc, _, _ = run_prefill_both(w)
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
+    check_decode(w, oc, gc, variants=(0, 1))
+    for step in range(40):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        if step in (0, 1, 25, 26, 39):
+            check_decode(w, oc, gc, step=step, variants=(0, 1))
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
