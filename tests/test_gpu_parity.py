@@ -248,6 +248,14 @@ def test_step_from_host_buffers_matches_separate_calls_and_oracle():
     assert gc.n_tokens == 340
 
 
+@pytest.mark.parametrize("r,G,bits", [(3, 64, 2), (6, 32, 4), (5, 128, 3), (16, 64, 2)])
+def test_query_heads_per_kv_head_not_a_multiple_of_four(r, G, bits):
+    # the fused kernel takes up to four query heads of a KV head per pass: partial and multiple passes
+    w = synth.tiny(n_tokens=450, group=G, k_bits=bits, v_bits=bits, n_q_heads=2 * r)
+    oc, gc, _, _ = run_prefill_both(w)
+    check_decode(w, oc, gc, variants=(3, 4, 1), splits=(0, 2))
+
+
 @pytest.mark.parametrize("w_sink,w_recent", [(0, 0), (0, 7), (5, 0)])
 def test_degenerate_windows(w_sink, w_recent):
     # no sink and / or no recent window: every token (w_recent = 0: even the newest) is quantised
