@@ -13,8 +13,10 @@
 //   values: thread c expands the codes of channel c for the tile's 128 tokens as row c of A_v; B_p has one column
 //           per chunk (= value group) holding p of that chunk's tokens; D_v[128 channels x 16] are the per-group
 //           sums, to which thread c applies the group's scale / zero-point of its channel.
-// The MMAs run asynchronously; the expansion of the next operand overlaps them.  Same records, same bulk-copy
-// pipeline, same split merge as the warp-level kernel.
+// The MMAs run asynchronously; the expansion of the next operand overlaps them.  A fifth warp starts the bulk copies
+// and issues the MMAs; it and the four compute warps hand work to each other through mbarriers only.  Same records,
+// same bulk-copy pipeline, same split merge as the warp-level kernel; the fp16 windows and the K/V skew zone are
+// handled with plain SIMT code, a slice per CTA, before its first tile.
 #include "innerq_device.cuh"
 #include "innerq_kernels.h"
 
@@ -40,7 +42,8 @@ constexpr int kStages = 3;
 constexpr int kOffBq = kStages * kTileBytes;       // B_q: 16 columns x 128 channels fp16, canonical K-major layout
 constexpr int kOffBp = kOffBq + 4096;              // B_p: 16 columns x 128 tokens
 constexpr int kOffMisc = kOffBp + 4096;            // barriers, reductions, tensor-memory base address
-constexpr int kT5Smem = kOffMisc + 512;
+constexpr int kOffScratch = kOffMisc + 512;        // scratch of the fp16 / skew token slice (3 * 128 + 8 floats)
+constexpr int kT5Smem = kOffScratch + 2048;
 
 // tensor memory (32-bit columns, 128 lanes), two allocations so that three CTAs fit into the SM's 512 columns:
 // operands A_k 64 + A_v 64, accumulators D_k 16 + D_v 16
@@ -157,7 +160,7 @@ struct T5Args {
   unsigned char* ws;
   const __half* q;
   __half* out;
-  int n_splits;        // CTAs per unit streaming packed tiles; CTA n_splits of a unit handles the fp16 tail
+  int n_splits;        // CTAs per unit (= gridDim.y)
   int k_ring_pos0, v_ring_pos0;
 };
 
@@ -181,11 +184,11 @@ __device__ __forceinline__ int b_offset(int n, int k) { return (k >> 3) * 256 + 
 // Log-sum-exp merge of the partial results of a unit (see innerq_decode_mma.cuh); four warps.
 __device__ __noinline__ void merge_parts4(const float* __restrict__ partials, float* wm, __half* __restrict__ out,
                                           int n_parts, int head, int max_splits) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;       // warps 0..3 work, a fifth only joins the barrier
   float M = -INFINITY, den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
   const float* Ph = partials + (size_t)head * max_splits * kPartialStride;
 #pragma unroll 1
-  for (int s0 = warp; s0 < n_parts; s0 += 4 * 4) {
+  for (int s0 = warp; s0 < n_parts && warp < 4; s0 += 4 * 4) {
     float4 v[4];
     float2 ml[4];
 #pragma unroll
@@ -209,11 +212,14 @@ __device__ __noinline__ void merge_parts4(const float* __restrict__ partials, fl
       n3 = fmaf(n3, a_old, v[e].w * a_new);
     }
   }
-  float* mine = wm + warp * (kD + 2);
-  *reinterpret_cast<float2*>(mine + 4 * lane) = make_float2(n0, n1);
-  *reinterpret_cast<float2*>(mine + 4 * lane + 2) = make_float2(n2, n3);
-  if (lane == 0) { mine[kD] = M; mine[kD + 1] = den; }
+  if (warp < 4) {
+    float* mine = wm + warp * (kD + 2);
+    *reinterpret_cast<float2*>(mine + 4 * lane) = make_float2(n0, n1);
+    *reinterpret_cast<float2*>(mine + 4 * lane + 2) = make_float2(n2, n3);
+    if (lane == 0) { mine[kD] = M; mine[kD + 1] = den; }
+  }
   __syncthreads();
+  if (warp >= 4) return;
   const int c = tid;
   float Mx = -INFINITY;
 #pragma unroll
@@ -229,12 +235,13 @@ __device__ __noinline__ void merge_parts4(const float* __restrict__ partials, fl
   out[(size_t)head * kD + c] = __float2half_rn(num / dn);
 }
 
-// block-wide max / sum over 128 threads through four shared words (two barriers each)
+// block-wide max / sum over the first 128 threads through four shared words (two barriers each; a fifth warp of
+// the CTA joins the barriers with a neutral value)
 __device__ __forceinline__ float block_max(float v, float* red4) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   __syncthreads();
-  if ((threadIdx.x & 31) == 0) red4[threadIdx.x >> 5] = v;
+  if ((threadIdx.x & 31) == 0 && threadIdx.x < kT5Threads) red4[threadIdx.x >> 5] = v;
   __syncthreads();
   return fmaxf(fmaxf(red4[0], red4[1]), fmaxf(red4[2], red4[3]));
 }
@@ -242,30 +249,32 @@ __device__ __forceinline__ float block_sum(float v, float* red4) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   __syncthreads();
-  if ((threadIdx.x & 31) == 0) red4[threadIdx.x >> 5] = v;
+  if ((threadIdx.x & 31) == 0 && threadIdx.x < kT5Threads) red4[threadIdx.x >> 5] = v;
   __syncthreads();
   return (red4[0] + red4[1]) + (red4[2] + red4[3]);
 }
 
-// The tokens outside the range where keys and values are both packed, by one CTA per unit with plain SIMT code
-// (at most a few hundred tokens): the K/V skew zone (packed key rows n_qv .., fp16 values from the value ring), the
-// sink window and the recent window (fp16 both).  Thread = token for the scores, thread = channel for the values.
+// The tokens outside the range where keys and values are both packed (at most a few hundred per unit): the K/V skew
+// zone (packed key rows n_qv .., fp16 values from the value ring), the sink window and the recent window (fp16
+// both), as one list of entries.  Every CTA of a unit takes a slice [e_lo, e_hi) of the list before it starts on
+// its packed tiles, with plain SIMT code: thread = token for the scores, thread = channel for the values.
 // fbuf: 3 * 128 + 8 floats of shared memory.  Results: this thread's channel sum, running max and sum.
-__device__ void tail_cta(const Layout& L, const Counts& cn, const T5Args& a, int u, float* fbuf, float& acc_out,
-                         float& m_out, float& l_out) {
+__device__ void tail_slice(const Layout& L, const Counts& cn, const T5Args& a, int u, int e_lo, int e_hi, float* fbuf,
+                           float& acc_out, float& m_out, float& l_out) {
   const int tid = threadIdx.x;
+  const bool act = tid < kT5Threads;        // the CTA's fifth warp only joins the barriers
   float* qs = fbuf;            // q'' raw
   float* qn = fbuf + 128;      // q'' * norm (packed key rows)
   float* ps = fbuf + 256;      // probabilities of the current round
   float* red4 = fbuf + 384;
   const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-  {
+  if (act) {
     const float v = __half2float(a.q[(size_t)u * kD + tid]) * (L.sm_scale * kLog2e);
     qs[tid] = v;
     qn[tid] = L.k_normalize ? v * norm[tid] : v;
   }
   __syncthreads();
-  const int n_skew = cn.n_qk - cn.n_qv, n_list = cn.n_sink + cn.n_k_recent, total = n_skew + n_list;
+  const int n_skew = cn.n_qk - cn.n_qv;
   const unsigned char* rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const __half* k_sink = reinterpret_cast<const __half*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
   const __half* k_ring = reinterpret_cast<const __half*>(a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride);
@@ -278,26 +287,33 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const T5Args& a, int
     return v_ring + (size_t)slot * kD;
   };
   float m_run = -INFINITY, l_run = 0.f, acc = 0.f;
-  for (int e0 = 0; e0 < total; e0 += kT5Threads) {
-    const int e = e0 + tid;
+  for (int e0 = e_lo; e0 < e_hi; e0 += kT5Threads) {
+    const int e = act ? e0 + tid : e_hi;
     float s = -INFINITY;
-    if (e < n_skew) {                                   // packed key row
+    if (e < n_skew && e < e_hi) {                       // packed key row
       const int i = cn.n_qv + e;
-      const uint32_t* row = reinterpret_cast<const uint32_t*>(rec + row_code_off(L.k, i));
-      const unsigned char* meta = rec + row_meta_off(L.k, i);
+      const uint4* row4 = reinterpret_cast<const uint4*>(rec + row_code_off(L.k, i));
+      const uint4 r0 = __ldg(row4), r1 = __ldg(row4 + 1);
+      const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+      const uint4 mw = __ldg(reinterpret_cast<const uint4*>(rec + row_meta_off(L.k, i)));
+      const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
       float d = 0.f;
-      for (int g = 0; g < kD / 32; ++g) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
         float sc, zc;
-        decode_meta(load_meta(meta, g, L.k.meta_bytes), L.k.bits, sc, zc);
+        decode_meta(mws[g], 2, sc, zc);
         float dg = 0.f, qg = 0.f;
-        for (int c = 32 * g; c < 32 * g + 32; ++c) {
-          dg = fmaf(qn[c], (float)row_code(row, c, L.k.bits), dg);
+#pragma unroll
+        for (int cc = 0; cc < 32; ++cc) {
+          const int c = 32 * g + cc, k = key_k_index(c);            // word (k / 2) / 8, field (k / 2) % 8, half k % 2
+          const uint32_t code = (w[k >> 4] >> (16 * (k & 1) + 2 * ((k >> 1) & 7))) & 3u;
+          dg = fmaf(qn[c], (float)code, dg);
           qg += qn[c];
         }
         d = fmaf(sc, dg, fmaf(zc, qg, d));
       }
       s = d;
-    } else if (e < total) {
+    } else if (e < e_hi) {
       const int le = e - n_skew;
       const __half* kr;
       if (le < cn.n_sink) kr = k_sink + (size_t)le * kD;
@@ -320,44 +336,65 @@ __device__ void tail_cta(const Layout& L, const Counts& cn, const T5Args& a, int
     }
     const float m_new = fmaxf(m_run, block_max(s, red4));
     const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
-    const float p = e < total ? ex2_approx(s - m_new) : 0.f;
-    ps[tid] = p;
+    const float p = e < e_hi ? ex2_approx(s - m_new) : 0.f;
+    if (act) ps[tid] = p;
     l_run = l_run * alpha + block_sum(p, red4);         // (its barriers also publish ps)
     m_run = m_new;
     acc *= alpha;
-    const int n = min(kT5Threads, total - e0);
-    for (int ee = 0; ee < n; ++ee) acc = fmaf(ps[ee], __half2float(v_row(e0 + ee)[tid]), acc);
+    const int n = min(kT5Threads, e_hi - e0);
+    if (act)
+      for (int ee = 0; ee < n; ++ee) acc = fmaf(ps[ee], __half2float(v_row(e0 + ee)[tid]), acc);
     __syncthreads();
   }
   acc_out = acc; m_out = m_run; l_out = l_run;
 }
 
-__global__ void __launch_bounds__(kT5Threads, 3) decode_tc5_kernel(const Layout L, const Counts cn, const T5Args a) {
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// warp-wide maximum of floats / sum of non-negative floats <= 1 with one redux instruction each
+__device__ __forceinline__ float warp_max(float v) {
+  int b = __float_as_int(v);
+  b ^= (b >> 31) & 0x7fffffff;                       // order-preserving map to signed integers (an involution)
+  b = __reduce_max_sync(0xffffffffu, b);
+  b ^= (b >> 31) & 0x7fffffff;
+  return __int_as_float(b);
+}
+__device__ __forceinline__ float warp_sum_unit(float v) {      // 24 fractional bits
+  return (float)__reduce_add_sync(0xffffffffu, (unsigned)__float2uint_rn(v * 0x1p24f)) * 0x1p-24f;
+}
+
+constexpr int kT5Block = kT5Threads + 32;            // four compute warps and the issuing warp
+
+// Compute warps 0..3: thread t is token t of the tile on the key side and channel t on the value side.  Warp 4:
+// its lane 0 starts the bulk copies and issues the MMAs.  They talk through mbarriers only (no CTA barrier in the
+// loop):   ak_ready / avbp_ready (128 arrivals: the operands of the key / value MMA are complete),
+//          dk_done / dv_done (the MMA's commit), full[s] / empty[s] (a stage's data has arrived / been consumed).
+// Software pipeline of a compute thread:  MMA-K(i) || expand V(i);  MMA-V(i) || expand K(i+1);  MMA-K(i+1) || output(i).
+__global__ void __launch_bounds__(kT5Block, 3) decode_tc5_kernel(const Layout L, const Counts cn, const T5Args a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool compute = warp < 4;
   const int u = blockIdx.x, split = blockIdx.y;
   unsigned char* misc = smem + kOffMisc;
-  const uint32_t bar_full = smem_u32(misc), bar_k = bar_full + 8 * kStages, bar_v = bar_k + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 48);       // [0] operands, [1] accumulators
-  float* redmax = reinterpret_cast<float*>(misc + 64);
-  float* redsum = reinterpret_cast<float*>(misc + 80);
-  float* qg_s = reinterpret_cast<float*>(misc + 96);
-  float* red4 = reinterpret_cast<float*>(misc + 112);
+  const uint32_t bar_full = smem_u32(misc), bar_empty = bar_full + 8 * kStages, bar_ak = bar_empty + 8 * kStages,
+                 bar_avbp = bar_ak + 8, bar_dk = bar_avbp + 8, bar_dv = bar_dk + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 96);       // [0] operands, [1] accumulators
+  float* redmax = reinterpret_cast<float*>(misc + 128);
+  float* redsum = reinterpret_cast<float*>(misc + 144);
+  float* qg_s = reinterpret_cast<float*>(misc + 160);
+  float* red4 = reinterpret_cast<float*>(misc + 176);
   __shared__ unsigned int s_ticket;
   const int n_parts = gridDim.y;
   float out_c = 0.f, m_run = -INFINITY, l_run = 0.f;      // this thread's channel of the partial result
   bool failed = false;
 
-  if (split == a.n_splits) {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    tail_cta(L, cn, a, u, reinterpret_cast<float*>(smem), out_c, m_run, l_run);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  } else {
+  {
     const int n_chunks = cn.n_qv / kChunk, n_tiles = (n_chunks + kChunksPerTile - 1) / kChunksPerTile;
     const int t_lo = (int)((long long)split * n_tiles / a.n_splits), t_hi = (int)((long long)(split + 1) * n_tiles / a.n_splits);
     const int n_my = t_hi - t_lo;
     const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
-    auto issue = [&](int it) {      // thread 0: tile t_lo + it into stage it % kStages
+    auto issue = [&](int it) {      // issuing lane: tile t_lo + it into stage it % kStages
       const int ti = t_lo + it, st = it % kStages;
       const int nv = min(kChunksPerTile, n_chunks - kChunksPerTile * ti);
       const uint32_t bytes = (uint32_t)nv * kRecBytes;
@@ -367,28 +404,44 @@ __global__ void __launch_bounds__(kT5Threads, 3) decode_tc5_kernel(const Layout 
     // ---------------- set-up that touches no global memory -------------------------------------------------------
     if (tid == 0) {
 #pragma unroll
-      for (int s = 0; s < kStages + 2; ++s) mbar_init(bar_full + 8 * s, 1);
+      for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, kT5Threads); }
+      mbar_init(bar_ak, kT5Threads);
+      mbar_init(bar_avbp, kT5Threads);
+      mbar_init(bar_dk, 1);
+      mbar_init(bar_dv, 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == 4) {
       tmem_alloc(smem_u32(tmem_slot), kTmemColsA);
       tmem_alloc(smem_u32(tmem_slot + 1), kTmemColsD);
       tmem_alloc_done();
     }
-    for (int i = tid; i < 8192 / 16; i += kT5Threads) reinterpret_cast<uint4*>(smem + kOffBq)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < 8192 / 16; i += kT5Block) reinterpret_cast<uint4*>(smem + kOffBq)[i] = make_uint4(0u, 0u, 0u, 0u);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // ---------------- q'' and the B_q operand ---------------------------------------------------------------------
     const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-    float qv = __half2float(a.q[(size_t)u * kD + tid]) * (L.sm_scale * kLog2e);
-    if (L.k_normalize) qv *= norm[tid];
+    float qv = 0.f;
+    if (compute) {
+      qv = __half2float(a.q[(size_t)u * kD + tid]) * (L.sm_scale * kLog2e);
+      if (L.k_normalize) qv *= norm[tid];
+    }
     __syncthreads();                 // barrier init, zero fill and the tensor-memory address are visible
-    if (tid == 0)
+    if (warp == 4 && lane == 0)
       for (int it = 0; it < kStages && it < n_my; ++it) issue(it);
-    const float amax = block_max(fabsf(qv), red4);
+    // this CTA's slice of the unit's fp16 / skew tokens, while the first tiles are on their way
+    {
+      const int total = (cn.n_qk - cn.n_qv) + cn.n_sink + cn.n_k_recent;
+      const int e_lo = (int)((long long)split * total / gridDim.y), e_hi = (int)((long long)(split + 1) * total / gridDim.y);
+      tail_slice(L, cn, a, u, e_lo, e_hi, reinterpret_cast<float*>(smem + kOffScratch), out_c, m_run, l_run);
+    }
+    float amax = warp_max(fabsf(qv));
+    if (compute && lane == 0) red4[warp] = amax;
+    __syncthreads();
+    amax = fmaxf(fmaxf(red4[0], red4[1]), fmaxf(red4[2], red4[3]));
     int e_q = 0;
     if (amax > 0.f && amax < INFINITY) e_q = ((__float_as_int(amax) >> 23) & 0xff) - 126;     // amax < 2^e_q
-    {
+    if (compute) {
       const int k = key_k_index(tid), g = tid >> 5;
       const uint32_t v = split_hi_lo(qv * pow2i(14 - e_q - 2 * key_field(tid)));
       *reinterpret_cast<uint16_t*>(smem + kOffBq + b_offset(2 * g, k)) = (uint16_t)(v & 0xFFFFu);
@@ -403,153 +456,160 @@ __global__ void __launch_bounds__(kT5Threads, 3) decode_tc5_kernel(const Layout 
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = tmem_slot[0], tbase_d = tmem_slot[1];
-    const uint32_t t_lane = tbase + ((uint32_t)(32 * warp) << 16);   // this warp's quarter of the 128 lanes
-    const uint32_t t_lane_d = tbase_d + ((uint32_t)(32 * warp) << 16);
-    const float kfac = pow2i(24 - (14 - e_q)), inv_kfac = pow2i(-(24 - (14 - e_q)));
-    const float Qg[4] = {qg_s[0] * inv_kfac, qg_s[1] * inv_kfac, qg_s[2] * inv_kfac, qg_s[3] * inv_kfac};
-    // this thread as a channel of the value side
-    const int vm_ = 4 * (tid >> 6) + ((tid >> 1) & 3), vgid = (tid >> 3) & 7, vrh = tid & 1;
-    const int v_word0 = (vm_ >> 2) * 128 + 16 * vgid + (vm_ & 3);          // + 4 * jj
-    const int v_meta_idx = block_meta_index(tid);
-    // this thread as a token of the key side: where its probability goes in B_p
-    const int p_off = b_offset(warp, val_k_index(warp, lane));
-    const float p_scale = pow2i(10 - 2 * val_field(lane));
 
-    // Software pipeline over the tiles of this CTA.  The two MMAs of a tile run asynchronously; while they do, the
-    // threads expand the next operand:   MMA-K(i) || expand V(i);   MMA-V(i) || expand K(i+1);   MMA-K(i+1) || output(i).
-    // (A wait that runs out does not leave the loop: every thread keeps passing the same CTA barriers; later waits
-    // are skipped and the result is discarded.)
-    auto expand_keys = [&](const unsigned char* sp) {       // packed row of token `tid` -> row `tid` of A_k
-      const uint4* row = reinterpret_cast<const uint4*>(sp + warp * kRecBytes + lane * kKRow);
-      const uint4 r0 = row[0], r1 = row[1];
-      const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+    if (!compute) {
+      // ======================= issuing warp ======================================================================
+      if (lane == 0) {
+        auto issue_mma = [&](int col_d, int col_a, int off_b, uint32_t bar) {
+          tc_fence_after();
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint32_t regs[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int wi = 2 * q4 + (i >> 3), fld = i & 7;
-          const uint32_t x = fld >= 4 ? (w[wi] >> 8) : w[wi];
-          regs[i] = x & (0x00030003u << (2 * (fld & 3)));
+          for (int ks = 0; ks < 8; ++ks)
+            mma_ts(tbase_d + col_d, tbase + col_a + 8 * ks, smem_desc(smem_u32(smem + off_b) + 512 * ks, 256, 128), ks > 0);
+          mma_commit(bar);
+        };
+        for (int it = 0; it < n_my && !failed; ++it) {
+          if (!mbar_wait(bar_ak, (uint32_t)it & 1u)) { failed = true; break; }
+          issue_mma(kColDk, kColAk, kOffBq, bar_dk);
+          if (it >= 1 && it - 1 + kStages < n_my) {                  // the stage of tile it-1 has been consumed: refill it
+            if (!mbar_wait(bar_empty + 8 * ((it - 1) % kStages), (uint32_t)((it - 1) / kStages) & 1u)) { failed = true; break; }
+            issue(it - 1 + kStages);
+          }
+          if (!mbar_wait(bar_avbp, (uint32_t)it & 1u)) { failed = true; break; }
+          issue_mma(kColDv, kColAv, kOffBp, bar_dv);
         }
-        tmem_st16(t_lane + kColAk + 16 * q4, regs);
       }
-    };
-    auto expand_values = [&](const unsigned char* sp) {     // codes of channel `tid` for the tile's tokens -> A_v
+      __syncwarp();
+    } else {
+      // ======================= compute warps =====================================================================
+      const uint32_t t_lane = tbase + ((uint32_t)(32 * warp) << 16);   // this warp's quarter of the 128 lanes
+      const uint32_t t_lane_d = tbase_d + ((uint32_t)(32 * warp) << 16);
+      const float kfac = pow2i(24 - (14 - e_q)), inv_kfac = pow2i(-(24 - (14 - e_q)));
+      const float Qg[4] = {qg_s[0] * inv_kfac, qg_s[1] * inv_kfac, qg_s[2] * inv_kfac, qg_s[3] * inv_kfac};
+      // this thread as a channel of the value side
+      const int vm_ = 4 * (tid >> 6) + ((tid >> 1) & 3), vgid = (tid >> 3) & 7, vrh = tid & 1;
+      const int v_word0 = (vm_ >> 2) * 128 + 16 * vgid + (vm_ & 3);          // + 4 * jj
+      const int v_meta_idx = block_meta_index(tid);
+      // this thread as a token of the key side: where its probability goes in B_p
+      const int p_off = b_offset(warp, val_k_index(warp, lane));
+      const float p_scale = pow2i(10 - 2 * val_field(lane));
+      auto expand_keys = [&](const unsigned char* sp) {       // packed row of token `tid` -> row `tid` of A_k
+        const uint4* row = reinterpret_cast<const uint4*>(sp + warp * kRecBytes + lane * kKRow);
+        const uint4 r0 = row[0], r1 = row[1];
+        const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
-      for (int ch = 0; ch < kChunksPerTile; ++ch) {
-        const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVCodes);
-        uint32_t regs[16];
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t regs[16];
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const uint32_t wv = vc[v_word0 + 4 * jj];
-          const uint32_t x = wv >> (8 * vrh);
-#pragma unroll
-          for (int fld = 0; fld < 4; ++fld) regs[4 * jj + fld] = x & (0x00030003u << (2 * fld));
+          for (int i = 0; i < 16; ++i) {
+            const int wi = 2 * q4 + (i >> 3), fld = i & 7;
+            const uint32_t x = fld >= 4 ? (w[wi] >> 8) : w[wi];
+            regs[i] = x & (0x00030003u << (2 * (fld & 3)));
+          }
+          tmem_st16(t_lane + kColAk + 16 * q4, regs);
         }
-        tmem_st16(t_lane + kColAv + 16 * ch, regs);
-      }
-    };
-    auto issue_mma = [&](int col_d, int col_a, int off_b, uint32_t bar) {   // thread 0
-      tc_fence_after();
+      };
+      auto expand_values = [&](const unsigned char* sp) {     // codes of channel `tid` for the tile's tokens -> A_v
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        mma_ts(tbase_d + col_d, tbase + col_a + 8 * ks, smem_desc(smem_u32(smem + off_b) + 512 * ks, 256, 128), ks > 0);
-      mma_commit(bar);
-    };
-    if (n_my > 0) {
-      if (!mbar_wait(bar_full, 0u)) failed = true;
-      expand_keys(smem);
-      tc_wait_st();
-      tc_fence_before();
-      __syncthreads();
-      if (tid == 0) issue_mma(kColDk, kColAk, kOffBq, bar_k);
-    }
-    for (int it = 0; it < n_my; ++it) {
-      const int st = it % kStages, ti = t_lo + it;
-      const int nv = min(kChunksPerTile, n_chunks - kChunksPerTile * ti);
-      const unsigned char* sp = smem + st * kTileBytes;
-      expand_values(sp);                                                       // || MMA-K(it)
-      // ---------------- scores of token `tid`; probabilities relative to the chunk's own maximum -------------------
-      if (!failed && !mbar_wait(bar_k, (uint32_t)it & 1u)) failed = true;
-      tc_fence_after();
-      float d[8];
-      tmem_ld8(t_lane_d + kColDk, d);
-      float s;
-      {
-        const uint4 mw = *reinterpret_cast<const uint4*>(sp + warp * kRecBytes + kOffKMeta + lane * kKMetaRow);
-        const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
-        float acc = 0.f;
+        for (int ch = 0; ch < kChunksPerTile; ++ch) {
+          const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVCodes);
+          uint32_t regs[16];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const __half2 h2 = *reinterpret_cast<const __half2*>(&mws[g]);
-          const float sg = __low2float(h2);
-          const float z = fmaf(-2.0f, fmaxf(sg, 0.f), __high2float(h2));       // symmetric groups: -s * 2^(b-1)
-          acc = fmaf(fabsf(sg), d[2 * g] + d[2 * g + 1], fmaf(z, Qg[g], acc));
+          for (int jj = 0; jj < 4; ++jj) {
+            const uint32_t x = vc[v_word0 + 4 * jj] >> (8 * vrh);
+#pragma unroll
+            for (int fld = 0; fld < 4; ++fld) regs[4 * jj + fld] = x & (0x00030003u << (2 * fld));
+          }
+          tmem_st16(t_lane + kColAv + 16 * ch, regs);
         }
-        s = warp < nv ? acc * kfac : -INFINITY;
-      }
-      float wmax = s;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
-      const float p = warp < nv ? ex2_approx(s - wmax) : 0.f;                  // chunk = warp = one column of B_p
-      float wsum = p;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-      if (lane == 0) { redmax[warp] = wmax; redsum[warp] = wsum; }
-      *reinterpret_cast<__half*>(smem + kOffBp + p_off) = __float2half_rn(p * p_scale);
-      tc_wait_st();                                                            // A_v
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");             // B_p
-      tc_fence_before();
-      __syncthreads();
-      if (tid == 0) issue_mma(kColDv, kColAv, kOffBp, bar_v);
-      // the chunks' maxima and sums, brought to the new running maximum
-      float cm[4], cs[4];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) { cm[ch] = redmax[ch]; cs[ch] = redsum[ch]; }
-      const float m_new = fmaxf(m_run, fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])));
-      const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
-      float cw[4];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) cw[ch] = cm[ch] == -INFINITY ? 0.f : ex2_approx(cm[ch] - m_new);
-      l_run = l_run * alpha + ((cs[0] * cw[0] + cs[1] * cw[1]) + (cs[2] * cw[2] + cs[3] * cw[3]));
-      m_run = m_new;
-      // value metadata of channel `tid` (the stage is handed back before it is used)
-      uint32_t vmeta[4];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch)
-        vmeta[ch] = *reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVMeta + 4 * v_meta_idx);
-      if (it + 1 < n_my) {                                                     // || MMA-V(it)
-        const int st1 = (it + 1) % kStages;
-        if (!failed && !mbar_wait(bar_full + 8 * st1, (uint32_t)((it + 1) / kStages) & 1u)) failed = true;
-        expand_keys(smem + st1 * kTileBytes);
+      };
+      // (A wait that runs out does not leave the loop; later waits are skipped and the result is discarded.)
+      if (n_my > 0) {
+        if (!mbar_wait(bar_full, 0u)) failed = true;
+        expand_keys(smem);
         tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_ak);
       }
-      if (!failed && !mbar_wait(bar_v, (uint32_t)it & 1u)) failed = true;
-      tc_fence_after();
-      float dv[4];
-      tmem_ld4(t_lane_d + kColDv, dv);
-      tc_fence_before();
-      __syncthreads();               // A_k(it+1) is complete; D_v, B_p, the reduction words and stage `st` are free
-      if (tid == 0) {
-        if (it + 1 < n_my) issue_mma(kColDk, kColAk, kOffBq, bar_k);
-        if (it + kStages < n_my) issue(it + kStages);
-      }
-      // ---------------- output channel `tid` ------------------------------------------------- || MMA-K(it+1) ------
-      out_c *= alpha;
+      for (int it = 0; it < n_my; ++it) {
+        const int st = it % kStages, ti = t_lo + it;
+        const int nv = min(kChunksPerTile, n_chunks - kChunksPerTile * ti);
+        const unsigned char* sp = smem + st * kTileBytes;
+        expand_values(sp);                                                       // || MMA-K(it)
+        // ---------------- scores of token `tid`; probabilities relative to the chunk's own maximum -----------------
+        if (!failed && !mbar_wait(bar_dk, (uint32_t)it & 1u)) failed = true;
+        tc_fence_after();
+        float d[8];
+        tmem_ld8(t_lane_d + kColDk, d);
+        float s;
+        {
+          const uint4 mw = *reinterpret_cast<const uint4*>(sp + warp * kRecBytes + kOffKMeta + lane * kKMetaRow);
+          const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+          float acc = 0.f;
 #pragma unroll
-      for (int ch = 0; ch < kChunksPerTile; ++ch) {
-        if (ch < nv) {
-          const __half2 h2 = *reinterpret_cast<const __half2*>(&vmeta[ch]);
-          const float sg = __low2float(h2);
-          const float z = fmaf(-2.0f, fmaxf(sg, 0.f), __high2float(h2));
-          out_c = fmaf(cw[ch], fmaf(fabsf(sg), dv[ch] * 0x1p14f, z * cs[ch]), out_c);
+          for (int g = 0; g < 4; ++g) {
+            const __half2 h2 = *reinterpret_cast<const __half2*>(&mws[g]);
+            const float sg = __low2float(h2);
+            const float z = fmaf(-2.0f, fmaxf(sg, 0.f), __high2float(h2));       // symmetric groups: -s * 2^(b-1)
+            acc = fmaf(fabsf(sg), d[2 * g] + d[2 * g + 1], fmaf(z, Qg[g], acc));
+          }
+          s = warp < nv ? acc * kfac : -INFINITY;
+        }
+        const float wmax = warp_max(s);
+        const float p = warp < nv ? ex2_approx(s - wmax) : 0.f;                  // chunk = warp = one column of B_p
+        const float wsum = warp_sum_unit(p);
+        if (lane == 0) { redmax[warp] = wmax; redsum[warp] = wsum; }
+        *reinterpret_cast<__half*>(smem + kOffBp + p_off) = __float2half_rn(p * p_scale);
+        tc_wait_st();                                                            // A_v
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");             // B_p
+        tc_fence_before();
+        mbar_arrive(bar_avbp);
+        // value metadata of channel `tid` (the stage is handed back before it is used)
+        uint32_t vmeta[4];
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+          vmeta[ch] = *reinterpret_cast<const uint32_t*>(sp + ch * kRecBytes + kOffVMeta + 4 * v_meta_idx);
+        if (it + 1 < n_my) {                                                     // || MMA-V(it)
+          const int st1 = (it + 1) % kStages;
+          if (!failed && !mbar_wait(bar_full + 8 * st1, (uint32_t)((it + 1) / kStages) & 1u)) failed = true;
+          expand_keys(smem + st1 * kTileBytes);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar_ak);
+        }
+        // the chunks' maxima and sums (all four warps have written theirs once avbp_ready has completed)
+        if (!failed && !mbar_wait(bar_avbp, (uint32_t)it & 1u)) failed = true;
+        float cm[4], cs[4];
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) { cm[ch] = redmax[ch]; cs[ch] = redsum[ch]; }
+        const float m_new = fmaxf(m_run, fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])));
+        const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
+        float cw[4];
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) cw[ch] = cm[ch] == -INFINITY ? 0.f : ex2_approx(cm[ch] - m_new);
+        l_run = l_run * alpha + ((cs[0] * cw[0] + cs[1] * cw[1]) + (cs[2] * cw[2] + cs[3] * cw[3]));
+        m_run = m_new;
+        if (!failed && !mbar_wait(bar_dv, (uint32_t)it & 1u)) failed = true;
+        tc_fence_after();
+        float dv[4];
+        tmem_ld4(t_lane_d + kColDv, dv);
+        tc_fence_before();
+        mbar_arrive(bar_empty + 8 * st);                                         // stage, D_v and B_p are free again
+        // ---------------- output channel `tid` ------------------------------------------------- || MMA-K(it+1) ----
+        out_c *= alpha;
+#pragma unroll
+        for (int ch = 0; ch < kChunksPerTile; ++ch) {
+          if (ch < nv) {
+            const __half2 h2 = *reinterpret_cast<const __half2*>(&vmeta[ch]);
+            const float sg = __low2float(h2);
+            const float z = fmaf(-2.0f, fmaxf(sg, 0.f), __high2float(h2));
+            out_c = fmaf(cw[ch], fmaf(fabsf(sg), dv[ch] * 0x1p14f, z * cs[ch]), out_c);
+          }
         }
       }
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     failed = __syncthreads_or(failed ? 1 : 0) != 0;
-    if (warp == 0) {
+    if (warp == 4) {
       tmem_dealloc(tmem_slot[0], kTmemColsA);
       tmem_dealloc(tmem_slot[1], kTmemColsD);
     }
@@ -561,7 +621,7 @@ __global__ void __launch_bounds__(kT5Threads, 3) decode_tc5_kernel(const Layout 
 
   // ---------------- partial result, ticket, merge by the last CTA of the unit ------------------------------------
   float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
-  {
+  if (compute) {
     float* P = partials + ((size_t)u * L.max_splits + split) * kPartialStride;
     P[tid] = m_run == -INFINITY ? 0.f : out_c;
     if (tid == 0) { P[kD] = m_run; P[kD + 1] = l_run; }
@@ -596,18 +656,17 @@ int launch_decode_tc5(const Layout& L, const unsigned char* cache, unsigned char
     configured = true;
   }
   const int n_tiles = (cn.n_qv / kChunk + kChunksPerTile - 1) / kChunksPerTile;
-  if (n_splits <= 0) n_splits = (3 * 148) / L.U - 1;     // three CTAs per SM, one of a unit's CTAs takes the fp16 tail
-  if (n_splits < 1) n_splits = 1;
+  if (n_splits <= 0) n_splits = (3 * 148) / L.U;         // three CTAs per SM
   if (n_splits > n_tiles) n_splits = n_tiles;
-  if (n_splits > L.max_splits - 1) n_splits = L.max_splits - 1;
-  if (n_splits < 0) n_splits = 0;
+  if (n_splits > L.max_splits) n_splits = L.max_splits;
+  if (n_splits < 1) n_splits = 1;                        // short contexts: the fp16 tokens only
   T5Args a;
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
   a.k_ring_pos0 = L.k.ring_cap ? cn.n_qk % L.k.ring_cap : 0;
   a.v_ring_pos0 = L.v.ring_cap ? cn.n_qv % L.v.ring_cap : 0;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(L.U, n_splits + 1); cfg.blockDim = dim3(kT5Threads); cfg.dynamicSmemBytes = kT5Smem; cfg.stream = st;
+  cfg.gridDim = dim3(L.U, n_splits); cfg.blockDim = dim3(kT5Block); cfg.dynamicSmemBytes = kT5Smem; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
