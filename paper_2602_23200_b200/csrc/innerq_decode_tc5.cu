@@ -42,7 +42,7 @@ constexpr int kStages = 3;
 constexpr int kOffBq = kStages * kTileBytes;       // B_q: 16 columns x 128 channels fp16, canonical K-major layout
 constexpr int kOffBp = kOffBq + 4096;              // B_p: 16 columns x 128 tokens
 constexpr int kOffMisc = kOffBp + 4096;            // barriers, reductions, tensor-memory base address
-constexpr int kOffScratch = kOffMisc + 512;        // scratch of the fp16 / skew token slice (3 * 128 + 8 floats)
+constexpr int kOffScratch = kOffMisc + 512;        // q'' raw and normalised, result of the fp16 / skew token slice
 constexpr int kT5Smem = kOffScratch + 2048;
 
 // tensor memory (32-bit columns, 128 lanes), two allocations so that three CTAs fit into the SM's 512 columns:
@@ -235,45 +235,29 @@ __device__ __noinline__ void merge_parts4(const float* __restrict__ partials, fl
   out[(size_t)head * kD + c] = __float2half_rn(num / dn);
 }
 
-// block-wide max / sum over the first 128 threads through four shared words (two barriers each; a fifth warp of
-// the CTA joins the barriers with a neutral value)
-__device__ __forceinline__ float block_max(float v, float* red4) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0 && threadIdx.x < kT5Threads) red4[threadIdx.x >> 5] = v;
-  __syncthreads();
-  return fmaxf(fmaxf(red4[0], red4[1]), fmaxf(red4[2], red4[3]));
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ float block_sum(float v, float* red4) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0 && threadIdx.x < kT5Threads) red4[threadIdx.x >> 5] = v;
-  __syncthreads();
-  return (red4[0] + red4[1]) + (red4[2] + red4[3]);
+// warp-wide maximum of floats / sum of non-negative floats <= 1 with one redux instruction each
+__device__ __forceinline__ float warp_max(float v) {
+  int b = __float_as_int(v);
+  b ^= (b >> 31) & 0x7fffffff;                       // order-preserving map to signed integers (an involution)
+  b = __reduce_max_sync(0xffffffffu, b);
+  b ^= (b >> 31) & 0x7fffffff;
+  return __int_as_float(b);
+}
+__device__ __forceinline__ float warp_sum_unit(float v) {      // 24 fractional bits
+  return (float)__reduce_add_sync(0xffffffffu, (unsigned)__float2uint_rn(v * 0x1p24f)) * 0x1p-24f;
 }
 
 // The tokens outside the range where keys and values are both packed (at most a few hundred per unit): the K/V skew
 // zone (packed key rows n_qv .., fp16 values from the value ring), the sink window and the recent window (fp16
-// both), as one list of entries.  Every CTA of a unit takes a slice [e_lo, e_hi) of the list before it starts on
-// its packed tiles, with plain SIMT code: thread = token for the scores, thread = channel for the values.
-// fbuf: 3 * 128 + 8 floats of shared memory.  Results: this thread's channel sum, running max and sum.
-__device__ void tail_slice(const Layout& L, const Counts& cn, const T5Args& a, int u, int e_lo, int e_hi, float* fbuf,
-                           float& acc_out, float& m_out, float& l_out) {
-  const int tid = threadIdx.x;
-  const bool act = tid < kT5Threads;        // the CTA's fifth warp only joins the barriers
-  float* qs = fbuf;            // q'' raw
-  float* qn = fbuf + 128;      // q'' * norm (packed key rows)
-  float* ps = fbuf + 256;      // probabilities of the current round
-  float* red4 = fbuf + 384;
-  const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
-  if (act) {
-    const float v = __half2float(a.q[(size_t)u * kD + tid]) * (L.sm_scale * kLog2e);
-    qs[tid] = v;
-    qn[tid] = L.k_normalize ? v * norm[tid] : v;
-  }
-  __syncthreads();
+// both), as one list of entries.  Every CTA of a unit takes a slice [e_lo, e_hi) of the list; ONE warp works it off
+// with plain SIMT code while the others stream the packed tiles: lane = entry for the scores (32 per round), lane =
+// four channels for the values.  qs / qn: q'' and q'' * norm in shared memory.  res: [128] channel sums, max, sum.
+__device__ void tail_slice_warp(const Layout& L, const Counts& cn, const T5Args& a, int u, int e_lo, int e_hi,
+                                const float* qs, const float* qn, float* res) {
+  const int lane = threadIdx.x & 31;
   const int n_skew = cn.n_qk - cn.n_qv;
   const unsigned char* rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const __half* k_sink = reinterpret_cast<const __half*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
@@ -286,9 +270,9 @@ __device__ void tail_slice(const Layout& L, const Counts& cn, const T5Args& a, i
     if (slot >= L.v.ring_cap) slot -= L.v.ring_cap;
     return v_ring + (size_t)slot * kD;
   };
-  float m_run = -INFINITY, l_run = 0.f, acc = 0.f;
-  for (int e0 = e_lo; e0 < e_hi; e0 += kT5Threads) {
-    const int e = act ? e0 + tid : e_hi;
+  float m_run = -INFINITY, l_run = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int e0 = e_lo; e0 < e_hi; e0 += 32) {
+    const int e = e0 + lane;
     float s = -INFINITY;
     if (e < n_skew && e < e_hi) {                       // packed key row
       const int i = cn.n_qv + e;
@@ -323,6 +307,7 @@ __device__ void tail_slice(const Layout& L, const Counts& cn, const T5Args& a, i
         kr = k_ring + (size_t)slot * kD;
       }
       float d = 0.f;
+#pragma unroll 4
       for (int i = 0; i < 16; ++i) {
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(kr) + i);
         const __half2* h = reinterpret_cast<const __half2*>(&v);
@@ -334,37 +319,31 @@ __device__ void tail_slice(const Layout& L, const Counts& cn, const T5Args& a, i
       }
       s = d;
     }
-    const float m_new = fmaxf(m_run, block_max(s, red4));
+    const float m_new = fmaxf(m_run, warp_max(s));
     const float alpha = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new);
     const float p = e < e_hi ? ex2_approx(s - m_new) : 0.f;
-    if (act) ps[tid] = p;
-    l_run = l_run * alpha + block_sum(p, red4);         // (its barriers also publish ps)
+    float ps = p;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    l_run = l_run * alpha + ps;
     m_run = m_new;
-    acc *= alpha;
-    const int n = min(kT5Threads, e_hi - e0);
-    if (act)
-      for (int ee = 0; ee < n; ++ee) acc = fmaf(ps[ee], __half2float(v_row(e0 + ee)[tid]), acc);
-    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] *= alpha;
+    const int n = min(32, e_hi - e0);
+    for (int ee = 0; ee < n; ++ee) {
+      const float pe = __shfl_sync(0xffffffffu, p, ee);
+      const uint2 v = __ldg(reinterpret_cast<const uint2*>(v_row(e0 + ee)) + lane);
+      const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+      const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+      acc[0] = fmaf(pe, f0.x, acc[0]); acc[1] = fmaf(pe, f0.y, acc[1]);
+      acc[2] = fmaf(pe, f1.x, acc[2]); acc[3] = fmaf(pe, f1.y, acc[3]);
+    }
   }
-  acc_out = acc; m_out = m_run; l_out = l_run;
+  *reinterpret_cast<float4*>(res + 4 * lane) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+  if (lane == 0) { res[kD] = m_run; res[kD + 1] = l_run; }
 }
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// warp-wide maximum of floats / sum of non-negative floats <= 1 with one redux instruction each
-__device__ __forceinline__ float warp_max(float v) {
-  int b = __float_as_int(v);
-  b ^= (b >> 31) & 0x7fffffff;                       // order-preserving map to signed integers (an involution)
-  b = __reduce_max_sync(0xffffffffu, b);
-  b ^= (b >> 31) & 0x7fffffff;
-  return __int_as_float(b);
-}
-__device__ __forceinline__ float warp_sum_unit(float v) {      // 24 fractional bits
-  return (float)__reduce_add_sync(0xffffffffu, (unsigned)__float2uint_rn(v * 0x1p24f)) * 0x1p-24f;
-}
-
-constexpr int kT5Block = kT5Threads + 32;            // four compute warps and the issuing warp
+constexpr int kT5Block = kT5Threads + 64;            // four compute warps, the issuing warp, the warp of the fp16 tokens
 
 // Compute warps 0..3: thread t is token t of the tile on the key side and channel t on the value side.  Warp 4:
 // its lane 0 starts the bulk copies and issues the MMAs.  They talk through mbarriers only (no CTA barrier in the
@@ -422,19 +401,18 @@ __global__ void __launch_bounds__(kT5Block, 3) decode_tc5_kernel(const Layout L,
     // ---------------- q'' and the B_q operand ---------------------------------------------------------------------
     const float* norm = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
     float qv = 0.f;
+    float* qs_s = reinterpret_cast<float*>(smem + kOffScratch);       // q'' raw, q'' * norm, result of the fp16 tokens
+    float* qn_s = qs_s + kD;
+    float* tail_res = qn_s + kD;
     if (compute) {
       qv = __half2float(a.q[(size_t)u * kD + tid]) * (L.sm_scale * kLog2e);
+      qs_s[tid] = qv;
       if (L.k_normalize) qv *= norm[tid];
+      qn_s[tid] = qv;
     }
     __syncthreads();                 // barrier init, zero fill and the tensor-memory address are visible
     if (warp == 4 && lane == 0)
       for (int it = 0; it < kStages && it < n_my; ++it) issue(it);
-    // this CTA's slice of the unit's fp16 / skew tokens, while the first tiles are on their way
-    {
-      const int total = (cn.n_qk - cn.n_qv) + cn.n_sink + cn.n_k_recent;
-      const int e_lo = (int)((long long)split * total / gridDim.y), e_hi = (int)((long long)(split + 1) * total / gridDim.y);
-      tail_slice(L, cn, a, u, e_lo, e_hi, reinterpret_cast<float*>(smem + kOffScratch), out_c, m_run, l_run);
-    }
     float amax = warp_max(fabsf(qv));
     if (compute && lane == 0) red4[warp] = amax;
     __syncthreads();
@@ -457,7 +435,12 @@ __global__ void __launch_bounds__(kT5Block, 3) decode_tc5_kernel(const Layout L,
     tc_fence_after();
     const uint32_t tbase = tmem_slot[0], tbase_d = tmem_slot[1];
 
-    if (!compute) {
+    if (warp == 5) {
+      // ======================= the unit's fp16 / skew tokens: this CTA's slice =====================================
+      const int total = (cn.n_qk - cn.n_qv) + cn.n_sink + cn.n_k_recent;
+      const int e_lo = (int)((long long)split * total / gridDim.y), e_hi = (int)((long long)(split + 1) * total / gridDim.y);
+      tail_slice_warp(L, cn, a, u, e_lo, e_hi, qs_s, qn_s, tail_res);
+    } else if (!compute) {
       // ======================= issuing warp ======================================================================
       if (lane == 0) {
         auto issue_mma = [&](int col_d, int col_a, int off_b, uint32_t bar) {
@@ -616,6 +599,13 @@ __global__ void __launch_bounds__(kT5Block, 3) decode_tc5_kernel(const Layout L,
     if (failed) {
       if (tid == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);
       m_run = -INFINITY; l_run = 0.f; out_c = 0.f;
+    } else if (compute) {          // add the slice of fp16 tokens (its results were published by the barrier above)
+      const float mt = tail_res[kD], lt = tail_res[kD + 1];
+      const float m_new = fmaxf(m_run, mt);
+      const float wa = m_run == -INFINITY ? 0.f : ex2_approx(m_run - m_new), wb = mt == -INFINITY ? 0.f : ex2_approx(mt - m_new);
+      out_c = out_c * wa + tail_res[tid] * wb;
+      l_run = l_run * wa + lt * wb;
+      m_run = m_new;
     }
   }
 
