@@ -97,6 +97,24 @@ def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
     return float(dense), float(minimal)
 
 
+def issue_roof_gbs(w, sm_mhz):
+    """Second roof of the packed decode kernel: instruction issue on the ALU and tensor pipes.
+
+    Per cached code the kernel spends one ALU-pipe instruction per code pair and plane (`word & mask` builds the fp16
+    operand pair) plus about 45 % other ALU-pipe work (measured mix), each occupying a 16-lane pipe for 2 cycles per
+    warp, and one warp-level MMA (m16n8k16: 256 codes, about 8 cycles of the tensor pipe) per plane; on this GPU the two
+    pipes were measured not to overlap, so their cycles add.  148 SMs x 4 sub-partitions at the sampled SM clock."""
+    if w.grouping != synth.INNER:
+        return None
+    def cycles_per_code(bits):
+        planes = 2 if bits == 3 else 1
+        return planes * (0.5 * 1.45 * 2.0 / 32.0 + 8.0 / 256.0)
+    k_bytes, v_bytes = payload_bytes(w)                       # per token: 128 codes each
+    cyc = 128 * (cycles_per_code(w.k_bits) + cycles_per_code(w.v_bits))
+    tokens_per_s = 148 * 4 * (sm_mhz or 1965.0) * 1e6 / cyc
+    return tokens_per_s * (k_bytes + v_bytes) / 1e9
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clocks and clock-event (throttle) reasons through NVML while the timed region runs.
 
@@ -418,6 +436,8 @@ def run_ours(args, w):
             "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
+            "second_roof": {"kind": "ALU-pipe + tensor-pipe issue of the packed decode kernel (model, see issue_roof_gbs)",
+                            "gbs": issue_roof_gbs(w, clocks.get("sm_mhz"))},
             "step_us_by_kind": step_split,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
