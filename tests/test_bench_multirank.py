@@ -37,3 +37,27 @@ def test_single_process_passthrough():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.whole_job_gbs(2e9, 1e-3, 1) == 2000.0
+
+
+def test_algorithmic_bytes_follow_the_library_payload():
+    # the roofline numerator: bytes per quantised token as bench.py counts them = what the C ABI says the packed
+    # cache holds per token, for every mode (zero-points stored or not) and both groupings
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_23200_b200 import binding as B, synth
+    for kw in (dict(), dict(k_bits=3, v_bits=2, k_mode=synth.SYM, v_mode=synth.HYBRID), dict(group=128, k_bits=4, v_bits=4),
+               dict(k_mode=synth.SYM, v_mode=synth.SYM, group=64),
+               dict(grouping=synth.OUTER, k_normalize=0, k_mode=synth.ASYM, v_mode=synth.ASYM, group=64)):
+        w = synth.tiny(**kw)
+        kb, vb = B.innerq_token_payload_bytes(B.make_config(w))
+        assert bench.payload_bytes(w) == (kb, vb), kw
+    # and the whole-call count on a case small enough to add up by hand: everything in windows -> fp16 rows only
+    w = synth.tiny(n_tokens=12, w_sink=4, w_recent=16)
+    dense, minimal = bench.decode_algorithmic_bytes(w, 12)
+    rows = w.n_units * 12 * 2 * 256
+    extras = w.batch * w.n_q_heads * 128 * 2 * 2 + w.n_units * 128 * 4
+    assert dense == minimal == rows + extras
+    # the issue roof exists for the inner-grouped formats only and scales with the bytes per token
+    assert bench.issue_roof_gbs(synth.tiny(grouping=synth.FP16, k_normalize=0), 1965.0) is None
+    r2, r4 = bench.issue_roof_gbs(synth.tiny(), 1965.0), bench.issue_roof_gbs(synth.tiny(k_bits=4, v_bits=4), 1965.0)
+    assert r4 > r2 > 0
