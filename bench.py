@@ -97,22 +97,30 @@ def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
     return float(dense), float(minimal)
 
 
-def issue_roof_gbs(w, sm_mhz):
-    """Second roof of the packed decode kernel: instruction issue on the ALU and tensor pipes.
-
-    Per cached code the kernel spends one ALU-pipe instruction per code pair and plane (`word & mask` builds the fp16
-    operand pair) plus about 45 % other ALU-pipe work (measured mix), each occupying a 16-lane pipe for 2 cycles per
-    warp, and one warp-level MMA (m16n8k16: 256 codes, about 8 cycles of the tensor pipe) per plane; on this GPU the two
-    pipes were measured not to overlap, so their cycles add.  148 SMs x 4 sub-partitions at the sampled SM clock."""
-    if w.grouping != synth.INNER:
+def stored_counters(workload: str):
+    """Counters of one decode launch of `workload` from the committed ncu summary (profiles/decode_counters.json)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "decode_counters.json")) as f:
+            return json.load(f).get(workload)
+    except Exception:
         return None
-    def cycles_per_code(bits):
-        planes = 2 if bits == 3 else 1
-        return planes * (0.5 * 1.45 * 2.0 / 32.0 + 8.0 / 256.0)
-    k_bytes, v_bytes = payload_bytes(w)                       # per token: 128 codes each
-    cyc = 128 * (cycles_per_code(w.k_bits) + cycles_per_code(w.v_bits))
-    tokens_per_s = 148 * 4 * (sm_mhz or 1965.0) * 1e6 / cyc
-    return tokens_per_s * (k_bytes + v_bytes) / 1e9
+
+
+def pipe_roofs_gbs(counters, bytes_per_decode, sm_mhz):
+    """Second roofs of the packed decode kernel from its measured instruction counts.
+
+    A sub-partition issues at most one warp instruction per cycle, its 16-lane ALU pipe takes one warp instruction
+    per 2 cycles and its tensor pipe one m16n8k16 MMA per 8 cycles (measured with a stand-alone loop on this GPU).
+    The time each of the three needs for the launch's instructions, spread evenly over 148 SMs x 4 sub-partitions at
+    the sampled SM clock, turns the launch's algorithmic bytes into a roof in GB/s; the lowest is returned first."""
+    if not counters:
+        return None
+    per_s = 148 * 4 * (sm_mhz or 1965.0) * 1e6
+    t = {"issue": counters["warp_instructions"] / per_s, "alu_pipe": 2.0 * counters["alu_pipe"] / per_s,
+         "tensor_pipe": 8.0 * counters["tensor_pipe"] / per_s}
+    roofs = {k: bytes_per_decode / v / 1e9 for k, v in t.items()}
+    low = min(roofs, key=roofs.get)
+    return {"lowest": low, "gbs": roofs[low], "all_gbs": roofs}
 
 
 class ClockSampler(threading.Thread):
@@ -169,12 +177,9 @@ def measured_peak_gbs():
 
 
 def stored_traffic(workload: str):
-    """DRAM bytes per decode launch from the committed ncu summary, if any."""
-    try:
-        with open(os.path.join(ROOT, "profiles", "decode_traffic.json")) as f:
-            return json.load(f).get(workload)
-    except Exception:
-        return None
+    """DRAM bytes (read + written) per decode launch from the committed ncu summary, if any."""
+    c = stored_counters(workload)
+    return c["dram_read_bytes"] + c["dram_write_bytes"] if c else None
 
 
 # ------------------------------------------------------------------------------------- oracle legs
@@ -436,8 +441,7 @@ def run_ours(args, w):
             "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
-            "second_roof": {"kind": "ALU-pipe + tensor-pipe issue of the packed decode kernel (model, see issue_roof_gbs)",
-                            "gbs": issue_roof_gbs(w, clocks.get("sm_mhz"))},
+            "second_roof": pipe_roofs_gbs(stored_counters(w.name), bytes_min / Kst, clocks.get("sm_mhz")),
             "step_us_by_kind": step_split,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -3,6 +3,8 @@ The path has no data-path collective (units are independent); ranks only agree o
 import os
 import sys
 
+import pytest
+
 import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -57,7 +59,16 @@ def test_algorithmic_bytes_follow_the_library_payload():
     rows = w.n_units * 12 * 2 * 256
     extras = w.batch * w.n_q_heads * 128 * 2 * 2 + w.n_units * 128 * 4
     assert dense == minimal == rows + extras
-    # the issue roof exists for the inner-grouped formats only and scales with the bytes per token
-    assert bench.issue_roof_gbs(synth.tiny(grouping=synth.FP16, k_normalize=0), 1965.0) is None
-    r2, r4 = bench.issue_roof_gbs(synth.tiny(), 1965.0), bench.issue_roof_gbs(synth.tiny(k_bits=4, v_bits=4), 1965.0)
-    assert r4 > r2 > 0
+    # second roofs from the stored instruction counts: one sub-partition issues 1 instruction, 1/2 ALU-pipe instruction
+    # and 1/8 MMA per cycle; the lowest of the three is reported
+    assert bench.pipe_roofs_gbs(None, 1e6, 1965.0) is None
+    c = {"warp_instructions": 592 * 1965, "alu_pipe": 592 * 1965, "tensor_pipe": 592 * 100}
+    r = bench.pipe_roofs_gbs(c, 1e6, 1965.0)      # 1 us of issue, 2 us of ALU pipe, 0.41 us of tensor pipe
+    assert r["lowest"] == "alu_pipe" and r["gbs"] == pytest.approx(500.0)
+    assert r["all_gbs"]["issue"] == pytest.approx(1000.0)
+    # every bench workload with a packed cache has its counters and DRAM traffic on file
+    for name in ("c1", "c2", "c3_4bit", "c3_2bit", "c4"):
+        w = bench.workload_by_name(name)
+        c = bench.stored_counters(w.name)
+        assert c is not None and c["alu_pipe"] < c["warp_instructions"], name
+        assert bench.stored_traffic(w.name) == c["dram_read_bytes"] + c["dram_write_bytes"]
