@@ -305,13 +305,17 @@ class OracleCache:
         Vt = np.concatenate([self.v.sink[u].astype(f64), self.v.dequant(u), self.v.recent[u].astype(f64)], axis=0)
         return Kt, Vt
 
-    def decode(self, q, units=None, return_probs=False):
+    def decode(self, q, units=None, return_probs=False, n_hidden=0):
         """q fp16 [B, Hq, D] -> float64 [B, Hq, D].  Query head j reads KV head j // (Hq/Hkv).
 
         Scores: raw q against the fp16 windows, q' = q * norm against the dequantised
         (normalised) key rows; softmax over all N tokens; values from V's own partition.
         `units` restricts the work to some (batch, KV head) units (other rows stay NaN).
+        `n_hidden` > 0 leaves the newest n_hidden tokens of the cache out (causal mask of a query that is
+        n_hidden positions before the newest token; not in the paper, which decodes one token at a time).
         """
+        n_vis = self.N - int(n_hidden)
+        assert 0 < n_vis <= self.N
         q = np.asarray(q).reshape(self.B, self.Hq, self.D).astype(f64)
         r = self.Hq // self.Hkv
         out = np.full((self.B, self.Hq, self.D), np.nan, dtype=f64)
@@ -321,7 +325,7 @@ class OracleCache:
             if self.grouping == FP16:
                 Kt, Vt = self.materialize(u)
                 for j in range(h * r, (h + 1) * r):
-                    out[b, j] = dense_attention(q[b, j], Kt, Vt, self.sm_scale)
+                    out[b, j] = dense_attention(q[b, j], Kt[:n_vis], Vt[:n_vis], self.sm_scale)
                 continue
             k_sink, k_rec = self.k.sink[u].astype(f64), self.k.recent[u].astype(f64)
             k_hat = self.k.dequant(u)
@@ -330,14 +334,26 @@ class OracleCache:
             for j in range(h * r, (h + 1) * r):
                 qj = q[b, j]
                 qn = qj * norm if self.k_normalize else qj
-                d = np.concatenate([k_sink @ qj, k_hat @ qn, k_rec @ qj])
+                d = np.concatenate([k_sink @ qj, k_hat @ qn, k_rec @ qj])[:n_vis]      # tokens oldest first
                 s = d * self.sm_scale
                 p = np.exp(s - s.max())
                 p = p / p.sum()
-                out[b, j] = p @ Vt
+                out[b, j] = p @ Vt[:n_vis]
                 if return_probs:
                     probs[(b, j)] = p
         return (out, probs) if return_probs else out
+
+    def decode_multi(self, q, units=None):
+        """q fp16 [B, n_q, Hq, D] -> float64 [B, n_q, Hq, D]: n_q consecutive query tokens whose own keys and
+        values are the newest n_q tokens of the cache; query i attends causally to tokens 0 .. N - n_q + i.
+        (Verification step of speculative decoding; the paper itself decodes one token per step, Section
+        "Preliminaries", so this is that definition applied n_q times to one cache state.)"""
+        q = np.asarray(q)
+        n_q = q.shape[1]
+        out = np.empty((self.B, n_q, self.Hq, self.D), dtype=f64)
+        for i in range(n_q):
+            out[:, i] = self.decode(q[:, i], units=units, n_hidden=n_q - 1 - i)
+        return out
 
     def export(self):
         """Canonical (unpacked) cache contents, tokens oldest first."""

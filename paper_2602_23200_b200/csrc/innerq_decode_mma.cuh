@@ -112,6 +112,13 @@ __device__ __forceinline__ uint32_t split_hi_lo(float x) {
   const __half lo = __float2half_rn(x - __half2float(hi));
   return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
 }
+// fp16(lo) in the low half-word, fp16(hi) in the high one, with one packing conversion (not the conversion unit's
+// single-value cvt, which costs a sub-partition 8 cycles per warp instruction)
+__device__ __forceinline__ uint32_t pack_half2_rn(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 __device__ __forceinline__ float pow2i(int e) { return __int_as_float((e + 127) << 23); }   // 2^e, -126 <= e <= 127
 
 // Per bit-width constants of the packed formats (see innerq_layout.h).
@@ -640,10 +647,9 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
       for (int st_ = 0; st_ < NSET; ++st_) {
         if constexpr (NG == 4)
-          pk[st_] = (uint32_t)__half_as_ushort(__float2half_rn(ps[2 * st_])) |
-                    ((uint32_t)__half_as_ushort(__float2half_rn(ps[2 * st_ + 1])) << 16);
+          pk[st_] = pack_half2_rn(ps[2 * st_], ps[2 * st_ + 1]);
         else
-          pk[st_] = (uint32_t)__half_as_ushort(__float2half_rn(ps[NG == 2 ? st_ : 0]));
+          pk[st_] = pack_half2_rn(ps[NG == 2 ? st_ : 0], 0.f);
       }
     };
 
@@ -877,7 +883,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
             }
             // p goes in as one fp16 (the lo column stays zero): its 2^-12 relative rounding is random per token and
             // far inside the output tolerance, and it saves the hi/lo split of every probability
-            uint32_t pk = (uint32_t)__half_as_ushort(__float2half_rn(p * pow2i(10 - VP * pos)));
+            uint32_t pk = pack_half2_rn(p * pow2i(10 - VP * pos), 0.f);
             if (SPLIT && j != slot) pk = 0u;                 // column pair of this chunk's window slot only
             Bp[mt][h] = movmatrix_trans(pk);
           }

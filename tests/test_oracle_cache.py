@@ -272,3 +272,39 @@ def test_quantised_keys_use_the_normalised_domain():
     s_norm = (r["scale_bits"] & 0x7FFF).view(np.float16).astype(np.float64).mean()
     s_raw = (raw["scale_bits"] & 0x7FFF).view(np.float16).astype(np.float64).mean()
     assert s_norm < 0.5 * s_raw
+
+
+@pytest.mark.parametrize("grouping", [O.INNER, O.OUTER, O.FP16])
+@pytest.mark.parametrize("n_q", [1, 2, 5])
+def test_multi_query_decode_is_causal_attention(grouping, n_q):
+    # n_q query tokens whose own keys / values are the newest n_q cache tokens: query i sees tokens 0 .. N-n_q+i.
+    # Pinned to the library's attention with an explicit boolean mask (a) on the raw fp16 tensors when every
+    # token is in a window and (b) on the materialised K~, V~ (themselves pinned element by element above)
+    # when most tokens are quantised.
+    for N, windows_only in ((9, True), (150, False)):
+        w = synth.tiny(n_tokens=N, grouping=grouping, k_normalize=int(grouping == O.INNER), w_sink=4,
+                       w_recent=8 if windows_only else 12)
+        K, V = synth.kv_all(w)
+        q = np.stack([synth.query(w, step) for step in range(n_q)], axis=1)          # [B, n_q, Hq, D]
+        c = O.from_workload(w)
+        c.prefill(K, V)
+        out = c.decode_multi(q)
+        assert out.shape == (w.batch, n_q, w.n_q_heads, w.head_dim)
+        r = w.q_per_kv
+        mask = torch.ones(n_q, N, dtype=torch.bool)
+        for i in range(n_q):
+            mask[i, N - n_q + i + 1:] = False
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                if windows_only:
+                    Km, Vm = K[b, h].astype(np.float64), V[b, h].astype(np.float64)
+                else:
+                    Km, Vm = c.materialize(b * w.n_kv_heads + h)
+                for j in range(h * r, (h + 1) * r):
+                    qt = torch.from_numpy(q[b, :, j].astype(np.float64))[None, None]        # [1, 1, n_q, D]
+                    ref = torch.nn.functional.scaled_dot_product_attention(
+                        qt, torch.from_numpy(Km)[None, None], torch.from_numpy(Vm)[None, None], attn_mask=mask,
+                        scale=1 / math.sqrt(w.head_dim))[0, 0].numpy()
+                    assert np.allclose(out[b, :, j], ref, rtol=1e-11, atol=1e-12)
+        # the newest query sees everything: the same as the single-token decode
+        assert np.array_equal(out[:, n_q - 1], c.decode(q[:, n_q - 1]))
