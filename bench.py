@@ -401,6 +401,24 @@ def run_ours(args, w):
     b1.record(stream)
     torch.cuda.synchronize()
     b2b_us = b0.elapsed_time(b1) / nb * 1e3
+    # several query tokens per sequence in one call (causal among the newest n_q tokens), back to back like the above
+    multi = None
+    if args.n_q > 1 and w.grouping != synth.FP16:
+        qm = torch.stack([q_all[i % len(qs)] for i in range(args.n_q)], dim=1).contiguous()     # [B, n_q, Hq, D]
+        om = torch.empty_like(qm)
+        for i in range(R):
+            caches[i].innerq_decode_attention_multi(qm, om)
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        m0.record(stream)
+        for i in range(nb):
+            caches[i % R].innerq_decode_attention_multi(qm, om)
+        m1.record(stream)
+        torch.cuda.synchronize()
+        multi_us = m0.elapsed_time(m1) / nb * 1e3
+        multi = {"n_q": args.n_q, "us_per_call_back_to_back": multi_us, "us_per_query_token": multi_us / args.n_q,
+                 "launches_per_call": caches[0].innerq_last_launch_count(2),
+                 "single_query_us_back_to_back": b2b_us}
     # steps timed one by one (events around append + decode): those on which a value group (inner grouping) or a key
     # group (outer grouping) of G tokens is quantised, against the others
     step_split = None
@@ -442,7 +460,7 @@ def run_ours(args, w):
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
             "second_roof": pipe_roofs_gbs(stored_counters(w.name), bytes_min / Kst, clocks.get("sm_mhz")),
-            "step_us_by_kind": step_split,
+            "step_us_by_kind": step_split, "multi_query": multi,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
@@ -478,6 +496,7 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--n-q", type=int, default=4, help="query tokens per call of the multi-query leg (0/1: skip it)")
     args = ap.parse_args()
     w = workload_by_name(args.workload)
     if args.impl == "reference":

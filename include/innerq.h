@@ -154,6 +154,26 @@ int innerq_decode_step_host(innerq_cache_t* cache, const void* k_new_host, const
 /* Bytes of device staging innerq_decode_step_host needs for this configuration.  Errors: INVALID_ARG. */
 int innerq_step_staging_bytes(const innerq_config_t* cfg, size_t* bytes);
 
+/* Decode attention for n_q consecutive query tokens per sequence in one call (the verification step of
+ * speculative decoding, or a short chunked prefill).  The paper decodes one token per step (Section
+ * "Preliminaries"); this is that definition applied to n_q queries against one cache state, with a causal mask:
+ * the cache already holds the n_q tokens' own keys and values as its newest tokens (append them first), and
+ * query token i (0 <= i < n_q) attends to tokens 0 .. N - n_q + i.
+ *   q, out        : device, fp16 [batch, n_q, n_q_heads, head_dim]; n_q = 1 is innerq_decode_attention.
+ *   dev_scratch   : device, 256-byte aligned, at least innerq_multi_query_scratch_bytes(cfg) bytes; owned by the
+ *                   caller, used only during the call (split partials of up to four query rows per KV head).
+ * The rows of a KV head (its n_q * r query heads) are processed four per pass over the packed cache: with one
+ * query head per KV head four query tokens share one pass, with four or more each token takes its own.
+ * Limits: the fused kernel only (packed inner- or outer-grouped cache in a format it supports; decode variant
+ * 0 or 2); the n_q - 1 newest tokens must all lie outside the token range in which keys AND values are packed
+ * (always true for n_q - 1 <= w_recent once the windows are full).  Otherwise UNSUPPORTED, nothing launched.
+ * Errors: INVALID_ARG (n_q < 1 or n_q > N included), BUFFER_TOO_SMALL, UNSUPPORTED, CUDA. */
+int innerq_decode_attention_multi(innerq_cache_t* cache, const void* q, void* out, int32_t n_q, void* dev_scratch,
+                                  size_t scratch_bytes, void* cuda_stream);
+
+/* Bytes of device scratch innerq_decode_attention_multi needs (independent of n_q).  Errors: INVALID_ARG. */
+int innerq_multi_query_scratch_bytes(const innerq_config_t* cfg, size_t* bytes);
+
 /* Same computation and arguments as innerq_decode_attention, for callers that cannot give the decode
  * step any scratch memory of their own.  (The paper has no counterpart; this is an integration aid.)
  * Typical cases: the workspace passed to innerq_cache_create was only lent for the prefill and has gone

@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = (
     "innerq_cache_bytes", "innerq_token_payload_bytes", "innerq_cache_create", "innerq_cache_destroy",
     "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
     "innerq_decode_attention_static", "innerq_decode_step_host", "innerq_step_staging_bytes",
+    "innerq_decode_attention_multi", "innerq_multi_query_scratch_bytes",
     "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
@@ -72,6 +73,8 @@ def lib() -> C.CDLL:
     L.innerq_decode_attention_static.argtypes = [vp, vp, vp, vp]
     L.innerq_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.innerq_step_staging_bytes.argtypes = [cfgp, C.POINTER(sz)]
+    L.innerq_decode_attention_multi.argtypes = [vp, vp, vp, i32, vp, sz, vp]
+    L.innerq_multi_query_scratch_bytes.argtypes = [cfgp, C.POINTER(sz)]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
@@ -210,6 +213,26 @@ class InnerQCache:
             out = torch.empty(shape, dtype=torch.float16, device=self.device)
         _check(lib().innerq_decode_attention_static(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
                                                     _stream_ptr(stream)), "innerq_decode_attention_static")
+        return out
+
+    def innerq_decode_attention_multi(self, q, out=None, stream=None):
+        """q fp16 [batch, n_q, n_q_heads, head_dim] (the n_q newest cache tokens are the queries' own) -> out of the
+        same shape, causal.  The device scratch the C call needs is a torch allocation made here on first use."""
+        import torch
+        c = self.cfg
+        if not (isinstance(q, torch.Tensor) and q.dim() == 4):
+            raise TypeError("q must be a [batch, n_q, n_q_heads, head_dim] tensor")
+        n_q = int(q.shape[1])
+        shape = (c.batch, n_q, c.n_q_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=torch.float16, device=self.device)
+        if getattr(self, "_multi_scratch", None) is None:
+            n = C.c_size_t()
+            _check(lib().innerq_multi_query_scratch_bytes(C.byref(c), C.byref(n)), "innerq_multi_query_scratch_bytes")
+            self._multi_scratch = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+        _check(lib().innerq_decode_attention_multi(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape), n_q,
+                                                   self._multi_scratch.data_ptr(), self._multi_scratch.numel(),
+                                                   _stream_ptr(stream)), "innerq_decode_attention_multi")
         return out
 
     def innerq_decode_step_host(self, k_new_host, v_new_host, q_host, out_host, stream=None):

@@ -280,6 +280,38 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   return INNERQ_OK;
 }
 
+// ---- several query tokens per sequence ----------------------------------------------------------------
+int innerq_multi_query_scratch_bytes(const innerq_config_t* cfg, size_t* bytes) {
+  if (!bytes) return INNERQ_ERR_INVALID_ARG;
+  const int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  Layout L;
+  make_layout(*cfg, L);
+  *bytes = align_up((size_t)L.U * 4 * L.max_splits * kPartialStride * 4, 256);
+  return INNERQ_OK;
+}
+
+int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, int32_t n_q, void* dev_scratch,
+                                  size_t scratch_bytes, void* cuda_stream) {
+  if (!c || !q || !out || !dev_scratch || n_q < 1 || n_q > c->N) return INNERQ_ERR_INVALID_ARG;
+  if ((uintptr_t)dev_scratch & 255u) return INNERQ_ERR_INVALID_ARG;
+  if (scratch_bytes < align_up((size_t)c->L.U * 4 * c->L.max_splits * kPartialStride * 4, 256)) return INNERQ_ERR_BUFFER_TOO_SMALL;
+  if ((c->opt_variant != 0 && c->opt_variant != 2) || c->L.k.kind == kNone || !decode_mma_supported(c->L))
+    return INNERQ_ERR_UNSUPPORTED;
+  // the hidden tokens (positions N - n_q + 1 .. N - 1) must be sink, skew-zone or recent tokens: those are
+  // scored in tiles that can mask by position; the chunks where keys and values are both packed cannot
+  const Counts cn = counts_for(c->L, c->N);
+  const int n_packed = cn.n_qk < cn.n_qv ? cn.n_qk : cn.n_qv;
+  if (n_packed > 0 && c->N - n_q + 1 < cn.n_sink + n_packed) return INNERQ_ERR_UNSUPPORTED;
+  const int n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
+                                  c->opt_splits, static_cast<cudaStream_t>(cuda_stream), n_q,
+                                  static_cast<float*>(dev_scratch));
+  if (n == -2) return INNERQ_ERR_UNSUPPORTED;
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->launches[2] = n;
+  return INNERQ_OK;
+}
+
 // ---- one step from host buffers ----------------------------------------------------------------------
 static size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 

@@ -42,8 +42,10 @@ bool decode_mma_supported(const Layout& L) { return format_launcher(L) != nullpt
 
 void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
 
+// n_q > 1: q and out are [B, n_q, Hq, D], the partials of a launch's (up to) four rows per unit go to
+// multi_partials [U * 4][max_splits][kPartialStride]
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st) {
+                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials) {
   const FormatLauncher launch = format_launcher(L);
   if (!launch) return -2;
   const Counts cn = counts_for(L, N);
@@ -66,6 +68,9 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.k_ring_pos0 = L.k.ring_cap ? cn.n_qk % L.k.ring_cap : 0;
   a.v_ring_pos0 = L.v.ring_cap ? cn.n_qv % L.v.ring_cap : 0;
   a.head0 = 0;
+  a.n_q = n_q;
+  a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
+  if (n_q < 1 || (n_q > 1 && !multi_partials)) return -1;
   return launch(L, cn, a, n_splits, g_chunks_per_iter, st);
 }
 

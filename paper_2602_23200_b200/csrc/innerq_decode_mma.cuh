@@ -165,10 +165,10 @@ template <int KB, int VB, int G, int KM, int VM, int CPI> struct StageLayout {
 
 
 // Cross-CTA merge, run by the last CTA of a unit to finish: log-sum-exp combination of the n_parts partial results
-// (rows of kPartialStride floats: acc[128], max, sum) of nh query heads starting at head_base, fp16 result to out.
+// (rows prow0 .. of kPartialStride floats: acc[128], max, sum) of nh query rows, fp16 results to rows orow of out.
 // Kept out of line so that its registers do not add to the streaming loop's.
 __device__ __noinline__ void merge_parts(const float* __restrict__ partials, float* wm, __half* __restrict__ out, int nh,
-                                         int n_parts, int head_base, int max_splits) {
+                                         int n_parts, int prow0, int4 orow, int max_splits) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // Warp w merges parts w, w + 8, ... (four parts per round of loads, lane l the channels 4l .. 4l+3, running
   // max / rescale as in the streaming loop), then the eight warp results are combined through shared memory.
@@ -177,7 +177,7 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 #pragma unroll 1
   for (int h = 0; h < nh; ++h) {
     float M = -INFINITY, den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
-    const float* Ph = partials + (size_t)(head_base + h) * max_splits * kPartialStride;
+    const float* Ph = partials + (size_t)(prow0 + h) * max_splits * kPartialStride;
 #pragma unroll 1
     for (int s0 = warp; s0 < n_parts; s0 += 4 * kWarps) {
       float4 v[4];
@@ -222,7 +222,8 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
       num = fmaf(r_[c], wgt, num);
       den = fmaf(r_[kD + 1], wgt, den);
     }
-    out[(size_t)(head_base + h) * kD + c] = __float2half_rn(num / den);
+    const int row = h == 0 ? orow.x : h == 1 ? orow.y : h == 2 ? orow.z : orow.w;
+    out[(size_t)row * kD + c] = __float2half_rn(num / den);
   }
 }
 
@@ -272,8 +273,14 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   const int gid = lane >> 2, j = lane & 3;
   const int u = blockIdx.x, split = blockIdx.y;
   const int b = u / L.Hkv, hkv = u % L.Hkv;
-  const int nh = min(SPLIT ? 1 : kHeads, L.r - a.head0);
-  const int head_base = b * L.Hq + hkv * L.r + a.head0;     // global index of this pass's first query head
+  const int nh = min(SPLIT ? 1 : kHeads, L.r * a.n_q - a.head0);
+  // Row of q / out of column h of this launch: head h' = (head0 + h) % r of query token i = (head0 + h) / r
+  // (q, out: [B, n_q, Hq, D]; n_q = 1: the pass's heads are consecutive rows), and the row of its split partials.
+  auto q_row = [&](int h) {
+    const int v = a.head0 + h, i = a.n_q > 1 ? v / L.r : 0;
+    return (b * a.n_q + i) * L.Hq + hkv * L.r + (v - i * L.r);
+  };
+  const int prow0 = a.n_q > 1 ? u * kHeads : q_row(0);
   const int n_parts = gridDim.y;
   const bool fast = split < a.n_splits;
   // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
@@ -369,7 +376,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
-      q_early[e] = h < nh ? __half2float(a.q[(size_t)(head_base + h) * kD + c]) : 0.f;
+      q_early[e] = h < nh ? __half2float(a.q[(size_t)q_row(h) * kD + c]) : 0.f;
       n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
     }
   }
@@ -467,6 +474,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     }
     // ---- as owner of C-fragment columns 2j, 2j+1: head j, or in SPLIT (head 0, key group j)
     const int my_head = SPLIT ? 0 : j;
+    // first absolute token position this lane's query row must not see (all tokens for the newest query)
+    const int pos_end = cn.n_sink + cn.n_qk + cn.n_k_recent - (a.n_q - 1 - (a.head0 + my_head) / L.r);
     const int e_c = qe_s[my_head];
     const float kfac = pow2i(24 - (QE - e_c));       // undoes the 2^-24 of the subnormal codes and bscale
     const float inv_kfac = pow2i(-(24 - (QE - e_c)));
@@ -692,12 +701,22 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       }
       if (gid >= cnt) sA = -INFINITY;
       if (gid + 8 >= cnt) sB = -INFINITY;
+      if (a.n_q > 1) {
+        // causal mask of this lane's query row: entries at absolute positions >= pos_end are newer than its token
+        auto pos = [&](int e) {
+          return skew ? cn.n_sink + min(cn.n_qk, cn.n_qv) + e
+                      : (e < cn.n_sink ? e : max(cn.n_qk, cn.n_qv) + e);      // n_sink + n_packed + (e - n_sink)
+        };
+        if (pos(e0 + gid) >= pos_end) sA = -INFINITY;
+        if (pos(e0 + gid + 8) >= pos_end) sB = -INFINITY;
+      }
       float cmax = fmaxf(sA, sB);
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
       cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
       const float m_new = fmaxf(m_run, cmax);
-      const float alpha = ex2_approx(m_run - m_new);            // 0 while m_run = -inf
+      // 0 while m_run = -inf; a tile that is masked completely for this row leaves the state as it is
+      const float alpha = m_new == -INFINITY ? 1.f : ex2_approx(m_run - m_new);
       m_run = m_new;
       l_part *= alpha;
 #pragma unroll
@@ -710,7 +729,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) accg[m][e] *= alpha;
       }
-      const float pA = ex2_approx(sA - m_new), pB = ex2_approx(sB - m_new);
+      const float pA = sA == -INFINITY ? 0.f : ex2_approx(sA - m_new), pB = sB == -INFINITY ? 0.f : ex2_approx(sB - m_new);
       l_part += pA + pB;
       if (OUTER && skew) {
         // values of the skew zone are packed (half a chunk: one k-step of 16 tokens), read straight from global memory
@@ -1067,7 +1086,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
       }
     }
     __syncthreads();
-    float* partials = reinterpret_cast<float*>(a.ws + L.ws_partial_off);
+    float* partials = a.partials;
     for (int i = tid; i < nh * kD; i += kThreads) {
       const int h = i >> 7, c = i & (kD - 1);
       float M = -INFINITY;
@@ -1081,7 +1100,7 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
         num = fmaf(r_[c], wgt, num);
         den = fmaf(r_[kD + 1], wgt, den);
       }
-      float* P = partials + ((size_t)(head_base + h) * L.max_splits + split) * kPartialStride;
+      float* P = partials + ((size_t)(prow0 + h) * L.max_splits + split) * kPartialStride;
       P[c] = num;
       if (c == 0) { P[kD] = M; P[kD + 1] = den; }
     }
@@ -1097,8 +1116,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   __syncthreads();
   if (s_ticket != gridDim.y - 1) return;
   __threadfence();
-  merge_parts(reinterpret_cast<const float*>(a.ws + L.ws_partial_off), reinterpret_cast<float*>(smem), a.out, nh, n_parts,
-              head_base, L.max_splits);
+  merge_parts(a.partials, reinterpret_cast<float*>(smem), a.out, nh, n_parts, prow0,
+              make_int4(q_row(0), q_row(1), q_row(2), q_row(3)), L.max_splits);
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
 }
 
@@ -1134,7 +1153,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   dim3 grid(L.U, grid_y);
   int launches = 0;
   const int step = SPLIT ? 1 : kHeads;
-  for (int h0 = 0; h0 < L.r; h0 += step) {
+  for (int h0 = 0; h0 < L.r * a.n_q; h0 += step) {
     a.head0 = h0;
     // launched as a programmatic dependent of whatever precedes it in the stream: its set-up overlaps that
     // kernel's tail, its first global access waits for it (grid_dependency_wait)
@@ -1163,7 +1182,7 @@ int launch_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_spl
 
 template <int KB, int VB, int KM, int VM>
 int launch_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1) return launch_cpi<KB, VB, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_cpi<KB, VB, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
   if (L.G == 32) return launch_cpi<KB, VB, 32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
   if (L.G == 64) return launch_cpi<KB, VB, 64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
   if (L.G == 128) return launch_cpi<KB, VB, 128, KM, VM, false>(L, cn, a, n_splits, cpi, st);

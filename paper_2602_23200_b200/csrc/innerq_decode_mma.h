@@ -22,7 +22,12 @@ struct DecodeArgs {
   int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
   int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
   int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
-  int head0;             // first query head (within the KV head's r) handled by this launch
+  int head0;             // first query row (within the KV head's r * n_q) handled by this launch
+  int n_q;               // consecutive query tokens per sequence (1: plain decode).  Row v = i * r + h of a KV head is
+                         // head h of query token i; q / out are [B, n_q, Hq, D]; query i does not see the newest
+                         // n_q - 1 - i tokens (all of them outside the chunks where keys AND values are packed)
+  float* partials;       // split partials [rows][max_splits][kPartialStride]: row = global query head (n_q == 1) or
+                         // unit * 4 + column of the launch (n_q > 1)
 };
 
 // Launchers by format: k<key bits>v<value bits>_m<bytes per key metadata entry><bytes per value metadata entry>.

@@ -31,7 +31,7 @@ int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned cha
 
 // Warp-MMA decode for the INNER layout.  Returns -2 if the configuration is not supported.
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st);
+                      __half* out, int n_splits, cudaStream_t st, int n_q = 1, float* multi_partials = nullptr);
 bool decode_mma_supported(const Layout& L);
 
 // Warp-MMA decode over an unquantised fp16 cache (grouping = FP16).  Returns -2 for other layouts.

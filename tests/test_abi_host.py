@@ -59,6 +59,21 @@ def test_step_staging_size_without_gpu():
     assert B.lib().innerq_step_staging_bytes(C.byref(cfg), None) == -1
 
 
+def test_multi_query_scratch_size_without_gpu():
+    # partials of four query rows per (batch, KV head) unit: the per-row size is the single-query workspace's
+    need, ws, cb = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    cfg1 = B.make_config(batch=1, n_q_heads=1, n_kv_heads=1, max_tokens=64)
+    cfg8 = B.make_config(batch=2, n_q_heads=8, n_kv_heads=4, max_tokens=64)
+    sizes = []
+    for cfg in (cfg1, cfg8):
+        assert B.lib().innerq_multi_query_scratch_bytes(C.byref(cfg), C.byref(need)) == 0
+        assert need.value > 0 and need.value % 256 == 0
+        sizes.append(need.value)
+    assert B.lib().innerq_multi_query_scratch_bytes(C.byref(cfg1), None) == -1
+    bad = B.make_config(batch=1, n_q_heads=3, n_kv_heads=2, max_tokens=64)
+    assert B.lib().innerq_multi_query_scratch_bytes(C.byref(bad), C.byref(need)) == -1
+
+
 def test_packed_payload_matches_table_bits():
     # Table "bits" (G = 32, head dim 128): effective bits per cached number = payload bytes * 8 / 128.
     rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table_bits.txt"))

@@ -272,6 +272,66 @@ def test_degenerate_windows(w_sink, w_recent):
     P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
 
 
+@pytest.mark.parametrize("grouping,r,G,bits,n_q", [(O.INNER, 1, 32, 2, 4), (O.INNER, 1, 32, 2, 7), (O.INNER, 4, 64, 2, 3),
+                                                    (O.INNER, 2, 128, 4, 5), (O.INNER, 1, 64, 3, 9), (O.OUTER, 1, 32, 2, 6),
+                                                    (O.OUTER, 4, 64, 4, 2)])
+def test_multi_query_decode(grouping, r, G, bits, n_q):
+    # n_q query tokens per sequence against one cache state, causal among the newest n_q tokens; rows of a KV
+    # head share passes over the packed cache four at a time
+    inner = grouping == O.INNER
+    w = synth.tiny(batch=2, n_q_heads=2 * r, n_kv_heads=2, n_tokens=4 + 20 * 32 + 77, group=G, k_bits=bits, v_bits=bits,
+                   w_sink=4, w_recent=24, grouping=grouping, k_normalize=int(inner),
+                   **({} if inner else dict(k_mode=O.ASYM, v_mode=O.ASYM)))
+    oc, gc, _, _ = run_prefill_both(w)
+    for step in range(3):                 # a few appended tokens, so the ring buffers are rotated
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+    q = np.stack([synth.query(w, 10 + i) for i in range(n_q)], axis=1)           # [B, n_q, Hq, D]
+    ref = oc.decode_multi(q)
+    for splits in (0, 1, 3):
+        gc.innerq_set_decode_options(splits, 0)
+        out = gc.innerq_decode_attention_multi(dev(q)).cpu().numpy()
+        P.assert_outputs_close(out, ref, f"multi-query n_q={n_q} splits={splits}")
+    gc.innerq_set_decode_options(0, 0)
+    # the newest query row is the plain decode of the same cache
+    one = gc.innerq_decode_attention(dev(q[:, n_q - 1])).cpu().numpy()
+    P.assert_outputs_close(one, ref[:, n_q - 1], "newest query = single-token decode")
+    assert gc.innerq_read_device_error() == 0
+
+
+def test_multi_query_short_contexts_and_limits():
+    from paper_2602_23200_b200 import binding as B
+    # everything in the windows: even sink tokens are masked by position
+    w = synth.tiny(n_tokens=11, w_sink=4, w_recent=16)
+    oc, gc, _, _ = run_prefill_both(w)
+    for n_q in (1, 2, 6, 11):
+        q = np.stack([synth.query(w, i) for i in range(n_q)], axis=1)
+        out = gc.innerq_decode_attention_multi(dev(q)).cpu().numpy()
+        P.assert_outputs_close(out, oc.decode_multi(q), f"windows only, n_q={n_q}")
+    q12 = np.stack([synth.query(w, i) for i in range(12)], axis=1)
+    with pytest.raises(B.InnerQError) as ei:              # more query tokens than cached tokens
+        gc.innerq_decode_attention_multi(dev(q12))
+    assert ei.value.status == -1
+    # hidden tokens would reach into the chunks where keys and values are both packed: refused, nothing launched
+    w = synth.tiny(n_tokens=4 + 64 + 8, w_sink=4, w_recent=8)
+    oc, gc, _, _ = run_prefill_both(w)
+    e = oc.export()
+    room = w.n_tokens - e["n_sink"] - min(e["n_qk"], e["n_qv"])       # tokens that can be hidden
+    q_ok = np.stack([synth.query(w, i) for i in range(room + 1)], axis=1)
+    P.assert_outputs_close(gc.innerq_decode_attention_multi(dev(q_ok)).cpu().numpy(), oc.decode_multi(q_ok), "at the limit")
+    q_bad = np.stack([synth.query(w, i) for i in range(room + 2)], axis=1)
+    with pytest.raises(B.InnerQError) as ei:
+        gc.innerq_decode_attention_multi(dev(q_bad))
+    assert ei.value.status == -2
+    # an unquantised cache has no fused kernel: refused as well
+    wf = synth.tiny(n_tokens=40, grouping=O.FP16, k_normalize=0)
+    _, gf, _, _ = run_prefill_both(wf)
+    with pytest.raises(B.InnerQError) as ei:
+        gf.innerq_decode_attention_multi(dev(np.stack([synth.query(wf, i) for i in range(2)], axis=1)))
+    assert ei.value.status == -2
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
