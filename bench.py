@@ -200,12 +200,31 @@ def oracle_steps(w, n_steps, units=None):
         oc.decode(q)
         times.append(time.perf_counter() - t0)
         nbytes.append(decode_algorithmic_bytes(sub, oc.N)[0])
+    extra = {}
     try:
-        from threadpoolctl import threadpool_info
+        from threadpoolctl import threadpool_info, threadpool_limits
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        with threadpool_limits(limits=1):          # one more step on a single thread
+            k1, v1 = synth.new_token(sub, n_steps)
+            q = synth.query(sub, n_steps)
+            t0 = time.perf_counter()
+            oc.append(k1, v1)
+            oc.decode(q)
+            extra["single_thread_s_per_step"] = time.perf_counter() - t0
     except Exception:
         cores = 1
-    return float(np.mean(times)), float(np.mean(nbytes)), cores
+    if sub.grouping != synth.FP16:
+        # hybrid groups whose two candidates' L1 errors differ by less than 1e-4 relative: either mask is right there
+        e = oc.export()
+        n_cont = n_all = 0
+        for name, mode in (("k", sub.k_mode), ("v", sub.v_mode)):
+            if mode == synth.HYBRID:
+                ea, es = e[f"{name}_err_asym"], e[f"{name}_err_sym"]
+                n_cont += int((np.abs(ea - es) <= 1e-4 * np.maximum(ea, es)).sum())
+                n_all += int(ea.size)
+        extra["contested_hybrid_groups"] = n_cont
+        extra["hybrid_groups"] = n_all
+    return float(np.mean(times)), float(np.mean(nbytes)), cores, extra
 
 
 def run_reference(args, w):
@@ -215,7 +234,7 @@ def run_reference(args, w):
     units = min(w.n_units, 4)
     for _ in range(args.warmup and 1):
         pass
-    t, b, cores = oracle_steps(w, max(1, min(args.steps, 8)), units=units)
+    t, b, cores, _ = oracle_steps(w, max(1, min(args.steps, 8)), units=units)
     gbs = b / t / 1e9
     line = {"impl": "reference", "metric": "decode_step_algorithmic_hbm_gbs", "value": gbs, "unit": "GB/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
@@ -271,7 +290,7 @@ def run_ours(args, w):
     total_steps = W + Kst
     e2e_steps = max(4, min(Kst, 32))
     split_steps = 2 * R * w.group if w.grouping != synth.FP16 else 0     # extra steps timed one by one (below)
-    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps + split_steps) // R + 8)
+    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps + split_steps) // R + 16)
     Kh, Vh = synth.kv_all(w)
     Kd, Vd = torch.from_numpy(Kh).cuda(), torch.from_numpy(Vh).cuda()
     caches = []
@@ -401,6 +420,16 @@ def run_ours(args, w):
     b1.record(stream)
     torch.cuda.synchronize()
     b2b_us = b0.elapsed_time(b1) / nb * 1e3
+    # the append kernel alone, each call between its own events (extra tokens beyond the timed steps)
+    app_n = 16
+    app_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(app_n)]
+    for j in range(app_n):
+        i = total_steps + e2e_steps + split_steps + j
+        app_ev[j][0].record(stream)
+        caches[j % R].innerq_append_token(k_new[i % n_in], v_new[i % n_in])
+        app_ev[j][1].record(stream)
+    torch.cuda.synchronize()
+    append_us = float(np.median([a.elapsed_time(b) for a, b in app_ev])) * 1e3
     # several query tokens per sequence in one call (causal among the newest n_q tokens), back to back like the above
     multi = None
     if args.n_q > 1 and w.grouping != synth.FP16:
@@ -454,6 +483,7 @@ def run_ours(args, w):
             "steps": Kst, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
             "us_per_decode": dec_us, "us_per_decode_median": float(np.median(dec_ms)) * 1e3,
             "us_per_decode_min": float(np.min(dec_ms)) * 1e3, "us_per_decode_back_to_back": b2b_us,
+            "us_per_append_median": append_us,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config_dict(w, args),
             "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
@@ -476,10 +506,14 @@ def run_ours(args, w):
         }
         if not args.no_cpu_baseline and world == 1:
             units = min(w.n_units, 4)
-            t, b, cores = oracle_steps(w, 3, units=units)
+            t, b, cores, extra = oracle_steps(w, 3, units=units)
             line["cpu_baseline"] = {"value": b / t / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                     "us_per_step_full_workload": t * 1e6 * (w.n_units / units),
                                     "sample": f"{units} of {w.n_units} KV heads, 3 steps of append+decode"}
+            if "single_thread_s_per_step" in extra:
+                line["cpu_baseline"]["single_thread_value"] = b / extra["single_thread_s_per_step"] / 1e9
+            if "hybrid_groups" in extra:
+                line["info"]["contested_hybrid_groups_in_sample"] = [extra["contested_hybrid_groups"], extra["hybrid_groups"]]
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
