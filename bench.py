@@ -317,6 +317,21 @@ def run_ours(args, w):
         rel_l2 = float(((o_q - o_ref).norm() / o_ref.norm()).item())
         ref_cache.close()
         del ref_cache, o_ref, o_q
+    # sequences of different lengths, one cache object each, decoded by one batched call (information; needs a batch)
+    ragged_sets, ragged_lengths = [], []
+    if w.batch > 1 and w.grouping != synth.FP16 and args.ragged:
+        fracs = [1.0, 0.125, 0.5, 0.25, 0.75, 1.0, 0.375, 0.625]
+        ragged_lengths = [max(w.w_sink + w.w_recent + w.group, int(w.n_tokens * fracs[i % len(fracs)])) for i in range(w.batch)]
+        w1 = w.with_(batch=1)
+        cfg1 = B.make_config(w1, max_tokens=w.n_tokens + 8)
+        per_set = sum(ragged_lengths) * w.n_kv_heads * sum(payload_bytes(w))
+        for _ in range(max(2, min(6, int(400e6 // max(per_set, 1)) + 1))):
+            cs = []
+            for i, n_i in enumerate(ragged_lengths):
+                c = B.InnerQCache(cfg1)
+                c.innerq_quantize_prefill(Kd[i:i + 1, :, :n_i].contiguous(), Vd[i:i + 1, :, :n_i].contiguous())
+                cs.append(c)
+            ragged_sets.append(cs)
     del Kd, Vd, Kh, Vh, ex
     torch.cuda.empty_cache()
 
@@ -448,6 +463,28 @@ def run_ours(args, w):
         multi = {"n_q": args.n_q, "us_per_call_back_to_back": multi_us, "us_per_query_token": multi_us / args.n_q,
                  "launches_per_call": caches[0].innerq_last_launch_count(2),
                  "single_query_us_back_to_back": b2b_us}
+    ragged = None
+    if ragged_sets:
+        qr = q_all[0].reshape(w.batch, 1, w.n_q_heads, w.head_dim).contiguous()
+        outr = torch.empty_like(qr)
+        for cs in ragged_sets:
+            B.innerq_decode_attention_batched(cs, qr, outr)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        r0.record(stream)
+        for i in range(nb):
+            B.innerq_decode_attention_batched(ragged_sets[i % len(ragged_sets)], qr, outr)
+        r1.record(stream)
+        torch.cuda.synchronize()
+        ragged_us = r0.elapsed_time(r1) / nb * 1e3
+        tok = sum(ragged_lengths)
+        ragged = {"lengths": ragged_lengths, "us_per_call_back_to_back": ragged_us,
+                  "tokens_per_call": tok * w.n_kv_heads,
+                  "us_if_time_scaled_with_tokens": b2b_us * tok / (w.batch * w.n_tokens),
+                  "cache_sets_rotated": len(ragged_sets)}
+        for cs in ragged_sets:
+            for c in cs:
+                c.close()
     # steps timed one by one (events around append + decode): those on which a value group (inner grouping) or a key
     # group (outer grouping) of G tokens is quantised, against the others
     step_split = None
@@ -490,7 +527,7 @@ def run_ours(args, w):
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
             "second_roof": pipe_roofs_gbs(stored_counters(w.name), bytes_min / Kst, clocks.get("sm_mhz")),
-            "step_us_by_kind": step_split, "multi_query": multi,
+            "step_us_by_kind": step_split, "multi_query": multi, "ragged_batch": ragged,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
@@ -530,6 +567,7 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ragged", type=int, default=1, help="1: also time a batched decode over sequences of mixed lengths")
     ap.add_argument("--n-q", type=int, default=4, help="query tokens per call of the multi-query leg (0/1: skip it)")
     args = ap.parse_args()
     w = workload_by_name(args.workload)

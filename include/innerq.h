@@ -174,6 +174,25 @@ int innerq_decode_attention_multi(innerq_cache_t* cache, const void* q, void* ou
 /* Bytes of device scratch innerq_decode_attention_multi needs (independent of n_q).  Errors: INVALID_ARG. */
 int innerq_multi_query_scratch_bytes(const innerq_config_t* cfg, size_t* bytes);
 
+/* Append and decode for several caches in one call each: sequences of different lengths that are decoded together
+ * (continuous batching).  The paper's kernels take one cache of one length; here every sequence has its own cache
+ * object (typically created with batch = 1), its own token count and its own eviction schedule, and one launch
+ * serves them all: block x of the grid is (cache i, unit u), and every cache brings its own token counts.
+ *   caches : host array of n handles (1 <= n <= 32), all created from the SAME configuration (max_tokens
+ *            included) and all different; each with its own workspace.
+ *   k_new, v_new : device, fp16 [n][batch, n_kv_heads, head_dim]  (cache i's rows at index i)
+ *   q, out       : device, fp16 [n][batch, n_q_heads, head_dim]
+ * innerq_append_token_batched appends one token to every listed cache (a cache that should not advance is left
+ * out of the list); innerq_decode_attention_batched attends for every listed cache over its own tokens.
+ * The decode needs the fused kernel (packed inner- or outer-grouped cache in a format it supports, decode variant
+ * 0 or 2 on the first cache): otherwise UNSUPPORTED.  Split counts follow the first cache's decode options.
+ * Errors: INVALID_ARG (different configurations, a cache listed twice, an empty cache in the decode), CAPACITY (a
+ * listed cache is full; nothing is appended to any), UNSUPPORTED, CUDA. */
+int innerq_append_token_batched(innerq_cache_t* const* caches, int32_t n, const void* k_new, const void* v_new,
+                                void* cuda_stream);
+int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, const void* q, void* out,
+                                    void* cuda_stream);
+
 /* Same computation and arguments as innerq_decode_attention, for callers that cannot give the decode
  * step any scratch memory of their own.  (The paper has no counterpart; this is an integration aid.)
  * Typical cases: the workspace passed to innerq_cache_create was only lent for the prefill and has gone

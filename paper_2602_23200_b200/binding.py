@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "innerq_cache_n_tokens", "innerq_quantize_prefill", "innerq_append_token", "innerq_decode_attention",
     "innerq_decode_attention_static", "innerq_decode_step_host", "innerq_step_staging_bytes",
     "innerq_decode_attention_multi", "innerq_multi_query_scratch_bytes",
+    "innerq_append_token_batched", "innerq_decode_attention_batched",
     "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
@@ -75,6 +76,8 @@ def lib() -> C.CDLL:
     L.innerq_step_staging_bytes.argtypes = [cfgp, C.POINTER(sz)]
     L.innerq_decode_attention_multi.argtypes = [vp, vp, vp, i32, vp, sz, vp]
     L.innerq_multi_query_scratch_bytes.argtypes = [cfgp, C.POINTER(sz)]
+    L.innerq_append_token_batched.argtypes = [C.POINTER(vp), i32, vp, vp, vp]
+    L.innerq_decode_attention_batched.argtypes = [C.POINTER(vp), i32, vp, vp, vp]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
@@ -141,6 +144,36 @@ def _dev_ptr(t, name: str, shape) -> int:
     if tuple(t.shape) != tuple(shape):
         raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
     return t.data_ptr()
+
+
+def _handles(caches):
+    if not caches or any(not isinstance(c, InnerQCache) for c in caches):
+        raise TypeError("caches must be a non-empty sequence of InnerQCache objects")
+    arr = (C.c_void_p * len(caches))(*[c._h for c in caches])
+    return arr
+
+
+def innerq_append_token_batched(caches, k_new, v_new, stream=None):
+    """Appends one token to every cache of the list (same configuration, own lengths): k_new, v_new are
+    fp16 [n, batch, n_kv_heads, head_dim] device tensors, row i for caches[i]."""
+    c = caches[0].cfg
+    shape = (len(caches), c.batch, c.n_kv_heads, c.head_dim)
+    _check(lib().innerq_append_token_batched(_handles(caches), len(caches), _dev_ptr(k_new, "k_new", shape),
+                                             _dev_ptr(v_new, "v_new", shape), _stream_ptr(stream)),
+           "innerq_append_token_batched")
+
+
+def innerq_decode_attention_batched(caches, q, out=None, stream=None):
+    """Decode attention for every cache of the list over its own tokens: q fp16 [n, batch, n_q_heads, head_dim]."""
+    import torch
+    c = caches[0].cfg
+    shape = (len(caches), c.batch, c.n_q_heads, c.head_dim)
+    if out is None:
+        out = torch.empty(shape, dtype=torch.float16, device=caches[0].device)
+    _check(lib().innerq_decode_attention_batched(_handles(caches), len(caches), _dev_ptr(q, "q", shape),
+                                                 _dev_ptr(out, "out", shape), _stream_ptr(stream)),
+           "innerq_decode_attention_batched")
+    return out
 
 
 class InnerQCache:

@@ -312,6 +312,64 @@ int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, i
   return INNERQ_OK;
 }
 
+// ---- several caches per call (sequences of different lengths) -----------------------------------------
+namespace {
+// All caches of a batched call must have been created from the same configuration: the kernels take one layout.
+bool same_layout(innerq_cache_t* const* caches, int n) {
+  for (int i = 0; i < n; ++i) {
+    if (!caches[i]) return false;
+    if (i && std::memcmp(&caches[i]->L, &caches[0]->L, sizeof(Layout)) != 0) return false;
+  }
+  return true;
+}
+}  // namespace
+
+int innerq_append_token_batched(innerq_cache_t* const* caches, int32_t n, const void* k_new, const void* v_new,
+                                void* cuda_stream) {
+  if (!caches || !k_new || !v_new || n < 1 || n > kMaxSeqs || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
+  unsigned char* ptr[kMaxSeqs];
+  int Ns[kMaxSeqs];
+  for (int i = 0; i < n; ++i) {
+    for (int j = 0; j < i; ++j)
+      if (caches[j] == caches[i]) return INNERQ_ERR_INVALID_ARG;      // one token per cache and call
+    if (caches[i]->N + 1 > caches[i]->L.max_tokens) return INNERQ_ERR_CAPACITY;
+    ptr[i] = caches[i]->cache;
+    Ns[i] = caches[i]->N + 1;
+  }
+  const int l = launch_append_batched(caches[0]->L, n, ptr, Ns, static_cast<const __half*>(k_new),
+                                      static_cast<const __half*>(v_new), static_cast<cudaStream_t>(cuda_stream));
+  if (l < 0) return INNERQ_ERR_CUDA;
+  for (int i = 0; i < n; ++i) {
+    caches[i]->N += 1;
+    caches[i]->launches[1] = l;
+  }
+  return INNERQ_OK;
+}
+
+int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, const void* q, void* out, void* cuda_stream) {
+  if (!caches || !q || !out || n < 1 || n > kMaxSeqs || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
+  const innerq_cache_t* c0 = caches[0];
+  if ((c0->opt_variant != 0 && c0->opt_variant != 2) || c0->L.k.kind == kNone || !decode_mma_supported(c0->L))
+    return INNERQ_ERR_UNSUPPORTED;
+  const unsigned char* ptr[kMaxSeqs];
+  unsigned char* ws[kMaxSeqs];
+  int Ns[kMaxSeqs];
+  for (int i = 0; i < n; ++i) {
+    if (caches[i]->N < 1) return INNERQ_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (caches[j]->ws == caches[i]->ws) return INNERQ_ERR_INVALID_ARG;      // partials and tickets are per cache
+    ptr[i] = caches[i]->cache;
+    ws[i] = caches[i]->ws;
+    Ns[i] = caches[i]->N;
+  }
+  const int l = launch_decode_mma_batched(c0->L, n, ptr, ws, Ns, static_cast<const __half*>(q), static_cast<__half*>(out),
+                                          c0->opt_splits, static_cast<cudaStream_t>(cuda_stream));
+  if (l == -2) return INNERQ_ERR_UNSUPPORTED;
+  if (l < 0) return INNERQ_ERR_CUDA;
+  for (int i = 0; i < n; ++i) caches[i]->launches[2] = l;
+  return INNERQ_OK;
+}
+
 // ---- one step from host buffers ----------------------------------------------------------------------
 static size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 

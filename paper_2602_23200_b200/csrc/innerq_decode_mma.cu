@@ -36,28 +36,25 @@ FormatLauncher format_launcher(const Layout& L) {
   return nullptr;
 }
 
-}  // namespace
+using BatchedLauncher = int (*)(const Layout&, SeqTable&, int, int, int, cudaStream_t);
 
-bool decode_mma_supported(const Layout& L) { return format_launcher(L) != nullptr; }
+BatchedLauncher batched_launcher(const Layout& L) {
+  const FormatLauncher one = format_launcher(L);
+  if (one == &launch_decode_mma_outer_k2v2) return &launch_decode_mma_outer_k2v2_batched;
+  if (one == &launch_decode_mma_outer_k4v4) return &launch_decode_mma_outer_k4v4_batched;
+  if (one == &launch_decode_mma_k2v2_m44) return &launch_decode_mma_k2v2_m44_batched;
+  if (one == &launch_decode_mma_k4v4_m44) return &launch_decode_mma_k4v4_m44_batched;
+  if (one == &launch_decode_mma_k3v3_m44) return &launch_decode_mma_k3v3_m44_batched;
+  if (one == &launch_decode_mma_k2v2_m22) return &launch_decode_mma_k2v2_m22_batched;
+  if (one == &launch_decode_mma_k3v3_m22) return &launch_decode_mma_k3v3_m22_batched;
+  if (one == &launch_decode_mma_k4v4_m22) return &launch_decode_mma_k4v4_m22_batched;
+  if (one == &launch_decode_mma_k3v2_m22) return &launch_decode_mma_k3v2_m22_batched;
+  if (one == &launch_decode_mma_k3v2_m24) return &launch_decode_mma_k3v2_m24_batched;
+  return nullptr;
+}
 
-void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
-
-// n_q > 1: q and out are [B, n_q, Hq, D], the partials of a launch's (up to) four rows per unit go to
-// multi_partials [U * 4][max_splits][kPartialStride]
-int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials) {
-  const FormatLauncher launch = format_launcher(L);
-  if (!launch) return -2;
-  const Counts cn = counts_for(L, N);
-  if (n_splits <= 0) {
-    n_splits = (2 * 148) / L.U;                  // two resident CTAs per SM, one wave
-    if (n_splits < 1) n_splits = 1;
-  }
-  if (n_splits > L.max_splits) n_splits = L.max_splits;
-  if (n_splits > 128) n_splits = 128;            // slots of the merge tables in shared memory
-  DecodeArgs a;
-  a.cache = cache; a.ws = ws; a.q = q; a.out = out;
-  a.n_splits = n_splits;
+// The launch parameters of one cache that follow from its token count alone.
+void fill_count_args(const Layout& L, const Counts& cn, DecodeArgs& a) {
   // tokens where only one tensor is packed (inner: keys, outer: values), then the tokens that are fp16 in both
   const bool outer = L.grouping == 1;
   a.n_skew_tiles = ((outer ? cn.n_qv - cn.n_qk : cn.n_qk - cn.n_qv) + 15) / 16;
@@ -68,6 +65,61 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.k_ring_pos0 = L.k.ring_cap ? cn.n_qk % L.k.ring_cap : 0;
   a.v_ring_pos0 = L.v.ring_cap ? cn.n_qv % L.v.ring_cap : 0;
   a.head0 = 0;
+}
+
+int default_splits(const Layout& L, int n_units_total) {
+  int n_splits = (2 * 148) / n_units_total;      // two resident CTAs per SM, one wave
+  if (n_splits < 1) n_splits = 1;
+  if (n_splits > L.max_splits) n_splits = L.max_splits;
+  if (n_splits > 128) n_splits = 128;            // slots of the merge tables in shared memory
+  return n_splits;
+}
+
+}  // namespace
+
+bool decode_mma_supported(const Layout& L) { return format_launcher(L) != nullptr; }
+
+// n caches of the same layout L with their own token counts: q and out are [n][B * Hq * D].
+int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const* caches, unsigned char* const* wss,
+                              const int* Ns, const __half* q, __half* out, int n_splits, cudaStream_t st) {
+  const BatchedLauncher launch = batched_launcher(L);
+  if (!launch) return -2;
+  if (n < 1 || n > kMaxSeqs) return -1;
+  if (n_splits <= 0) n_splits = default_splits(L, n * L.U);
+  if (n_splits > L.max_splits) n_splits = L.max_splits;
+  if (n_splits > 128) n_splits = 128;
+  SeqTable T;
+  for (int i = 0; i < n; ++i) {
+    SeqArgs& e = T.s[i];
+    e.cn = counts_for(L, Ns[i]);
+    e.a.cache = caches[i]; e.a.ws = wss[i];
+    e.a.q = q + (size_t)i * L.B * L.Hq * kD;
+    e.a.out = out + (size_t)i * L.B * L.Hq * kD;
+    e.a.n_splits = n_splits;
+    fill_count_args(L, e.cn, e.a);
+    e.a.n_q = 1;
+    e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
+  }
+  for (int i = n; i < kMaxSeqs; ++i) T.s[i] = T.s[0];
+  return launch(L, T, n, n_splits, g_chunks_per_iter, st);
+}
+
+void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
+
+// n_q > 1: q and out are [B, n_q, Hq, D], the partials of a launch's (up to) four rows per unit go to
+// multi_partials [U * 4][max_splits][kPartialStride]
+int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
+                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials) {
+  const FormatLauncher launch = format_launcher(L);
+  if (!launch) return -2;
+  const Counts cn = counts_for(L, N);
+  if (n_splits <= 0) n_splits = default_splits(L, L.U);
+  if (n_splits > L.max_splits) n_splits = L.max_splits;
+  if (n_splits > 128) n_splits = 128;            // slots of the merge tables in shared memory
+  DecodeArgs a;
+  a.cache = cache; a.ws = ws; a.q = q; a.out = out;
+  a.n_splits = n_splits;
+  fill_count_args(L, cn, a);
   a.n_q = n_q;
   a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
   if (n_q < 1 || (n_q > 1 && !multi_partials)) return -1;

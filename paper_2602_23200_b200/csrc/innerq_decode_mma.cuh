@@ -245,8 +245,7 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 // m-tile's rows fall into); zero-points contribute sum_c q''_c Z_jc per group and sum_t p_t Z_{t,g} per channel
 // group.  One chunk per iteration, four heads per pass.
 template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
-__global__ void __launch_bounds__(kThreads, 2)
-decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
+__device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u) {
   constexpr int KP = KB == 3 ? 2 : KB, VP = VB == 3 ? 2 : VB;     // bits of the primary code plane
   using F = Fmt<KP>;
   using FV = Fmt<VP>;
@@ -271,7 +270,8 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, j = lane & 3;
-  const int u = blockIdx.x, split = blockIdx.y;
+  const int split = blockIdx.y;
+  if (split >= a.grid_y) return;      // batched launch: this sequence uses fewer grid rows than the longest one
   const int b = u / L.Hkv, hkv = u % L.Hkv;
   const int nh = min(SPLIT ? 1 : kHeads, L.r * a.n_q - a.head0);
   // Row of q / out of column h of this launch: head h' = (head0 + h) % r of query token i = (head0 + h) / r
@@ -281,12 +281,12 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     return (b * a.n_q + i) * L.Hq + hkv * L.r + (v - i * L.r);
   };
   const int prow0 = a.n_q > 1 ? u * kHeads : q_row(0);
-  const int n_parts = gridDim.y;
+  const int n_parts = a.grid_y;
   const bool fast = split < a.n_splits;
   // ---------------- this warp's work: tail tiles and a range of packed chunks ----------------------
   // Tail tiles of the unit are dealt round-robin to CTAs, then to warps.  A tile costs about as much as
   // `tail_cost_units` range units, so packed ranges are shortened accordingly (contiguous, ordered).
-  const int Gy = gridDim.y, cst = a.tail_cost_units;
+  const int Gy = a.grid_y, cst = a.tail_cost_units;
   const int n_chunks_total = (OUTER ? cn.n_qk : cn.n_qv) / kChunk;   // chunks in which keys AND values are packed
   const int n_units_total = (n_chunks_total + RU - 1) / RU;
   const int q_cta = a.tiles_q0 + (split < a.tiles_rem ? 1 : 0);                 // tail tiles of this CTA
@@ -1114,11 +1114,52 @@ decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
     s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
   }
   __syncthreads();
-  if (s_ticket != gridDim.y - 1) return;
+  if (s_ticket != a.grid_y - 1) return;
   __threadfence();
   merge_parts(a.partials, reinterpret_cast<float*>(smem), a.out, nh, n_parts, prow0,
               make_int4(q_row(0), q_row(1), q_row(2), q_row(3)), L.max_splits);
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
+}
+
+// One cache: block x = unit.
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>(L, cn, a, blockIdx.x);
+}
+// Several caches of one configuration: block x = sequence * U + unit, the sequence's counts and parameters come
+// from its table entry (read in place from the parameter space).
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_mma_batched_kernel(const __grid_constant__ Layout L, const __grid_constant__ SeqTable T) {
+  const int seq = blockIdx.x / L.U;
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
+}
+
+// Split-dependent launch parameters of one cache for a grid of grid_y rows (0: choose it): how many of the rows
+// stream packed chunks, the range units per row, the tail tiles per row.  Returns grid_y.
+template <int RU>
+int fill_split_args(const Layout& L, const Counts& cn, DecodeArgs& a, bool outer, int n_splits, int grid_y) {
+  const int n_chunks = (outer ? cn.n_qk : cn.n_qv) / kChunk;
+  const int n_units = (n_chunks + RU - 1) / RU;
+  const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
+  if (n_splits > by_work) n_splits = by_work;
+  if (n_units == 0) n_splits = 0;
+  if (grid_y <= 0) {
+    // without packed chunks the CTAs only share the tail tiles (eight per CTA)
+    grid_y = n_splits > 0 ? n_splits : (a.n_tail_tiles + kWarps - 1) / kWarps;
+    if (grid_y < 1) grid_y = 1;
+    if (grid_y > L.max_splits) grid_y = L.max_splits;
+  }
+  if (n_splits > grid_y) n_splits = grid_y;
+  a.grid_y = grid_y;
+  a.n_splits = n_splits;
+  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about as much as one value group's chunks
+  const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
+  a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
+  a.tiles_q0 = a.n_tail_tiles / grid_y;
+  a.tiles_rem = a.n_tail_tiles % grid_y;
+  return grid_y;
 }
 
 template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
@@ -1133,23 +1174,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
       return -1;
     configured = true;
   }
-  const int n_chunks = (OUTER ? cn.n_qk : cn.n_qv) / kChunk;
-  const int n_units = (n_chunks + RU - 1) / RU;
-  const int by_work = (n_units + kWarps - 1) / kWarps;      // at least one range unit per warp
-  if (n_splits > by_work) n_splits = by_work;
-  if (n_units == 0) n_splits = 0;
-  // without packed chunks the CTAs only share the tail tiles (eight per CTA)
-  int grid_y = n_splits > 0 ? n_splits : (a.n_tail_tiles + kWarps - 1) / kWarps;
-  if (grid_y < 1) grid_y = 1;
-  if (grid_y > L.max_splits) grid_y = L.max_splits;
-  a.n_splits = n_splits;
-  a.tail_cost_units = n_splits ? 1 : 0;     // a tail tile costs a warp about as much as one value group's chunks
-  {
-    const int virt = n_units + a.tail_cost_units * a.n_tail_tiles;
-    a.units_per_split = n_splits ? (virt + n_splits - 1) / n_splits : 0;
-  }
-  a.tiles_q0 = a.n_tail_tiles / grid_y;
-  a.tiles_rem = a.n_tail_tiles % grid_y;
+  const int grid_y = fill_split_args<RU>(L, cn, a, OUTER, n_splits, 0);
   dim3 grid(L.U, grid_y);
   int launches = 0;
   const int step = SPLIT ? 1 : kHeads;
@@ -1169,6 +1194,51 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
+// The same kernel over a table of caches.  Every sequence splits its own chunks over as many of the launch's
+// grid rows as it has work for; the rows beyond that only take their share of its tail tiles.
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
+  using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
+  constexpr int kSmem = SL::kCtaBytes;
+  constexpr int RU = SL::kCH;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+      return -1;
+    configured = true;
+  }
+  // Grid rows per sequence in proportion to its packed chunks (n_splits is what a sequence of average length gets),
+  // so that short sequences do not hold as many CTAs as long ones; the launch has the largest count.
+  long long total_chunks = 0;
+  for (int i = 0; i < n_seqs; ++i) total_chunks += (OUTER ? T.s[i].cn.n_qk : T.s[i].cn.n_qv) / kChunk;
+  int grid_y = 1;
+  for (int i = 0; i < n_seqs; ++i) {
+    const long long mine = (OUTER ? T.s[i].cn.n_qk : T.s[i].cn.n_qv) / kChunk;
+    int want = total_chunks > 0 ? (int)((mine * n_splits * n_seqs + total_chunks / 2) / total_chunks) : 1;
+    if (want < 1) want = 1;
+    if (want > L.max_splits) want = L.max_splits;
+    if (want > 128) want = 128;
+    const int gy = fill_split_args<RU>(L, T.s[i].cn, T.s[i].a, OUTER, want, 0);
+    if (gy > grid_y) grid_y = gy;
+  }
+  dim3 grid(n_seqs * L.U, grid_y);
+  int launches = 0;
+  const int step = SPLIT ? 1 : kHeads;
+  for (int h0 = 0; h0 < L.r; h0 += step) {
+    for (int i = 0; i < n_seqs; ++i) T.s[i].a.head0 = h0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, T) != cudaSuccess) return -1;
+    ++launches;
+  }
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
 // One packed format (key bits, value bits, metadata entry bytes of each) at every group size.  cpi: chunks of 32
 // tokens per loop iteration, 0 = automatic.  Two per iteration need twice the stage bytes, which only the
 // 2-bit/2-bit formats can afford with two resident CTAs per SM.
@@ -1178,6 +1248,31 @@ int launch_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_spl
     if (cpi != 1) return launch_one<KB, VB, G, KM, VM, SPLIT, 2>(L, cn, a, n_splits, st);
   }
   return launch_one<KB, VB, G, KM, VM, SPLIT, 1>(L, cn, a, n_splits, st);
+}
+
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT>
+int launch_cpi_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
+  if constexpr (KB == 2 && VB == 2) {
+    if (cpi != 1) return launch_one_batched<KB, VB, G, KM, VM, SPLIT, 2>(L, T, n_seqs, n_splits, st);
+  }
+  return launch_one_batched<KB, VB, G, KM, VM, SPLIT, 1>(L, T, n_seqs, n_splits, st);
+}
+
+template <int KB, int VB, int KM, int VM>
+int launch_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
+  if (L.G == 32 && L.r == 1) return launch_cpi_batched<KB, VB, 32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 32) return launch_cpi_batched<KB, VB, 32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 64) return launch_cpi_batched<KB, VB, 64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 128) return launch_cpi_batched<KB, VB, 128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  return -2;
+}
+
+template <int KB, int VB>
+int launch_format_outer_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
+  if (L.G == 32) return launch_one_batched<KB, VB, 32, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
+  if (L.G == 64) return launch_one_batched<KB, VB, 64, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
+  if (L.G == 128) return launch_one_batched<KB, VB, 128, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
+  return -2;
 }
 
 template <int KB, int VB, int KM, int VM>
@@ -1202,16 +1297,25 @@ int launch_format_outer(const Layout& L, const Counts& cn, const DecodeArgs& a, 
 
 // Defines the externally visible launcher of one format in the translation unit that compiles its kernels.
 #define IQ_MMA_FORMAT_NAME(KB, VB, KM, VM) launch_decode_mma_k##KB##v##VB##_m##KM##VM
+#define IQ_MMA_FORMAT_NAME_BATCHED(KB, VB, KM, VM) launch_decode_mma_k##KB##v##VB##_m##KM##VM##_batched
 #define IQ_DEFINE_MMA_FORMAT(KB, VB, KM, VM)                                                                  \
   int IQ_MMA_FORMAT_NAME(KB, VB, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, \
                                          int cpi, cudaStream_t st) {                                            \
     return launch_format<KB, VB, KM, VM>(L, cn, a, n_splits, cpi, st);                                          \
+  }                                                                                                             \
+  int IQ_MMA_FORMAT_NAME_BATCHED(KB, VB, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi,  \
+                                                    cudaStream_t st) {                                           \
+    return launch_format_batched<KB, VB, KM, VM>(L, T, n_seqs, n_splits, cpi, st);                               \
   }
 
 #define IQ_DEFINE_MMA_OUTER_FORMAT(KB, VB)                                                                          \
   int launch_decode_mma_outer_k##KB##v##VB(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,    \
                                            int, cudaStream_t st) {                                                   \
     return launch_format_outer<KB, VB>(L, cn, a, n_splits, st);                                                      \
+  }                                                                                                                  \
+  int launch_decode_mma_outer_k##KB##v##VB##_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int,    \
+                                                     cudaStream_t st) {                                              \
+    return launch_format_outer_batched<KB, VB>(L, T, n_seqs, n_splits, st);                                          \
   }
 
 }  // namespace iq

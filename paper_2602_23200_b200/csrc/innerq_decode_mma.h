@@ -14,11 +14,13 @@ struct DecodeArgs {
   unsigned char* ws;
   const __half* q;
   __half* out;
-  int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits)
+  int grid_y;            // grid rows (blockIdx.y) that work on this cache: the launch's gridDim.y, or fewer for a
+                         // short sequence of a batched launch (the rows beyond it return at once)
+  int n_splits;          // CTAs per unit that stream packed chunks (blockIdx.y < n_splits <= grid_y)
   int n_tail_tiles;      // tiles of 16 tokens outside the packed-K/packed-V range: skew tiles first, then fp16 tiles;
-                         // tile x belongs to CTA x % gridDim.y, warp (x / gridDim.y) % 8
+                         // tile x belongs to CTA x % grid_y, warp (x / grid_y) % 8
   int n_skew_tiles;      // of those, tiles whose keys are packed rows (values still fp16)
-  int tiles_q0, tiles_rem;   // n_tail_tiles / gridDim.y and n_tail_tiles % gridDim.y
+  int tiles_q0, tiles_rem;   // n_tail_tiles / grid_y and n_tail_tiles % grid_y
   int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
   int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
   int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
@@ -28,6 +30,16 @@ struct DecodeArgs {
                          // n_q - 1 - i tokens (all of them outside the chunks where keys AND values are packed)
   float* partials;       // split partials [rows][max_splits][kPartialStride]: row = global query head (n_q == 1) or
                          // unit * 4 + column of the launch (n_q > 1)
+};
+
+// Batched launch over several caches of one configuration, each with its own length (continuous batching):
+// block x = sequence * U + unit; every sequence has its own token counts and launch parameters.
+struct SeqArgs {
+  Counts cn;
+  DecodeArgs a;
+};
+struct SeqTable {
+  SeqArgs s[kMaxSeqs];
 };
 
 // Launchers by format: k<key bits>v<value bits>_m<bytes per key metadata entry><bytes per value metadata entry>.
@@ -40,6 +52,21 @@ int launch_decode_mma_k3v3_m22(const Layout& L, const Counts& cn, const DecodeAr
 int launch_decode_mma_k4v4_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
 int launch_decode_mma_k3v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
 int launch_decode_mma_k3v2_m24(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
+
+// The same for a table of sequences (n_seqs <= kMaxSeqs entries with cn and the N-dependent fields of a filled in).
+#define IQ_DECLARE_MMA_BATCHED(name) \
+  int name##_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st);
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k2v2_m44)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k4v4_m44)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v3_m44)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k2v2_m22)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v3_m22)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k4v4_m22)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v2_m22)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v2_m24)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_outer_k2v2)
+IQ_DECLARE_MMA_BATCHED(launch_decode_mma_outer_k4v4)
+#undef IQ_DECLARE_MMA_BATCHED
 
 // Outer-grouped comparison cache (same argument list; cpi is ignored).
 int launch_decode_mma_outer_k2v2(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);

@@ -100,6 +100,9 @@ struct Layout {
 constexpr int kPartialStride = kD + 4;   // acc[D], m, l, pad, pad
 
 // Token bookkeeping: a function of N alone.
+// Most caches one batched call (append / decode over independent caches of one configuration) takes.
+constexpr int kMaxSeqs = 32;
+
 struct Counts {
   int N, n_sink, n_qk, n_qv, n_k_recent, n_v_recent;
 };

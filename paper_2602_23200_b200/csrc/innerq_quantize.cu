@@ -267,6 +267,20 @@ __device__ __forceinline__ void append_evict_block(const Layout& L, const Store&
                      nq_before / L.G);
 }
 
+// One appended token of one unit: ring write of the new key / value rows, eviction of the oldest key row and, when
+// a group of G tokens has filled up, of the oldest G value rows (outer grouping: the other way round).
+__device__ __forceinline__ void append_unit(const Layout& L, const __half* __restrict__ xk, const __half* __restrict__ xv,
+                                            int N, int u, unsigned char* __restrict__ cache, __half* tile, uint32_t* words) {
+  const __half k_x = xk[threadIdx.x], v_x = xv[threadIdx.x];
+  const bool k_norm = L.k_normalize != 0;
+  append_evict_row(L, L.k, xk, N, u, cache, k_norm, words);
+  append_evict_row(L, L.v, xv, N, u, cache, false, words);
+  append_write(L, L.k, k_x, N, u, cache);
+  append_write(L, L.v, v_x, N, u, cache);
+  append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
+  append_evict_block(L, L.v, N, u, cache, false, tile, words);
+}
+
 __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
                                                      const __half* __restrict__ v_new, int N,
                                                      unsigned char* __restrict__ cache) {
@@ -277,16 +291,28 @@ __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __r
   // for this kernel's completion before its first global access); this kernel in turn waits for its predecessor.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const __half* xk = k_new + (size_t)u * kD;
-  const __half* xv = v_new + (size_t)u * kD;
-  const __half k_x = xk[threadIdx.x], v_x = xv[threadIdx.x];
-  const bool k_norm = L.k_normalize != 0;
-  append_evict_row(L, L.k, xk, N, u, cache, k_norm, words);
-  append_evict_row(L, L.v, xv, N, u, cache, false, words);
-  append_write(L, L.k, k_x, N, u, cache);
-  append_write(L, L.v, v_x, N, u, cache);
-  append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
-  append_evict_block(L, L.v, N, u, cache, false, tile, words);
+  append_unit(L, k_new + (size_t)u * kD, v_new + (size_t)u * kD, N, u, cache, tile, words);
+}
+
+// The same for several caches of one configuration, each with its own token count: block x = sequence * U + unit,
+// k_new / v_new are [n][U][D].
+struct AppendSeq {
+  unsigned char* cache;
+  int N;       // token count after this append
+};
+struct AppendTable {
+  AppendSeq s[kMaxSeqs];
+};
+__global__ void __launch_bounds__(128) append_batched_kernel(const __grid_constant__ Layout L,
+                                                             const __half* __restrict__ k_new,
+                                                             const __half* __restrict__ v_new,
+                                                             const __grid_constant__ AppendTable T) {
+  __shared__ __align__(16) __half tile[128 * kD];
+  __shared__ uint32_t words[4 * 512];
+  const int seq = blockIdx.x / L.U, u = blockIdx.x - seq * L.U;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  append_unit(L, k_new + (size_t)blockIdx.x * kD, v_new + (size_t)blockIdx.x * kD, T.s[seq].N, u, T.s[seq].cache, tile, words);
 }
 
 // ------------------------------------------------------------------ canonical export
@@ -412,6 +438,23 @@ int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, co
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, append_kernel, L, k_new, v_new, N_after, cache) == cudaSuccess ? 1 : -1;
+}
+
+int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const __half* k_new,
+                          const __half* v_new, cudaStream_t st) {
+  if (n < 1 || n > kMaxSeqs) return -1;
+  AppendTable T;
+  for (int i = 0; i < kMaxSeqs; ++i) {
+    T.s[i].cache = caches[i < n ? i : 0];
+    T.s[i].N = Ns_after[i < n ? i : 0];
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n * L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, append_batched_kernel, L, k_new, v_new, T) == cudaSuccess ? 1 : -1;
 }
 
 int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st) {

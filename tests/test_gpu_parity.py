@@ -332,6 +332,77 @@ def test_multi_query_short_contexts_and_limits():
     assert ei.value.status == -2
 
 
+@pytest.mark.parametrize("grouping,r,G,bits", [(O.INNER, 1, 32, 2), (O.INNER, 4, 64, 2), (O.INNER, 2, 128, 4), (O.INNER, 1, 32, 3),
+                                               (O.OUTER, 2, 32, 2)])
+def test_batched_calls_over_sequences_of_different_lengths(grouping, r, G, bits):
+    # every sequence has its own cache object and length; one launch appends to / decodes all of them
+    from paper_2602_23200_b200 import binding as B
+    inner = grouping == O.INNER
+    lengths = [1, 37, 164, 700, 333, 4 + 16 + G]
+    base = synth.tiny(batch=1, n_q_heads=2 * r, n_kv_heads=2, group=G, k_bits=bits, v_bits=bits, grouping=grouping,
+                      k_normalize=int(inner), **({} if inner else dict(k_mode=O.ASYM, v_mode=O.ASYM)))
+    ws, ocs, gcs = [], [], []
+    for i, n in enumerate(lengths):
+        w = base.with_(n_tokens=n, wid=base.wid + 100 + i)
+        oc, gc, _, _ = run_prefill_both(w, max_tokens=1000)
+        ws.append(w); ocs.append(oc); gcs.append(gc)
+
+    def decode_all(step, who=None):
+        who = list(range(len(gcs))) if who is None else who
+        q = np.stack([synth.query(ws[i], step) for i in who])                      # [n, 1, Hq, D]
+        out = B.innerq_decode_attention_batched([gcs[i] for i in who], dev(q)).cpu().numpy()
+        for row, i in enumerate(who):
+            P.assert_outputs_close(out[row], ocs[i].decode(q[row]), f"sequence {i} (N={ocs[i].N}) step {step}")
+
+    decode_all(0)
+    for step in range(2 * G + 3):                   # every sequence crosses group evictions at its own steps
+        who = [i for i in range(len(gcs)) if not (i == 2 and step % 3 == 0)]       # sequence 2 skips some steps
+        toks = [synth.new_token(ws[i], step) for i in who]
+        for (k1, v1), i in zip(toks, who):
+            ocs[i].append(k1, v1)
+        B.innerq_append_token_batched([gcs[i] for i in who], dev(np.stack([t[0] for t in toks])),
+                                      dev(np.stack([t[1] for t in toks])))
+        if step in (0, 1, G - 1, G, 2 * G + 2):
+            decode_all(step + 1)
+            decode_all(step + 1, who=[3, 0])                                        # any subset, any order
+    for i, (oc, gc) in enumerate(zip(ocs, gcs)):
+        assert gc.n_tokens == oc.N
+        P.assert_export_equal(gc.innerq_cache_export(), oc.export(), grouping, G, k_hybrid=inner, v_hybrid=inner)
+        assert gc.innerq_read_device_error() == 0
+    # a single-cache call on one of them still agrees
+    q = synth.query(ws[4], 99)
+    P.assert_outputs_close(gcs[4].innerq_decode_attention(dev(q)).cpu().numpy(), ocs[4].decode(q), "single after batched")
+
+
+def test_batched_calls_argument_checks():
+    from paper_2602_23200_b200 import binding as B
+    w = synth.tiny(batch=1, n_q_heads=2, n_kv_heads=2, n_tokens=50)
+    _, a, _, _ = run_prefill_both(w, max_tokens=51)
+    _, b, _, _ = run_prefill_both(w, max_tokens=51)
+    _, other, _, _ = run_prefill_both(w.with_(group=64), max_tokens=51)
+    q2 = dev(np.stack([synth.query(w, 0), synth.query(w, 1)]))
+    k1, v1 = synth.new_token(w, 0)
+    kv2 = dev(np.stack([k1, k1])), dev(np.stack([v1, v1]))
+    for bad in ([a, a], [a, other]):                       # the same cache twice; different configurations
+        with pytest.raises(B.InnerQError) as ei:
+            B.innerq_decode_attention_batched(bad, q2)
+        assert ei.value.status == -1
+        with pytest.raises(B.InnerQError) as ei:
+            B.innerq_append_token_batched(bad, *kv2)
+        assert ei.value.status == -1
+    B.innerq_append_token_batched([a], dev(k1[None]), dev(v1[None]))           # a is full now (51 of 51)
+    with pytest.raises(B.InnerQError) as ei:
+        B.innerq_append_token_batched([b, a], *kv2)
+    assert ei.value.status == -3 and b.n_tokens == 50 and a.n_tokens == 51      # nothing was appended to b either
+    wf = w.with_(grouping=O.FP16, k_normalize=0)
+    _, f, _, _ = run_prefill_both(wf, max_tokens=51)
+    with pytest.raises(B.InnerQError) as ei:
+        B.innerq_decode_attention_batched([f], dev(synth.query(wf, 0)[None]))
+    assert ei.value.status == -2
+    out = B.innerq_decode_attention_batched([b, a], q2)
+    assert _torch().isfinite(out.float()).all()
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
