@@ -4,10 +4,11 @@ batch 1, 32 query heads, 8 KV heads, head_dim 128, group 32, sink 32, recent 96.
 
 Presets: Base (3-bit symmetric K and V), Hybrid (3-bit symmetric K, 2-bit hybrid V), Small (3-bit symmetric K,
 2-bit symmetric V), the 2-bit and 4-bit hybrid caches of the benchmark configurations, an outer-grouped
-(per-channel K, per-token V) 2-bit cache and the unquantised fp16 cache.  The hybrid mask density cannot be
-forced from outside (it is decided by the data), so the mask rows use the two readings of the symmetric formula
-and the all-asymmetric mode to reach about 0 %, 2 %, 93 % and 100 % flagged groups; the measured fraction is
-printed.  Key side and value side are one fused kernel here and are not timed separately.
+(per-channel K, per-token V) 2-bit cache and the unquantised fp16 cache.  The hybrid mask is decided by the data:
+besides the presets on the workload's own values (whose measured asymmetric fraction is printed), the mask
+ablation rows rebuild the values group by group so that 1, 10, 50 and 99 % of the value groups prefer the
+asymmetric candidate (values_with_mask_density).  Key side and value side are one fused kernel here and are not
+timed separately.
 
     python -m paper_2602_23200_b200.latency_study [--out table.md] [--lengths 512,4096,32768]
 
@@ -39,6 +40,34 @@ PRESETS = [
                                  v_mode=synth.ASYM)),
     ("fp16", dict(grouping=synth.FP16, k_normalize=0)),
 ]
+
+# The hybrid-mask ablation (Table "hybrid_ablation": the value kernel against the fraction of asymmetric groups),
+# on the "Hybrid" preset.  The mask is decided by the data, so the values are built group by group to land on
+# the wanted fraction: see values_with_mask_density.
+MASK_DENSITIES = [0.01, 0.10, 0.50, 0.99]
+MASK_PRESET = dict(k_bits=3, v_bits=2, k_mode=synth.SYM, v_mode=synth.HYBRID)
+
+
+def values_with_mask_density(V, w_sink: int, G: int, density: float, seed: int = 5):
+    """Copy of the fp16 values V [B, Hkv, N, D] in which a fraction `density` of the (G tokens x 1 channel) groups
+    behind the sink prefers the asymmetric candidate and the rest the symmetric one.  Asymmetric groups: the
+    original values shifted by +3 (far from zero-centred).  Symmetric groups: values from {-1, 0, 1} with at least
+    one -1, which the 2-bit symmetric quantiser (codes -1, 0, 1 times the scale max|x|) reproduces exactly, while
+    the asymmetric one (four levels between min and max) cannot hit 0 when both signs occur, and ties go to the
+    symmetric candidate."""
+    V = np.array(V, dtype=np.float16, copy=True)
+    Bn, H, N, D = V.shape
+    n_groups = max(0, (N - w_sink) // G)
+    if n_groups == 0:
+        return V
+    body = V[:, :, w_sink:w_sink + n_groups * G].astype(np.float32).reshape(Bn, H, n_groups, G, D)
+    rng = np.random.default_rng(seed)
+    asym = rng.random((Bn, H, n_groups, 1, D)) < density
+    sym_vals = np.where(np.abs(body) > 0.67, np.sign(body), 0.0).astype(np.float32)
+    sym_vals[:, :, :, 0, :] = -1.0
+    body = np.where(asym, body + 3.0, sym_vals)
+    V[:, :, w_sink:w_sink + n_groups * G] = body.reshape(Bn, H, n_groups * G, D).astype(np.float16)
+    return V
 
 
 def layer_workload(n_tokens: int, **kw) -> synth.Workload:
@@ -114,6 +143,27 @@ def main(argv=None) -> int:
             cache.close()
         rows.append((name, frac_v, cells))
         print(f"{name:28s} " + " ".join(f"{c:7.1f}/{wm:<7.1f}" for c, wm in cells), flush=True)
+    base_w = layer_workload(n_max)
+    for density in MASK_DENSITIES:
+        name = f"Hybrid K3s/V2h, mask {100 * density:g} % wanted"
+        Vm = torch.from_numpy(values_with_mask_density(V, base_w.w_sink, base_w.group, density)).cuda()
+        cells = []
+        frac_v = float("nan")
+        for n in lengths:
+            w = layer_workload(n, **MASK_PRESET)
+            cache = B.InnerQCache(B.make_config(w, max_tokens=n + 64))
+            cache.innerq_quantize_prefill(Kd[:, :, :n].contiguous(), Vm[:, :, :n].contiguous())
+            q = torch.from_numpy(synth.query(w)).cuda()
+            out = torch.empty_like(q)
+            cold, warm = time_decode(cache, q, out, flush, args.reps)
+            if n == n_max:
+                frac_v = asym_fraction(cache, "v_scale")
+            cells.append((cold, warm))
+            records.append({"preset": name, "n_tokens": n, "cold_us": round(cold, 2), "warm_us": round(warm, 2)})
+            cache.close()
+        rows.append((name, frac_v, cells))
+        print(f"{name:28s} " + " ".join(f"{c:7.1f}/{wm:<7.1f}" for c, wm in cells), flush=True)
+        del Vm
     lines = ["| preset (asym fraction of V groups) | " + " | ".join(str(n) for n in lengths) + " |",
              "|---|" + "---|" * len(lengths)]
     for name, fv, cells in rows:
