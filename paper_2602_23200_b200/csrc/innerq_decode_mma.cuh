@@ -1167,13 +1167,8 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
   using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSmem) != cudaSuccess)
-      return -1;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured)) return -1;
   const int grid_y = fill_split_args<RU>(L, cn, a, OUTER, n_splits, 0);
   dim3 grid(L.U, grid_y);
   int launches = 0;
@@ -1201,13 +1196,8 @@ int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, c
   using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
-      return -1;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (!opt_in_dynamic_smem(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured)) return -1;
   // Grid rows per sequence in proportion to its packed chunks (n_splits is what a sequence of average length gets),
   // so that short sequences do not hold as many CTAs as long ones; the launch has the largest count.
   long long total_chunks = 0;

@@ -640,11 +640,8 @@ int launch_decode_tc5(const Layout& L, const unsigned char* cache, unsigned char
                       int n_splits, cudaStream_t st) {
   if (!decode_tc5_supported(L)) return -2;
   const Counts cn = counts_for(L, N);
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(decode_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kT5Smem) != cudaSuccess) return -1;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  if (!opt_in_dynamic_smem(decode_tc5_kernel, kT5Smem, configured)) return -1;
   const int n_tiles = (cn.n_qv / kChunk + kChunksPerTile - 1) / kChunksPerTile;
   if (n_splits <= 0) n_splits = (3 * 148) / L.U;         // three CTAs per SM
   if (n_splits > n_tiles) n_splits = n_tiles;

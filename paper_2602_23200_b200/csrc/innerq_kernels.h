@@ -4,9 +4,24 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "innerq_layout.h"
 
 namespace iq {
+
+// More than 48 KB of dynamic shared memory is an opt-in per kernel AND per device: `done` (one per kernel, a bit per
+// device ordinal) remembers where it has been set, so a process that drives several GPUs sets it on each of them.
+template <typename Kernel>
+inline bool opt_in_dynamic_smem(Kernel kernel, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  const unsigned long long bit = 1ull << dev;
+  if (done.load(std::memory_order_acquire) & bit) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done.fetch_or(bit, std::memory_order_release);
+  return true;
+}
 
 struct ExportPtrs {
   uint8_t *k_code, *v_code;
