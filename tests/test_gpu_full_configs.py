@@ -138,3 +138,51 @@ def test_config5_sweep_point(bits, G, mode, grouping, variant):
         P.assert_outputs_close(q_rows(w, out, units), oc.decode(q_rows(w, q, units)), "fp16 cache")
         return
     compare(w, gc, oc, units)
+
+
+def test_config2_multi_query_call():
+    # four query tokens per call on the 32-head / 32768-token cache (the configuration bench.py's multi-query leg
+    # times): sampled heads against the oracle's causal decode of the same cache state
+    w = synth.config2()
+    K, V = synth.kv_all(w)
+    units = [2, 30]
+    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    n_q = 4
+    q = np.stack([synth.query(w, 200 + i) for i in range(n_q)], axis=1)                  # [B, n_q, Hq, D]
+    out = gc.innerq_decode_attention_multi(dev(q)).cpu().numpy()
+    q_sub = np.stack([q_rows(w, q[:, i], units)[0] for i in range(n_q)], axis=0)[None]   # [1, n_q, len(units)*r, D]
+    ref = oc.decode_multi(q_sub)
+    got = np.stack([q_rows(w, out[:, i], units)[0] for i in range(n_q)], axis=0)[None]
+    worst = P.assert_outputs_close(got, ref, "config2 multi-query")
+    assert gc.innerq_read_device_error() == 0
+    print(f"config2, 4 query tokens per call: worst err/tol {worst:.3f}")
+
+
+def test_config3_shape_sequences_of_different_lengths():
+    # the batched call of bench.py's ragged leg: 16 sequences (8 KV heads, r = 4, 2-bit, G = 64) of 1024 .. 8192
+    # tokens, one cache object each; two of the sequences are checked against their own oracle caches
+    from paper_2602_23200_b200 import binding as B
+    w = synth.config3(2)
+    fracs = [1.0, 0.125, 0.5, 0.25, 0.75, 1.0, 0.375, 0.625]
+    lengths = [int(w.n_tokens * fracs[i % len(fracs)]) for i in range(w.batch)]
+    w1 = w.with_(batch=1)
+    K, V = synth.kv_all(w1)                       # one sequence's data, cut to each length
+    cfg = B.make_config(w1, max_tokens=w.n_tokens + 8)
+    caches = []
+    for n in lengths:
+        c = B.InnerQCache(cfg)
+        c.innerq_quantize_prefill(dev(K[:, :, :n]), dev(V[:, :, :n]))
+        caches.append(c)
+    q = np.stack([synth.query(w1, i) for i in range(w.batch)])                           # [16, 1, Hq, D]
+    out = B.innerq_decode_attention_batched(caches, dev(q)).cpu().numpy()
+    worst = 0.0
+    for i in (1, 4):                              # 1024 and 6144 tokens
+        wi = w1.with_(n_tokens=lengths[i])
+        Ki, Vi = K[:, :, :lengths[i]], V[:, :, :lengths[i]]
+        units = [0, 5]
+        oc = sub_oracle(wi, np.ascontiguousarray(Ki), np.ascontiguousarray(Vi), units)
+        ref = oc.decode(q_rows(wi, q[i], units))
+        worst = max(worst, P.assert_outputs_close(q_rows(wi, out[i], units), ref, f"sequence {i}"))
+    for c in caches:
+        assert c.innerq_read_device_error() == 0
+    print(f"config-3 shape, 16 sequences of mixed lengths: worst err/tol {worst:.3f}")
