@@ -97,7 +97,8 @@ __device__ __forceinline__ void decode_fast(uint32_t meta, float neg_half, float
   const __half2 h = *reinterpret_cast<const __half2*>(&meta);
   const float sg = __low2float(h), Z = __high2float(h);
   s = fabsf(sg);
-  z = fmaf(neg_half, fmaxf(sg, 0.f), Z);
+  // neg_half * max(sg, 0) as (neg_half / 2) * (sg + |sg|): the same value exactly, on the fp32 pipe only
+  z = fmaf(0.5f * neg_half, sg + fabsf(sg), Z);
 }
 __device__ __forceinline__ float h2f_bits(uint32_t bits) { return __half2float(__ushort_as_half((unsigned short)bits)); }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
