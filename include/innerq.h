@@ -178,8 +178,8 @@ int innerq_multi_query_scratch_bytes(const innerq_config_t* cfg, size_t* bytes);
  * (continuous batching).  The paper's kernels take one cache of one length; here every sequence has its own cache
  * object (typically created with batch = 1), its own token count and its own eviction schedule, and one launch
  * serves them all: block x of the grid is (cache i, unit u), and every cache brings its own token counts.
- *   caches : host array of n handles (1 <= n <= 32), all created from the SAME configuration (max_tokens
- *            included) and all different; each with its own workspace.
+ *   caches : host array of n handles (1 <= n <= 4096; one launch per 32 of them), all created from the SAME
+ *            configuration (max_tokens included) and all different; each with its own workspace.
  *   k_new, v_new : device, fp16 [n][batch, n_kv_heads, head_dim]  (cache i's rows at index i)
  *   q, out       : device, fp16 [n][batch, n_q_heads, head_dim]
  * innerq_append_token_batched appends one token to every listed cache (a cache that should not advance is left

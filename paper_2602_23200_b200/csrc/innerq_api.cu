@@ -314,6 +314,7 @@ int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, i
 
 // ---- several caches per call (sequences of different lengths) -----------------------------------------
 namespace {
+constexpr int kMaxBatchedCaches = 4096;      // per call; a launch takes kMaxSeqs of them
 // All caches of a batched call must have been created from the same configuration: the kernels take one layout.
 bool same_layout(innerq_cache_t* const* caches, int n) {
   for (int i = 0; i < n; ++i) {
@@ -326,47 +327,64 @@ bool same_layout(innerq_cache_t* const* caches, int n) {
 
 int innerq_append_token_batched(innerq_cache_t* const* caches, int32_t n, const void* k_new, const void* v_new,
                                 void* cuda_stream) {
-  if (!caches || !k_new || !v_new || n < 1 || n > kMaxSeqs || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
-  unsigned char* ptr[kMaxSeqs];
-  int Ns[kMaxSeqs];
+  if (!caches || !k_new || !v_new || n < 1 || n > kMaxBatchedCaches || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
   for (int i = 0; i < n; ++i) {
     for (int j = 0; j < i; ++j)
       if (caches[j] == caches[i]) return INNERQ_ERR_INVALID_ARG;      // one token per cache and call
     if (caches[i]->N + 1 > caches[i]->L.max_tokens) return INNERQ_ERR_CAPACITY;
-    ptr[i] = caches[i]->cache;
-    Ns[i] = caches[i]->N + 1;
   }
-  const int l = launch_append_batched(caches[0]->L, n, ptr, Ns, static_cast<const __half*>(k_new),
-                                      static_cast<const __half*>(v_new), static_cast<cudaStream_t>(cuda_stream));
-  if (l < 0) return INNERQ_ERR_CUDA;
-  for (int i = 0; i < n; ++i) {
-    caches[i]->N += 1;
-    caches[i]->launches[1] = l;
+  const Layout& L = caches[0]->L;
+  const size_t row = (size_t)L.U * kD;                                 // fp16 elements per cache in k_new / v_new
+  int launches = 0;
+  for (int i0 = 0; i0 < n; i0 += kMaxSeqs) {                          // one launch per kMaxSeqs caches
+    const int m = n - i0 < kMaxSeqs ? n - i0 : kMaxSeqs;
+    unsigned char* ptr[kMaxSeqs];
+    int Ns[kMaxSeqs];
+    for (int i = 0; i < m; ++i) {
+      ptr[i] = caches[i0 + i]->cache;
+      Ns[i] = caches[i0 + i]->N + 1;
+    }
+    const int l = launch_append_batched(L, m, ptr, Ns, static_cast<const __half*>(k_new) + i0 * row,
+                                        static_cast<const __half*>(v_new) + i0 * row, static_cast<cudaStream_t>(cuda_stream));
+    if (l < 0) return INNERQ_ERR_CUDA;
+    for (int i = 0; i < m; ++i) caches[i0 + i]->N += 1;
+    launches += l;
   }
+  for (int i = 0; i < n; ++i) caches[i]->launches[1] = launches;
   return INNERQ_OK;
 }
 
 int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, const void* q, void* out, void* cuda_stream) {
-  if (!caches || !q || !out || n < 1 || n > kMaxSeqs || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
+  if (!caches || !q || !out || n < 1 || n > kMaxBatchedCaches || !same_layout(caches, n)) return INNERQ_ERR_INVALID_ARG;
   const innerq_cache_t* c0 = caches[0];
   if ((c0->opt_variant != 0 && c0->opt_variant != 2) || c0->L.k.kind == kNone || !decode_mma_supported(c0->L))
     return INNERQ_ERR_UNSUPPORTED;
-  const unsigned char* ptr[kMaxSeqs];
-  unsigned char* ws[kMaxSeqs];
-  int Ns[kMaxSeqs];
   for (int i = 0; i < n; ++i) {
     if (caches[i]->N < 1) return INNERQ_ERR_INVALID_ARG;
     for (int j = 0; j < i; ++j)
       if (caches[j]->ws == caches[i]->ws) return INNERQ_ERR_INVALID_ARG;      // partials and tickets are per cache
-    ptr[i] = caches[i]->cache;
-    ws[i] = caches[i]->ws;
-    Ns[i] = caches[i]->N;
   }
-  const int l = launch_decode_mma_batched(c0->L, n, ptr, ws, Ns, static_cast<const __half*>(q), static_cast<__half*>(out),
-                                          c0->opt_splits, static_cast<cudaStream_t>(cuda_stream));
-  if (l == -2) return INNERQ_ERR_UNSUPPORTED;
-  if (l < 0) return INNERQ_ERR_CUDA;
-  for (int i = 0; i < n; ++i) caches[i]->launches[2] = l;
+  const Layout& L = c0->L;
+  const size_t row = (size_t)L.B * L.Hq * kD;                          // fp16 elements per cache in q / out
+  int launches = 0;
+  for (int i0 = 0; i0 < n; i0 += kMaxSeqs) {
+    const int m = n - i0 < kMaxSeqs ? n - i0 : kMaxSeqs;
+    const unsigned char* ptr[kMaxSeqs];
+    unsigned char* ws[kMaxSeqs];
+    int Ns[kMaxSeqs];
+    for (int i = 0; i < m; ++i) {
+      ptr[i] = caches[i0 + i]->cache;
+      ws[i] = caches[i0 + i]->ws;
+      Ns[i] = caches[i0 + i]->N;
+    }
+    const int l = launch_decode_mma_batched(L, m, ptr, ws, Ns, static_cast<const __half*>(q) + i0 * row,
+                                            static_cast<__half*>(out) + i0 * row, c0->opt_splits,
+                                            static_cast<cudaStream_t>(cuda_stream));
+    if (l == -2) return INNERQ_ERR_UNSUPPORTED;
+    if (l < 0) return INNERQ_ERR_CUDA;
+    launches += l;
+  }
+  for (int i = 0; i < n; ++i) caches[i]->launches[2] = launches;
   return INNERQ_OK;
 }
 

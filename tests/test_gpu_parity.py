@@ -403,6 +403,27 @@ def test_batched_calls_argument_checks():
     assert _torch().isfinite(out.float()).all()
 
 
+def test_batched_calls_with_more_caches_than_one_launch_takes():
+    from paper_2602_23200_b200 import binding as B
+    n = 37                                                  # a launch takes 32: two launches
+    base = synth.tiny(batch=1, n_q_heads=2, n_kv_heads=1)
+    ws, ocs, gcs = [], [], []
+    for i in range(n):
+        w = base.with_(n_tokens=20 + 13 * i, wid=base.wid + 300 + i)
+        oc, gc, _, _ = run_prefill_both(w, max_tokens=600)
+        ws.append(w); ocs.append(oc); gcs.append(gc)
+    toks = [synth.new_token(ws[i], 0) for i in range(n)]
+    for (k1, v1), oc in zip(toks, ocs):
+        oc.append(k1, v1)
+    B.innerq_append_token_batched(gcs, dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks])))
+    assert gcs[0].innerq_last_launch_count(1) == 2
+    q = np.stack([synth.query(ws[i], 1) for i in range(n)])
+    out = B.innerq_decode_attention_batched(gcs, dev(q)).cpu().numpy()
+    for i in range(n):
+        assert gcs[i].n_tokens == ocs[i].N
+        P.assert_outputs_close(out[i], ocs[i].decode(q[i]), f"sequence {i} of {n}")
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
