@@ -85,9 +85,9 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
   const BatchedLauncher launch = batched_launcher(L);
   if (!launch) return -2;
   if (n < 1 || n > kMaxSeqs) return -1;
-  if (n_splits <= 0) n_splits = default_splits(L, n * L.U);
-  if (n_splits > L.max_splits) n_splits = L.max_splits;
-  if (n_splits > 128) n_splits = 128;
+  // rows (of U CTAs each) for all sequences together: one wave of two CTAs per SM, or n_splits per sequence on average
+  int row_budget = n_splits > 0 ? n_splits * n : (2 * 148) / L.U;
+  if (row_budget < n) row_budget = n;
   SeqTable T;
   for (int i = 0; i < n; ++i) {
     SeqArgs& e = T.s[i];
@@ -95,13 +95,13 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
     e.a.cache = caches[i]; e.a.ws = wss[i];
     e.a.q = q + (size_t)i * L.B * L.Hq * kD;
     e.a.out = out + (size_t)i * L.B * L.Hq * kD;
-    e.a.n_splits = n_splits;
+    e.a.n_splits = 0;
     fill_count_args(L, e.cn, e.a);
     e.a.n_q = 1;
     e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
   }
   for (int i = n; i < kMaxSeqs; ++i) T.s[i] = T.s[0];
-  return launch(L, T, n, n_splits, g_chunks_per_iter, st);
+  return launch(L, T, n, row_budget, g_chunks_per_iter, st);
 }
 
 void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }

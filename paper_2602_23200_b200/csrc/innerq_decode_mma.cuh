@@ -1199,15 +1199,28 @@ int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, c
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
   if (!opt_in_dynamic_smem(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured)) return -1;
-  // Grid rows per sequence in proportion to its packed chunks (n_splits is what a sequence of average length gets),
-  // so that short sequences do not hold as many CTAs as long ones; the launch has the largest count.
-  long long total_chunks = 0;
-  for (int i = 0; i < n_seqs; ++i) total_chunks += (OUTER ? T.s[i].cn.n_qk : T.s[i].cn.n_qv) / kChunk;
+  // Grid rows per sequence: the fewest chunks per row T such that all sequences together, each cut into rows of at
+  // most T chunks, need no more than n_splits rows in total (so the longest row, which sets the time, is as short
+  // as one wave of CTAs allows, and short sequences hold few CTAs).
+  long long chunks[kMaxSeqs], longest = 1;
+  for (int i = 0; i < n_seqs; ++i) {
+    chunks[i] = (OUTER ? T.s[i].cn.n_qk : T.s[i].cn.n_qv) / kChunk;
+    if (chunks[i] > longest) longest = chunks[i];
+  }
+  const long long budget = n_splits;                    // rows of all sequences together (each row is U CTAs)
+  auto rows_needed = [&](long long t) {
+    long long r = 0;
+    for (int i = 0; i < n_seqs; ++i) r += chunks[i] > 0 ? (chunks[i] + t - 1) / t : 1;
+    return r;
+  };
+  long long lo = 1, hi = longest;                       // smallest t with rows_needed(t) <= budget (hi always fits)
+  while (lo < hi) {
+    const long long mid = (lo + hi) / 2;
+    if (rows_needed(mid) <= budget) hi = mid; else lo = mid + 1;
+  }
   int grid_y = 1;
   for (int i = 0; i < n_seqs; ++i) {
-    const long long mine = (OUTER ? T.s[i].cn.n_qk : T.s[i].cn.n_qv) / kChunk;
-    int want = total_chunks > 0 ? (int)((mine * n_splits * n_seqs + total_chunks / 2) / total_chunks) : 1;
-    if (want < 1) want = 1;
+    int want = chunks[i] > 0 ? (int)((chunks[i] + lo - 1) / lo) : 1;
     if (want > L.max_splits) want = L.max_splits;
     if (want > 128) want = 128;
     const int gy = fill_split_args<RU>(L, T.s[i].cn, T.s[i].a, OUTER, want, 0);
