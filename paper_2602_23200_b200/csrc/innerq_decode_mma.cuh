@@ -621,8 +621,10 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       Bqr[s][1] = tw > 0 ? bqr_s[(s * 2 + 1) * 32 + lane] : 0u;
     }
     const float kfac_raw = pow2i(-(14 - qe_s[4 + my_head]));       // fp16 key rows: accumulator * kfac_raw
+    // From here on every warp uses its slice of the table area as scratch (the side ring of SPLIT, the exchange of
+    // decoded value metadata otherwise): all warps have taken their table entries into registers by now.
+    __syncthreads();
     if constexpr (SPLIT) {
-      __syncthreads();
       for (int i = lane; i < SL::kSideBytes / 4; i += 32) side[i] = 0u;
       __syncwarp();
     }
@@ -838,16 +840,21 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       }
 
       // ---------------- online softmax (log2 domain; raw scores still carry 1/kfac) -------------------
+      // The reference m_run of the running sums is any value within kLazy of the largest score so far, not the
+      // maximum itself: it only moves (with the cross-lane reduction and the rescaling that takes) when a score of
+      // this iteration exceeds it by more than kLazy, so p <= 2^kLazy and the usual iteration needs one vote.
+      constexpr float kLazy = OUTER ? 0.f : 4.f;
       float cmax = -INFINITY;
 #pragma unroll
       for (int cc = 0; cc < CPI; ++cc)
         cmax = fmaxf(cmax, fmaxf(fmaxf(sc[cc][0][0], sc[cc][0][1]), fmaxf(sc[cc][1][0], sc[cc][1][1])));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-      cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
       const float kf = OUTER ? 1.0f : kfac;                    // what the raw scores still have to be multiplied by
-      const float m_new = fmaxf(m_run, cmax * kf);
-      if (__any_sync(0xffffffffu, m_new > m_run)) {
+      float m_new = m_run;
+      if (__any_sync(0xffffffffu, cmax * kf > m_run + kLazy)) {
+        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 4));
+        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
+        m_new = fmaxf(m_run, cmax * kf);
         const float alpha = ex2_approx(m_run - m_new);     // 0 on the first iteration (m_run = -inf)
         l_part *= alpha;
         psum *= alpha;
@@ -986,7 +993,35 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
           pg += __shfl_xor_sync(0xffffffffu, pg, 16);
           pg *= 0x1p-14f;                               // accumulators carry p * 2^10 * 2^-24
           const uint32_t* vmg = SPLIT ? side + j * (SL::kVMeta / 4) : vm;    // this group's entries (slot j's in SPLIT)
-          if constexpr (VM == 4) {
+          // The value sums of a lane sit in the even accumulator columns (p enters as one fp16 per token, the lo
+          // column of its pair is zero), except in the outer-grouped variant.
+          auto acc_sum = [&](int m, int rh) { return OUTER ? accg[m][2 * rh] + accg[m][2 * rh + 1] : accg[m][2 * rh]; };
+          if constexpr (!SPLIT && VM == 4) {
+            // The four lanes of a quad need the same 16 entries: every lane decodes 4 of the group's 128 once, the
+            // warp exchanges (scale, zero-point) pairs through its side area (rows of 16 pairs, padded to 36 words
+            // so that the 128-bit reads of the eight lane groups fall into different banks), each lane reads its 16.
+            float* ds = reinterpret_cast<float*>(side);
+            {
+              const uint4 mw = *reinterpret_cast<const uint4*>(vmg + lane * 4);
+              const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
+              float sz[8];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) decode_fast(mws[e], neg_half_v, sz[2 * e], sz[2 * e + 1]);
+              float* dst = ds + (lane >> 2) * 36 + (lane & 3) * 8;       // entries 4*lane .. 4*lane+3 = row lane/4
+              *reinterpret_cast<float4*>(dst) = make_float4(sz[0], sz[1], sz[2], sz[3]);
+              *reinterpret_cast<float4*>(dst + 4) = make_float4(sz[4], sz[5], sz[6], sz[7]);
+            }
+            __syncwarp();
+            const float4* row = reinterpret_cast<const float4*>(ds + gid * 36);
+#pragma unroll
+            for (int q8 = 0; q8 < 8; ++q8) {
+              const float4 v = row[q8];                                   // entries 2*q8, 2*q8 + 1: (s, z, s, z)
+              const int m = q8;                                           // entry idx = 2 * m + rh
+              out_acc[m][0] = fmaf(v.x, acc_sum(m, 0), fmaf(v.y, pg, out_acc[m][0]));
+              out_acc[m][1] = fmaf(v.z, acc_sum(m, 1), fmaf(v.w, pg, out_acc[m][1]));
+            }
+            __syncwarp();                                                 // the side area is reused at the next group end
+          } else if constexpr (VM == 4) {
             const uint4* vm4 = reinterpret_cast<const uint4*>(vmg + gid * 16);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
@@ -997,7 +1032,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
                 const int idx = q4 * 4 + e, m = idx >> 1, rh = idx & 1;    // fragment row (m, rh) of lane group gid
                 float s_, z_;
                 decode_fast(mws[e], neg_half_v, s_, z_);
-                out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(z_, pg, out_acc[m][rh]));
+                out_acc[m][rh] = fmaf(s_, acc_sum(m, rh), fmaf(z_, pg, out_acc[m][rh]));
               }
             }
           } else {
@@ -1010,7 +1045,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
               for (int e = 0; e < 8; ++e) {
                 const int idx = q4 * 8 + e, m = idx >> 1, rh = idx & 1;
                 const float s_ = h2f_bits((uint16_t)((mws[e >> 1] >> (16 * (e & 1))) & 0x7FFFu));
-                out_acc[m][rh] = fmaf(s_, accg[m][2 * rh] + accg[m][2 * rh + 1], fmaf(neg_half_v * s_, pg, out_acc[m][rh]));
+                out_acc[m][rh] = fmaf(s_, acc_sum(m, rh), fmaf(neg_half_v * s_, pg, out_acc[m][rh]));
               }
             }
           }
