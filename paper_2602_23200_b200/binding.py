@@ -131,16 +131,23 @@ def innerq_token_payload_bytes(cfg: innerq_config_t):
     return kb.value, vb.value
 
 
-def _stream_ptr(stream) -> int:
+def _stream_ptr(stream, device=None) -> int:
+    """Raw cudaStream_t of `stream` (default: the current stream).  The library launches on the CURRENT device,
+    so a call for a cache that lives on another device is refused here instead of faulting on the GPU."""
     import torch
+    if device is not None and torch.cuda.current_device() != device.index:
+        raise RuntimeError(f"the current CUDA device is {torch.cuda.current_device()}, the cache lives on {device}: "
+                           "make the cache's device current (torch.cuda.set_device / torch.cuda.device) for the call")
     s = torch.cuda.current_stream() if stream is None else stream
     return int(s.cuda_stream)
 
 
-def _dev_ptr(t, name: str, shape) -> int:
+def _dev_ptr(t, name: str, shape, device=None) -> int:
     import torch
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float16 and t.is_contiguous()):
         raise TypeError(f"{name} must be a contiguous CUDA fp16 tensor")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name} is on {t.device}, the cache on {device}")
     if tuple(t.shape) != tuple(shape):
         raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
     return t.data_ptr()
@@ -158,8 +165,8 @@ def innerq_append_token_batched(caches, k_new, v_new, stream=None):
     fp16 [n, batch, n_kv_heads, head_dim] device tensors, row i for caches[i]."""
     c = caches[0].cfg
     shape = (len(caches), c.batch, c.n_kv_heads, c.head_dim)
-    _check(lib().innerq_append_token_batched(_handles(caches), len(caches), _dev_ptr(k_new, "k_new", shape),
-                                             _dev_ptr(v_new, "v_new", shape), _stream_ptr(stream)),
+    _check(lib().innerq_append_token_batched(_handles(caches), len(caches), _dev_ptr(k_new, "k_new", shape, caches[0].device),
+                                             _dev_ptr(v_new, "v_new", shape, caches[0].device), _stream_ptr(stream, caches[0].device)),
            "innerq_append_token_batched")
 
 
@@ -170,8 +177,8 @@ def innerq_decode_attention_batched(caches, q, out=None, stream=None):
     shape = (len(caches), c.batch, c.n_q_heads, c.head_dim)
     if out is None:
         out = torch.empty(shape, dtype=torch.float16, device=caches[0].device)
-    _check(lib().innerq_decode_attention_batched(_handles(caches), len(caches), _dev_ptr(q, "q", shape),
-                                                 _dev_ptr(out, "out", shape), _stream_ptr(stream)),
+    _check(lib().innerq_decode_attention_batched(_handles(caches), len(caches), _dev_ptr(q, "q", shape, caches[0].device),
+                                                 _dev_ptr(out, "out", shape, caches[0].device), _stream_ptr(stream, caches[0].device)),
            "innerq_decode_attention_batched")
     return out
 
@@ -179,10 +186,13 @@ def innerq_decode_attention_batched(caches, q, out=None, stream=None):
 class InnerQCache:
     """A packed KV cache living in caller-side torch device buffers, driven through the C ABI."""
 
-    def __init__(self, cfg: innerq_config_t, device="cuda:0", stream=None):
+    def __init__(self, cfg: innerq_config_t, device=None, stream=None):
         import torch
         self.cfg = cfg
-        self.device = torch.device(device)
+        # default: the current device (one process per GPU sets it once with torch.cuda.set_device)
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        if self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
         cb, wb = innerq_cache_bytes(cfg)
         self.cache_bytes, self.workspace_bytes = cb, wb
         with torch.cuda.device(self.device):
@@ -190,7 +200,7 @@ class InnerQCache:
             self._ws_buf = torch.empty(wb, dtype=torch.uint8, device=self.device)
             h = C.c_void_p()
             _check(lib().innerq_cache_create(C.byref(cfg), self._cache_buf.data_ptr(), cb, self._ws_buf.data_ptr(), wb,
-                                             _stream_ptr(stream), C.byref(h)), "innerq_cache_create")
+                                             _stream_ptr(stream, self.device), C.byref(h)), "innerq_cache_create")
         self._h = h
 
     def close(self):
@@ -216,14 +226,14 @@ class InnerQCache:
         c = self.cfg
         n = int(k.shape[2]) if k.dim() == 4 else -1
         shape = (c.batch, c.n_kv_heads, n, c.head_dim)
-        kp, vp = (_dev_ptr(k, "k", shape), _dev_ptr(v, "v", shape)) if n > 0 else (k.data_ptr(), v.data_ptr())
-        _check(lib().innerq_quantize_prefill(self._h, kp, vp, n, _stream_ptr(stream)), "innerq_quantize_prefill")
+        kp, vp = (_dev_ptr(k, "k", shape, self.device), _dev_ptr(v, "v", shape, self.device)) if n > 0 else (k.data_ptr(), v.data_ptr())
+        _check(lib().innerq_quantize_prefill(self._h, kp, vp, n, _stream_ptr(stream, self.device)), "innerq_quantize_prefill")
 
     def innerq_append_token(self, k_new, v_new, stream=None):
         c = self.cfg
         shape = (c.batch, c.n_kv_heads, c.head_dim)
-        _check(lib().innerq_append_token(self._h, _dev_ptr(k_new, "k_new", shape), _dev_ptr(v_new, "v_new", shape),
-                                         _stream_ptr(stream)), "innerq_append_token")
+        _check(lib().innerq_append_token(self._h, _dev_ptr(k_new, "k_new", shape, self.device), _dev_ptr(v_new, "v_new", shape, self.device),
+                                         _stream_ptr(stream, self.device)), "innerq_append_token")
 
     def innerq_decode_attention(self, q, out=None, stream=None):
         import torch
@@ -231,8 +241,8 @@ class InnerQCache:
         shape = (c.batch, c.n_q_heads, c.head_dim)
         if out is None:
             out = torch.empty(shape, dtype=torch.float16, device=self.device)
-        _check(lib().innerq_decode_attention(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
-                                             _stream_ptr(stream)), "innerq_decode_attention")
+        _check(lib().innerq_decode_attention(self._h, _dev_ptr(q, "q", shape, self.device), _dev_ptr(out, "out", shape, self.device),
+                                             _stream_ptr(stream, self.device)), "innerq_decode_attention")
         return out
 
     def innerq_decode_attention_static(self, q, out=None, stream=None):
@@ -244,8 +254,8 @@ class InnerQCache:
         shape = (c.batch, c.n_q_heads, c.head_dim)
         if out is None:
             out = torch.empty(shape, dtype=torch.float16, device=self.device)
-        _check(lib().innerq_decode_attention_static(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape),
-                                                    _stream_ptr(stream)), "innerq_decode_attention_static")
+        _check(lib().innerq_decode_attention_static(self._h, _dev_ptr(q, "q", shape, self.device), _dev_ptr(out, "out", shape, self.device),
+                                                    _stream_ptr(stream, self.device)), "innerq_decode_attention_static")
         return out
 
     def innerq_decode_attention_multi(self, q, out=None, stream=None):
@@ -263,9 +273,9 @@ class InnerQCache:
             n = C.c_size_t()
             _check(lib().innerq_multi_query_scratch_bytes(C.byref(c), C.byref(n)), "innerq_multi_query_scratch_bytes")
             self._multi_scratch = torch.empty(n.value, dtype=torch.uint8, device=self.device)
-        _check(lib().innerq_decode_attention_multi(self._h, _dev_ptr(q, "q", shape), _dev_ptr(out, "out", shape), n_q,
+        _check(lib().innerq_decode_attention_multi(self._h, _dev_ptr(q, "q", shape, self.device), _dev_ptr(out, "out", shape, self.device), n_q,
                                                    self._multi_scratch.data_ptr(), self._multi_scratch.numel(),
-                                                   _stream_ptr(stream)), "innerq_decode_attention_multi")
+                                                   _stream_ptr(stream, self.device)), "innerq_decode_attention_multi")
         return out
 
     def innerq_decode_step_host(self, k_new_host, v_new_host, q_host, out_host, stream=None):
@@ -285,14 +295,14 @@ class InnerQCache:
             _check(lib().innerq_step_staging_bytes(C.byref(c), C.byref(n)), "innerq_step_staging_bytes")
             self._staging = torch.empty(n.value, dtype=torch.uint8, device=self.device)
         _check(lib().innerq_decode_step_host(self._h, k_new_host.data_ptr(), v_new_host.data_ptr(), q_host.data_ptr(),
-                                             out_host.data_ptr(), self._staging.data_ptr(), _stream_ptr(stream)),
+                                             out_host.data_ptr(), self._staging.data_ptr(), _stream_ptr(stream, self.device)),
                "innerq_decode_step_host")
 
     def innerq_set_decode_options(self, n_splits: int = 0, variant: int = 0):
         _check(lib().innerq_set_decode_options(self._h, n_splits, variant), "innerq_set_decode_options")
 
     def innerq_read_device_error(self, stream=None) -> int:
-        return _check(lib().innerq_read_device_error(self._h, _stream_ptr(stream)), "innerq_read_device_error")
+        return _check(lib().innerq_read_device_error(self._h, _stream_ptr(stream, self.device)), "innerq_read_device_error")
 
     def innerq_last_launch_count(self, which: int) -> int:
         return _check(lib().innerq_last_launch_count(self._h, which), "innerq_last_launch_count")
@@ -325,7 +335,7 @@ class InnerQCache:
         ex = innerq_export_t()
         for name, ten in t.items():
             setattr(ex, name, ten.data_ptr())
-        _check(lib().innerq_cache_export(self._h, C.byref(ex), _stream_ptr(stream)), "innerq_cache_export")
+        _check(lib().innerq_cache_export(self._h, C.byref(ex), _stream_ptr(stream, self.device)), "innerq_cache_export")
         torch.cuda.synchronize(dev)
         out = {k: getattr(ex, k) for k in ("n_tokens", "n_sink", "n_qk", "n_qv", "n_k_recent", "n_v_recent")}
         host = {k: v.cpu().numpy() for k, v in t.items()}
