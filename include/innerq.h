@@ -132,7 +132,14 @@ int innerq_append_token(innerq_cache_t* cache, const void* k_new, const void* v_
  * fully overwritten.  Attends over all N cached tokens (append the step's token first); N >= 1.
  * Scores of quantised key rows use q' = q * norm; dequantisation happens in registers, scale and
  * zero-point are applied once per group.  Uses the workspace; two decodes on the same cache must
- * not overlap.  Errors: INVALID_ARG (N == 0 included), CUDA. */
+ * not overlap.
+ * Stream order: the kernels of append and decode are launched as programmatic dependents of the kernel before
+ * them in the stream, and the decode streams the part of the cache that no earlier call can still be writing
+ * (what was packed when the cache's previous decode was launched) and reads `q` BEFORE it waits for that kernel.
+ * All calls on one cache must therefore be enqueued in order on one stream (or be ordered by events), and `q`
+ * must not come from a kernel that signals programmatic launch completion before it has written `q`; ordinary
+ * kernels and copies earlier in the stream are always complete by then.
+ * Errors: INVALID_ARG (N == 0 included), CUDA. */
 int innerq_decode_attention(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
 
 /* One decode step from HOST buffers (the sequence the paper's Section "Latency" times per generated token:

@@ -15,6 +15,8 @@ struct innerq_cache {
   unsigned char* cache;
   unsigned char* ws;
   int N;
+  int N_safe;      // token count when the last decode of this cache was launched (or at prefill): what was packed by then
+                   // is complete and is not written again; a later decode may stream it before its predecessors finish
   int opt_splits, opt_variant;
   int launches[3];
 };
@@ -211,6 +213,7 @@ int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cach
   c->cache = static_cast<unsigned char*>(dev_cache);
   c->ws = static_cast<unsigned char*>(dev_workspace);
   c->N = 0;
+  c->N_safe = 0;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(c->cache, 0, c->L.cache_bytes, s) != cudaSuccess ||
       cudaMemsetAsync(c->ws, 0, c->L.workspace_bytes, s) != cudaSuccess) {
@@ -241,6 +244,7 @@ int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int
                          static_cast<cudaStream_t>(cuda_stream));
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N = n_tokens;
+  c->N_safe = n_tokens;
   c->launches[0] = n;
   return INNERQ_OK;
 }
@@ -269,13 +273,14 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L))
     n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
-                          c->opt_splits, s);
+                          c->opt_splits, s, 1, nullptr, c->N_safe);
   if (n == -2) {
     if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
     n = launch_decode_simt(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
   }
   if (n < 0) return INNERQ_ERR_CUDA;
+  c->N_safe = c->N;
   c->launches[2] = n;
   return INNERQ_OK;
 }
@@ -305,9 +310,10 @@ int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, i
   if (n_packed > 0 && c->N - n_q + 1 < cn.n_sink + n_packed) return INNERQ_ERR_UNSUPPORTED;
   const int n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                                   c->opt_splits, static_cast<cudaStream_t>(cuda_stream), n_q,
-                                  static_cast<float*>(dev_scratch));
+                                  static_cast<float*>(dev_scratch), c->N_safe);
   if (n == -2) return INNERQ_ERR_UNSUPPORTED;
   if (n < 0) return INNERQ_ERR_CUDA;
+  c->N_safe = c->N;
   c->launches[2] = n;
   return INNERQ_OK;
 }
@@ -371,17 +377,19 @@ int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, co
     const int m = n - i0 < kMaxSeqs ? n - i0 : kMaxSeqs;
     const unsigned char* ptr[kMaxSeqs];
     unsigned char* ws[kMaxSeqs];
-    int Ns[kMaxSeqs];
+    int Ns[kMaxSeqs], Ns_safe[kMaxSeqs];
     for (int i = 0; i < m; ++i) {
       ptr[i] = caches[i0 + i]->cache;
       ws[i] = caches[i0 + i]->ws;
       Ns[i] = caches[i0 + i]->N;
+      Ns_safe[i] = caches[i0 + i]->N_safe;
     }
-    const int l = launch_decode_mma_batched(L, m, ptr, ws, Ns, static_cast<const __half*>(q) + i0 * row,
+    const int l = launch_decode_mma_batched(L, m, ptr, ws, Ns, Ns_safe, static_cast<const __half*>(q) + i0 * row,
                                             static_cast<__half*>(out) + i0 * row, c0->opt_splits,
                                             static_cast<cudaStream_t>(cuda_stream));
     if (l == -2) return INNERQ_ERR_UNSUPPORTED;
     if (l < 0) return INNERQ_ERR_CUDA;
+    for (int i = 0; i < m; ++i) caches[i0 + i]->N_safe = caches[i0 + i]->N;
     launches += l;
   }
   for (int i = 0; i < n; ++i) caches[i]->launches[2] = launches;
@@ -482,13 +490,14 @@ int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, 
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L))
     n = launch_decode_mma(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
-                          c->opt_splits, s);
+                          c->opt_splits, s, 1, nullptr, c->N_safe);
   if (n == -2) {
     if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
     n = launch_decode_simt(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
   }
   if (n < 0) return INNERQ_ERR_CUDA;
+  c->N_safe = c->N;
   c->launches[2] = n;
   return INNERQ_OK;
 }

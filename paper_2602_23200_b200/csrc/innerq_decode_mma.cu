@@ -79,9 +79,12 @@ int default_splits(const Layout& L, int n_units_total) {
 
 bool decode_mma_supported(const Layout& L) { return format_launcher(L) != nullptr; }
 
+static int safe_chunks_for(const Layout& L, int N_safe, const Counts& cn_now);
+
 // n caches of the same layout L with their own token counts: q and out are [n][B * Hq * D].
 int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const* caches, unsigned char* const* wss,
-                              const int* Ns, const __half* q, __half* out, int n_splits, cudaStream_t st) {
+                              const int* Ns, const int* Ns_safe, const __half* q, __half* out, int n_splits,
+                              cudaStream_t st) {
   const BatchedLauncher launch = batched_launcher(L);
   if (!launch) return -2;
   if (n < 1 || n > kMaxSeqs) return -1;
@@ -97,6 +100,7 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
     e.a.out = out + (size_t)i * L.B * L.Hq * kD;
     e.a.n_splits = 0;
     fill_count_args(L, e.cn, e.a);
+    e.a.safe_chunks = safe_chunks_for(L, Ns_safe[i], e.cn);
     e.a.n_q = 1;
     e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
   }
@@ -108,8 +112,18 @@ void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n ==
 
 // n_q > 1: q and out are [B, n_q, Hq, D], the partials of a launch's (up to) four rows per unit go to
 // multi_partials [U * 4][max_splits][kPartialStride]
+// N_safe: token count of the cache when its previous decode was launched (or it was prefilled): chunks packed by
+// then are not written by any kernel that can still be running.
+static int safe_chunks_for(const Layout& L, int N_safe, const Counts& cn_now) {
+  const Counts old = counts_for(L, N_safe < 0 ? 0 : N_safe);
+  const bool outer = L.grouping == 1;
+  int s = (outer ? old.n_qk : old.n_qv) / kChunk;
+  const int now = (outer ? cn_now.n_qk : cn_now.n_qv) / kChunk;
+  return s < now ? s : now;
+}
+
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials) {
+                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials, int N_safe) {
   const FormatLauncher launch = format_launcher(L);
   if (!launch) return -2;
   const Counts cn = counts_for(L, N);
@@ -120,6 +134,7 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.cache = cache; a.ws = ws; a.q = q; a.out = out;
   a.n_splits = n_splits;
   fill_count_args(L, cn, a);
+  a.safe_chunks = safe_chunks_for(L, N_safe, cn);
   a.n_q = n_q;
   a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
   if (n_q < 1 || (n_q > 1 && !multi_partials)) return -1;

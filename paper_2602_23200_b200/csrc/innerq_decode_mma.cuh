@@ -365,10 +365,21 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  // Everything above touches no global memory: under a programmatic dependent launch it runs while the kernel
-  // before this one in the stream (the step's append, or the previous decode's merge) is still finishing.
-  // From here on its results are needed.
-  grid_dependency_wait();
+  // Everything above touches no global memory: under a programmatic dependent launch it runs while the kernels
+  // before this one in the stream (the step's append, the previous decode's merge) are still running.  What they may
+  // still be writing is known: the fp16 rings, and packed rows / groups that did not exist when the previous decode
+  // of this cache was launched (that decode made sure of its own predecessors before it let this one start).  So
+  // this kernel waits for its predecessors (dep_wait) only before it touches those: the tail tiles and the chunks
+  // from safe_chunks on.  q and the norms are inputs that are complete before the call (see innerq.h); the chunks
+  // below safe_chunks are streamed, and the q tables built, while the append is still running.
+  bool dep_waited = false;
+  auto dep_wait = [&]() {
+    if (!dep_waited) { grid_dependency_wait(); dep_waited = true; }
+  };
+  // an iteration's copy covers the chunks [c_lo + i * CPI, c_lo + (i + 1) * CPI)
+  auto dep_wait_for_iteration = [&](int i) {
+    if (c_lo + (i + 1) * CPI > a.safe_chunks) dep_wait();
+  };
   // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
   // hundred KB of queued chunk data per SM they would take microseconds to arrive.
   float q_early[2], n_early[2];
@@ -381,11 +392,12 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
     }
   }
-  if (lane == 0) {
 #pragma unroll
-    for (int s = 0; s < NST; ++s)
-      if (s < n_iters) issue(s);
-  }
+  for (int s = 0; s < NST; ++s)
+    if (s < n_iters) {
+      dep_wait_for_iteration(s);
+      if (lane == 0) issue(s);
+    }
 
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
   float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
@@ -670,6 +682,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     // running soft-max state.  Keys: fp16 rows against raw q'' (pieces tid4 + 4i of rows gid, gid + 8), or the
     // packed rows of the skew zone through the same path as the main loop.  Values: fp16 rows, pieces gid and
     // gid + 8 of token rows 2*tid4, 2*tid4 + 1 (+8), byte-permuted into (channel; token pair) fragments.
+    if (tw > 0) dep_wait();          // the rings and the newest packed rows are what the append writes
     for (int k = 0; k < tw; ++k) {
       bool skew; int e0, cnt;
       tail_tile(k, skew, e0, cnt);
@@ -1054,9 +1067,15 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       }
 
       __syncwarp();
-      if (lane == 0 && it + NST < n_iters) issue(st);
+      if (it + NST < n_iters) {
+        dep_wait_for_iteration(it + NST);
+        if (lane == 0) issue(st);
+      }
     }
 
+    // Before the next kernel in the stream may start (and stream its own safe chunks), this one has made sure that
+    // everything before it is complete; the partials and tickets written below are also shared with the previous decode.
+    dep_wait();
     grid_launch_dependents();     // the next kernel in the stream may start its own set-up during this epilogue
     if (failed) {
       // a copy never arrived: flag it for the host and contribute nothing

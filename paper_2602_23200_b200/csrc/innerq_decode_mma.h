@@ -24,6 +24,9 @@ struct DecodeArgs {
   int k_ring_pos0, v_ring_pos0;   // ring slot of the oldest recent key token / oldest fp16 value token
   int units_per_split;   // range units (max(value group, iteration) of chunks) per CTA, before the tail discount
   int tail_cost_units;   // a warp streams this many range units less per tail tile it handles (load balance)
+  int safe_chunks;       // chunks [0, safe_chunks) of every unit were complete before the previous decode of this cache
+                         // was launched: no kernel that may still be running writes them, so they are streamed
+                         // before this kernel waits for its predecessors (programmatic dependent launch)
   int head0;             // first query row (within the KV head's r * n_q) handled by this launch
   int n_q;               // consecutive query tokens per sequence (1: plain decode).  Row v = i * r + h of a KV head is
                          // head h of query token i; q / out are [B, n_q, Hq, D]; query i does not see the newest

@@ -46,9 +46,11 @@ int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned cha
 
 // Warp-MMA decode for the INNER layout.  Returns -2 if the configuration is not supported.
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st, int n_q = 1, float* multi_partials = nullptr);
+                      __half* out, int n_splits, cudaStream_t st, int n_q = 1, float* multi_partials = nullptr,
+                      int N_safe = 0);
 int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const* caches, unsigned char* const* wss,
-                              const int* Ns, const __half* q, __half* out, int n_splits, cudaStream_t st);
+                              const int* Ns, const int* Ns_safe, const __half* q, __half* out, int n_splits,
+                              cudaStream_t st);
 int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const __half* k_new,
                           const __half* v_new, cudaStream_t st);
 bool decode_mma_supported(const Layout& L);

@@ -76,7 +76,7 @@ def test_config2_prefill_then_steps():
     w = synth.config2()
     K, V = synth.kv_all(w)
     units = [0, 13, 31]
-    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    gc, oc = make_gpu(w, K, V, extra=128), sub_oracle(w, K, V, units, extra=128)
     compare(w, gc, oc, units, step=1000)
     worst = 0.0
     for step in range(40):                      # crosses value-group evictions (every 32 steps) and 40 key evictions
@@ -87,6 +87,29 @@ def test_config2_prefill_then_steps():
             _, e = compare(w, gc, oc, units, step=step, check_export=step in (4, 39))
             worst = max(worst, e)
     print(f"config2: worst err/tol over steps {worst:.3f}")
+    # 40 more steps enqueued back to back, no host synchronisation in between (the way bench.py's timed loop runs:
+    # the kernels of consecutive steps overlap), every step's output checked afterwards
+    import torch
+    n_more = 40
+    toks = [synth.new_token(w, 100 + s) for s in range(n_more)]
+    qs = [synth.query(w, 100 + s) for s in range(n_more)]
+    k_all, v_all, q_all = dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks])), dev(np.stack(qs))
+    outs = torch.empty_like(q_all)
+    torch.cuda.synchronize()
+    for s in range(n_more):
+        gc.innerq_append_token(k_all[s], v_all[s])
+        gc.innerq_decode_attention(q_all[s], outs[s])
+    torch.cuda.synchronize()
+    got = outs.cpu().numpy()
+    worst_b2b = 0.0
+    for s in range(n_more):
+        k1, v1 = toks[s]
+        oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+        ref = oc.decode(q_rows(w, qs[s], units))
+        worst_b2b = max(worst_b2b, P.assert_outputs_close(q_rows(w, got[s], units), ref, f"back-to-back step {s}"))
+    P.assert_export_equal(slice_export(gc.innerq_cache_export(), units), oc.export(), w.grouping, w.group, True, True)
+    assert gc.innerq_read_device_error() == 0
+    print(f"config2, 40 steps back to back: worst err/tol {worst_b2b:.3f}")
     # the tcgen05 kernel on the same cache (full size, its default split), same tolerance
     gc.innerq_set_decode_options(0, 5)
     _, e5 = compare(w, gc, oc, units, step=77, check_export=False)

@@ -424,6 +424,37 @@ def test_batched_calls_with_more_caches_than_one_launch_takes():
         P.assert_outputs_close(out[i], ocs[i].decode(q[i]), f"sequence {i} of {n}")
 
 
+@pytest.mark.parametrize("grouping,r,G", [(O.INNER, 1, 32), (O.INNER, 4, 64), (O.OUTER, 2, 32)])
+def test_steps_enqueued_back_to_back_without_host_synchronisation(grouping, r, G):
+    # The kernels of consecutive steps overlap on the GPU (each is a programmatic dependent of the one before it and
+    # the decode streams the settled part of the cache before it waits): enqueue many steps with no host
+    # synchronisation in between, then check every step's output and the final cache against the oracle.
+    torch = _torch()
+    inner = grouping == O.INNER
+    w = synth.tiny(batch=2, n_q_heads=4 * r, n_kv_heads=4, n_tokens=4 + 16 + 40 * 32 + 11, group=G, grouping=grouping,
+                   k_normalize=int(inner), **({} if inner else dict(k_mode=O.ASYM, v_mode=O.ASYM)))
+    n_steps = 2 * G + 9
+    oc, gc, _, _ = run_prefill_both(w, max_tokens=w.n_tokens + n_steps + 4)
+    toks = [synth.new_token(w, s) for s in range(n_steps)]
+    qs = [synth.query(w, s) for s in range(n_steps)]
+    k_all, v_all = dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks]))
+    q_all = dev(np.stack(qs))
+    outs = torch.empty_like(q_all)
+    torch.cuda.synchronize()
+    for s in range(n_steps):                       # nothing here waits for the GPU
+        gc.innerq_append_token(k_all[s], v_all[s])
+        gc.innerq_decode_attention(q_all[s], outs[s])
+        if s % 7 == 3:                             # some steps decode twice, some append twice in a row
+            gc.innerq_decode_attention(q_all[s], outs[s])
+    torch.cuda.synchronize()
+    got = outs.cpu().numpy()
+    for s in range(n_steps):
+        oc.append(*toks[s])
+        P.assert_outputs_close(got[s], oc.decode(qs[s]), f"step {s}")
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), grouping, G, k_hybrid=inner, v_hybrid=inner)
+    assert gc.innerq_read_device_error() == 0
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
