@@ -17,6 +17,8 @@ struct innerq_cache {
   int N;
   int N_safe;      // token count when the last decode of this cache was launched (or at prefill): what was packed by then
                    // is complete and is not written again; a later decode may stream it before its predecessors finish
+  int reads_settled;   // the last kernel enqueued for this cache was a fused decode: when its dependents may start, it
+                       // has read everything it reads from the cache (an append can then run without waiting first)
   int opt_splits, opt_variant;
   int launches[3];
 };
@@ -214,6 +216,7 @@ int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cach
   c->ws = static_cast<unsigned char*>(dev_workspace);
   c->N = 0;
   c->N_safe = 0;
+  c->reads_settled = 0;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(c->cache, 0, c->L.cache_bytes, s) != cudaSuccess ||
       cudaMemsetAsync(c->ws, 0, c->L.workspace_bytes, s) != cudaSuccess) {
@@ -245,6 +248,7 @@ int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N = n_tokens;
   c->N_safe = n_tokens;
+  c->reads_settled = 0;
   c->launches[0] = n;
   return INNERQ_OK;
 }
@@ -253,8 +257,9 @@ int innerq_append_token(innerq_cache_t* c, const void* k_new, const void* v_new,
   if (!c || !k_new || !v_new) return INNERQ_ERR_INVALID_ARG;
   if (c->N + 1 > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
   int n = launch_append(c->L, c->cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new), c->N + 1,
-                        static_cast<cudaStream_t>(cuda_stream));
+                        static_cast<cudaStream_t>(cuda_stream), c->reads_settled);
   if (n < 0) return INNERQ_ERR_CUDA;
+  c->reads_settled = 0;
   c->N += 1;
   c->launches[1] = n;
   return INNERQ_OK;
@@ -264,6 +269,7 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int n = -2;
+  bool fused = false;
   if (c->opt_variant == 5) {          // tcgen05 kernel, where it exists; no fallback
     n = launch_decode_tc5(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                           c->opt_splits, s);
@@ -271,9 +277,11 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   } else if (c->opt_variant != 1 && c->L.k.kind == kNone)
     n = launch_decode_fp16(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
-  else if (c->opt_variant != 1 && decode_mma_supported(c->L))
+  else if (c->opt_variant != 1 && decode_mma_supported(c->L)) {
     n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                           c->opt_splits, s, 1, nullptr, c->N_safe);
+    fused = n >= 0;
+  }
   if (n == -2) {
     if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
     n = launch_decode_simt(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
@@ -281,6 +289,7 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   }
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N_safe = c->N;
+  c->reads_settled = fused ? 1 : 0;
   c->launches[2] = n;
   return INNERQ_OK;
 }
@@ -314,6 +323,7 @@ int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, i
   if (n == -2) return INNERQ_ERR_UNSUPPORTED;
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N_safe = c->N;
+  c->reads_settled = 1;
   c->launches[2] = n;
   return INNERQ_OK;
 }
@@ -345,15 +355,19 @@ int innerq_append_token_batched(innerq_cache_t* const* caches, int32_t n, const 
   for (int i0 = 0; i0 < n; i0 += kMaxSeqs) {                          // one launch per kMaxSeqs caches
     const int m = n - i0 < kMaxSeqs ? n - i0 : kMaxSeqs;
     unsigned char* ptr[kMaxSeqs];
-    int Ns[kMaxSeqs];
+    int Ns[kMaxSeqs], late[kMaxSeqs];
     for (int i = 0; i < m; ++i) {
       ptr[i] = caches[i0 + i]->cache;
       Ns[i] = caches[i0 + i]->N + 1;
+      late[i] = caches[i0 + i]->reads_settled;
     }
-    const int l = launch_append_batched(L, m, ptr, Ns, static_cast<const __half*>(k_new) + i0 * row,
+    const int l = launch_append_batched(L, m, ptr, Ns, late, static_cast<const __half*>(k_new) + i0 * row,
                                         static_cast<const __half*>(v_new) + i0 * row, static_cast<cudaStream_t>(cuda_stream));
     if (l < 0) return INNERQ_ERR_CUDA;
-    for (int i = 0; i < m; ++i) caches[i0 + i]->N += 1;
+    for (int i = 0; i < m; ++i) {
+      caches[i0 + i]->N += 1;
+      caches[i0 + i]->reads_settled = 0;
+    }
     launches += l;
   }
   for (int i = 0; i < n; ++i) caches[i]->launches[1] = launches;
@@ -389,7 +403,10 @@ int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, co
                                             static_cast<cudaStream_t>(cuda_stream));
     if (l == -2) return INNERQ_ERR_UNSUPPORTED;
     if (l < 0) return INNERQ_ERR_CUDA;
-    for (int i = 0; i < m; ++i) caches[i0 + i]->N_safe = caches[i0 + i]->N;
+    for (int i = 0; i < m; ++i) {
+      caches[i0 + i]->N_safe = caches[i0 + i]->N;
+      caches[i0 + i]->reads_settled = 1;
+    }
     launches += l;
   }
   for (int i = 0; i < n; ++i) caches[i]->launches[2] = launches;
@@ -485,12 +502,15 @@ int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, 
   // the array keeps whatever the previous call (of any cache) left: tickets and the error word must start at zero
   if (cudaMemsetAsync(scratch + c->L.ws_ticket_off, 0, (size_t)(c->L.U + 8) * 4, s) != cudaSuccess) return INNERQ_ERR_CUDA;
   int n = -2;
+  bool fused = false;
   if (c->opt_variant != 1 && c->L.k.kind == kNone)
     n = launch_decode_fp16(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
-  else if (c->opt_variant != 1 && decode_mma_supported(c->L))
+  else if (c->opt_variant != 1 && decode_mma_supported(c->L)) {
     n = launch_decode_mma(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                           c->opt_splits, s, 1, nullptr, c->N_safe);
+    fused = n >= 0;
+  }
   if (n == -2) {
     if (c->opt_variant == 2) return INNERQ_ERR_UNSUPPORTED;
     n = launch_decode_simt(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
@@ -498,6 +518,7 @@ int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, 
   }
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N_safe = c->N;
+  c->reads_settled = fused ? 1 : 0;
   c->launches[2] = n;
   return INNERQ_OK;
 }

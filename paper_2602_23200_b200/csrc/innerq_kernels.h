@@ -37,7 +37,7 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
 int launch_quantize_store_prefill(const Layout& L, const Store& S, const __half* X, int N, int n_q, unsigned char* cache,
                                   const float* inv_norm, cudaStream_t st);
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
-                  cudaStream_t st);
+                  cudaStream_t st, int late_wait = 0);
 int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st);
 
 // Generic SIMT decode (any store kinds, bits, group sizes): split kernel + merge kernel.
@@ -51,8 +51,8 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
 int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const* caches, unsigned char* const* wss,
                               const int* Ns, const int* Ns_safe, const __half* q, __half* out, int n_splits,
                               cudaStream_t st);
-int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const __half* k_new,
-                          const __half* v_new, cudaStream_t st);
+int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const int* late_wait,
+                          const __half* k_new, const __half* v_new, cudaStream_t st);
 bool decode_mma_supported(const Layout& L);
 
 // Warp-MMA decode over an unquantised fp16 cache (grouping = FP16).  Returns -2 for other layouts.

@@ -281,24 +281,30 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
   append_evict_block(L, L.v, N, u, cache, false, tile, words);
 }
 
+// Programmatic dependent launch: the decode that follows may start while this kernel runs (it streams what this
+// kernel cannot write and waits for this kernel's completion before it touches the rest).  This kernel in turn
+// waits for the kernels before it, either before its first global access or, with late_wait (the host knows that
+// the last kernel on this cache was a fused decode, which lets its dependents start only after its last read of
+// the cache), after its work: it then runs during that decode's merge, and still completes after it, so that
+// whatever follows sees both finished.
 __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
                                                      const __half* __restrict__ v_new, int N,
-                                                     unsigned char* __restrict__ cache) {
+                                                     unsigned char* __restrict__ cache, int late_wait) {
   __shared__ __align__(16) __half tile[128 * kD];
   __shared__ uint32_t words[4 * 512];
   const int u = blockIdx.x;
-  // Programmatic dependent launch: the decode that follows may set itself up while this kernel runs (it waits
-  // for this kernel's completion before its first global access); this kernel in turn waits for its predecessor.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
   append_unit(L, k_new + (size_t)u * kD, v_new + (size_t)u * kD, N, u, cache, tile, words);
+  if (late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // The same for several caches of one configuration, each with its own token count: block x = sequence * U + unit,
 // k_new / v_new are [n][U][D].
 struct AppendSeq {
   unsigned char* cache;
-  int N;       // token count after this append
+  int N;           // token count after this append
+  int late_wait;   // as for append_kernel
 };
 struct AppendTable {
   AppendSeq s[kMaxSeqs];
@@ -311,8 +317,10 @@ __global__ void __launch_bounds__(128) append_batched_kernel(const __grid_consta
   __shared__ uint32_t words[4 * 512];
   const int seq = blockIdx.x / L.U, u = blockIdx.x - seq * L.U;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int late_wait = T.s[seq].late_wait;
+  if (!late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
   append_unit(L, k_new + (size_t)blockIdx.x * kD, v_new + (size_t)blockIdx.x * kD, T.s[seq].N, u, T.s[seq].cache, tile, words);
+  if (late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ------------------------------------------------------------------ canonical export
@@ -430,23 +438,24 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
 }
 
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
-                  cudaStream_t st) {
+                  cudaStream_t st, int late_wait) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, append_kernel, L, k_new, v_new, N_after, cache) == cudaSuccess ? 1 : -1;
+  return cudaLaunchKernelEx(&cfg, append_kernel, L, k_new, v_new, N_after, cache, late_wait) == cudaSuccess ? 1 : -1;
 }
 
-int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const __half* k_new,
-                          const __half* v_new, cudaStream_t st) {
+int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, const int* Ns_after, const int* late_wait,
+                          const __half* k_new, const __half* v_new, cudaStream_t st) {
   if (n < 1 || n > kMaxSeqs) return -1;
   AppendTable T;
   for (int i = 0; i < kMaxSeqs; ++i) {
     T.s[i].cache = caches[i < n ? i : 0];
     T.s[i].N = Ns_after[i < n ? i : 0];
+    T.s[i].late_wait = late_wait[i < n ? i : 0];
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n * L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
