@@ -532,8 +532,10 @@ def run_ours(args, w):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
                          "note": "achieved is from decodes bracketed by their own events (every 8th step), which "
-                                 "cannot overlap their neighbours; back to back the same kernel averages "
-                                 "us_per_decode_back_to_back",
+                                 "cannot overlap their neighbours; in the timed loop consecutive kernels overlap "
+                                 "(a whole step, append included, takes us_per_step: frac_of_step); back to back "
+                                 "the decode kernel averages us_per_decode_back_to_back",
+                         "frac_of_step": value_gbs / world / peak,
                          "achieved_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9,
                          "frac_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9 / peak,
                          "kernel": "innerq_decode_attention (split + merge)"},
