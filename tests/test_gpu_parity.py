@@ -455,6 +455,66 @@ def test_steps_enqueued_back_to_back_without_host_synchronisation(grouping, r, G
     assert gc.innerq_read_device_error() == 0
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_interleaving_of_calls_on_one_stream(seed):
+    # Three caches of different formats share one stream; appends, decodes (fused and plain kernels), multi-query
+    # decodes and exports are enqueued in random order with no host synchronisation except at exports.  Every output is
+    # checked afterwards: the overlap of consecutive kernels must never let a decode miss an append.
+    torch = _torch()
+    rng = np.random.default_rng(seed)
+    specs = [dict(n_q_heads=4, n_kv_heads=4, group=32, k_bits=2, v_bits=2, w_recent=16),
+             dict(n_q_heads=8, n_kv_heads=2, group=64, k_bits=4, v_bits=4, w_recent=24),
+             dict(n_q_heads=4, n_kv_heads=2, group=32, k_bits=2, v_bits=2, w_recent=16, grouping=O.OUTER, k_normalize=0,
+                  k_mode=O.ASYM, v_mode=O.ASYM)]
+    ws, ocs, gcs, steps = [], [], [], []
+    pool = 160                                     # inputs are put on the device up front: no copy between the calls
+    toks, qs, toks_d, qs_d = [], [], [], []
+    for i, kw in enumerate(specs):
+        w = synth.tiny(batch=1, n_tokens=4 + kw["w_recent"] + 60 * 32 + 5 * i, wid=500 + 10 * seed + i, **kw)
+        oc, gc, _, _ = run_prefill_both(w, max_tokens=w.n_tokens + pool + 8)
+        ws.append(w); ocs.append(oc); gcs.append(gc); steps.append(0)
+        toks.append([synth.new_token(w, s_) for s_ in range(pool)])
+        qs.append([synth.query(w, 1000 + s_) for s_ in range(pool)])
+        toks_d.append((dev(np.stack([t[0] for t in toks[i]])), dev(np.stack([t[1] for t in toks[i]]))))
+        qs_d.append(dev(np.stack(qs[i])))
+    torch.cuda.synchronize()
+    pending = []                                   # (device output, reference) pairs, checked at the end
+    n_queries = [0] * len(gcs)
+    for it in range(260):
+        i = int(rng.integers(len(gcs)))
+        w, oc, gc = ws[i], ocs[i], gcs[i]
+        op = rng.choice(["append", "append", "decode", "decode", "plain", "multi", "export"], p=[.3, .2, .2, .1, .05, .1, .05])
+        if op == "append":
+            if steps[i] >= pool:
+                continue
+            k1, v1 = toks[i][steps[i]]
+            oc.append(k1, v1)
+            gc.innerq_append_token(toks_d[i][0][steps[i]], toks_d[i][1][steps[i]])
+            steps[i] += 1
+        elif op in ("decode", "plain"):
+            j = n_queries[i] % pool; n_queries[i] += 1
+            gc.innerq_set_decode_options(0, 1 if op == "plain" else 0)
+            pending.append((gc.innerq_decode_attention(qs_d[i][j]), oc.decode(qs[i][j]), f"{op} cache {i} op {it}"))
+            gc.innerq_set_decode_options(0, 0)
+        elif op == "multi":
+            n_q = int(rng.integers(2, 5))
+            e = oc.export()
+            j = n_queries[i] % (pool - 4); n_queries[i] += n_q
+            if oc.N - e["n_sink"] - min(e["n_qk"], e["n_qv"]) < n_q - 1:
+                continue
+            q = np.stack(qs[i][j:j + n_q], axis=1)                                   # [1, n_q, Hq, D]
+            qd = qs_d[i][j:j + n_q].transpose(0, 1).contiguous()
+            pending.append((gc.innerq_decode_attention_multi(qd), oc.decode_multi(q), f"multi cache {i} op {it}"))
+        else:
+            P.assert_export_equal(gc.innerq_cache_export(), oc.export(), w.grouping, w.group,
+                                  k_hybrid=w.k_mode == O.HYBRID, v_hybrid=w.v_mode == O.HYBRID)
+    torch.cuda.synchronize()
+    for out, ref, what in pending:
+        P.assert_outputs_close(out.cpu().numpy(), ref, what)
+    for i, gc in enumerate(gcs):
+        assert gc.n_tokens == ocs[i].N and gc.innerq_read_device_error() == 0
+
+
 def test_capacity_and_argument_errors():
     from paper_2602_23200_b200 import binding as B
     torch = _torch()
