@@ -374,6 +374,29 @@ def test_batched_calls_over_sequences_of_different_lengths(grouping, r, G, bits)
     P.assert_outputs_close(gcs[4].innerq_decode_attention(dev(q)).cpu().numpy(), ocs[4].decode(q), "single after batched")
 
 
+def test_batched_calls_with_caches_that_hold_a_batch_themselves():
+    # every cache object may itself hold several sequences of one length: rows of k_new / q are [cache][batch, ...]
+    from paper_2602_23200_b200 import binding as B
+    base = synth.tiny(batch=3, n_q_heads=4, n_kv_heads=2, group=64)
+    ws, ocs, gcs = [], [], []
+    for i, n in enumerate([90, 333, 200]):
+        w = base.with_(n_tokens=n, wid=base.wid + 700 + i)
+        oc, gc, _, _ = run_prefill_both(w, max_tokens=500)
+        ws.append(w); ocs.append(oc); gcs.append(gc)
+    for step in range(70):
+        toks = [synth.new_token(w, step) for w in ws]
+        for (k1, v1), oc in zip(toks, ocs):
+            oc.append(k1, v1)
+        B.innerq_append_token_batched(gcs, dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks])))
+        if step in (0, 63, 64, 69):
+            q = np.stack([synth.query(w, step) for w in ws])                     # [3, batch, Hq, D]
+            out = B.innerq_decode_attention_batched(gcs, dev(q)).cpu().numpy()
+            for i in range(3):
+                P.assert_outputs_close(out[i], ocs[i].decode(q[i]), f"cache {i} step {step}")
+    for w, oc, gc in zip(ws, ocs, gcs):
+        P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
+
+
 def test_batched_calls_argument_checks():
     from paper_2602_23200_b200 import binding as B
     w = synth.tiny(batch=1, n_q_heads=2, n_kv_heads=2, n_tokens=50)
