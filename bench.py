@@ -332,6 +332,18 @@ def run_ours(args, w):
                 c.innerq_quantize_prefill(Kd[i:i + 1, :, :n_i].contiguous(), Vd[i:i + 1, :, :n_i].contiguous())
                 cs.append(c)
             ragged_sets.append(cs)
+    # the same caches with their packed records in pages of a shared pool, pages handed out in a shuffled order
+    # (information: what the page table costs the decode kernel)
+    paged_caches = []
+    if args.paged and w.grouping != synth.FP16:
+        per_cache = -(-cfg.max_tokens // args.paged) + 1
+        order = np.random.default_rng(5).permutation(R * per_cache)
+        pool = B.PagePool(cfg, args.paged, R * per_cache, order=order)
+        for _ in range(R):
+            c = B.InnerQCache(cfg, pool=pool)
+            c.ensure_pages(w.n_tokens)
+            c.innerq_quantize_prefill(Kd, Vd)
+            paged_caches.append(c)
     del Kd, Vd, Kh, Vh, ex
     torch.cuda.empty_cache()
 
@@ -435,6 +447,20 @@ def run_ours(args, w):
     b1.record(stream)
     torch.cuda.synchronize()
     b2b_us = b0.elapsed_time(b1) / nb * 1e3
+    paged = None
+    if paged_caches:
+        for c in paged_caches:
+            c.innerq_decode_attention(q_all[0], out)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        p0.record(stream)
+        for i in range(nb):
+            paged_caches[i % R].innerq_decode_attention(q_all[i % len(qs)], out)
+        p1.record(stream)
+        torch.cuda.synchronize()
+        paged = {"page_tokens": args.paged, "pages_per_cache": paged_caches[0].pages_assigned,
+                 "page_bytes": pool.page_bytes, "us_per_decode_back_to_back": p0.elapsed_time(p1) / nb * 1e3,
+                 "contiguous_us_per_decode_back_to_back": b2b_us}
     # the append kernel alone, each call between its own events (extra tokens beyond the timed steps)
     app_n = 16
     app_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(app_n)]
@@ -527,7 +553,7 @@ def run_ours(args, w):
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
             "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
             "second_roof": pipe_roofs_gbs(stored_counters(w.name), bytes_min / Kst, clocks.get("sm_mhz")),
-            "step_us_by_kind": step_split, "multi_query": multi, "ragged_batch": ragged,
+            "step_us_by_kind": step_split, "multi_query": multi, "ragged_batch": ragged, "paged_cache": paged,
             "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
@@ -569,6 +595,7 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--paged", type=int, default=1024, help="page size in tokens of the paged-cache leg (0: skip it)")
     ap.add_argument("--ragged", type=int, default=1, help="1: also time a batched decode over sequences of mixed lengths")
     ap.add_argument("--n-q", type=int, default=4, help="query tokens per call of the multi-query leg (0/1: skip it)")
     args = ap.parse_args()

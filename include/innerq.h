@@ -104,6 +104,50 @@ int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cach
 /* Frees the host handle only. */
 int innerq_cache_destroy(innerq_cache_t* cache);
 
+/* ---- Paged caches -------------------------------------------------------------------------------------
+ * The packed part of a cache (codes and scale / zero-point words of the quantised middle, which is what grows
+ * with the context; Section "High-precision Window" keeps the rest in two fixed-size fp16 windows) can live in
+ * pages of `page_tokens` tokens drawn from a pool that many caches share, instead of inside the cache buffer.
+ * page_tokens is a power of two, at least 128 (so a page holds whole groups for every G); a page holds those tokens of all
+ * batch * n_kv_heads units of the cache.  The cache buffer then holds only the norms, the fp16 windows and a page
+ * table; the pool is one caller-owned device buffer of pool_pages * page_bytes bytes, 256-byte aligned, and a page
+ * is named by its index in it.  The caller decides which page goes to which cache (free list, eviction, reuse);
+ * the library checks indices against pool_pages and against the cache's own pages, not across caches.
+ * Kernels, results and every other entry point are the same as for a contiguous cache; batched calls need caches
+ * on one pool.  Not available for grouping FP16 (UNSUPPORTED) or with the tcgen05 kernel variant. */
+
+/* Sizes for a paged cache: bytes of the cache buffer and the workspace, bytes of one page, and the most page slots
+ * a cache can use (max_tokens tokens).  Host pointers.  Errors: INVALID_ARG (page_tokens), UNSUPPORTED. */
+int innerq_paged_cache_bytes(const innerq_config_t* cfg, int32_t page_tokens, size_t* cache_bytes,
+                             size_t* workspace_bytes, size_t* page_bytes, int32_t* max_pages);
+
+/* As innerq_cache_create, over the page pool `dev_pool` of `pool_pages` pages.  The cache starts with no pages. */
+int innerq_cache_create_paged(const innerq_config_t* cfg, int32_t page_tokens, void* dev_cache, size_t cache_bytes,
+                              void* dev_workspace, size_t workspace_bytes, void* dev_pool, int32_t pool_pages,
+                              void* cuda_stream, innerq_cache_t** out);
+
+/* Page slots that the cache needs to hold n_tokens tokens (0 for a contiguous cache), or a negative error code.
+ * A prefill to n tokens or an append that makes N = n returns INNERQ_ERR_CAPACITY unless at least this many
+ * pages are assigned. */
+int innerq_cache_pages_for(const innerq_cache_t* cache, int32_t n_tokens);
+
+/* Pages assigned so far, or a negative error code. */
+int innerq_cache_pages_assigned(const innerq_cache_t* cache);
+
+/* Gives the cache `n` more pages: page slots [assigned, assigned + n) map to pool pages pages_host[0..n) (HOST
+ * array; read before the call returns).  Enqueues the copy of the new table entries on `cuda_stream` (the
+ * stream of the cache's other calls); the pages' old contents are dead from then on.  Pages may be assigned any
+ * time before the call that needs them; assigning them a few steps early keeps the copy out of the step that
+ * crosses the page boundary.  Errors: INVALID_ARG (contiguous cache, index out of range or already in this
+ * cache), CAPACITY (more than max_pages), CUDA. */
+int innerq_cache_assign_pages(innerq_cache_t* cache, const int32_t* pages_host, int32_t n, void* cuda_stream);
+
+/* Empties the cache (N = 0) and hands its pages back: writes their pool indices to pages_host[0..count) (HOST
+ * array of `capacity` entries) and returns count, or a negative error code (BUFFER_TOO_SMALL leaves the cache as
+ * it was).  Host-side only: kernels already enqueued for this cache still read the pages, so the caller may give
+ * them to another cache only on the same stream (or after synchronising). */
+int innerq_cache_release_pages(innerq_cache_t* cache, int32_t* pages_host, int32_t capacity);
+
 /* Number of tokens currently cached (host value), or a negative error code. */
 int innerq_cache_n_tokens(const innerq_cache_t* cache);
 

@@ -25,6 +25,8 @@ EXPORTED_SYMBOLS = (
     "innerq_decode_attention_static", "innerq_decode_step_host", "innerq_step_staging_bytes",
     "innerq_decode_attention_multi", "innerq_multi_query_scratch_bytes",
     "innerq_append_token_batched", "innerq_decode_attention_batched",
+    "innerq_paged_cache_bytes", "innerq_cache_create_paged", "innerq_cache_pages_for", "innerq_cache_pages_assigned",
+    "innerq_cache_assign_pages", "innerq_cache_release_pages",
     "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
@@ -78,6 +80,12 @@ def lib() -> C.CDLL:
     L.innerq_multi_query_scratch_bytes.argtypes = [cfgp, C.POINTER(sz)]
     L.innerq_append_token_batched.argtypes = [C.POINTER(vp), i32, vp, vp, vp]
     L.innerq_decode_attention_batched.argtypes = [C.POINTER(vp), i32, vp, vp, vp]
+    L.innerq_paged_cache_bytes.argtypes = [cfgp, i32, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz), C.POINTER(i32)]
+    L.innerq_cache_create_paged.argtypes = [cfgp, i32, vp, sz, vp, sz, vp, i32, vp, C.POINTER(vp)]
+    L.innerq_cache_pages_for.argtypes = [vp, i32]
+    L.innerq_cache_pages_assigned.argtypes = [vp]
+    L.innerq_cache_assign_pages.argtypes = [vp, C.POINTER(i32), i32, vp]
+    L.innerq_cache_release_pages.argtypes = [vp, C.POINTER(i32), i32]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
@@ -129,6 +137,38 @@ def innerq_token_payload_bytes(cfg: innerq_config_t):
     kb, vb = C.c_double(), C.c_double()
     _check(lib().innerq_token_payload_bytes(C.byref(cfg), C.byref(kb), C.byref(vb)), "innerq_token_payload_bytes")
     return kb.value, vb.value
+
+
+def innerq_paged_cache_bytes(cfg: innerq_config_t, page_tokens: int):
+    """(cache_bytes, workspace_bytes, page_bytes, max_pages) of a paged cache."""
+    cb, wb, pb, mp = C.c_size_t(), C.c_size_t(), C.c_size_t(), C.c_int32()
+    _check(lib().innerq_paged_cache_bytes(C.byref(cfg), int(page_tokens), C.byref(cb), C.byref(wb), C.byref(pb), C.byref(mp)),
+           "innerq_paged_cache_bytes")
+    return cb.value, wb.value, pb.value, mp.value
+
+
+class PagePool:
+    """A pool of cache pages in one torch device buffer, with the free list a caller of the C ABI keeps itself.
+    `order` (a permutation of range(n_pages)) sets the order in which free pages are handed out."""
+
+    def __init__(self, cfg: innerq_config_t, page_tokens: int, n_pages: int, device=None, order=None):
+        import torch
+        self.cfg, self.page_tokens, self.n_pages = cfg, int(page_tokens), int(n_pages)
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.page_bytes = innerq_paged_cache_bytes(cfg, page_tokens)[2]
+        self.buf = torch.empty(self.n_pages * self.page_bytes, dtype=torch.uint8, device=self.device)
+        self.free = list(range(self.n_pages)) if order is None else [int(i) for i in order]
+        if sorted(self.free) != list(range(self.n_pages)):
+            raise ValueError("order must be a permutation of range(n_pages)")
+
+    def take(self, n: int):
+        if n > len(self.free):
+            raise RuntimeError(f"page pool exhausted: {n} pages wanted, {len(self.free)} free")
+        out, self.free = self.free[:n], self.free[n:]
+        return out
+
+    def give_back(self, pages):
+        self.free.extend(int(i) for i in pages)
 
 
 def _stream_ptr(stream, device=None) -> int:
@@ -186,22 +226,65 @@ def innerq_decode_attention_batched(caches, q, out=None, stream=None):
 class InnerQCache:
     """A packed KV cache living in caller-side torch device buffers, driven through the C ABI."""
 
-    def __init__(self, cfg: innerq_config_t, device=None, stream=None):
+    def __init__(self, cfg: innerq_config_t, device=None, stream=None, pool: "PagePool | None" = None):
+        """pool: keep the packed part of the cache in pages of this pool (innerq_cache_create_paged) instead of inside
+        the cache's own buffer; pages are assigned with ensure_pages / innerq_cache_assign_pages."""
         import torch
         self.cfg = cfg
+        self.pool = pool
         # default: the current device (one process per GPU sets it once with torch.cuda.set_device)
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         if self.device.index is None:
             self.device = torch.device("cuda", torch.cuda.current_device())
-        cb, wb = innerq_cache_bytes(cfg)
+        if pool is not None and pool.device != self.device:
+            raise ValueError(f"the pool is on {pool.device}, the cache on {self.device}")
+        cb, wb = innerq_cache_bytes(cfg) if pool is None else innerq_paged_cache_bytes(cfg, pool.page_tokens)[:2]
         self.cache_bytes, self.workspace_bytes = cb, wb
         with torch.cuda.device(self.device):
             self._cache_buf = torch.empty(cb, dtype=torch.uint8, device=self.device)
             self._ws_buf = torch.empty(wb, dtype=torch.uint8, device=self.device)
             h = C.c_void_p()
-            _check(lib().innerq_cache_create(C.byref(cfg), self._cache_buf.data_ptr(), cb, self._ws_buf.data_ptr(), wb,
-                                             _stream_ptr(stream, self.device), C.byref(h)), "innerq_cache_create")
+            if pool is None:
+                _check(lib().innerq_cache_create(C.byref(cfg), self._cache_buf.data_ptr(), cb, self._ws_buf.data_ptr(), wb,
+                                                 _stream_ptr(stream, self.device), C.byref(h)), "innerq_cache_create")
+            else:
+                _check(lib().innerq_cache_create_paged(C.byref(cfg), pool.page_tokens, self._cache_buf.data_ptr(), cb,
+                                                       self._ws_buf.data_ptr(), wb, pool.buf.data_ptr(), pool.n_pages,
+                                                       _stream_ptr(stream, self.device), C.byref(h)),
+                       "innerq_cache_create_paged")
         self._h = h
+
+    # ---- paged caches
+    def innerq_cache_pages_for(self, n_tokens: int) -> int:
+        return _check(lib().innerq_cache_pages_for(self._h, int(n_tokens)), "innerq_cache_pages_for")
+
+    @property
+    def pages_assigned(self) -> int:
+        return _check(lib().innerq_cache_pages_assigned(self._h), "innerq_cache_pages_assigned")
+
+    def innerq_cache_assign_pages(self, pages, stream=None):
+        arr = (C.c_int32 * len(pages))(*[int(i) for i in pages])
+        _check(lib().innerq_cache_assign_pages(self._h, arr, len(pages), _stream_ptr(stream, self.device)),
+               "innerq_cache_assign_pages")
+
+    def innerq_cache_release_pages(self):
+        """Empties the cache and returns the pool indices of the pages it held."""
+        n = self.pages_assigned
+        arr = (C.c_int32 * max(n, 1))()
+        got = _check(lib().innerq_cache_release_pages(self._h, arr, n), "innerq_cache_release_pages")
+        return [int(arr[i]) for i in range(got)]
+
+    def ensure_pages(self, n_tokens: int, stream=None):
+        """Takes from the pool's free list whatever the cache still lacks to hold n_tokens tokens."""
+        if self.pool is None:
+            return
+        lack = self.innerq_cache_pages_for(n_tokens) - self.pages_assigned
+        if lack > 0:
+            self.innerq_cache_assign_pages(self.pool.take(lack), stream)
+
+    def release_to_pool(self):
+        if self.pool is not None:
+            self.pool.give_back(self.innerq_cache_release_pages())
 
     def close(self):
         h, self._h = getattr(self, "_h", None), None

@@ -3,6 +3,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "../../include/innerq.h"
 #include "innerq_kernels.h"
@@ -21,6 +22,8 @@ struct innerq_cache {
                        // has read everything it reads from the cache (an append can then run without waiting first)
   int opt_splits, opt_variant;
   int launches[3];
+  int pool_pages;                 // paged cache: pages in the pool (page ids are checked against it)
+  std::vector<uint32_t> pages;    // paged cache: pool page of every assigned page slot (host copy of the device table)
 };
 
 namespace {
@@ -62,7 +65,9 @@ void place_store(Store& S, int kind, int bits, int mode, const innerq_config_t& 
   const int G = c.group;
   int mid = c.max_tokens - c.w_sink - c.w_recent;
   if (mid < 1) mid = 1;
-  S.cap_q = (int)align_up((size_t)mid, kTile);
+  // one chunk to spare: the decode kernel's copies take two chunks at a time and may read (never use) the one behind
+  // the last packed token
+  S.cap_q = (int)align_up((size_t)mid + kChunk, kTile);
   S.ring_cap = kind == kRow ? c.w_recent + 1 : c.w_recent + G;
   S.n_groups = kind == kRow ? kD / G : kD;
   S.meta_bytes = mode == INNERQ_MODE_SYM ? 2 : 4;
@@ -73,7 +78,7 @@ void place_store(Store& S, int kind, int bits, int mode, const innerq_config_t& 
 }
 
 // Geometry of the shared record area of a ROW store and a BLOCK store (see struct Store).
-void place_records(Store& row, Store& blk, int G, int U, size_t& off) {
+void place_records(Store& row, Store& blk, int G, int U, size_t& off, int page_groups) {
   const int row_codes = kChunk * row_bytes(row.bits);
   const int row_meta = kChunk * row.n_groups * row.meta_bytes;
   const int blk_codes = chunk_bytes(blk.bits);
@@ -81,7 +86,7 @@ void place_records(Store& row, Store& blk, int G, int U, size_t& off) {
   const int chunk_stride = row_codes + row_meta + blk_codes;
   const int cpg = G / kChunk;
   const int group_stride = cpg * chunk_stride + blk_meta;
-  const size_t unit = align_up((size_t)(row.cap_q / G) * group_stride, 256);
+  const size_t unit = page_groups > 0 ? (size_t)page_groups * group_stride : align_up((size_t)(row.cap_q / G) * group_stride, 256);
   Store* both[2] = {&row, &blk};
   for (Store* S : both) {
     S->rec_off = off;
@@ -94,14 +99,14 @@ void place_records(Store& row, Store& blk, int G, int U, size_t& off) {
   row.meta_in_rec = row_codes;
   blk.code_in_rec = row_codes + row_meta;
   blk.meta_in_rec = cpg * chunk_stride;
-  off = align_up(off + unit * U, 256);
+  if (page_groups == 0) off = align_up(off + unit * U, 256);
 }
 
 // Outer grouping: keys are grouped per channel along tokens (kBlock metadata) but keep one packed row per token,
 // values are grouped per token along channels (kRow metadata) but keep 32-token chunks.  A chunk record holds the
 // key rows, the values' metadata rows and the value chunk; the keys' per-group metadata comes FIRST in the group
 // record, because scores need it from the group's first token on.
-void place_records_outer(Store& k, Store& v, int G, int U, size_t& off) {
+void place_records_outer(Store& k, Store& v, int G, int U, size_t& off, int page_groups) {
   k.code_kind = kRow;
   v.code_kind = kBlock;
   const int row_codes = kChunk * row_bytes(k.bits);
@@ -111,7 +116,7 @@ void place_records_outer(Store& k, Store& v, int G, int U, size_t& off) {
   const int chunk_stride = row_codes + row_meta + blk_codes;
   const int cpg = G / kChunk;
   const int group_stride = blk_meta + cpg * chunk_stride;
-  const size_t unit = align_up((size_t)(v.cap_q / G) * group_stride, 256);
+  const size_t unit = page_groups > 0 ? (size_t)page_groups * group_stride : align_up((size_t)(v.cap_q / G) * group_stride, 256);
   Store* both[2] = {&k, &v};
   for (Store* S : both) {
     S->rec_off = off;
@@ -125,10 +130,11 @@ void place_records_outer(Store& k, Store& v, int G, int U, size_t& off) {
   k.meta_in_rec = 0;
   v.meta_in_rec = row_codes;
   v.code_in_rec = row_codes + row_meta;
-  off = align_up(off + unit * U, 256);
+  if (page_groups == 0) off = align_up(off + unit * U, 256);
 }
 
-void make_layout(const innerq_config_t& c, Layout& L) {
+// page_tokens > 0: paged record area (see struct Layout); the pool pointer is set by the caller.
+void make_layout(const innerq_config_t& c, Layout& L, int page_tokens = 0) {
   std::memset(&L, 0, sizeof(L));
   L.B = c.batch; L.Hq = c.n_q_heads; L.Hkv = c.n_kv_heads;
   L.U = c.batch * c.n_kv_heads;
@@ -151,11 +157,19 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   } else if (c.grouping == INNERQ_GROUPING_INNER) {
     place_store(L.k, kRow, c.k_bits, c.k_mode, c, L.U, off);
     place_store(L.v, kBlock, c.v_bits, c.v_mode, c, L.U, off);
-    place_records(L.k, L.v, L.G, L.U, off);
+    place_records(L.k, L.v, L.G, L.U, off, page_tokens / L.G);
   } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
     place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);
     place_store(L.v, kRow, c.v_bits, INNERQ_MODE_ASYM, c, L.U, off);
-    place_records_outer(L.k, L.v, L.G, L.U, off);
+    place_records_outer(L.k, L.v, L.G, L.U, off, page_tokens / L.G);
+  }
+  L.page_chunk_mask = page_tokens > 0 ? page_tokens / kChunk - 1 : 0x3fffffff;
+  if (page_tokens > 0) {
+    L.page_groups = page_tokens / L.G;
+    L.max_pages = (L.k.cap_q / L.G + L.page_groups - 1) / L.page_groups;
+    L.page_bytes = align_up(L.k.rec_unit_stride * L.U, 256);
+    L.page_table_off = off;
+    off = align_up(off + (size_t)L.max_pages * 4, 256);
   }
   L.cache_bytes = off;
   size_t w = 0;
@@ -163,6 +177,60 @@ void make_layout(const innerq_config_t& c, Layout& L) {
   L.ws_absmax_off = w; w = align_up(w + (size_t)L.U * kD * 4, 256);
   L.ws_ticket_off = w; w = align_up(w + (size_t)(L.U + 8) * 4, 256);   // tickets [U], then the device error word
   L.workspace_bytes = w;
+}
+
+// Page slots that a cache of N tokens uses: every group record that holds a packed key row or value chunk.
+int pages_for(const Layout& L, int N) {
+  if (L.page_groups == 0) return 0;
+  const Counts cn = counts_for(L, N);
+  const int n_rec = cn.n_qk > cn.n_qv ? cn.n_qk : cn.n_qv;
+  const int groups = (n_rec + L.G - 1) / L.G;
+  return (groups + L.page_groups - 1) / L.page_groups;
+}
+bool has_pages_for(const innerq_cache* c, int N) { return (int)c->pages.size() >= pages_for(c->L, N); }
+
+int create_cache(const innerq_config_t* cfg, int page_tokens, void* dev_cache, size_t cache_bytes, void* dev_workspace,
+                 size_t workspace_bytes, void* dev_pool, int pool_pages, void* cuda_stream, innerq_cache_t** out) {
+  int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  if (!dev_cache || !dev_workspace || !out) return INNERQ_ERR_INVALID_ARG;
+  if (((uintptr_t)dev_cache & 255u) || ((uintptr_t)dev_workspace & 255u)) return INNERQ_ERR_INVALID_ARG;
+  innerq_cache* c = new (std::nothrow) innerq_cache();
+  if (!c) return INNERQ_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  make_layout(*cfg, c->L, page_tokens);
+  c->L.pool = static_cast<unsigned char*>(dev_pool);
+  c->pool_pages = pool_pages;
+  if (cache_bytes < c->L.cache_bytes || workspace_bytes < c->L.workspace_bytes) {
+    delete c;
+    return INNERQ_ERR_BUFFER_TOO_SMALL;
+  }
+  c->cache = static_cast<unsigned char*>(dev_cache);
+  c->ws = static_cast<unsigned char*>(dev_workspace);
+  c->N = 0;
+  c->N_safe = 0;
+  c->reads_settled = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(c->cache, 0, c->L.cache_bytes, s) != cudaSuccess ||
+      cudaMemsetAsync(c->ws, 0, c->L.workspace_bytes, s) != cudaSuccess) {
+    delete c;
+    return INNERQ_ERR_CUDA;
+  }
+  // norm = 1 until a prefill computes it
+  if (launch_prefill(c->L, c->cache, c->ws, nullptr, nullptr, 0, s) < 0) {
+    delete c;
+    return INNERQ_ERR_CUDA;
+  }
+  *out = c;
+  return INNERQ_OK;
+}
+
+int check_page_tokens(const innerq_config_t* cfg, int page_tokens) {
+  int st = check_config(cfg);
+  if (st != INNERQ_OK) return st;
+  if (page_tokens < kTile || (page_tokens & (page_tokens - 1)) != 0) return INNERQ_ERR_INVALID_ARG;
+  if (cfg->grouping == INNERQ_GROUPING_FP16) return INNERQ_ERR_UNSUPPORTED;    // only packed records are paged
+  return INNERQ_OK;
 }
 
 }  // namespace
@@ -200,36 +268,82 @@ int innerq_token_payload_bytes(const innerq_config_t* cfg, double* k_bytes, doub
 
 int innerq_cache_create(const innerq_config_t* cfg, void* dev_cache, size_t cache_bytes, void* dev_workspace,
                         size_t workspace_bytes, void* cuda_stream, innerq_cache_t** out) {
-  int st = check_config(cfg);
+  return create_cache(cfg, 0, dev_cache, cache_bytes, dev_workspace, workspace_bytes, nullptr, 0, cuda_stream, out);
+}
+
+// ---- paged record area --------------------------------------------------------------------------------
+int innerq_paged_cache_bytes(const innerq_config_t* cfg, int32_t page_tokens, size_t* cache_bytes, size_t* workspace_bytes,
+                             size_t* page_bytes, int32_t* max_pages) {
+  const int st = check_page_tokens(cfg, page_tokens);
   if (st != INNERQ_OK) return st;
-  if (!dev_cache || !dev_workspace || !out) return INNERQ_ERR_INVALID_ARG;
-  if (((uintptr_t)dev_cache & 255u) || ((uintptr_t)dev_workspace & 255u)) return INNERQ_ERR_INVALID_ARG;
-  innerq_cache* c = new (std::nothrow) innerq_cache();
-  if (!c) return INNERQ_ERR_INVALID_ARG;
-  c->cfg = *cfg;
-  make_layout(*cfg, c->L);
-  if (cache_bytes < c->L.cache_bytes || workspace_bytes < c->L.workspace_bytes) {
-    delete c;
-    return INNERQ_ERR_BUFFER_TOO_SMALL;
+  if (!cache_bytes || !workspace_bytes || !page_bytes || !max_pages) return INNERQ_ERR_INVALID_ARG;
+  Layout L;
+  make_layout(*cfg, L, page_tokens);
+  *cache_bytes = L.cache_bytes;
+  *workspace_bytes = L.workspace_bytes;
+  *page_bytes = L.page_bytes;
+  *max_pages = L.max_pages;
+  return INNERQ_OK;
+}
+
+int innerq_cache_create_paged(const innerq_config_t* cfg, int32_t page_tokens, void* dev_cache, size_t cache_bytes,
+                              void* dev_workspace, size_t workspace_bytes, void* dev_pool, int32_t pool_pages,
+                              void* cuda_stream, innerq_cache_t** out) {
+  const int st = check_page_tokens(cfg, page_tokens);
+  if (st != INNERQ_OK) return st;
+  if (!dev_pool || ((uintptr_t)dev_pool & 255u) || pool_pages < 1) return INNERQ_ERR_INVALID_ARG;
+  return create_cache(cfg, page_tokens, dev_cache, cache_bytes, dev_workspace, workspace_bytes, dev_pool, pool_pages,
+                      cuda_stream, out);
+}
+
+int innerq_cache_pages_for(const innerq_cache_t* c, int32_t n_tokens) {
+  if (!c || n_tokens < 0) return INNERQ_ERR_INVALID_ARG;
+  if (n_tokens > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  return pages_for(c->L, n_tokens);
+}
+
+int innerq_cache_pages_assigned(const innerq_cache_t* c) { return c ? (int)c->pages.size() : INNERQ_ERR_INVALID_ARG; }
+
+int innerq_cache_assign_pages(innerq_cache_t* c, const int32_t* pages_host, int32_t n, void* cuda_stream) {
+  if (!c || !pages_host || n < 1 || c->L.page_groups == 0) return INNERQ_ERR_INVALID_ARG;
+  const size_t have = c->pages.size();
+  if (have + (size_t)n > (size_t)c->L.max_pages) return INNERQ_ERR_CAPACITY;
+  for (int i = 0; i < n; ++i) {
+    if (pages_host[i] < 0 || pages_host[i] >= c->pool_pages) return INNERQ_ERR_INVALID_ARG;
+    for (size_t j = 0; j < have; ++j)
+      if (c->pages[j] == (uint32_t)pages_host[i]) return INNERQ_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (pages_host[j] == pages_host[i]) return INNERQ_ERR_INVALID_ARG;
   }
-  c->cache = static_cast<unsigned char*>(dev_cache);
-  c->ws = static_cast<unsigned char*>(dev_workspace);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (c->L.k.code_kind != c->L.k.kind) {
+    // outer grouping fills chunk words token by token with OR: its pages start from zero
+    for (int i = 0; i < n; ++i)
+      if (cudaMemsetAsync(c->L.pool + (size_t)pages_host[i] * c->L.page_bytes, 0, c->L.page_bytes, s) != cudaSuccess)
+        return INNERQ_ERR_CUDA;
+  }
+  c->pages.reserve(c->L.max_pages);        // the copy below reads the vector's storage: it must not move later
+  for (int i = 0; i < n; ++i) c->pages.push_back((uint32_t)pages_host[i]);
+  // a copy is ordered after every kernel before it in the stream and before every kernel after it, whatever their
+  // launch attributes: no kernel ever sees a table entry half-way
+  if (cudaMemcpyAsync(c->cache + c->L.page_table_off + have * 4, c->pages.data() + have, (size_t)n * 4,
+                      cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    c->pages.resize(have);
+    return INNERQ_ERR_CUDA;
+  }
+  return INNERQ_OK;
+}
+
+int innerq_cache_release_pages(innerq_cache_t* c, int32_t* pages_host, int32_t capacity) {
+  if (!c || c->L.page_groups == 0 || capacity < 0 || (capacity > 0 && !pages_host)) return INNERQ_ERR_INVALID_ARG;
+  const int n = (int)c->pages.size();
+  if (capacity < n) return INNERQ_ERR_BUFFER_TOO_SMALL;
+  for (int i = 0; i < n; ++i) pages_host[i] = (int32_t)c->pages[i];
+  c->pages.clear();
   c->N = 0;
   c->N_safe = 0;
   c->reads_settled = 0;
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  if (cudaMemsetAsync(c->cache, 0, c->L.cache_bytes, s) != cudaSuccess ||
-      cudaMemsetAsync(c->ws, 0, c->L.workspace_bytes, s) != cudaSuccess) {
-    delete c;
-    return INNERQ_ERR_CUDA;
-  }
-  // norm = 1 until a prefill computes it
-  if (launch_prefill(c->L, c->cache, c->ws, nullptr, nullptr, 0, s) < 0) {
-    delete c;
-    return INNERQ_ERR_CUDA;
-  }
-  *out = c;
-  return INNERQ_OK;
+  return n;
 }
 
 int innerq_cache_destroy(innerq_cache_t* cache) {
@@ -242,7 +356,7 @@ int innerq_cache_n_tokens(const innerq_cache_t* cache) { return cache ? cache->N
 
 int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int32_t n_tokens, void* cuda_stream) {
   if (!c || n_tokens < 0 || (n_tokens > 0 && (!k || !v))) return INNERQ_ERR_INVALID_ARG;
-  if (n_tokens > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  if (n_tokens > c->L.max_tokens || !has_pages_for(c, n_tokens)) return INNERQ_ERR_CAPACITY;
   int n = launch_prefill(c->L, c->cache, c->ws, static_cast<const __half*>(k), static_cast<const __half*>(v), n_tokens,
                          static_cast<cudaStream_t>(cuda_stream));
   if (n < 0) return INNERQ_ERR_CUDA;
@@ -255,7 +369,7 @@ int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int
 
 int innerq_append_token(innerq_cache_t* c, const void* k_new, const void* v_new, void* cuda_stream) {
   if (!c || !k_new || !v_new) return INNERQ_ERR_INVALID_ARG;
-  if (c->N + 1 > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  if (c->N + 1 > c->L.max_tokens || !has_pages_for(c, c->N + 1)) return INNERQ_ERR_CAPACITY;
   int n = launch_append(c->L, c->cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new), c->N + 1,
                         static_cast<cudaStream_t>(cuda_stream), c->reads_settled);
   if (n < 0) return INNERQ_ERR_CUDA;
@@ -347,7 +461,7 @@ int innerq_append_token_batched(innerq_cache_t* const* caches, int32_t n, const 
   for (int i = 0; i < n; ++i) {
     for (int j = 0; j < i; ++j)
       if (caches[j] == caches[i]) return INNERQ_ERR_INVALID_ARG;      // one token per cache and call
-    if (caches[i]->N + 1 > caches[i]->L.max_tokens) return INNERQ_ERR_CAPACITY;
+    if (caches[i]->N + 1 > caches[i]->L.max_tokens || !has_pages_for(caches[i], caches[i]->N + 1)) return INNERQ_ERR_CAPACITY;
   }
   const Layout& L = caches[0]->L;
   const size_t row = (size_t)L.U * kD;                                 // fp16 elements per cache in k_new / v_new
@@ -427,7 +541,7 @@ int innerq_step_staging_bytes(const innerq_config_t* cfg, size_t* bytes) {
 int innerq_decode_step_host(innerq_cache_t* c, const void* k_new_host, const void* v_new_host, const void* q_host,
                             void* out_host, void* dev_staging, void* cuda_stream) {
   if (!c || !k_new_host || !v_new_host || !q_host || !out_host || !dev_staging) return INNERQ_ERR_INVALID_ARG;
-  if (c->N + 1 > c->L.max_tokens) return INNERQ_ERR_CAPACITY;
+  if (c->N + 1 > c->L.max_tokens || !has_pages_for(c, c->N + 1)) return INNERQ_ERR_CAPACITY;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const size_t kv_bytes = (size_t)c->L.U * kD * 2, q_bytes = (size_t)c->L.B * c->L.Hq * kD * 2;
   unsigned char* d = static_cast<unsigned char*>(dev_staging);

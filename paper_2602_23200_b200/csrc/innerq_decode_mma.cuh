@@ -245,7 +245,7 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 // metadata, which leads the group record), for values p_t * S_{t,g} (one operand set per channel group the
 // m-tile's rows fall into); zero-points contribute sum_c q''_c Z_jc per group and sum_t p_t Z_{t,g} per channel
 // group.  One chunk per iteration, four heads per pass.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
 __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u) {
   constexpr int KP = KB == 3 ? 2 : KB, VP = VB == 3 ? 2 : VB;     // bits of the primary code plane
   using F = Fmt<KP>;
@@ -312,11 +312,17 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
   unsigned char* ring = smem + (size_t)warp * SL::kWarpBytes;
   uint32_t* side = reinterpret_cast<uint32_t*>(smem + SL::kOffSide + (size_t)warp * SL::kSideBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
-  const unsigned char* g_rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
   const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
+  // Group record g of this unit (a paged cache looks the group's page up in the cache's page table).
+  auto group_rec = [&](int g) -> const unsigned char* {
+    if constexpr (PAGED) return group_ptr(unit_rec(L, a.cache, u), g);
+    else return a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride + (size_t)g * SL::kGroupRec;
+  };
 
   // Copies of consecutive iterations read consecutive byte ranges of the record area: keep a running source.
-  const unsigned char* nx_src = g_rec + (size_t)(c_lo / CH) * SL::kGroupRec + (size_t)(c_lo % CH) * SL::kRec;
+  // In a paged cache (PAGED) that holds inside a page (2^k chunks): the copy that starts a page is re-based, and the
+  // copy whose two chunks lie in two pages is split.
+  const unsigned char* nx_src = n_iters > 0 ? group_rec(c_lo / CH) + (size_t)(c_lo % CH) * SL::kRec : nullptr;
   int nx_ci = c_lo;
   auto issue = [&](int st) {   // one lane: arm the barrier, start the copy of the next iteration into stage st
     // the value group's scale/zero words sit right behind its last chunk
@@ -325,6 +331,19 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
                              : (CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0));
     const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
+    const int in_page = PAGED ? nx_ci & L.page_chunk_mask : 1;
+    if (in_page == 0) {
+      nx_src = group_rec(nx_ci / CH);
+    } else if (PAGED && in_page + CPI > L.page_chunk_mask + 1) {
+      // CPI = 2 with one chunk per group, first chunk at the end of a page: two copies of one group record each.
+      // A second chunk beyond this warp's range is not used (and its page may not exist): the first one again.
+      const unsigned char* second = nx_ci + 1 < c_lo + n_chunks_w ? group_rec((nx_ci + 1) / CH) : nx_src;
+      bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes / 2, bars_u32 + 8 * st);
+      bulk_g2s(ring_u32 + st * SL::kBytes + bytes / 2, second, bytes / 2, bars_u32 + 8 * st);
+      nx_src = second + bytes / 2;
+      nx_ci += CPI;
+      return;
+    }
     bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes, bars_u32 + 8 * st);
     nx_src += bytes;
     nx_ci += CPI;
@@ -689,8 +708,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       float sA, sB;                                            // true log2-domain scores of entries e0+gid, e0+gid+8
       if (skew && !OUTER) {
         const int iq = cn.n_qv + e0;                           // first packed key row of the tile (16-aligned)
-        const unsigned char* rec = g_rec + (size_t)((iq / kChunk) / CH) * SL::kGroupRec +
-                                   (size_t)((iq / kChunk) % CH) * SL::kRec;
+        const unsigned char* rec = group_rec((iq / kChunk) / CH) + (size_t)((iq / kChunk) % CH) * SL::kRec;
         k_mtile(reinterpret_cast<const uint32_t*>(rec), reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta),
                 iq % kChunk, sA, sB);
         sA *= kfac;
@@ -750,7 +768,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       if (OUTER && skew) {
         // values of the skew zone are packed (half a chunk: one k-step of 16 tokens), read straight from global memory
         const int iq = cn.n_qk + e0, ci = iq / kChunk, ks = (iq % kChunk) / 16;
-        const unsigned char* rec = g_rec + (size_t)(ci / CH) * SL::kGroupRec + SL::kVMeta + (size_t)(ci % CH) * SL::kRec;
+        const unsigned char* rec = group_rec(ci / CH) + SL::kVMeta + (size_t)(ci % CH) * SL::kRec;
         const uint32_t* vmr = reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta);
         const uint32_t* vcg = reinterpret_cast<const uint32_t*>(rec + SL::kOffVCodes);
         uint32_t Bt[NSET][2];
@@ -1177,18 +1195,18 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
 }
 
 // One cache: block x = unit.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>(L, cn, a, blockIdx.x);
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>(L, cn, a, blockIdx.x);
 }
 // Several caches of one configuration: block x = sequence * U + unit, the sequence's counts and parameters come
 // from its table entry (read in place from the parameter space).
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_batched_kernel(const __grid_constant__ Layout L, const __grid_constant__ SeqTable T) {
   const int seq = blockIdx.x / L.U;
-  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
 }
 
 // Split-dependent launch parameters of one cache for a grid of grid_y rows (0: choose it): how many of the rows
@@ -1217,13 +1235,13 @@ int fill_split_args(const Layout& L, const Counts& cn, DecodeArgs& a, bool outer
   return grid_y;
 }
 
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
-int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
+int launch_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
   using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, kSmem, configured)) return -1;
   const int grid_y = fill_split_args<RU>(L, cn, a, OUTER, n_splits, 0);
   dim3 grid(L.U, grid_y);
   int launches = 0;
@@ -1238,7 +1256,7 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, cn, a) != cudaSuccess) return -1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -1246,13 +1264,13 @@ int launch_one(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cu
 
 // The same kernel over a table of caches.  Every sequence splits its own chunks over as many of the launch's
 // grid rows as it has work for; the rows beyond that only take their share of its tail tiles.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
-int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
+int launch_one_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
   using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, kSmem, configured)) return -1;
   // Grid rows per sequence: the fewest chunks per row T such that all sequences together, each cut into rows of at
   // most T chunks, need no more than n_splits rows in total (so the longest row, which sets the time, is as short
   // as one wave of CTAs allows, and short sequences hold few CTAs).
@@ -1291,10 +1309,23 @@ int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, c
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, T) != cudaSuccess) return -1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, T) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+// Contiguous or paged record area: two instances of every kernel, so that the contiguous one carries none of the
+// page arithmetic.
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+int launch_one(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, cudaStream_t st) {
+  return L.page_groups > 0 ? launch_one_p<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, true>(L, cn, a, n_splits, st)
+                           : launch_one_p<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false>(L, cn, a, n_splits, st);
+}
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
+  return L.page_groups > 0 ? launch_one_batched_p<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, true>(L, T, n_seqs, n_splits, st)
+                           : launch_one_batched_p<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false>(L, T, n_seqs, n_splits, st);
 }
 
 // One packed format (key bits, value bits, metadata entry bytes of each) at every group size.  cpi: chunks of 32

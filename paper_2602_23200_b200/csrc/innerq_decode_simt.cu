@@ -13,7 +13,7 @@ constexpr int kSimtTile = 32;
 struct TensorView {              // one unit's view of a store
   const __half* sink;
   const __half* ring;
-  const unsigned char* rec;
+  Rec rec;
   Store S;
   int kind, bits, ring_cap, n_groups, meta_bytes;
   int n_sink, n_q, w_sink;
@@ -24,7 +24,7 @@ __device__ __forceinline__ TensorView make_view(const Layout& L, const Store& S,
   TensorView v;
   v.sink = reinterpret_cast<const __half*>(cache + S.sink_off + (size_t)u * S.sink_stride);
   v.ring = reinterpret_cast<const __half*>(cache + S.ring_off + (size_t)u * S.ring_stride);
-  v.rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  v.rec = unit_rec(L, cache, u);
   v.S = S;
   v.meta_bytes = S.meta_bytes;
   v.kind = S.kind; v.bits = S.bits; v.ring_cap = S.ring_cap; v.n_groups = S.n_groups;
@@ -42,12 +42,12 @@ __device__ __forceinline__ float element(const TensorView& v, int G, int t, int 
   quant = true;
   float s, z;
   uint32_t code;
-  if (v.kind == kRow) decode_meta(load_meta(v.rec + row_meta_off(v.S, i), c / G, v.meta_bytes), v.bits, s, z);
-  else decode_meta(load_meta(v.rec + block_meta_off(v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
+  if (v.kind == kRow) decode_meta(load_meta(row_meta_ptr(v.rec, v.S, i), c / G, v.meta_bytes), v.bits, s, z);
+  else decode_meta(load_meta(block_meta_ptr(v.rec, v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
   if (v.S.code_kind == kRow)
-    code = row_code(reinterpret_cast<const uint32_t*>(v.rec + row_code_off(v.S, i)), c, v.bits);
+    code = row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(v.rec, v.S, i)), c, v.bits);
   else
-    code = chunk_code(reinterpret_cast<const uint32_t*>(v.rec + block_code_off(v.S, i / kChunk)), i % kChunk, c, v.bits);
+    code = chunk_code(reinterpret_cast<const uint32_t*>(block_code_ptr(v.rec, v.S, i / kChunk)), i % kChunk, c, v.bits);
   return fmaf(s, (float)code, z);
 }
 

@@ -259,7 +259,7 @@ __device__ void tail_slice_warp(const Layout& L, const Counts& cn, const T5Args&
                                 const float* qs, const float* qn, float* res) {
   const int lane = threadIdx.x & 31;
   const int n_skew = cn.n_qk - cn.n_qv;
-  const unsigned char* rec = a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride;
+  const Rec rec = unit_rec(L, a.cache, u);
   const __half* k_sink = reinterpret_cast<const __half*>(a.cache + L.k.sink_off + (size_t)u * L.k.sink_stride);
   const __half* k_ring = reinterpret_cast<const __half*>(a.cache + L.k.ring_off + (size_t)u * L.k.ring_stride);
   const __half* v_sink = reinterpret_cast<const __half*>(a.cache + L.v.sink_off + (size_t)u * L.v.sink_stride);
@@ -276,10 +276,10 @@ __device__ void tail_slice_warp(const Layout& L, const Counts& cn, const T5Args&
     float s = -INFINITY;
     if (e < n_skew && e < e_hi) {                       // packed key row
       const int i = cn.n_qv + e;
-      const uint4* row4 = reinterpret_cast<const uint4*>(rec + row_code_off(L.k, i));
+      const uint4* row4 = reinterpret_cast<const uint4*>(row_code_ptr(rec, L.k, i));
       const uint4 r0 = __ldg(row4), r1 = __ldg(row4 + 1);
       const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-      const uint4 mw = __ldg(reinterpret_cast<const uint4*>(rec + row_meta_off(L.k, i)));
+      const uint4 mw = __ldg(reinterpret_cast<const uint4*>(row_meta_ptr(rec, L.k, i)));
       const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w};
       float d = 0.f;
 #pragma unroll
@@ -632,7 +632,7 @@ __global__ void __launch_bounds__(kT5Block, 3) decode_tc5_kernel(const Layout L,
 
 // The format this kernel is built for.
 bool decode_tc5_supported(const Layout& L) {
-  return L.grouping == 0 && L.r == 1 && L.G == 32 && L.k.kind == kRow && L.v.kind == kBlock && L.k.bits == 2 &&
+  return L.page_groups == 0 && L.grouping == 0 && L.r == 1 && L.G == 32 && L.k.kind == kRow && L.v.kind == kBlock && L.k.bits == 2 &&
          L.v.bits == 2 && L.k.meta_bytes == 4 && L.v.meta_bytes == 4;
 }
 

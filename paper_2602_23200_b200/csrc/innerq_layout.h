@@ -67,20 +67,10 @@ struct Store {
                                       // BLOCK: offset of the group's metadata inside a group record
 };
 
-// Byte offset (from the unit's record area) of chunk record ci.
-IQ_HD size_t chunk_rec_off(const Store& S, int ci) {
-  return (size_t)(ci / S.chunks_per_group) * S.group_stride + S.chunk0 + (size_t)(ci % S.chunks_per_group) * S.chunk_stride;
+// Byte offset of chunk record ci inside its group record.
+IQ_HD size_t chunk_in_group_off(const Store& S, int ci) {
+  return S.chunk0 + (size_t)(ci % S.chunks_per_group) * S.chunk_stride;
 }
-// Row-coded tensor: packed row of quantised token i.  kRow tensor: index base of token i's metadata entries.
-IQ_HD size_t row_code_off(const Store& S, int i) {
-  return chunk_rec_off(S, i / kChunk) + S.code_in_rec + (size_t)(i % kChunk) * (16 * S.bits);
-}
-IQ_HD size_t row_meta_off(const Store& S, int i) {
-  return chunk_rec_off(S, i / kChunk) + S.meta_in_rec + (size_t)(i % kChunk) * S.n_groups * S.meta_bytes;
-}
-// Chunk-coded tensor: packed chunk ci.  kBlock tensor: metadata of group j.
-IQ_HD size_t block_code_off(const Store& S, int ci) { return chunk_rec_off(S, ci) + S.code_in_rec; }
-IQ_HD size_t block_meta_off(const Store& S, int j) { return (size_t)j * S.group_stride + S.meta_in_rec; }
 
 struct Layout {
   int B, Hq, Hkv, U, r;
@@ -94,8 +84,55 @@ struct Layout {
   size_t ws_absmax_off;    // uint32 [U][D]
   size_t ws_ticket_off;    // uint32 [U]
   size_t workspace_bytes;
+  // Paged record area (page_groups > 0): the group records of a cache live in pages of a pool that several caches
+  // share, `page_groups` consecutive groups of every unit per page, and a table in the cache's own memory names the
+  // page of each page slot.  Inside a page the layout is the contiguous one ([unit][group]) with rec_unit_stride =
+  // page_groups * group_stride.  page_groups == 0: one contiguous record area per unit inside the cache buffer.
+  int page_groups, max_pages;
+  int page_chunk_mask;     // chunks per page - 1 (a page holds 2^k chunks of 32 tokens); contiguous: 0x3fffffff
+  size_t page_bytes;
+  size_t page_table_off;   // uint32 [max_pages] in the cache buffer: pool page of page slot p
+  unsigned char* pool;     // device address of page 0
   Store k, v;
 };
+
+// The record area of one unit, as the kernels address it: group record g starts at group_ptr(R, g).
+struct Rec {
+  unsigned char* base;       // contiguous: the unit's record area; paged: the unit's slice of pool page 0
+  const uint32_t* table;     // paged: pool page of every page slot of the cache (device memory); null when contiguous
+  size_t page_bytes;
+  int page_groups;
+  int group_stride;
+};
+IQ_HD Rec unit_rec(const Layout& L, const unsigned char* cache, int u) {
+  Rec R;
+  unsigned char* c = const_cast<unsigned char*>(cache);
+  const bool paged = L.page_groups > 0;
+  R.base = (paged ? L.pool : c + L.k.rec_off) + (size_t)u * L.k.rec_unit_stride;
+  R.table = paged ? reinterpret_cast<const uint32_t*>(c + L.page_table_off) : nullptr;
+  R.page_bytes = L.page_bytes;
+  R.page_groups = L.page_groups;
+  R.group_stride = L.k.group_stride;
+  return R;
+}
+IQ_HD unsigned char* group_ptr(const Rec& R, int g) {
+  if (!R.table) return R.base + (size_t)g * R.group_stride;
+  const int slot = g / R.page_groups;
+  return R.base + (size_t)R.table[slot] * R.page_bytes + (size_t)(g - slot * R.page_groups) * R.group_stride;
+}
+IQ_HD unsigned char* chunk_rec_ptr(const Rec& R, const Store& S, int ci) {
+  return group_ptr(R, ci / S.chunks_per_group) + chunk_in_group_off(S, ci);
+}
+// Row-coded tensor: packed row of quantised token i.  kRow tensor: base of token i's metadata entries.
+IQ_HD unsigned char* row_code_ptr(const Rec& R, const Store& S, int i) {
+  return chunk_rec_ptr(R, S, i / kChunk) + S.code_in_rec + (size_t)(i % kChunk) * (16 * S.bits);
+}
+IQ_HD unsigned char* row_meta_ptr(const Rec& R, const Store& S, int i) {
+  return chunk_rec_ptr(R, S, i / kChunk) + S.meta_in_rec + (size_t)(i % kChunk) * S.n_groups * S.meta_bytes;
+}
+// Chunk-coded tensor: packed chunk ci.  kBlock tensor: metadata of group j.
+IQ_HD unsigned char* block_code_ptr(const Rec& R, const Store& S, int ci) { return chunk_rec_ptr(R, S, ci) + S.code_in_rec; }
+IQ_HD unsigned char* block_meta_ptr(const Rec& R, const Store& S, int j) { return group_ptr(R, j) + S.meta_in_rec; }
 
 constexpr int kPartialStride = kD + 4;   // acc[D], m, l, pad, pad
 

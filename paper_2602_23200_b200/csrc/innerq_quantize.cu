@@ -64,7 +64,7 @@ __global__ void fill_float_kernel(float* p, float v, int n) {
 // global memory, whose words other tokens share: that area must be zero before its first token arrives.
 __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src, const float* __restrict__ inv_norm4,
                                                   const Layout& L, const Store& S, uint32_t* stage,
-                                                  unsigned char* __restrict__ rec, int i_row) {
+                                                  const Rec& rec, int i_row) {
   const int lane = threadIdx.x & 31;
   const int gl = L.G >> 2;   // lanes per group
   float x[4];
@@ -102,7 +102,7 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
   const bool asym = choose_asym(S.mode, ea, es);
   if (S.code_kind == kRow) {
     const int words = row_bytes(S.bits) / 4;
-    uint32_t* dst_row = reinterpret_cast<uint32_t*>(rec + row_code_off(S, i_row));
+    uint32_t* dst_row = reinterpret_cast<uint32_t*>(row_code_ptr(rec, S, i_row));
     if (lane < words) stage[lane] = 0u;
     __syncwarp();
 #pragma unroll
@@ -113,14 +113,14 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
     __syncwarp();
     if (lane < words) dst_row[lane] = stage[lane];
   } else {
-    uint32_t* chunk = reinterpret_cast<uint32_t*>(rec + block_code_off(S, i_row / kChunk));
+    uint32_t* chunk = reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, i_row / kChunk));
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
       chunk_put(chunk, i_row % kChunk, 4 * lane + i, S.bits, code);
     }
   }
-  if ((lane % gl) == 0) store_meta(rec + row_meta_off(S, i_row), lane / gl, S.meta_bytes, group_meta(p, asym));
+  if ((lane % gl) == 0) store_meta(row_meta_ptr(rec, S, i_row), lane / gl, S.meta_bytes, group_meta(p, asym));
   __syncwarp();
 }
 
@@ -128,7 +128,7 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
 // A 128-thread CTA quantises one group of G tokens x 128 channels; thread c owns channel c.
 // tile: fp16 [G][D] staging; words: the group's packed chunks, or its packed rows (row-coded tensor), zeroed here.
 __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* __restrict__ norm, const Layout& L,
-                                   const Store& S, __half* tile, uint32_t* words, unsigned char* __restrict__ rec, int group_j) {
+                                   const Store& S, __half* tile, uint32_t* words, const Rec& rec, int group_j) {
   const int G = L.G, c = threadIdx.x;
   const int cw = chunk_bytes(S.bits) / 4, rw = row_bytes(S.bits) / 4;
   const bool rows = S.code_kind == kRow;
@@ -164,15 +164,15 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     if (rows) row_put(words + t * rw, c, S.bits, code);
     else chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
   }
-  store_meta(rec + block_meta_off(S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
+  store_meta(block_meta_ptr(rec, S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
   __syncthreads();
   for (int i = threadIdx.x; i < n_words; i += 128) {
     if (rows) {
       const int t = i / rw;
-      reinterpret_cast<uint32_t*>(rec + row_code_off(S, group_j * G + t))[i - t * rw] = words[i];
+      reinterpret_cast<uint32_t*>(row_code_ptr(rec, S, group_j * G + t))[i - t * rw] = words[i];
     } else {
       const int ch = i / cw;
-      reinterpret_cast<uint32_t*>(rec + block_code_off(S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
+      reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, group_j * (G / kChunk) + ch))[i - ch * cw] = words[i];
     }
   }
   __syncthreads();
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(128) quantize_rows_generic_kernel(Layout L, St
                                                                     int n_q, unsigned char* __restrict__ cache) {
   __shared__ uint32_t stage[4][16];
   const int u = blockIdx.y, warp = threadIdx.x >> 5;
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   for (int i = blockIdx.x * 4 + warp; i < n_q; i += gridDim.x * 4)
     quantize_row_warp(X + ((size_t)u * N + L.w_sink + i) * kD, nullptr, L, S, stage[warp], rec, i);
 }
@@ -193,10 +193,19 @@ __global__ void __launch_bounds__(128) quantize_blocks_generic_kernel(Layout L, 
   __shared__ __align__(16) __half tile[128 * kD];
   __shared__ uint32_t words[4 * 512];
   const int u = blockIdx.y;
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   TokSrc src{X + (size_t)u * N * kD, 0, 0};
   for (int j = blockIdx.x; j < n_q / L.G; j += gridDim.x)
     quantize_block_cta(src, L.w_sink + j * L.G, nullptr, L, S, tile, words, rec, j);
+}
+
+// Paged record area: zeroes the pool page of page slot blockIdx.y.
+__global__ void zero_pages_kernel(Layout L, const unsigned char* __restrict__ cache) {
+  const uint32_t page = reinterpret_cast<const uint32_t*>(cache + L.page_table_off)[blockIdx.y];
+  uint4* dst = reinterpret_cast<uint4*>(L.pool + (size_t)page * L.page_bytes);
+  const size_t n = L.page_bytes / 16;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // ------------------------------------------------------------------ window copies (prefill)
@@ -235,7 +244,7 @@ __device__ __forceinline__ void append_evict_row(const Layout& L, const Store& R
   float inv4[4];
 #pragma unroll
   for (int e = 0; e < 4; ++e) inv4[e] = use_norm ? __fdiv_rn(1.0f, norm[4 * threadIdx.x + e]) : 1.0f;
-  unsigned char* rec = cache + R.rec_off + (size_t)u * R.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   TokSrc src{ring, R.ring_cap, L.w_sink};
   // with an empty recent window the evicted token is the new one, which is not in the ring yet
   const __half* row = L.w_sink + nq_before == t_new ? x_new : src.row(L.w_sink + nq_before);
@@ -263,7 +272,7 @@ __device__ __forceinline__ void append_evict_block(const Layout& L, const Store&
   const float* norm = use_norm ? reinterpret_cast<const float*>(cache + L.norm_off) + (size_t)u * kD : nullptr;
   const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
   TokSrc src{ring, R.ring_cap, L.w_sink};
-  quantize_block_cta(src, L.w_sink + nq_before, norm, L, R, tile, words, cache + R.rec_off + (size_t)u * R.rec_unit_stride,
+  quantize_block_cta(src, L.w_sink + nq_before, norm, L, R, tile, words, unit_rec(L, cache, u),
                      nq_before / L.G);
 }
 
@@ -330,14 +339,14 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
                                     uint16_t* __restrict__ recent_out) {
   const int u = blockIdx.y;
   const int cap = L.max_tokens;
-  const unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   const int stride = gridDim.x * blockDim.x, tid0 = blockIdx.x * blockDim.x + threadIdx.x;
   if (code && S.kind != kNone) {
     for (int i = tid0; i < n_q * kD; i += stride) {
       int t = i / kD, c = i % kD;
       uint32_t v = S.code_kind == kRow
-                       ? row_code(reinterpret_cast<const uint32_t*>(rec + row_code_off(S, t)), c, S.bits)
-                       : chunk_code(reinterpret_cast<const uint32_t*>(rec + block_code_off(S, t / kChunk)), t % kChunk, c,
+                       ? row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(rec, S, t)), c, S.bits)
+                       : chunk_code(reinterpret_cast<const uint32_t*>(block_code_ptr(rec, S, t / kChunk)), t % kChunk, c,
                                     S.bits);
       code[((size_t)u * cap + t) * kD + c] = (uint8_t)v;
     }
@@ -347,8 +356,8 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
     const int rows_cap = S.kind == kRow ? cap : cap / L.G + 1;
     for (int i = tid0; i < n_meta_rows * S.n_groups; i += stride) {
       const int mr = i / S.n_groups, me = i % S.n_groups;
-      uint32_t m = S.kind == kRow ? load_meta(rec + row_meta_off(S, mr), me, S.meta_bytes)
-                                  : load_meta(rec + block_meta_off(S, mr), me, S.meta_bytes);
+      uint32_t m = S.kind == kRow ? load_meta(row_meta_ptr(rec, S, mr), me, S.meta_bytes)
+                                  : load_meta(block_meta_ptr(rec, S, mr), me, S.meta_bytes);
       const int ic = S.kind == kRow ? i : mr * kD + block_meta_channel(me);   // canonical position
       size_t o = (size_t)u * rows_cap * S.n_groups + ic;
       if (scale) scale[o] = (uint16_t)(m & 0xFFFFu);
@@ -395,7 +404,16 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
   }
   if (L.k.kind != kNone && L.k.code_kind != L.k.kind) {
     // chunk words of the outer-grouped cache are filled token by token with OR: they start from zero
-    if (cudaMemsetAsync(cache + L.k.rec_off, 0, L.k.rec_unit_stride * L.U, st) != cudaSuccess) return -1;
+    if (L.page_groups == 0) {
+      if (cudaMemsetAsync(cache + L.k.rec_off, 0, L.k.rec_unit_stride * L.U, st) != cudaSuccess) return -1;
+    } else {      // the pages this prefill fills (the caller has assigned them)
+      const int n_rec = cn.n_qk > cn.n_qv ? cn.n_qk : cn.n_qv;
+      const int n_pages = ((n_rec + L.G - 1) / L.G + L.page_groups - 1) / L.page_groups;
+      if (n_pages > 0) {
+        zero_pages_kernel<<<dim3(64, n_pages), 256, 0, st>>>(L, cache);
+        launches += 1;
+      }
+    }
   }
   const Store* stores[2] = {&L.k, &L.v};
   const __half* srcs[2] = {K, V};

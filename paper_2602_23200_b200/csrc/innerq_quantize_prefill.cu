@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
   constexpr int WM = PB == 2 ? 2 : 4;        // row words between consecutive local words
   const int w_add = PB == 2 ? (seg >> 1) : seg;
   const int sh_lo = PB == 2 ? 8 * (seg & 1) : 0, sh_hi = 4 * seg;
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD + kSeg * seg;
   const int n_batches = (n_q + 7) >> 3;
   const int stride = gridDim.x * 4;
@@ -246,9 +246,9 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
     }
     const int i = i0 + tk;
     if (i < n_q && (lane & (gl - 1)) == 0)
-      store_meta(rec + row_meta_off(S, i0), (size_t)tk * S.n_groups + (seg >> (gl >> 1)), S.meta_bytes, group_meta(p, asym));
+      store_meta(row_meta_ptr(rec, S, i0), (size_t)tk * S.n_groups + (seg >> (gl >> 1)), S.meta_bytes, group_meta(p, asym));
     __syncwarp();
-    uint32_t* dst = reinterpret_cast<uint32_t*>(rec + row_code_off(S, i0));
+    uint32_t* dst = reinterpret_cast<uint32_t*>(row_code_ptr(rec, S, i0));
 #pragma unroll
     for (int k = 0; k < RW / 4; ++k) {
       const int idx = lane + 32 * k;
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
   const int u = blockIdx.y, tid = threadIdx.x, cp = tid & 63, k = tid >> 6, c0 = 2 * cp;
   float inv[2] = {1.0f, 1.0f};
   if constexpr (NORM) { inv[0] = inv_norm[(size_t)u * kD + c0]; inv[1] = inv_norm[(size_t)u * kD + c0 + 1]; }
-  unsigned char* rec = cache + S.rec_off + (size_t)u * S.rec_unit_stride;
+  const Rec rec = unit_rec(L, cache, u);
   const __half* Xu = X + ((size_t)u * N + L.w_sink) * kD + c0;
   // positions (see block_pos_plane): fragment coordinates of the pair (row halves rh = 0, 1)
   const int m = 4 * (c0 >> 6) + ((c0 >> 1) & 3), gid = (c0 >> 3) & 7;
@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
       }
       meta2[rh] = group_meta(p, asym);
     }
-    uint32_t* chunk = reinterpret_cast<uint32_t*>(rec + block_code_off(S, j * CH + k));
+    uint32_t* chunk = reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, j * CH + k));
 #pragma unroll
     for (int i = 0; i < NW; ++i) chunk[base_lo + 4 * (i & 3) + 256 * (i >> 2)] = wlo[i];
     if constexpr (BITS == 3) {
@@ -354,8 +354,8 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
       }
     }
     if (k == 0) {
-      store_meta(rec + block_meta_off(S, j), block_meta_index(c0), S.meta_bytes, meta2[0]);
-      store_meta(rec + block_meta_off(S, j), block_meta_index(c0 + 1), S.meta_bytes, meta2[1]);
+      store_meta(block_meta_ptr(rec, S, j), block_meta_index(c0), S.meta_bytes, meta2[0]);
+      store_meta(block_meta_ptr(rec, S, j), block_meta_index(c0 + 1), S.meta_bytes, meta2[1]);
     }
   }
 }

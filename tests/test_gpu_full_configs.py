@@ -117,6 +117,49 @@ def test_config2_prefill_then_steps():
     print(f"config2, tcgen05 kernel: err/tol {e5:.3f}")
 
 
+def test_config2_paged_cache():
+    # the same workload with the packed records in 512-token pages of a pool, handed out in a shuffled order; the
+    # steps are enqueued back to back and cross a page boundary (the 32636 packed key rows of the prefill fill 63.7 pages)
+    import torch
+    from paper_2602_23200_b200 import binding as B
+    w = synth.config2()
+    K, V = synth.kv_all(w)
+    units = [5, 30]
+    n_steps, page = 140, 512
+    cfg = B.make_config(w, max_tokens=w.n_tokens + n_steps + 8)
+    n_pages = (w.n_tokens + n_steps) // page + 3
+    pool = B.PagePool(cfg, page, n_pages, order=np.random.default_rng(17).permutation(n_pages))
+    pool.buf.fill_(0x5A)
+    gc = B.InnerQCache(cfg, pool=pool)
+    gc.ensure_pages(w.n_tokens)
+    gc.innerq_quantize_prefill(dev(K), dev(V))
+    oc = sub_oracle(w, K, V, units, extra=n_steps + 8)
+    compare(w, gc, oc, units, step=500)
+    toks = [synth.new_token(w, 300 + s) for s in range(n_steps)]
+    qs = [synth.query(w, 300 + s) for s in range(n_steps)]
+    k_all, v_all, q_all = dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks])), dev(np.stack(qs))
+    outs = torch.empty_like(q_all)
+    pages_before = gc.pages_assigned
+    torch.cuda.synchronize()
+    for s in range(n_steps):
+        gc.ensure_pages(gc.n_tokens + 1)
+        gc.innerq_append_token(k_all[s], v_all[s])
+        gc.innerq_decode_attention(q_all[s], outs[s])
+    torch.cuda.synchronize()
+    assert gc.pages_assigned == pages_before + 1
+    got = outs.cpu().numpy()
+    worst = 0.0
+    for s in range(n_steps):
+        k1, v1 = toks[s]
+        oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+        if s < 2 or 124 <= s < 134 or s == n_steps - 1:
+            ref = oc.decode(q_rows(w, qs[s], units))
+            worst = max(worst, P.assert_outputs_close(q_rows(w, got[s], units), ref, f"paged, step {s}"))
+    P.assert_export_equal(slice_export(gc.innerq_cache_export(), units), oc.export(), w.grouping, w.group, True, True)
+    assert gc.innerq_read_device_error() == 0
+    print(f"config2, paged cache, {n_steps} steps back to back: worst err/tol {worst:.3f}")
+
+
 @pytest.mark.parametrize("bits", [4, 2])
 def test_config3_gqa_batch16(bits):
     w = synth.config3(bits)
