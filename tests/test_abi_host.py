@@ -100,3 +100,28 @@ def test_cache_size_tracks_payload():
     payload = w.n_units * w.n_tokens * (k_bytes + v_bytes)
     assert payload <= cb <= 1.02 * payload
     assert cb < 0.16 * (2 * w.n_units * w.n_tokens * 128 * 2)      # 2.25 bits vs 16 bits per number
+
+
+def test_paged_sizes_without_gpu():
+    # a page holds page_tokens tokens of every unit, at exactly the payload the effective-bits table counts;
+    # the cache buffer of a paged cache keeps only what does not grow with the context
+    for w in (synth.config2(), synth.config3(4), synth.config4()):
+        for kw in ({}, dict(grouping=B.GROUPING_OUTER, k_normalize=0, k_mode=B.MODE_ASYM, v_mode=B.MODE_ASYM)):
+            cfg = B.make_config(w, **kw)
+            k_bytes, v_bytes = B.innerq_token_payload_bytes(cfg)
+            full, _ = B.innerq_cache_bytes(cfg)
+            for page in (128, 1024, 4096):
+                cb, wb, pb, mp = B.innerq_paged_cache_bytes(cfg, page)
+                assert pb == page * w.n_units * (k_bytes + v_bytes), (w.name, page)
+                packed_tokens = w.n_tokens - w.w_sink - w.w_recent
+                assert mp * page >= packed_tokens and (mp - 1) * page < packed_tokens + 32 + 128
+                assert cb < 0.02 * full + 2 * w.n_units * (w.w_sink + w.w_recent + w.group + 1) * 128 * 2 + 4 * mp + 4096
+                assert wb == B.innerq_cache_bytes(cfg)[1]
+    cfg = B.make_config(synth.config2())
+    for bad in (0, 100, 64, 384, -1024):
+        with pytest.raises(B.InnerQError) as ei:
+            B.innerq_paged_cache_bytes(cfg, bad)
+        assert ei.value.status == -1
+    with pytest.raises(B.InnerQError) as ei:
+        B.innerq_paged_cache_bytes(B.make_config(synth.config2(), grouping=B.GROUPING_FP16), 1024)
+    assert ei.value.status == -2
