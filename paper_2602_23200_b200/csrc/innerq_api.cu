@@ -165,6 +165,7 @@ void make_layout(const innerq_config_t& c, Layout& L, int page_tokens = 0) {
   }
   L.page_chunk_mask = page_tokens > 0 ? page_tokens / kChunk - 1 : 0x3fffffff;
   if (page_tokens > 0) {
+    for (int n = page_tokens / kChunk; n > 1; n >>= 1) L.page_chunk_shift += 1;
     L.page_groups = page_tokens / L.G;
     L.max_pages = (L.k.cap_q / L.G + L.page_groups - 1) / L.page_groups;
     L.page_bytes = align_up(L.k.rec_unit_stride * L.U, 256);
@@ -393,7 +394,7 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L)) {
     n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
-                          c->opt_splits, s, 1, nullptr, c->N_safe);
+                          c->opt_splits, s, 1, nullptr, c->N_safe, c->pages.data(), (int)c->pages.size());
     fused = n >= 0;
   }
   if (n == -2) {
@@ -433,7 +434,7 @@ int innerq_decode_attention_multi(innerq_cache_t* c, const void* q, void* out, i
   if (n_packed > 0 && c->N - n_q + 1 < cn.n_sink + n_packed) return INNERQ_ERR_UNSUPPORTED;
   const int n = launch_decode_mma(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                                   c->opt_splits, static_cast<cudaStream_t>(cuda_stream), n_q,
-                                  static_cast<float*>(dev_scratch), c->N_safe);
+                                  static_cast<float*>(dev_scratch), c->N_safe, c->pages.data(), (int)c->pages.size());
   if (n == -2) return INNERQ_ERR_UNSUPPORTED;
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N_safe = c->N;
@@ -622,7 +623,7 @@ int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, 
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L)) {
     n = launch_decode_mma(c->L, c->cache, scratch, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
-                          c->opt_splits, s, 1, nullptr, c->N_safe);
+                          c->opt_splits, s, 1, nullptr, c->N_safe, c->pages.data(), (int)c->pages.size());
     fused = n >= 0;
   }
   if (n == -2) {

@@ -103,6 +103,8 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
     e.a.safe_chunks = safe_chunks_for(L, Ns_safe[i], e.cn);
     e.a.n_q = 1;
     e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
+    e.a.pages_host = nullptr;      // paged caches: a batched launch reads every cache's table from its buffer
+    e.a.n_pages_host = 0;
   }
   for (int i = n; i < kMaxSeqs; ++i) T.s[i] = T.s[0];
   return launch(L, T, n, row_budget, g_chunks_per_iter, st);
@@ -123,7 +125,8 @@ static int safe_chunks_for(const Layout& L, int N_safe, const Counts& cn_now) {
 }
 
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials, int N_safe) {
+                      __half* out, int n_splits, cudaStream_t st, int n_q, float* multi_partials, int N_safe,
+                      const uint32_t* pages_host, int n_pages_host) {
   const FormatLauncher launch = format_launcher(L);
   if (!launch) return -2;
   const Counts cn = counts_for(L, N);
@@ -137,6 +140,8 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.safe_chunks = safe_chunks_for(L, N_safe, cn);
   a.n_q = n_q;
   a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
+  a.pages_host = pages_host;
+  a.n_pages_host = n_pages_host;
   if (n_q < 1 || (n_q > 1 && !multi_partials)) return -1;
   return launch(L, cn, a, n_splits, g_chunks_per_iter, st);
 }

@@ -246,7 +246,8 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 // m-tile's rows fall into); zero-points contribute sum_c q''_c Z_jc per group and sum_t p_t Z_{t,g} per channel
 // group.  One chunk per iteration, four heads per pass.
 template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
-__device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u) {
+__device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u,
+                                                const PageIds* ptab = nullptr) {
   constexpr int KP = KB == 3 ? 2 : KB, VP = VB == 3 ? 2 : VB;     // bits of the primary code plane
   using F = Fmt<KP>;
   using FV = Fmt<VP>;
@@ -314,16 +315,37 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kOffBars) + warp * NST;
   const uint32_t ring_u32 = smem_u32(ring), bars_u32 = smem_u32(bars);
   // Group record g of this unit (a paged cache looks the group's page up in the cache's page table).
+  // (ptab: the table as a kernel parameter, when the launcher could pass it; else it is read from the cache buffer)
+  [[maybe_unused]] auto page_of = [&](int slot) -> uint32_t {
+    return ptab ? ptab->id[slot] : reinterpret_cast<const uint32_t*>(a.cache + L.page_table_off)[slot];
+  };
+  [[maybe_unused]] auto page_start = [&](uint32_t page) -> const unsigned char* {
+    return L.pool + (size_t)page * L.page_bytes + (size_t)u * L.k.rec_unit_stride;
+  };
   auto group_rec = [&](int g) -> const unsigned char* {
-    if constexpr (PAGED) return group_ptr(unit_rec(L, a.cache, u), g);
-    else return a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride + (size_t)g * SL::kGroupRec;
+    if constexpr (PAGED) {
+      const int slot = g / L.page_groups;
+      return page_start(page_of(slot)) + (size_t)(g - slot * L.page_groups) * SL::kGroupRec;
+    } else {
+      return a.cache + L.k.rec_off + (size_t)u * L.k.rec_unit_stride + (size_t)g * SL::kGroupRec;
+    }
   };
 
   // Copies of consecutive iterations read consecutive byte ranges of the record area: keep a running source.
   // In a paged cache (PAGED) that holds inside a page (2^k chunks): the copy that starts a page is re-based, and the
-  // copy whose two chunks lie in two pages is split.
+  // copy whose two chunks lie in two pages is split.  The table entry of the page after the current one is loaded
+  // one page ahead (page_next), so that no copy waits for a table lookup except a warp's first one.
   const unsigned char* nx_src = n_iters > 0 ? group_rec(c_lo / CH) + (size_t)(c_lo % CH) * SL::kRec : nullptr;
   int nx_ci = c_lo;
+  [[maybe_unused]] uint32_t page_next = 0;
+  [[maybe_unused]] auto load_page_next = [&](int ci) {      // ci: a chunk of the page that is current from now on
+    const int slot = (ci >> L.page_chunk_shift) + 1;
+    if ((slot << L.page_chunk_shift) < c_lo + n_chunks_w)   // this warp will read that page: it exists
+      page_next = page_of(slot);
+  };
+  if constexpr (PAGED) {
+    if (n_iters > 0) load_page_next(c_lo);
+  }
   auto issue = [&](int st) {   // one lane: arm the barrier, start the copy of the next iteration into stage st
     // the value group's scale/zero words sit right behind its last chunk
     // (OUTER: the key group's words sit in front of its first chunk)
@@ -331,18 +353,23 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
                              : (CPI >= CH ? CPI / CH : (((nx_ci + CPI) & (CH - 1)) == 0 ? 1 : 0));
     const uint32_t bytes = CPI * SL::kRec + n_meta * SL::kVMeta;
     mbar_expect_tx(bars_u32 + 8 * st, bytes);
-    const int in_page = PAGED ? nx_ci & L.page_chunk_mask : 1;
-    if (in_page == 0) {
-      nx_src = group_rec(nx_ci / CH);
-    } else if (PAGED && in_page + CPI > L.page_chunk_mask + 1) {
-      // CPI = 2 with one chunk per group, first chunk at the end of a page: two copies of one group record each.
-      // A second chunk beyond this warp's range is not used (and its page may not exist): the first one again.
-      const unsigned char* second = nx_ci + 1 < c_lo + n_chunks_w ? group_rec((nx_ci + 1) / CH) : nx_src;
-      bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes / 2, bars_u32 + 8 * st);
-      bulk_g2s(ring_u32 + st * SL::kBytes + bytes / 2, second, bytes / 2, bars_u32 + 8 * st);
-      nx_src = second + bytes / 2;
-      nx_ci += CPI;
-      return;
+    if constexpr (PAGED) {
+      const int in_page = nx_ci & L.page_chunk_mask;
+      if (in_page == 0 && nx_ci != c_lo) {
+        nx_src = page_start(page_next);
+        load_page_next(nx_ci);
+      } else if (in_page + CPI > L.page_chunk_mask + 1) {
+        // CPI = 2 with one chunk per group, first chunk at the end of a page: two copies of one group record each.
+        // A second chunk beyond this warp's range is not used (and its page may not exist): the first one again.
+        const bool used = nx_ci + 1 < c_lo + n_chunks_w;
+        const unsigned char* second = used ? page_start(page_next) : nx_src;
+        bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes / 2, bars_u32 + 8 * st);
+        bulk_g2s(ring_u32 + st * SL::kBytes + bytes / 2, second, bytes / 2, bars_u32 + 8 * st);
+        nx_src = second + bytes / 2;
+        if (used) load_page_next(nx_ci + 1);
+        nx_ci += CPI;
+        return;
+      }
     }
     bulk_g2s(ring_u32 + st * SL::kBytes, nx_src, bytes, bars_u32 + 8 * st);
     nx_src += bytes;
@@ -1200,6 +1227,13 @@ __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
   decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>(L, cn, a, blockIdx.x);
 }
+
+// One paged cache with its page table in the parameter space (read in place: no look-up in device memory).
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_mma_paged_kernel(const Layout L, const Counts cn, const DecodeArgs a, const __grid_constant__ PageIds P) {
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, true>(L, cn, a, blockIdx.x, &P);
+}
 // Several caches of one configuration: block x = sequence * U + unit, the sequence's counts and parameters come
 // from its table entry (read in place from the parameter space).
 template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
@@ -1242,6 +1276,17 @@ int launch_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, 
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
   if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, kSmem, configured)) return -1;
+  // a paged cache whose page list fits the parameter space: the kernel that takes the table as a parameter
+  [[maybe_unused]] PageIds ids;
+  bool table_in_params = false;
+  if constexpr (PAGED) {
+    static std::atomic<unsigned long long> configured_p{0};
+    if (a.pages_host && a.n_pages_host <= kParamPages) {
+      if (!opt_in_dynamic_smem(decode_mma_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, kSmem, configured_p)) return -1;
+      for (int i = 0; i < a.n_pages_host; ++i) ids.id[i] = a.pages_host[i];
+      table_in_params = true;
+    }
+  }
   const int grid_y = fill_split_args<RU>(L, cn, a, OUTER, n_splits, 0);
   dim3 grid(L.U, grid_y);
   int launches = 0;
@@ -1256,7 +1301,14 @@ int launch_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a) != cudaSuccess) return -1;
+    cudaError_t err;
+    if constexpr (PAGED) {
+      err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_mma_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, cn, a, ids)
+                            : cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a);
+    } else {
+      err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a);
+    }
+    if (err != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

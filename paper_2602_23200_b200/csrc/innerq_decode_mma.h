@@ -33,6 +33,16 @@ struct DecodeArgs {
                          // n_q - 1 - i tokens (all of them outside the chunks where keys AND values are packed)
   float* partials;       // split partials [rows][max_splits][kPartialStride]: row = global query head (n_q == 1) or
                          // unit * 4 + column of the launch (n_q > 1)
+  // HOST side only (paged caches): the cache's page list, which the launcher copies into the kernel's parameter
+  // space when it fits (PageIds), so that no copy of a CTA waits for a look-up in the table in device memory
+  const uint32_t* pages_host;
+  int n_pages_host;
+};
+
+// A paged cache's table (pool page of every page slot) as a kernel parameter.
+constexpr int kParamPages = 512;
+struct PageIds {
+  uint32_t id[kParamPages];
 };
 
 // Batched launch over several caches of one configuration, each with its own length (continuous batching):

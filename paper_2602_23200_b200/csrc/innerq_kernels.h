@@ -45,9 +45,10 @@ int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned cha
                        __half* out, int n_splits, cudaStream_t st);
 
 // Warp-MMA decode for the INNER layout.  Returns -2 if the configuration is not supported.
+// pages_host: a paged cache's page list on the host (optional: saves the kernel its look-ups in device memory).
 int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                       __half* out, int n_splits, cudaStream_t st, int n_q = 1, float* multi_partials = nullptr,
-                      int N_safe = 0);
+                      int N_safe = 0, const uint32_t* pages_host = nullptr, int n_pages_host = 0);
 int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const* caches, unsigned char* const* wss,
                               const int* Ns, const int* Ns_safe, const __half* q, __half* out, int n_splits,
                               cudaStream_t st);

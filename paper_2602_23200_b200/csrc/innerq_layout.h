@@ -90,6 +90,7 @@ struct Layout {
   // page_groups * group_stride.  page_groups == 0: one contiguous record area per unit inside the cache buffer.
   int page_groups, max_pages;
   int page_chunk_mask;     // chunks per page - 1 (a page holds 2^k chunks of 32 tokens); contiguous: 0x3fffffff
+  int page_chunk_shift;    // k
   size_t page_bytes;
   size_t page_table_off;   // uint32 [max_pages] in the cache buffer: pool page of page slot p
   unsigned char* pool;     // device address of page 0
