@@ -284,3 +284,119 @@ def test_paged_argument_and_capacity_errors():
     with pytest.raises(B.InnerQError) as e:
         cc.innerq_cache_assign_pages([0])
     assert e.value.status == ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_interleaving_of_calls_on_paged_caches(seed):
+    # Two pools (two formats), two caches on each; appends (pages taken just in time), decodes with both kernels,
+    # multi-query decodes and restarts (a cache hands its pages back and is prefilled with a new sequence out of the
+    # same pool) are enqueued in random order on one stream with no host synchronisation; every output is checked
+    # against the oracle afterwards.
+    from paper_2602_23200_b200 import binding as B
+    torch = _torch()
+    rng = np.random.default_rng(100 + seed)
+    specs = [dict(n_q_heads=4, n_kv_heads=4, group=32, k_bits=2, v_bits=2, w_recent=16),
+             dict(n_q_heads=8, n_kv_heads=2, group=64, k_bits=3, v_bits=2, k_mode=O.SYM, w_recent=24)]
+    n_in, cap = 200, 1400
+    slots = []                                     # one per cache: dict(w, oc, gc, step, spec index, pool)
+    inputs = {}                                    # wid -> host and device copies of the tokens and queries
+
+    def sequence(si, wid, n_tokens):
+        w = synth.tiny(batch=1, n_tokens=n_tokens, wid=wid, **specs[si])
+        toks = [synth.new_token(w, s) for s in range(n_in)]
+        qs = [synth.query(w, 1000 + s) for s in range(n_in)]
+        K, V = synth.kv_all(w)
+        inputs[wid] = dict(w=w, toks=toks, qs=qs, K=K, V=V, Kd=dev(K), Vd=dev(V),
+                           kd=dev(np.stack([t[0] for t in toks])), vd=dev(np.stack([t[1] for t in toks])),
+                           qd=dev(np.stack(qs)))
+        return w
+
+    wid = 700 + 50 * seed
+    for si in range(len(specs)):
+        w0 = sequence(si, wid, 500); wid += 1
+        cfg = B.make_config(w0, max_tokens=cap)
+        pool = make_pool(cfg, 128, 2 * (cap // 128 + 2), seed=seed + si)
+        for k in range(2):
+            w = w0
+            if k == 1:
+                w = sequence(si, wid, 300 + 64 * seed); wid += 1
+            gc = B.InnerQCache(cfg, pool=pool)
+            gc.ensure_pages(w.n_tokens)
+            gc.innerq_quantize_prefill(inputs[w.wid]["Kd"], inputs[w.wid]["Vd"])
+            slots.append(dict(wid=w.wid, gc=gc, step=0, nq=0, si=si))
+    # sequences that restarts will switch to, made (and copied to the device) up front
+    spare = []
+    for k in range(6):
+        si = k % len(specs)
+        w = sequence(si, wid, 200 + 90 * k); wid += 1
+        spare.append(w.wid)
+    torch.cuda.synchronize()
+    ops = []
+    for it in range(320):
+        i = int(rng.integers(len(slots)))
+        s = slots[i]
+        op = str(rng.choice(["append", "decode", "plain", "multi", "restart"], p=[.5, .3, .05, .1, .05]))
+        if op == "append":
+            if s["step"] >= n_in:
+                continue
+            ops.append((op, i, s["wid"], s["step"], 0)); s["step"] += 1
+        elif op == "restart":
+            cand = [x for x in spare if inputs[x]["w"].group == specs[s["si"]]["group"]]
+            if not cand:
+                continue
+            spare.remove(cand[0])
+            s.update(wid=cand[0], step=0, nq=0)
+            ops.append((op, i, cand[0], 0, 0))
+        elif op == "multi":
+            n_q = int(rng.integers(2, 5))
+            ops.append((op, i, s["wid"], s["nq"] % (n_in - 4), n_q)); s["nq"] += n_q
+        else:
+            ops.append((op, i, s["wid"], s["nq"] % n_in, 0)); s["nq"] += 1
+    outs = []
+    for op, i, w_id, j, n_q in ops:                # nothing here waits for the GPU
+        gc, x = slots[i]["gc"], inputs[w_id]
+        if op == "append":
+            gc.ensure_pages(gc.n_tokens + 1)
+            gc.innerq_append_token(x["kd"][j], x["vd"][j])
+            outs.append(None)
+        elif op == "restart":
+            gc.release_to_pool()
+            gc.ensure_pages(x["w"].n_tokens)
+            gc.innerq_quantize_prefill(x["Kd"], x["Vd"])
+            outs.append(None)
+        elif op == "multi":
+            outs.append(gc.innerq_decode_attention_multi(x["qd"][j:j + n_q].transpose(0, 1).contiguous()))
+        else:
+            gc.innerq_set_decode_options(0, 1 if op == "plain" else 0)
+            outs.append(gc.innerq_decode_attention(x["qd"][j]))
+            gc.innerq_set_decode_options(0, 0)
+    torch.cuda.synchronize()
+    ocs = {}
+
+    def oracle_for(i, w_id):
+        x = inputs[w_id]
+        oc = O.from_workload(x["w"], max_tokens=cap)
+        oc.prefill(x["K"], x["V"])
+        ocs[i] = oc
+
+    started = set()
+    for (op, i, w_id, j, n_q), out in zip(ops, outs):
+        if i not in started:                        # the sequence the cache was created with
+            started.add(i)
+            if op != "restart":
+                oracle_for(i, w_id)
+        x = inputs[w_id]
+        if op == "restart":
+            oracle_for(i, w_id)
+        elif op == "append":
+            ocs[i].append(*x["toks"][j])
+        elif op == "multi":
+            P.assert_outputs_close(out.cpu().numpy(), ocs[i].decode_multi(np.stack(x["qs"][j:j + n_q], axis=1)), f"multi, cache {i}")
+        else:
+            P.assert_outputs_close(out.cpu().numpy(), ocs[i].decode(x["qs"][j]), f"{op}, cache {i}")
+    for i, oc in ocs.items():
+        gc, w = slots[i]["gc"], inputs[slots[i]["wid"]]["w"]
+        assert gc.n_tokens == oc.N and gc.innerq_read_device_error() == 0
+        assert gc.pages_assigned == gc.innerq_cache_pages_for(gc.n_tokens)
+        P.assert_export_equal(gc.innerq_cache_export(), oc.export(), w.grouping, w.group,
+                              k_hybrid=w.k_mode == O.HYBRID, v_hybrid=w.v_mode == O.HYBRID)
