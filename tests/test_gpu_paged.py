@@ -400,3 +400,14 @@ def test_random_interleaving_of_calls_on_paged_caches(seed):
         assert gc.pages_assigned == gc.innerq_cache_pages_for(gc.n_tokens)
         P.assert_export_equal(gc.innerq_cache_export(), oc.export(), w.grouping, w.group,
                               k_hybrid=w.k_mode == O.HYBRID, v_hybrid=w.v_mode == O.HYBRID)
+
+
+def test_paged_table_longer_than_the_kernel_parameter_takes():
+    # a single-cache launch passes up to 512 page indices in its parameter space; a cache with more pages makes the
+    # same kernel read the table from the cache buffer (as batched launches always do)
+    w = synth.tiny(batch=1, n_kv_heads=1, n_q_heads=2, n_tokens=66100, group=32)
+    oc, gc = paged_pair(w, 128, 66100 + 140, seed=4)
+    assert gc.pages_assigned > 512
+    check_decode(w, oc, gc, variants=(0,), splits=(0, 5))
+    steps(w, oc, gc, 0, 130, check_every=43, variants=(0,))
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, 32)
