@@ -168,8 +168,9 @@ int innerq_quantize_prefill(innerq_cache_t* cache, const void* k, const void* v,
  * window while it is not full, else the recent window; tokens leaving the recent window are
  * normalised with the norm fixed at prefill (keys) and quantised into the packed cache.
  * Stream order as for innerq_decode_attention: when the cache's previous call was a decode, this kernel reads
- * k_new, v_new and writes the cache while that decode is still merging its partial results (the decode has read
- * the cache by then), so k_new and v_new must be complete before the call under the same rule as `q`.
+ * k_new, v_new and writes the cache while that decode is still running (the decode lets it start once it has
+ * read everything an append writes: the fp16 windows and the newest packed rows; the packed range it goes on
+ * streaming is never written again), so k_new and v_new must be complete before the call under the same rule as `q`.
  * Errors: INVALID_ARG, CAPACITY, CUDA. */
 int innerq_append_token(innerq_cache_t* cache, const void* k_new, const void* v_new, void* cuda_stream);
 

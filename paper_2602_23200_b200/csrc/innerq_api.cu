@@ -19,7 +19,8 @@ struct innerq_cache {
   int N_safe;      // token count when the last decode of this cache was launched (or at prefill): what was packed by then
                    // is complete and is not written again; a later decode may stream it before its predecessors finish
   int reads_settled;   // the last kernel enqueued for this cache was a fused decode: when its dependents may start, it
-                       // has read everything it reads from the cache (an append can then run without waiting first)
+                       // has read everything that an append writes (the fp16 rings, the newest packed rows); an
+                       // append can then run without waiting first
   int opt_splits, opt_variant;
   int launches[3];
   int pool_pages;                 // paged cache: pages in the pool (page ids are checked against it)

@@ -445,6 +445,8 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       if (lane == 0) issue(s);
     }
 
+  __shared__ unsigned int s_past_tail;      // warps of this CTA that are past their tail tiles (see the main loop's head)
+  if (tid == 0) s_past_tail = 0u;           // ordered before its first use by the barriers of the prologue
   // ---------------- prologue: q'' = q * sm_scale * log2(e) (* norm for packed key rows) -------------
   float* q_nrm_s = reinterpret_cast<float*>(smem + SL::kOffSide);  // [4][128]   (the side area is not in use yet)
   float* q_raw_s = q_nrm_s + kHeads * kD;                          // [4][128]
@@ -857,6 +859,16 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       }
     }
 
+    // From here on this warp reads nothing that the next step's append writes (the fp16 rings and packed rows /
+    // groups that do not exist yet).  When that holds for every warp of the CTA, the CTA lets the next kernel in the
+    // stream start (one call per CTA counts, so the last warp to get here makes it); dependents start when every
+    // CTA has.  One warp per unit gets here only after it has waited for this kernel's own predecessors, so
+    // whatever starts then finds everything before this kernel complete (an append relies on that: it works first
+    // and waits afterwards).  The step's append thus runs while this kernel streams, not after it.
+    if (split == 0 && warp == 0) dep_wait();
+    __syncwarp();
+    if (lane == 0 && atomicAdd(&s_past_tail, 1u) == kWarps - 1) grid_launch_dependents();
+
     // The loop body is deliberately not unrolled over iterations: two CTAs of eight warps walk it at
     // different phases, so it has to stay resident in the instruction cache.
 #pragma unroll 1
@@ -1118,10 +1130,8 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       }
     }
 
-    // Before the next kernel in the stream may start (and stream its own safe chunks), this one has made sure that
-    // everything before it is complete; the partials and tickets written below are also shared with the previous decode.
+    // the partials and tickets written below are also shared with the previous decode
     dep_wait();
-    grid_launch_dependents();     // the next kernel in the stream may start its own set-up during this epilogue
     if (failed) {
       // a copy never arrived: flag it for the host and contribute nothing
       if (lane == 0) atomicExch(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + L.U, 1u);

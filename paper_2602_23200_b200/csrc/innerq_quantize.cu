@@ -294,13 +294,15 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
 // kernel cannot write and waits for this kernel's completion before it touches the rest).  This kernel in turn
 // waits for the kernels before it, either before its first global access or, with late_wait (the host knows that
 // the last kernel on this cache was a fused decode, which lets its dependents start only after its last read of
-// the cache), after its work: it then runs during that decode's merge, and still completes after it, so that
-// whatever follows sees both finished.
+// what an append writes: the fp16 rings and the packed rows / groups behind the range it streams), after its work:
+// it then runs while that decode streams the packed cache, and still completes after it, so that whatever follows
+// sees both finished.
 __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
                                                      const __half* __restrict__ v_new, int N,
                                                      unsigned char* __restrict__ cache, int late_wait) {
-  __shared__ __align__(16) __half tile[128 * kD];
-  __shared__ uint32_t words[4 * 512];
+  extern __shared__ __align__(16) unsigned char append_smem[];      // see append_smem_bytes
+  __half* tile = reinterpret_cast<__half*>(append_smem);
+  uint32_t* words = reinterpret_cast<uint32_t*>(append_smem + (size_t)L.G * kD * 2);
   const int u = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -322,8 +324,9 @@ __global__ void __launch_bounds__(128) append_batched_kernel(const __grid_consta
                                                              const __half* __restrict__ k_new,
                                                              const __half* __restrict__ v_new,
                                                              const __grid_constant__ AppendTable T) {
-  __shared__ __align__(16) __half tile[128 * kD];
-  __shared__ uint32_t words[4 * 512];
+  extern __shared__ __align__(16) unsigned char append_smem[];
+  __half* tile = reinterpret_cast<__half*>(append_smem);
+  uint32_t* words = reinterpret_cast<uint32_t*>(append_smem + (size_t)L.G * kD * 2);
   const int seq = blockIdx.x / L.U, u = blockIdx.x - seq * L.U;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int late_wait = T.s[seq].late_wait;
@@ -455,10 +458,16 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
+// Shared memory of an append CTA: the fp16 staging tile of one group of G tokens and the group's packed words (a
+// 32-token chunk is at most 512 words; a row-coded group G rows of at most 16 words).  Sized by G, not for the
+// largest G: with G = 32 four of these CTAs fit beside a resident decode CTA, so the append of every unit of the
+// benchmark shapes runs while the previous decode is still streaming.
+static size_t append_smem_bytes(const Layout& L) { return (size_t)L.G * kD * 2 + (size_t)(L.G / kChunk) * 512 * 4; }
+
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
                   cudaStream_t st, int late_wait) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cfg.gridDim = dim3(L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = append_smem_bytes(L); cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -476,7 +485,7 @@ int launch_append_batched(const Layout& L, int n, unsigned char* const* caches, 
     T.s[i].late_wait = late_wait[i < n ? i : 0];
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n * L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cfg.gridDim = dim3(n * L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = append_smem_bytes(L); cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
