@@ -187,8 +187,8 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
       for (int e = 0; e < 4; ++e) {
         const int s = s0 + e * kWarps;
         const float* P = Ph + (size_t)(s < n_parts ? s : s0) * kPartialStride;
-        v[e] = __ldcg(reinterpret_cast<const float4*>(P) + lane);
-        ml[e] = __ldcg(reinterpret_cast<const float2*>(P + kD));
+        v[e] = __ldg(reinterpret_cast<const float4*>(P) + lane);
+        ml[e] = __ldg(reinterpret_cast<const float2*>(P + kD));
         if (s >= n_parts) ml[e] = make_float2(-INFINITY, 0.f);
       }
 #pragma unroll
@@ -422,6 +422,22 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
   auto dep_wait = [&]() {
     if (!dep_waited) { grid_dependency_wait(); dep_waited = true; }
   };
+  // What the step's append writes for this unit (rings, newest packed rows) is complete when the unit's counter in
+  // the cache buffer holds this decode's N: the append publishes it (release) after its last write, long before it
+  // ends (it ends after the previous decode).  A decode that follows an append in the stream waits for its
+  // predecessor's completion (the append is most likely still at work, and that wait wakes up faster than any
+  // polling).  A decode that follows another decode looks once (acquire): the count is there, since that decode
+  // saw the append complete before it let this one start, and the warp goes on at once, while the previous decode
+  // may still be merging; should it not be there, the wait for the predecessor is always right.
+  auto wait_for_append = [&]() {
+    if (dep_waited) return;
+    if (a.after_append) { dep_wait(); return; }
+    const uint32_t* flag = reinterpret_cast<const uint32_t*>(a.cache + L.appended_off) + u;
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (!__all_sync(0xffffffffu, v == (uint32_t)cn.N)) dep_wait();
+  };
+  auto ld_tail = [&](const uint4* p) -> uint4 { return dep_waited ? __ldg(p) : __ldcg(p); };
   // an iteration's copy covers the chunks [c_lo + i * CPI, c_lo + (i + 1) * CPI)
   auto dep_wait_for_iteration = [&](int i) {
     if (c_lo + (i + 1) * CPI > a.safe_chunks) dep_wait();
@@ -730,7 +746,10 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     // running soft-max state.  Keys: fp16 rows against raw q'' (pieces tid4 + 4i of rows gid, gid + 8), or the
     // packed rows of the skew zone through the same path as the main loop.  Values: fp16 rows, pieces gid and
     // gid + 8 of token rows 2*tid4, 2*tid4 + 1 (+8), byte-permuted into (channel; token pair) fragments.
-    if (tw > 0) dep_wait();          // the rings and the newest packed rows are what the append writes
+    // After the wait for the predecessor kernel these rows go through the read-only path; a warp that went on after
+    // its look at the append's counter reads them at the L2 cache (the acquire covers ordinary loads, and this SM's
+    // read-only cache may still hold the rows as an earlier decode saw them).
+    if (tw > 0) wait_for_append();   // the rings and the newest packed rows are what the append writes
     for (int k = 0; k < tw; ++k) {
       bool skew; int e0, cnt;
       tail_tile(k, skew, e0, cnt);
@@ -747,7 +766,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
         const uint4* rb = k_row(skew, e0 + min(gid + 8, cnt - 1));
         uint4 ka[4], kb[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { ka[i] = __ldg(ra + j + 4 * i); kb[i] = __ldg(rb + j + 4 * i); }
+        for (int i = 0; i < 4; ++i) { ka[i] = ld_tail(ra + j + 4 * i); kb[i] = ld_tail(rb + j + 4 * i); }
         float c4[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -809,8 +828,8 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
           for (int st_ = 0; st_ < NSET; ++st_) Bt[st_][h] = movmatrix_trans(pk[st_]);
         }
         if constexpr (VP == 2) {
-          const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(vcg + lane * 4));
-          const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(vcg + 128 + lane * 4));
+          const uint4 v0 = ld_tail(reinterpret_cast<const uint4*>(vcg + lane * 4));
+          const uint4 v1 = ld_tail(reinterpret_cast<const uint4*>(vcg + 128 + lane * 4));
           const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
           for (int m = 0; m < 8; ++m) {
@@ -821,7 +840,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
         } else {
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(vcg + ks * 256 + hh * 128 + lane * 4));
+            const uint4 v = ld_tail(reinterpret_cast<const uint4*>(vcg + ks * 256 + hh * 128 + lane * 4));
             const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int mm = 0; mm < 4; ++mm) {
@@ -842,7 +861,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       for (int hh = 0; hh < 2; ++hh) {
         uint4 v4[4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) v4[r] = __ldg(vr[r] + gid + 8 * hh);
+        for (int r = 0; r < 4; ++r) v4[r] = ld_tail(vr[r] + gid + 8 * hh);
         const uint32_t* T0 = reinterpret_cast<const uint32_t*>(&v4[0]);
         const uint32_t* T1 = reinterpret_cast<const uint32_t*>(&v4[1]);
         const uint32_t* T8 = reinterpret_cast<const uint32_t*>(&v4[2]);
@@ -862,10 +881,10 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     // From here on this warp reads nothing that the next step's append writes (the fp16 rings and packed rows /
     // groups that do not exist yet).  When that holds for every warp of the CTA, the CTA lets the next kernel in the
     // stream start (one call per CTA counts, so the last warp to get here makes it); dependents start when every
-    // CTA has.  One warp per unit gets here only after it has waited for this kernel's own predecessors, so
-    // whatever starts then finds everything before this kernel complete (an append relies on that: it works first
-    // and waits afterwards).  The step's append thus runs while this kernel streams, not after it.
-    if (split == 0 && warp == 0) dep_wait();
+    // CTA has.  One warp per unit gets here only after it has seen the unit's last append complete, so the next
+    // append (which works first and waits afterwards) finds its predecessor's writes in place and nobody reading
+    // what it is about to overwrite.  The step's append thus runs while this kernel streams, not after it.
+    if (split == 0 && warp == 0) wait_for_append();
     __syncwarp();
     if (lane == 0 && atomicAdd(&s_past_tail, 1u) == kWarps - 1) grid_launch_dependents();
 

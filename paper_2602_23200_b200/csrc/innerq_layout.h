@@ -78,6 +78,8 @@ struct Layout {
   int max_tokens, max_splits;
   float sm_scale;
   size_t norm_off;     // float [U][D]
+  size_t appended_off; // uint32 [U]: token count of the unit after the last append (or prefill) whose writes are
+                       // complete; a decode of N tokens that reads N there may read the rings and the newest rows
   size_t cache_bytes;
   // workspace
   size_t ws_partial_off;   // float [B*Hq][max_splits][kPartialStride]

@@ -51,6 +51,10 @@ __global__ void finalize_norm_kernel(uint32_t* __restrict__ absmax, float* __res
   }
 }
 
+__global__ void fill_u32_kernel(uint32_t* p, uint32_t v, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
 __global__ void fill_float_kernel(float* p, float v, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;
@@ -288,6 +292,15 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
   append_write(L, L.v, v_x, N, u, cache);
   append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
   append_evict_block(L, L.v, N, u, cache, false, tile, words);
+  // Publish: everything this unit's append writes is written.  A decode of N tokens that reads N here (acquire)
+  // may read the rings and the newest packed rows without waiting for this kernel to end.
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(reinterpret_cast<uint32_t*>(cache + L.appended_off) + u),
+                 "r"((uint32_t)N)
+                 : "memory");
+  }
 }
 
 // Programmatic dependent launch: the decode that follows may start while this kernel runs (it streams what this
@@ -455,6 +468,9 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
       launches += 1;
     }
   }
+  // the counts the decode kernel compares with its own N (see append_unit)
+  fill_u32_kernel<<<(L.U + 255) / 256, 256, 0, st>>>(reinterpret_cast<uint32_t*>(cache + L.appended_off), (uint32_t)N, L.U);
+  launches += 1;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
