@@ -560,7 +560,9 @@ def run_ours(args, w):
                          "note": "achieved is from decodes bracketed by their own events (every 8th step), which "
                                  "cannot overlap their neighbours; in the timed loop consecutive kernels overlap "
                                  "(a whole step, append included, takes us_per_step: frac_of_step); back to back "
-                                 "the decode kernel averages us_per_decode_back_to_back",
+                                 "the decode kernel averages us_per_decode_back_to_back (time per decode of a chain "
+                                 "of launches over rotating cache instances, in which the next launch's CTAs fill "
+                                 "the slots the current one leaves idle: a rate, not one launch's duration)",
                          "frac_of_step": value_gbs / world / peak,
                          "achieved_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9,
                          "frac_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9 / peak,
