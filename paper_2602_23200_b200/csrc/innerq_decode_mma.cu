@@ -101,7 +101,6 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
     e.a.n_splits = 0;
     fill_count_args(L, e.cn, e.a);
     e.a.safe_chunks = safe_chunks_for(L, Ns_safe[i], e.cn);
-    e.a.after_append = Ns[i] != Ns_safe[i];
     e.a.n_q = 1;
     e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
     e.a.pages_host = nullptr;      // paged caches: a batched launch reads every cache's table from its buffer
@@ -139,7 +138,6 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   a.n_splits = n_splits;
   fill_count_args(L, cn, a);
   a.safe_chunks = safe_chunks_for(L, N_safe, cn);
-  a.after_append = N != N_safe;
   a.n_q = n_q;
   a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
   a.pages_host = pages_host;

@@ -423,15 +423,13 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     if (!dep_waited) { grid_dependency_wait(); dep_waited = true; }
   };
   // What the step's append writes for this unit (rings, newest packed rows) is complete when the unit's counter in
-  // the cache buffer holds this decode's N: the append publishes it (release) after its last write, long before it
-  // ends (it ends after the previous decode).  A decode that follows an append in the stream waits for its
-  // predecessor's completion (the append is most likely still at work, and that wait wakes up faster than any
-  // polling).  A decode that follows another decode looks once (acquire): the count is there, since that decode
-  // saw the append complete before it let this one start, and the warp goes on at once, while the previous decode
-  // may still be merging; should it not be there, the wait for the predecessor is always right.
+  // the cache buffer holds this decode's N: the append publishes it (release) after its last write, long before the
+  // append kernel ends (one of its CTAs stays until the previous decode has ended).  A warp looks once (acquire): if
+  // the count is there it goes on at once, while the append's other units and the previous decode's merge may still
+  // be running; if not (the append is still at work on this unit), it waits for its predecessor's completion, which
+  // is always right and wakes up faster than any polling would.
   auto wait_for_append = [&]() {
     if (dep_waited) return;
-    if (a.after_append) { dep_wait(); return; }
     const uint32_t* flag = reinterpret_cast<const uint32_t*>(a.cache + L.appended_off) + u;
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");

@@ -27,8 +27,6 @@ struct DecodeArgs {
   int safe_chunks;       // chunks [0, safe_chunks) of every unit were complete before the previous decode of this cache
                          // was launched: no kernel that may still be running writes them, so they are streamed
                          // before this kernel waits for its predecessors (programmatic dependent launch)
-  int after_append;      // tokens were appended since this cache's previous decode was launched: the kernel before this
-                         // one in the stream is (or follows) an append that may still be running
   int head0;             // first query row (within the KV head's r * n_q) handled by this launch
   int n_q;               // consecutive query tokens per sequence (1: plain decode).  Row v = i * r + h of a KV head is
                          // head h of query token i; q / out are [B, n_q, Hq, D]; query i does not see the newest

@@ -308,8 +308,9 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
 // waits for the kernels before it, either before its first global access or, with late_wait (the host knows that
 // the last kernel on this cache was a fused decode, which lets its dependents start only after its last read of
 // what an append writes: the fp16 rings and the packed rows / groups behind the range it streams), after its work:
-// it then runs while that decode streams the packed cache, and still completes after it, so that whatever follows
-// sees both finished.
+// it then runs while that decode streams the packed cache.  The kernel still completes after that decode, so that
+// whatever follows sees both finished: the CTA of unit 0 waits at its end; the others leave (and free their SM
+// slots for the next decode's first CTAs) as soon as their unit's token count is published.
 __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __restrict__ k_new,
                                                      const __half* __restrict__ v_new, int N,
                                                      unsigned char* __restrict__ cache, int late_wait) {
@@ -320,7 +321,8 @@ __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __r
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
   append_unit(L, k_new + (size_t)u * kD, v_new + (size_t)u * kD, N, u, cache, tile, words);
-  if (late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // one CTA keeps the kernel alive until its predecessor has ended (the chain of completions); the others leave
+  if (late_wait && u == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // The same for several caches of one configuration, each with its own token count: block x = sequence * U + unit,
