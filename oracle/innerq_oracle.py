@@ -74,7 +74,11 @@ def quantize_groups(x, bits: int, mode: int, sym_variant: int = FULLRANGE):
 
     Returns a dict: code uint8 [..., G] (unsigned; offset-binary for symmetric groups),
     scale_bits uint16 [...] (fp16 scale, bit 15 = M), zero_bits uint16 [...] (fp16 Z if
-    M else 0), flag bool [...], err_asym / err_sym float64 [...] (sum |x - x^|).
+    M else 0), flag bool [...], err_asym / err_sym float64 [...] (sum |x - x^|), and
+    alt_code / alt_scale_bits / alt_zero_bits: the stored form of the candidate that was
+    NOT chosen (what a group holds if M takes the other value; Figure "hybrid" computes
+    both candidates and the mask selects one).  Tests compare against it the groups whose
+    two errors are so close that float32 summation may order them the other way.
     """
     x = np.asarray(x, dtype=f32)
     L = 2 ** bits - 1
@@ -110,10 +114,14 @@ def quantize_groups(x, bits: int, mode: int, sym_variant: int = FULLRANGE):
         flag = np.ones(mn.shape, dtype=bool)
     else:
         flag = e_a < e_s          # tie -> symmetric
-    code = np.where(flag[..., None], u_a, q_s + f32(half)).astype(np.uint8)
-    scale_bits = np.where(flag, S_a.view(np.uint16) | np.uint16(0x8000), S_s.view(np.uint16)).astype(np.uint16)
-    zero_bits = np.where(flag, Z.view(np.uint16), np.uint16(0)).astype(np.uint16)
-    return dict(code=code, scale_bits=scale_bits, zero_bits=zero_bits, flag=flag, err_asym=e_a, err_sym=e_s)
+    code_a, code_s = u_a.astype(np.uint8), (q_s + f32(half)).astype(np.uint8)
+    scale_a, scale_s = (S_a.view(np.uint16) | np.uint16(0x8000)).astype(np.uint16), S_s.view(np.uint16)
+    zero_a, zero_s = Z.view(np.uint16), np.zeros(mn.shape, dtype=np.uint16)
+    pick = lambda m, a, s_: np.where(m, a, s_).astype(a.dtype)       # asymmetric candidate where m, else symmetric
+    return dict(code=pick(flag[..., None], code_a, code_s), scale_bits=pick(flag, scale_a, scale_s),
+                zero_bits=pick(flag, zero_a, zero_s), flag=flag, err_asym=e_a, err_sym=e_s,
+                alt_code=pick(~flag[..., None], code_a, code_s), alt_scale_bits=pick(~flag, scale_a, scale_s),
+                alt_zero_bits=pick(~flag, zero_a, zero_s))
 
 
 def dequantize_groups(code, scale_bits, zero_bits, bits: int):
@@ -169,6 +177,10 @@ class _Store:
         self.zero = np.zeros((U,) + n_meta, dtype=np.uint16)
         self.err_asym = np.zeros((U,) + n_meta, dtype=f64)
         self.err_sym = np.zeros((U,) + n_meta, dtype=f64)
+        # the candidate that was not chosen, in stored form (only tests read it)
+        self.alt_code = np.zeros((U, cap, D), dtype=np.uint8)
+        self.alt_scale = np.zeros((U,) + n_meta, dtype=np.uint16)
+        self.alt_zero = np.zeros((U,) + n_meta, dtype=np.uint16)
 
     # x: float32 [U, n, D] tokens to quantise (already normalised if K), n multiple of G for 'block'
     def _quantize_and_store(self, x):
@@ -179,17 +191,21 @@ class _Store:
         if self.kind == "row":
             r = quantize_groups(x.reshape(U, n, D // G, G), self.bits, self.mode, self.sym_variant)
             self.code[:, self.n_q:self.n_q + n] = r["code"].reshape(U, n, D)
+            self.alt_code[:, self.n_q:self.n_q + n] = r["alt_code"].reshape(U, n, D)
             sl = slice(self.n_q, self.n_q + n)
         else:
             assert n % G == 0 and self.n_q % G == 0
             xg = x.reshape(U, n // G, G, D).transpose(0, 1, 3, 2)       # [U, groups, D, G]
             r = quantize_groups(xg, self.bits, self.mode, self.sym_variant)
             self.code[:, self.n_q:self.n_q + n] = r["code"].transpose(0, 1, 3, 2).reshape(U, n, D)
+            self.alt_code[:, self.n_q:self.n_q + n] = r["alt_code"].transpose(0, 1, 3, 2).reshape(U, n, D)
             sl = slice(self.n_q // G, (self.n_q + n) // G)
         self.scale[:, sl] = r["scale_bits"]
         self.zero[:, sl] = r["zero_bits"]
         self.err_asym[:, sl] = r["err_asym"]
         self.err_sym[:, sl] = r["err_sym"]
+        self.alt_scale[:, sl] = r["alt_scale_bits"]
+        self.alt_zero[:, sl] = r["alt_zero_bits"]
         self.n_q += n
 
     def prefill(self, X, inv_norm):
@@ -369,6 +385,8 @@ class OracleCache:
             v_code=v.code[:, :v.n_q], v_scale=v.scale[:, :v.n_meta()], v_zero=v.zero[:, :v.n_meta()],
             k_err_asym=k.err_asym[:, :k.n_meta()], k_err_sym=k.err_sym[:, :k.n_meta()],
             v_err_asym=v.err_asym[:, :v.n_meta()], v_err_sym=v.err_sym[:, :v.n_meta()],
+            k_alt_code=k.alt_code[:, :k.n_q], k_alt_scale=k.alt_scale[:, :k.n_meta()], k_alt_zero=k.alt_zero[:, :k.n_meta()],
+            v_alt_code=v.alt_code[:, :v.n_q], v_alt_scale=v.alt_scale[:, :v.n_meta()], v_alt_zero=v.alt_zero[:, :v.n_meta()],
         )
 
 

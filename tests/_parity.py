@@ -11,6 +11,8 @@ OUT_RTOL, OUT_ATOL = 2e-3, 1e-3
 # relative margin in the oracle's float64 sums; the CUDA path sums in float32 in another order,
 # so either mask value is correct there.
 CONTEST_RTOL = 1e-4
+# Largest share of a tensor's groups that may be contested AND resolved the other way (observed: 1e-5 .. 2e-4)
+MAX_FLIP_SHARE = 4e-4
 
 
 def assert_outputs_close(out_gpu, out_ref, what=""):
@@ -30,7 +32,11 @@ def _contested(e_a, e_s):
 
 
 def assert_store_equal(g, o, name, kind, G, hybrid):
-    """Compare one tensor's canonical arrays (g: CUDA export, o: oracle export).  Returns #contested flips."""
+    """Compare one tensor's canonical arrays (g: CUDA export, o: oracle export).  Returns #contested flips.
+
+    Where both sides chose the same mask, codes, scale bits and zero bits must be identical.  Where they chose
+    differently the group must be contested, and the CUDA path's codes, scale bits and zero bits must be identical to
+    the oracle's OTHER candidate (the one its mask did not select), so every stored bit of every group is checked."""
     sc_g, sc_o = g[f"{name}_scale"], o[f"{name}_scale"]
     assert sc_g.shape == sc_o.shape, (name, sc_g.shape, sc_o.shape)
     flag_g, flag_o = (sc_g & 0x8000) != 0, (sc_o & 0x8000) != 0
@@ -40,20 +46,22 @@ def assert_store_equal(g, o, name, kind, G, hybrid):
         assert hybrid, f"{name}: mask differs in a non-hybrid mode"
         cont = _contested(o[f"{name}_err_asym"], o[f"{name}_err_sym"])
         assert np.all(cont[flips]), f"{name}: {int((flips & ~cont).sum())} uncontested groups chose another mode"
-        assert n_flips <= max(2, int(2e-3 * flips.size)), f"{name}: too many contested flips ({n_flips})"
-    same = ~flips
-    assert np.array_equal(sc_g[same], sc_o[same]), f"{name}_scale"
-    assert np.array_equal(g[f"{name}_zero"][same], o[f"{name}_zero"][same]), f"{name}_zero"
+        assert n_flips <= max(2, int(MAX_FLIP_SHARE * flips.size)), f"{name}: too many contested flips ({n_flips})"
+    # expected stored form per group: the oracle's chosen candidate, or its other one where the masks differ
+    sc_e = np.where(flips, o[f"{name}_alt_scale"], sc_o)
+    ze_e = np.where(flips, o[f"{name}_alt_zero"], o[f"{name}_zero"])
+    assert np.array_equal(sc_g, sc_e), f"{name}_scale"
+    assert np.array_equal(g[f"{name}_zero"], ze_e), f"{name}_zero"
     # zero-point is 0 wherever the mask is 0
     assert not np.any(g[f"{name}_zero"][~flag_g])
     cg, co = g[f"{name}_code"], o[f"{name}_code"]
     assert cg.shape == co.shape
     U, n, D = cg.shape
     if kind == "row":
-        same_e = np.repeat(same, G, axis=-1).reshape(U, n, D)
+        flips_e = np.repeat(flips, G, axis=-1).reshape(U, n, D)
     else:
-        same_e = np.repeat(same, G, axis=1).reshape(U, n, D)
-    assert np.array_equal(cg[same_e], co[same_e]), f"{name}_code"
+        flips_e = np.repeat(flips, G, axis=1).reshape(U, n, D)
+    assert np.array_equal(cg, np.where(flips_e, o[f"{name}_alt_code"], co)), f"{name}_code"
     return n_flips
 
 

@@ -211,6 +211,9 @@ def test_hybrid_is_the_better_of_the_two_modes(bits, variant):
     for name in ("code", "scale_bits", "zero_bits"):
         assert np.array_equal(rh[name][flag], ra[name][flag])
         assert np.array_equal(rh[name][~flag], rs[name][~flag])
+        # the candidate hybrid did not choose is the other pure mode's result, for every group
+        assert np.array_equal(rh["alt_" + name][flag], rs[name][flag])
+        assert np.array_equal(rh["alt_" + name][~flag], ra[name][~flag])
     assert not np.any(rh["zero_bits"][~flag])
     xh = O.dequantize_groups(rh["code"], rh["scale_bits"], rh["zero_bits"], bits)
     assert np.allclose(np.abs(x - xh).sum(1), np.minimum(ea, es), rtol=1e-12)
