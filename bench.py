@@ -10,6 +10,16 @@ The packed cache of that workload (about 100 MB) would fit in the 126 MB L2, so 
 over several independent cache instances (same contents, different memory; total several times
 the L2 size) and step i uses instance i mod R: every decode streams its cache from HBM.
 
+What is timed (all with CUDA events on the launching stream, after untimed warm steps that run
+straight into the timed ones):
+  * `value`, `ms_per_step`: EXACTLY --steps steps of append + decode between two events;
+  * `us_per_step_fixed_leg`: the same loop over a fixed number of steps, whatever --steps says;
+  * `roofline`: the decode kernel alone, 48 launches each between its own events, MEDIAN;
+  * `us_per_decode_back_to_back`: a chain of decode launches;
+  * `e2e`: the host-buffer entry point, one step at a time with a synchronisation per step;
+  * `per_config`: the long-context GQA workload (decode alone / chained / step and the full prefill
+    quantisation) and the batch-16 GQA workload at 4 and 2 bits, same legs.
+
 Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead (host cores).
 """
 from __future__ import annotations
@@ -84,7 +94,6 @@ def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
     row_q, blk_q = mid, (mid // G) * G
     n_qk, n_qv = (row_q, blk_q) if w.grouping == synth.INNER else (blk_q, row_q)
     kb, vb = payload_bytes(w)
-    n_sink = min(N, ws)
     per_unit = n_qk * kb + n_qv * vb + (N - n_qk) * 2 * D + (N - n_qv) * 2 * D
     extra = 2 * w.batch * w.n_q_heads * D * 2 + (U * D * 4 if w.k_normalize else 0)
     dense = U * per_unit + extra
@@ -93,7 +102,6 @@ def decode_algorithmic_bytes(w, N, sym_frac_k=0.0, sym_frac_v=0.0):
     k_has_z = (w.k_mode != synth.SYM) or w.grouping == synth.OUTER
     v_has_z = (w.v_mode != synth.SYM) or w.grouping == synth.OUTER
     minimal = dense - U * 2 * (k_groups * sym_frac_k * k_has_z + v_groups * sym_frac_v * v_has_z)
-    del n_sink
     return float(dense), float(minimal)
 
 
@@ -232,8 +240,6 @@ def run_reference(args, w):
     if rank != 0:
         return
     units = min(w.n_units, 4)
-    for _ in range(args.warmup and 1):
-        pass
     t, b, cores, _ = oracle_steps(w, max(1, min(args.steps, 8)), units=units)
     gbs = b / t / 1e9
     line = {"impl": "reference", "metric": "decode_step_algorithmic_hbm_gbs", "value": gbs, "unit": "GB/s",
@@ -272,6 +278,196 @@ def whole_job_gbs(bytes_per_step_per_rank: float, seconds_per_step: float, world
 
 
 # ------------------------------------------------------------------------------------- CUDA arm
+class Legs:
+    """Timed legs over a set of cache instances of one workload (rotated so that every decode streams from HBM).
+
+    Every leg starts behind a short device-side delay (`torch.cuda._sleep`), recorded BEFORE the leg's first event,
+    so that the host has its launches queued when the GPU reaches them: what the events then bracket is device time,
+    the way a serving loop that runs ahead of the GPU sees it, not the host's launch latency from an idle stream."""
+
+    def __init__(self, w, caches, k_new, v_new, q_all, out, first_step=0):
+        import torch
+        self.torch, self.w, self.caches, self.R = torch, w, caches, len(caches)
+        self.k_new, self.v_new, self.q_all, self.out = k_new, v_new, q_all, out
+        self.stream = torch.cuda.current_stream()
+        self.i = first_step                 # index of the next unused (k_new, v_new, q) triple
+
+    def _ev(self):
+        return self.torch.cuda.Event(enable_timing=True)
+
+    def delay(self, cycles=300_000):
+        self.torch.cuda._sleep(cycles)      # ~0.15 ms at 1.9 GHz; outside every timed region
+
+    def step(self):
+        i = self.i
+        c = self.caches[i % self.R]
+        c.innerq_append_token(self.k_new[i], self.v_new[i])
+        c.innerq_decode_attention(self.q_all[i], self.out)
+        self.i += 1
+        return c
+
+    def steps(self, n, warm=0):
+        """n steps (append + decode) between two events, after `warm` untimed steps that run straight into them."""
+        self.delay()
+        for _ in range(warm):
+            self.step()
+        e0, e1 = self._ev(), self._ev()
+        e0.record(self.stream)
+        for _ in range(n):
+            self.step()
+        e1.record(self.stream)
+        self.torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n
+
+    def decodes_bracketed(self, n):
+        """n decodes, each between its own pair of events (no overlap with its neighbours).  Returns a list of us."""
+        evs = [(self._ev(), self._ev()) for _ in range(n)]
+        self.delay()
+        for j in range(4):                                      # untimed, so that the first bracket is not the coldest
+            self.caches[j % self.R].innerq_decode_attention(self.q_all[j], self.out)
+        for j, (a, b) in enumerate(evs):
+            a.record(self.stream)
+            self.caches[j % self.R].innerq_decode_attention(self.q_all[j % len(self.q_all)], self.out)
+            b.record(self.stream)
+        self.torch.cuda.synchronize()
+        return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+    def decodes_chained(self, n, caches=None, call=None):
+        """n decodes launched back to back over the rotating instances: us per decode of the chain."""
+        caches = caches or self.caches
+        call = call or (lambda c, j: c.innerq_decode_attention(self.q_all[j % len(self.q_all)], self.out))
+        self.delay()
+        for j in range(4):
+            call(caches[j % len(caches)], j)
+        e0, e1 = self._ev(), self._ev()
+        e0.record(self.stream)
+        for j in range(n):
+            call(caches[j % len(caches)], j)
+        e1.record(self.stream)
+        self.torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n
+
+    def appends_bracketed(self, n):
+        evs = [(self._ev(), self._ev()) for _ in range(n)]
+        self.delay()
+        for j, (a, b) in enumerate(evs):
+            i = self.i
+            a.record(self.stream)
+            self.caches[i % self.R].innerq_append_token(self.k_new[i], self.v_new[i])
+            b.record(self.stream)
+            self.i += 1
+        self.torch.cuda.synchronize()
+        return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+    def steps_one_by_one(self, n):
+        """n steps, each between its own events; returns (us list, mask of the steps that evict a group of G tokens)."""
+        w = self.w
+        evs = [(self._ev(), self._ev()) for _ in range(n)]
+        evict = []
+        self.delay()
+        for a, b in evs:
+            n_before = self.caches[self.i % self.R].n_tokens
+            a.record(self.stream)
+            self.step()
+            b.record(self.stream)
+            mid0, mid1 = n_before - w.w_sink - w.w_recent, n_before + 1 - w.w_sink - w.w_recent
+            evict.append(mid1 > 0 and mid1 // w.group > max(mid0, 0) // w.group)
+        self.torch.cuda.synchronize()
+        return np.array([a.elapsed_time(b) * 1e3 for a, b in evs]), np.array(evict)
+
+
+def stats(us):
+    us = np.asarray(us, dtype=np.float64)
+    return {"median": float(np.median(us)), "min": float(us.min()), "mean": float(us.mean()), "n": int(us.size)}
+
+
+def make_inputs(w, n):
+    import torch
+    toks = [synth.new_token(w, s) for s in range(n)]
+    qs = [synth.query(w, s) for s in range(n)]
+    kh, vh, qh = np.stack([t[0] for t in toks]), np.stack([t[1] for t in toks]), np.stack(qs)
+    return (kh, vh, qh), (torch.from_numpy(kh).cuda(), torch.from_numpy(vh).cuda(), torch.from_numpy(qh).cuda())
+
+
+def kv_device(w, tiled):
+    """fp16 K, V of the workload on the device.  tiled: batch entry 0 is generated and repeated over the batch
+    (host generation time of the large shapes; units are independent, so timings do not depend on it)."""
+    import torch
+    if tiled and w.batch > 1:
+        K1, V1 = synth.kv_all(w.with_(batch=1))
+        Kd, Vd = torch.from_numpy(K1).cuda(), torch.from_numpy(V1).cuda()
+        return Kd.expand(w.batch, -1, -1, -1).contiguous(), Vd.expand(w.batch, -1, -1, -1).contiguous()
+    Kh, Vh = synth.kv_all(w)
+    return torch.from_numpy(Kh).cuda(), torch.from_numpy(Vh).cuda()
+
+
+def sym_fractions(cache):
+    ex = cache.innerq_cache_export(codes=False)
+    f = lambda a: float(1.0 - ((a & 0x8000) != 0).mean()) if a is not None and a.size else 0.0
+    return f(ex.get("k_scale")), f(ex.get("v_scale"))
+
+
+def prefill_algorithmic_bytes(w):
+    """Bytes a prefill quantisation must move: fp16 K and V read once, the packed cache and the windows written."""
+    U, N = w.n_units, w.n_tokens
+    dense, _ = decode_algorithmic_bytes(w, N)
+    return float(U * N * D * 2 * 2 + dense)
+
+
+def measure_config(name, peak, R=2, n_steps=128):
+    """One more workload for the line's `per_config` block: decode alone / chained, the step, and (c4) the prefill."""
+    import torch
+    from paper_2602_23200_b200 import binding as B
+    w = workload_by_name(name)
+    n_in = 32 + n_steps + 8
+    cfg = B.make_config(w, max_tokens=w.n_tokens + n_in // R + 16)
+    Kd, Vd = kv_device(w, tiled=True)
+    caches = []
+    pre_us = []
+    for _ in range(R):
+        c = B.InnerQCache(cfg)
+        c.innerq_quantize_prefill(Kd, Vd)
+        caches.append(c)
+    res = {"config": {"batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "context": w.n_tokens,
+                      "bits": w.k_bits, "group": w.group, "instances_rotated": R}}
+    if name == "c4":
+        # the full prefill quantisation of the 131072-token cache, each call between its own events
+        for rep in range(4):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            caches[rep % R].innerq_quantize_prefill(Kd, Vd)
+            e1.record()
+            torch.cuda.synchronize()
+            pre_us.append(e0.elapsed_time(e1) * 1e3)
+        pb = prefill_algorithmic_bytes(w)
+        med = float(np.median(pre_us[1:]))
+        res["prefill"] = {"us": stats(pre_us[1:]), "algorithmic_bytes": pb, "gbs": pb / med / 1e3,
+                          "frac_of_measured_peak": pb / med / 1e3 / peak, "pct_of_nominal_8TBs": pb / med / 1e3 / 80.0,
+                          "launches": caches[0].innerq_last_launch_count(0)}
+    sym_k, sym_v = sym_fractions(caches[0])
+    del Kd, Vd
+    torch.cuda.empty_cache()
+    _, (k_new, v_new, q_all) = make_inputs(w, n_in)
+    legs = Legs(w, caches, k_new, v_new, q_all, torch.empty_like(q_all[0]))
+    nbytes = decode_algorithmic_bytes(w, w.n_tokens + 1, sym_k, sym_v)[1]
+    alone = stats(legs.decodes_bracketed(32))
+    chain = legs.decodes_chained(64)
+    step = legs.steps(n_steps, warm=32)
+    gbs = lambda us: nbytes / us / 1e3
+    res.update({
+        "bytes_per_decode_minimal": nbytes, "sym_group_fraction": {"k": sym_k, "v": sym_v},
+        "us_per_decode_alone": alone, "us_per_decode_chained": chain, "us_per_step": step,
+        "frac_of_measured_peak": {"alone_median": gbs(alone["median"]) / peak, "chained": gbs(chain) / peak,
+                                  "step": gbs(step) / peak},
+        "pct_of_nominal_8TBs": {"alone_median": gbs(alone["median"]) / 80.0, "chained": gbs(chain) / 80.0,
+                                "step": gbs(step) / 80.0},
+    })
+    for c in caches:
+        assert c.innerq_read_device_error() == 0
+        c.close()
+    return res
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -287,12 +483,14 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     R, Kst, W = args.instances, args.steps, max(args.warmup, 3)
-    total_steps = W + Kst
+    packed = w.grouping != synth.FP16
+    WARM = 64                       # untimed steps that run straight into the timed region (besides the W warm-up steps)
+    LEG = args.leg_steps            # the step-rate leg that does not depend on --steps
     e2e_steps = max(4, min(Kst, 32))
-    split_steps = 2 * R * w.group if w.grouping != synth.FP16 else 0     # extra steps timed one by one (below)
-    cfg = B.make_config(w, max_tokens=w.n_tokens + (total_steps + e2e_steps + split_steps) // R + 16)
-    Kh, Vh = synth.kv_all(w)
-    Kd, Vd = torch.from_numpy(Kh).cuda(), torch.from_numpy(Vh).cuda()
+    split_steps = 2 * R * w.group if packed else 0           # steps timed one by one (below)
+    n_in = W + WARM + Kst + 32 + LEG + e2e_steps + split_steps + 16
+    cfg = B.make_config(w, max_tokens=w.n_tokens + n_in // R + 16)
+    Kd, Vd = kv_device(w, tiled=False)
     caches = []
     for _ in range(R):
         c = B.InnerQCache(cfg)
@@ -300,14 +498,11 @@ def run_ours(args, w):
         if args.splits or args.variant:
             c.innerq_set_decode_options(args.splits, args.variant)
         caches.append(c)
-    # fraction of symmetric groups (their zero-points are not needed by the result)
-    ex = caches[0].innerq_cache_export(codes=False)
-    sym_k = float(1.0 - ((ex["k_scale"] & 0x8000) != 0).mean()) if "k_scale" in ex and ex["k_scale"].size else 0.0
-    sym_v = float(1.0 - ((ex["v_scale"] & 0x8000) != 0).mean()) if "v_scale" in ex and ex["v_scale"].size else 0.0
+    sym_k, sym_v = sym_fractions(caches[0]) if packed else (0.0, 0.0)
     # information only: how far the quantised cache moves the attention output away from the unquantised one
     # (relative L2 over all heads, same q), measured against the library's fp16 cache of the same inputs
     rel_l2 = None
-    if w.grouping != synth.FP16:
+    if packed:
         wf = w.with_(grouping=synth.FP16, k_normalize=0)
         ref_cache = B.InnerQCache(B.make_config(wf, max_tokens=w.n_tokens + 8))
         ref_cache.innerq_quantize_prefill(Kd, Vd)
@@ -317,9 +512,17 @@ def run_ours(args, w):
         rel_l2 = float(((o_q - o_ref).norm() / o_ref.norm()).item())
         ref_cache.close()
         del ref_cache, o_ref, o_q
+    # the paper-literal symmetric variant (clipped signed range): the regime in which most groups stay symmetric
+    literal_caches = []
+    if packed and args.literal and w.sym_variant == 0 and (w.k_mode == synth.HYBRID or w.v_mode == synth.HYBRID):
+        cfg_l = B.make_config(w.with_(sym_variant=1), max_tokens=w.n_tokens + 16)
+        for _ in range(R):
+            c = B.InnerQCache(cfg_l)
+            c.innerq_quantize_prefill(Kd, Vd)
+            literal_caches.append(c)
     # sequences of different lengths, one cache object each, decoded by one batched call (information; needs a batch)
     ragged_sets, ragged_lengths = [], []
-    if w.batch > 1 and w.grouping != synth.FP16 and args.ragged:
+    if w.batch > 1 and packed and args.ragged:
         fracs = [1.0, 0.125, 0.5, 0.25, 0.75, 1.0, 0.375, 0.625]
         ragged_lengths = [max(w.w_sink + w.w_recent + w.group, int(w.n_tokens * fracs[i % len(fracs)])) for i in range(w.batch)]
         w1 = w.with_(batch=1)
@@ -335,7 +538,7 @@ def run_ours(args, w):
     # the same caches with their packed records in pages of a shared pool, pages handed out in a shuffled order
     # (information: what the page table costs the decode kernel)
     paged_caches = []
-    if args.paged and w.grouping != synth.FP16:
+    if args.paged and packed:
         per_cache = -(-cfg.max_tokens // args.paged) + 1
         order = np.random.default_rng(5).permutation(R * per_cache)
         pool = B.PagePool(cfg, args.paged, R * per_cache, order=order)
@@ -344,148 +547,104 @@ def run_ours(args, w):
             c.ensure_pages(w.n_tokens)
             c.innerq_quantize_prefill(Kd, Vd)
             paged_caches.append(c)
-    del Kd, Vd, Kh, Vh, ex
+    del Kd, Vd
     torch.cuda.empty_cache()
 
-    n_in = total_steps + e2e_steps + split_steps
-    toks = [synth.new_token(w, s) for s in range(n_in)]
-    qs = [synth.query(w, s) for s in range(n_in)]
-    k_new = torch.from_numpy(np.stack([t[0] for t in toks])).cuda()
-    v_new = torch.from_numpy(np.stack([t[1] for t in toks])).cuda()
-    q_all = torch.from_numpy(np.stack(qs)).cuda()
+    (kh_np, vh_np, qh_np), (k_new, v_new, q_all) = make_inputs(w, n_in)
     out = torch.empty_like(q_all[0])
-    stream = torch.cuda.current_stream()
-
-    def step(i):
-        c = caches[i % R]
-        c.innerq_append_token(k_new[i], v_new[i])
-        c.innerq_decode_attention(q_all[i], out)
-        return c
+    legs = Legs(w, caches, k_new, v_new, q_all, out)
+    stream = legs.stream
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(W):
-        step(i)
+    # ---- the timed region of the contract: W warm-up steps, then EXACTLY Kst steps between two events --------
+    for _ in range(W):
+        legs.step()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    time.sleep(0.15)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # The decode kernel is bracketed by its own events on every 8th step only: an event between append and decode
-    # keeps the decode from being launched as a programmatic dependent of the append, so the other steps run the
-    # way a serving loop would.  The bracketed decodes are the ones the roofline figure is computed from.
-    ev_every = 8
-    dec_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range((Kst + ev_every - 1) // ev_every)]
+    time.sleep(0.05)
     barrier()
+    legs.delay()
+    for _ in range(WARM):           # untimed; they run straight into the timed steps, so those start on a busy GPU
+        legs.step()
+    i_first = legs.i
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
-    for j in range(Kst):
-        i = W + j
-        c = caches[i % R]
-        c.innerq_append_token(k_new[i], v_new[i])
-        if j % ev_every == 0:
-            dec_ev[j // ev_every][0].record(stream)
-            c.innerq_decode_attention(q_all[i], out)
-            dec_ev[j // ev_every][1].record(stream)
-        else:
-            c.innerq_decode_attention(q_all[i], out)
+    for _ in range(Kst):
+        legs.step()
     ev1.record(stream)
     barrier()
-    clocks = sampler.stop()
-    # bookkeeping outside the timed region: launches and bytes per step follow from N alone
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), "cuda")
+    ms_step = ms_total / Kst
     launches = Kst * (caches[0].innerq_last_launch_count(1) + caches[0].innerq_last_launch_count(2))
     bytes_dense = bytes_min = 0.0
-    n_now = [w.n_tokens + (W + Kst - 1 - r) // R + 1 for r in range(R)]       # tokens per cache after the loop
-    for j in range(Kst):
-        i = W + j
-        n_step = w.n_tokens + i // R + 1
-        bd, bm = decode_algorithmic_bytes(w, n_step, sym_k, sym_v)
+    for i in range(i_first, i_first + Kst):
+        bd, bm = decode_algorithmic_bytes(w, w.n_tokens + i // R + 1, sym_k, sym_v)
         bytes_dense += bd
         bytes_min += bm
-    assert all(caches[r].n_tokens == n_now[r] for r in range(R))
-    ms_total = ev0.elapsed_time(ev1)
-    dec_ms = [a.elapsed_time(b) for a, b in dec_ev]
-    ms_total = max_over_ranks(ms_total, "cuda")
-    ms_step = ms_total / Kst
-    value_gbs = whole_job_gbs(bytes_min / Kst, ms_step * 1e-3, world)
+    bytes_dense /= Kst
+    bytes_min /= Kst                 # bytes per decode vary by < 0.1 % over the whole run
+    value_gbs = whole_job_gbs(bytes_min, ms_step * 1e-3, world)
+    # ---- the same step loop over a fixed number of steps (does not depend on --steps) ------------------------
+    leg_us = legs.steps(LEG, warm=32)
+    # ---- the decode kernel alone: every launch between its own events (the roofline figure), and chained -------
+    alone = stats(legs.decodes_bracketed(48))
+    b2b_us = legs.decodes_chained(64)
+    clocks = sampler.stop()
+    assert all(c.n_tokens == w.n_tokens + (legs.i - 1 - r) // R + 1 for r, c in enumerate(caches))
 
-    # end to end: host buffers in, host buffer out, copies inside the timed region
-    kh = torch.from_numpy(np.stack([t[0] for t in toks])).pin_memory()
-    vh = torch.from_numpy(np.stack([t[1] for t in toks])).pin_memory()
-    qh = torch.from_numpy(np.stack(qs)).pin_memory()
+    # ---- end to end: host buffers in, host buffer out, through the C-ABI call that takes host pointers --------
+    kh = torch.from_numpy(kh_np).pin_memory()
+    vh = torch.from_numpy(vh_np).pin_memory()
+    qh = torch.from_numpy(qh_np).pin_memory()
     oh = torch.empty_like(qh[0]).pin_memory()
 
-    def e2e_step(i):
-        # the C-ABI call with host buffers: three host -> device copies, append, decode, device -> host copy
+    def e2e_step():
+        i = legs.i
         c = caches[i % R]
         c.innerq_decode_step_host(kh[i], vh[i], qh[i], oh)
         torch.cuda.synchronize()
+        legs.i += 1
         return c
 
-    base = total_steps
-    e2e_step(base)
+    e2e_step()
     barrier()
     t0 = time.perf_counter()
     e2e_bytes = 0.0
-    for j in range(1, e2e_steps):
-        c = e2e_step(base + j)
+    for _ in range(1, e2e_steps):
+        c = e2e_step()
         e2e_bytes += decode_algorithmic_bytes(w, c.n_tokens, sym_k, sym_v)[1]
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / (e2e_steps - 1)
     e2e_s = max_over_ranks(e2e_s, "cuda")
     e2e_gbs = whole_job_gbs(e2e_bytes / (e2e_steps - 1), e2e_s, world)
-    # decode kernel alone, launches back to back (no host work between them), same rotation over instances
-    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    nb = max(16, min(Kst, 64))
-    barrier()
-    b0.record(stream)
-    for i in range(nb):
-        caches[i % R].innerq_decode_attention(q_all[i % len(qs)], out)
-    b1.record(stream)
-    torch.cuda.synchronize()
-    b2b_us = b0.elapsed_time(b1) / nb * 1e3
+    h2d = (kh[0].numel() + vh[0].numel() + qh[0].numel()) * 2
+    d2h = oh.numel() * 2
+
+    # ---- information legs ----------------------------------------------------------------------------------
     paged = None
     if paged_caches:
-        for c in paged_caches:
-            c.innerq_decode_attention(q_all[0], out)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        p0.record(stream)
-        for i in range(nb):
-            paged_caches[i % R].innerq_decode_attention(q_all[i % len(qs)], out)
-        p1.record(stream)
-        torch.cuda.synchronize()
         paged = {"page_tokens": args.paged, "pages_per_cache": paged_caches[0].pages_assigned,
-                 "page_bytes": pool.page_bytes, "us_per_decode_back_to_back": p0.elapsed_time(p1) / nb * 1e3,
+                 "page_bytes": pool.page_bytes, "us_per_decode_back_to_back": legs.decodes_chained(64, caches=paged_caches),
                  "contiguous_us_per_decode_back_to_back": b2b_us}
-    # the append kernel alone, each call between its own events (extra tokens beyond the timed steps)
-    app_n = 16
-    app_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(app_n)]
-    for j in range(app_n):
-        i = total_steps + e2e_steps + split_steps + j
-        app_ev[j][0].record(stream)
-        caches[j % R].innerq_append_token(k_new[i % n_in], v_new[i % n_in])
-        app_ev[j][1].record(stream)
-    torch.cuda.synchronize()
-    append_us = float(np.median([a.elapsed_time(b) for a, b in app_ev])) * 1e3
-    # several query tokens per sequence in one call (causal among the newest n_q tokens), back to back like the above
+    literal = None
+    if literal_caches:
+        lk, lv = sym_fractions(literal_caches[0])
+        literal = {"sym_group_fraction": {"k": lk, "v": lv},
+                   "bytes_per_decode_minimal": decode_algorithmic_bytes(w.with_(sym_variant=1), w.n_tokens, lk, lv)[1],
+                   "us_per_decode_back_to_back": legs.decodes_chained(64, caches=literal_caches)}
+        for c in literal_caches:
+            c.close()
+    append_us = float(np.median(legs.appends_bracketed(16)))
     multi = None
-    if args.n_q > 1 and w.grouping != synth.FP16:
-        qm = torch.stack([q_all[i % len(qs)] for i in range(args.n_q)], dim=1).contiguous()     # [B, n_q, Hq, D]
+    if args.n_q > 1 and packed:
+        qm = torch.stack([q_all[i] for i in range(args.n_q)], dim=1).contiguous()     # [B, n_q, Hq, D]
         om = torch.empty_like(qm)
-        for i in range(R):
-            caches[i].innerq_decode_attention_multi(qm, om)
-        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        m0.record(stream)
-        for i in range(nb):
-            caches[i % R].innerq_decode_attention_multi(qm, om)
-        m1.record(stream)
-        torch.cuda.synchronize()
-        multi_us = m0.elapsed_time(m1) / nb * 1e3
+        multi_us = legs.decodes_chained(64, call=lambda c, j: c.innerq_decode_attention_multi(qm, om))
         multi = {"n_q": args.n_q, "us_per_call_back_to_back": multi_us, "us_per_query_token": multi_us / args.n_q,
                  "launches_per_call": caches[0].innerq_last_launch_count(2),
                  "single_query_us_back_to_back": b2b_us}
@@ -493,16 +652,8 @@ def run_ours(args, w):
     if ragged_sets:
         qr = q_all[0].reshape(w.batch, 1, w.n_q_heads, w.head_dim).contiguous()
         outr = torch.empty_like(qr)
-        for cs in ragged_sets:
-            B.innerq_decode_attention_batched(cs, qr, outr)
-        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        r0.record(stream)
-        for i in range(nb):
-            B.innerq_decode_attention_batched(ragged_sets[i % len(ragged_sets)], qr, outr)
-        r1.record(stream)
-        torch.cuda.synchronize()
-        ragged_us = r0.elapsed_time(r1) / nb * 1e3
+        ragged_us = legs.decodes_chained(64, caches=ragged_sets,
+                                         call=lambda cs, j: B.innerq_decode_attention_batched(cs, qr, outr))
         tok = sum(ragged_lengths)
         ragged = {"lengths": ragged_lengths, "us_per_call_back_to_back": ragged_us,
                   "tokens_per_call": tok * w.n_kv_heads,
@@ -511,66 +662,65 @@ def run_ours(args, w):
         for cs in ragged_sets:
             for c in cs:
                 c.close()
-    # steps timed one by one (events around append + decode): those on which a value group (inner grouping) or a key
-    # group (outer grouping) of G tokens is quantised, against the others
+    # steps timed one by one: those on which a value group (inner grouping) or a key group (outer grouping) of G
+    # tokens is quantised, against the others
     step_split = None
     if split_steps:
-        base2 = total_steps + e2e_steps
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(split_steps)]
-        evict = []
-        for j in range(split_steps):
-            i = base2 + j
-            c = caches[i % R]
-            n_before = c.n_tokens
-            evs[j][0].record(stream)
-            c.innerq_append_token(k_new[i], v_new[i])
-            c.innerq_decode_attention(q_all[i], out)
-            evs[j][1].record(stream)
-            mid0, mid1 = n_before - w.w_sink - w.w_recent, n_before + 1 - w.w_sink - w.w_recent
-            evict.append(mid1 > 0 and mid1 // w.group > max(mid0, 0) // w.group)
-        torch.cuda.synchronize()
-        t_us = np.array([a_.elapsed_time(b_) * 1e3 for a_, b_ in evs])
-        ev_mask = np.array(evict)
+        t_us, ev_mask = legs.steps_one_by_one(split_steps)
         step_split = {"steps": split_steps, "group_eviction_steps": int(ev_mask.sum()),
                       "us_median_group_eviction": float(np.median(t_us[ev_mask])) if ev_mask.any() else None,
                       "us_median_other": float(np.median(t_us[~ev_mask])) if (~ev_mask).any() else None}
-    h2d = (kh[0].numel() + vh[0].numel() + qh[0].numel()) * 2
-    d2h = oh.numel() * 2
+    dev_err = max(c.innerq_read_device_error() for c in caches)
+    for c in caches + paged_caches:
+        c.close()
+    del caches, paged_caches, legs
+    torch.cuda.empty_cache()
 
     if rank == 0:
         peak, which = measured_peak_gbs()
-        dec_us = float(np.mean(dec_ms)) * 1e3
-        achieved = (bytes_min / Kst) / (dec_us * 1e-6) / 1e9      # bytes per decode vary by < 0.1 % over the steps
+        gbs = lambda us: bytes_min / us / 1e3
+        achieved = gbs(alone["median"])
+        counters = stored_counters(w.name)
         line = {
             "metric": "decode_step_algorithmic_hbm_gbs", "value": value_gbs, "unit": "GB/s", "n_gpus": world,
             "steps": Kst, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
-            "us_per_decode": dec_us, "us_per_decode_median": float(np.median(dec_ms)) * 1e3,
-            "us_per_decode_min": float(np.min(dec_ms)) * 1e3, "us_per_decode_back_to_back": b2b_us,
+            "us_per_step_fixed_leg": {"steps": LEG, "us": leg_us, "frac_of_measured_peak": gbs(leg_us) / peak},
+            "us_per_decode": alone["median"], "us_per_decode_alone": alone, "us_per_decode_back_to_back": b2b_us,
             "us_per_append_median": append_us,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config_dict(w, args),
-            "bytes_per_decode": {"dense_zero_points": bytes_dense / Kst, "minimal": bytes_min / Kst,
+            "bytes_per_decode": {"dense_zero_points": bytes_dense, "minimal": bytes_min,
                                  "sym_group_fraction": {"k": sym_k, "v": sym_v}},
-            "info": {"rel_l2_vs_fp16_cache_attention": rel_l2},
-            "second_roof": pipe_roofs_gbs(stored_counters(w.name), bytes_min / Kst, clocks.get("sm_mhz")),
+            "info": {"rel_l2_vs_fp16_cache_attention": rel_l2, "device_error_word": dev_err,
+                     "untimed_steps_before_the_timed_region": W + WARM},
+            "paper_literal_sym_variant": literal,
+            "second_roof": pipe_roofs_gbs(counters, bytes_min, clocks.get("sm_mhz")),
             "step_us_by_kind": step_split, "multi_query": multi, "ragged_batch": ragged, "paged_cache": paged,
-            "pct_of_nominal_8TBs": 100.0 * achieved / 8000.0,
+            "pct_of_nominal_8TBs": {"decode_alone_median": achieved / 80.0, "decode_back_to_back": gbs(b2b_us) / 80.0,
+                                    "step": value_gbs / world / 80.0},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
-                         "note": "achieved is from decodes bracketed by their own events (every 8th step), which "
-                                 "cannot overlap their neighbours; in the timed loop consecutive kernels overlap "
-                                 "(a whole step, append included, takes us_per_step: frac_of_step); back to back "
-                                 "the decode kernel averages us_per_decode_back_to_back (time per decode of a chain "
-                                 "of launches over rotating cache instances, in which the next launch's CTAs fill "
-                                 "the slots the current one leaves idle: a rate, not one launch's duration)",
+                         "traffic_source": ("stored: ncu capture of one launch of this workload, "
+                                            + str((counters or {}).get("captured_at", "profiles/decode_counters.json")))
+                         if counters else None,
+                         "note": "achieved = algorithmic bytes of one decode / MEDIAN duration of 48 decode launches "
+                                 "that are each bracketed by their own events (us_per_decode_alone), so none "
+                                 "overlaps its neighbours; in the step loop consecutive kernels overlap (a whole "
+                                 "step, append included, takes us_per_step: frac_of_step); launched back to back "
+                                 "the decode kernel averages us_per_decode_back_to_back (a rate: the next "
+                                 "launch's CTAs fill the slots the current one leaves idle)",
                          "frac_of_step": value_gbs / world / peak,
-                         "achieved_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9,
-                         "frac_back_to_back": (bytes_min / Kst) / (b2b_us * 1e-6) / 1e9 / peak,
+                         "achieved_back_to_back": gbs(b2b_us), "frac_back_to_back": gbs(b2b_us) / peak,
                          "kernel": "innerq_decode_attention (split + merge)"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "us_per_step": e2e_s * 1e6, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": launches, "clocks": clocks,
         }
+        if args.per_config and world == 1:
+            line["per_config"] = {}
+            for name in args.per_config.split(","):
+                if name and workload_by_name(name).name != w.name:
+                    line["per_config"][name] = measure_config(name, peak)
         if not args.no_cpu_baseline and world == 1:
             units = min(w.n_units, 4)
             t, b, cores, extra = oracle_steps(w, 3, units=units)
@@ -589,7 +739,7 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1024)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
@@ -600,6 +750,10 @@ def main():
     ap.add_argument("--paged", type=int, default=1024, help="page size in tokens of the paged-cache leg (0: skip it)")
     ap.add_argument("--ragged", type=int, default=1, help="1: also time a batched decode over sequences of mixed lengths")
     ap.add_argument("--n-q", type=int, default=4, help="query tokens per call of the multi-query leg (0/1: skip it)")
+    ap.add_argument("--leg-steps", type=int, default=512, help="steps of the step-rate leg that does not depend on --steps")
+    ap.add_argument("--literal", type=int, default=1, help="1: also report the paper-literal symmetric variant")
+    ap.add_argument("--per-config", default="c4,c3_4bit,c3_2bit",
+                    help="further workloads measured into the line's per_config block ('' to skip)")
     args = ap.parse_args()
     w = workload_by_name(args.workload)
     if args.impl == "reference":

@@ -263,7 +263,11 @@ int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, co
  *   - All caches and all calls on a device share the one array, which keeps the contents of the previous
  *     call; the parts that must start at zero are cleared on `cuda_stream` before the launch.  Two such
  *     calls must not overlap on the GPU (different streams without ordering): they would race on the array.
- *   - The caller's workspace is not touched, so innerq_read_device_error does not see this call.
+ *   - The array that is used belongs to the CURRENT device: the cache must live on it (INVALID_ARG if not).
+ *   - The caller's workspace is not touched.  The error word of this call is in the array as well;
+ *     innerq_read_device_error (called with the same device current) reports it together with the
+ *     workspace's own word.  It tells about the last such call only: the next one clears it.
+ *   - Decode variant 5 (tcgen05 kernel) is not served from the array: UNSUPPORTED.
  * Errors: INVALID_ARG (N == 0 included), BUFFER_TOO_SMALL, UNSUPPORTED, CUDA. */
 int innerq_decode_attention_static(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
 
@@ -284,7 +288,8 @@ int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t v
  * runs out it records that in a device-side error word, contributes nothing for the affected token
  * range and returns normally.  This call copies the word to the host and SYNCHRONISES `cuda_stream`
  * (the only entry point that does).  Returns 0 (no error), 1 (a wait ran out since the cache was
- * created) or a negative error code. */
+ * created, or in the last innerq_decode_attention_static call of this cache's configuration on the
+ * current device) or a negative error code. */
 int innerq_read_device_error(innerq_cache_t* cache, void* cuda_stream);
 
 /* Number of kernels the last call of each kind launched (for launch accounting):

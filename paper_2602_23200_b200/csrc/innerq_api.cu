@@ -364,7 +364,10 @@ int innerq_quantize_prefill(innerq_cache_t* c, const void* k, const void* v, int
                          static_cast<cudaStream_t>(cuda_stream));
   if (n < 0) return INNERQ_ERR_CUDA;
   c->N = n_tokens;
-  c->N_safe = n_tokens;
+  // Nothing of a fresh prefill counts as settled: the first decode after it waits for its predecessors before it
+  // reads any packed chunk (the prefill kernels are ordinary launches, whose writes a dependent launch may rely on
+  // only after that wait).  The decode that follows then streams ahead again.
+  c->N_safe = 0;
   c->reads_settled = 0;
   c->launches[0] = n;
   return INNERQ_OK;
@@ -611,7 +614,16 @@ int static_scratch_for_current_device(unsigned char** out) {
 
 int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, void* cuda_stream) {
   if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
+  if (c->opt_variant == 5) return INNERQ_ERR_UNSUPPORTED;      // the tcgen05 kernel is not served from this array
   if (c->L.workspace_bytes > kStaticScratchBytes) return INNERQ_ERR_BUFFER_TOO_SMALL;
+  // the array that is used is the current device's: the cache has to live on that device
+  {
+    int dev = -1;
+    cudaPointerAttributes at;
+    if (cudaGetDevice(&dev) != cudaSuccess) return INNERQ_ERR_CUDA;
+    if (cudaPointerGetAttributes(&at, c->cache) != cudaSuccess) { cudaGetLastError(); return INNERQ_ERR_INVALID_ARG; }
+    if (at.type != cudaMemoryTypeDevice || at.device != dev) return INNERQ_ERR_INVALID_ARG;
+  }
   unsigned char* scratch = nullptr;
   int st = static_scratch_for_current_device(&scratch);
   if (st != INNERQ_OK) return st;
@@ -673,6 +685,24 @@ int innerq_read_device_error(innerq_cache_t* c, void* cuda_stream) {
   if (cudaMemcpyAsync(&flag, c->ws + c->L.ws_ticket_off + (size_t)c->L.U * 4, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
       cudaStreamSynchronize(s) != cudaSuccess)
     return INNERQ_ERR_CUDA;
+  // a call of innerq_decode_attention_static keeps its error word in the library's own array (same offset, this
+  // cache's layout; every such call clears it first, so it tells about the last one on the current device)
+  int dev = -1;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices && c->L.workspace_bytes <= kStaticScratchBytes) {
+    void* p = nullptr;
+    {
+      std::lock_guard<std::mutex> lock(g_scratch_mutex);
+      p = g_scratch_ptr[dev];
+    }
+    if (p) {
+      unsigned int flag2 = 0;
+      if (cudaMemcpyAsync(&flag2, static_cast<unsigned char*>(p) + c->L.ws_ticket_off + (size_t)c->L.U * 4, 4,
+                          cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+          cudaStreamSynchronize(s) != cudaSuccess)
+        return INNERQ_ERR_CUDA;
+      flag |= flag2;
+    }
+  }
   return (int)flag;
 }
 

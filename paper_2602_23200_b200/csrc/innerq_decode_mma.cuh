@@ -434,6 +434,9 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (!__all_sync(0xffffffffu, v == (uint32_t)cn.N)) dep_wait();
+    // what was acquired is ordered ahead of bulk async copies too (this kernel's later ones, and through
+    // launch_dependents the next kernel's, which stream the rows that append packed)
+    asm volatile("fence.proxy.async.global;" ::: "memory");
   };
   auto ld_tail = [&](const uint4* p) -> uint4 { return dep_waited ? __ldg(p) : __ldcg(p); };
   // an iteration's copy covers the chunks [c_lo + i * CPI, c_lo + (i + 1) * CPI)

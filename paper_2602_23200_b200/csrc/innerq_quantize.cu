@@ -293,7 +293,10 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
   append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
   append_evict_block(L, L.v, N, u, cache, false, tile, words);
   // Publish: everything this unit's append writes is written.  A decode of N tokens that reads N here (acquire)
-  // may read the rings and the newest packed rows without waiting for this kernel to end.
+  // may read the rings and the newest packed rows without waiting for this kernel to end.  The packed rows will be
+  // read by bulk async copies (another memory proxy than these ordinary stores): every thread orders its stores
+  // ahead of that proxy before the count is released.
+  asm volatile("fence.proxy.async.global;" ::: "memory");
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();

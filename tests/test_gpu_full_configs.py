@@ -117,6 +117,48 @@ def test_config2_prefill_then_steps():
     print(f"config2, tcgen05 kernel: err/tol {e5:.3f}")
 
 
+def test_config2_inputs_written_by_the_kernel_right_before_each_call():
+    # The way a model uses the library: q, k_new and v_new of every step are produced on the same stream by an
+    # ordinary kernel (here an elementwise op into three buffers that are REUSED by every step) immediately before
+    # innerq_append_token / innerq_decode_attention, which are launched as programmatic dependents and read their
+    # inputs before they wait for their predecessors.  120 steps enqueued without host synchronisation; every
+    # output and the final cache contents against the oracle.
+    import torch
+    w = synth.config2()
+    K, V = synth.kv_all(w)
+    units = [7, 24]
+    n_steps = 120
+    gc, oc = make_gpu(w, K, V, extra=n_steps + 8), sub_oracle(w, K, V, units, extra=n_steps + 8)
+    del K, V
+    toks = [synth.new_token(w, 500 + s) for s in range(n_steps)]
+    qs = [synth.query(w, 500 + s) for s in range(n_steps)]
+    k_src, v_src, q_src = dev(np.stack([t[0] for t in toks])), dev(np.stack([t[1] for t in toks])), dev(np.stack(qs))
+    k_buf, v_buf, q_buf = torch.zeros_like(k_src[0]), torch.zeros_like(v_src[0]), torch.zeros_like(q_src[0])
+    one = torch.ones((), dtype=torch.float16, device="cuda")
+    outs = torch.empty_like(q_src)
+    torch.cuda.synchronize()
+    for s in range(n_steps):
+        torch.mul(k_src[s], one, out=k_buf)              # three ordinary kernels: the step's inputs come into being
+        torch.mul(v_src[s], one, out=v_buf)
+        if s % 2 == 0:
+            torch.mul(q_src[s], one, out=q_buf)          # q before the append on even steps ...
+        gc.innerq_append_token(k_buf, v_buf)
+        if s % 2 == 1:
+            torch.mul(q_src[s], one, out=q_buf)          # ... and between append and decode on odd ones
+        gc.innerq_decode_attention(q_buf, outs[s])
+    torch.cuda.synchronize()
+    got = outs.cpu().numpy()
+    worst = 0.0
+    for s in range(n_steps):
+        k1, v1 = toks[s]
+        oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+        ref = oc.decode(q_rows(w, qs[s], units))
+        worst = max(worst, P.assert_outputs_close(q_rows(w, got[s], units), ref, f"produced inputs, step {s}"))
+    P.assert_export_equal(slice_export(gc.innerq_cache_export(), units), oc.export(), w.grouping, w.group, True, True)
+    assert gc.innerq_read_device_error() == 0
+    print(f"config2, inputs produced on the stream, {n_steps} steps back to back: worst err/tol {worst:.3f}")
+
+
 def test_config2_paged_cache():
     # the same workload with the packed records in 512-token pages of a pool, handed out in a shuffled order; the
     # steps are enqueued back to back and cross a page boundary (the 32636 packed key rows of the prefill fill 63.7 pages)

@@ -1,12 +1,14 @@
 """The decode entry point that runs on the library's built-in scratch array (needs a B200).
 
 Collected last on purpose: a run that stops at the first failure has then already run everything else.
-It checks the variant against the regular entry point on two calls in a row (the shared array keeps the
-first call's contents when the second starts), and that an over-sized configuration is refused.
+It checks the variant against the regular entry point AND against the CPU oracle on two calls in a row (the
+shared array keeps the first call's contents when the second starts), and that an over-sized configuration
+and the tcgen05 decode variant are refused.
 """
 import numpy as np
 import pytest
 
+from oracle import innerq_oracle as O
 from paper_2602_23200_b200 import synth
 from tests import _parity as P
 
@@ -26,12 +28,17 @@ def _setup(w):
 def test_static_scratch_decode_matches_regular_decode_twice(w):
     import torch
     gc = _setup(w)
+    oc = O.from_workload(w)
+    oc.prefill(*synth.kv_all(w))
     for call in range(2):
-        q = torch.from_numpy(synth.query(w, call)).cuda()
+        qh = synth.query(w, call)
+        q = torch.from_numpy(qh).cuda()
         ref = gc.innerq_decode_attention(q).cpu().numpy()
         got = gc.innerq_decode_attention_static(q).cpu().numpy()
         assert np.isfinite(got).all()
-        P.assert_outputs_close(got, ref, f"static scratch, call {call}")
+        P.assert_outputs_close(got, ref, f"static scratch against the regular entry point, call {call}")
+        P.assert_outputs_close(got, oc.decode(qh), f"static scratch against the oracle, call {call}")
+        assert gc.innerq_read_device_error() == 0      # covers the error word inside the shared array as well
     # a different cache on the same device shares the array: its call must not be disturbed by the leftovers
     w2 = synth.tiny(n_tokens=333, group=64, k_bits=4, v_bits=4)
     gc2 = _setup(w2)
@@ -55,3 +62,17 @@ def test_static_scratch_refuses_configurations_beyond_its_size():
     assert ei.value.status == -4
     out = gc.innerq_decode_attention(q)          # the regular entry point still serves it
     assert torch.isfinite(out.float()).all()
+
+
+def test_static_scratch_refuses_the_tcgen05_variant():
+    import torch
+    from paper_2602_23200_b200 import binding as B
+    w = synth.tiny(n_tokens=300)
+    gc = _setup(w)
+    q = torch.from_numpy(synth.query(w)).cuda()
+    gc.innerq_set_decode_options(0, 5)
+    with pytest.raises(B.InnerQError) as ei:
+        gc.innerq_decode_attention_static(q)
+    assert ei.value.status == -2
+    gc.innerq_set_decode_options(0, 0)
+    assert torch.isfinite(gc.innerq_decode_attention_static(q).float()).all()
