@@ -291,6 +291,16 @@ class Legs:
         self.k_new, self.v_new, self.q_all, self.out = k_new, v_new, q_all, out
         self.stream = torch.cuda.current_stream()
         self.i = first_step                 # index of the next unused (k_new, v_new, q) triple
+        # the step loop passes addresses (buffers validated here once), so that the host stays ahead of the GPU
+        from paper_2602_23200_b200.binding import _dev_ptr
+        c = caches[0].cfg
+        n = k_new.shape[0]
+        self.kp = _dev_ptr(k_new, "k_new", (n, c.batch, c.n_kv_heads, c.head_dim), caches[0].device)
+        self.vp = _dev_ptr(v_new, "v_new", (n, c.batch, c.n_kv_heads, c.head_dim), caches[0].device)
+        self.qp = _dev_ptr(q_all, "q", (n, c.batch, c.n_q_heads, c.head_dim), caches[0].device)
+        self.op = _dev_ptr(out, "out", (c.batch, c.n_q_heads, c.head_dim), caches[0].device)
+        self.kv_stride, self.q_stride = k_new[0].numel() * 2, q_all[0].numel() * 2
+        self.sp = int(self.stream.cuda_stream)
 
     def _ev(self):
         return self.torch.cuda.Event(enable_timing=True)
@@ -301,23 +311,26 @@ class Legs:
     def step(self):
         i = self.i
         c = self.caches[i % self.R]
-        c.innerq_append_token(self.k_new[i], self.v_new[i])
-        c.innerq_decode_attention(self.q_all[i], self.out)
+        c.innerq_append_token_ptr(self.kp + i * self.kv_stride, self.vp + i * self.kv_stride, self.sp)
+        c.innerq_decode_attention_ptr(self.qp + i * self.q_stride, self.op, self.sp)
         self.i += 1
         return c
 
     def steps(self, n, warm=0):
-        """n steps (append + decode) between two events, after `warm` untimed steps that run straight into them."""
+        """n steps (append + decode) between two events, after `warm` untimed steps that run straight into them.
+        Returns (us per step on the device, us per step the host needed to enqueue them)."""
         self.delay()
         for _ in range(warm):
             self.step()
         e0, e1 = self._ev(), self._ev()
         e0.record(self.stream)
+        t0 = time.perf_counter()
         for _ in range(n):
             self.step()
+        host_us = (time.perf_counter() - t0) * 1e6 / n
         e1.record(self.stream)
         self.torch.cuda.synchronize()
-        return e0.elapsed_time(e1) * 1e3 / n
+        return e0.elapsed_time(e1) * 1e3 / n, host_us
 
     def decodes_bracketed(self, n):
         """n decodes, each between its own pair of events (no overlap with its neighbours).  Returns a list of us."""
@@ -452,11 +465,12 @@ def measure_config(name, peak, R=2, n_steps=128):
     nbytes = decode_algorithmic_bytes(w, w.n_tokens + 1, sym_k, sym_v)[1]
     alone = stats(legs.decodes_bracketed(32))
     chain = legs.decodes_chained(64)
-    step = legs.steps(n_steps, warm=32)
+    step, step_host = legs.steps(n_steps, warm=32)
     gbs = lambda us: nbytes / us / 1e3
     res.update({
         "bytes_per_decode_minimal": nbytes, "sym_group_fraction": {"k": sym_k, "v": sym_v},
         "us_per_decode_alone": alone, "us_per_decode_chained": chain, "us_per_step": step,
+        "host_us_per_step_enqueue": step_host,
         "frac_of_measured_peak": {"alone_median": gbs(alone["median"]) / peak, "chained": gbs(chain) / peak,
                                   "step": gbs(step) / peak},
         "pct_of_nominal_8TBs": {"alone_median": gbs(alone["median"]) / 80.0, "chained": gbs(chain) / 80.0,
@@ -590,7 +604,7 @@ def run_ours(args, w):
     bytes_min /= Kst                 # bytes per decode vary by < 0.1 % over the whole run
     value_gbs = whole_job_gbs(bytes_min, ms_step * 1e-3, world)
     # ---- the same step loop over a fixed number of steps (does not depend on --steps) ------------------------
-    leg_us = legs.steps(LEG, warm=32)
+    leg_us, leg_host_us = legs.steps(LEG, warm=32)
     # ---- the decode kernel alone: every launch between its own events (the roofline figure), and chained -------
     alone = stats(legs.decodes_bracketed(48))
     b2b_us = legs.decodes_chained(64)
@@ -684,7 +698,8 @@ def run_ours(args, w):
         line = {
             "metric": "decode_step_algorithmic_hbm_gbs", "value": value_gbs, "unit": "GB/s", "n_gpus": world,
             "steps": Kst, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
-            "us_per_step_fixed_leg": {"steps": LEG, "us": leg_us, "frac_of_measured_peak": gbs(leg_us) / peak},
+            "us_per_step_fixed_leg": {"steps": LEG, "us": leg_us, "frac_of_measured_peak": gbs(leg_us) / peak,
+                                      "host_us_per_step_enqueue": leg_host_us},
             "us_per_decode": alone["median"], "us_per_decode_alone": alone, "us_per_decode_back_to_back": b2b_us,
             "us_per_append_median": append_us,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",

@@ -328,6 +328,19 @@ class InnerQCache:
                                              _stream_ptr(stream, self.device)), "innerq_decode_attention")
         return out
 
+    # The two calls of a decode step with addresses instead of tensors, for loops that have validated their buffers
+    # once (contiguous fp16 CUDA tensors of the shapes above, on this cache's device, which is current) and then
+    # step through them by pointer arithmetic: the same C entry points, without the per-call checks.
+    def innerq_append_token_ptr(self, k_new_ptr: int, v_new_ptr: int, stream_ptr: int):
+        st = _lib.innerq_append_token(self._h, k_new_ptr, v_new_ptr, stream_ptr)
+        if st:
+            _check(st, "innerq_append_token")
+
+    def innerq_decode_attention_ptr(self, q_ptr: int, out_ptr: int, stream_ptr: int):
+        st = _lib.innerq_decode_attention(self._h, q_ptr, out_ptr, stream_ptr)
+        if st:
+            _check(st, "innerq_decode_attention")
+
     def innerq_decode_attention_static(self, q, out=None, stream=None):
         """Decode on the library's built-in scratch array: for callers that cannot supply device scratch
         themselves.  Allocates nothing inside the library (the `out` tensor, if not passed, is still a
