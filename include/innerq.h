@@ -114,7 +114,7 @@ int innerq_cache_destroy(innerq_cache_t* cache);
  * is named by its index in it.  The caller decides which page goes to which cache (free list, eviction, reuse);
  * the library checks indices against pool_pages and against the cache's own pages, not across caches.
  * Kernels, results and every other entry point are the same as for a contiguous cache; batched calls need caches
- * on one pool.  Not available for grouping FP16 (UNSUPPORTED) or with the tcgen05 kernel variant. */
+ * on one pool.  Not available for grouping FP16 (UNSUPPORTED). */
 
 /* Sizes for a paged cache: bytes of the cache buffer and the workspace, bytes of one page, and the most page slots
  * a cache can use (max_tokens tokens).  Host pointers.  Errors: INVALID_ARG (page_tokens), UNSUPPORTED. */
@@ -267,7 +267,6 @@ int innerq_decode_attention_batched(innerq_cache_t* const* caches, int32_t n, co
  *   - The caller's workspace is not touched.  The error word of this call is in the array as well;
  *     innerq_read_device_error (called with the same device current) reports it together with the
  *     workspace's own word.  It tells about the last such call only: the next one clears it.
- *   - Decode variant 5 (tcgen05 kernel) is not served from the array: UNSUPPORTED.
  * Errors: INVALID_ARG (N == 0 included), BUFFER_TOO_SMALL, UNSUPPORTED, CUDA. */
 int innerq_decode_attention_static(innerq_cache_t* cache, const void* q, void* out, void* cuda_stream);
 
@@ -280,7 +279,6 @@ int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_s
  *   n_splits : number of token ranges each unit is split into by the decode kernel.
  *   variant  : 0 automatic, 1 plain SIMT kernel, 2 warp-MMA kernel (where supported; UNSUPPORTED otherwise),
  *              3 / 4 warp-MMA kernel with one / two 32-token chunks per loop iteration (sets a process-wide knob).
- *              5 tcgen05 kernel (2-bit keys and values, group 32, one query head per KV head; UNSUPPORTED otherwise).
  * Errors: INVALID_ARG. */
 int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
 

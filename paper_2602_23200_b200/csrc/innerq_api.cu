@@ -159,6 +159,8 @@ void make_layout(const innerq_config_t& c, Layout& L, int page_tokens = 0) {
   } else if (c.grouping == INNERQ_GROUPING_INNER) {
     place_store(L.k, kRow, c.k_bits, c.k_mode, c, L.U, off);
     place_store(L.v, kBlock, c.v_bits, c.v_mode, c, L.U, off);
+    // 2-bit keys with 2-bit values: codes in byte order, for the decode kernel built on the 8-bit integer MMA
+    if (c.k_bits == 2 && c.v_bits == 2) L.k.perm = L.v.perm = 1;
     place_records(L.k, L.v, L.G, L.U, off, page_tokens / L.G);
   } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
     place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);
@@ -390,11 +392,7 @@ int innerq_decode_attention(innerq_cache_t* c, const void* q, void* out, void* c
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int n = -2;
   bool fused = false;
-  if (c->opt_variant == 5) {          // tcgen05 kernel, where it exists; no fallback
-    n = launch_decode_tc5(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
-                          c->opt_splits, s);
-    if (n == -2) return INNERQ_ERR_UNSUPPORTED;
-  } else if (c->opt_variant != 1 && c->L.k.kind == kNone)
+  if (c->opt_variant != 1 && c->L.k.kind == kNone)
     n = launch_decode_fp16(c->L, c->cache, c->ws, c->N, static_cast<const __half*>(q), static_cast<__half*>(out),
                            c->opt_splits, s);
   else if (c->opt_variant != 1 && decode_mma_supported(c->L)) {
@@ -614,7 +612,6 @@ int static_scratch_for_current_device(unsigned char** out) {
 
 int innerq_decode_attention_static(innerq_cache_t* c, const void* q, void* out, void* cuda_stream) {
   if (!c || !q || !out || c->N < 1) return INNERQ_ERR_INVALID_ARG;
-  if (c->opt_variant == 5) return INNERQ_ERR_UNSUPPORTED;      // the tcgen05 kernel is not served from this array
   if (c->L.workspace_bytes > kStaticScratchBytes) return INNERQ_ERR_BUFFER_TOO_SMALL;
   // the array that is used is the current device's: the cache has to live on that device
   {
@@ -669,7 +666,7 @@ int innerq_cache_export(innerq_cache_t* c, innerq_export_t* ex, void* cuda_strea
 }
 
 int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t variant) {
-  if (!c || n_splits < 0 || variant < 0 || variant > 5) return INNERQ_ERR_INVALID_ARG;
+  if (!c || n_splits < 0 || variant < 0 || variant > 4) return INNERQ_ERR_INVALID_ARG;
   c->opt_splits = n_splits;
   // variants 3 and 4 force the fast kernel with one / two 32-token chunks per loop iteration (process-wide knob)
   if (variant == 3 || variant == 4) { decode_mma_set_chunks_per_iter(variant - 2); variant = 2; }

@@ -45,9 +45,9 @@ __device__ __forceinline__ float element(const TensorView& v, int G, int t, int 
   if (v.kind == kRow) decode_meta(load_meta(row_meta_ptr(v.rec, v.S, i), c / G, v.meta_bytes), v.bits, s, z);
   else decode_meta(load_meta(block_meta_ptr(v.rec, v.S, i / G), block_meta_index(c), v.meta_bytes), v.bits, s, z);
   if (v.S.code_kind == kRow)
-    code = row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(v.rec, v.S, i)), c, v.bits);
+    code = row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(v.rec, v.S, i)), c, v.bits, v.S.perm);
   else
-    code = chunk_code(reinterpret_cast<const uint32_t*>(block_code_ptr(v.rec, v.S, i / kChunk)), i % kChunk, c, v.bits);
+    code = chunk_code(reinterpret_cast<const uint32_t*>(block_code_ptr(v.rec, v.S, i / kChunk)), i % kChunk, c, v.bits, v.S.perm);
   return fmaf(s, (float)code, z);
 }
 

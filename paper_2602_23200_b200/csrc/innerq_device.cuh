@@ -12,7 +12,11 @@ __device__ __forceinline__ float h2f_bits(uint16_t b) { return __half2float(__us
 __device__ __forceinline__ uint16_t f2h_bits(float f) { return __half_as_ushort(__float2half_rn(f)); }
 
 // ---- packed-code accessors (generic, slow; the fast kernels extract fragments directly) ----
-__device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, int c, int bits) {
+__device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, int c, int bits, int perm = 0) {
+  if (perm == 1) {
+    BitPos p = row_pos_i8(c);
+    return (row[p.word] >> p.bit) & 3u;
+  }
   if (bits == 3) {
     BitPos lo = row_pos_plane(c, 2), hi = row_pos_plane(c, 1);
     return ((row[lo.word] >> lo.bit) & 3u) | (((row[row_hi_plane_word() + hi.word] >> hi.bit) & 1u) << 2);
@@ -21,7 +25,11 @@ __device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, i
   return (row[p.word] >> p.bit) & ((1u << bits) - 1u);
 }
 
-__device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chunk, int tau, int c, int bits) {
+__device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chunk, int tau, int c, int bits, int perm = 0) {
+  if (perm == 1) {
+    BitPos p = block_pos_i8(tau, c);
+    return (chunk[p.word] >> p.bit) & 3u;
+  }
   if (bits == 3) {
     BitPos lo = block_pos_plane(tau, c, 2), hi = block_pos_plane(tau, c, 1);
     return ((chunk[lo.word] >> lo.bit) & 3u) | (((chunk[chunk_hi_plane_word() + hi.word] >> hi.bit) & 1u) << 2);
@@ -31,8 +39,11 @@ __device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chun
 }
 
 // OR a code into a zero-initialised packed row / chunk held in shared memory.
-__device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t code) {
-  if (bits == 3) {
+__device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t code, int perm = 0) {
+  if (perm == 1) {
+    BitPos p = row_pos_i8(c);
+    atomicOr(&row[p.word], code << p.bit);
+  } else if (bits == 3) {
     BitPos lo = row_pos_plane(c, 2), hi = row_pos_plane(c, 1);
     atomicOr(&row[lo.word], (code & 3u) << lo.bit);
     atomicOr(&row[row_hi_plane_word() + hi.word], (code >> 2) << hi.bit);
@@ -41,8 +52,11 @@ __device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t
     atomicOr(&row[p.word], code << p.bit);
   }
 }
-__device__ __forceinline__ void chunk_put(uint32_t* chunk, int tau, int c, int bits, uint32_t code) {
-  if (bits == 3) {
+__device__ __forceinline__ void chunk_put(uint32_t* chunk, int tau, int c, int bits, uint32_t code, int perm = 0) {
+  if (perm == 1) {
+    BitPos p = block_pos_i8(tau, c);
+    atomicOr(&chunk[p.word], code << p.bit);
+  } else if (bits == 3) {
     BitPos lo = block_pos_plane(tau, c, 2), hi = block_pos_plane(tau, c, 1);
     atomicOr(&chunk[lo.word], (code & 3u) << lo.bit);
     atomicOr(&chunk[chunk_hi_plane_word() + hi.word], (code >> 2) << hi.bit);

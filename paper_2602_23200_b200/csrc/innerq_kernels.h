@@ -61,9 +61,5 @@ int launch_decode_fp16(const Layout& L, const unsigned char* cache, unsigned cha
                        __half* out, int n_splits, cudaStream_t st);
 void decode_mma_set_chunks_per_iter(int n);   // tuning: 32-token chunks per loop iteration (1 or 2)
 
-// tcgen05 decode for 2-bit keys and values, G = 32, one query head per KV head.  Returns -2 for other layouts.
-int launch_decode_tc5(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
-                      __half* out, int n_splits, cudaStream_t st);
-bool decode_tc5_supported(const Layout& L);
 
 }  // namespace iq

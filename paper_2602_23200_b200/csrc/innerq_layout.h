@@ -46,6 +46,9 @@ struct Store {
                        // kBlock = 32-token chunks (the operand order of p.V).  Equal to `kind` under inner grouping;
                        // under outer grouping keys keep rows and values keep chunks, only the metadata changes sides.
   int bits, mode;
+  int perm;            // order of the codes inside a packed row / chunk: 0 = pairs for the fp16 tensor-core fragments
+                       // (word & mask is a half2), 1 = bytes for the 8-bit integer fragments (2-bit codes of an
+                       // inner-grouped cache whose keys and values are both 2-bit; see row_pos_i8 / block_pos_i8)
   int ring_cap;        // slots of the recent ring: w_recent + 1 (ROW) or w_recent + G (BLOCK)
   int cap_q;           // capacity in quantised tokens (multiple of kTile)
   int n_groups;        // metadata entries per row (ROW: D/G) or per group (BLOCK: D)
@@ -210,6 +213,35 @@ IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
     p.bit = 16 * tp + (((m & 1) * 2 + rh) * 4 + 2 * ks + kh);
   }
   return p;
+}
+
+// ---- 2-bit codes in byte order (Store::perm = 1): operands of the integer tensor-core instruction m16n8k32 -------
+// A byte holds four codes at bit positions 0, 2, 4, 6; `word & (0x03030303 << 2p)` is four 8-bit operand values
+// (the codes at position p times 4^p; the factor is taken out after the sum).
+// ROW store: byte k (0..31) of the 32-byte row holds channels k, 32 + k, 64 + k, 96 + k at positions 0..3, so that
+// position p is one k-step of 32 channels = the p-th run of 32 channels (a whole group at G = 32).  The fragment of
+// lane (gid, j) is bytes 4j..4j+3 and 16+4j..16+4j+3 of rows gid and gid + 8: the two words are stored next to each
+// other (physical word 2j + h holds bytes 16h + 4j ..), one 64-bit load per row.
+IQ_HD BitPos row_pos_i8(int c) {
+  const int p = c >> 5, k = c & 31, lw = k >> 2;
+  BitPos r;
+  r.word = 2 * (lw & 3) + (lw >> 2);
+  r.bit = 8 * (k & 3) + 2 * p;
+  return r;
+}
+// BLOCK store: one chunk = one k-step of 32 tokens for each of 8 m-tiles of 16 channels.  Token tau sits at
+// k = 4 * (tau % 8) + tau / 8 (the four tokens whose scores one lane holds after the key MMAs are adjacent in k).
+// Channel c = 64 W + 8 gid + 2 p + rh is fragment row gid (rh = 0) or gid + 8 (rh = 1) of m-tile 4 W + p, the same
+// ownership as with perm = 0; the four m-tiles 4 W .. 4 W + 3 share their words, one per bit position.
+// Lane 4 gid + j holds words [W][2 * (k / 16) + rh] with bytes k % 4, for k / 4 % 4 == j.
+IQ_HD BitPos block_pos_i8(int tau, int c) {
+  const int k = 4 * (tau & 7) + (tau >> 3);
+  const int W = c >> 6, p = (c >> 1) & 3, gid = (c >> 3) & 7, rh = c & 1;
+  const int j = (k & 15) >> 2, half = k >> 4;
+  BitPos r;
+  r.word = W * 128 + (4 * gid + j) * 4 + 2 * half + rh;
+  r.bit = 8 * (k & 3) + 2 * p;
+  return r;
 }
 
 // BLOCK store metadata: the 128 per-channel entries of a group are ordered so that the 16 channels a

@@ -112,7 +112,7 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
-      row_put(stage, 4 * lane + i, S.bits, code);
+      row_put(stage, 4 * lane + i, S.bits, code, S.perm);
     }
     __syncwarp();
     if (lane < words) dst_row[lane] = stage[lane];
@@ -121,7 +121,7 @@ __device__ __forceinline__ void quantize_row_warp(const __half* __restrict__ src
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t code = (uint32_t)(int)(asym ? ua[i] : qs[i] + p.half);
-      chunk_put(chunk, i_row % kChunk, 4 * lane + i, S.bits, code);
+      chunk_put(chunk, i_row % kChunk, 4 * lane + i, S.bits, code, S.perm);
     }
   }
   if ((lane % gl) == 0) store_meta(row_meta_ptr(rec, S, i_row), lane / gl, S.meta_bytes, group_meta(p, asym));
@@ -165,8 +165,8 @@ __device__ void quantize_block_cta(const TokSrc& src, int t_first, const float* 
     float x = __half2float(tile[t * kD + c]);
     if (norm) x = __fmul_rn(x, inv);
     uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
-    if (rows) row_put(words + t * rw, c, S.bits, code);
-    else chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code);
+    if (rows) row_put(words + t * rw, c, S.bits, code, S.perm);
+    else chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code, S.perm);
   }
   store_meta(block_meta_ptr(rec, S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
   __syncthreads();
@@ -366,9 +366,9 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
     for (int i = tid0; i < n_q * kD; i += stride) {
       int t = i / kD, c = i % kD;
       uint32_t v = S.code_kind == kRow
-                       ? row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(rec, S, t)), c, S.bits)
+                       ? row_code(reinterpret_cast<const uint32_t*>(row_code_ptr(rec, S, t)), c, S.bits, S.perm)
                        : chunk_code(reinterpret_cast<const uint32_t*>(block_code_ptr(rec, S, t / kChunk)), t % kChunk, c,
-                                    S.bits);
+                                    S.bits, S.perm);
       code[((size_t)u * cap + t) * kD + c] = (uint8_t)v;
     }
   }

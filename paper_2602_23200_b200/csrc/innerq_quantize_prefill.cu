@@ -148,6 +148,42 @@ __device__ __forceinline__ void pack_block_segment(const ChosenCoder& cc, const 
   for (int i = 0; i < NW; ++i) lw[i] -= cw[i];
 }
 
+// Byte-order layout (Store::perm = 1, 2-bit codes).  ROW segment = 32 consecutive channels = one bit position of all
+// 32 bytes of the row: the codes go to position 0 of the 8 row words here, the caller shifts them to its position.
+template <bool CLAMP>
+__device__ __forceinline__ void pack_row_segment_i8(const ChosenCoder& cc, const float (&x)[kSeg], uint32_t (&w8)[8]) {
+  uint32_t cw[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { w8[i] = 0u; cw[i] = 0u; }
+#pragma unroll
+  for (int e = 0; e < kSeg; ++e) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[e]);
+    const BitPos p = row_pos_i8(e);                     // constants: positions of channels 0..31 (bit position 0)
+    w8[p.word] += code << p.bit;
+    cw[p.word] += kMagicBits << p.bit;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w8[i] -= cw[i];
+}
+// BLOCK segment = 32 tokens of one channel: bytes of the 8 words [j][half] of its fragment row (see block_pos_i8), at
+// bit position 0 here.  Word index: 2 * j + half.
+template <bool CLAMP>
+__device__ __forceinline__ void pack_block_segment_i8(const ChosenCoder& cc, const float (&x)[kSeg], uint32_t (&w8)[8]) {
+  uint32_t cw[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { w8[i] = 0u; cw[i] = 0u; }
+#pragma unroll
+  for (int t = 0; t < kSeg; ++t) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[t]);
+    const BitPos p = block_pos_i8(t, 0);                // constants: channel 0 (W = 0, gid = 0, position 0, rh = 0)
+    const int li = 2 * ((p.word >> 2) & 3) + ((p.word >> 1) & 1);      // 2 * j + half
+    w8[li] += code << p.bit;
+    cw[li] += kMagicBits << p.bit;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w8[i] -= cw[i];
+}
+
 __device__ __forceinline__ void unpack8(const uint4& v, float* x) {
   const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
@@ -162,7 +198,7 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* x) {
 // channels 32*seg .. 32*seg+31.  The 8 packed rows and their metadata entries are contiguous in the chunk record.
 // Positions of the segment's codes (see row_pos_plane): element e of segment 0 sits in local word j = tid4(e);
 // for segment seg the word index and the bit offset move by a per-plane amount that depends on seg only.
-template <int BITS, bool NORM>
+template <int BITS, bool NORM, bool I8 = false>
 __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, Store S, const __half* __restrict__ X, int N,
                                                                     int n_q, unsigned char* __restrict__ cache,
                                                                     const float* __restrict__ inv_norm) {
@@ -234,15 +270,25 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
       asym = ea < es;
     }
     const ChosenCoder cc(sc, asym);
-    uint32_t lw[4], hw[4];
-    if (no_clip) pack_row_segment<BITS, false>(cc, x, lw, hw);
-    else pack_row_segment<BITS, true>(cc, x, lw, hw);
-    __syncwarp();                                          // the stage is zero and no longer being read
     uint32_t* row = stage + tk * RW;
+    if constexpr (I8) {
+      static_assert(!I8 || BITS == 2, "byte order is defined for 2-bit codes");
+      uint32_t w8[8];
+      if (no_clip) pack_row_segment_i8<false>(cc, x, w8);
+      else pack_row_segment_i8<true>(cc, x, w8);
+      __syncwarp();                                        // the stage is zero and no longer being read
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      atomicOr(&row[WM * jj + w_add], lw[jj] << sh_lo);
-      if constexpr (BITS == 3) atomicOr(&row[row_hi_plane_word() + jj], hw[jj] << sh_hi);
+      for (int jj = 0; jj < 8; ++jj) atomicOr(&row[jj], w8[jj] << (2 * seg));
+    } else {
+      uint32_t lw[4], hw[4];
+      if (no_clip) pack_row_segment<BITS, false>(cc, x, lw, hw);
+      else pack_row_segment<BITS, true>(cc, x, lw, hw);
+      __syncwarp();                                        // the stage is zero and no longer being read
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        atomicOr(&row[WM * jj + w_add], lw[jj] << sh_lo);
+        if constexpr (BITS == 3) atomicOr(&row[row_hi_plane_word() + jj], hw[jj] << sh_hi);
+      }
     }
     const int i = i0 + tk;
     if (i < n_q && (lane & (gl - 1)) == 0)
@@ -264,7 +310,7 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
 // (one 32-bit load per token: a warp reads 128 contiguous bytes of each token row).  The two channels of a pair
 // are the two row halves of one MMA fragment row pair, so between them they fill whole words of the packed chunk
 // and no staging or atomics are needed (3-bit: the 1-bit plane's words are shared with the neighbouring pair).
-template <int BITS, bool NORM>
+template <int BITS, bool NORM, bool I8 = false>
 __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, Store S, const __half* __restrict__ X,
                                                                       int N, int n_q, unsigned char* __restrict__ cache,
                                                                       const float* __restrict__ inv_norm) {
@@ -290,6 +336,7 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
     uint32_t wlo[NW], whi[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int i = 0; i < NW; ++i) wlo[i] = 0u;
+    [[maybe_unused]] uint32_t w16[2][8];      // byte order: words [rh][2 * j + half] of this channel pair, at its bit position
     uint32_t meta2[2];
     if (CH > 1) __syncthreads();       // the previous group's reduction words are no longer read
 #pragma unroll
@@ -332,20 +379,56 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
         asym = ea < es;
       }
       const ChosenCoder cc(sc, asym);
-      uint32_t lw[NW], hw[4];
-      if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
-      else pack_block_segment<BITS, true>(cc, x, lw, hw);
+      if constexpr (I8) {
+        if (no_clip) pack_block_segment_i8<false>(cc, x, w16[rh]);
+        else pack_block_segment_i8<true>(cc, x, w16[rh]);
 #pragma unroll
-      for (int i = 0; i < NW; ++i) wlo[i] |= lw[i] << (8 * rh);
-      if constexpr (BITS == 3) {
+        for (int i = 0; i < 8; ++i) w16[rh][i] <<= 2 * (cp & 3);      // this pair's bit position: (c >> 1) & 3
+      } else {
+        uint32_t lw[NW], hw[4];
+        if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
+        else pack_block_segment<BITS, true>(cc, x, lw, hw);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) whi[i] |= hw[i] << (4 * (2 * (m & 1) + rh));
+        for (int i = 0; i < NW; ++i) wlo[i] |= lw[i] << (8 * rh);
+        if constexpr (BITS == 3) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) whi[i] |= hw[i] << (4 * (2 * (m & 1) + rh));
+        }
       }
       meta2[rh] = group_meta(p, asym);
     }
     uint32_t* chunk = reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, j * CH + k));
+    if constexpr (I8) {
+      // The four channel pairs cp = 4q .. 4q+3 (adjacent lanes) fill the four bit positions of the same 16 words.
+      // Reduce-scatter by OR: after two exchange steps lane `pos` holds the complete words of j = pos (two halves,
+      // two row halves), which are 16 contiguous bytes of the chunk.
+      const int pos = cp & 3;
+      uint32_t h8[2][4];                      // step 1: keep j of my parity (j = 2 * i + (pos & 1)), index [rh][2 * i + half]
 #pragma unroll
-    for (int i = 0; i < NW; ++i) chunk[base_lo + 4 * (i & 3) + 256 * (i >> 2)] = wlo[i];
+      for (int rh = 0; rh < 2; ++rh)
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint32_t keep = (pos & 1) ? w16[rh][2 * (2 * i + 1) + half] : w16[rh][2 * (2 * i) + half];
+            const uint32_t give = (pos & 1) ? w16[rh][2 * (2 * i) + half] : w16[rh][2 * (2 * i + 1) + half];
+            h8[rh][2 * i + half] = keep | __shfl_xor_sync(0xffffffffu, give, 1);
+          }
+      uint32_t f4[4];                         // step 2: keep i = pos >> 1; index 2 * half + rh (the word order in the chunk)
+#pragma unroll
+      for (int rh = 0; rh < 2; ++rh)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t keep = (pos & 2) ? h8[rh][2 + half] : h8[rh][half];
+          const uint32_t give = (pos & 2) ? h8[rh][half] : h8[rh][2 + half];
+          f4[2 * half + rh] = keep | __shfl_xor_sync(0xffffffffu, give, 2);
+        }
+      const int W = c0 >> 6;
+      *reinterpret_cast<uint4*>(chunk + W * 128 + (4 * gid + pos) * 4) = make_uint4(f4[0], f4[1], f4[2], f4[3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < NW; ++i) chunk[base_lo + 4 * (i & 3) + 256 * (i >> 2)] = wlo[i];
+    }
     if constexpr (BITS == 3) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -372,12 +455,23 @@ static int launch_store_bits(const Layout& L, const Store& S, const __half* X, i
     const int n_batches = (n_q + 7) / 8;
     const int per_unit = grid_cap((n_batches + 4 * 8 - 1) / (4 * 8), grid_cap(148 * 16 / L.U, 1 << 16));
     dim3 grid(per_unit, L.U);
+    if constexpr (BITS == 2) {
+      if (S.perm == 1) {
+        if (inv_norm) quantize_rows_prefill_kernel<2, true, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
+        else quantize_rows_prefill_kernel<2, false, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+      }
+    }
     if (inv_norm) quantize_rows_prefill_kernel<BITS, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
     else quantize_rows_prefill_kernel<BITS, false><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
   } else {
     const int CH = L.G / kChunk;
     const int smem = CH * 128 * 16;                   // reduction words of groups spanning several chunks
     auto kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true> : quantize_blocks_prefill_kernel<BITS, false>;
+    if constexpr (BITS == 2) {
+      if (S.perm == 1)
+        kern = inv_norm ? quantize_blocks_prefill_kernel<2, true, true> : quantize_blocks_prefill_kernel<2, false, true>;
+    }
     const int n_groups = n_q / L.G;
     dim3 grid(grid_cap(n_groups, grid_cap(148 * 16 / L.U, 1 << 16)), L.U);
     kern<<<grid, 64 * CH, smem, st>>>(L, S, X, N, n_q, cache, inv_norm);

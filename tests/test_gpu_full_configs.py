@@ -110,11 +110,11 @@ def test_config2_prefill_then_steps():
     P.assert_export_equal(slice_export(gc.innerq_cache_export(), units), oc.export(), w.grouping, w.group, True, True)
     assert gc.innerq_read_device_error() == 0
     print(f"config2, 40 steps back to back: worst err/tol {worst_b2b:.3f}")
-    # the tcgen05 kernel on the same cache (full size, its default split), same tolerance
-    gc.innerq_set_decode_options(0, 5)
-    _, e5 = compare(w, gc, oc, units, step=77, check_export=False)
+    # the generic kernel on the same cache (full size): an on-device cross-check of the packed layout
+    gc.innerq_set_decode_options(0, 1)
+    _, e1 = compare(w, gc, oc, units, step=77, check_export=False)
     gc.innerq_set_decode_options(0, 0)
-    print(f"config2, tcgen05 kernel: err/tol {e5:.3f}")
+    print(f"config2, generic kernel: err/tol {e1:.3f}")
 
 
 def test_config2_inputs_written_by_the_kernel_right_before_each_call():

@@ -273,11 +273,6 @@ def test_paged_argument_and_capacity_errors():
     with pytest.raises(B.InnerQError) as e:             # at most max_pages
         gc.innerq_cache_assign_pages([0, 2, 3])
     assert e.value.status == ERR_CAPACITY
-    gc.innerq_set_decode_options(0, 5)                  # the tcgen05 variant reads contiguous caches only
-    with pytest.raises(B.InnerQError) as e:
-        gc.innerq_decode_attention(dev(synth.query(w)))
-    assert e.value.status == ERR_UNSUPPORTED
-    gc.innerq_set_decode_options(0, 0)
     # a contiguous cache has no pages
     cc = B.InnerQCache(cfg)
     assert cc.innerq_cache_pages_for(500) == 0 and cc.pages_assigned == 0

@@ -99,26 +99,20 @@ def test_outer_grouped_fused_kernel(bits, G, r, N):
 
 
 @pytest.mark.parametrize("N,mode", [(700, O.HYBRID), (1333, O.ASYM), (164, O.HYBRID), (37, O.HYBRID)])
-def test_tcgen05_decode_kernel(N, mode):
-    # the tcgen05 kernel (variant 5: 2-bit, G = 32, one query head per KV head) against the oracle and the warp-level
-    # kernel, for several split counts and through appends that cross a value-group eviction
+def test_one_query_head_per_kv_head_kernel_instance(N, mode):
+    # 2-bit, G = 32, one query head per KV head: the instance of the fused kernel whose tensor-core columns are
+    # (channel group, digit), against the oracle and the generic kernel, for several split counts, one and two chunks
+    # per loop iteration, and through appends that cross a value-group eviction
     w = synth.tiny(n_tokens=N, group=32, n_q_heads=2, k_mode=mode, v_mode=mode)
     oc, gc, _, _ = run_prefill_both(w)
-    check_decode(w, oc, gc, variants=(5, 2), splits=(0, 1, 3))
+    check_decode(w, oc, gc, variants=(2, 3, 4, 1), splits=(0, 1, 3))
     for step in range(40):
         k1, v1 = synth.new_token(w, step)
         oc.append(k1, v1)
         gc.innerq_append_token(dev(k1), dev(v1))
         if step in (0, 7, 31, 32, 39):
-            check_decode(w, oc, gc, step=step, variants=(5,), splits=(0, 2))
-    from paper_2602_23200_b200 import binding as B
-    other = gpu_cache(synth.tiny(n_tokens=64, group=64, n_q_heads=2))
-    other.innerq_set_decode_options(0, 5)
-    K, V = synth.kv_all(synth.tiny(n_tokens=64, group=64, n_q_heads=2))
-    other.innerq_quantize_prefill(dev(K), dev(V))
-    with pytest.raises(B.InnerQError) as ei:                 # not the format the kernel is built for
-        other.innerq_decode_attention(dev(synth.query(w)))
-    assert ei.value.status == -2
+            check_decode(w, oc, gc, step=step, variants=(3, 4), splits=(0, 2))
+
 
 
 def test_fp16_cache_decode():

@@ -3,7 +3,7 @@
 Collected last on purpose: a run that stops at the first failure has then already run everything else.
 It checks the variant against the regular entry point AND against the CPU oracle on two calls in a row (the
 shared array keeps the first call's contents when the second starts), and that an over-sized configuration
-and the tcgen05 decode variant are refused.
+is refused.
 """
 import numpy as np
 import pytest
@@ -62,17 +62,3 @@ def test_static_scratch_refuses_configurations_beyond_its_size():
     assert ei.value.status == -4
     out = gc.innerq_decode_attention(q)          # the regular entry point still serves it
     assert torch.isfinite(out.float()).all()
-
-
-def test_static_scratch_refuses_the_tcgen05_variant():
-    import torch
-    from paper_2602_23200_b200 import binding as B
-    w = synth.tiny(n_tokens=300)
-    gc = _setup(w)
-    q = torch.from_numpy(synth.query(w)).cuda()
-    gc.innerq_set_decode_options(0, 5)
-    with pytest.raises(B.InnerQError) as ei:
-        gc.innerq_decode_attention_static(q)
-    assert ei.value.status == -2
-    gc.innerq_set_decode_options(0, 0)
-    assert torch.isfinite(gc.innerq_decode_attention_static(q).float()).all()
