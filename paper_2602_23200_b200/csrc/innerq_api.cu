@@ -152,7 +152,7 @@ void make_layout(const innerq_config_t& c, Layout& L, int page_tokens = 0) {
   L.max_splits = ms + (c.w_sink + c.w_recent + L.G + 31) / 32 + 1;
   size_t off = 0;
   L.norm_off = off; off = align_up(off + (size_t)L.U * kD * 4, 256);
-  L.appended_off = off; off = align_up(off + (size_t)L.U * 4, 256);
+  L.appended_off = off; off = align_up(off + (size_t)L.U * 8, 256);      // counts [U], then append part tickets [U]
   if (c.grouping == INNERQ_GROUPING_FP16) {
     place_store(L.k, kNone, 16, 0, c, L.U, off);
     place_store(L.v, kNone, 16, 0, c, L.U, off);

@@ -82,7 +82,8 @@ struct Layout {
   float sm_scale;
   size_t norm_off;     // float [U][D]
   size_t appended_off; // uint32 [U]: token count of the unit after the last append (or prefill) whose writes are
-                       // complete; a decode of N tokens that reads N there may read the rings and the newest rows
+                       // complete; a decode of N tokens that reads N there may read the rings and the newest rows.
+                       // Then uint32 [U]: tickets of the CTAs that share the append of one unit (zero between appends)
   size_t cache_bytes;
   // workspace
   size_t ws_partial_off;   // float [B*Hq][max_splits][kPartialStride]

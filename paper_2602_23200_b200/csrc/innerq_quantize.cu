@@ -282,8 +282,30 @@ __device__ __forceinline__ void append_evict_block(const Layout& L, const Store&
 
 // One appended token of one unit: ring write of the new key / value rows, eviction of the oldest key row and, when
 // a group of G tokens has filled up, of the oldest G value rows (outer grouping: the other way round).
+// Publish: everything this unit's append writes is written.  A decode of N tokens that reads N in the unit's counter
+// (acquire) may read the rings and the newest packed rows without waiting for this kernel to end.  The packed rows
+// will be read by bulk async copies (another memory proxy than these ordinary stores): every thread orders its
+// stores ahead of that proxy first.  n_parts CTAs share the unit's append (one, or five on the step that packs a
+// chunk-coded group): each takes a ticket after its writes, the last one publishes.
+__device__ __forceinline__ void append_publish(const Layout& L, int N, int u, unsigned char* __restrict__ cache, int n_parts) {
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t* counts = reinterpret_cast<uint32_t*>(cache + L.appended_off);
+    __threadfence();
+    if (n_parts > 1) {
+      if (atomicAdd(counts + L.U + u, 1u) != (uint32_t)(n_parts - 1)) return;
+      counts[L.U + u] = 0u;          // ready for the next append
+      __threadfence();               // the other parts' writes (published before their tickets) precede the count
+    }
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(counts + u), "r"((uint32_t)N) : "memory");
+  }
+}
+
+// skip_v_block: the value store's group eviction of this step is done by other CTAs (quarters, see append_kernel)
 __device__ __forceinline__ void append_unit(const Layout& L, const __half* __restrict__ xk, const __half* __restrict__ xv,
-                                            int N, int u, unsigned char* __restrict__ cache, __half* tile, uint32_t* words) {
+                                            int N, int u, unsigned char* __restrict__ cache, __half* tile, uint32_t* words,
+                                            bool skip_v_block = false, int n_parts = 1) {
   const __half k_x = xk[threadIdx.x], v_x = xv[threadIdx.x];
   const bool k_norm = L.k_normalize != 0;
   append_evict_row(L, L.k, xk, N, u, cache, k_norm, words);
@@ -291,18 +313,70 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
   append_write(L, L.k, k_x, N, u, cache);
   append_write(L, L.v, v_x, N, u, cache);
   append_evict_block(L, L.k, N, u, cache, k_norm, tile, words);
-  append_evict_block(L, L.v, N, u, cache, false, tile, words);
-  // Publish: everything this unit's append writes is written.  A decode of N tokens that reads N here (acquire)
-  // may read the rings and the newest packed rows without waiting for this kernel to end.  The packed rows will be
-  // read by bulk async copies (another memory proxy than these ordinary stores): every thread orders its stores
-  // ahead of that proxy before the count is released.
-  asm volatile("fence.proxy.async.global;" ::: "memory");
+  if (!skip_v_block) append_evict_block(L, L.v, N, u, cache, false, tile, words);
+  append_publish(L, N, u, cache, n_parts);
+}
+
+// Quarter of a group eviction of a chunk-coded BLOCK store: channels 32 q .. 32 q + 31 of the G oldest ring tokens
+// (first token t_first; the row appended by this very step, token N - 1, is taken from the call's input x_new, which
+// another CTA is writing to the ring at the same time).  128 threads: lane = channel, warp = quarter of the tokens.
+// The words of a packed chunk that hold these channels hold no others (see block_pos_plane / block_pos_i8: a word
+// belongs to one lane group gid and one half W of the channels), so the quarters write disjoint words.
+__device__ __forceinline__ int chunk_word_quarter(int i, int bits, int perm) {
+  if (bits == 3 && i >= chunk_hi_plane_word()) {
+    const int r = i - chunk_hi_plane_word();
+    return 2 * ((r & 3) >> 1) + ((r >> 2) >> 4);          // word = lane * 4 + (m >> 1), m >> 1 = 2 W + ..; gid = lane / 4
+  }
+  (void)perm;
+  const int r = i & 255;                                   // 4-bit codes: two k-step halves of 256 words
+  return 2 * (r >> 7) + (((r & 127) >> 2) >> 4);           // W = r / 128, gid = ((r % 128) / 4) / 4 -> 2 W + gid / 4
+}
+__device__ void quantize_block_quarter(const TokSrc& src, const __half* __restrict__ x_new, int t_new, int t_first,
+                                       const Layout& L, const Store& S, __half* tile, uint32_t* words, float* red,
+                                       const Rec& rec, int group_j, int q) {
+  const int G = L.G, cl = threadIdx.x & 31, part = threadIdx.x >> 5, c = 32 * q + cl;
+  const int cw = chunk_bytes(S.bits) / 4, n_words = (G / kChunk) * cw, per = G >> 2;
+  for (int i = threadIdx.x; i < G * 4; i += 128) {         // 4 x 16-byte pieces of the quarter per token row
+    const int t = i >> 2, piece = i & 3;
+    const __half* row = t_first + t == t_new ? x_new : src.row(t_first + t);
+    reinterpret_cast<uint4*>(tile)[i] = *reinterpret_cast<const uint4*>(row + 32 * q + piece * 8);
+  }
+  for (int i = threadIdx.x; i < n_words; i += 128) words[i] = 0u;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(reinterpret_cast<uint32_t*>(cache + L.appended_off) + u),
-                 "r"((uint32_t)N)
-                 : "memory");
+  float mn = INFINITY, mx = -INFINITY;
+  for (int t = part * per; t < (part + 1) * per; ++t) {
+    const float x = __half2float(tile[t * 32 + cl]);
+    mn = fminf(mn, x); mx = fmaxf(mx, x);
+  }
+  red[(part * 32 + cl) * 2] = mn; red[(part * 32 + cl) * 2 + 1] = mx;
+  __syncthreads();
+  for (int pp = 0; pp < 4; ++pp) { mn = fminf(mn, red[(pp * 32 + cl) * 2]); mx = fmaxf(mx, red[(pp * 32 + cl) * 2 + 1]); }
+  const GroupParams p = group_params(mn, mx, fmaxf(fabsf(mn), fabsf(mx)), S.bits, L.sym_variant);
+  float ea = 0.f, es = 0.f;
+  if (S.mode == 2) {
+    for (int t = part * per; t < (part + 1) * per; ++t) {
+      const float x = __half2float(tile[t * 32 + cl]);
+      ea += asym_err(p, x, asym_code(p, x));
+      es += sym_err(p, x, sym_code(p, x));
+    }
+    __syncthreads();                                       // the minima / maxima have been read
+    red[(part * 32 + cl) * 2] = ea; red[(part * 32 + cl) * 2 + 1] = es;
+    __syncthreads();
+    ea = 0.f; es = 0.f;
+    for (int pp = 0; pp < 4; ++pp) { ea += red[(pp * 32 + cl) * 2]; es += red[(pp * 32 + cl) * 2 + 1]; }
+  }
+  const bool asym = choose_asym(S.mode, ea, es);
+  for (int t = part * per; t < (part + 1) * per; ++t) {
+    const float x = __half2float(tile[t * 32 + cl]);
+    const uint32_t code = (uint32_t)(int)(asym ? asym_code(p, x) : sym_code(p, x) + p.half);
+    chunk_put(words + (t / kChunk) * cw, t % kChunk, c, S.bits, code, S.perm);
+  }
+  if (part == 0) store_meta(block_meta_ptr(rec, S, group_j), block_meta_index(c), S.meta_bytes, group_meta(p, asym));
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_words; i += 128) {
+    const int ch = i / cw, wi = i - ch * cw;
+    if (chunk_word_quarter(wi, S.bits, S.perm) == q)
+      reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, group_j * (G / kChunk) + ch))[wi] = words[i];
   }
 }
 
@@ -323,9 +397,23 @@ __global__ void __launch_bounds__(128) append_kernel(Layout L, const __half* __r
   const int u = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
-  append_unit(L, k_new + (size_t)u * kD, v_new + (size_t)u * kD, N, u, cache, tile, words);
+  // gridDim.y = 5 on the step that packs a group of G value tokens (inner grouping): row 0 does the per-token work,
+  // rows 1 .. 4 a quarter of the group's channels each, so that this step costs about as much as any other
+  const int n_parts = gridDim.y;
+  if (blockIdx.y == 0) {
+    append_unit(L, k_new + (size_t)u * kD, v_new + (size_t)u * kD, N, u, cache, tile, words, n_parts > 1, n_parts);
+  } else {
+    const Store& R = L.v;
+    const int nq_before = n_quantised(kBlock, N - 1, L.w_sink, L.w_recent, L.G);
+    const __half* ring = reinterpret_cast<const __half*>(cache + R.ring_off + (size_t)u * R.ring_stride);
+    TokSrc src{ring, R.ring_cap, L.w_sink};
+    quantize_block_quarter(src, v_new + (size_t)u * kD, N - 1, L.w_sink + nq_before, L, R, tile, words,
+                           reinterpret_cast<float*>(words + (L.G / kChunk) * 512), unit_rec(L, cache, u), nq_before / L.G,
+                           blockIdx.y - 1);
+    append_publish(L, N, u, cache, n_parts);
+  }
   // one CTA keeps the kernel alive until its predecessor has ended (the chain of completions); the others leave
-  if (late_wait && u == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (late_wait && u == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // The same for several caches of one configuration, each with its own token count: block x = sequence * U + unit,
@@ -483,12 +571,18 @@ int launch_prefill(const Layout& L, unsigned char* cache, unsigned char* ws, con
 // 32-token chunk is at most 512 words; a row-coded group G rows of at most 16 words).  Sized by G, not for the
 // largest G: with G = 32 four of these CTAs fit beside a resident decode CTA, so the append of every unit of the
 // benchmark shapes runs while the previous decode is still streaming.
-static size_t append_smem_bytes(const Layout& L) { return (size_t)L.G * kD * 2 + (size_t)(L.G / kChunk) * 512 * 4; }
+static size_t append_smem_bytes(const Layout& L) {
+  return (size_t)L.G * kD * 2 + (size_t)(L.G / kChunk) * 512 * 4 + 4 * 32 * 2 * 4;      // + the quarters' reduction words
+}
 
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
                   cudaStream_t st, int late_wait) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(L.U); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = append_smem_bytes(L); cfg.stream = st;
+  // the step on which a chunk-coded group of G value tokens is packed gets four more CTAs per unit (see append_kernel)
+  const bool v_group = L.v.kind == kBlock && L.v.code_kind == kBlock && N_after - 1 >= L.w_sink &&
+                       n_quantised(kBlock, N_after, L.w_sink, L.w_recent, L.G) !=
+                           n_quantised(kBlock, N_after - 1, L.w_sink, L.w_recent, L.G);
+  cfg.gridDim = dim3(L.U, v_group ? 5 : 1); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = append_smem_bytes(L); cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
