@@ -666,11 +666,14 @@ int innerq_cache_export(innerq_cache_t* c, innerq_export_t* ex, void* cuda_strea
 }
 
 int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t variant) {
-  if (!c || n_splits < 0 || variant < 0 || variant > 4) return INNERQ_ERR_INVALID_ARG;
+  if (!c || n_splits < 0 || variant < 0 || variant > 7 || variant == 5) return INNERQ_ERR_INVALID_ARG;
   c->opt_splits = n_splits;
   // variants 3 and 4 force the fast kernel with one / two 32-token chunks per loop iteration (process-wide knob)
   if (variant == 3 || variant == 4) { decode_mma_set_chunks_per_iter(variant - 2); variant = 2; }
   else decode_mma_set_chunks_per_iter(0);
+  // variants 6 and 7: the fast kernel without its key-side / value-side arithmetic (timing only, process-wide knob)
+  if (variant == 6 || variant == 7) { decode_mma_set_ablation(variant - 5); variant = 2; }
+  else decode_mma_set_ablation(0);
   c->opt_variant = variant;
   return INNERQ_OK;
 }

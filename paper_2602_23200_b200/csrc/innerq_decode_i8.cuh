@@ -608,7 +608,10 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         const uint32_t* kc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc));
         const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) k_mtile(kc, km, 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
+        for (int mt = 0; mt < 2; ++mt) {
+          if (a.ablation & 1) sc[cc][mt][0] = sc[cc][mt][1] = 0.f;      // timing experiment: no key side
+          else k_mtile(kc, km, 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
+        }
       }
 
       // ---------------- online softmax (log2 domain; raw scores are in integer units: times kfac) -----
@@ -687,7 +690,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         if (SPLIT && (gid >> 1) != slot) { b0 = 0u; b1 = 0u; }      // column pair of this chunk's window slot only
 
         // ---------------- values: 8 m-tiles of 16 channels x one k-step of 32 tokens --------------------
-        {
+        if (!(a.ablation & 2)) {
           const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
           const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
           const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};

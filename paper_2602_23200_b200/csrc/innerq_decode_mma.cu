@@ -9,6 +9,7 @@ namespace iq {
 namespace {
 
 int g_chunks_per_iter = 0;    // tuning knob: 0 automatic, else 1 or 2 chunks of 32 tokens per loop iteration
+int g_ablation = 0;           // timing experiments: see DecodeArgs::ablation
 
 using FormatLauncher = int (*)(const Layout&, const Counts&, const DecodeArgs&, int, int, cudaStream_t);
 
@@ -102,6 +103,7 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
     fill_count_args(L, e.cn, e.a);
     e.a.safe_chunks = safe_chunks_for(L, Ns_safe[i], e.cn);
     e.a.n_q = 1;
+    e.a.ablation = g_ablation;
     e.a.partials = reinterpret_cast<float*>(wss[i] + L.ws_partial_off);
     e.a.pages_host = nullptr;      // paged caches: a batched launch reads every cache's table from its buffer
     e.a.n_pages_host = 0;
@@ -111,6 +113,7 @@ int launch_decode_mma_batched(const Layout& L, int n, const unsigned char* const
 }
 
 void decode_mma_set_chunks_per_iter(int n) { g_chunks_per_iter = (n == 1 || n == 2) ? n : 0; }
+void decode_mma_set_ablation(int mask) { g_ablation = mask & 3; }
 
 // n_q > 1: q and out are [B, n_q, Hq, D], the partials of a launch's (up to) four rows per unit go to
 // multi_partials [U * 4][max_splits][kPartialStride]
@@ -139,6 +142,7 @@ int launch_decode_mma(const Layout& L, const unsigned char* cache, unsigned char
   fill_count_args(L, cn, a);
   a.safe_chunks = safe_chunks_for(L, N_safe, cn);
   a.n_q = n_q;
+  a.ablation = g_ablation;
   a.partials = n_q > 1 ? multi_partials : reinterpret_cast<float*>(ws + L.ws_partial_off);
   a.pages_host = pages_host;
   a.n_pages_host = n_pages_host;

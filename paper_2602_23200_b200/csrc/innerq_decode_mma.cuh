@@ -917,8 +917,8 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
         const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + lead + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
-          float sA, sB;
-          k_mtile(kc, km, 16 * mt, sA, sB);
+          float sA = 0.f, sB = 0.f;
+          if (!(a.ablation & 1)) k_mtile(kc, km, 16 * mt, sA, sB);      // (timing experiment: no key side)
           if constexpr (OUTER) {       // true log2-domain scores right away (the scaling changes from group to group)
             sA = fmaf(sA, kfac_cur, kconst);
             sB = fmaf(sB, kfac_cur, kconst);
@@ -1010,7 +1010,9 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
         else psum += psum_c;
 
         // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
-        if constexpr (VP == 2) {
+        if (a.ablation & 2) {
+          // timing experiment: no value side
+        } else if constexpr (VP == 2) {
           const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
           const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
           const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -1044,7 +1046,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
           }
         }
 
-        if constexpr (VB == 3) {
+        if constexpr (VB == 3) if (!(a.ablation & 2)) {
           // 1-bit plane (weight 4): 4 words per lane, word m/2 holds fields ((m%2)*2 + rh)*4 + 2*ks + kh
           const uint4 hv = *reinterpret_cast<const uint4*>(vc + 256 + lane * 4);
           const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};

@@ -31,6 +31,8 @@ struct DecodeArgs {
   int n_q;               // consecutive query tokens per sequence (1: plain decode).  Row v = i * r + h of a KV head is
                          // head h of query token i; q / out are [B, n_q, Hq, D]; query i does not see the newest
                          // n_q - 1 - i tokens (all of them outside the chunks where keys AND values are packed)
+  int ablation;          // timing experiments only (results are then wrong on purpose): bit 0 leaves out the key side's
+                         // unpack + MMA work of the streaming loop (scores are taken as 0), bit 1 the value side's
   float* partials;       // split partials [rows][max_splits][kPartialStride]: row = global query head (n_q == 1) or
                          // unit * 4 + column of the launch (n_q > 1)
   // HOST side only (paged caches): the cache's page list, which the launcher copies into the kernel's parameter

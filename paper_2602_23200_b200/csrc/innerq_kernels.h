@@ -60,6 +60,7 @@ bool decode_mma_supported(const Layout& L);
 int launch_decode_fp16(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                        __half* out, int n_splits, cudaStream_t st);
 void decode_mma_set_chunks_per_iter(int n);   // tuning: 32-token chunks per loop iteration (1 or 2)
+void decode_mma_set_ablation(int mask);       // timing experiments: bit 0 / 1 = no key-side / value-side work in the loop
 
 
 }  // namespace iq

@@ -7,8 +7,10 @@ Presets: Base (3-bit symmetric K and V), Hybrid (3-bit symmetric K, 2-bit hybrid
 (per-channel K, per-token V) 2-bit cache and the unquantised fp16 cache.  The hybrid mask is decided by the data:
 besides the presets on the workload's own values (whose measured asymmetric fraction is printed), the mask
 ablation rows rebuild the values group by group so that 1, 10, 50 and 99 % of the value groups prefer the
-asymmetric candidate (values_with_mask_density).  Key side and value side are one fused kernel here and are not
-timed separately.
+asymmetric candidate (values_with_mask_density).  Key side and value side are one fused kernel here; what each side
+costs is measured as the difference between the full kernel and the same kernel with that side's unpack + MMA work
+left out of its streaming loop (decode variants 6 and 7 of innerq_set_decode_options, timing only), all bytes still
+streamed: the second table.
 
     python -m paper_2602_23200_b200.latency_study [--out table.md] [--lengths 512,4096,32768]
 
@@ -101,6 +103,32 @@ def time_decode(cache, q, out, flush, reps: int):
     return statistics.median(cold), e0.elapsed_time(e1) * 1e3 / n
 
 
+def time_sides(cache, q, out, reps: int):
+    """(full, without the key side, without the value side) in us per call, back to back; None where the cache's
+    format has no fused kernel."""
+    import torch
+    from . import binding as B
+    res = []
+    for variant in (2, 6, 7):
+        try:
+            cache.innerq_set_decode_options(0, variant)
+            for _ in range(3):
+                cache.innerq_decode_attention(q, out)
+        except B.InnerQError:
+            cache.innerq_set_decode_options(0, 0)
+            return None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 4 * reps
+        e0.record()
+        for _ in range(n):
+            cache.innerq_decode_attention(q, out)
+        e1.record()
+        torch.cuda.synchronize()
+        res.append(e0.elapsed_time(e1) * 1e3 / n)
+    cache.innerq_set_decode_options(0, 0)
+    return tuple(res)
+
+
 def asym_fraction(cache, which: str) -> float:
     e = cache.innerq_cache_export(codes=False)
     s = e.get(which)
@@ -123,9 +151,10 @@ def main(argv=None) -> int:
     K, V = synth.kv_all(layer_workload(n_max))
     Kd, Vd = torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than L2
-    rows, records = [], []
+    rows, records, side_rows = [], [], []
     for name, kw in PRESETS:
         cells = []
+        sides = []
         frac_v = float("nan")
         for n in lengths:
             w = layer_workload(n, **kw)
@@ -139,9 +168,18 @@ def main(argv=None) -> int:
             if n == n_max and w.grouping == synth.INNER:
                 frac_v = asym_fraction(cache, "v_scale")
             cells.append((cold, warm))
-            records.append({"preset": name, "n_tokens": n, "cold_us": round(cold, 2), "warm_us": round(warm, 2)})
+            rec = {"preset": name, "n_tokens": n, "cold_us": round(cold, 2), "warm_us": round(warm, 2)}
+            if w.grouping != synth.FP16:
+                sd = time_sides(cache, q, out, args.reps)
+                sides.append(sd)
+                if sd:
+                    rec.update({"full_us": round(sd[0], 2), "without_key_side_us": round(sd[1], 2),
+                                "without_value_side_us": round(sd[2], 2)})
+            records.append(rec)
             cache.close()
         rows.append((name, frac_v, cells))
+        if sides and all(sides):
+            side_rows.append((name, sides))
         print(f"{name:28s} " + " ".join(f"{c:7.1f}/{wm:<7.1f}" for c, wm in cells), flush=True)
     base_w = layer_workload(n_max)
     for density in MASK_DENSITIES:
@@ -171,6 +209,13 @@ def main(argv=None) -> int:
         lines.append(f"| {tag} | " + " | ".join(f"{c:.1f} / {wm:.1f}" for c, wm in cells) + " |")
     table = "\n".join(lines)
     print("\nµs per decode call, cold (L2 flushed) / warm (back to back):\n" + table)
+    lines = ["| preset | " + " | ".join(str(n) for n in lengths) + " |", "|---|" + "---|" * len(lengths)]
+    for name, sides in side_rows:
+        lines.append(f"| {name} | " + " | ".join(f"{f - nk:.1f} + {f - nv:.1f} of {f:.1f}" for f, nk, nv in sides) + " |")
+    side_table = "\n".join(lines)
+    print("\nµs per call, back to back: key side + value side (full minus the kernel without that side) of the full "
+          "kernel's time; the rest is streaming, soft-max, metadata and fixed cost, which both sides share:\n" + side_table)
+    table = table + "\n\n" + side_table
     if args.out:
         with open(args.out, "w") as f:
             f.write(table + "\n\n" + "\n".join(json.dumps(r) for r in records) + "\n")
