@@ -980,10 +980,13 @@ int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, 
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
-// cpi: chunks of 32 tokens per loop iteration, 0 = automatic (two).
+// cpi: chunks of 32 tokens per loop iteration, 0 = automatic: two, unless a warp gets so few chunks that the second
+// half of an iteration would often be empty (G = 32, where a warp's range may be an odd number of chunks, and fewer
+// than four chunks per warp: short contexts split over many CTAs).
 template <int G, int KM, int VM, bool SPLIT>
 int launch_i8_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
   const bool paged = L.page_groups > 0;
+  if (cpi == 0 && G == 32 && cn.n_qv / kChunk < 4 * kWarps * (n_splits > 0 ? n_splits : 1)) cpi = 1;
   if (cpi == 1)
     return paged ? launch_i8_one_p<G, KM, VM, SPLIT, 1, true>(L, cn, a, n_splits, st)
                  : launch_i8_one_p<G, KM, VM, SPLIT, 1, false>(L, cn, a, n_splits, st);

@@ -13,45 +13,44 @@ int g_ablation = 0;           // timing experiments: see DecodeArgs::ablation
 
 using FormatLauncher = int (*)(const Layout&, const Counts&, const DecodeArgs&, int, int, cudaStream_t);
 
-// The formats with kernels: equal key and value bit widths with full or symmetric-only metadata, and the mixed
-// 3-bit-key / 2-bit-value combinations with symmetric keys.
-FormatLauncher format_launcher(const Layout& L) {
+// The formats with kernels: every combination of 2 / 3 / 4-bit keys and values with full or scale-only metadata
+// (2-bit keys with 2-bit values: the integer-MMA kernel), and the outer-grouped comparison cache at 2 and 4 bits.
+struct FormatEntry {
+  int kb, vb, km, vm;
+  FormatLauncher one;
+  int (*batched)(const Layout&, SeqTable&, int, int, int, cudaStream_t);
+};
+#define IQ_FORMAT_ENTRY(KB, VB, KM, VM) \
+  {KB, VB, KM, VM, &launch_decode_mma_k##KB##v##VB##_m##KM##VM, &launch_decode_mma_k##KB##v##VB##_m##KM##VM##_batched},
+const FormatEntry kFormats[] = {IQ_FOR_EACH_MMA_FORMAT(IQ_FORMAT_ENTRY)};
+#undef IQ_FORMAT_ENTRY
+
+const FormatEntry* find_format(const Layout& L) {
   if (L.G != 32 && L.G != 64 && L.G != 128) return nullptr;
-  if (L.grouping == 1) {      // outer grouping: per-channel key groups on token rows, per-token value groups on chunks
-    if (L.k.kind != kBlock || L.k.code_kind != kRow || L.v.kind != kRow || L.v.code_kind != kBlock) return nullptr;
-    if (L.k.meta_bytes != 4 || L.v.meta_bytes != 4 || L.k.bits != L.v.bits) return nullptr;
-    if (L.k.bits == 2) return &launch_decode_mma_outer_k2v2;
-    if (L.k.bits == 4) return &launch_decode_mma_outer_k4v4;
-    return nullptr;
-  }
   if (L.grouping != 0 || L.k.kind != kRow || L.v.kind != kBlock) return nullptr;
-  const int kb = L.k.bits, vb = L.v.bits, km = L.k.meta_bytes, vm = L.v.meta_bytes;
-  if (kb == 2 && vb == 2 && km == 4 && vm == 4) return &launch_decode_mma_k2v2_m44;
-  if (kb == 4 && vb == 4 && km == 4 && vm == 4) return &launch_decode_mma_k4v4_m44;
-  if (kb == 3 && vb == 3 && km == 4 && vm == 4) return &launch_decode_mma_k3v3_m44;
-  if (kb == 2 && vb == 2 && km == 2 && vm == 2) return &launch_decode_mma_k2v2_m22;
-  if (kb == 3 && vb == 3 && km == 2 && vm == 2) return &launch_decode_mma_k3v3_m22;
-  if (kb == 4 && vb == 4 && km == 2 && vm == 2) return &launch_decode_mma_k4v4_m22;
-  if (kb == 3 && vb == 2 && km == 2 && vm == 2) return &launch_decode_mma_k3v2_m22;
-  if (kb == 3 && vb == 2 && km == 2 && vm == 4) return &launch_decode_mma_k3v2_m24;
+  for (const FormatEntry& f : kFormats)
+    if (f.kb == L.k.bits && f.vb == L.v.bits && f.km == L.k.meta_bytes && f.vm == L.v.meta_bytes) return &f;
   return nullptr;
+}
+
+bool is_outer(const Layout& L) {
+  return L.grouping == 1 && (L.G == 32 || L.G == 64 || L.G == 128) && L.k.kind == kBlock && L.k.code_kind == kRow &&
+         L.v.kind == kRow && L.v.code_kind == kBlock && L.k.meta_bytes == 4 && L.v.meta_bytes == 4 &&
+         L.k.bits == L.v.bits && (L.k.bits == 2 || L.k.bits == 4);
+}
+
+FormatLauncher format_launcher(const Layout& L) {
+  if (is_outer(L)) return L.k.bits == 2 ? &launch_decode_mma_outer_k2v2 : &launch_decode_mma_outer_k4v4;
+  const FormatEntry* f = find_format(L);
+  return f ? f->one : nullptr;
 }
 
 using BatchedLauncher = int (*)(const Layout&, SeqTable&, int, int, int, cudaStream_t);
 
 BatchedLauncher batched_launcher(const Layout& L) {
-  const FormatLauncher one = format_launcher(L);
-  if (one == &launch_decode_mma_outer_k2v2) return &launch_decode_mma_outer_k2v2_batched;
-  if (one == &launch_decode_mma_outer_k4v4) return &launch_decode_mma_outer_k4v4_batched;
-  if (one == &launch_decode_mma_k2v2_m44) return &launch_decode_mma_k2v2_m44_batched;
-  if (one == &launch_decode_mma_k4v4_m44) return &launch_decode_mma_k4v4_m44_batched;
-  if (one == &launch_decode_mma_k3v3_m44) return &launch_decode_mma_k3v3_m44_batched;
-  if (one == &launch_decode_mma_k2v2_m22) return &launch_decode_mma_k2v2_m22_batched;
-  if (one == &launch_decode_mma_k3v3_m22) return &launch_decode_mma_k3v3_m22_batched;
-  if (one == &launch_decode_mma_k4v4_m22) return &launch_decode_mma_k4v4_m22_batched;
-  if (one == &launch_decode_mma_k3v2_m22) return &launch_decode_mma_k3v2_m22_batched;
-  if (one == &launch_decode_mma_k3v2_m24) return &launch_decode_mma_k3v2_m24_batched;
-  return nullptr;
+  if (is_outer(L)) return L.k.bits == 2 ? &launch_decode_mma_outer_k2v2_batched : &launch_decode_mma_outer_k4v4_batched;
+  const FormatEntry* f = find_format(L);
+  return f ? f->batched : nullptr;
 }
 
 // The launch parameters of one cache that follow from its token count alone.

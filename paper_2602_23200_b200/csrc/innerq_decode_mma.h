@@ -57,31 +57,24 @@ struct SeqTable {
   SeqArgs s[kMaxSeqs];
 };
 
-// Launchers by format: k<key bits>v<value bits>_m<bytes per key metadata entry><bytes per value metadata entry>.
-// cpi: chunks of 32 tokens per loop iteration (0 = automatic).  Return the number of launches, or < 0.
-int launch_decode_mma_k2v2_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k4v4_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k3v3_m44(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k2v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k3v3_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k4v4_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k3v2_m22(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-int launch_decode_mma_k3v2_m24(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);
-
-// The same for a table of sequences (n_seqs <= kMaxSeqs entries with cn and the N-dependent fields of a filled in).
-#define IQ_DECLARE_MMA_BATCHED(name) \
-  int name##_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st);
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k2v2_m44)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k4v4_m44)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v3_m44)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k2v2_m22)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v3_m22)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k4v4_m22)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v2_m22)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_k3v2_m24)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_outer_k2v2)
-IQ_DECLARE_MMA_BATCHED(launch_decode_mma_outer_k4v4)
-#undef IQ_DECLARE_MMA_BATCHED
+// Launchers by format: k<key bits>v<value bits>_m<bytes per key metadata entry><bytes per value metadata entry>, every
+// combination of 2 / 3 / 4-bit keys and values with 2-byte (scale only: symmetric mode) or 4-byte (scale | zero-point)
+// metadata.  cpi: chunks of 32 tokens per loop iteration (0 = automatic).  Return the number of launches, or < 0.
+// The _batched form takes a table of sequences (n_seqs <= kMaxSeqs entries with cn and the N-dependent fields of a).
+#define IQ_FOR_EACH_META(X, KB, VB) X(KB, VB, 2, 2) X(KB, VB, 2, 4) X(KB, VB, 4, 2) X(KB, VB, 4, 4)
+#define IQ_FOR_EACH_MMA_FORMAT(X)                                                                        \
+  IQ_FOR_EACH_META(X, 2, 2)                                                                              \
+  IQ_FOR_EACH_META(X, 2, 3) IQ_FOR_EACH_META(X, 2, 4) IQ_FOR_EACH_META(X, 3, 2) IQ_FOR_EACH_META(X, 3, 3) \
+  IQ_FOR_EACH_META(X, 3, 4) IQ_FOR_EACH_META(X, 4, 2) IQ_FOR_EACH_META(X, 4, 3) IQ_FOR_EACH_META(X, 4, 4)
+#define IQ_DECLARE_MMA_FORMAT(KB, VB, KM, VM)                                                                      \
+  int launch_decode_mma_k##KB##v##VB##_m##KM##VM(const Layout& L, const Counts& cn, const DecodeArgs& a,          \
+                                                 int n_splits, int cpi, cudaStream_t st);                           \
+  int launch_decode_mma_k##KB##v##VB##_m##KM##VM##_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, \
+                                                           int cpi, cudaStream_t st);
+IQ_FOR_EACH_MMA_FORMAT(IQ_DECLARE_MMA_FORMAT)
+#undef IQ_DECLARE_MMA_FORMAT
+int launch_decode_mma_outer_k2v2_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st);
+int launch_decode_mma_outer_k4v4_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st);
 
 // Outer-grouped comparison cache (same argument list; cpi is ignored).
 int launch_decode_mma_outer_k2v2(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st);

@@ -1,0 +1,6 @@
+// Decode kernels of one packed format: 3-bit keys, 2-bit values, 4 / 2 bytes per key / value metadata entry.
+#include "innerq_decode_mma.cuh"
+
+namespace iq {
+IQ_DEFINE_MMA_FORMAT(3, 2, 4, 2)
+}  // namespace iq

@@ -135,9 +135,9 @@ def test_mixed_bits_and_modes():
     check_decode(w, oc, gc, variants=(0, 1, 3))
 
 
-# key bits, value bits, key mode, value mode, G, query heads per KV head, N: the packed formats the fused kernel
-# is built for beyond equal-width hybrid ones (3-bit planes, symmetric-only 2-byte metadata, 3-bit keys with
-# 2-bit values), with one query head per KV head (group-per-column kernel), several, and two passes of four
+# key bits, value bits, key mode, value mode, G, query heads per KV head, N: packed formats of the fused kernel
+# beyond equal-width hybrid ones (3-bit planes, symmetric-only 2-byte metadata, keys and values of different widths
+# or metadata forms), with one query head per KV head (group-per-column kernel), several, and two passes of four
 FORMATS = [
     (3, 3, O.HYBRID, O.HYBRID, 32, 1, 700),
     (3, 3, O.SYM, O.SYM, 32, 1, 700),
@@ -149,6 +149,14 @@ FORMATS = [
     (4, 4, O.SYM, O.SYM, 32, 1, 500),
     (3, 3, O.ASYM, O.ASYM, 128, 8, 900),
     (3, 3, O.SYM, O.SYM, 64, 8, 555),
+    # keys and values of different widths, and 2-bit caches whose two tensors differ in metadata form
+    (2, 4, O.HYBRID, O.HYBRID, 32, 1, 700),
+    (4, 2, O.HYBRID, O.ASYM, 64, 4, 600),
+    (2, 3, O.SYM, O.HYBRID, 32, 2, 500),
+    (4, 3, O.HYBRID, O.SYM, 128, 4, 900),
+    (3, 4, O.SYM, O.SYM, 64, 1, 450),
+    (2, 2, O.SYM, O.HYBRID, 32, 1, 1200),
+    (2, 2, O.HYBRID, O.SYM, 64, 4, 640),
 ]
 
 
