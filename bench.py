@@ -360,6 +360,23 @@ class Legs:
         self.torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / n
 
+    def sides(self, n=64):
+        """us per decode in a chain for the full fused kernel, without its key-side arithmetic and without its
+        value-side arithmetic (decode options 6 / 7: timing only, all bytes still streamed); None if the cache's format
+        has no fused kernel."""
+        from paper_2602_23200_b200.binding import InnerQError
+        res = {}
+        try:
+            for name, variant in (("full", 2), ("without_key_side", 6), ("without_value_side", 7)):
+                for c in self.caches:
+                    c.innerq_set_decode_options(0, variant)
+                res[name] = self.decodes_chained(n)
+        except InnerQError:
+            res = None
+        for c in self.caches:
+            c.innerq_set_decode_options(0, 0)
+        return res
+
     def appends_bracketed(self, n):
         evs = [(self._ev(), self._ev()) for _ in range(n)]
         self.delay()
@@ -466,11 +483,12 @@ def measure_config(name, peak, R=2, n_steps=128):
     alone = stats(legs.decodes_bracketed(32))
     chain = legs.decodes_chained(64)
     step, step_host = legs.steps(n_steps, warm=32)
+    sides = legs.sides()
     gbs = lambda us: nbytes / us / 1e3
     res.update({
         "bytes_per_decode_minimal": nbytes, "sym_group_fraction": {"k": sym_k, "v": sym_v},
         "us_per_decode_alone": alone, "us_per_decode_chained": chain, "us_per_step": step,
-        "host_us_per_step_enqueue": step_host,
+        "host_us_per_step_enqueue": step_host, "us_per_decode_chained_by_side": sides,
         "frac_of_measured_peak": {"alone_median": gbs(alone["median"]) / peak, "chained": gbs(chain) / peak,
                                   "step": gbs(step) / peak},
         "pct_of_nominal_8TBs": {"alone_median": gbs(alone["median"]) / 80.0, "chained": gbs(chain) / 80.0,
@@ -653,6 +671,7 @@ def run_ours(args, w):
                    "us_per_decode_back_to_back": legs.decodes_chained(64, caches=literal_caches)}
         for c in literal_caches:
             c.close()
+    sides = legs.sides() if packed and not (args.splits or args.variant) else None
     append_us = float(np.median(legs.appends_bracketed(16)))
     multi = None
     if args.n_q > 1 and packed:
@@ -701,7 +720,7 @@ def run_ours(args, w):
             "us_per_step_fixed_leg": {"steps": LEG, "us": leg_us, "frac_of_measured_peak": gbs(leg_us) / peak,
                                       "host_us_per_step_enqueue": leg_host_us},
             "us_per_decode": alone["median"], "us_per_decode_alone": alone, "us_per_decode_back_to_back": b2b_us,
-            "us_per_append_median": append_us,
+            "us_per_append_median": append_us, "us_per_decode_back_to_back_by_side": sides,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config_dict(w, args),
             "bytes_per_decode": {"dense_zero_points": bytes_dense, "minimal": bytes_min,

@@ -281,7 +281,9 @@ int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_s
  *              3 / 4 warp-MMA kernel with one / two 32-token chunks per loop iteration (sets a process-wide knob).
  *              6 / 7 TIMING ONLY, the output is wrong on purpose: the warp-MMA kernel with the unpack + MMA work of
  *              its key side (6) or value side (7) left out of the streaming loop, the bytes still streamed; what
- *              a side costs is the difference to the full kernel (process-wide knob; any other variant clears it).
+ *              a side costs is the difference to the full kernel (process-wide knob; any other variant clears it;
+ *              contiguous caches in the 2-bit formats, the 3-bit / 3-bit, 3-bit / 2-bit and 4-bit / 4-bit formats of
+ *              the latency study and the outer-grouped cache: UNSUPPORTED elsewhere).
  * Errors: INVALID_ARG. */
 int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
 

@@ -135,9 +135,15 @@ def dequantize_groups(code, scale_bits, zero_bits, bits: int):
     return s[..., None] * np.asarray(code).astype(f64) + z_eff[..., None]
 
 
-def channel_norm(K):
-    """norm[c] = sqrt(max_t |K[t, c]|) in float32, 0 -> 1.  K: fp16 [..., N, D] -> float32 [..., D]."""
+def channel_norm(K, all_heads: bool = False):
+    """norm[c] = sqrt(max_t |K[t, c]|) in float32, 0 -> 1.  K: fp16 [..., N, D] -> float32 [..., D].
+
+    all_heads: the literal scope of the paper's formula, max over ALL leading axes (batch, heads) and tokens: one
+    vector of D factors, broadcast back to every unit.  The default (the reading taken here, and the only one the
+    CUDA path has) is one vector per (batch, KV head) unit."""
     m = np.abs(np.asarray(K).astype(f32)).max(axis=-2)
+    if all_heads:
+        m = np.broadcast_to(m.reshape(-1, m.shape[-1]).max(axis=0), m.shape)
     n = np.sqrt(m).astype(f32)
     return np.where(n == 0, f32(1.0), n).astype(f32)
 
@@ -260,13 +266,14 @@ class OracleCache:
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, group, k_bits, v_bits,
                  k_mode=HYBRID, v_mode=HYBRID, sym_variant=FULLRANGE, w_sink=4, w_recent=128,
-                 grouping=INNER, k_normalize=1, sm_scale=0.0):
+                 grouping=INNER, k_normalize=1, sm_scale=0.0, norm_all_heads=False):
         assert n_q_heads % n_kv_heads == 0 and head_dim % group == 0
         self.B, self.Hq, self.Hkv, self.D = batch, n_q_heads, n_kv_heads, head_dim
         self.U = batch * n_kv_heads
         self.G, self.grouping = group, grouping
         self.w_sink, self.w_recent = w_sink, w_recent
         self.k_normalize = bool(k_normalize) and grouping == INNER
+        self.norm_all_heads = bool(norm_all_heads)      # literal cross-head scope of the key norm (oracle only)
         self.sm_scale = float(sm_scale) if sm_scale else 1.0 / np.sqrt(head_dim)
         self.N = 0
         self.norm = np.ones((self.U, head_dim), dtype=f32)
@@ -294,7 +301,7 @@ class OracleCache:
             self.K, self.V = K.copy(), V.copy()
             return
         if self.k_normalize:
-            self.norm = channel_norm(K) if norm is None else np.asarray(norm, dtype=f32).reshape(self.U, self.D)
+            self.norm = channel_norm(K, self.norm_all_heads) if norm is None else np.asarray(norm, dtype=f32).reshape(self.U, self.D)
         self.k.prefill(K, self._inv_norm())
         self.v.prefill(V, None)
 

@@ -57,7 +57,9 @@ constexpr float kPScale = 65535.0f;          // p <= 1 as 16 bits: two unsigned 
 // head, G = 32): the 8 columns are 4 groups x 2 digits for keys and 4 value groups of a window x 2 digits for
 // values, which removes the 4x redundancy a quad otherwise has in decoding per-group metadata; CPI: chunks of 32
 // tokens per loop iteration.
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
+// ABL (timing experiments only, results wrong on purpose): bit 0 leaves out the key side's unpack + MMA work of the
+// streaming loop (scores taken as 0), bit 1 the value side's; all bytes are still streamed.
+template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u,
                                                const PageIds* ptab = nullptr) {
   using SL = StageLayout<2, 2, G, KM, VM, CPI>;
@@ -609,7 +611,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffKMeta);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
-          if (a.ablation & 1) sc[cc][mt][0] = sc[cc][mt][1] = 0.f;      // timing experiment: no key side
+          if constexpr (ABL & 1) sc[cc][mt][0] = sc[cc][mt][1] = 0.f;      // timing experiment: no key side
           else k_mtile(kc, km, 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
         }
       }
@@ -690,7 +692,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         if (SPLIT && (gid >> 1) != slot) { b0 = 0u; b1 = 0u; }      // column pair of this chunk's window slot only
 
         // ---------------- values: 8 m-tiles of 16 channels x one k-step of 32 tokens --------------------
-        if (!(a.ablation & 2)) {
+        if constexpr (!(ABL & 2)) {
           const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
           const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
           const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -867,10 +869,10 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 
 
 // One cache: block x = unit.
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
+template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  decode_i8_body<G, KM, VM, SPLIT, CPI, PAGED>(L, cn, a, blockIdx.x);
+  decode_i8_body<G, KM, VM, SPLIT, CPI, PAGED, ABL>(L, cn, a, blockIdx.x);
 }
 // One paged cache with its page table in the parameter space (read in place: no look-up in device memory).
 template <int G, int KM, int VM, bool SPLIT, int CPI>
@@ -920,8 +922,18 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
     cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t err;
     if constexpr (PAGED) {
+      if (a.ablation) return -2;      // the timing instances exist for contiguous caches only
       err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
                             : cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
+    } else if (a.ablation == 1 || a.ablation == 2) {
+      static std::atomic<unsigned long long> configured_a1{0}, configured_a2{0};
+      if (a.ablation == 1) {
+        if (!opt_in_dynamic_smem(decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 1>, L, cn, a);
+      } else {
+        if (!opt_in_dynamic_smem(decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
+      }
     } else {
       err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     }

@@ -245,7 +245,9 @@ __device__ __noinline__ void merge_parts(const float* __restrict__ partials, flo
 // metadata, which leads the group record), for values p_t * S_{t,g} (one operand set per channel group the
 // m-tile's rows fall into); zero-points contribute sum_c q''_c Z_jc per group and sum_t p_t Z_{t,g} per channel
 // group.  One chunk per iteration, four heads per pass.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
+// ABL (timing experiments only, results wrong on purpose): bit 0 leaves out the key side's unpack + MMA work of the
+// streaming loop (scores taken as 0), bit 1 the value side's; all bytes are still streamed.
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false, int ABL = 0>
 __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u,
                                                 const PageIds* ptab = nullptr) {
   constexpr int KP = KB == 3 ? 2 : KB, VP = VB == 3 ? 2 : VB;     // bits of the primary code plane
@@ -918,7 +920,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           float sA = 0.f, sB = 0.f;
-          if (!(a.ablation & 1)) k_mtile(kc, km, 16 * mt, sA, sB);      // (timing experiment: no key side)
+          if constexpr (!(ABL & 1)) k_mtile(kc, km, 16 * mt, sA, sB);      // (else: timing experiment, no key side)
           if constexpr (OUTER) {       // true log2-domain scores right away (the scaling changes from group to group)
             sA = fmaf(sA, kfac_cur, kconst);
             sB = fmaf(sB, kfac_cur, kconst);
@@ -1010,7 +1012,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
         else psum += psum_c;
 
         // ---------------- values: 8 m-tiles of 16 channels x 2 k-steps of 16 tokens ------------------
-        if (a.ablation & 2) {
+        if constexpr (ABL & 2) {
           // timing experiment: no value side
         } else if constexpr (VP == 2) {
           const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
@@ -1046,7 +1048,7 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
           }
         }
 
-        if constexpr (VB == 3) if (!(a.ablation & 2)) {
+        if constexpr (VB == 3 && !(ABL & 2)) {
           // 1-bit plane (weight 4): 4 words per lane, word m/2 holds fields ((m%2)*2 + rh)*4 + 2*ks + kh
           const uint4 hv = *reinterpret_cast<const uint4*>(vc + 256 + lane * 4);
           const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
@@ -1254,10 +1256,10 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
 }
 
 // One cache: block x = unit.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool OUTER = false, bool PAGED = false, int ABL = 0>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>(L, cn, a, blockIdx.x);
+  decode_mma_body<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED, ABL>(L, cn, a, blockIdx.x);
 }
 
 // One paged cache with its page table in the parameter space (read in place: no look-up in device memory).
@@ -1335,8 +1337,22 @@ int launch_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, 
     cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t err;
     if constexpr (PAGED) {
+      if (a.ablation) return -2;      // the timing instances exist for contiguous caches only
       err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_mma_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER>, L, cn, a, ids)
                             : cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a);
+    } else if (a.ablation == 1 || a.ablation == 2) {
+#ifdef IQ_WITH_TIMING_INSTANCES      // defined by the translation units of the formats the latency study times
+      static std::atomic<unsigned long long> configured_a1{0}, configured_a2{0};
+      if (a.ablation == 1) {
+        if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false, 1>, kSmem, configured_a1)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false, 1>, L, cn, a);
+      } else {
+        if (!opt_in_dynamic_smem(decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false, 2>, kSmem, configured_a2)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false, 2>, L, cn, a);
+      }
+#else
+      return -2;
+#endif
     } else {
       err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, PAGED>, L, cn, a);
     }

@@ -308,3 +308,28 @@ def test_multi_query_decode_is_causal_attention(grouping, n_q):
                     assert np.allclose(out[b, :, j], ref, rtol=1e-11, atol=1e-12)
         # the newest query sees everything: the same as the single-token decode
         assert np.array_equal(out[:, n_q - 1], c.decode(q[:, n_q - 1]))
+
+
+def test_key_norm_scopes_per_unit_and_across_heads():
+    # Section "Per-channel Normalization of K": norm_k = sqrt(max |K[:, :, k]|).  Read per (batch, KV head) unit by
+    # default; the literal scope takes the maximum over all heads as well (oracle-only switch).  Either way the norm
+    # cancels between q' = q * norm and k / norm, so with every token inside the windows both give plain attention,
+    # and with quantised rows the two differ only through the quantisation grid.
+    rng = np.random.default_rng(11)
+    K = rng.standard_normal((2, 3, 40, 128)).astype(np.float16)
+    K[1, 2, 7, 5] = 50.0                                        # one large key entry in one head
+    per_unit = O.channel_norm(K)
+    literal = O.channel_norm(K, all_heads=True)
+    assert per_unit.shape == literal.shape == (2, 3, 128)
+    assert per_unit[1, 2, 5] == np.float32(np.sqrt(np.float32(50.0))) and per_unit[0, 0, 5] < 3
+    assert np.all(literal == literal[0, 0]) and literal[0, 0, 5] == np.float32(np.sqrt(np.float32(50.0)))
+    assert np.all(literal >= per_unit)
+    V = rng.standard_normal((2, 3, 40, 128)).astype(np.float16)
+    q = rng.standard_normal((2, 3, 128)).astype(np.float16)
+    outs = []
+    for flag in (False, True):
+        oc = O.OracleCache(2, 3, 3, 128, 64, 32, 2, 2, w_sink=4, w_recent=8, norm_all_heads=flag)
+        oc.prefill(K, V)
+        assert np.array_equal(oc.norm.reshape(2, 3, 128), literal if flag else per_unit)
+        outs.append(oc.decode(q))
+    assert np.allclose(outs[0], outs[1], atol=0.5) and not np.array_equal(outs[0], outs[1])
