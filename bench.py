@@ -44,7 +44,8 @@ D = 128
 
 
 def workload_by_name(name: str):
-    """c1 .. c4 (c3_4bit / c3_2bit); a suffix "+fp16" or "+outer" selects the comparison cache of the same shape."""
+    """c1 .. c4 (c3_4bit / c3_2bit), c5_b<bits>_g<group>_<hybrid|asym|sym|literal> (sweep on the config-3 shape);
+    a suffix "+fp16" or "+outer" selects the comparison cache of the same shape."""
     if "+" in name:
         base, variant = name.split("+", 1)
         w = workload_by_name(base)
@@ -63,6 +64,14 @@ def workload_by_name(name: str):
         return synth.config3(2)
     if name == "c4":
         return synth.config4()
+    if name.startswith("c5_"):      # sweep point on the config-3 shape: c5_b<bits>_g<group>_<hybrid|asym|sym|literal>
+        try:
+            _, b, g, mode = name.split("_")
+            bits, group = int(b[1:]), int(g[1:])
+            m = {"hybrid": synth.HYBRID, "asym": synth.ASYM, "sym": synth.SYM, "literal": synth.HYBRID}[mode]
+            return synth.config5(bits, group, m, synth.INNER, 1 if mode == "literal" else 0).with_(name=name)
+        except (ValueError, KeyError):
+            pass
     raise SystemExit(f"unknown workload {name}")
 
 

@@ -275,6 +275,17 @@ int innerq_decode_attention_static(innerq_cache_t* cache, const void* q, void* o
  * stream reaches the enqueued kernels.  Errors: INVALID_ARG, CUDA. */
 int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_stream);
 
+/* The inverse of innerq_cache_export (checkpoint / resume, moving a sequence between caches or processes): fills the
+ * cache for `n_tokens` tokens from canonical arrays of the SAME configuration, in the shapes and order that the
+ * export writes (innerq_export_t; its count fields are ignored: the partition of n_tokens into sink, packed and recent
+ * tokens is a function of n_tokens and the configuration).  Replaces the cache's contents like a prefill; a cache
+ * restored this way continues (append, decode) exactly like the one that was exported.  The arrays are read when the
+ * stream reaches the enqueued kernels and must stay valid until then.  Codes are taken as given (values above 2^b - 1
+ * would corrupt neighbouring fields: the caller's responsibility).  The paper has no counterpart.
+ * Errors: INVALID_ARG (a needed array is NULL), CAPACITY (n_tokens > max_tokens, or a paged cache without the pages
+ * for n_tokens), CUDA. */
+int innerq_cache_import(innerq_cache_t* cache, const innerq_export_t* ex, int32_t n_tokens, void* cuda_stream);
+
 /* Tuning knobs for experiments; both default to 0 = automatic.
  *   n_splits : number of token ranges each unit is split into by the decode kernel.
  *   variant  : 0 automatic, 1 plain SIMT kernel, 2 warp-MMA kernel (where supported; UNSUPPORTED otherwise),

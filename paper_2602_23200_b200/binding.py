@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "innerq_append_token_batched", "innerq_decode_attention_batched",
     "innerq_paged_cache_bytes", "innerq_cache_create_paged", "innerq_cache_pages_for", "innerq_cache_pages_assigned",
     "innerq_cache_assign_pages", "innerq_cache_release_pages",
-    "innerq_cache_export", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
+    "innerq_cache_export", "innerq_cache_import", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
     "innerq_status_string",
 )
 
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
     L.innerq_cache_assign_pages.argtypes = [vp, C.POINTER(i32), i32, vp]
     L.innerq_cache_release_pages.argtypes = [vp, C.POINTER(i32), i32]
     L.innerq_cache_export.argtypes = [vp, C.POINTER(innerq_export_t), vp]
+    L.innerq_cache_import.argtypes = [vp, C.POINTER(innerq_export_t), C.c_int32, vp]
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
     L.innerq_read_device_error.argtypes = [vp, vp]
@@ -402,6 +403,41 @@ class InnerQCache:
 
     def innerq_last_launch_count(self, which: int) -> int:
         return _check(lib().innerq_last_launch_count(self._h, which), "innerq_last_launch_count")
+
+    def innerq_cache_import(self, arrays: dict, stream=None):
+        """Fills the cache from the dict innerq_cache_export returned for a cache of the same configuration (numpy
+        arrays trimmed to the live counts; they are padded back to the capacity shapes here and copied to the device)."""
+        import torch
+        c = self.cfg
+        U, D, G, cap = self.units, c.head_dim, c.group, c.max_tokens
+        fp16 = c.grouping == GROUPING_FP16
+        inner = c.grouping == GROUPING_INNER
+        n_tokens = int(arrays["n_tokens"])
+
+        def pad(a, shape, dtype):
+            t = torch.zeros(shape, dtype=dtype, device=self.device)
+            if a is not None and a.size:
+                src = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+                t[tuple(slice(0, n) for n in src.shape)] = src.to(self.device)
+            return t
+
+        row_meta, blk_meta = (U, cap, D // G), (U, cap // G + 1, D)
+        t = {"norm": pad(arrays["norm"].reshape(U, D), (U, D), torch.float32)}
+        sink_cap = cap if fp16 else c.w_sink
+        for k in ("k_sink", "v_sink"):
+            t[k] = pad(arrays[k], (U, max(sink_cap, 1), D), torch.float16)
+        if not fp16:
+            km, vm = (row_meta, blk_meta) if inner else (blk_meta, row_meta)
+            t["k_code"], t["v_code"] = pad(arrays["k_code"], (U, cap, D), torch.uint8), pad(arrays["v_code"], (U, cap, D), torch.uint8)
+            t["k_scale"], t["k_zero"] = pad(arrays["k_scale"], km, torch.int16), pad(arrays["k_zero"], km, torch.int16)
+            t["v_scale"], t["v_zero"] = pad(arrays["v_scale"], vm, torch.int16), pad(arrays["v_zero"], vm, torch.int16)
+            t["k_recent"] = pad(arrays["k_recent"], (U, c.w_recent + G, D), torch.float16)
+            t["v_recent"] = pad(arrays["v_recent"], (U, c.w_recent + G, D), torch.float16)
+        ex = innerq_export_t()
+        for name, ten in t.items():
+            setattr(ex, name, ten.data_ptr())
+        _check(lib().innerq_cache_import(self._h, C.byref(ex), n_tokens, _stream_ptr(stream, self.device)), "innerq_cache_import")
+        torch.cuda.synchronize(self.device)      # the temporaries above may go once the kernels have read them
 
     def innerq_cache_export(self, stream=None, codes: bool = True) -> dict:
         """Canonical (unpacked) cache contents as numpy arrays trimmed to the live counts."""

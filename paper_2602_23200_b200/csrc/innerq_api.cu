@@ -665,6 +665,26 @@ int innerq_cache_export(innerq_cache_t* c, innerq_export_t* ex, void* cuda_strea
   return INNERQ_OK;
 }
 
+int innerq_cache_import(innerq_cache_t* c, const innerq_export_t* ex, int32_t n_tokens, void* cuda_stream) {
+  if (!c || !ex || n_tokens < 0) return INNERQ_ERR_INVALID_ARG;
+  if (n_tokens > c->L.max_tokens || !has_pages_for(c, n_tokens)) return INNERQ_ERR_CAPACITY;
+  const bool fp16 = c->L.k.kind == kNone;
+  if (!ex->norm || !ex->k_sink || !ex->v_sink) return INNERQ_ERR_INVALID_ARG;
+  if (!fp16) {
+    if (!ex->k_code || !ex->v_code || !ex->k_scale || !ex->v_scale || !ex->k_recent || !ex->v_recent) return INNERQ_ERR_INVALID_ARG;
+    if ((c->L.k.meta_bytes == 4 && !ex->k_zero) || (c->L.v.meta_bytes == 4 && !ex->v_zero)) return INNERQ_ERR_INVALID_ARG;
+  }
+  ExportPtrs p{ex->k_code, ex->v_code, ex->k_scale, ex->k_zero, ex->v_scale, ex->v_zero,
+               ex->norm,   ex->k_sink, ex->v_sink,  ex->k_recent, ex->v_recent};
+  const int n = launch_import(c->L, c->cache, n_tokens, p, static_cast<cudaStream_t>(cuda_stream));
+  if (n < 0) return INNERQ_ERR_CUDA;
+  c->N = n_tokens;
+  c->N_safe = 0;              // as after a prefill: the next decode waits for these kernels before it reads anything
+  c->reads_settled = 0;
+  c->launches[0] = n;
+  return INNERQ_OK;
+}
+
 int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t variant) {
   if (!c || n_splits < 0 || variant < 0 || variant > 7 || variant == 5) return INNERQ_ERR_INVALID_ARG;
   c->opt_splits = n_splits;

@@ -39,6 +39,8 @@ int launch_quantize_store_prefill(const Layout& L, const Store& S, const __half*
 int launch_append(const Layout& L, unsigned char* cache, const __half* k_new, const __half* v_new, int N_after,
                   cudaStream_t st, int late_wait = 0);
 int launch_export(const Layout& L, const unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st);
+// The inverse: fills the cache (packed records, windows, norms, counts) for N tokens from canonical arrays.
+int launch_import(const Layout& L, unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st);
 
 // Generic SIMT decode (any store kinds, bits, group sizes): split kernel + merge kernel.
 int launch_decode_simt(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,

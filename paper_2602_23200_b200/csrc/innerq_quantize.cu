@@ -487,6 +487,58 @@ __global__ void export_store_kernel(Layout L, Store S, const unsigned char* __re
   }
 }
 
+// ------------------------------------------------------------------ canonical import (the inverse of the export)
+// Pass 0 clears the packed rows / chunks of the first n_q tokens (the codes are OR-ed in), pass 1 writes codes,
+// metadata and the fp16 windows from the canonical arrays (same shapes as export_store_kernel's).
+__global__ void import_store_kernel(Layout L, Store S, unsigned char* __restrict__ cache, int n_q, int n_sink, int n_recent,
+                                    const uint8_t* __restrict__ code, const uint16_t* __restrict__ scale,
+                                    const uint16_t* __restrict__ zero, const uint16_t* __restrict__ sink_in,
+                                    const uint16_t* __restrict__ recent_in, int pass) {
+  const int u = blockIdx.y;
+  const int cap = L.max_tokens;
+  const Rec rec = unit_rec(L, cache, u);
+  const int stride = gridDim.x * blockDim.x, tid0 = blockIdx.x * blockDim.x + threadIdx.x;
+  if (S.kind != kNone && pass == 0) {
+    if (S.code_kind == kRow) {
+      const int rw = row_bytes(S.bits) / 4;
+      for (int i = tid0; i < n_q * rw; i += stride) reinterpret_cast<uint32_t*>(row_code_ptr(rec, S, i / rw))[i % rw] = 0u;
+    } else {
+      const int cw = chunk_bytes(S.bits) / 4, n_ch = (n_q + kChunk - 1) / kChunk;
+      for (int i = tid0; i < n_ch * cw; i += stride) reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, i / cw))[i % cw] = 0u;
+    }
+    return;
+  }
+  if (S.kind != kNone) {
+    for (int i = tid0; i < n_q * kD; i += stride) {
+      const int t = i / kD, c = i % kD;
+      const uint32_t v = code[((size_t)u * cap + t) * kD + c];
+      if (S.code_kind == kRow) row_put(reinterpret_cast<uint32_t*>(row_code_ptr(rec, S, t)), c, S.bits, v, S.perm);
+      else chunk_put(reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, t / kChunk)), t % kChunk, c, S.bits, v, S.perm);
+    }
+    const int n_meta_rows = S.kind == kRow ? n_q : n_q / L.G;
+    const int rows_cap = S.kind == kRow ? cap : cap / L.G + 1;
+    for (int i = tid0; i < n_meta_rows * S.n_groups; i += stride) {
+      const int mr = i / S.n_groups, me = i % S.n_groups;
+      const int ic = S.kind == kRow ? i : mr * kD + block_meta_channel(me);   // canonical position
+      const size_t o = (size_t)u * rows_cap * S.n_groups + ic;
+      const uint32_t m = (uint32_t)scale[o] | ((uint32_t)(zero ? zero[o] : 0) << 16);
+      if (S.kind == kRow) store_meta(row_meta_ptr(rec, S, mr), me, S.meta_bytes, m);
+      else store_meta(block_meta_ptr(rec, S, mr), me, S.meta_bytes, m);
+    }
+  }
+  uint16_t* sink = reinterpret_cast<uint16_t*>(cache + S.sink_off + (size_t)u * S.sink_stride);
+  uint16_t* ring = reinterpret_cast<uint16_t*>(cache + S.ring_off + (size_t)u * S.ring_stride);
+  const int sink_cap = S.kind == kNone ? L.max_tokens : L.w_sink;
+  for (int i = tid0; i < n_sink * kD; i += stride) sink[i] = sink_in[(size_t)u * sink_cap * kD + i];
+  if (S.kind != kNone) {
+    const int t_first = n_sink + n_q;   // absolute token of the oldest recent entry
+    for (int i = tid0; i < n_recent * kD; i += stride) {
+      const int t = t_first + i / kD, c = i % kD;
+      ring[(size_t)((t - L.w_sink) % S.ring_cap) * kD + c] = recent_in[(size_t)u * (L.w_recent + L.G) * kD + i];
+    }
+  }
+}
+
 // ------------------------------------------------------------------ host launchers
 static inline int grid_for(int n, int per_block, int cap) {
   int g = (n + per_block - 1) / per_block;
@@ -619,6 +671,29 @@ int launch_export(const Layout& L, const unsigned char* cache, int N, const Expo
     if (cudaMemcpyAsync(e.norm, cache + L.norm_off, (size_t)L.U * kD * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return -1;
   return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+int launch_import(const Layout& L, unsigned char* cache, int N, const ExportPtrs& e, cudaStream_t st) {
+  const Counts cn = counts_for(L, N);
+  const bool fp16 = L.k.kind == kNone;
+  const Store* S[2] = {&L.k, &L.v};
+  const int nq[2] = {cn.n_qk, cn.n_qv}, nrec[2] = {cn.n_k_recent, cn.n_v_recent};
+  const uint8_t* code[2] = {e.k_code, e.v_code};
+  const uint16_t* scale[2] = {e.k_scale, e.v_scale};
+  const uint16_t* zero[2] = {e.k_zero, e.v_zero};
+  const uint16_t* sink[2] = {e.k_sink, e.v_sink};
+  const uint16_t* recent[2] = {e.k_recent, e.v_recent};
+  int launches = 0;
+  for (int pass = 0; pass < 2; ++pass)      // all packed words are cleared before any code is OR-ed in
+    for (int i = 0; i < 2; ++i) {
+      if (pass == 0 && (S[i]->kind == kNone || nq[i] == 0)) continue;
+      import_store_kernel<<<dim3(64, L.U), 256, 0, st>>>(L, *S[i], cache, nq[i], fp16 ? N : cn.n_sink, nrec[i], code[i],
+                                                        scale[i], zero[i], sink[i], recent[i], pass);
+      ++launches;
+    }
+  if (cudaMemcpyAsync(cache + L.norm_off, e.norm, (size_t)L.U * kD * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return -1;
+  fill_u32_kernel<<<(L.U + 255) / 256, 256, 0, st>>>(reinterpret_cast<uint32_t*>(cache + L.appended_off), (uint32_t)N, L.U);
+  return cudaGetLastError() == cudaSuccess ? launches + 1 : -1;
 }
 
 }  // namespace iq

@@ -580,3 +580,38 @@ def test_config1_full_parity():
     flips = P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, w.group)
     worst = check_decode(w, oc, gc, variants=(0, 1, 3, 4), splits=(0, 1, 4, 13))
     print(f"config1: contested flips {flips}, worst err/tol {worst:.3f}")
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(group=64, k_bits=3, v_bits=3, n_q_heads=8), dict(k_bits=4, v_bits=2, k_mode=O.SYM),
+                                dict(grouping=O.OUTER, k_normalize=0, k_mode=O.ASYM, v_mode=O.ASYM, group=64),
+                                dict(grouping=O.FP16, k_normalize=0)],
+                         ids=["2bit", "3bit_g64", "k4sym_v2", "outer", "fp16"])
+def test_import_restores_an_exported_cache(kw):
+    # checkpoint / resume: export a cache that has been prefilled and stepped, import the arrays into a fresh cache of
+    # the same configuration: identical export, identical decode output (same bits), and both caches continue alike
+    import torch
+    w = synth.tiny(n_tokens=500, **kw)
+    oc, gc, _, _ = run_prefill_both(w)
+    for step in range(w.group + 5):
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        gc.innerq_append_token(dev(k1), dev(v1))
+    saved = gc.innerq_cache_export()
+    g2 = gpu_cache(w)
+    g2.innerq_cache_import(saved)
+    assert g2.n_tokens == gc.n_tokens
+    again = g2.innerq_cache_export()
+    for key, val in saved.items():
+        assert np.array_equal(np.asarray(val), np.asarray(again[key])), key
+    q = dev(synth.query(w, 3))
+    assert torch.equal(gc.innerq_decode_attention(q), g2.innerq_decode_attention(q))
+    check_decode(w, oc, g2, step=3)
+    for step in range(100, 100 + w.group + 2):                 # both continue through another group eviction
+        k1, v1 = synth.new_token(w, step)
+        oc.append(k1, v1)
+        for c in (gc, g2):
+            c.innerq_append_token(dev(k1), dev(v1))
+    a, b = gc.innerq_cache_export(), g2.innerq_cache_export()
+    for key, val in a.items():
+        assert np.array_equal(np.asarray(val), np.asarray(b[key])), key
+    check_decode(w, oc, g2, step=9)
