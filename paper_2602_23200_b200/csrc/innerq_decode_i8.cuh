@@ -1,10 +1,11 @@
-// Fused decode attention over the packed InnerQ cache with 2-bit keys and 2-bit values, on the 8-bit integer
-// tensor-core instruction (mma.sync m16n8k32, u8 x s8 / u8 x u8, s32 accumulate).
+// Fused decode attention over the packed InnerQ cache with 2-bit keys and 2-bit values, or 4-bit and 4-bit, on the
+// 8-bit integer tensor-core instruction (mma.sync m16n8k32, u8 x s8 / u8 x u8, s32 accumulate).
 //
 // Same launch shape, pipeline, tail tiles and merge as the fp16-operand kernel (innerq_decode_mma.cuh, whose helpers
-// this file uses); what differs is the arithmetic core.  The cache keeps its 2-bit codes in byte order
-// (Store::perm = 1, see row_pos_i8 / block_pos_i8), so `word & (0x03030303 << 2p)` is four operand bytes at once:
-// half the unpack instructions and half the MMAs of the fp16 path per cached element.
+// this file uses); what differs is the arithmetic core.  The cache keeps its codes in byte order
+// (Store::perm = 1, see row_pos_i8 / block_pos_i8), so `word & (0x03030303 << 2p)` (2-bit codes; 4-bit:
+// `word & 0x0F0F0F0F`, `word & 0xF0F0F0F0`) is four operand bytes at once: half the unpack instructions and half the
+// MMAs of the fp16 path per cached element.
 //   Keys.   q'' (scaled, normalised query) is split into two signed base-128 digits per channel; columns of the
 //           second operand are (head, digit), or (channel group, digit) when there is one query head per KV head and
 //           G = 32 (SPLIT).  The integer code sums come out exact; scale and zero-point are applied once per
@@ -59,14 +60,16 @@ constexpr float kPScale = 65535.0f;          // p <= 1 as 16 bits: two unsigned 
 // tokens per loop iteration.
 // ABL (timing experiments only, results wrong on purpose): bit 0 leaves out the key side's unpack + MMA work of the
 // streaming loop (scores taken as 0), bit 1 the value side's; all bytes are still streamed.
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
+// BITS: 2 or 4 (keys and values alike).
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u,
                                                const PageIds* ptab = nullptr) {
-  using SL = StageLayout<2, 2, G, KM, VM, CPI>;
+  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
+  static_assert(BITS == 2 || BITS == 4, "byte order exists for 2- and 4-bit codes");
   constexpr int NG = SL::kNG;                   // key groups per token
   constexpr int CH = SL::kCH;                   // chunks per value group
   constexpr int NST = SL::kStages;
-  constexpr int RW = 8;                         // 32-bit words per packed key row
+  constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
   constexpr int RU = CH;                        // chunks per range unit: one value group
   constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
   static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
@@ -366,8 +369,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
       for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g];
     }
-    const float wj = pow2i(-2 * j), wjm = -wj * kMagicSf;           // SPLIT: group j sits at bit position j (weight 4^j)
-    const float neg_half = -2.0f, neg_half_v = -2.0f;               // -2^(b-1)
+    // SPLIT: group j sits at bit position j of a byte (weight 4^j), with 4-bit codes in nibble j % 2 (weight 16^(j % 2))
+    const float wj = BITS == 2 ? pow2i(-2 * j) : pow2i(-4 * (j & 1)), wjm = -wj * kMagicSf;
+    const float neg_half = -(float)(1 << (BITS - 1)), neg_half_v = neg_half;               // -2^(b-1)
     // 128 * hi + lo of one accumulator pair (bit patterns of kMagicSf + sum), times the power of two w: exact
     auto digits = [&](int hi, int lo, float w, float wm) {
       return fmaf(128.f, fmaf(w, __int_as_float(hi), wm), fmaf(w, __int_as_float(lo), wm));
@@ -376,8 +380,6 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
     // are r0 + gid and r0 + gid + 8.  kc / km: packed rows and metadata rows of the chunk (shared or global memory).
     auto k_mtile = [&](const uint32_t* kc, const uint32_t* km, int r0, float& sA_out, float& sB_out) {
       const int rA = r0 + gid, rB = rA + 8;
-      const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + 2 * j);      // bytes 4j.. and 16+4j.. of row rA
-      const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + 2 * j);
       auto kmeta = [&](int row, int g, float& s_, float& z_) {      // decoder parameters of (row, group)
         if constexpr (KM == 4) decode_fast(km[row * NG + g], neg_half, s_, z_);
         else {
@@ -386,6 +388,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         }
       };
       float sA, sB, s_, z_;
+      if constexpr (BITS == 2) {
+      const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + 2 * j);      // bytes 4j.. and 16+4j.. of row rA
+      const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + 2 * j);
       if constexpr (SPLIT) {
         // column pair g carries q'' of group g only, so one accumulator chain leaves group j's sums with lane j
         int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
@@ -444,6 +449,73 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           sA = fmaf(s_, tA[0] + tA[1], z_ * Qg[0]);
           kmeta(rB, 0, s_, z_);
           sB = fmaf(s_, tB[0] + tB[1], z_ * Qg[0]);
+        }
+      }
+      } else {
+        // 4-bit codes: words [2 h2 + h] = bytes 16 h + 4 j .. of row half h2; channel run s = low (s even) or high
+        // (s odd) nibbles of half s / 2
+        const uint4 xa4 = *reinterpret_cast<const uint4*>(kc + rA * RW + 4 * j);
+        const uint4 xb4 = *reinterpret_cast<const uint4*>(kc + rB * RW + 4 * j);
+        const uint32_t xa[4] = {xa4.x, xa4.y, xa4.z, xa4.w}, xb[4] = {xb4.x, xb4.y, xb4.z, xb4.w};
+        if constexpr (SPLIT || G == 32) {
+          int cs[SPLIT ? 1 : 4][4];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            int (&c4)[4] = cs[SPLIT ? 0 : g];
+            if (!SPLIT || g == 0) { c4[0] = c4[1] = c4[2] = c4[3] = kMagicS; }
+            const uint32_t mk = (g & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
+            const int h2 = g >> 1;
+            imma_us(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[g][0], Bq[g][1]);
+          }
+          if constexpr (SPLIT) {
+            kmeta(rA, j, s_, z_);
+            sA = fmaf(s_, digits(cs[0][0], cs[0][1], wj, wjm), z_ * Qg[0]);
+            kmeta(rB, j, s_, z_);
+            sB = fmaf(s_, digits(cs[0][2], cs[0][3], wj, wjm), z_ * Qg[0]);
+            sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+            sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+            sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+            sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+          } else {
+            sA = 0.f; sB = 0.f;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const float w = pow2i(-4 * (g & 1)), wm = -w * kMagicSf;
+              kmeta(rA, g, s_, z_);
+              sA = fmaf(s_, digits(cs[SPLIT ? 0 : g][0], cs[SPLIT ? 0 : g][1], w, wm), fmaf(z_, Qg[SPLIT ? 0 : g], sA));
+              kmeta(rB, g, s_, z_);
+              sB = fmaf(s_, digits(cs[SPLIT ? 0 : g][2], cs[SPLIT ? 0 : g][3], w, wm), fmaf(z_, Qg[SPLIT ? 0 : g], sB));
+            }
+          }
+        } else {
+          // G = 64 / 128: the high nibbles are shifted down, so that the two channel runs of a row half (G = 64: one
+          // group) or all four (G = 128) share an accumulator at weight 1
+          float tA[2], tB[2];
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+            const uint32_t mk = 0x0F0F0F0Fu;
+            imma_us(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[2 * h2][0], Bq[2 * h2][1]);
+            imma_us(c4, (xa[2 * h2] >> 4) & mk, (xb[2 * h2] >> 4) & mk, (xa[2 * h2 + 1] >> 4) & mk, (xb[2 * h2 + 1] >> 4) & mk,
+                    Bq[2 * h2 + 1][0], Bq[2 * h2 + 1][1]);
+            tA[h2] = digits(c4[0], c4[1], 1.0f, -kMagicSf);
+            tB[h2] = digits(c4[2], c4[3], 1.0f, -kMagicSf);
+          }
+          if constexpr (G == 64) {
+            kmeta(rA, 0, s_, z_);
+            sA = fmaf(s_, tA[0], z_ * Qg[0]);
+            kmeta(rB, 0, s_, z_);
+            sB = fmaf(s_, tB[0], z_ * Qg[0]);
+            kmeta(rA, 1, s_, z_);
+            sA = fmaf(s_, tA[1], fmaf(z_, Qg[1], sA));
+            kmeta(rB, 1, s_, z_);
+            sB = fmaf(s_, tB[1], fmaf(z_, Qg[1], sB));
+          } else {
+            kmeta(rA, 0, s_, z_);
+            sA = fmaf(s_, tA[0] + tA[1], z_ * Qg[0]);
+            kmeta(rB, 0, s_, z_);
+            sB = fmaf(s_, tB[0] + tB[1], z_ * Qg[0]);
+          }
         }
       }
       sA_out = sA;
@@ -692,7 +764,21 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         if (SPLIT && (gid >> 1) != slot) { b0 = 0u; b1 = 0u; }      // column pair of this chunk's window slot only
 
         // ---------------- values: 8 m-tiles of 16 channels x one k-step of 32 tokens --------------------
-        if constexpr (!(ABL & 2)) {
+        if constexpr (!(ABL & 2) && BITS == 4) {
+          // 4-bit codes: word set W = m / 2 (four words: the roles a0 .. a3), nibble m % 2
+#pragma unroll
+          for (int W = 0; W < 4; ++W) {
+            const uint4 v = *reinterpret_cast<const uint4*>(vc + W * 128 + lane * 4);
+#pragma unroll
+            for (int pos = 0; pos < 2; ++pos) {
+              const uint32_t mk = pos ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
+              if constexpr (kFreshEveryChunk)
+                imma_uu_init(accg[2 * W + pos], v.x & mk, v.y & mk, v.z & mk, v.w & mk, b0, b1, kMagicU);
+              else
+                imma_uu(accg[2 * W + pos], v.x & mk, v.y & mk, v.z & mk, v.w & mk, b0, b1);
+            }
+          }
+        } else if constexpr (!(ABL & 2)) {
           const uint4 v0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
           const uint4 v1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
           const uint32_t vw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -725,7 +811,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           pg *= kPScale;                                // out_acc is in units of 1 / kPScale
           const uint32_t* vmg = SPLIT ? side + j * (SL::kVMeta / 4) : vm;    // this group's entries (slot j's in SPLIT)
           // code sum of fragment row (m, rh): m-tile m sits at bit position m % 4 of its words (weight 4^(m % 4))
-          auto acc_sum = [&](int m, int rh) { return vdigits(accg[m][2 * rh], accg[m][2 * rh + 1], pow2i(-2 * (m & 3))); };
+          auto acc_sum = [&](int m, int rh) {
+            return vdigits(accg[m][2 * rh], accg[m][2 * rh + 1], BITS == 2 ? pow2i(-2 * (m & 3)) : pow2i(-4 * (m & 1)));
+          };
           if constexpr (!SPLIT && VM == 4) {
             // The four lanes of a quad need the same 16 entries: every lane decodes 4 of the group's 128 once, the
             // warp exchanges (scale, zero-point) pairs through its side area (rows of 16 pairs, padded to 36 words
@@ -869,40 +957,40 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 
 
 // One cache: block x = unit.
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  decode_i8_body<G, KM, VM, SPLIT, CPI, PAGED, ABL>(L, cn, a, blockIdx.x);
+  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, PAGED, ABL>(L, cn, a, blockIdx.x);
 }
 // One paged cache with its page table in the parameter space (read in place: no look-up in device memory).
-template <int G, int KM, int VM, bool SPLIT, int CPI>
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_paged_kernel(const Layout L, const Counts cn, const DecodeArgs a, const __grid_constant__ PageIds P) {
-  decode_i8_body<G, KM, VM, SPLIT, CPI, true>(L, cn, a, blockIdx.x, &P);
+  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, true>(L, cn, a, blockIdx.x, &P);
 }
 // Several caches of one configuration: block x = sequence * U + unit.
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_batched_kernel(const __grid_constant__ Layout L, const __grid_constant__ SeqTable T) {
   const int seq = blockIdx.x / L.U;
-  decode_i8_body<G, KM, VM, SPLIT, CPI, PAGED>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
+  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, PAGED>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
 }
 
 // ---- host side: the launchers of one metadata format (KM, VM) at every group size ---------------------------
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
 int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
-  using SL = StageLayout<2, 2, G, KM, VM, CPI>;
+  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_i8_kernel<G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
   // a paged cache whose page list fits the parameter space: the kernel that takes the table as a parameter
   [[maybe_unused]] PageIds ids;
   bool table_in_params = false;
   if constexpr (PAGED) {
     static std::atomic<unsigned long long> configured_p{0};
     if (a.pages_host && a.n_pages_host <= kParamPages) {
-      if (!opt_in_dynamic_smem(decode_i8_paged_kernel<G, KM, VM, SPLIT, CPI>, kSmem, configured_p)) return -1;
+      if (!opt_in_dynamic_smem(decode_i8_paged_kernel<BITS, G, KM, VM, SPLIT, CPI>, kSmem, configured_p)) return -1;
       for (int i = 0; i < a.n_pages_host; ++i) ids.id[i] = a.pages_host[i];
       table_in_params = true;
     }
@@ -923,19 +1011,19 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
     cudaError_t err;
     if constexpr (PAGED) {
       if (a.ablation) return -2;      // the timing instances exist for contiguous caches only
-      err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
-                            : cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
+      err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<BITS, G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
+                            : cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     } else if (a.ablation == 1 || a.ablation == 2) {
       static std::atomic<unsigned long long> configured_a1{0}, configured_a2{0};
       if (a.ablation == 1) {
-        if (!opt_in_dynamic_smem(decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
-        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 1>, L, cn, a);
+        if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 1>, L, cn, a);
       } else {
-        if (!opt_in_dynamic_smem(decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
-        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
+        if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
       }
     } else {
-      err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
+      err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     }
     if (err != cudaSuccess) return -1;
     ++launches;
@@ -944,13 +1032,13 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
 }
 
 // The same kernel over a table of caches (rows per sequence: see launch_one_batched_p of the fp16-operand kernel).
-template <int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
+template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
 int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
-  using SL = StageLayout<2, 2, G, KM, VM, CPI>;
+  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_i8_batched_kernel<G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_i8_batched_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
   long long chunks[kMaxSeqs], longest = 1;
   for (int i = 0; i < n_seqs; ++i) {
     chunks[i] = T.s[i].cn.n_qv / kChunk;
@@ -986,49 +1074,54 @@ int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_i8_batched_kernel<G, KM, VM, SPLIT, CPI, PAGED>, L, T) != cudaSuccess) return -1;
+    if (cudaLaunchKernelEx(&cfg, decode_i8_batched_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, T) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
-// cpi: chunks of 32 tokens per loop iteration, 0 = automatic: two, unless a warp gets so few chunks that the second
-// half of an iteration would often be empty (G = 32, where a warp's range may be an odd number of chunks, and fewer
-// than four chunks per warp: short contexts split over many CTAs).
-template <int G, int KM, int VM, bool SPLIT>
+// cpi: chunks of 32 tokens per loop iteration, 0 = automatic: two for 2-bit codes (4-bit stages are twice the size:
+// always one), unless a warp gets so few chunks that the second half of an iteration would often be empty (G = 32,
+// where a warp's range may be an odd number of chunks, and fewer than four chunks per warp: short contexts split
+// over many CTAs).
+template <int BITS, int G, int KM, int VM, bool SPLIT>
 int launch_i8_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
   const bool paged = L.page_groups > 0;
   if (cpi == 0 && G == 32 && cn.n_qv / kChunk < 4 * kWarps * (n_splits > 0 ? n_splits : 1)) cpi = 1;
-  if (cpi == 1)
-    return paged ? launch_i8_one_p<G, KM, VM, SPLIT, 1, true>(L, cn, a, n_splits, st)
-                 : launch_i8_one_p<G, KM, VM, SPLIT, 1, false>(L, cn, a, n_splits, st);
-  return paged ? launch_i8_one_p<G, KM, VM, SPLIT, 2, true>(L, cn, a, n_splits, st)
-               : launch_i8_one_p<G, KM, VM, SPLIT, 2, false>(L, cn, a, n_splits, st);
+  if constexpr (BITS == 2) {
+    if (cpi != 1)
+      return paged ? launch_i8_one_p<BITS, G, KM, VM, SPLIT, 2, true>(L, cn, a, n_splits, st)
+                   : launch_i8_one_p<BITS, G, KM, VM, SPLIT, 2, false>(L, cn, a, n_splits, st);
+  }
+  return paged ? launch_i8_one_p<BITS, G, KM, VM, SPLIT, 1, true>(L, cn, a, n_splits, st)
+               : launch_i8_one_p<BITS, G, KM, VM, SPLIT, 1, false>(L, cn, a, n_splits, st);
 }
-template <int G, int KM, int VM, bool SPLIT>
+template <int BITS, int G, int KM, int VM, bool SPLIT>
 int launch_i8_cpi_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
   const bool paged = L.page_groups > 0;
-  if (cpi == 1)
-    return paged ? launch_i8_batched_p<G, KM, VM, SPLIT, 1, true>(L, T, n_seqs, n_splits, st)
-                 : launch_i8_batched_p<G, KM, VM, SPLIT, 1, false>(L, T, n_seqs, n_splits, st);
-  return paged ? launch_i8_batched_p<G, KM, VM, SPLIT, 2, true>(L, T, n_seqs, n_splits, st)
-               : launch_i8_batched_p<G, KM, VM, SPLIT, 2, false>(L, T, n_seqs, n_splits, st);
+  if constexpr (BITS == 2) {
+    if (cpi != 1)
+      return paged ? launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 2, true>(L, T, n_seqs, n_splits, st)
+                   : launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 2, false>(L, T, n_seqs, n_splits, st);
+  }
+  return paged ? launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 1, true>(L, T, n_seqs, n_splits, st)
+               : launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 1, false>(L, T, n_seqs, n_splits, st);
 }
 
-template <int KM, int VM>
+template <int BITS, int KM, int VM>
 int launch_i8_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_i8_cpi<32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 32) return launch_i8_cpi<32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 64) return launch_i8_cpi<64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 128) return launch_i8_cpi<128, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_i8_cpi<BITS, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 32) return launch_i8_cpi<BITS, 32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 64) return launch_i8_cpi<BITS, 64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 128) return launch_i8_cpi<BITS, 128, KM, VM, false>(L, cn, a, n_splits, cpi, st);
   return -2;
 }
-template <int KM, int VM>
+template <int BITS, int KM, int VM>
 int launch_i8_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1) return launch_i8_cpi_batched<32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 32) return launch_i8_cpi_batched<32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 64) return launch_i8_cpi_batched<64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 128) return launch_i8_cpi_batched<128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 32 && L.r == 1) return launch_i8_cpi_batched<BITS, 32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 32) return launch_i8_cpi_batched<BITS, 32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 64) return launch_i8_cpi_batched<BITS, 64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 128) return launch_i8_cpi_batched<BITS, 128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
   return -2;
 }
 
@@ -1036,14 +1129,14 @@ int launch_i8_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_spl
 
 // Defines the externally visible launchers of one metadata format in the translation unit that compiles its kernels
 // (same names as the fp16-operand kernel's: the host dispatch does not change).
-#define IQ_DEFINE_I8_FORMAT(KM, VM)                                                                             \
-  int IQ_MMA_FORMAT_NAME(2, 2, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,   \
-                                       int cpi, cudaStream_t st) {                                              \
-    return launch_i8_format<KM, VM>(L, cn, a, n_splits, cpi, st);                                               \
-  }                                                                                                             \
-  int IQ_MMA_FORMAT_NAME_BATCHED(2, 2, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, \
-                                               cudaStream_t st) {                                               \
-    return launch_i8_format_batched<KM, VM>(L, T, n_seqs, n_splits, cpi, st);                                   \
+#define IQ_DEFINE_I8_FORMAT(BITS, KM, VM)                                                                            \
+  int IQ_MMA_FORMAT_NAME(BITS, BITS, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,   \
+                                             int cpi, cudaStream_t st) {                                              \
+    return launch_i8_format<BITS, KM, VM>(L, cn, a, n_splits, cpi, st);                                               \
+  }                                                                                                                   \
+  int IQ_MMA_FORMAT_NAME_BATCHED(BITS, BITS, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, \
+                                                     cudaStream_t st) {                                               \
+    return launch_i8_format_batched<BITS, KM, VM>(L, T, n_seqs, n_splits, cpi, st);                                   \
   }
 
 }  // namespace iq

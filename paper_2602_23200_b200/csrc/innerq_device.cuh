@@ -14,8 +14,8 @@ __device__ __forceinline__ uint16_t f2h_bits(float f) { return __half_as_ushort(
 // ---- packed-code accessors (generic, slow; the fast kernels extract fragments directly) ----
 __device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, int c, int bits, int perm = 0) {
   if (perm == 1) {
-    BitPos p = row_pos_i8(c);
-    return (row[p.word] >> p.bit) & 3u;
+    BitPos p = row_pos_i8(c, bits);
+    return (row[p.word] >> p.bit) & ((1u << bits) - 1u);
   }
   if (bits == 3) {
     BitPos lo = row_pos_plane(c, 2), hi = row_pos_plane(c, 1);
@@ -27,8 +27,8 @@ __device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, i
 
 __device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chunk, int tau, int c, int bits, int perm = 0) {
   if (perm == 1) {
-    BitPos p = block_pos_i8(tau, c);
-    return (chunk[p.word] >> p.bit) & 3u;
+    BitPos p = block_pos_i8(tau, c, bits);
+    return (chunk[p.word] >> p.bit) & ((1u << bits) - 1u);
   }
   if (bits == 3) {
     BitPos lo = block_pos_plane(tau, c, 2), hi = block_pos_plane(tau, c, 1);
@@ -41,7 +41,7 @@ __device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chun
 // OR a code into a zero-initialised packed row / chunk held in shared memory.
 __device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t code, int perm = 0) {
   if (perm == 1) {
-    BitPos p = row_pos_i8(c);
+    BitPos p = row_pos_i8(c, bits);
     atomicOr(&row[p.word], code << p.bit);
   } else if (bits == 3) {
     BitPos lo = row_pos_plane(c, 2), hi = row_pos_plane(c, 1);
@@ -54,7 +54,7 @@ __device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t
 }
 __device__ __forceinline__ void chunk_put(uint32_t* chunk, int tau, int c, int bits, uint32_t code, int perm = 0) {
   if (perm == 1) {
-    BitPos p = block_pos_i8(tau, c);
+    BitPos p = block_pos_i8(tau, c, bits);
     atomicOr(&chunk[p.word], code << p.bit);
   } else if (bits == 3) {
     BitPos lo = block_pos_plane(tau, c, 2), hi = block_pos_plane(tau, c, 1);

@@ -47,8 +47,8 @@ struct Store {
                        // under outer grouping keys keep rows and values keep chunks, only the metadata changes sides.
   int bits, mode;
   int perm;            // order of the codes inside a packed row / chunk: 0 = pairs for the fp16 tensor-core fragments
-                       // (word & mask is a half2), 1 = bytes for the 8-bit integer fragments (2-bit codes of an
-                       // inner-grouped cache whose keys and values are both 2-bit; see row_pos_i8 / block_pos_i8)
+                       // (word & mask is a half2), 1 = bytes for the 8-bit integer fragments (inner-grouped caches
+                       // whose keys and values are both 2-bit or both 4-bit; see row_pos_i8 / block_pos_i8)
   int ring_cap;        // slots of the recent ring: w_recent + 1 (ROW) or w_recent + G (BLOCK)
   int cap_q;           // capacity in quantised tokens (multiple of kTile)
   int n_groups;        // metadata entries per row (ROW: D/G) or per group (BLOCK: D)
@@ -223,11 +223,19 @@ IQ_HD BitPos block_pos_plane(int tau, int c, int plane_bits) {
 // position p is one k-step of 32 channels = the p-th run of 32 channels (a whole group at G = 32).  The fragment of
 // lane (gid, j) is bytes 4j..4j+3 and 16+4j..16+4j+3 of rows gid and gid + 8: the two words are stored next to each
 // other (physical word 2j + h holds bytes 16h + 4j ..), one 64-bit load per row.
-IQ_HD BitPos row_pos_i8(int c) {
+// 4-bit codes: a byte holds two codes (masks 0x0F0F0F0F / 0xF0F0F0F0, the high one times 16); the 64-byte row is two
+// halves of 32 bytes, half h2 holding channel runs 2 h2 (low nibbles) and 2 h2 + 1 (high nibbles); a lane's four words
+// per row (bytes 4j.. and 16+4j.. of both halves) are adjacent: one 128-bit load.
+IQ_HD BitPos row_pos_i8(int c, int bits = 2) {
   const int p = c >> 5, k = c & 31, lw = k >> 2;
   BitPos r;
-  r.word = 2 * (lw & 3) + (lw >> 2);
-  r.bit = 8 * (k & 3) + 2 * p;
+  if (bits == 4) {
+    r.word = 4 * (lw & 3) + 2 * (p >> 1) + (lw >> 2);
+    r.bit = 8 * (k & 3) + 4 * (p & 1);
+  } else {
+    r.word = 2 * (lw & 3) + (lw >> 2);
+    r.bit = 8 * (k & 3) + 2 * p;
+  }
   return r;
 }
 // BLOCK store: one chunk = one k-step of 32 tokens for each of 8 m-tiles of 16 channels.  Token tau sits at
@@ -235,13 +243,15 @@ IQ_HD BitPos row_pos_i8(int c) {
 // Channel c = 64 W + 8 gid + 2 p + rh is fragment row gid (rh = 0) or gid + 8 (rh = 1) of m-tile 4 W + p, the same
 // ownership as with perm = 0; the four m-tiles 4 W .. 4 W + 3 share their words, one per bit position.
 // Lane 4 gid + j holds words [W][2 * (k / 16) + rh] with bytes k % 4, for k / 4 % 4 == j.
-IQ_HD BitPos block_pos_i8(int tau, int c) {
+// 4-bit codes: the two m-tiles 2 W, 2 W + 1 share their words (low / high nibble), W = 0 .. 3: 16 words per lane.
+IQ_HD BitPos block_pos_i8(int tau, int c, int bits = 2) {
   const int k = 4 * (tau & 7) + (tau >> 3);
-  const int W = c >> 6, p = (c >> 1) & 3, gid = (c >> 3) & 7, rh = c & 1;
+  const int m = 4 * (c >> 6) + ((c >> 1) & 3), gid = (c >> 3) & 7, rh = c & 1;
   const int j = (k & 15) >> 2, half = k >> 4;
+  const int W = bits == 4 ? m >> 1 : m >> 2, p = bits == 4 ? m & 1 : m & 3;
   BitPos r;
   r.word = W * 128 + (4 * gid + j) * 4 + 2 * half + rh;
-  r.bit = 8 * (k & 3) + 2 * p;
+  r.bit = 8 * (k & 3) + bits * p;
   return r;
 }
 

@@ -327,8 +327,9 @@ __device__ __forceinline__ int chunk_word_quarter(int i, int bits, int perm) {
     const int r = i - chunk_hi_plane_word();
     return 2 * ((r & 3) >> 1) + ((r >> 2) >> 4);          // word = lane * 4 + (m >> 1), m >> 1 = 2 W + ..; gid = lane / 4
   }
-  (void)perm;
-  const int r = i & 255;                                   // 4-bit codes: two k-step halves of 256 words
+  if (perm == 1 && bits == 4)                              // byte order, 16 words per lane: word set W = i / 128 = m / 2
+    return 2 * (i >> 8) + (((i & 127) >> 2) >> 4);
+  const int r = i & 255;                                   // 4-bit codes in pair order: two k-step halves of 256 words
   return 2 * (r >> 7) + (((r & 127) >> 2) >> 4);           // W = r / 128, gid = ((r % 128) / 4) / 4 -> 2 W + gid / 4
 }
 __device__ void quantize_block_quarter(const TokSrc& src, const __half* __restrict__ x_new, int t_new, int t_first,

@@ -148,9 +148,10 @@ __device__ __forceinline__ void pack_block_segment(const ChosenCoder& cc, const 
   for (int i = 0; i < NW; ++i) lw[i] -= cw[i];
 }
 
-// Byte-order layout (Store::perm = 1, 2-bit codes).  ROW segment = 32 consecutive channels = one bit position of all
-// 32 bytes of the row: the codes go to position 0 of the 8 row words here, the caller shifts them to its position.
-template <bool CLAMP>
+// Byte-order layout (Store::perm = 1, 2- or 4-bit codes).  ROW segment = 32 consecutive channels = one bit position of
+// 32 bytes of the row: the codes go to position 0 of 8 words here (index 2 * j + h, see row_pos_i8), the caller
+// places them in the row and shifts them to its position.
+template <int BITS, bool CLAMP>
 __device__ __forceinline__ void pack_row_segment_i8(const ChosenCoder& cc, const float (&x)[kSeg], uint32_t (&w8)[8]) {
   uint32_t cw[8];
 #pragma unroll
@@ -158,16 +159,17 @@ __device__ __forceinline__ void pack_row_segment_i8(const ChosenCoder& cc, const
 #pragma unroll
   for (int e = 0; e < kSeg; ++e) {
     const uint32_t code = cc.template code_bits<CLAMP>(x[e]);
-    const BitPos p = row_pos_i8(e);                     // constants: positions of channels 0..31 (bit position 0)
-    w8[p.word] += code << p.bit;
-    cw[p.word] += kMagicBits << p.bit;
+    const BitPos p = row_pos_i8(e, BITS);               // constants: positions of channels 0..31 (bit position 0)
+    const int li = BITS == 4 ? 2 * (p.word >> 2) + (p.word & 1) : p.word;
+    w8[li] += code << p.bit;
+    cw[li] += kMagicBits << p.bit;
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) w8[i] -= cw[i];
 }
 // BLOCK segment = 32 tokens of one channel: bytes of the 8 words [j][half] of its fragment row (see block_pos_i8), at
 // bit position 0 here.  Word index: 2 * j + half.
-template <bool CLAMP>
+template <int BITS, bool CLAMP>
 __device__ __forceinline__ void pack_block_segment_i8(const ChosenCoder& cc, const float (&x)[kSeg], uint32_t (&w8)[8]) {
   uint32_t cw[8];
 #pragma unroll
@@ -175,7 +177,7 @@ __device__ __forceinline__ void pack_block_segment_i8(const ChosenCoder& cc, con
 #pragma unroll
   for (int t = 0; t < kSeg; ++t) {
     const uint32_t code = cc.template code_bits<CLAMP>(x[t]);
-    const BitPos p = block_pos_i8(t, 0);                // constants: channel 0 (W = 0, gid = 0, position 0, rh = 0)
+    const BitPos p = block_pos_i8(t, 0, BITS);          // constants: channel 0 (W = 0, gid = 0, position 0, rh = 0)
     const int li = 2 * ((p.word >> 2) & 3) + ((p.word >> 1) & 1);      // 2 * j + half
     w8[li] += code << p.bit;
     cw[li] += kMagicBits << p.bit;
@@ -272,13 +274,16 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
     const ChosenCoder cc(sc, asym);
     uint32_t* row = stage + tk * RW;
     if constexpr (I8) {
-      static_assert(!I8 || BITS == 2, "byte order is defined for 2-bit codes");
+      static_assert(!I8 || BITS == 2 || BITS == 4, "byte order is defined for 2- and 4-bit codes");
       uint32_t w8[8];
-      if (no_clip) pack_row_segment_i8<false>(cc, x, w8);
-      else pack_row_segment_i8<true>(cc, x, w8);
+      if (no_clip) pack_row_segment_i8<BITS, false>(cc, x, w8);
+      else pack_row_segment_i8<BITS, true>(cc, x, w8);
       __syncwarp();                                        // the stage is zero and no longer being read
 #pragma unroll
-      for (int jj = 0; jj < 8; ++jj) atomicOr(&row[jj], w8[jj] << (2 * seg));
+      for (int jj = 0; jj < 8; ++jj) {
+        if constexpr (BITS == 2) atomicOr(&row[jj], w8[jj] << (2 * seg));
+        else atomicOr(&row[4 * (jj >> 1) + 2 * (seg >> 1) + (jj & 1)], w8[jj] << (4 * (seg & 1)));
+      }
     } else {
       uint32_t lw[4], hw[4];
       if (no_clip) pack_row_segment<BITS, false>(cc, x, lw, hw);
@@ -380,10 +385,10 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
       }
       const ChosenCoder cc(sc, asym);
       if constexpr (I8) {
-        if (no_clip) pack_block_segment_i8<false>(cc, x, w16[rh]);
-        else pack_block_segment_i8<true>(cc, x, w16[rh]);
+        if (no_clip) pack_block_segment_i8<BITS, false>(cc, x, w16[rh]);
+        else pack_block_segment_i8<BITS, true>(cc, x, w16[rh]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) w16[rh][i] <<= 2 * (cp & 3);      // this pair's bit position: (c >> 1) & 3
+        for (int i = 0; i < 8; ++i) w16[rh][i] <<= BITS * (BITS == 2 ? cp & 3 : cp & 1);      // this pair's bit position
       } else {
         uint32_t lw[NW], hw[4];
         if (no_clip) pack_block_segment<BITS, false>(cc, x, lw, hw);
@@ -398,7 +403,24 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
       meta2[rh] = group_meta(p, asym);
     }
     uint32_t* chunk = reinterpret_cast<uint32_t*>(block_code_ptr(rec, S, j * CH + k));
-    if constexpr (I8) {
+    if constexpr (I8 && BITS == 4) {
+      // The two channel pairs cp = 2q, 2q + 1 (adjacent lanes) fill the two nibbles of the same 16 words: after one
+      // exchange lane `pos` holds the complete words of j = 2 pos, 2 pos + 1 (16 contiguous bytes each).
+      const int pos = cp & 1, W = m >> 1;
+#pragma unroll
+      for (int jj = 0; jj < 2; ++jj) {
+        uint32_t f4[4];
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh)
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint32_t keep = pos ? w16[rh][2 * (2 + jj) + half] : w16[rh][2 * jj + half];
+            const uint32_t give = pos ? w16[rh][2 * jj + half] : w16[rh][2 * (2 + jj) + half];
+            f4[2 * half + rh] = keep | __shfl_xor_sync(0xffffffffu, give, 1);
+          }
+        *reinterpret_cast<uint4*>(chunk + W * 128 + (4 * gid + 2 * pos + jj) * 4) = make_uint4(f4[0], f4[1], f4[2], f4[3]);
+      }
+    } else if constexpr (I8) {
       // The four channel pairs cp = 4q .. 4q+3 (adjacent lanes) fill the four bit positions of the same 16 words.
       // Reduce-scatter by OR: after two exchange steps lane `pos` holds the complete words of j = pos (two halves,
       // two row halves), which are 16 contiguous bytes of the chunk.
@@ -455,10 +477,10 @@ static int launch_store_bits(const Layout& L, const Store& S, const __half* X, i
     const int n_batches = (n_q + 7) / 8;
     const int per_unit = grid_cap((n_batches + 4 * 8 - 1) / (4 * 8), grid_cap(148 * 16 / L.U, 1 << 16));
     dim3 grid(per_unit, L.U);
-    if constexpr (BITS == 2) {
+    if constexpr (BITS == 2 || BITS == 4) {
       if (S.perm == 1) {
-        if (inv_norm) quantize_rows_prefill_kernel<2, true, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
-        else quantize_rows_prefill_kernel<2, false, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
+        if (inv_norm) quantize_rows_prefill_kernel<BITS, true, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
+        else quantize_rows_prefill_kernel<BITS, false, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
         return cudaGetLastError() == cudaSuccess ? 1 : -1;
       }
     }
@@ -468,9 +490,9 @@ static int launch_store_bits(const Layout& L, const Store& S, const __half* X, i
     const int CH = L.G / kChunk;
     const int smem = CH * 128 * 16;                   // reduction words of groups spanning several chunks
     auto kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true> : quantize_blocks_prefill_kernel<BITS, false>;
-    if constexpr (BITS == 2) {
+    if constexpr (BITS == 2 || BITS == 4) {
       if (S.perm == 1)
-        kern = inv_norm ? quantize_blocks_prefill_kernel<2, true, true> : quantize_blocks_prefill_kernel<2, false, true>;
+        kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true, true> : quantize_blocks_prefill_kernel<BITS, false, true>;
     }
     const int n_groups = n_q / L.G;
     dim3 grid(grid_cap(n_groups, grid_cap(148 * 16 / L.U, 1 << 16)), L.U);
