@@ -30,17 +30,25 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs = []
-    procs = []
+    pending = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
         objs.append(obj)
-        cmd = [nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]
-        procs.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
-    for cmd, p in procs:
+        pending.append([nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj])
+    # one compiler process per core at a time (there are several dozen translation units: one per packed format)
+    jobs = max(1, min(len(pending), os.cpu_count() or 4))
+    running = []
+    while pending or running:
+        while pending and len(running) < jobs:
+            cmd = pending.pop(0)
+            running.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+        cmd, p = running.pop(0)
         out, _ = p.communicate()
         if verbose or p.returncode:
             sys.stderr.write(out)
         if p.returncode:
+            for _, q in running:
+                q.kill()
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
     cmd = [nvcc, *ARCH, "-shared", "-o", LIB, *objs, "-lcudart"]
     subprocess.run(cmd, check=True)
