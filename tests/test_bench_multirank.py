@@ -72,3 +72,23 @@ def test_algorithmic_bytes_follow_the_library_payload():
         c = bench.stored_counters(w.name)
         assert c is not None and c["alu_pipe"] < c["warp_instructions"], name
         assert bench.stored_traffic(w.name) == c["dram_read_bytes"] + c["dram_write_bytes"]
+
+
+def test_sweep_workload_names_and_prefill_bytes():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_23200_b200 import synth
+    w = bench.workload_by_name("c5_b4_g128_asym")
+    assert (w.k_bits, w.v_bits, w.group, w.k_mode, w.v_mode, w.sym_variant) == (4, 4, 128, synth.ASYM, synth.ASYM, 0)
+    assert (w.batch, w.n_kv_heads, w.n_tokens) == (16, 8, 8192)
+    w = bench.workload_by_name("c5_b2_g64_literal")
+    assert (w.k_mode, w.sym_variant) == (synth.HYBRID, 1)
+    w = bench.workload_by_name("c5_b2_g32_hybrid+outer")
+    assert w.grouping == synth.OUTER and w.k_normalize == 0 and w.group == 32
+    with pytest.raises(SystemExit):
+        bench.workload_by_name("c5_b2_g64_nonsense")
+    # a prefill quantisation reads K and V once (fp16) and writes what a decode then reads
+    w = synth.tiny(n_tokens=400)
+    assert bench.prefill_algorithmic_bytes(w) == w.n_units * 400 * 128 * 2 * 2 + bench.decode_algorithmic_bytes(w, 400)[0]
+    st = bench.stats([3.0, 1.0, 2.0, 10.0])
+    assert (st["median"], st["min"], st["mean"], st["n"]) == (2.5, 1.0, 4.0, 4)
