@@ -223,14 +223,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fp16_kernel(const Layout L
   }
 
   // ---- cross-CTA merge by the last CTA of the unit to arrive
-  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's fence below
+  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's ticket below
   if (tid == 0) {
-    __threadfence();               // cumulative: publishes the whole CTA's partial before the ticket is taken
-    s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+    // release: publishes the whole CTA's partial (ordered before this thread by the barrier) with the ticket;
+    // acquire: the CTA that draws the last ticket sees every other CTA's partial
+    unsigned int t;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;"
+                 : "=r"(t) : "l"(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u) : "memory");
+    s_ticket = t;
   }
   __syncthreads();
   if (s_ticket != gridDim.y - 1) return;
-  __threadfence();
   const int n_parts = gridDim.y;
   for (int i = tid; i < nh * n_parts; i += kThreads) {
     const int h = i / n_parts, s = i % n_parts;

@@ -1242,14 +1242,17 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
 
   // ---------------- cross-CTA merge: the last CTA of the unit to arrive combines all parts -----------
   __shared__ unsigned int s_ticket;
-  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's fence below
+  __syncthreads();                 // all partial writes of this CTA happen-before thread 0's ticket below
   if (tid == 0) {
-    __threadfence();               // cumulative: publishes the whole CTA's partial before the ticket is taken
-    s_ticket = atomicAdd(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u, 1u);
+    // release: publishes the whole CTA's partial (ordered before this thread by the barrier) with the ticket;
+    // acquire: the CTA that draws the last ticket sees every other CTA's partial
+    unsigned int t;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;"
+                 : "=r"(t) : "l"(reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off) + u) : "memory");
+    s_ticket = t;
   }
   __syncthreads();
   if (s_ticket != a.grid_y - 1) return;
-  __threadfence();
   merge_parts(a.partials, reinterpret_cast<float*>(smem), a.out, nh, n_parts, prow0,
               make_int4(q_row(0), q_row(1), q_row(2), q_row(3)), L.max_splits);
   if (tid == 0) reinterpret_cast<unsigned int*>(a.ws + L.ws_ticket_off)[u] = 0u;   // ready for the next launch
