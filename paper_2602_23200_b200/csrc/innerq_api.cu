@@ -159,9 +159,8 @@ void make_layout(const innerq_config_t& c, Layout& L, int page_tokens = 0) {
   } else if (c.grouping == INNERQ_GROUPING_INNER) {
     place_store(L.k, kRow, c.k_bits, c.k_mode, c, L.U, off);
     place_store(L.v, kBlock, c.v_bits, c.v_mode, c, L.U, off);
-    // 2-bit keys with 2-bit values, 4-bit with 4-bit: codes in byte order, for the decode kernel built on the 8-bit
-    // integer MMA
-    if ((c.k_bits == 2 && c.v_bits == 2) || (c.k_bits == 4 && c.v_bits == 4)) L.k.perm = L.v.perm = 1;
+    // codes in byte order, for the decode kernel built on the 8-bit integer MMA
+    L.k.perm = L.v.perm = 1;
     place_records(L.k, L.v, L.G, L.U, off, page_tokens / L.G);
   } else {   // outer grouping: asymmetric, K per channel along tokens, V per token along channels
     place_store(L.k, kBlock, c.k_bits, INNERQ_MODE_ASYM, c, L.U, off);

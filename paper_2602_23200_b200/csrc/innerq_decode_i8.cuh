@@ -1,11 +1,12 @@
-// Fused decode attention over the packed InnerQ cache with 2-bit keys and 2-bit values, or 4-bit and 4-bit, on the
-// 8-bit integer tensor-core instruction (mma.sync m16n8k32, u8 x s8 / u8 x u8, s32 accumulate).
+// Fused decode attention over the inner-grouped packed InnerQ cache (2-, 3- or 4-bit keys, 2-, 3- or 4-bit values) on
+// the 8-bit integer tensor-core instruction (mma.sync m16n8k32, u8 x s8 / u8 x u8, s32 accumulate).
 //
-// Same launch shape, pipeline, tail tiles and merge as the fp16-operand kernel (innerq_decode_mma.cuh, whose helpers
-// this file uses); what differs is the arithmetic core.  The cache keeps its codes in byte order
-// (Store::perm = 1, see row_pos_i8 / block_pos_i8), so `word & (0x03030303 << 2p)` (2-bit codes; 4-bit:
-// `word & 0x0F0F0F0F`, `word & 0xF0F0F0F0`) is four operand bytes at once: half the unpack instructions and half the
-// MMAs of the fp16 path per cached element.
+// Same launch shape, pipeline, tail tiles and merge as the fp16-operand kernel of the outer-grouped comparison cache
+// (innerq_decode_mma.cuh, whose helpers this file uses); what differs is the arithmetic core.  The cache keeps its
+// codes in byte order (Store::perm = 1, see row_pos_i8 / block_pos_i8), so `word & (0x03030303 << 2p)` (2-bit codes;
+// 4-bit: `word & 0x0F0F0F0F`, `word & 0xF0F0F0F0`) is four operand bytes at once: half the unpack instructions and
+// half the MMAs of the fp16 path per cached element.  3-bit codes are a 2-bit and a 1-bit plane that one bit-select
+// per pair of bit positions joins into 3-bit fields (see row_pos_i8_3): 1.5 logic instructions per operand word.
 //   Keys.   q'' (scaled, normalised query) is split into two signed base-128 digits per channel; columns of the
 //           second operand are (head, digit), or (channel group, digit) when there is one query head per KV head and
 //           G = 32 (SPLIT).  The integer code sums come out exact; scale and zero-point are applied once per
@@ -60,16 +61,16 @@ constexpr float kPScale = 65535.0f;          // p <= 1 as 16 bits: two unsigned 
 // tokens per loop iteration.
 // ABL (timing experiments only, results wrong on purpose): bit 0 leaves out the key side's unpack + MMA work of the
 // streaming loop (scores taken as 0), bit 1 the value side's; all bytes are still streamed.
-// BITS: 2 or 4 (keys and values alike).
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
+// KB / VB: bits per key / value code (2, 3 or 4).
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn, const DecodeArgs& a, const int u,
                                                const PageIds* ptab = nullptr) {
-  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
-  static_assert(BITS == 2 || BITS == 4, "byte order exists for 2- and 4-bit codes");
+  using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
+  static_assert(KB >= 2 && KB <= 4 && VB >= 2 && VB <= 4, "2-, 3- and 4-bit codes");
   constexpr int NG = SL::kNG;                   // key groups per token
   constexpr int CH = SL::kCH;                   // chunks per value group
   constexpr int NST = SL::kStages;
-  constexpr int RW = 4 * BITS;                  // 32-bit words per packed key row
+  constexpr int RW = 4 * KB;                    // 32-bit words per packed key row
   constexpr int RU = CH;                        // chunks per range unit: one value group
   constexpr int WIN = 4;                        // SPLIT: value groups per window (one per lane of a quad)
   static_assert(!SPLIT || (G == 32), "SPLIT is built for G = 32");
@@ -369,9 +370,11 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
       for (int g = 0; g < NG; ++g) Qg[g] = qg_s[j * 4 + g];
     }
-    // SPLIT: group j sits at bit position j of a byte (weight 4^j), with 4-bit codes in nibble j % 2 (weight 16^(j % 2))
-    const float wj = BITS == 2 ? pow2i(-2 * j) : pow2i(-4 * (j & 1)), wjm = -wj * kMagicSf;
-    const float neg_half = -(float)(1 << (BITS - 1)), neg_half_v = neg_half;               // -2^(b-1)
+    // SPLIT: group j sits at bit position j of a byte (weight 4^j), with 4-bit codes in nibble j % 2 (weight
+    // 16^(j % 2)), with 3-bit codes in the field of position j (weight 1, 2, 16, 32)
+    const float wj = KB == 2 ? pow2i(-2 * j) : KB == 4 ? pow2i(-4 * (j & 1)) : pow2i(-(4 * (j >> 1) + (j & 1)));
+    const float wjm = -wj * kMagicSf;
+    const float neg_half = -(float)(1 << (KB - 1)), neg_half_v = -(float)(1 << (VB - 1));               // -2^(b-1)
     // 128 * hi + lo of one accumulator pair (bit patterns of kMagicSf + sum), times the power of two w: exact
     auto digits = [&](int hi, int lo, float w, float wm) {
       return fmaf(128.f, fmaf(w, __int_as_float(hi), wm), fmaf(w, __int_as_float(lo), wm));
@@ -388,7 +391,58 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         }
       };
       float sA, sB, s_, z_;
-      if constexpr (BITS == 2) {
+      if constexpr (KB == 3) {
+        // 3-bit codes: one bit-select of a 2-bit plane word and the 1-bit plane word (as it is for the row's first
+        // half, shifted by one for the second) per parity of the bit position gives the 3-bit fields of two positions
+        const uint2 la = *reinterpret_cast<const uint2*>(kc + rA * RW + 2 * j);
+        const uint2 lb = *reinterpret_cast<const uint2*>(kc + rB * RW + 2 * j);
+        const uint32_t ha = kc[rA * RW + 8 + j], hb = kc[rB * RW + 8 + j];
+        const uint32_t lo[4] = {la.x, lb.x, la.y, lb.y};                        // operand registers a0 .. a3
+        const uint32_t ze[4] = {ha, hb, ha >> 1, hb >> 1}, zo[4] = {ha, hb, ha << 1, hb << 1};
+        uint32_t we[4], wo[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          we[r] = (lo[r] & 0x33333333u) | (ze[r] & 0xCCCCCCCCu);                // positions 0, 2: bits 0-2, 4-6
+          wo[r] = (lo[r] & 0xCCCCCCCCu) | (zo[r] & 0x33333333u);                // positions 1, 3: bits 1-3, 5-7
+        }
+        auto areg = [&](int p, int r) {
+          return (p & 1) ? (wo[r] & (0x0E0E0E0Eu << (4 * (p >> 1)))) : (we[r] & (0x07070707u << (4 * (p >> 1))));
+        };
+        if constexpr (SPLIT) {
+          int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+#pragma unroll
+          for (int g = 0; g < 4; ++g) imma_us(c4, areg(g, 0), areg(g, 1), areg(g, 2), areg(g, 3), Bq[g][0], Bq[g][1]);
+          kmeta(rA, j, s_, z_);
+          sA = fmaf(s_, digits(c4[0], c4[1], wj, wjm), z_ * Qg[0]);
+          kmeta(rB, j, s_, z_);
+          sB = fmaf(s_, digits(c4[2], c4[3], wj, wjm), z_ * Qg[0]);
+          sA += __shfl_xor_sync(0xffffffffu, sA, 1);
+          sB += __shfl_xor_sync(0xffffffffu, sB, 1);
+          sA += __shfl_xor_sync(0xffffffffu, sA, 2);
+          sB += __shfl_xor_sync(0xffffffffu, sB, 2);
+        } else {
+          // the four positions carry different weights: one accumulator each, joined per group in fp32
+          float tA[NG], tB[NG];
+#pragma unroll
+          for (int g = 0; g < NG; ++g) tA[g] = tB[g] = 0.f;
+#pragma unroll
+          for (int p = 0; p < 4; ++p) {
+            int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+            imma_us(c4, areg(p, 0), areg(p, 1), areg(p, 2), areg(p, 3), Bq[p][0], Bq[p][1]);
+            const float w = pow2i(-(4 * (p >> 1) + (p & 1))), wm = -w * kMagicSf;
+            tA[(32 * p) / G] += digits(c4[0], c4[1], w, wm);
+            tB[(32 * p) / G] += digits(c4[2], c4[3], w, wm);
+          }
+          sA = 0.f; sB = 0.f;
+#pragma unroll
+          for (int g = 0; g < NG; ++g) {
+            kmeta(rA, g, s_, z_);
+            sA = fmaf(s_, tA[g], fmaf(z_, Qg[g], sA));
+            kmeta(rB, g, s_, z_);
+            sB = fmaf(s_, tB[g], fmaf(z_, Qg[g], sB));
+          }
+        }
+      } else if constexpr (KB == 2) {
       const uint2 xa = *reinterpret_cast<const uint2*>(kc + rA * RW + 2 * j);      // bytes 4j.. and 16+4j.. of row rA
       const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + 2 * j);
       if constexpr (SPLIT) {
@@ -764,7 +818,34 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         if (SPLIT && (gid >> 1) != slot) { b0 = 0u; b1 = 0u; }      // column pair of this chunk's window slot only
 
         // ---------------- values: 8 m-tiles of 16 channels x one k-step of 32 tokens --------------------
-        if constexpr (!(ABL & 2) && BITS == 4) {
+        if constexpr (!(ABL & 2) && VB == 3) {
+          // 3-bit codes: word sets W = 0, 1 of the 2-bit plane (as with 2-bit codes) and one set of the 1-bit plane,
+          // as it is for W = 0 and shifted by one for W = 1
+          const uint4 l0 = *reinterpret_cast<const uint4*>(vc + lane * 4);
+          const uint4 l1 = *reinterpret_cast<const uint4*>(vc + 128 + lane * 4);
+          const uint4 h4 = *reinterpret_cast<const uint4*>(vc + 256 + lane * 4);
+          const uint32_t lw[2][4] = {{l0.x, l0.y, l0.z, l0.w}, {l1.x, l1.y, l1.z, l1.w}};
+          const uint32_t hw[4] = {h4.x, h4.y, h4.z, h4.w};
+#pragma unroll
+          for (int W = 0; W < 2; ++W) {
+            uint32_t we[4], wo[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              const uint32_t ze = W ? hw[r] >> 1 : hw[r], zo = W ? hw[r] << 1 : hw[r];
+              we[r] = (lw[W][r] & 0x33333333u) | (ze & 0xCCCCCCCCu);
+              wo[r] = (lw[W][r] & 0xCCCCCCCCu) | (zo & 0x33333333u);
+            }
+#pragma unroll
+            for (int pos = 0; pos < 4; ++pos) {
+              const uint32_t mk = (pos & 1) ? (0x0E0E0E0Eu << (4 * (pos >> 1))) : (0x07070707u << (4 * (pos >> 1)));
+              const uint32_t* src = (pos & 1) ? wo : we;
+              if constexpr (kFreshEveryChunk)
+                imma_uu_init(accg[4 * W + pos], src[0] & mk, src[1] & mk, src[2] & mk, src[3] & mk, b0, b1, kMagicU);
+              else
+                imma_uu(accg[4 * W + pos], src[0] & mk, src[1] & mk, src[2] & mk, src[3] & mk, b0, b1);
+            }
+          }
+        } else if constexpr (!(ABL & 2) && VB == 4) {
           // 4-bit codes: word set W = m / 2 (four words: the roles a0 .. a3), nibble m % 2
 #pragma unroll
           for (int W = 0; W < 4; ++W) {
@@ -810,9 +891,11 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           pg += __shfl_xor_sync(0xffffffffu, pg, 16);
           pg *= kPScale;                                // out_acc is in units of 1 / kPScale
           const uint32_t* vmg = SPLIT ? side + j * (SL::kVMeta / 4) : vm;    // this group's entries (slot j's in SPLIT)
-          // code sum of fragment row (m, rh): m-tile m sits at bit position m % 4 of its words (weight 4^(m % 4))
+          // code sum of fragment row (m, rh): m-tile m sits at bit position m % 4 of its words (weight 4^(m % 4);
+          // 3-bit fields: 1, 2, 16, 32), with 4-bit codes in nibble m % 2
           auto acc_sum = [&](int m, int rh) {
-            return vdigits(accg[m][2 * rh], accg[m][2 * rh + 1], BITS == 2 ? pow2i(-2 * (m & 3)) : pow2i(-4 * (m & 1)));
+            return vdigits(accg[m][2 * rh], accg[m][2 * rh + 1],
+                           VB == 2 ? pow2i(-2 * (m & 3)) : VB == 4 ? pow2i(-4 * (m & 1)) : pow2i(-(2 * (m & 2) + (m & 1))));
           };
           if constexpr (!SPLIT && VM == 4) {
             // The four lanes of a quad need the same 16 entries: every lane decodes 4 of the group's 128 once, the
@@ -960,40 +1043,40 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 
 
 // One cache: block x = unit.
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false, int ABL = 0>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_kernel(const Layout L, const Counts cn, const DecodeArgs a) {
-  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, PAGED, ABL>(L, cn, a, blockIdx.x);
+  decode_i8_body<KB, VB, G, KM, VM, SPLIT, CPI, PAGED, ABL>(L, cn, a, blockIdx.x);
 }
 // One paged cache with its page table in the parameter space (read in place: no look-up in device memory).
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_paged_kernel(const Layout L, const Counts cn, const DecodeArgs a, const __grid_constant__ PageIds P) {
-  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, true>(L, cn, a, blockIdx.x, &P);
+  decode_i8_body<KB, VB, G, KM, VM, SPLIT, CPI, true>(L, cn, a, blockIdx.x, &P);
 }
 // Several caches of one configuration: block x = sequence * U + unit.
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED = false>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_i8_batched_kernel(const __grid_constant__ Layout L, const __grid_constant__ SeqTable T) {
   const int seq = blockIdx.x / L.U;
-  decode_i8_body<BITS, G, KM, VM, SPLIT, CPI, PAGED>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
+  decode_i8_body<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>(L, T.s[seq].cn, T.s[seq].a, blockIdx.x - seq * L.U);
 }
 
 // ---- host side: the launchers of one metadata format (KM, VM) at every group size ---------------------------
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
 int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_splits, cudaStream_t st) {
-  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
+  using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
   // a paged cache whose page list fits the parameter space: the kernel that takes the table as a parameter
   [[maybe_unused]] PageIds ids;
   bool table_in_params = false;
   if constexpr (PAGED) {
     static std::atomic<unsigned long long> configured_p{0};
     if (a.pages_host && a.n_pages_host <= kParamPages) {
-      if (!opt_in_dynamic_smem(decode_i8_paged_kernel<BITS, G, KM, VM, SPLIT, CPI>, kSmem, configured_p)) return -1;
+      if (!opt_in_dynamic_smem(decode_i8_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, kSmem, configured_p)) return -1;
       for (int i = 0; i < a.n_pages_host; ++i) ids.id[i] = a.pages_host[i];
       table_in_params = true;
     }
@@ -1014,19 +1097,19 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
     cudaError_t err;
     if constexpr (PAGED) {
       if (a.ablation) return -2;      // the timing instances exist for contiguous caches only
-      err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<BITS, G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
-                            : cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
+      err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
+                            : cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     } else if (a.ablation == 1 || a.ablation == 2) {
       static std::atomic<unsigned long long> configured_a1{0}, configured_a2{0};
       if (a.ablation == 1) {
-        if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
-        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 1>, L, cn, a);
+        if (!opt_in_dynamic_smem(decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 1>, L, cn, a);
       } else {
-        if (!opt_in_dynamic_smem(decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
-        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
+        if (!opt_in_dynamic_smem(decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
+        err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
       }
     } else {
-      err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
+      err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     }
     if (err != cudaSuccess) return -1;
     ++launches;
@@ -1035,13 +1118,13 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
 }
 
 // The same kernel over a table of caches (rows per sequence: see launch_one_batched_p of the fp16-operand kernel).
-template <int BITS, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT, int CPI, bool PAGED>
 int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
-  using SL = StageLayout<BITS, BITS, G, KM, VM, CPI>;
+  using SL = StageLayout<KB, VB, G, KM, VM, CPI>;
   constexpr int kSmem = SL::kCtaBytes;
   constexpr int RU = SL::kCH;
   static std::atomic<unsigned long long> configured{0};
-  if (!opt_in_dynamic_smem(decode_i8_batched_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
+  if (!opt_in_dynamic_smem(decode_i8_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, kSmem, configured)) return -1;
   long long chunks[kMaxSeqs], longest = 1;
   for (int i = 0; i < n_seqs; ++i) {
     chunks[i] = T.s[i].cn.n_qv / kChunk;
@@ -1077,7 +1160,7 @@ int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_i8_batched_kernel<BITS, G, KM, VM, SPLIT, CPI, PAGED>, L, T) != cudaSuccess) return -1;
+    if (cudaLaunchKernelEx(&cfg, decode_i8_batched_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, L, T) != cudaSuccess) return -1;
     ++launches;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -1087,44 +1170,44 @@ int launch_i8_batched_p(const Layout& L, SeqTable& T, int n_seqs, int n_splits, 
 // always one), unless a warp gets so few chunks that the second half of an iteration would often be empty (G = 32,
 // where a warp's range may be an odd number of chunks, and fewer than four chunks per warp: short contexts split
 // over many CTAs).
-template <int BITS, int G, int KM, int VM, bool SPLIT>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT>
 int launch_i8_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
   const bool paged = L.page_groups > 0;
   if (cpi == 0 && G == 32 && cn.n_qv / kChunk < 4 * kWarps * (n_splits > 0 ? n_splits : 1)) cpi = 1;
-  if constexpr (BITS == 2) {
+  if constexpr (KB == 2 && VB == 2) {
     if (cpi != 1)
-      return paged ? launch_i8_one_p<BITS, G, KM, VM, SPLIT, 2, true>(L, cn, a, n_splits, st)
-                   : launch_i8_one_p<BITS, G, KM, VM, SPLIT, 2, false>(L, cn, a, n_splits, st);
+      return paged ? launch_i8_one_p<KB, VB, G, KM, VM, SPLIT, 2, true>(L, cn, a, n_splits, st)
+                   : launch_i8_one_p<KB, VB, G, KM, VM, SPLIT, 2, false>(L, cn, a, n_splits, st);
   }
-  return paged ? launch_i8_one_p<BITS, G, KM, VM, SPLIT, 1, true>(L, cn, a, n_splits, st)
-               : launch_i8_one_p<BITS, G, KM, VM, SPLIT, 1, false>(L, cn, a, n_splits, st);
+  return paged ? launch_i8_one_p<KB, VB, G, KM, VM, SPLIT, 1, true>(L, cn, a, n_splits, st)
+               : launch_i8_one_p<KB, VB, G, KM, VM, SPLIT, 1, false>(L, cn, a, n_splits, st);
 }
-template <int BITS, int G, int KM, int VM, bool SPLIT>
+template <int KB, int VB, int G, int KM, int VM, bool SPLIT>
 int launch_i8_cpi_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
   const bool paged = L.page_groups > 0;
-  if constexpr (BITS == 2) {
+  if constexpr (KB == 2 && VB == 2) {
     if (cpi != 1)
-      return paged ? launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 2, true>(L, T, n_seqs, n_splits, st)
-                   : launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 2, false>(L, T, n_seqs, n_splits, st);
+      return paged ? launch_i8_batched_p<KB, VB, G, KM, VM, SPLIT, 2, true>(L, T, n_seqs, n_splits, st)
+                   : launch_i8_batched_p<KB, VB, G, KM, VM, SPLIT, 2, false>(L, T, n_seqs, n_splits, st);
   }
-  return paged ? launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 1, true>(L, T, n_seqs, n_splits, st)
-               : launch_i8_batched_p<BITS, G, KM, VM, SPLIT, 1, false>(L, T, n_seqs, n_splits, st);
+  return paged ? launch_i8_batched_p<KB, VB, G, KM, VM, SPLIT, 1, true>(L, T, n_seqs, n_splits, st)
+               : launch_i8_batched_p<KB, VB, G, KM, VM, SPLIT, 1, false>(L, T, n_seqs, n_splits, st);
 }
 
-template <int BITS, int KM, int VM>
+template <int KB, int VB, int KM, int VM>
 int launch_i8_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_i8_cpi<BITS, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 32) return launch_i8_cpi<BITS, 32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 64) return launch_i8_cpi<BITS, 64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 128) return launch_i8_cpi<BITS, 128, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_i8_cpi<KB, VB, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 32) return launch_i8_cpi<KB, VB, 32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 64) return launch_i8_cpi<KB, VB, 64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
+  if (L.G == 128) return launch_i8_cpi<KB, VB, 128, KM, VM, false>(L, cn, a, n_splits, cpi, st);
   return -2;
 }
-template <int BITS, int KM, int VM>
+template <int KB, int VB, int KM, int VM>
 int launch_i8_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1) return launch_i8_cpi_batched<BITS, 32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 32) return launch_i8_cpi_batched<BITS, 32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 64) return launch_i8_cpi_batched<BITS, 64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 128) return launch_i8_cpi_batched<BITS, 128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 32 && L.r == 1) return launch_i8_cpi_batched<KB, VB, 32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 32) return launch_i8_cpi_batched<KB, VB, 32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 64) return launch_i8_cpi_batched<KB, VB, 64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
+  if (L.G == 128) return launch_i8_cpi_batched<KB, VB, 128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
   return -2;
 }
 
@@ -1132,14 +1215,14 @@ int launch_i8_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_spl
 
 // Defines the externally visible launchers of one metadata format in the translation unit that compiles its kernels
 // (same names as the fp16-operand kernel's: the host dispatch does not change).
-#define IQ_DEFINE_I8_FORMAT(BITS, KM, VM)                                                                            \
-  int IQ_MMA_FORMAT_NAME(BITS, BITS, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,   \
+#define IQ_DEFINE_I8_FORMAT(KB, VB, KM, VM)                                                                           \
+  int IQ_MMA_FORMAT_NAME(KB, VB, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,   \
                                              int cpi, cudaStream_t st) {                                              \
-    return launch_i8_format<BITS, KM, VM>(L, cn, a, n_splits, cpi, st);                                               \
+    return launch_i8_format<KB, VB, KM, VM>(L, cn, a, n_splits, cpi, st);                                               \
   }                                                                                                                   \
-  int IQ_MMA_FORMAT_NAME_BATCHED(BITS, BITS, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, \
+  int IQ_MMA_FORMAT_NAME_BATCHED(KB, VB, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, \
                                                      cudaStream_t st) {                                               \
-    return launch_i8_format_batched<BITS, KM, VM>(L, T, n_seqs, n_splits, cpi, st);                                   \
+    return launch_i8_format_batched<KB, VB, KM, VM>(L, T, n_seqs, n_splits, cpi, st);                                   \
   }
 
 }  // namespace iq

@@ -3,5 +3,5 @@
 #include "innerq_decode_i8.cuh"
 
 namespace iq {
-IQ_DEFINE_I8_FORMAT(2, 4, 4)
+IQ_DEFINE_I8_FORMAT(2, 2, 4, 4)
 }  // namespace iq

@@ -1,6 +1,7 @@
-// Decode kernels of one packed format: 3-bit keys, 4-bit values, 2 / 4 bytes per key / value metadata entry.
-#include "innerq_decode_mma.cuh"
+// Decode kernels of one packed format: 3-bit keys, 4-bit values (byte order, integer MMA), 2 / 4 bytes per key /
+// value metadata entry.
+#include "innerq_decode_i8.cuh"
 
 namespace iq {
-IQ_DEFINE_MMA_FORMAT(3, 4, 2, 4)
+IQ_DEFINE_I8_FORMAT(3, 4, 2, 4)
 }  // namespace iq

@@ -1,6 +1,7 @@
-// Decode kernels of one packed format: 4-bit keys, 2-bit values, 4 / 2 bytes per key / value metadata entry.
-#include "innerq_decode_mma.cuh"
+// Decode kernels of one packed format: 4-bit keys, 2-bit values (byte order, integer MMA), 4 / 2 bytes per key /
+// value metadata entry.
+#include "innerq_decode_i8.cuh"
 
 namespace iq {
-IQ_DEFINE_MMA_FORMAT(4, 2, 4, 2)
+IQ_DEFINE_I8_FORMAT(4, 2, 4, 2)
 }  // namespace iq

@@ -3,5 +3,5 @@
 #include "innerq_decode_i8.cuh"
 
 namespace iq {
-IQ_DEFINE_I8_FORMAT(4, 2, 2)
+IQ_DEFINE_I8_FORMAT(4, 4, 2, 2)
 }  // namespace iq

@@ -13,6 +13,10 @@ __device__ __forceinline__ uint16_t f2h_bits(float f) { return __half_as_ushort(
 
 // ---- packed-code accessors (generic, slow; the fast kernels extract fragments directly) ----
 __device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, int c, int bits, int perm = 0) {
+  if (perm == 1 && bits == 3) {
+    const BitPos3 p = row_pos_i8_3(c);
+    return code3_join((row[p.lo.word] >> p.lo.bit) & 3u, (row[p.hi.word] >> p.hi.bit) & 1u, p.odd);
+  }
   if (perm == 1) {
     BitPos p = row_pos_i8(c, bits);
     return (row[p.word] >> p.bit) & ((1u << bits) - 1u);
@@ -26,6 +30,10 @@ __device__ __forceinline__ uint32_t row_code(const uint32_t* __restrict__ row, i
 }
 
 __device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chunk, int tau, int c, int bits, int perm = 0) {
+  if (perm == 1 && bits == 3) {
+    const BitPos3 p = block_pos_i8_3(tau, c);
+    return code3_join((chunk[p.lo.word] >> p.lo.bit) & 3u, (chunk[p.hi.word] >> p.hi.bit) & 1u, p.odd);
+  }
   if (perm == 1) {
     BitPos p = block_pos_i8(tau, c, bits);
     return (chunk[p.word] >> p.bit) & ((1u << bits) - 1u);
@@ -40,7 +48,11 @@ __device__ __forceinline__ uint32_t chunk_code(const uint32_t* __restrict__ chun
 
 // OR a code into a zero-initialised packed row / chunk held in shared memory.
 __device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t code, int perm = 0) {
-  if (perm == 1) {
+  if (perm == 1 && bits == 3) {
+    const BitPos3 p = row_pos_i8_3(c);
+    atomicOr(&row[p.lo.word], code3_lo(code, p.odd) << p.lo.bit);
+    atomicOr(&row[p.hi.word], code3_hi(code, p.odd) << p.hi.bit);
+  } else if (perm == 1) {
     BitPos p = row_pos_i8(c, bits);
     atomicOr(&row[p.word], code << p.bit);
   } else if (bits == 3) {
@@ -53,7 +65,11 @@ __device__ __forceinline__ void row_put(uint32_t* row, int c, int bits, uint32_t
   }
 }
 __device__ __forceinline__ void chunk_put(uint32_t* chunk, int tau, int c, int bits, uint32_t code, int perm = 0) {
-  if (perm == 1) {
+  if (perm == 1 && bits == 3) {
+    const BitPos3 p = block_pos_i8_3(tau, c);
+    atomicOr(&chunk[p.lo.word], code3_lo(code, p.odd) << p.lo.bit);
+    atomicOr(&chunk[p.hi.word], code3_hi(code, p.odd) << p.hi.bit);
+  } else if (perm == 1) {
     BitPos p = block_pos_i8(tau, c, bits);
     atomicOr(&chunk[p.word], code << p.bit);
   } else if (bits == 3) {

@@ -47,8 +47,8 @@ struct Store {
                        // under outer grouping keys keep rows and values keep chunks, only the metadata changes sides.
   int bits, mode;
   int perm;            // order of the codes inside a packed row / chunk: 0 = pairs for the fp16 tensor-core fragments
-                       // (word & mask is a half2), 1 = bytes for the 8-bit integer fragments (inner-grouped caches
-                       // whose keys and values are both 2-bit or both 4-bit; see row_pos_i8 / block_pos_i8)
+                       // (word & mask is a half2; outer-grouped caches), 1 = bytes for the 8-bit integer fragments
+                       // (inner-grouped caches; see row_pos_i8 / block_pos_i8 / row_pos_i8_3 / block_pos_i8_3)
   int ring_cap;        // slots of the recent ring: w_recent + 1 (ROW) or w_recent + G (BLOCK)
   int cap_q;           // capacity in quantised tokens (multiple of kTile)
   int n_groups;        // metadata entries per row (ROW: D/G) or per group (BLOCK: D)
@@ -254,6 +254,51 @@ IQ_HD BitPos block_pos_i8(int tau, int c, int bits = 2) {
   r.bit = 8 * (k & 3) + bits * p;
   return r;
 }
+
+// 3-bit codes in byte order: a 2-bit plane laid out exactly as the 2-bit codes above (row words 0..7, chunk words
+// 0..255) followed by a 1-bit plane (row words 8..11, chunk words 256..383).  The split of a code between the planes
+// alternates with the bit position p of its 2-bit field, so that one bit-select of the two planes yields 3-bit fields
+// that no shift has to align:
+//   p even: 2-bit plane = code & 3,  1-bit plane = code >> 2, put right ABOVE the field: bits 4(p/2) + {0,1,2},
+//           i.e. the code times 16^(p/2);
+//   p odd:  2-bit plane = code >> 1, 1-bit plane = code & 1,  put right BELOW the field: bits 4(p/2) + {1,2,3},
+//           i.e. the code times 2 * 16^(p/2).
+// The 1-bit plane word of a lane pairs with two 2-bit words (ROW: h = 0, 1, the two k halves of a row; BLOCK: W = 0,
+// 1, the two sets of four m-tiles); its bits for the first one sit where they are used (p = 0,1,2,3 -> bit 2,1,6,5 of
+// the byte), those for the second one next to them (bit 3,0,7,4: `>> 1` for even p, `<< 1` for odd p).
+IQ_HD int hi_bit_i8(int p, int second) {
+  const int b = ((p & 1) ? 1 : 2) + 4 * (p >> 1);
+  return second ? b + ((p & 1) ? -1 : 1) : b;
+}
+// weight of the 3-bit field of bit position p after the bit-select: 1, 2, 16, 32
+IQ_HD int field_weight_i8_3(int p) { return (1 + (p & 1)) << (4 * (p >> 1)); }
+struct BitPos3 { BitPos lo, hi; int odd; };      // positions in the two planes; odd: the split of the code (see above)
+IQ_HD BitPos3 row_pos_i8_3(int c) {
+  const int p = c >> 5, k = c & 31, lw = k >> 2, j = lw & 3, h = lw >> 2;
+  BitPos3 r;
+  r.lo.word = 2 * j + h;
+  r.lo.bit = 8 * (k & 3) + 2 * p;
+  r.hi.word = 8 + j;
+  r.hi.bit = 8 * (k & 3) + hi_bit_i8(p, h);
+  r.odd = p & 1;
+  return r;
+}
+IQ_HD BitPos3 block_pos_i8_3(int tau, int c) {
+  const int k = 4 * (tau & 7) + (tau >> 3);
+  const int m = 4 * (c >> 6) + ((c >> 1) & 3), gid = (c >> 3) & 7, rh = c & 1;
+  const int j = (k & 15) >> 2, half = k >> 4, W = m >> 2, p = m & 3;
+  BitPos3 r;
+  r.lo.word = W * 128 + (4 * gid + j) * 4 + 2 * half + rh;
+  r.lo.bit = 8 * (k & 3) + 2 * p;
+  r.hi.word = 256 + (4 * gid + j) * 4 + 2 * half + rh;
+  r.hi.bit = 8 * (k & 3) + hi_bit_i8(p, W);
+  r.odd = p & 1;
+  return r;
+}
+// the two plane values of a 3-bit code, and the code from them
+IQ_HD uint32_t code3_lo(uint32_t code, int odd) { return odd ? (code >> 1) & 3u : code & 3u; }
+IQ_HD uint32_t code3_hi(uint32_t code, int odd) { return odd ? code & 1u : (code >> 2) & 1u; }
+IQ_HD uint32_t code3_join(uint32_t lo, uint32_t hi, int odd) { return odd ? (lo << 1) | hi : lo | (hi << 2); }
 
 // BLOCK store metadata: the 128 per-channel entries of a group are ordered so that the 16 channels a
 // lane owns in the PV fragments are contiguous (entry 2*m + rh of lane gid): 4 x 128-bit loads.

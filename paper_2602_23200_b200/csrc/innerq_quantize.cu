@@ -317,30 +317,34 @@ __device__ __forceinline__ void append_unit(const Layout& L, const __half* __res
   append_publish(L, N, u, cache, n_parts);
 }
 
-// Quarter of a group eviction of a chunk-coded BLOCK store: channels 32 q .. 32 q + 31 of the G oldest ring tokens
-// (first token t_first; the row appended by this very step, token N - 1, is taken from the call's input x_new, which
-// another CTA is writing to the ring at the same time).  128 threads: lane = channel, warp = quarter of the tokens.
-// The words of a packed chunk that hold these channels hold no others (see block_pos_plane / block_pos_i8: a word
-// belongs to one lane group gid and one half W of the channels), so the quarters write disjoint words.
+// Quarter of a group eviction of a chunk-coded BLOCK store: 32 channels of the G oldest ring tokens (first token
+// t_first; the row appended by this very step, token N - 1, is taken from the call's input x_new, which another CTA
+// is writing to the ring at the same time).  128 threads: lane = channel of the quarter, warp = quarter of the tokens.
+// The quarters write disjoint words of the packed chunks.  Pair order (perm = 0): quarter q = channels 32 q ..
+// 32 q + 31; a word belongs to one lane group gid and one half W of the channels (see block_pos_plane).  Byte order
+// (perm = 1): a word belongs to one lane group gid, and the 1-bit plane of 3-bit codes holds both halves W in one
+// word, so quarter q is the channels of lane groups 2 q and 2 q + 1: 16 q .. 16 q + 15 and 64 + 16 q .. 64 + 16 q + 15.
+__device__ __forceinline__ int quarter_channel(int q, int cl, int perm) {      // channel of lane cl of quarter q
+  return perm == 1 ? 64 * (cl >> 4) + 16 * q + (cl & 15) : 32 * q + cl;
+}
 __device__ __forceinline__ int chunk_word_quarter(int i, int bits, int perm) {
+  if (perm == 1) return (i & 127) >> 5;                    // word = set * 128 + lane * 4 + role, gid = lane / 4
   if (bits == 3 && i >= chunk_hi_plane_word()) {
     const int r = i - chunk_hi_plane_word();
     return 2 * ((r & 3) >> 1) + ((r >> 2) >> 4);          // word = lane * 4 + (m >> 1), m >> 1 = 2 W + ..; gid = lane / 4
   }
-  if (perm == 1 && bits == 4)                              // byte order, 16 words per lane: word set W = i / 128 = m / 2
-    return 2 * (i >> 8) + (((i & 127) >> 2) >> 4);
   const int r = i & 255;                                   // 4-bit codes in pair order: two k-step halves of 256 words
   return 2 * (r >> 7) + (((r & 127) >> 2) >> 4);           // W = r / 128, gid = ((r % 128) / 4) / 4 -> 2 W + gid / 4
 }
 __device__ void quantize_block_quarter(const TokSrc& src, const __half* __restrict__ x_new, int t_new, int t_first,
                                        const Layout& L, const Store& S, __half* tile, uint32_t* words, float* red,
                                        const Rec& rec, int group_j, int q) {
-  const int G = L.G, cl = threadIdx.x & 31, part = threadIdx.x >> 5, c = 32 * q + cl;
+  const int G = L.G, cl = threadIdx.x & 31, part = threadIdx.x >> 5, c = quarter_channel(q, cl, S.perm);
   const int cw = chunk_bytes(S.bits) / 4, n_words = (G / kChunk) * cw, per = G >> 2;
   for (int i = threadIdx.x; i < G * 4; i += 128) {         // 4 x 16-byte pieces of the quarter per token row
     const int t = i >> 2, piece = i & 3;
     const __half* row = t_first + t == t_new ? x_new : src.row(t_first + t);
-    reinterpret_cast<uint4*>(tile)[i] = *reinterpret_cast<const uint4*>(row + 32 * q + piece * 8);
+    reinterpret_cast<uint4*>(tile)[i] = *reinterpret_cast<const uint4*>(row + quarter_channel(q, piece * 8, S.perm));
   }
   for (int i = threadIdx.x; i < n_words; i += 128) words[i] = 0u;
   __syncthreads();

@@ -186,6 +186,39 @@ __device__ __forceinline__ void pack_block_segment_i8(const ChosenCoder& cc, con
   for (int i = 0; i < 8; ++i) w8[i] -= cw[i];
 }
 
+// 3-bit codes in byte order (see row_pos_i8_3 / block_pos_i8_3): the 2-bit plane's words as above (bit position 0)
+// and the 1-bit plane's bits at bit 0 of their bytes; `odd` (bit position of the segment is odd) picks the split of
+// a code between the planes.  ROW: hw[h][j] = 1-bit plane word j, bits of row half h.
+template <bool CLAMP>
+__device__ __forceinline__ void pack_row_segment_i8_3(const ChosenCoder& cc, const float (&x)[kSeg], int odd,
+                                                      uint32_t (&w8)[8], uint32_t (&hw)[2][4]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { w8[i] = 0u; hw[i >> 2][i & 3] = 0u; }
+  const int sh_lo = odd, sh_hi = odd ? 0 : 2;
+#pragma unroll
+  for (int e = 0; e < kSeg; ++e) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[e]);      // kMagicBits + code: the low bits are the code
+    const int lw = e >> 2, j = lw & 3, h = lw >> 2, sh = 8 * (e & 3);
+    w8[2 * j + h] |= ((code >> sh_lo) & 3u) << sh;
+    hw[h][j] |= ((code >> sh_hi) & 1u) << sh;
+  }
+}
+// BLOCK: word index 2 * j + half in both planes.
+template <bool CLAMP>
+__device__ __forceinline__ void pack_block_segment_i8_3(const ChosenCoder& cc, const float (&x)[kSeg], int odd,
+                                                        uint32_t (&w8)[8], uint32_t (&h8)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { w8[i] = 0u; h8[i] = 0u; }
+  const int sh_lo = odd, sh_hi = odd ? 0 : 2;
+#pragma unroll
+  for (int t = 0; t < kSeg; ++t) {
+    const uint32_t code = cc.template code_bits<CLAMP>(x[t]);
+    const int k = 4 * (t & 7) + (t >> 3), li = 2 * ((k & 15) >> 2) + (k >> 4), sh = 8 * (k & 3);
+    w8[li] |= ((code >> sh_lo) & 3u) << sh;
+    h8[li] |= ((code >> sh_hi) & 1u) << sh;
+  }
+}
+
 __device__ __forceinline__ void unpack8(const uint4& v, float* x) {
   const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
@@ -273,8 +306,17 @@ __global__ void __launch_bounds__(128) quantize_rows_prefill_kernel(Layout L, St
     }
     const ChosenCoder cc(sc, asym);
     uint32_t* row = stage + tk * RW;
-    if constexpr (I8) {
-      static_assert(!I8 || BITS == 2 || BITS == 4, "byte order is defined for 2- and 4-bit codes");
+    if constexpr (I8 && BITS == 3) {
+      uint32_t w8[8], hw[2][4];
+      if (no_clip) pack_row_segment_i8_3<false>(cc, x, seg & 1, w8, hw);
+      else pack_row_segment_i8_3<true>(cc, x, seg & 1, w8, hw);
+      __syncwarp();                                        // the stage is zero and no longer being read
+      const int b0 = hi_bit_i8(seg, 0), b1 = hi_bit_i8(seg, 1);
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) atomicOr(&row[jj], w8[jj] << (2 * seg));
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) atomicOr(&row[8 + jj], (hw[0][jj] << b0) | (hw[1][jj] << b1));
+    } else if constexpr (I8) {
       uint32_t w8[8];
       if (no_clip) pack_row_segment_i8<BITS, false>(cc, x, w8);
       else pack_row_segment_i8<BITS, true>(cc, x, w8);
@@ -342,8 +384,9 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
 #pragma unroll
     for (int i = 0; i < NW; ++i) wlo[i] = 0u;
     [[maybe_unused]] uint32_t w16[2][8];      // byte order: words [rh][2 * j + half] of this channel pair, at its bit position
+    [[maybe_unused]] uint32_t h16[I8 && BITS == 3 ? 2 : 1][8];      // ... of the 1-bit plane of 3-bit codes
     uint32_t meta2[2];
-    if (CH > 1) __syncthreads();       // the previous group's reduction words are no longer read
+    if (CH > 1 || (I8 && BITS == 3)) __syncthreads();       // the previous group's exchange words are no longer read
 #pragma unroll
     for (int rh = 0; rh < 2; ++rh) {
       float x[kSeg];
@@ -384,7 +427,13 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
         asym = ea < es;
       }
       const ChosenCoder cc(sc, asym);
-      if constexpr (I8) {
+      if constexpr (I8 && BITS == 3) {
+        if (no_clip) pack_block_segment_i8_3<false>(cc, x, cp & 1, w16[rh], h16[rh]);
+        else pack_block_segment_i8_3<true>(cc, x, cp & 1, w16[rh], h16[rh]);
+        const int sh_hi = hi_bit_i8(cp & 3, c0 >> 6);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { w16[rh][i] <<= 2 * (cp & 3); h16[rh][i] <<= sh_hi; }
+      } else if constexpr (I8) {
         if (no_clip) pack_block_segment_i8<BITS, false>(cc, x, w16[rh]);
         else pack_block_segment_i8<BITS, true>(cc, x, w16[rh]);
 #pragma unroll
@@ -425,33 +474,49 @@ __global__ void __launch_bounds__(256) quantize_blocks_prefill_kernel(Layout L, 
       // Reduce-scatter by OR: after two exchange steps lane `pos` holds the complete words of j = pos (two halves,
       // two row halves), which are 16 contiguous bytes of the chunk.
       const int pos = cp & 3;
-      uint32_t h8[2][4];                      // step 1: keep j of my parity (j = 2 * i + (pos & 1)), index [rh][2 * i + half]
+      auto reduce_scatter = [&](const uint32_t (&w)[2][8]) {
+        uint32_t h8[2][4];                    // step 1: keep j of my parity (j = 2 * i + (pos & 1)), index [rh][2 * i + half]
 #pragma unroll
-      for (int rh = 0; rh < 2; ++rh)
+        for (int rh = 0; rh < 2; ++rh)
 #pragma unroll
-        for (int i = 0; i < 2; ++i)
+          for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const uint32_t keep = (pos & 1) ? w[rh][2 * (2 * i + 1) + half] : w[rh][2 * (2 * i) + half];
+              const uint32_t give = (pos & 1) ? w[rh][2 * (2 * i) + half] : w[rh][2 * (2 * i + 1) + half];
+              h8[rh][2 * i + half] = keep | __shfl_xor_sync(0xffffffffu, give, 1);
+            }
+        uint32_t f4[4];                       // step 2: keep i = pos >> 1; index 2 * half + rh (the word order in the chunk)
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh)
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            const uint32_t keep = (pos & 1) ? w16[rh][2 * (2 * i + 1) + half] : w16[rh][2 * (2 * i) + half];
-            const uint32_t give = (pos & 1) ? w16[rh][2 * (2 * i) + half] : w16[rh][2 * (2 * i + 1) + half];
-            h8[rh][2 * i + half] = keep | __shfl_xor_sync(0xffffffffu, give, 1);
+            const uint32_t keep = (pos & 2) ? h8[rh][2 + half] : h8[rh][half];
+            const uint32_t give = (pos & 2) ? h8[rh][half] : h8[rh][2 + half];
+            f4[2 * half + rh] = keep | __shfl_xor_sync(0xffffffffu, give, 2);
           }
-      uint32_t f4[4];                         // step 2: keep i = pos >> 1; index 2 * half + rh (the word order in the chunk)
-#pragma unroll
-      for (int rh = 0; rh < 2; ++rh)
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t keep = (pos & 2) ? h8[rh][2 + half] : h8[rh][half];
-          const uint32_t give = (pos & 2) ? h8[rh][half] : h8[rh][2 + half];
-          f4[2 * half + rh] = keep | __shfl_xor_sync(0xffffffffu, give, 2);
-        }
+        return make_uint4(f4[0], f4[1], f4[2], f4[3]);
+      };
       const int W = c0 >> 6;
-      *reinterpret_cast<uint4*>(chunk + W * 128 + (4 * gid + pos) * 4) = make_uint4(f4[0], f4[1], f4[2], f4[3]);
+      *reinterpret_cast<uint4*>(chunk + W * 128 + (4 * gid + pos) * 4) = reduce_scatter(w16);
+      if constexpr (BITS == 3) {
+        // 1-bit plane: the words of lane group gid hold the bits of both halves W of the channels, which two warps
+        // of this chunk's 64 threads computed: the second hands its words to the first through shared memory
+        uint4* hx = reinterpret_cast<uint4*>(smem_q + (size_t)CH * 128 * 16) + k * 32 + (cp & 31);
+        const uint4 mine = reduce_scatter(h16);
+        if (W == 1) *hx = mine;
+        __syncthreads();
+        if (W == 0) {
+          const uint4 o = *hx;
+          *reinterpret_cast<uint4*>(chunk + 256 + (4 * gid + pos) * 4) =
+              make_uint4(mine.x | o.x, mine.y | o.y, mine.z | o.z, mine.w | o.w);
+        }
+      }
     } else {
 #pragma unroll
       for (int i = 0; i < NW; ++i) chunk[base_lo + 4 * (i & 3) + 256 * (i >> 2)] = wlo[i];
     }
-    if constexpr (BITS == 3) {
+    if constexpr (BITS == 3 && !I8) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const uint32_t full = whi[i] | __shfl_xor_sync(0xffffffffu, whi[i], 1);   // the pair with the other m & 1
@@ -477,23 +542,20 @@ static int launch_store_bits(const Layout& L, const Store& S, const __half* X, i
     const int n_batches = (n_q + 7) / 8;
     const int per_unit = grid_cap((n_batches + 4 * 8 - 1) / (4 * 8), grid_cap(148 * 16 / L.U, 1 << 16));
     dim3 grid(per_unit, L.U);
-    if constexpr (BITS == 2 || BITS == 4) {
-      if (S.perm == 1) {
-        if (inv_norm) quantize_rows_prefill_kernel<BITS, true, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
-        else quantize_rows_prefill_kernel<BITS, false, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
-        return cudaGetLastError() == cudaSuccess ? 1 : -1;
-      }
+    if (S.perm == 1) {
+      if (inv_norm) quantize_rows_prefill_kernel<BITS, true, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
+      else quantize_rows_prefill_kernel<BITS, false, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
+      return cudaGetLastError() == cudaSuccess ? 1 : -1;
     }
     if (inv_norm) quantize_rows_prefill_kernel<BITS, true><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, inv_norm);
     else quantize_rows_prefill_kernel<BITS, false><<<grid, 128, 0, st>>>(L, S, X, N, n_q, cache, nullptr);
   } else {
     const int CH = L.G / kChunk;
-    const int smem = CH * 128 * 16;                   // reduction words of groups spanning several chunks
+    // reduction words of groups spanning several chunks; 3-bit codes in byte order: exchange of the 1-bit plane's words
+    const int smem = CH * 128 * 16 + (BITS == 3 && S.perm == 1 ? CH * 32 * 16 : 0);
     auto kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true> : quantize_blocks_prefill_kernel<BITS, false>;
-    if constexpr (BITS == 2 || BITS == 4) {
-      if (S.perm == 1)
-        kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true, true> : quantize_blocks_prefill_kernel<BITS, false, true>;
-    }
+    if (S.perm == 1)
+      kern = inv_norm ? quantize_blocks_prefill_kernel<BITS, true, true> : quantize_blocks_prefill_kernel<BITS, false, true>;
     const int n_groups = n_q / L.G;
     dim3 grid(grid_cap(n_groups, grid_cap(148 * 16 / L.U, 1 << 16)), L.U);
     kern<<<grid, 64 * CH, smem, st>>>(L, S, X, N, n_q, cache, inv_norm);
