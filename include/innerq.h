@@ -293,8 +293,9 @@ int innerq_cache_import(innerq_cache_t* cache, const innerq_export_t* ex, int32_
  *              6 / 7 TIMING ONLY, the output is wrong on purpose: the warp-MMA kernel with the unpack + MMA work of
  *              its key side (6) or value side (7) left out of the streaming loop, the bytes still streamed; what
  *              a side costs is the difference to the full kernel (process-wide knob; any other variant clears it;
- *              contiguous caches in the 2-bit formats, the 3-bit / 3-bit, 3-bit / 2-bit and 4-bit / 4-bit formats of
- *              the latency study and the outer-grouped cache: UNSUPPORTED elsewhere).
+ *              contiguous caches with 2-bit keys and values or 4-bit keys and values, the 3-bit / 3-bit and
+ *              3-bit / 2-bit formats of the latency study (both sides with zero-points, both without, and 3 / 2 with
+ *              scale-only keys and full values) and the outer-grouped cache: UNSUPPORTED elsewhere).
  * Errors: INVALID_ARG. */
 int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t variant);
 

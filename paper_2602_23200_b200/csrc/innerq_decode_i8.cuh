@@ -1100,6 +1100,7 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
       err = table_in_params ? cudaLaunchKernelEx(&cfg, decode_i8_paged_kernel<KB, VB, G, KM, VM, SPLIT, CPI>, L, cn, a, ids)
                             : cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     } else if (a.ablation == 1 || a.ablation == 2) {
+#ifdef IQ_WITH_TIMING_INSTANCES      // defined by the translation units of the formats the latency study and the bench time
       static std::atomic<unsigned long long> configured_a1{0}, configured_a2{0};
       if (a.ablation == 1) {
         if (!opt_in_dynamic_smem(decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 1>, kSmem, configured_a1)) return -1;
@@ -1108,6 +1109,9 @@ int launch_i8_one_p(const Layout& L, const Counts& cn, DecodeArgs a, int n_split
         if (!opt_in_dynamic_smem(decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 2>, kSmem, configured_a2)) return -1;
         err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, false, 2>, L, cn, a);
       }
+#else
+      return -2;
+#endif
     } else {
       err = cudaLaunchKernelEx(&cfg, decode_i8_kernel<KB, VB, G, KM, VM, SPLIT, CPI, PAGED>, L, cn, a);
     }

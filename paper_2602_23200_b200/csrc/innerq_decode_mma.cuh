@@ -1,4 +1,8 @@
-// Fused decode attention over the packed InnerQ cache (INNER layout), one launch:
+// Fused decode attention over a packed cache with pair-ordered codes (Store::perm = 0), one launch.  Built today for
+// the outer-grouped comparison cache only (OUTER = true: innerq_decode_mma_outer.cu); inner-grouped caches keep their
+// codes in byte order and are decoded by the integer-operand kernel (innerq_decode_i8.cuh), which shares this file's
+// launch shape, pipeline helpers, tail tiles and merge.  The description below is of the inner-grouped form, from
+// which the outer-grouped one differs in where scales and zero-points are applied (see OUTER in the kernel).
 //   q.K^T on packed key rows  ->  online softmax  ->  p.V on packed value chunks, split over token
 //   ranges, fp16 windows and the K/V skew zone as 16-token tiles dealt to the same warps, cross-CTA merge by
 //   the last CTA to finish.
@@ -154,6 +158,7 @@ template <int KB, int VB, int G, int KM, int VM, int CPI> struct StageLayout {
   // group spans several iterations, inside one group)
   __host__ __device__ static constexpr int off(int cc) { return cc * kRec + (cc / kCH) * kVMeta; }
   static constexpr int kBytes = CPI * kRec + (CPI / kCH > 0 ? CPI / kCH : 1) * kVMeta;
+  // (three stages of the 4 KB records of 3-bit keys with 3-bit values fit as well and were measured: no gain)
   static constexpr int kStages = kBytes <= 3072 ? 4 : 2;
   static constexpr int kWarpBytes = kBytes * kStages;
   static constexpr int kSideBytes = 4 * kD * 4;                   // per warp: value metadata of the last 4 groups
