@@ -743,8 +743,8 @@ def run_ours(args, w):
                                     "step": value_gbs / world / 80.0},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": which, "traffic": stored_traffic(w.name),
-                         "traffic_source": ("stored: ncu capture of one launch of this workload, "
-                                            + str((counters or {}).get("captured_at", "profiles/decode_counters.json")))
+                         "traffic_source": ("stored in profiles/decode_counters.json: "
+                                            + str((counters or {}).get("captured_at", "ncu capture of one launch")))
                          if counters else None,
                          "note": "achieved = algorithmic bytes of one decode / MEDIAN duration of 48 decode launches "
                                  "that are each bracketed by their own events (us_per_decode_alone), so none "
