@@ -1,6 +1,6 @@
 // Host side of the fused decode kernel over the packed InnerQ cache: picks the kernel family of the cache's
-// packed format and fills the launch parameters.  The kernels are in innerq_decode_mma.cuh and are compiled
-// one translation unit per format (innerq_decode_mma_k*v*_m*.cu).
+// packed format and fills the launch parameters.  The kernels are in innerq_decode_i8.cuh (inner-grouped caches,
+// one translation unit per format: innerq_decode_mma_k*v*_m*.cu) and innerq_decode_mma.cuh (outer-grouped caches).
 #include "innerq_decode_mma.h"
 #include "innerq_kernels.h"
 
@@ -14,7 +14,8 @@ int g_ablation = 0;           // timing experiments: see DecodeArgs::ablation
 using FormatLauncher = int (*)(const Layout&, const Counts&, const DecodeArgs&, int, int, cudaStream_t);
 
 // The formats with kernels: every combination of 2 / 3 / 4-bit keys and values with full or scale-only metadata
-// (2-bit keys with 2-bit values: the integer-MMA kernel), and the outer-grouped comparison cache at 2 and 4 bits.
+// (all instances of the integer-MMA kernel, innerq_decode_i8.cuh), and the outer-grouped comparison cache at 2 and 4
+// bits (the fp16-operand kernel, innerq_decode_mma.cuh).
 struct FormatEntry {
   int kb, vb, km, vm;
   FormatLauncher one;

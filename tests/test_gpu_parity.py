@@ -171,6 +171,8 @@ def test_fused_kernel_formats(kb, vb, km, vm, G, r, N):
         oc.append(k1, v1)
         gc.innerq_append_token(dev(k1), dev(v1))
     check_decode(w, oc, gc, step=7, variants=(3,), splits=(0, 3))
+    # what the appends packed (one row per step, one value group on the way), bit for bit
+    P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, km == O.HYBRID, vm == O.HYBRID)
 
 
 @pytest.mark.parametrize("N", [1, 3, 4, 5, 19, 20, 21, 52, 53])
