@@ -345,19 +345,40 @@ class Legs:
         """n decodes, each between its own pair of events (no overlap with its neighbours).  Returns a list of us."""
         evs = [(self._ev(), self._ev()) for _ in range(n)]
         self.delay()
+        nq = len(self.q_all)
         for j in range(4):                                      # untimed, so that the first bracket is not the coldest
-            self.caches[j % self.R].innerq_decode_attention(self.q_all[j], self.out)
-        for j, (a, b) in enumerate(evs):
+            self.caches[j % self.R].innerq_decode_attention_ptr(self.qp + (j % nq) * self.q_stride, self.op, self.sp)
+        # Event timestamps advance in steps of about 2 us on this GPU: a spacer of random length in front of every
+        # bracket keeps the brackets from all falling on the same side of a step (median and mean then tell more).
+        spacer = np.random.default_rng(7).integers(0, 8000, size=n)
+        for j, (a, b) in enumerate(evs):                        # calls by address: the host stays ahead of the GPU
+            self.torch.cuda._sleep(int(spacer[j]))
             a.record(self.stream)
-            self.caches[j % self.R].innerq_decode_attention(self.q_all[j % len(self.q_all)], self.out)
+            self.caches[j % self.R].innerq_decode_attention_ptr(self.qp + (j % nq) * self.q_stride, self.op, self.sp)
             b.record(self.stream)
         self.torch.cuda.synchronize()
         return [a.elapsed_time(b) * 1e3 for a, b in evs]
 
+    def bracket_floor(self, n=32):
+        """Median us between the two events of a bracket that holds one trivial kernel (a 32-byte torch fill): what the
+        bracketing itself and a kernel launch cost on this machine, for reading `us_per_decode_alone`."""
+        x = self.torch.zeros(8, device=self.out.device)
+        evs = [(self._ev(), self._ev()) for _ in range(n)]
+        self.delay()
+        for _ in range(4):
+            x.fill_(1.0)
+        for a, b in evs:
+            a.record(self.stream)
+            x.fill_(1.0)
+            b.record(self.stream)
+        self.torch.cuda.synchronize()
+        return float(np.median([a.elapsed_time(b) * 1e3 for a, b in evs]))
+
     def decodes_chained(self, n, caches=None, call=None):
         """n decodes launched back to back over the rotating instances: us per decode of the chain."""
         caches = caches or self.caches
-        call = call or (lambda c, j: c.innerq_decode_attention(self.q_all[j % len(self.q_all)], self.out))
+        nq = len(self.q_all)
+        call = call or (lambda c, j: c.innerq_decode_attention_ptr(self.qp + (j % nq) * self.q_stride, self.op, self.sp))
         self.delay()
         for j in range(4):
             call(caches[j % len(caches)], j)
@@ -634,6 +655,7 @@ def run_ours(args, w):
     leg_us, leg_host_us = legs.steps(LEG, warm=32)
     # ---- the decode kernel alone: every launch between its own events (the roofline figure), and chained -------
     alone = stats(legs.decodes_bracketed(48))
+    alone["trivial_kernel_in_the_same_bracket_us"] = legs.bracket_floor()
     b2b_us = legs.decodes_chained(64)
     clocks = sampler.stop()
     assert all(c.n_tokens == w.n_tokens + (legs.i - 1 - r) // R + 1 for r, c in enumerate(caches))
@@ -797,8 +819,11 @@ def main():
     ap.add_argument("--literal", type=int, default=1, help="1: also report the paper-literal symmetric variant")
     ap.add_argument("--per-config", default="c4,c3_4bit,c3_2bit",
                     help="further workloads measured into the line's per_config block ('' to skip)")
+    ap.add_argument("--tokens", type=int, default=0, help="context length instead of the workload's own (experiments)")
     args = ap.parse_args()
     w = workload_by_name(args.workload)
+    if args.tokens > 0:
+        w = w.with_(n_tokens=args.tokens, name=f"{w.name}@{args.tokens}")
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -17,6 +17,8 @@
 // Integer accumulators start from the bit pattern of a float constant (2^23 or 1.5 * 2^23), so that reading them
 // as floats and subtracting the constant converts them exactly with one fp32 addition instead of a conversion.
 #pragma once
+#include <type_traits>
+
 #include "innerq_decode_mma.cuh"
 
 namespace iq {
@@ -375,16 +377,23 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
     const float wj = KB == 2 ? pow2i(-2 * j) : KB == 4 ? pow2i(-4 * (j & 1)) : pow2i(-(4 * (j >> 1) + (j & 1)));
     const float wjm = -wj * kMagicSf;
     const float neg_half = -(float)(1 << (KB - 1)), neg_half_v = -(float)(1 << (VB - 1));               // -2^(b-1)
-    // 128 * hi + lo of one accumulator pair (bit patterns of kMagicSf + sum), times the power of two w: exact
+    // 128 * hi + lo of one accumulator pair (bit patterns of kMagicSf + sum), times the power of two w (wm = -w *
+    // kMagicSf).  The inner product, 128 w H - w kMagicSf, is a multiple of 128 w below 2^24 of them: exact; the outer one
+    // rounds w (128 H + L) once.
     auto digits = [&](int hi, int lo, float w, float wm) {
-      return fmaf(128.f, fmaf(w, __int_as_float(hi), wm), fmaf(w, __int_as_float(lo), wm));
+      return fmaf(w, __int_as_float(lo), fmaf(128.f * w, __int_as_float(hi), 129.f * wm));
     };
     // Raw scores (integer units: multiply by kfac) of the 16 packed key rows r0 .. r0+15 of a chunk: this lane's rows
     // are r0 + gid and r0 + gid + 8.  kc / km: packed rows and metadata rows of the chunk (shared or global memory).
-    auto k_mtile = [&](const uint32_t* kc, const uint32_t* km, int r0, float& sA_out, float& sB_out) {
+    // decoded: std::true_type when km points to decoder parameters that the warp has already worked out for the whole
+    // chunk ((scale, zero-point) float pairs, see kShareKMeta below), std::false_type for the stored metadata words.
+    auto k_mtile = [&](auto decoded, const uint32_t* kc, const uint32_t* km, int r0, float& sA_out, float& sB_out) {
       const int rA = r0 + gid, rB = rA + 8;
       auto kmeta = [&](int row, int g, float& s_, float& z_) {      // decoder parameters of (row, group)
-        if constexpr (KM == 4) decode_fast(km[row * NG + g], neg_half, s_, z_);
+        if constexpr (decltype(decoded)::value) {
+          const float2 v = reinterpret_cast<const float2*>(km)[row * NG + g];
+          s_ = v.x; z_ = v.y;
+        } else if constexpr (KM == 4) decode_fast(km[row * NG + g], neg_half, s_, z_);
         else {
           s_ = h2f_bits(reinterpret_cast<const uint16_t*>(km)[row * NG + g] & 0x7FFFu);
           z_ = neg_half * s_;
@@ -424,14 +433,14 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           // the four positions carry different weights: one accumulator each, joined per group in fp32
           float tA[NG], tB[NG];
 #pragma unroll
-          for (int g = 0; g < NG; ++g) tA[g] = tB[g] = 0.f;
-#pragma unroll
           for (int p = 0; p < 4; ++p) {
             int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
             imma_us(c4, areg(p, 0), areg(p, 1), areg(p, 2), areg(p, 3), Bq[p][0], Bq[p][1]);
             const float w = pow2i(-(4 * (p >> 1) + (p & 1))), wm = -w * kMagicSf;
-            tA[(32 * p) / G] += digits(c4[0], c4[1], w, wm);
-            tB[(32 * p) / G] += digits(c4[2], c4[3], w, wm);
+            const float dA = digits(c4[0], c4[1], w, wm), dB = digits(c4[2], c4[3], w, wm);
+            constexpr int PG = G / 32;                      // bit positions per group
+            if (p % PG == 0) { tA[p / PG] = dA; tB[p / PG] = dB; }
+            else { tA[p / PG] += dA; tB[p / PG] += dB; }
           }
           sA = 0.f; sB = 0.f;
 #pragma unroll
@@ -620,7 +629,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
       if (skew) {
         const int iq = cn.n_qv + e0;                           // first packed key row of the tile (16-aligned)
         const unsigned char* rec = group_rec((iq / kChunk) / CH) + (size_t)((iq / kChunk) % CH) * SL::kRec;
-        k_mtile(reinterpret_cast<const uint32_t*>(rec), reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta),
+        k_mtile(std::false_type{}, reinterpret_cast<const uint32_t*>(rec), reinterpret_cast<const uint32_t*>(rec + SL::kOffKMeta),
                 iq % kChunk, sA, sB);
         sA *= kfac;
         sB *= kfac;
@@ -706,9 +715,14 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
     if (lane == 0 && atomicAdd(&s_past_tail, 1u) == kWarps - 1) grid_launch_dependents();
 
     constexpr bool kFreshEveryChunk = !SPLIT && CH == 1;      // a value group is one chunk: nothing is carried over
-    // 256 * hi + lo of a value accumulator pair (bit patterns of kMagicUf + sum), times the power of two w: exact
+    // see the raw scores below; measured: 2.4 % faster in a chain where an iteration holds two chunks of four groups per
+    // row (one exchange for 256 entries), 0-2 % SLOWER with one chunk per iteration (3- and 4-bit keys) or two groups
+    constexpr bool kShareKMeta = !SPLIT && NG == 4 && CPI == 2;
+    static_assert(!kShareKMeta || CPI * kChunk * NG * 8 <= SL::kSideBytes, "decoded key metadata of an iteration fit the side area");
+    // 256 * hi + lo of a value accumulator pair (bit patterns of kMagicUf + sum), times the power of two w: the inner
+    // product, 256 w H - w kMagicUf, is exact (a multiple of 256 w), the outer one rounds w (256 H + L) once
     auto vdigits = [&](int hi, int lo, float w) {
-      return fmaf(256.f, fmaf(w, __int_as_float(hi), -w * kMagicUf), fmaf(w, __int_as_float(lo), -w * kMagicUf));
+      return fmaf(w, __int_as_float(lo), fmaf(256.f * w, __int_as_float(hi), -257.f * w * kMagicUf));
     };
     // lanes this lane fetches its value-side B registers from: the lane that holds the probabilities of tokens
     // k = 4j .. 4j+3 (register 0) and 16 + 4j .. (register 1) for this column's head
@@ -726,6 +740,47 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
       const bool last_valid = CPI == 1 || (it * CPI + 1 < n_chunks_w);   // odd chunk count: the last half is empty
 
       // ---------------- raw scores: CPI * 2 m-tiles of 16 tokens -------------------------------------
+      // With several key groups per token and several heads per pass, the four lanes of a quad need the decoder
+      // parameters of the same (row, group) entries: lane = row decodes its row's NG entries once, the warp exchanges
+      // them through its side area (free between the value groups' ends), each lane reads its two rows per m-tile.
+      if constexpr (kShareKMeta && !(ABL & 1)) {
+#pragma unroll
+        for (int cc = 0; cc < CPI; ++cc) {
+          if (cc > 0 && !last_valid) continue;
+          const unsigned char* kmb = sp + SL::off(cc) + SL::kOffKMeta + lane * (NG * KM);
+          float* dst = reinterpret_cast<float*>(side) + cc * (kChunk * NG * 2) + lane * (NG * 2);
+          float sz[2 * NG];
+          if constexpr (KM == 4) {
+            uint32_t mw[NG];
+            if constexpr (NG == 4) {
+              const uint4 t = *reinterpret_cast<const uint4*>(kmb);
+              mw[0] = t.x; mw[1] = t.y; mw[2] = t.z; mw[3] = t.w;
+            } else {
+              const uint2 t = *reinterpret_cast<const uint2*>(kmb);
+              mw[0] = t.x; mw[1] = t.y;
+            }
+#pragma unroll
+            for (int g = 0; g < NG; ++g) decode_fast(mw[g], neg_half, sz[2 * g], sz[2 * g + 1]);
+          } else {
+            uint32_t hw[NG / 2];
+            if constexpr (NG == 4) {
+              const uint2 t = *reinterpret_cast<const uint2*>(kmb);
+              hw[0] = t.x; hw[1] = t.y;
+            } else {
+              hw[0] = *reinterpret_cast<const uint32_t*>(kmb);
+            }
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+              sz[2 * g] = h2f_bits((hw[g >> 1] >> (16 * (g & 1))) & 0x7FFFu);
+              sz[2 * g + 1] = neg_half * sz[2 * g];
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < NG; g += 2)
+            *reinterpret_cast<float4*>(dst + 2 * g) = make_float4(sz[2 * g], sz[2 * g + 1], sz[2 * g + 2], sz[2 * g + 3]);
+        }
+        __syncwarp();
+      }
       float sc[CPI][2][2];
 #pragma unroll
       for (int cc = 0; cc < CPI; ++cc) {
@@ -738,9 +793,12 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           if constexpr (ABL & 1) sc[cc][mt][0] = sc[cc][mt][1] = 0.f;      // timing experiment: no key side
-          else k_mtile(kc, km, 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
+          else if constexpr (kShareKMeta)
+            k_mtile(std::true_type{}, kc, side + cc * (kChunk * NG * 2), 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
+          else k_mtile(std::false_type{}, kc, km, 16 * mt, sc[cc][mt][0], sc[cc][mt][1]);
         }
       }
+      if constexpr (kShareKMeta && !(ABL & 1)) __syncwarp();      // the side area goes back to the value groups' ends
 
       // ---------------- online softmax (log2 domain; raw scores are in integer units: times kfac) -----
       // The reference m_run of the running sums is an INTEGER that no score so far exceeds (the ceiling of the
