@@ -390,6 +390,25 @@ class Legs:
         self.torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / n
 
+    def small_launches(self, nbytes, peak, n_steps=96):
+        """The same legs with one CTA per SM and launch (148 / units splits per unit instead of one wave of two CTAs
+        per SM): consecutive launches then share the GPU, which hides each launch's start and end behind its
+        neighbours' streaming (higher step rate) and makes a launch that runs alone slower (half the warps per SM).
+        The library's default stays the latency-optimal split; `innerq_set_decode_options` selects this one."""
+        sp = max(1, 148 // self.w.n_units)
+        for c in self.caches:
+            c.innerq_set_decode_options(sp, 0)
+        try:
+            step, _ = self.steps(n_steps, warm=16)
+            chain = self.decodes_chained(64)
+            alone = float(np.median(self.decodes_bracketed(16)))
+        finally:
+            for c in self.caches:
+                c.innerq_set_decode_options(0, 0)
+        gbs = lambda us: nbytes / us / 1e3
+        return {"n_splits": sp, "us_per_step": step, "us_per_decode_back_to_back": chain, "us_per_decode_alone_median": alone,
+                "frac_of_measured_peak": {"step": gbs(step) / peak, "chained": gbs(chain) / peak, "alone_median": gbs(alone) / peak}}
+
     def sides(self, n=64):
         """us per decode in a chain for the full fused kernel, without its key-side arithmetic and without its
         value-side arithmetic (decode options 6 / 7: timing only, all bytes still streamed); None if the cache's format
@@ -479,7 +498,7 @@ def measure_config(name, peak, R=2, n_steps=128):
     import torch
     from paper_2602_23200_b200 import binding as B
     w = workload_by_name(name)
-    n_in = 32 + n_steps + 8
+    n_in = 32 + n_steps + 8 + 16 + 96
     cfg = B.make_config(w, max_tokens=w.n_tokens + n_in // R + 16)
     Kd, Vd = kv_device(w, tiled=True)
     caches = []
@@ -514,8 +533,10 @@ def measure_config(name, peak, R=2, n_steps=128):
     chain = legs.decodes_chained(64)
     step, step_host = legs.steps(n_steps, warm=32)
     sides = legs.sides()
+    small = legs.small_launches(nbytes, peak)
     gbs = lambda us: nbytes / us / 1e3
     res.update({
+        "one_cta_per_sm_launches": small,
         "bytes_per_decode_minimal": nbytes, "sym_group_fraction": {"k": sym_k, "v": sym_v},
         "us_per_decode_alone": alone, "us_per_decode_chained": chain, "us_per_step": step,
         "host_us_per_step_enqueue": step_host, "us_per_decode_chained_by_side": sides,
@@ -550,7 +571,7 @@ def run_ours(args, w):
     LEG = args.leg_steps            # the step-rate leg that does not depend on --steps
     e2e_steps = max(4, min(Kst, 32))
     split_steps = 2 * R * w.group if packed else 0           # steps timed one by one (below)
-    n_in = W + WARM + Kst + 32 + LEG + e2e_steps + split_steps + 16
+    n_in = W + WARM + Kst + 32 + LEG + e2e_steps + split_steps + 16 + 16 + 96
     cfg = B.make_config(w, max_tokens=w.n_tokens + n_in // R + 16)
     Kd, Vd = kv_device(w, tiled=False)
     caches = []
@@ -703,6 +724,7 @@ def run_ours(args, w):
         for c in literal_caches:
             c.close()
     sides = legs.sides() if packed and not (args.splits or args.variant) else None
+    small = legs.small_launches(bytes_min, measured_peak_gbs()[0]) if packed and not (args.splits or args.variant) else None
     append_us = float(np.median(legs.appends_bracketed(16)))
     multi = None
     if args.n_q > 1 and packed:
@@ -760,7 +782,7 @@ def run_ours(args, w):
                      "untimed_steps_before_the_timed_region": W + WARM},
             "paper_literal_sym_variant": literal,
             "second_roof": pipe_roofs_gbs(counters, bytes_min, clocks.get("sm_mhz")),
-            "step_us_by_kind": step_split, "multi_query": multi, "ragged_batch": ragged, "paged_cache": paged,
+            "step_us_by_kind": step_split, "one_cta_per_sm_launches": small, "multi_query": multi, "ragged_batch": ragged, "paged_cache": paged,
             "pct_of_nominal_8TBs": {"decode_alone_median": achieved / 80.0, "decode_back_to_back": gbs(b2b_us) / 80.0,
                                     "step": value_gbs / world / 80.0},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -231,16 +231,14 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
   };
   // What the step's append writes for this unit (rings, newest packed rows) is complete when the unit's counter in
   // the cache buffer holds this decode's N: the append publishes it (release) after its last write, long before the
-  // append kernel ends (one of its CTAs stays until the previous decode has ended).  A warp looks once (acquire): if
-  // the count is there it goes on at once, while the append's other units and the previous decode's merge may still
-  // be running; if not (the append is still at work on this unit), it waits for its predecessor's completion, which
-  // is always right and wakes up faster than any polling would.
+  // append kernel ends (one of its CTAs stays until the previous decode has ended).  A warp looks for a bounded time
+  // (acquire; see append_count_is): when the count is there it goes on, while the append's other units and the
+  // previous decode may still be running; if it never shows, it waits for its predecessor's completion, which is
+  // always right.
   auto wait_for_append = [&]() {
     if (dep_waited) return;
     const uint32_t* flag = reinterpret_cast<const uint32_t*>(a.cache + L.appended_off) + u;
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    if (!__all_sync(0xffffffffu, v == (uint32_t)cn.N)) dep_wait();
+    if (!append_count_is(flag, (uint32_t)cn.N)) dep_wait();
     // what was acquired is ordered ahead of bulk async copies too (this kernel's later ones, and through
     // launch_dependents the next kernel's, which stream the rows that append packed)
     asm volatile("fence.proxy.async.global;" ::: "memory");

@@ -170,6 +170,26 @@ template <int KB, int VB, int G, int KM, int VM, int CPI> struct StageLayout {
 };
 
 
+// True when the unit's append counter (see Layout::appended_off) holds N, looked at up to kAppendPolls times about
+// 0.2 us apart (whole warp, same answer in every lane).  The append that writes it precedes this kernel in the
+// stream and lets its dependents start only once all of its CTAs are running, so it makes progress whatever this
+// kernel does, and it publishes the counter long before it ends (its last CTA stays until the previous decode has
+// ended).  A caller that gets false waits for its predecessor's completion instead, which is always right; looking
+// only once sent most warps down that road and tied this decode's tail tiles to the END of the previous decode, which
+// costs nothing with one wave of CTAs per launch and most of the overlap when launches are small enough to share
+// the GPU (config 2 at four splits per unit: 28.1 us per step, 17.5 us with the bounded look).
+constexpr int kAppendPolls = 48;
+__device__ __forceinline__ bool append_count_is(const uint32_t* flag, uint32_t N) {
+  bool there = false;
+  for (int tries = 0; tries < kAppendPolls && !there; ++tries) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    there = __all_sync(0xffffffffu, v == N);
+    if (!there) __nanosleep(200);
+  }
+  return there;
+}
+
 // Cross-CTA merge, run by the last CTA of a unit to finish: log-sum-exp combination of the n_parts partial results
 // (rows prow0 .. of kPartialStride floats: acc[128], max, sum) of nh query rows, fp16 results to rows orow of out.
 // Kept out of line so that its registers do not add to the streaming loop's.
@@ -431,16 +451,14 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
   };
   // What the step's append writes for this unit (rings, newest packed rows) is complete when the unit's counter in
   // the cache buffer holds this decode's N: the append publishes it (release) after its last write, long before the
-  // append kernel ends (one of its CTAs stays until the previous decode has ended).  A warp looks once (acquire): if
-  // the count is there it goes on at once, while the append's other units and the previous decode's merge may still
-  // be running; if not (the append is still at work on this unit), it waits for its predecessor's completion, which
-  // is always right and wakes up faster than any polling would.
+  // append kernel ends (one of its CTAs stays until the previous decode has ended).  A warp looks for a bounded time
+  // (acquire; see append_count_is): when the count is there it goes on, while the append's other units and the
+  // previous decode may still be running; if it never shows, it waits for its predecessor's completion, which is
+  // always right.
   auto wait_for_append = [&]() {
     if (dep_waited) return;
     const uint32_t* flag = reinterpret_cast<const uint32_t*>(a.cache + L.appended_off) + u;
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    if (!__all_sync(0xffffffffu, v == (uint32_t)cn.N)) dep_wait();
+    if (!append_count_is(flag, (uint32_t)cn.N)) dep_wait();
     // what was acquired is ordered ahead of bulk async copies too (this kernel's later ones, and through
     // launch_dependents the next kernel's, which stream the rows that append packed)
     asm volatile("fence.proxy.async.global;" ::: "memory");
