@@ -287,7 +287,10 @@ int innerq_cache_export(innerq_cache_t* cache, innerq_export_t* ex, void* cuda_s
 int innerq_cache_import(innerq_cache_t* cache, const innerq_export_t* ex, int32_t n_tokens, void* cuda_stream);
 
 /* Tuning knobs for experiments; both default to 0 = automatic.
- *   n_splits : number of token ranges each unit is split into by the decode kernel.
+ *   n_splits : number of token ranges each unit is split into by the decode kernel.  0 = automatic: one wave of two
+ *              CTAs per SM, the lowest latency for a launch that runs alone.  148 / (batch * n_kv_heads), i.e. one
+ *              CTA per SM and launch, lets consecutive launches share the GPU and hide each other's start and end:
+ *              10-15 % more steps per second in a loop of back-to-back calls, 10-25 % slower for a launch alone.
  *   variant  : 0 automatic, 1 plain SIMT kernel, 2 warp-MMA kernel (where supported; UNSUPPORTED otherwise),
  *              3 / 4 warp-MMA kernel with one / two 32-token chunks per loop iteration (sets a process-wide knob).
  *              6 / 7 TIMING ONLY, the output is wrong on purpose: the warp-MMA kernel with the unpack + MMA work of

@@ -1454,48 +1454,11 @@ int launch_one_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, c
                            : launch_one_batched_p<KB, VB, G, KM, VM, SPLIT, CPI, OUTER, false>(L, T, n_seqs, n_splits, st);
 }
 
-// One packed format (key bits, value bits, metadata entry bytes of each) at every group size.  cpi: chunks of 32
-// tokens per loop iteration, 0 = automatic.  Two per iteration need twice the stage bytes, which only the
-// 2-bit/2-bit formats can afford with two resident CTAs per SM.
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT>
-int launch_cpi(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
-  if constexpr (KB == 2 && VB == 2) {
-    if (cpi != 1) return launch_one<KB, VB, G, KM, VM, SPLIT, 2>(L, cn, a, n_splits, st);
-  }
-  return launch_one<KB, VB, G, KM, VM, SPLIT, 1>(L, cn, a, n_splits, st);
-}
-
-template <int KB, int VB, int G, int KM, int VM, bool SPLIT>
-int launch_cpi_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
-  if constexpr (KB == 2 && VB == 2) {
-    if (cpi != 1) return launch_one_batched<KB, VB, G, KM, VM, SPLIT, 2>(L, T, n_seqs, n_splits, st);
-  }
-  return launch_one_batched<KB, VB, G, KM, VM, SPLIT, 1>(L, T, n_seqs, n_splits, st);
-}
-
-template <int KB, int VB, int KM, int VM>
-int launch_format_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1) return launch_cpi_batched<KB, VB, 32, KM, VM, true>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 32) return launch_cpi_batched<KB, VB, 32, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 64) return launch_cpi_batched<KB, VB, 64, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  if (L.G == 128) return launch_cpi_batched<KB, VB, 128, KM, VM, false>(L, T, n_seqs, n_splits, cpi, st);
-  return -2;
-}
-
 template <int KB, int VB>
 int launch_format_outer_batched(const Layout& L, SeqTable& T, int n_seqs, int n_splits, cudaStream_t st) {
   if (L.G == 32) return launch_one_batched<KB, VB, 32, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
   if (L.G == 64) return launch_one_batched<KB, VB, 64, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
   if (L.G == 128) return launch_one_batched<KB, VB, 128, 4, 4, false, 1, true>(L, T, n_seqs, n_splits, st);
-  return -2;
-}
-
-template <int KB, int VB, int KM, int VM>
-int launch_format(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, int cpi, cudaStream_t st) {
-  if (L.G == 32 && L.r == 1 && a.n_q == 1) return launch_cpi<KB, VB, 32, KM, VM, true>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 32) return launch_cpi<KB, VB, 32, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 64) return launch_cpi<KB, VB, 64, KM, VM, false>(L, cn, a, n_splits, cpi, st);
-  if (L.G == 128) return launch_cpi<KB, VB, 128, KM, VM, false>(L, cn, a, n_splits, cpi, st);
   return -2;
 }
 
@@ -1510,19 +1473,10 @@ int launch_format_outer(const Layout& L, const Counts& cn, const DecodeArgs& a, 
 
 }  // namespace
 
-// Defines the externally visible launcher of one format in the translation unit that compiles its kernels.
+// Names of the externally visible launchers of one inner-grouped format (defined by the integer-operand kernel's
+// translation units), and the definition of the outer-grouped ones in the translation unit that compiles their kernels.
 #define IQ_MMA_FORMAT_NAME(KB, VB, KM, VM) launch_decode_mma_k##KB##v##VB##_m##KM##VM
 #define IQ_MMA_FORMAT_NAME_BATCHED(KB, VB, KM, VM) launch_decode_mma_k##KB##v##VB##_m##KM##VM##_batched
-#define IQ_DEFINE_MMA_FORMAT(KB, VB, KM, VM)                                                                  \
-  int IQ_MMA_FORMAT_NAME(KB, VB, KM, VM)(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits, \
-                                         int cpi, cudaStream_t st) {                                            \
-    return launch_format<KB, VB, KM, VM>(L, cn, a, n_splits, cpi, st);                                          \
-  }                                                                                                             \
-  int IQ_MMA_FORMAT_NAME_BATCHED(KB, VB, KM, VM)(const Layout& L, SeqTable& T, int n_seqs, int n_splits, int cpi,  \
-                                                    cudaStream_t st) {                                           \
-    return launch_format_batched<KB, VB, KM, VM>(L, T, n_seqs, n_splits, cpi, st);                               \
-  }
-
 #define IQ_DEFINE_MMA_OUTER_FORMAT(KB, VB)                                                                          \
   int launch_decode_mma_outer_k##KB##v##VB(const Layout& L, const Counts& cn, const DecodeArgs& a, int n_splits,    \
                                            int, cudaStream_t st) {                                                   \
