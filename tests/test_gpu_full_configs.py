@@ -117,7 +117,10 @@ def test_config2_prefill_then_steps():
     print(f"config2, generic kernel: err/tol {e1:.3f}")
 
 
-def test_config2_inputs_written_by_the_kernel_right_before_each_call():
+@pytest.mark.parametrize("splits", [0, 4])
+def test_config2_inputs_written_by_the_kernel_right_before_each_call(splits):
+    # splits = 4: one CTA per SM and launch, so that two or three consecutive decodes are resident at the same time
+    # (the operating point bench.py reports as one_cta_per_sm_launches); 0: the default, one wave per launch.
     # The way a model uses the library: q, k_new and v_new of every step are produced on the same stream by an
     # ordinary kernel (here an elementwise op into three buffers that are REUSED by every step) immediately before
     # innerq_append_token / innerq_decode_attention, which are launched as programmatic dependents and read their
@@ -129,6 +132,7 @@ def test_config2_inputs_written_by_the_kernel_right_before_each_call():
     units = [7, 24]
     n_steps = 120
     gc, oc = make_gpu(w, K, V, extra=n_steps + 8), sub_oracle(w, K, V, units, extra=n_steps + 8)
+    gc.innerq_set_decode_options(splits, 0)
     del K, V
     toks = [synth.new_token(w, 500 + s) for s in range(n_steps)]
     qs = [synth.query(w, 500 + s) for s in range(n_steps)]
