@@ -310,6 +310,13 @@ int innerq_set_decode_options(innerq_cache_t* cache, int32_t n_splits, int32_t v
  * current device) or a negative error code. */
 int innerq_read_device_error(innerq_cache_t* cache, void* cuda_stream);
 
+/* Test support for the call above: enqueues a one-warp kernel that waits, with the decode kernels' own bounded
+ * wait (256 polls), on a barrier on which nothing ever arrives, gives up, and records that in the cache's device
+ * error word exactly as a decode warp would; the kernel returns normally and the context stays usable.  After it
+ * innerq_read_device_error returns 1 for this cache for good (the word is never cleared), so use a cache made for
+ * the test.  Does not synchronise.  Errors: INVALID_ARG, CUDA. */
+int innerq_selftest_wait_expiry(innerq_cache_t* cache, void* cuda_stream);
+
 /* Number of kernels the last call of each kind launched (for launch accounting):
  * which = 0 prefill, 1 append, 2 decode.  Returns the count or a negative error code. */
 int innerq_last_launch_count(const innerq_cache_t* cache, int32_t which);

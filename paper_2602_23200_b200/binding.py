@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "innerq_paged_cache_bytes", "innerq_cache_create_paged", "innerq_cache_pages_for", "innerq_cache_pages_assigned",
     "innerq_cache_assign_pages", "innerq_cache_release_pages",
     "innerq_cache_export", "innerq_cache_import", "innerq_set_decode_options", "innerq_last_launch_count", "innerq_read_device_error",
-    "innerq_status_string",
+    "innerq_selftest_wait_expiry", "innerq_status_string",
 )
 
 
@@ -91,6 +91,7 @@ def lib() -> C.CDLL:
     L.innerq_set_decode_options.argtypes = [vp, i32, i32]
     L.innerq_last_launch_count.argtypes = [vp, i32]
     L.innerq_read_device_error.argtypes = [vp, vp]
+    L.innerq_selftest_wait_expiry.argtypes = [vp, vp]
     L.innerq_status_string.argtypes = [C.c_int]
     L.innerq_status_string.restype = C.c_char_p
     for name in EXPORTED_SYMBOLS:
@@ -400,6 +401,9 @@ class InnerQCache:
 
     def innerq_read_device_error(self, stream=None) -> int:
         return _check(lib().innerq_read_device_error(self._h, _stream_ptr(stream, self.device)), "innerq_read_device_error")
+
+    def innerq_selftest_wait_expiry(self, stream=None):
+        _check(lib().innerq_selftest_wait_expiry(self._h, _stream_ptr(stream, self.device)), "innerq_selftest_wait_expiry")
 
     def innerq_last_launch_count(self, which: int) -> int:
         return _check(lib().innerq_last_launch_count(self._h, which), "innerq_last_launch_count")

@@ -698,6 +698,11 @@ int innerq_set_decode_options(innerq_cache_t* c, int32_t n_splits, int32_t varia
   return INNERQ_OK;
 }
 
+int innerq_selftest_wait_expiry(innerq_cache_t* c, void* cuda_stream) {
+  if (!c) return INNERQ_ERR_INVALID_ARG;
+  return launch_wait_expiry_selftest(c->L, c->ws, static_cast<cudaStream_t>(cuda_stream)) < 0 ? INNERQ_ERR_CUDA : INNERQ_OK;
+}
+
 int innerq_read_device_error(innerq_cache_t* c, void* cuda_stream) {
   if (!c) return INNERQ_ERR_INVALID_ARG;
   unsigned int flag = 0;

@@ -61,6 +61,8 @@ bool decode_mma_supported(const Layout& L);
 // Warp-MMA decode over an unquantised fp16 cache (grouping = FP16).  Returns -2 for other layouts.
 int launch_decode_fp16(const Layout& L, const unsigned char* cache, unsigned char* ws, int N, const __half* q,
                        __half* out, int n_splits, cudaStream_t st);
+// Test support: a one-warp kernel whose bounded wait runs out and sets the workspace's error word.
+int launch_wait_expiry_selftest(const Layout& L, unsigned char* ws, cudaStream_t st);
 void decode_mma_set_chunks_per_iter(int n);   // tuning: 32-token chunks per loop iteration (1 or 2)
 void decode_mma_set_ablation(int mask);       // timing experiments: bit 0 / 1 = no key-side / value-side work in the loop
 

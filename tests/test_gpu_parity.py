@@ -175,6 +175,24 @@ def test_fused_kernel_formats(kb, vb, km, vm, G, r, N):
     P.assert_export_equal(gc.innerq_cache_export(), oc.export(), O.INNER, G, km == O.HYBRID, vm == O.HYBRID)
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    # The decode kernels wait for their asynchronous copies a bounded number of times and, if a wait runs out, set
+    # the cache's device error word and return.  The self-test kernel takes that road on purpose: the kernels' own
+    # wait routine, on a barrier nothing ever arrives on.  No fault, no hang: the kernel gives up after 256 polls.
+    w = synth.tiny(n_tokens=300)
+    oc, gc, _, _ = run_prefill_both(w)
+    check_decode(w, oc, gc)                                   # error word still 0 (asserted there)
+    gc.innerq_selftest_wait_expiry()
+    assert gc.innerq_read_device_error() == 1                 # the expiry is reported ...
+    assert gc.innerq_read_device_error() == 1                 # ... for good: the word is sticky
+    q = synth.query(w, 3)
+    out = gc.innerq_decode_attention(dev(q)).cpu().numpy()    # ... and the context and the cache still work
+    P.assert_outputs_close(out, oc.decode(q), "after a wait that ran out")
+    # another cache has its own error word
+    _, g2, _, _ = run_prefill_both(w)
+    assert g2.innerq_read_device_error() == 0
+
+
 @pytest.mark.parametrize("N", [1, 3, 4, 5, 19, 20, 21, 52, 53])
 def test_short_contexts_and_window_edges(N):
     # N <= w_sink, N <= w_sink + w_recent (nothing quantised), first quantised key token, first value group
