@@ -38,6 +38,12 @@ __device__ __forceinline__ void imma_uu(int (&c)[4], uint32_t a0, uint32_t a1, u
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // the same with a constant accumulator input (every element = c0): no registers to set up for a fresh sum
+__device__ __forceinline__ void imma_us_init(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1, int c0) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c0));
+}
 __device__ __forceinline__ void imma_uu_init(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                              uint32_t b1, int c0) {
   asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
@@ -416,9 +422,12 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           return (p & 1) ? (wo[r] & (0x0E0E0E0Eu << (4 * (p >> 1)))) : (we[r] & (0x07070707u << (4 * (p >> 1))));
         };
         if constexpr (SPLIT) {
-          int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+          int c4[4];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) imma_us(c4, areg(g, 0), areg(g, 1), areg(g, 2), areg(g, 3), Bq[g][0], Bq[g][1]);
+          for (int g = 0; g < 4; ++g) {
+            if (g == 0) imma_us_init(c4, areg(g, 0), areg(g, 1), areg(g, 2), areg(g, 3), Bq[g][0], Bq[g][1], kMagicS);
+            else imma_us(c4, areg(g, 0), areg(g, 1), areg(g, 2), areg(g, 3), Bq[g][0], Bq[g][1]);
+          }
           kmeta(rA, j, s_, z_);
           sA = fmaf(s_, digits(c4[0], c4[1], wj, wjm), z_ * Qg[0]);
           kmeta(rB, j, s_, z_);
@@ -432,8 +441,8 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           float tA[NG], tB[NG];
 #pragma unroll
           for (int p = 0; p < 4; ++p) {
-            int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
-            imma_us(c4, areg(p, 0), areg(p, 1), areg(p, 2), areg(p, 3), Bq[p][0], Bq[p][1]);
+            int c4[4];
+            imma_us_init(c4, areg(p, 0), areg(p, 1), areg(p, 2), areg(p, 3), Bq[p][0], Bq[p][1], kMagicS);
             const float w = pow2i(-(4 * (p >> 1) + (p & 1))), wm = -w * kMagicSf;
             const float dA = digits(c4[0], c4[1], w, wm), dB = digits(c4[2], c4[3], w, wm);
             constexpr int PG = G / 32;                      // bit positions per group
@@ -454,11 +463,12 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
       const uint2 xb = *reinterpret_cast<const uint2*>(kc + rB * RW + 2 * j);
       if constexpr (SPLIT) {
         // column pair g carries q'' of group g only, so one accumulator chain leaves group j's sums with lane j
-        int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+        int c4[4];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const uint32_t mk = 0x03030303u << (2 * g);
-          imma_us(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[g][0], Bq[g][1]);
+          if (g == 0) imma_us_init(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[g][0], Bq[g][1], kMagicS);
+          else imma_us(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[g][0], Bq[g][1]);
         }
         kmeta(rA, j, s_, z_);
         sA = fmaf(s_, digits(c4[0], c4[1], wj, wjm), z_ * Qg[0]);
@@ -472,9 +482,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         sA = 0.f; sB = 0.f;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {                 // bit position g = group g: its own accumulator
-          int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+          int c4[4];
           const uint32_t mk = 0x03030303u << (2 * g);
-          imma_us(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[g][0], Bq[g][1]);
+          imma_us_init(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[g][0], Bq[g][1], kMagicS);
           const float w = pow2i(-2 * g), wm = -w * kMagicSf;
           kmeta(rA, g, s_, z_);
           sA = fmaf(s_, digits(c4[0], c4[1], w, wm), fmaf(z_, Qg[g], sA));
@@ -488,9 +498,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         float tA[2], tB[2];
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+          int c4[4];
           const uint32_t mk = 0x03030303u << (4 * c);
-          imma_us(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[2 * c][0], Bq[2 * c][1]);
+          imma_us_init(c4, xa.x & mk, xb.x & mk, xa.y & mk, xb.y & mk, Bq[2 * c][0], Bq[2 * c][1], kMagicS);
           imma_us(c4, ya0 & mk, yb0 & mk, ya1 & mk, yb1 & mk, Bq[2 * c + 1][0], Bq[2 * c + 1][1]);
           const float w = pow2i(-4 * c), wm = -w * kMagicSf;
           tA[c] = digits(c4[0], c4[1], w, wm);
@@ -523,10 +533,12 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             int (&c4)[4] = cs[SPLIT ? 0 : g];
-            if (!SPLIT || g == 0) { c4[0] = c4[1] = c4[2] = c4[3] = kMagicS; }
             const uint32_t mk = (g & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
             const int h2 = g >> 1;
-            imma_us(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[g][0], Bq[g][1]);
+            if (!SPLIT || g == 0)
+              imma_us_init(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[g][0], Bq[g][1], kMagicS);
+            else
+              imma_us(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[g][0], Bq[g][1]);
           }
           if constexpr (SPLIT) {
             kmeta(rA, j, s_, z_);
@@ -554,9 +566,9 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
           float tA[2], tB[2];
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
-            int c4[4] = {kMagicS, kMagicS, kMagicS, kMagicS};
+            int c4[4];
             const uint32_t mk = 0x0F0F0F0Fu;
-            imma_us(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[2 * h2][0], Bq[2 * h2][1]);
+            imma_us_init(c4, xa[2 * h2] & mk, xb[2 * h2] & mk, xa[2 * h2 + 1] & mk, xb[2 * h2 + 1] & mk, Bq[2 * h2][0], Bq[2 * h2][1], kMagicS);
             imma_us(c4, (xa[2 * h2] >> 4) & mk, (xb[2 * h2] >> 4) & mk, (xa[2 * h2 + 1] >> 4) & mk, (xb[2 * h2 + 1] >> 4) & mk,
                     Bq[2 * h2 + 1][0], Bq[2 * h2 + 1][1]);
             tA[h2] = digits(c4[0], c4[1], 1.0f, -kMagicSf);
@@ -713,6 +725,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
     if (lane == 0 && atomicAdd(&s_past_tail, 1u) == kWarps - 1) grid_launch_dependents();
 
     constexpr bool kFreshEveryChunk = !SPLIT && CH == 1;      // a value group is one chunk: nothing is carried over
+    constexpr bool kStaticSlots = !SPLIT && CH == CPI && CH > 1;   // a value group is one iteration (G = 64, two chunks)
     // see the raw scores below; measured: 2.4 % faster in a chain where an iteration holds two chunks of four groups per
     // row (one exchange for 256 entries), 0-2 % SLOWER with one chunk per iteration (3- and 4-bit keys) or two groups
     constexpr bool kShareKMeta = !SPLIT && NG == 4 && CPI == 2;
@@ -817,7 +830,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         psum *= alpha;
 #pragma unroll
         for (int m = 0; m < 8; ++m) { out_acc[m][0] *= alpha; out_acc[m][1] *= alpha; }
-        if constexpr (!kFreshEveryChunk) {
+        if constexpr (!kFreshEveryChunk && !kStaticSlots) {      // (else no value group is open between iterations)
           // sums of the open value group: (256 hi + lo) >> k, the bits that leave hi carried into lo (they weigh 256)
           const int k = m_run == -INFINITY ? 23 : min(23, (int)(m_new - m_run));
           const int keep = k < 23 ? -1 : 0, low = (1 << k) - 1;
@@ -840,11 +853,14 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
         const uint32_t* vc = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kOffVCodes);
         const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + SL::off(cc) + SL::kRec);
         // slot: position of this chunk's value group in the SPLIT window / position of the chunk in its group
-        const int slot = SPLIT ? (ci - c_lo) & (WIN - 1) : ci % CH;
+        // (kStaticSlots: an iteration is exactly one value group, so the position is the chunk's index in the iteration)
+        const int slot = SPLIT ? (ci - c_lo) & (WIN - 1) : (kStaticSlots ? cc : ci % CH);
         const bool group_start = slot == 0;
+        // the first MMA of a sum takes the constant as its accumulator input instead of registers set up for it
+        const bool init_here = kFreshEveryChunk || (kStaticSlots && cc == 0);
         const bool group_end = SPLIT ? (slot == WIN - 1 || (it == n_iters - 1 && (cc == CPI - 1 || !last_valid)))
                                      : (slot == CH - 1);
-        if (!kFreshEveryChunk && group_start) {
+        if (!kFreshEveryChunk && !kStaticSlots && group_start) {
 #pragma unroll
           for (int m = 0; m < 8; ++m)
 #pragma unroll
@@ -895,7 +911,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
             for (int pos = 0; pos < 4; ++pos) {
               const uint32_t mk = (pos & 1) ? (0x0E0E0E0Eu << (4 * (pos >> 1))) : (0x07070707u << (4 * (pos >> 1)));
               const uint32_t* src = (pos & 1) ? wo : we;
-              if constexpr (kFreshEveryChunk)
+              if (init_here)
                 imma_uu_init(accg[4 * W + pos], src[0] & mk, src[1] & mk, src[2] & mk, src[3] & mk, b0, b1, kMagicU);
               else
                 imma_uu(accg[4 * W + pos], src[0] & mk, src[1] & mk, src[2] & mk, src[3] & mk, b0, b1);
@@ -909,7 +925,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
             for (int pos = 0; pos < 2; ++pos) {
               const uint32_t mk = pos ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
-              if constexpr (kFreshEveryChunk)
+              if (init_here)
                 imma_uu_init(accg[2 * W + pos], v.x & mk, v.y & mk, v.z & mk, v.w & mk, b0, b1, kMagicU);
               else
                 imma_uu(accg[2 * W + pos], v.x & mk, v.y & mk, v.z & mk, v.w & mk, b0, b1);
@@ -924,7 +940,7 @@ __device__ __forceinline__ void decode_i8_body(const Layout& L, const Counts& cn
 #pragma unroll
             for (int pos = 0; pos < 4; ++pos) {
               const uint32_t mk = 0x03030303u << (2 * pos);
-              if constexpr (kFreshEveryChunk)
+              if (init_here)
                 imma_uu_init(accg[4 * W + pos], vw[4 * W] & mk, vw[4 * W + 1] & mk, vw[4 * W + 2] & mk, vw[4 * W + 3] & mk,
                              b0, b1, kMagicU);
               else
