@@ -470,14 +470,18 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
   };
   // q and the key norms are requested first of all, ahead of the bulk copies below: behind several
   // hundred KB of queued chunk data per SM they would take microseconds to arrive.
-  float q_early[2], n_early[2];
+  // Only requested here: nothing may USE the loaded values before the copies below are issued (a warp issues in
+  // order, so a conversion or a select on them would hold the copies back until q has arrived from memory).
+  unsigned short q_bits[2];
+  float n_raw[2];
   {
     const float* norm_g = reinterpret_cast<const float*>(a.cache + L.norm_off) + (size_t)u * kD;
+    const unsigned short* q16 = reinterpret_cast<const unsigned short*>(a.q);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int i = tid + e * kThreads, h = i >> 7, c = i & (kD - 1);
-      q_early[e] = h < nh ? __half2float(a.q[(size_t)q_row(h) * kD + c]) : 0.f;
-      n_early[e] = L.k_normalize ? norm_g[c] : 1.0f;
+      q_bits[e] = q16[(size_t)q_row(h < nh ? h : 0) * kD + c];
+      n_raw[e] = norm_g[c];
     }
   }
 #pragma unroll
@@ -486,6 +490,13 @@ __device__ __forceinline__ void decode_mma_body(const Layout& L, const Counts& c
       dep_wait_for_iteration(s);
       if (lane == 0) issue(s);
     }
+  float q_early[2], n_early[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int h = (tid + e * kThreads) >> 7;
+    q_early[e] = h < nh ? __half2float(__ushort_as_half(q_bits[e])) : 0.f;
+    n_early[e] = L.k_normalize ? n_raw[e] : 1.0f;
+  }
 
   __shared__ unsigned int s_past_tail;      // warps of this CTA that are past their tail tiles (see the main loop's head)
   if (tid == 0) s_past_tail = 0u;           // ordered before its first use by the barriers of the prologue
