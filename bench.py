@@ -45,10 +45,17 @@ D = 128
 
 def workload_by_name(name: str):
     """c1 .. c4 (c3_4bit / c3_2bit), c5_b<bits>_g<group>_<hybrid|asym|sym|literal> (sweep on the config-3 shape);
-    a suffix "+fp16" or "+outer" selects the comparison cache of the same shape."""
+    a suffix "+fp16" or "+outer" selects the comparison cache of the same shape, "+k<K>v<V>" (e.g. c2+k3v3) other
+    code widths and "+k<K>v<V>sym" those widths in all-symmetric mode (the paper's Base preset is +k3v3sym)."""
     if "+" in name:
         base, variant = name.split("+", 1)
         w = workload_by_name(base)
+        if len(variant) in (4, 7) and variant[0] == "k" and variant[2] == "v" and variant[1] in "234" and variant[3] in "234" \
+                and variant[4:] in ("", "sym"):
+            kw = dict(name=w.name + "+" + variant, k_bits=int(variant[1]), v_bits=int(variant[3]))
+            if variant[4:] == "sym":
+                kw.update(k_mode=synth.SYM, v_mode=synth.SYM)
+            return w.with_(**kw)
         if variant == "fp16":
             return w.with_(name=w.name + "+fp16", grouping=synth.FP16, k_normalize=0)
         if variant == "outer":

@@ -87,6 +87,13 @@ def test_sweep_workload_names_and_prefill_bytes():
     assert w.grouping == synth.OUTER and w.k_normalize == 0 and w.group == 32
     with pytest.raises(SystemExit):
         bench.workload_by_name("c5_b2_g64_nonsense")
+    # other code widths on a named shape: the paper's presets on the 32-head shape
+    w = bench.workload_by_name("c2+k3v2")
+    assert (w.k_bits, w.v_bits, w.n_kv_heads, w.n_tokens, w.k_mode) == (3, 2, 32, 32768, synth.HYBRID)
+    w = bench.workload_by_name("c2+k3v3sym")
+    assert (w.k_bits, w.v_bits, w.k_mode, w.v_mode) == (3, 3, synth.SYM, synth.SYM)
+    with pytest.raises(SystemExit):
+        bench.workload_by_name("c2+k5v3")
     # a prefill quantisation reads K and V once (fp16) and writes what a decode then reads
     w = synth.tiny(n_tokens=400)
     assert bench.prefill_algorithmic_bytes(w) == w.n_units * 400 * 128 * 2 * 2 + bench.decode_algorithmic_bytes(w, 400)[0]
