@@ -220,6 +220,26 @@ def test_config3_gqa_batch16(bits):
     print(f"config3 {bits}-bit: contested flips {flips}, worst err/tol {max(worst, worst2):.3f}")
 
 
+@pytest.mark.parametrize("kb,vb,sym", [(3, 3, False), (3, 2, True), (4, 4, False)])
+def test_config2_shape_with_other_code_widths(kb, vb, sym):
+    # the 32-head, 32768-token shape with 3- and 4-bit codes (one query head per KV head and G = 32: the kernel
+    # instance whose MMA columns are groups, not heads); sym: the paper's presets keep the keys symmetric
+    w = synth.config2().with_(k_bits=kb, v_bits=vb)
+    if sym:
+        w = w.with_(k_mode=O.SYM)
+    K, V = synth.kv_all(w)
+    units = [3, 18]
+    gc, oc = make_gpu(w, K, V), sub_oracle(w, K, V, units)
+    del K, V
+    flips, worst = compare(w, gc, oc, units)
+    for step in range(3):
+        k1, v1 = synth.new_token(w, step)
+        gc.innerq_append_token(dev(k1), dev(v1))
+        oc.append(k1.reshape(w.n_units, -1)[units][None], v1.reshape(w.n_units, -1)[units][None])
+    _, worst2 = compare(w, gc, oc, units, step=3)
+    print(f"config-2 shape k{kb}v{vb}: contested flips {flips}, worst err/tol {max(worst, worst2):.3f}")
+
+
 def test_config4_long_context_prefill_and_decode():
     # batch 4 x 8 KV heads x 131072 tokens, 2-bit, G = 128: full prefill quantisation, then decode.
     w = synth.config4()
